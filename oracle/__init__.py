@@ -1,0 +1,143 @@
+"""CPU oracle for FusedDQP -- test infrastructure, not the product.
+
+Only tests, the smoke check and the benchmark's CPU-baseline / reference arm
+may import this package.  It never imports the CUDA package.
+
+The arithmetic lives in ``oracle_q4nx.c`` (plain C, fp64); this module builds
+it with gcc on first use and exposes thin numpy wrappers.  Each wrapper names
+the passage of the paper its C routine follows.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "oracle_q4nx.c")
+_LIB = os.path.join(_HERE, "liboracle_q4nx.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fast-math, no FMA contraction)."""
+    with _lock:
+        if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+            tmp = _LIB + f".tmp{os.getpid()}"
+            subprocess.check_call(
+                ["gcc", "-std=c11", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-shared",
+                 "-fPIC", "-o", tmp, _SRC, "-lm"])
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i64, p, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+        lib.oracle_packed_bytes.restype = ctypes.c_size_t
+        lib.oracle_packed_bytes.argtypes = [i64, i64]
+        lib.oracle_unpack.restype = ci
+        lib.oracle_unpack.argtypes = [p, i64, i64, p, p, p]
+        lib.oracle_dequant.restype = ci
+        lib.oracle_dequant.argtypes = [p, p, p, i64, i64, i64, i64, p, p]
+        lib.oracle_project.restype = ci
+        lib.oracle_project.argtypes = [p, p, p, p, i64, i64, i64, i64, i64, ci, ci, p, p]
+        lib.oracle_project_packed.restype = ci
+        lib.oracle_project_packed.argtypes = [p, p, i64, i64, i64, i64, i64, ci, ci, p, p]
+        lib.oracle_max_threads.restype = ci
+        _lib = lib
+    return _lib
+
+
+def _ptr(a: np.ndarray):
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def packed_bytes(K: int, N: int) -> int:
+    """Size of a packed K x N matrix: 5 bits per weight (a 32 x 256 block is 5120 bytes)."""
+    return int(_load().oracle_packed_bytes(K, N))
+
+
+def max_threads() -> int:
+    return int(_load().oracle_max_threads())
+
+
+def unpack(packed, K: int, N: int):
+    """Packed Q4NX bytes -> (codes[N,K] u8, scales[N,K/32] u16, offsets[N,K/32] u16)."""
+    packed = _c(packed, np.uint8)
+    if packed.size != packed_bytes(K, N) or packed.size == 0:
+        raise ValueError("packed size does not match K, N")
+    codes = np.empty((N, K), np.uint8)
+    scales = np.empty((N, K // 32), np.uint16)
+    offsets = np.empty((N, K // 32), np.uint16)
+    rc = _load().oracle_unpack(_ptr(packed), K, N, _ptr(codes), _ptr(scales), _ptr(offsets))
+    if rc != 0:
+        raise ValueError(f"oracle_unpack failed ({rc})")
+    return codes, scales, offsets
+
+
+def dequant(codes, scales, offsets, n0: int = 0, n1: int | None = None):
+    """Eq. 3: (w32[K, n1-n0] float32, w16[K, n1-n0] bf16 bits) for columns n0..n1."""
+    codes = _c(codes, np.uint8)
+    scales = _c(scales, np.uint16)
+    offsets = _c(offsets, np.uint16)
+    N, K = codes.shape
+    n1 = N if n1 is None else n1
+    w32 = np.empty((K, n1 - n0), np.float32)
+    w16 = np.empty((K, n1 - n0), np.uint16)
+    rc = _load().oracle_dequant(_ptr(codes), _ptr(scales), _ptr(offsets), K, N, n0, n1, _ptr(w32), _ptr(w16))
+    if rc != 0:
+        raise ValueError(f"oracle_dequant failed ({rc})")
+    return w32, w16
+
+
+def project(x_bf16, codes, scales, offsets, n0: int = 0, n1: int | None = None, use_w16: bool = False,
+            nthreads: int = 1):
+    """Eq. 14/15: (y[M, n1-n0] fp64, abs_sum[M, n1-n0] fp64) from unpacked weights."""
+    x_bf16 = _c(x_bf16, np.uint16)
+    codes = _c(codes, np.uint8)
+    scales = _c(scales, np.uint16)
+    offsets = _c(offsets, np.uint16)
+    N, K = codes.shape
+    M = x_bf16.shape[0]
+    if x_bf16.shape != (M, K):
+        raise ValueError("x must be [M, K]")
+    n1 = N if n1 is None else n1
+    y = np.empty((M, n1 - n0), np.float64)
+    a = np.empty((M, n1 - n0), np.float64)
+    rc = _load().oracle_project(_ptr(x_bf16), _ptr(codes), _ptr(scales), _ptr(offsets), M, K, N, n0, n1,
+                                int(use_w16), nthreads, _ptr(y), _ptr(a))
+    if rc != 0:
+        raise ValueError(f"oracle_project failed ({rc})")
+    return y, a
+
+
+def project_packed(x_bf16, packed, K: int, N: int, n0: int = 0, n1: int | None = None, use_w16: bool = False,
+                   nthreads: int = 1):
+    """Eq. 14/15 straight from packed bytes (column range n0..n1)."""
+    x_bf16 = _c(x_bf16, np.uint16)
+    packed = _c(packed, np.uint8)
+    M = x_bf16.shape[0]
+    if x_bf16.shape != (M, K):
+        raise ValueError("x must be [M, K]")
+    if packed.size != packed_bytes(K, N) or packed.size == 0:
+        raise ValueError("packed size does not match K, N")
+    n1 = N if n1 is None else n1
+    y = np.empty((M, n1 - n0), np.float64)
+    a = np.empty((M, n1 - n0), np.float64)
+    rc = _load().oracle_project_packed(_ptr(x_bf16), _ptr(packed), M, K, N, n0, n1, int(use_w16), nthreads,
+                                       _ptr(y), _ptr(a))
+    if rc != 0:
+        raise ValueError(f"oracle_project_packed failed ({rc})")
+    return y, a

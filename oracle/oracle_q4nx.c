@@ -1,0 +1,230 @@
+/*
+ * CPU oracle for FusedDQP (fused Q4NX dequantisation + projection).
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  Only the tests, the smoke
+ * check and the benchmark's cpu_baseline / reference arm may build, load or
+ * call it.  It shares no code with the CUDA library: its own layout reader,
+ * its own bf16 helpers, its own arithmetic.
+ *
+ * What it computes, and where the paper states it:
+ *   - Q4NX container (Sec. "Dequantization Engine"): weights are tiled into
+ *     32 x 256 blocks, each holding 32*256 int4 codes, 256 bf16 scales and
+ *     256 bf16 minimum-value offsets = 5120 bytes; group size g = 32.
+ *   - Eq. 3 (block-wise dequantisation):  w_hat_i = d_g * w_qi + m_g,
+ *     w_qi in {0..15}.
+ *   - Eq. 14 / Eq. 15 (FusedDQP): Y = W x A, accumulated block by block as
+ *     y_acc += dequant(w) x a.  The method is an exact restructuring of a
+ *     matrix-vector product with the dequantised matrix, so the oracle is
+ *     that product written out: sequential over k, in fp64.
+ *
+ * Naming: x is [M][K] (M token rows, K input features), the logical weight
+ * matrix is w_hat[k][n] (N output features), y is [M][N].  The paper's
+ * "M x K" matrix W has our N as its row count.
+ *
+ * Byte layout read here ("layout v1"; the paper fixes only the byte budget of
+ * a block, every other choice is this build's reading and is listed in the
+ * design notes):
+ *   strip  s = n / 32, row r = n % 32; strips are stored one after another,
+ *   a strip is 20*K bytes.  Inside a strip, blocks b = k / 256 follow each
+ *   other; block b holds j_b = min(8, K/32 - 8*b) groups of 32 k-indices and
+ *   is 640*j_b bytes: [codes 512*j_b][scales 64*j_b][offsets 64*j_b].
+ *   With c = k % 256, t = c / 32, i = c % 32:
+ *     code   byte  t*512 + r*16 + i/2   (low nibble when i is even)
+ *     scale  u16   at 512*j_b + 2*(t*32 + r)      little-endian bf16 bits
+ *     offset u16   at 576*j_b + 2*(t*32 + r)
+ *
+ * Precision: eq. 3 is evaluated once-rounded to fp32 (w32) from the exactly
+ * widened bf16 scale/offset; w16 is the round-to-nearest-even bf16 of w32.
+ * The projection accumulates (double)x * (double)w32 sequentially in k.
+ *
+ * Pins (tests/test_oracle_pins.py): the paper's 5120-byte block, hand-written
+ * byte dumps, closed-form worked examples, exact rational evaluation of eq. 3
+ * over all codes, an independent fp64 matmul, and invariants.  Parity with
+ * the authors' on-disk files and with the NPU's own rounding of eq. 3 is
+ * unpinned (no such data exists here).
+ */
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+#include <math.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ---- bf16 helpers (oracle's own) ------------------------------------- */
+
+static double bf16_bits_to_double(uint16_t h) {
+    uint32_t u = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f; /* widening is exact */
+}
+
+static uint16_t fp32_to_bf16_rne(float f) {
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7fffffffu) > 0x7f800000u) /* NaN: keep it a NaN */
+        return (uint16_t)((u >> 16) | 0x0040u);
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+/* ---- container geometry ----------------------------------------------- */
+
+/* Bytes of a packed K x N matrix: exactly 5 bits per weight.  0 when the
+ * shape is not representable (K or N not a positive multiple of 32). */
+size_t oracle_packed_bytes(int64_t K, int64_t N) {
+    if (K <= 0 || N <= 0 || (K % 32) != 0 || (N % 32) != 0) return 0;
+    return (size_t)(N / 32) * (size_t)(20 * K);
+}
+
+/* Locate element (n, k): offsets of its code byte, scale and offset words. */
+static void locate(int64_t K, int64_t n, int64_t k, size_t *code_byte, int *high_nibble,
+                   size_t *scale_at, size_t *offset_at) {
+    int64_t s = n / 32, r = n % 32;
+    int64_t b = k / 256, c = k % 256, t = c / 32, i = c % 32;
+    int64_t groups_left = K / 32 - 8 * b;
+    int64_t jb = groups_left < 8 ? groups_left : 8;
+    size_t block_off = (size_t)s * (size_t)(20 * K) + (size_t)b * 5120u;
+    *code_byte = block_off + (size_t)(t * 512 + r * 16 + i / 2);
+    *high_nibble = (int)(i & 1);
+    *scale_at = block_off + (size_t)(512 * jb) + (size_t)(2 * (t * 32 + r));
+    *offset_at = block_off + (size_t)(576 * jb) + (size_t)(2 * (t * 32 + r));
+}
+
+static uint16_t read_u16le(const uint8_t *p) { return (uint16_t)(p[0] | ((uint16_t)p[1] << 8)); }
+
+/* Packed bytes -> codes[N][K] (one code per byte), scales[N][K/32],
+ * offsets[N][K/32] (raw bf16 bits).  Returns 0, or -1 on a bad shape. */
+int oracle_unpack(const uint8_t *packed, int64_t K, int64_t N, uint8_t *codes, uint16_t *scales,
+                  uint16_t *offsets) {
+    if (oracle_packed_bytes(K, N) == 0 || !packed || !codes || !scales || !offsets) return -1;
+    int64_t G = K / 32;
+    for (int64_t n = 0; n < N; ++n) {
+        for (int64_t k = 0; k < K; ++k) {
+            size_t cb, sa, oa;
+            int hi;
+            locate(K, n, k, &cb, &hi, &sa, &oa);
+            uint8_t byte = packed[cb];
+            codes[n * K + k] = hi ? (uint8_t)(byte >> 4) : (uint8_t)(byte & 0x0f);
+            if ((k % 32) == 0) {
+                scales[n * G + k / 32] = read_u16le(packed + sa);
+                offsets[n * G + k / 32] = read_u16le(packed + oa);
+            }
+        }
+    }
+    return 0;
+}
+
+/* ---- eq. 3 --------------------------------------------------------------- */
+
+/* w32 = RN_fp32(d * q + m) with d, m the exact values of the bf16 words.
+ * d*q is exact in double (8-bit x 4-bit significands); the sum is exact in
+ * double whenever the two exponents are within ~40 binades, and otherwise the
+ * small term cannot move the result across an fp32 rounding boundary. */
+static float dequant_one(uint16_t d_bits, uint16_t m_bits, unsigned q) {
+    double d = bf16_bits_to_double(d_bits);
+    double m = bf16_bits_to_double(m_bits);
+    return (float)(d * (double)q + m);
+}
+
+/* Dequantise columns [n0, n1) of the matrix given as codes/scales/offsets.
+ * w32 / w16 are [K][n1-n0] row-major (logical w_hat[k][n]); either may be
+ * NULL. */
+int oracle_dequant(const uint8_t *codes, const uint16_t *scales, const uint16_t *offsets, int64_t K,
+                   int64_t N, int64_t n0, int64_t n1, float *w32, uint16_t *w16) {
+    if (oracle_packed_bytes(K, N) == 0 || !codes || !scales || !offsets) return -1;
+    if (n0 < 0 || n1 > N || n0 > n1) return -1;
+    int64_t G = K / 32, W = n1 - n0;
+    for (int64_t n = n0; n < n1; ++n) {
+        for (int64_t k = 0; k < K; ++k) {
+            unsigned q = codes[n * K + k];
+            if (q > 15u) return -2;
+            float w = dequant_one(scales[n * G + k / 32], offsets[n * G + k / 32], q);
+            if (w32) w32[k * W + (n - n0)] = w;
+            if (w16) w16[k * W + (n - n0)] = fp32_to_bf16_rne(w);
+        }
+    }
+    return 0;
+}
+
+/* ---- eq. 14 / eq. 15 ----------------------------------------------------- */
+
+/* y[m][n - n0] = sum_k x[m][k] * w32[k][n]  for n in [n0, n1), fp64, k ascending.
+ * abs_sum (optional) gets sum_k |x * w32|, the quantity the acceptance bound
+ * is stated in.  use_w16 != 0 multiplies by the bf16-rounded weights instead
+ * (what a dequantise-to-bf16 tensor-core path sees); the acceptance bound is
+ * always taken against use_w16 == 0.
+ * nthreads > 1 splits the independent output columns over OpenMP threads. */
+int oracle_project(const uint16_t *x_bf16, const uint8_t *codes, const uint16_t *scales,
+                   const uint16_t *offsets, int64_t M, int64_t K, int64_t N, int64_t n0, int64_t n1,
+                   int use_w16, int nthreads, double *y, double *abs_sum) {
+    if (oracle_packed_bytes(K, N) == 0 || M < 1 || !x_bf16 || !codes || !scales || !offsets || !y)
+        return -1;
+    if (n0 < 0 || n1 > N || n0 > n1) return -1;
+    int64_t G = K / 32, W = n1 - n0;
+    int bad = 0;
+    (void)nthreads;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(static) num_threads(nthreads > 0 ? nthreads : 1) reduction(| : bad)
+#endif
+    for (int64_t n = n0; n < n1; ++n) {
+        for (int64_t m = 0; m < M; ++m) {
+            double acc = 0.0, aacc = 0.0;
+            for (int64_t k = 0; k < K; ++k) {
+                unsigned q = codes[n * K + k];
+                if (q > 15u) bad = 1;
+                float w = dequant_one(scales[n * G + k / 32], offsets[n * G + k / 32], q & 15u);
+                double wd = use_w16 ? bf16_bits_to_double(fp32_to_bf16_rne(w)) : (double)w;
+                double p = bf16_bits_to_double(x_bf16[m * K + k]) * wd;
+                acc += p;
+                aacc += fabs(p);
+            }
+            y[m * W + (n - n0)] = acc;
+            if (abs_sum) abs_sum[m * W + (n - n0)] = aacc;
+        }
+    }
+    return bad ? -2 : 0;
+}
+
+/* Same projection, reading the packed bytes directly (unpacks one column at
+ * a time), for sizes where codes[N][K] would not be worth materialising. */
+int oracle_project_packed(const uint16_t *x_bf16, const uint8_t *packed, int64_t M, int64_t K,
+                          int64_t N, int64_t n0, int64_t n1, int use_w16, int nthreads, double *y,
+                          double *abs_sum) {
+    if (oracle_packed_bytes(K, N) == 0 || M < 1 || !x_bf16 || !packed || !y) return -1;
+    if (n0 < 0 || n1 > N || n0 > n1) return -1;
+    int64_t W = n1 - n0;
+    (void)nthreads;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(static) num_threads(nthreads > 0 ? nthreads : 1)
+#endif
+    for (int64_t n = n0; n < n1; ++n) {
+        for (int64_t m = 0; m < M; ++m) {
+            double acc = 0.0, aacc = 0.0;
+            for (int64_t k = 0; k < K; ++k) {
+                size_t cb, sa, oa;
+                int hi;
+                locate(K, n, k, &cb, &hi, &sa, &oa);
+                unsigned q = hi ? (unsigned)(packed[cb] >> 4) : (unsigned)(packed[cb] & 0x0f);
+                float w = dequant_one(read_u16le(packed + sa), read_u16le(packed + oa), q);
+                double wd = use_w16 ? bf16_bits_to_double(fp32_to_bf16_rne(w)) : (double)w;
+                double p = bf16_bits_to_double(x_bf16[m * K + k]) * wd;
+                acc += p;
+                aacc += fabs(p);
+            }
+            y[m * W + (n - n0)] = acc;
+            if (abs_sum) abs_sum[m * W + (n - n0)] = aacc;
+        }
+    }
+    return 0;
+}
+
+int oracle_max_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

@@ -1,0 +1,333 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked without a GPU.
+
+Each test is chosen so that a plausible mistake in the oracle (a dropped term, a
+wrong sign or index, a transposed operand, a wrong rounding) fails at least one.
+Nothing here touches the CUDA library.
+"""
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+import synthgen
+from q4nx_seq import read_sequential, write_sequential
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+
+
+# --------------------------------------------------------------------------- helpers
+
+def bf16_fraction(bits: int) -> Fraction:
+    """Exact value of a bf16 bit pattern (finite), by integer arithmetic only."""
+    sign = -1 if bits & 0x8000 else 1
+    e = (bits >> 7) & 0xFF
+    man = bits & 0x7F
+    if e == 0:
+        return sign * Fraction(man, 1 << 7) * Fraction(1, 1 << 126)
+    return sign * (1 + Fraction(man, 1 << 7)) * (Fraction(2) ** (e - 127))
+
+
+def round_to_binary(v: Fraction, p: int, emin: int) -> Fraction:
+    """Round v to nearest-even in a binary format with p significand bits and minimum
+    normal exponent emin (subnormals kept), exactly."""
+    if v == 0:
+        return Fraction(0)
+    s = -1 if v < 0 else 1
+    a = abs(v)
+    e = a.numerator.bit_length() - a.denominator.bit_length()
+    if Fraction(2) ** e > a:
+        e -= 1
+    e = max(e, emin)
+    ulp = Fraction(2) ** (e - (p - 1))
+    q, r = divmod(a, ulp)
+    if r * 2 > ulp or (r * 2 == ulp and q % 2 == 1):
+        q += 1
+    return s * q * ulp
+
+
+def f32_bits_of(v: Fraction) -> int:
+    return int(np.float32(float(v)).view(np.uint32))  # v is already fp32-exact: float() is exact
+
+
+def structured(K, N, code_fn, d_fn, m_fn):
+    n = np.arange(N)[:, None]
+    k = np.arange(K)[None, :]
+    g = np.arange(K // 32)[None, :]
+    codes = (code_fn(n, k) % 16).astype(np.uint8)
+    scales = synthgen.bf16_bits(d_fn(n, g).astype(np.float32) + np.zeros((N, K // 32), np.float32))
+    offsets = synthgen.bf16_bits(m_fn(n, g).astype(np.float32) + np.zeros((N, K // 32), np.float32))
+    return codes, scales, offsets
+
+
+# --------------------------------------------------------------------------- container size
+
+def test_block_byte_budget_from_paper():
+    # Sec. "Dequantization Engine": a 32 x 256 block is 4096 + 512 + 512 = 5120 bytes (5 bits / weight).
+    assert oracle.packed_bytes(256, 32) == 5120
+    assert oracle.packed_bytes(1152, 6912) == 1152 * 6912 * 5 // 8 == 4976640
+    assert oracle.packed_bytes(288, 32) == 5120 + 640
+    for K, N in [(0, 32), (32, 0), (48, 32), (32, 48), (-32, 32)]:
+        assert oracle.packed_bytes(K, N) == 0
+
+
+# --------------------------------------------------------------------------- layout
+
+def test_layout_hand_located_element():
+    # K = 288 (one full block + a one-group tail), N = 32.  Element (n=5, k=270) sits in the tail
+    # block: block offset 5120, tile 0, row 5, i = 14 -> code byte 5120 + 5*16 + 7 = 5207 (low nibble);
+    # the tail has one group, so scales start at 5120 + 512 and offsets at 5120 + 576.
+    K, N = 288, 32
+    buf = np.zeros(oracle.packed_bytes(K, N), np.uint8)
+    buf[5207] = 0x0B
+    buf[5642], buf[5643] = 0x00, 0x3F      # scale (row 5, group 8) = 0.5
+    buf[5706], buf[5707] = 0x80, 0xBF      # offset = -1
+    codes, scales, offsets = oracle.unpack(buf, K, N)
+    assert codes[5, 270] == 11 and codes.sum() == 11
+    assert scales[5, 8] == 0x3F00 and np.count_nonzero(scales) == 1
+    assert offsets[5, 8] == 0xBF80 and np.count_nonzero(offsets) == 1
+    # high nibble of the same byte is the next k
+    buf[5207] = 0xB0
+    codes, _, _ = oracle.unpack(buf, K, N)
+    assert codes[5, 271] == 11 and codes.sum() == 11
+    # first block of the second strip would start at 20*K
+    K, N = 288, 64
+    buf = np.zeros(oracle.packed_bytes(K, N), np.uint8)
+    buf[20 * K + 7 * 512 + 31 * 16 + 15] = 0xF0   # strip 1, block 0, tile 7, row 31, i = 31
+    codes, _, _ = oracle.unpack(buf, K, N)
+    assert codes[63, 255] == 15 and codes.sum() == 15
+
+
+def test_layout_golden_dump():
+    # tests/golden/q4nx_k32_n32.hex: the 640-byte container of the K = N = 32 matrix with
+    # code[n][k] = (k + 3n) mod 16, every scale 0.5 (0x3F00), every offset -1 (0xBF80),
+    # written out by hand rule: line r of the code section is row r, 16 bytes, low nibble first.
+    with open(os.path.join(GOLDEN, "q4nx_k32_n32.hex")) as f:
+        data = bytes.fromhex("".join(line.split("#")[0] for line in f))
+    assert len(data) == 640
+    codes, scales, offsets = oracle.unpack(np.frombuffer(data, np.uint8), 32, 32)
+    n, k = np.arange(32)[:, None], np.arange(32)[None, :]
+    assert np.array_equal(codes, (k + 3 * n) % 16)
+    assert np.all(scales == 0x3F00) and np.all(offsets == 0xBF80)
+
+
+@pytest.mark.parametrize("K,N", [(32, 32), (64, 64), (256, 32), (288, 32), (544, 96), (1152, 64)])
+def test_layout_against_sequential_writer(K, N):
+    w = synthgen.weights(100 + K + N, K, N)
+    packed = write_sequential(w.codes, w.scales, w.offsets)
+    assert packed.size == oracle.packed_bytes(K, N)
+    codes, scales, offsets = oracle.unpack(packed, K, N)
+    assert np.array_equal(codes, w.codes)
+    assert np.array_equal(scales, w.scales)
+    assert np.array_equal(offsets, w.offsets)
+    c2, s2, o2 = read_sequential(packed, K, N)
+    assert np.array_equal(c2, w.codes) and np.array_equal(s2, w.scales) and np.array_equal(o2, w.offsets)
+
+
+# --------------------------------------------------------------------------- eq. 3
+
+def _special_bf16():
+    vals = [0x0000, 0x8000, 0x0001, 0x8001, 0x007F, 0x0080, 0x0081, 0x3F80, 0xBF80, 0x3F00, 0x3E80,
+            0x7F7F, 0xFF7F, 0x7F00, 0x0100, 0x4B00, 0x3C23, 0xBC23, 0x3CA4, 0x5000, 0x2000]
+    return vals
+
+
+def test_dequant_exact_rational_all_codes():
+    # Eq. 3 over all 16 codes for a sweep of (d, m) bf16 pairs, against exact rational arithmetic
+    # rounded once to fp32 (and then to bf16) with integer arithmetic -- no floating point involved.
+    rng = np.random.default_rng(7)
+    special = _special_bf16()
+    pairs = [(d, m) for d in special for m in special]
+    rnd = rng.integers(0, 0x7F80, size=(3000, 2))                # finite magnitudes
+    sgn = rng.integers(0, 2, size=(3000, 2)) << 15
+    pairs += [tuple(int(v) for v in row) for row in (rnd | sgn)]
+    near = rng.integers(0x3800, 0x4000, size=(3000, 2)) | (rng.integers(0, 2, size=(3000, 2)) << 15)
+    pairs += [tuple(int(v) for v in row) for row in near]       # comparable magnitudes: real cancellation
+    # lay the pairs out as a K = 32 * ceil(P/1) ... simpler: one group per (pair), N = 32 rows reuse
+    P = len(pairs)
+    G = (P + 31) // 32
+    N, K = 32, 32 * G
+    codes = np.tile(np.arange(32, dtype=np.uint8) % 16, (N, G))   # every code appears in each group
+    scales = np.zeros((N, G), np.uint16)
+    offsets = np.zeros((N, G), np.uint16)
+    flat = pairs + [(0, 0)] * (N * G - P)
+    for idx, (d, m) in enumerate(flat):
+        scales[idx % N, idx // N] = d
+        offsets[idx % N, idx // N] = m
+    w32, w16 = oracle.dequant(codes, scales, offsets)
+    w32b = w32.view(np.uint32)
+    max_f32 = (2 - Fraction(1, 1 << 23)) * Fraction(2) ** 127
+    checked = 0
+    for idx, (d, m) in enumerate(pairs):
+        n, g = idx % N, idx // N
+        dv, mv = bf16_fraction(d), bf16_fraction(m)
+        for q in range(16):
+            exact = dv * q + mv
+            r32 = round_to_binary(exact, 24, -126)
+            if abs(r32) > max_f32:
+                continue  # overflow to inf: outside the tested domain
+            k = 32 * g + q
+            got = int(w32b[k, n])
+            want = f32_bits_of(r32)
+            if r32 == 0:
+                assert got & 0x7FFFFFFF == 0
+            else:
+                assert got == want, (hex(d), hex(m), q, hex(got), hex(want))
+            r16 = round_to_binary(r32, 8, -126)
+            if abs(r16) <= (2 - Fraction(1, 1 << 7)) * Fraction(2) ** 127 and r16 != 0:
+                assert int(w16[k, n]) == f32_bits_of(r16) >> 16
+            checked += 1
+    assert checked > 90000
+
+
+def test_dequant_special_cases():
+    K, N = 32, 32
+    codes = np.tile(np.arange(32, dtype=np.uint8) % 16, (N, 1))
+    one, half, neg1 = 0x3F80, 0x3F00, 0xBF80
+    # d = 0 -> offset only; m = 0 -> scale only; layout of the result is [K][N]
+    w32, _ = oracle.dequant(codes, np.zeros((N, 1), np.uint16), np.full((N, 1), neg1, np.uint16))
+    assert w32.shape == (K, N) and np.all(w32 == -1.0)
+    w32, w16 = oracle.dequant(codes, np.full((N, 1), half, np.uint16), np.zeros((N, 1), np.uint16))
+    assert np.array_equal(w32[:, 3], 0.5 * (np.arange(32) % 16))
+    assert np.array_equal(synthgen.bf16_to_f32(w16), w32)
+    # double rounding matters: 1 + 2^-8 + 2^-24-ish cases are covered by the rational sweep; here the
+    # plain tie: w32 = 1 + 2^-8 exactly (d = 2^-8, q = 1, m = 1) -> bf16 tie rounds to even = 1.0
+    w32, w16 = oracle.dequant(np.ones((N, K), np.uint8), np.full((N, 1), 0x3B80, np.uint16),
+                              np.full((N, 1), one, np.uint16))
+    assert np.all(w32 == np.float32(1 + 2.0 ** -8)) and np.all(w16 == 0x3F80)
+    # 1 + 3*2^-8 is also a tie: rounds up to even mantissa 0x3F82
+    w32, w16 = oracle.dequant(np.full((N, K), 3, np.uint8), np.full((N, 1), 0x3B80, np.uint16),
+                              np.full((N, 1), one, np.uint16))
+    assert np.all(w16 == 0x3F82)
+    with pytest.raises(ValueError):
+        oracle.dequant(np.full((N, K), 16, np.uint8), np.zeros((N, 1), np.uint16), np.zeros((N, 1), np.uint16))
+
+
+# --------------------------------------------------------------------------- eq. 14 / 15: worked examples
+
+def test_worked_example_E1_E2():
+    # K = N = 32, code = (k + 3n) mod 16, d = 0.5, m = -1.
+    # E1: x = 1 -> every row sees two full cycles 0..15: y = 0.5 * 240 - 32 = 88.
+    # E2: x = one-hot at k = 5 -> y[n] = 0.5 * ((5 + 3n) mod 16) - 1 -> 1.5, 3, 4.5, 6, -0.5, 1, ...
+    codes, scales, offsets = structured(32, 32, lambda n, k: k + 3 * n, lambda n, g: 0.5 + 0 * n, lambda n, g: -1.0 + 0 * n)
+    x = synthgen.bf16_bits(np.ones((1, 32), np.float32))
+    y, a = oracle.project(x, codes, scales, offsets)
+    assert np.all(y == 88.0)
+    x = synthgen.bf16_bits(np.eye(32, dtype=np.float32)[5:6])
+    y, a = oracle.project(x, codes, scales, offsets)
+    assert list(y[0, :6]) == [1.5, 3.0, 4.5, 6.0, -0.5, 1.0]
+    assert np.array_equal(a, np.abs(y))
+
+
+def _e3_inputs():
+    K = N = 64
+    codes, scales, offsets = structured(
+        K, N, lambda n, k: 7 * k + 3 * n, lambda n, g: 2.0 ** -(1.0 + g) + 0 * n, lambda n, g: (n - 32) / 16.0 + g)
+    m_idx, k_idx = np.arange(2)[:, None], np.arange(K)[None, :]
+    xf = (((k_idx + m_idx) % 5) - 2).astype(np.float32)
+    return K, N, codes, scales, offsets, xf
+
+
+def test_worked_example_E3_closed_form():
+    # K = N = 64, M = 2, code = (7k + 3n) mod 16, d[n][g] = 2^-(1+g), m[n][g] = (n-32)/16 + g,
+    # x[m][k] = ((k + m) mod 5) - 2.  All values are small dyadics, so every sum is exact.
+    K, N, codes, scales, offsets, xf = _e3_inputs()
+    w32, _ = oracle.dequant(codes, scales, offsets)
+    assert w32[33, 5] == 0.8125            # 0.25 * 6 + (-27/16 + 1)
+    y, a = oracle.project(synthgen.bf16_bits(xf), codes, scales, offsets)
+    expect = {(0, 0): 10.25, (0, 1): -1.625, (0, 31): -5.875, (0, 32): 6.25, (0, 63): -9.875,
+              (1, 0): -9.5, (1, 17): -6.625, (1, 63): -6.375}
+    for (m, n), v in expect.items():
+        assert y[m, n] == v, (m, n, y[m, n], v)
+    assert y[0].sum() == -532 and y[1].sum() == 308
+    assert a[0, 0] == 137.25 and a[0, 63] == 402.75
+    # the same numbers from the definition with exact rationals (independent of the oracle's code)
+    for m in range(2):
+        for n in (0, 1, 17, 31, 32, 63):
+            acc = Fraction(0)
+            for k in range(K):
+                g = k // 32
+                wq = (7 * k + 3 * n) % 16
+                acc += Fraction(int(xf[m, k])) * (Fraction(1, 2 ** (1 + g)) * wq + Fraction(n - 32, 16) + g)
+            assert Fraction(y[m, n]) == acc
+
+
+# --------------------------------------------------------------------------- projection vs an independent fp64 matmul
+
+@pytest.mark.parametrize("K,N,M", [(64, 32, 1), (288, 64, 3), (1152, 96, 2), (2560, 64, 8)])
+def test_projection_against_numpy_matmul(K, N, M):
+    w = synthgen.weights(200 + K, K, N)
+    x = synthgen.activations(300 + K, M, K)
+    packed = write_sequential(w.codes, w.scales, w.offsets) if K * N <= 300000 else None
+    # independent dequantised matrix: numpy, fp64 (exact for these magnitudes up to one fp32 rounding)
+    d = synthgen.bf16_to_f32(w.scales).astype(np.float64)
+    m = synthgen.bf16_to_f32(w.offsets).astype(np.float64)
+    W = (np.repeat(d, 32, axis=1) * w.codes + np.repeat(m, 32, axis=1)).astype(np.float32).astype(np.float64)  # [N, K]
+    xd = synthgen.bf16_to_f32(x).astype(np.float64)
+    y_np = xd @ W.T
+    a_np = np.abs(xd) @ np.abs(W.T)
+    y, a = oracle.project(x, w.codes, w.scales, w.offsets)
+    assert y.shape == (M, N)
+    assert np.allclose(a, a_np, rtol=1e-12, atol=0)
+    assert np.all(np.abs(y - y_np) <= 1e-13 * a_np)
+    w32, _ = oracle.dequant(w.codes, w.scales, w.offsets)
+    assert np.array_equal(w32.astype(np.float64), W.T)
+    if packed is not None:
+        y2, a2 = oracle.project_packed(x, packed, K, N)
+        assert np.array_equal(y2, y) and np.array_equal(a2, a)
+    # column ranges and threads give the same bits
+    y3, a3 = oracle.project(x, w.codes, w.scales, w.offsets, n0=32, n1=N, nthreads=4) if N > 32 else (y[:, 0:0], a[:, 0:0])
+    assert np.array_equal(y3, y[:, 32:]) if N > 32 else True
+
+
+# --------------------------------------------------------------------------- invariants
+
+def test_invariants_zero_offsets_only_scales_only_onehot():
+    K, N, M = 320, 64, 2
+    w = synthgen.weights(5, K, N)
+    x = synthgen.activations(6, M, K)
+    xf = synthgen.bf16_to_f32(x).astype(np.float64)
+    zc = np.zeros_like(w.codes)
+    z16 = np.zeros_like(w.scales)
+    # zero weights
+    y, a = oracle.project(x, zc, w.scales, z16)
+    assert np.all(y == 0) and np.all(a == 0)
+    # offsets only: y[m][n] = sum_g m[n][g] * sum_{k in g} x[m][k]
+    y, _ = oracle.project(x, zc, w.scales, w.offsets)
+    X = xf.reshape(M, K // 32, 32)
+    mo = synthgen.bf16_to_f32(w.offsets).astype(np.float64)
+    want = np.einsum("mgk,ng->mn", X, mo)
+    assert np.allclose(y, want, rtol=0, atol=1e-12)
+    # scales only
+    y, _ = oracle.project(x, w.codes, w.scales, z16)
+    d = synthgen.bf16_to_f32(w.scales).astype(np.float64)
+    want = np.einsum("mgk,ngk->mn", X, d[:, :, None] * w.codes.reshape(N, K // 32, 32))
+    assert np.allclose(y, want, rtol=0, atol=1e-12)
+    # one-hot x reads out a row of the dequantised matrix, exactly
+    w32, w16 = oracle.dequant(w.codes, w.scales, w.offsets)
+    for k in (0, 31, 32, 255, 256, 319):
+        e = np.zeros((1, K), np.float32)
+        e[0, k] = 1
+        y, _ = oracle.project(synthgen.bf16_bits(e), w.codes, w.scales, w.offsets)
+        assert np.array_equal(y[0], w32[k].astype(np.float64))
+        y, _ = oracle.project(synthgen.bf16_bits(e), w.codes, w.scales, w.offsets, use_w16=True)
+        assert np.array_equal(y[0], synthgen.bf16_to_f32(w16[k]).astype(np.float64))
+
+
+def test_invariants_linearity_and_rows():
+    K, N = 512, 32
+    w = synthgen.weights(8, K, N)
+    # small-integer activations: sums of them are bf16-exact and fp64 accumulation is exact enough
+    r = synthgen.u64(9, 0, 2 * K).reshape(2, K)
+    x1 = ((r[0] >> 60).astype(np.int64) - 8).astype(np.float32)[None]
+    x2 = ((r[1] >> 60).astype(np.int64) - 8).astype(np.float32)[None]
+    y1, _ = oracle.project(synthgen.bf16_bits(x1), w.codes, w.scales, w.offsets)
+    y2, _ = oracle.project(synthgen.bf16_bits(x2), w.codes, w.scales, w.offsets)
+    y12, a12 = oracle.project(synthgen.bf16_bits(x1 + x2), w.codes, w.scales, w.offsets)
+    assert np.all(np.abs(y12 - (y1 + y2)) <= 1e-13 * (a12 + 1))
+    ys, _ = oracle.project(synthgen.bf16_bits(2 * x1), w.codes, w.scales, w.offsets)
+    assert np.array_equal(ys, 2 * y1)
+    # each row of a batched call equals the single-row call; rows are not mixed up or transposed
+    yb, _ = oracle.project(synthgen.bf16_bits(np.concatenate([x1, x2])), w.codes, w.scales, w.offsets)
+    assert np.array_equal(yb[0], y1[0]) and np.array_equal(yb[1], y2[0])
