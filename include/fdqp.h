@@ -1,0 +1,183 @@
+/*
+ * fdqp.h -- C ABI of the FusedDQP library for NVIDIA B200 (sm_100a).
+ *
+ * FusedDQP is the decode-time projection of the paper "Mapping Gemma3 onto an
+ * Edge Dataflow Architecture": a matrix-vector (or thin matrix-matrix) product
+ * whose weight matrix is stored in the 4-bit Q4NX container and is dequantised
+ * inside the same kernel that multiplies it (Sec. "FusedDQP", Eq. 14 and 15),
+ * using the block-wise rule of Eq. 3 (Sec. "Dequantization Engine").
+ *
+ * Naming used by every entry point
+ *   x      activations, [M][K] row-major, bf16           (M token rows)
+ *   w_hat  logical dequantised weights, w_hat[k][n]       (K inputs, N outputs)
+ *   y      result, [M][N] row-major, fp32:  y[m][n] = sum_k x[m][k] * w_hat[k][n]
+ * The paper writes the same product as Y = W x A with W of size "M x K"; its M
+ * (output features) is N here, and M here counts tokens.
+ *
+ * Q4NX container ("layout v1").  The paper fixes the content and size of a
+ * block -- 32 x 256 int4 codes, 256 bf16 scales, 256 bf16 minimum-value
+ * offsets, 5120 bytes, group size 32 -- and that blocks are consumed left to
+ * right along K.  The remaining byte-level choices are this library's:
+ *   - a block covers 32 output features (a "strip", s = n / 32, r = n % 32)
+ *     by 256 input features (b = k / 256); groups of 32 run along K;
+ *   - strips are stored one after another, and the blocks of a strip follow
+ *     each other, so a strip is one contiguous run of 20*K bytes;
+ *   - a block with j groups (j = 8, or (K/32) % 8 for the last block of a strip
+ *     when K is not a multiple of 256) is 640*j bytes:
+ *         [codes 512*j] [scales 64*j] [offsets 64*j];
+ *   - with c = k % 256, t = c / 32, i = c % 32: the code of (r, c) is in byte
+ *     t*512 + r*16 + i/2, low nibble for even i; the group's scale is the
+ *     little-endian bf16 word 512*j + 2*(t*32 + r), its offset the word at
+ *     576*j + 2*(t*32 + r).
+ * K and N must be positive multiples of 32.  Codes are unsigned 0..15.
+ *
+ * Dequantisation (Eq. 3):  w_hat = d * code + m, evaluated with d and m widened
+ * exactly from bf16 and ONE rounding to fp32.  fdqp_dequant returns exactly that
+ * value (or its round-to-nearest-even bf16).  fdqp_run accumulates in fp32 in an
+ * unspecified but run-to-run reproducible order; for M >= 9 the weights pass
+ * through bf16 before a tensor-core contraction.  Acceptance bound for y against
+ * an fp64 evaluation: |y - y_ref| <= 2e-3 * sum_k |x*w_hat| + 1e-5.
+ *
+ * Conventions
+ *   - "host" / "device" on every pointer says where the memory must live.
+ *   - No entry point throws; each returns an fdqp_status (FDQP_OK == 0).
+ *   - Device work is enqueued on the caller's CUDA stream (a cudaStream_t passed
+ *     as void*; NULL is the legacy default stream) and is asynchronous unless
+ *     stated otherwise.
+ *   - There is no CPU fallback: without an sm_100 device fdqp_create fails.
+ */
+#ifndef FDQP_H
+#define FDQP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define FDQP_API __attribute__((visibility("default")))
+#else
+#define FDQP_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fdqp_ctx fdqp_ctx; /* opaque, owned by the library */
+
+typedef enum {
+    FDQP_OK = 0,
+    FDQP_ERR_ARG = 1,     /* null pointer, bad flag, code > 15 */
+    FDQP_ERR_SHAPE = 2,   /* M < 1, K or N not a positive multiple of 32 */
+    FDQP_ERR_ALIGN = 3,   /* a device pointer is not 16-byte aligned */
+    FDQP_ERR_SIZE = 4,    /* output buffer too small, or shape beyond the context's maxima */
+    FDQP_ERR_ARCH = 5,    /* device is not compute capability 10.x */
+    FDQP_ERR_CUDA = 6,    /* a CUDA runtime call failed; see fdqp_last_cuda_error */
+    FDQP_ERR_NOMEM = 7,   /* allocation failed */
+    FDQP_ERR_TIMEOUT = 8  /* a bounded wait inside a kernel ran out (sticky, see fdqp_last_status) */
+} fdqp_status;
+
+/* ---- Q4NX container (host side; Sec. "Dequantization Engine") ------------- */
+
+/* Bytes of a packed K x N matrix: K*N*5/8 (a 32 x 256 block is 5120 bytes).
+ * Returns 0 if K or N is not a positive multiple of 32. */
+FDQP_API size_t q4nx_packed_bytes(int64_t K, int64_t N);
+
+/* Pack codes, scales and offsets into the container described above.
+ *   codes        host, [N][K], one code per byte, each 0..15 (else FDQP_ERR_ARG)
+ *   scales_bf16  host, [N][K/32], raw bf16 bits of d
+ *   offsets_bf16 host, [N][K/32], raw bf16 bits of m
+ *   out          host, out_bytes >= q4nx_packed_bytes(K, N) (else FDQP_ERR_SIZE)
+ * Lossless; the caller keeps ownership of every buffer.  How float weights are
+ * turned into (code, d, m) is outside this library. */
+FDQP_API fdqp_status q4nx_pack(const uint8_t* codes, const uint16_t* scales_bf16, const uint16_t* offsets_bf16,
+                      int64_t K, int64_t N, void* out, size_t out_bytes);
+
+/* Inverse of q4nx_pack (all buffers host, sized as above). */
+FDQP_API fdqp_status q4nx_unpack(const void* packed, int64_t K, int64_t N, uint8_t* codes, uint16_t* scales_bf16,
+                        uint16_t* offsets_bf16);
+
+/* ---- context --------------------------------------------------------------- */
+
+/* Create a context on CUDA device `device` for projections up to max_M x max_K x
+ * max_N.  Allocates (device) the split-K workspace, its arrival counters, and the
+ * staging buffers of fdqp_run_host; reads the SM count and shared-memory limits.
+ * A context serves one stream at a time: its workspace is not re-entrant.
+ * Errors: FDQP_ERR_ARG (null), FDQP_ERR_SHAPE, FDQP_ERR_ARCH (not sm_100),
+ * FDQP_ERR_CUDA, FDQP_ERR_NOMEM.  On error *ctx is NULL. */
+FDQP_API fdqp_status fdqp_create(fdqp_ctx** ctx, int device, int64_t max_M, int64_t max_K, int64_t max_N);
+
+/* Free everything fdqp_create allocated.  The caller must have synchronised the
+ * streams that used the context.  NULL is accepted. */
+FDQP_API fdqp_status fdqp_destroy(fdqp_ctx* ctx);
+
+/* ---- the projection (Sec. "FusedDQP", Eq. 14 / 15, with Eq. 3 fused) ------- */
+
+/* y = x * dequant(W).
+ *   x_bf16  device, [M][K] bf16, 16-byte aligned
+ *   W_q4nx  device, q4nx_packed_bytes(K, N) bytes, 16-byte aligned
+ *   y       device, [M][N] fp32, 16-byte aligned; fully overwritten (no accumulate, no bias)
+ * Dispatch: M = 1 and 2..8 run the streaming GEMV kernels (weights fetched once
+ * from HBM through a shared-memory ring, nibbles unpacked in registers, scale and
+ * offset applied in fp32, split-K across CTAs reduced in a fixed order); M >= 9
+ * runs the dequantise-into-shared-memory tensor-core path.
+ * Asynchronous on `cuda_stream`; no allocation and no host synchronisation.  W, x
+ * and y must stay valid until the stream has passed the call.  Two calls that
+ * share a context must be ordered on one stream.
+ * Errors (nothing is launched): FDQP_ERR_ARG, FDQP_ERR_SHAPE, FDQP_ERR_ALIGN,
+ * FDQP_ERR_SIZE (beyond the maxima given to fdqp_create), FDQP_ERR_CUDA. */
+FDQP_API fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, float* y, int64_t M, int64_t K,
+                     int64_t N, void* cuda_stream);
+
+/* Same projection with HOST activations and result: copies x (host, [M][K] bf16)
+ * to the context's device staging buffer, runs fdqp_run, copies y back to `y_host`
+ * (host, [M][N] fp32) and synchronises the stream before returning.  W stays a
+ * device pointer (weights are resident model state).  Pinned host memory makes
+ * the copies asynchronous but is not required. */
+FDQP_API fdqp_status fdqp_run_host(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,
+                          int64_t M, int64_t K, int64_t N, void* cuda_stream);
+
+/* ---- the dequantisation engine (Sec. "Dequantization Engine", Eq. 3) ------- */
+
+/* Write the dequantised matrix w_hat[k][n] to `out` (device, [K][N] row-major,
+ * 16-byte aligned): fp32 when out_is_bf16 == 0, else bf16 = RNE(fp32 value).
+ * Bit-exact by definition (one rounding to fp32).  Asynchronous on the stream. */
+FDQP_API fdqp_status fdqp_dequant(fdqp_ctx* ctx, const void* W_q4nx, void* out, int out_is_bf16, int64_t K, int64_t N,
+                         void* cuda_stream);
+
+/* ---- status, tuning, introspection ---------------------------------------- */
+
+/* Sticky device-side status: FDQP_ERR_TIMEOUT once any kernel of this context gave
+ * up on a bounded wait (its output is then undefined), else FDQP_OK.  Reads a
+ * host-mapped word: call it after synchronising the stream; it synchronises
+ * nothing itself.  Cleared only by fdqp_destroy. */
+FDQP_API fdqp_status fdqp_last_status(fdqp_ctx* ctx);
+
+/* Text of the last CUDA runtime error seen by this context ("" if none).  The
+ * pointer stays valid until the next failing call or fdqp_destroy. */
+FDQP_API const char* fdqp_last_cuda_error(fdqp_ctx* ctx);
+
+/* Human-readable name of a status code (static storage). */
+FDQP_API const char* fdqp_status_string(fdqp_status s);
+
+/* Override a launch parameter; value < 0 restores the built-in choice.  Keys:
+ *   "path"          0 = dispatch on M (default), 1 = force the plain CUDA-core kernel
+ *   "ctas_per_sm"   persistent CTAs per SM for the GEMV kernels (1 or 2; 2 implies 8 consumer warps)
+ *   "consumer_warps" 8 or 16 consumer warps per CTA
+ *   "stages"        shared-memory ring depth in Q4NX blocks
+ *   "split_k"       number of K slices (1, 2 or 4)
+ *   "l2_evict_first" 1 = weight copies carry an evict-first L2 hint
+ * Unknown key or unusable value: FDQP_ERR_ARG.  Meant for benchmarks and tests. */
+FDQP_API fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t value);
+
+/* Number of kernels this context has launched since it was created. */
+FDQP_API int64_t fdqp_launch_count(fdqp_ctx* ctx);
+
+/* Describe the launch fdqp_run would make for (M, K, N) into `buf` (host,
+ * NUL-terminated, truncated to buf_bytes): kernel name, grid, block, shared
+ * memory, stages, split.  Launches nothing. */
+FDQP_API fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N, char* buf, size_t buf_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FDQP_H */

@@ -1,0 +1,202 @@
+"""ctypes binding of the FusedDQP C ABI (see include/fdqp.h for the contract of each call).
+
+Only marshals arguments: numpy arrays for host buffers, torch tensors (or raw integer
+addresses) for device buffers, ``torch.cuda.current_stream()`` when no stream is given.
+The library is built in-tree by ``build.py``; if it is missing or cannot be loaded the
+import of a symbol fails loudly -- there is no Python or CPU fallback for any operation.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libfdqp.so")
+_lib = None
+
+STATUS = {
+    0: "FDQP_OK", 1: "FDQP_ERR_ARG", 2: "FDQP_ERR_SHAPE", 3: "FDQP_ERR_ALIGN", 4: "FDQP_ERR_SIZE",
+    5: "FDQP_ERR_ARCH", 6: "FDQP_ERR_CUDA", 7: "FDQP_ERR_NOMEM", 8: "FDQP_ERR_TIMEOUT",
+}
+
+EXPORTS = [
+    "q4nx_packed_bytes", "q4nx_pack", "q4nx_unpack", "fdqp_create", "fdqp_destroy", "fdqp_run", "fdqp_run_host",
+    "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
+    "fdqp_launch_count", "fdqp_describe",
+]
+
+
+class FdqpError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        self.name = STATUS.get(code, f"status {code}")
+        super().__init__(f"{where}: {self.name}" + (f" ({detail})" if detail else ""))
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load libfdqp.so (building it first if the sources are newer)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        from . import build as _build
+        _build.build()
+    lib = ctypes.CDLL(_LIB_PATH)
+    i64, vp, ci, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.q4nx_packed_bytes.restype = sz
+    lib.q4nx_packed_bytes.argtypes = [i64, i64]
+    lib.q4nx_pack.restype = ci
+    lib.q4nx_pack.argtypes = [vp, vp, vp, i64, i64, vp, sz]
+    lib.q4nx_unpack.restype = ci
+    lib.q4nx_unpack.argtypes = [vp, i64, i64, vp, vp, vp]
+    lib.fdqp_create.restype = ci
+    lib.fdqp_create.argtypes = [ctypes.POINTER(vp), ci, i64, i64, i64]
+    lib.fdqp_destroy.restype = ci
+    lib.fdqp_destroy.argtypes = [vp]
+    lib.fdqp_run.restype = ci
+    lib.fdqp_run.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.fdqp_run_host.restype = ci
+    lib.fdqp_run_host.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.fdqp_dequant.restype = ci
+    lib.fdqp_dequant.argtypes = [vp, vp, vp, ci, i64, i64, vp]
+    lib.fdqp_last_status.restype = ci
+    lib.fdqp_last_status.argtypes = [vp]
+    lib.fdqp_last_cuda_error.restype = ctypes.c_char_p
+    lib.fdqp_last_cuda_error.argtypes = [vp]
+    lib.fdqp_status_string.restype = ctypes.c_char_p
+    lib.fdqp_status_string.argtypes = [ci]
+    lib.fdqp_set_param.restype = ci
+    lib.fdqp_set_param.argtypes = [vp, ctypes.c_char_p, i64]
+    lib.fdqp_launch_count.restype = i64
+    lib.fdqp_launch_count.argtypes = [vp]
+    lib.fdqp_describe.restype = ci
+    lib.fdqp_describe.argtypes = [vp, i64, i64, i64, ctypes.c_char_p, sz]
+    _lib = lib
+    return lib
+
+
+# ---- marshalling helpers ------------------------------------------------------------------------
+
+def _addr(buf) -> int:
+    """Address of a torch tensor, a numpy array, or an integer that already is one."""
+    if buf is None:
+        return 0
+    if isinstance(buf, int):
+        return buf
+    if isinstance(buf, np.ndarray):
+        return buf.ctypes.data
+    return int(buf.data_ptr())  # torch tensor
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return stream
+    return int(stream.cuda_stream)
+
+
+def _check(code: int, where: str, ctx=None):
+    if code != 0:
+        detail = ""
+        if ctx is not None and code == 6:
+            detail = load_library().fdqp_last_cuda_error(ctx).decode()
+        raise FdqpError(code, where, detail)
+
+
+# ---- container ------------------------------------------------------------------------------------
+
+def q4nx_packed_bytes(K: int, N: int) -> int:
+    return int(load_library().q4nx_packed_bytes(K, N))
+
+
+def q4nx_pack(codes: np.ndarray, scales_bf16: np.ndarray, offsets_bf16: np.ndarray) -> np.ndarray:
+    """codes[N,K] u8, scales/offsets[N,K/32] u16 (bf16 bits) -> packed bytes (host numpy)."""
+    codes = np.ascontiguousarray(codes, np.uint8)
+    scales_bf16 = np.ascontiguousarray(scales_bf16, np.uint16)
+    offsets_bf16 = np.ascontiguousarray(offsets_bf16, np.uint16)
+    N, K = codes.shape
+    size = q4nx_packed_bytes(K, N)
+    if size == 0:
+        raise FdqpError(2, "q4nx_pack")
+    if scales_bf16.shape != (N, K // 32) or offsets_bf16.shape != (N, K // 32):
+        raise FdqpError(2, "q4nx_pack", "scales/offsets must be [N, K/32]")
+    out = np.empty(size, np.uint8)
+    _check(load_library().q4nx_pack(codes.ctypes.data, scales_bf16.ctypes.data, offsets_bf16.ctypes.data, K, N,
+                                    out.ctypes.data, out.size), "q4nx_pack")
+    return out
+
+
+def q4nx_unpack(packed: np.ndarray, K: int, N: int):
+    packed = np.ascontiguousarray(packed, np.uint8)
+    if q4nx_packed_bytes(K, N) == 0 or packed.size != q4nx_packed_bytes(K, N):
+        raise FdqpError(2, "q4nx_unpack")
+    codes = np.empty((N, K), np.uint8)
+    scales = np.empty((N, K // 32), np.uint16)
+    offsets = np.empty((N, K // 32), np.uint16)
+    _check(load_library().q4nx_unpack(packed.ctypes.data, K, N, codes.ctypes.data, scales.ctypes.data,
+                                      offsets.ctypes.data), "q4nx_unpack")
+    return codes, scales, offsets
+
+
+# ---- context and projection -------------------------------------------------------------------------
+
+def fdqp_create(device: int, max_M: int, max_K: int, max_N: int) -> int:
+    """Returns the context handle (an integer address); release it with fdqp_destroy."""
+    h = ctypes.c_void_p()
+    _check(load_library().fdqp_create(ctypes.byref(h), device, max_M, max_K, max_N), "fdqp_create")
+    return h.value
+
+
+def fdqp_destroy(ctx: int) -> None:
+    _check(load_library().fdqp_destroy(ctx), "fdqp_destroy")
+
+
+def fdqp_run(ctx: int, x_bf16, W_q4nx, y, M: int, K: int, N: int, stream=None) -> None:
+    """x, W, y: device tensors (or addresses).  Asynchronous on `stream`."""
+    _check(load_library().fdqp_run(ctx, _addr(x_bf16), _addr(W_q4nx), _addr(y), M, K, N, _stream(stream)),
+           "fdqp_run", ctx)
+
+
+def fdqp_run_host(ctx: int, x_host_bf16, W_q4nx, y_host, M: int, K: int, N: int, stream=None) -> None:
+    """x, y: HOST buffers (numpy or pinned torch); W: device.  Returns after y_host is filled."""
+    _check(load_library().fdqp_run_host(ctx, _addr(x_host_bf16), _addr(W_q4nx), _addr(y_host), M, K, N,
+                                        _stream(stream)), "fdqp_run_host", ctx)
+
+
+def fdqp_dequant(ctx: int, W_q4nx, out, out_is_bf16: bool, K: int, N: int, stream=None) -> None:
+    _check(load_library().fdqp_dequant(ctx, _addr(W_q4nx), _addr(out), int(out_is_bf16), K, N, _stream(stream)),
+           "fdqp_dequant", ctx)
+
+
+def fdqp_last_status(ctx: int) -> int:
+    return int(load_library().fdqp_last_status(ctx))
+
+
+def fdqp_last_cuda_error(ctx: int) -> str:
+    return load_library().fdqp_last_cuda_error(ctx).decode()
+
+
+def fdqp_status_string(code: int) -> str:
+    return load_library().fdqp_status_string(code).decode()
+
+
+def fdqp_set_param(ctx: int, key: str, value: int) -> None:
+    _check(load_library().fdqp_set_param(ctx, key.encode(), value), f"fdqp_set_param({key})")
+
+
+def fdqp_launch_count(ctx: int) -> int:
+    return int(load_library().fdqp_launch_count(ctx))
+
+
+def fdqp_describe(ctx: int, M: int, K: int, N: int) -> str:
+    buf = ctypes.create_string_buffer(512)
+    _check(load_library().fdqp_describe(ctx, M, K, N, buf, len(buf)), "fdqp_describe")
+    return buf.value.decode()

@@ -1,0 +1,336 @@
+// C ABI of the FusedDQP library: context, argument checks, launch planning and dispatch.
+// Every operation of the projection runs in the CUDA kernels; nothing here computes on the host
+// and there is no fallback when the device is not an sm_100 part.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "fdqp.h"
+#include "fdqp_plan.h"
+
+namespace fdqp {
+cudaError_t gemv_launch(const GemvPlan& p, int consumer_warps, cudaStream_t stream);
+cudaError_t gemv_set_smem_limit(int bytes);
+cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
+cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
+}  // namespace fdqp
+
+using namespace fdqp;
+
+struct fdqp_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int smem_optin = 0;
+    int64_t max_M = 0, max_K = 0, max_N = 0;
+    float* ws_edge = nullptr;
+    float* ws_full = nullptr;
+    int* tickets = nullptr;
+    int* status_host = nullptr;  // pinned, mapped
+    int* status_dev = nullptr;   // device alias of status_host
+    void* x_stage = nullptr;     // fdqp_run_host staging (allocated on its first use)
+    float* y_stage = nullptr;
+    int64_t launches = 0;
+    std::string last_err;
+    // overrides (-1 = automatic)
+    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1;
+};
+
+namespace {
+
+constexpr int kMaxStages = 40;
+constexpr uint32_t kXsBudget = 100u * 1024u;  // shared memory the staged activations may take
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && (prev == dev || cudaSetDevice(dev) == cudaSuccess)) ok = true;
+        if (prev == dev) prev = -1;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+fdqp_status cuda_fail(fdqp_ctx* ctx, cudaError_t e, const char* what) {
+    if (ctx) ctx->last_err = std::string(what) + ": " + cudaGetErrorString(e);
+    cudaGetLastError();  // clear the sticky-less error state
+    return e == cudaErrorMemoryAllocation ? FDQP_ERR_NOMEM : FDQP_ERR_CUDA;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline uint32_t round_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
+
+fdqp_status check_shape(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
+    if (M < 1 || K <= 0 || N <= 0 || (K % kGroup) != 0 || (N % kStripRows) != 0) return FDQP_ERR_SHAPE;
+    if (M > ctx->max_M || K > ctx->max_K || N > ctx->max_N) return FDQP_ERR_SIZE;
+    return FDQP_OK;
+}
+
+// Fill the launch plan of one GEMV launch (M <= 8).  Returns false if no ring fits.
+bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, GemvPlan* p) {
+    std::memset(p, 0, sizeof(*p));
+    p->M = M;
+    p->K = K;
+    p->N = N;
+    p->S = N / kStripRows;
+    p->nb = (K + kBlockK - 1) / kBlockK;
+    int ctas_per_sm = ctx->p_ctas_per_sm > 0 ? (int)ctx->p_ctas_per_sm : 1;
+    if (ctas_per_sm > kMaxCtasPerSm) ctas_per_sm = kMaxCtasPerSm;
+    // register file: one 18-warp CTA or two 10-warp CTAs fit an SM
+    const int cw = ctas_per_sm > 1 ? 8 : ((ctx->p_cw == 8 || ctx->p_cw == 16) ? (int)ctx->p_cw : 16);
+    // K slices: as few as keep the staged activations within budget
+    int Z = 1;
+    if (ctx->p_split_k > 0) {
+        Z = (int)ctx->p_split_k;
+    } else {
+        while (Z < kMaxSplit && (uint32_t)((p->nb + Z - 1) / Z) * 8u * 64u * (uint32_t)M > kXsBudget / (uint32_t)ctas_per_sm)
+            Z *= 2;
+    }
+    if (Z > p->nb) Z = p->nb;
+    int nbz = (p->nb + Z - 1) / Z;
+    Z = (p->nb + nbz - 1) / nbz;  // drop slices that would be empty
+    p->Z = Z;
+    p->nbz = nbz;
+    int grid = ctx->sm_count * ctas_per_sm;
+    const int64_t total_blocks = (int64_t)p->S * p->nb;
+    if (grid > total_blocks) grid = (int)total_blocks;
+    int Gz = grid / Z;
+    if (Gz < 1) Gz = 1;
+    p->Gz = Gz;
+    // shared-memory carve-up
+    const uint32_t tiles = (uint32_t)nbz * 8u;
+    const uint32_t xs_bytes = tiles * 64u * (uint32_t)M;
+    const uint32_t xsum_bytes = tiles * kMaxTokens * 4u;
+    const uint32_t part_bytes = 2u * (uint32_t)cw * kStripRows * (uint32_t)M * 4u;
+    const uint32_t fixed = round_up(xs_bytes, 128) + 128 + round_up(xsum_bytes, 128) + round_up(part_bytes, 128) +
+                           (2u * kMaxStages + 4u) * 8u + 128u;
+    const uint32_t per_cta = (uint32_t)ctx->smem_optin / (uint32_t)ctas_per_sm - (ctas_per_sm > 1 ? 1024u : 0u);
+    if (fixed + 2u * kBlockBytes > per_cta) return false;
+    int nstage = (int)((per_cta - fixed) / kBlockBytes);
+    if (nstage > kMaxStages) nstage = kMaxStages;
+    if (ctx->p_stages > 0 && ctx->p_stages < nstage) nstage = (int)ctx->p_stages;
+    if (nstage < cw / 8) return false;
+    p->nstage = nstage;
+    p->off_xs = (uint32_t)nstage * kBlockBytes;
+    p->off_zero = p->off_xs + round_up(xs_bytes, 128);
+    p->off_xsum = p->off_zero + 128;
+    p->off_part = p->off_xsum + round_up(xsum_bytes, 128);
+    p->off_bar = p->off_part + round_up(part_bytes, 128);
+    p->smem_bytes = p->off_bar + (2u * (uint32_t)nstage + 4u) * 8u;
+    p->evict_first = ctx->p_evict >= 0 ? (ctx->p_evict != 0) : 1;
+    p->ws_edge = ctx->ws_edge;
+    p->ws_full = ctx->ws_full;
+    p->tickets = ctx->tickets;
+    p->status = ctx->status_dev;
+    *consumer_warps = cw;
+    return true;
+}
+
+}  // namespace
+
+extern "C" const char* fdqp_status_string(fdqp_status s) {
+    switch (s) {
+        case FDQP_OK: return "ok";
+        case FDQP_ERR_ARG: return "bad argument";
+        case FDQP_ERR_SHAPE: return "bad shape (M >= 1, K and N positive multiples of 32)";
+        case FDQP_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case FDQP_ERR_SIZE: return "size beyond buffer or context maxima";
+        case FDQP_ERR_ARCH: return "device is not compute capability 10.x";
+        case FDQP_ERR_CUDA: return "CUDA runtime error";
+        case FDQP_ERR_NOMEM: return "out of memory";
+        case FDQP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, int64_t max_K, int64_t max_N) {
+    if (!out) return FDQP_ERR_ARG;
+    *out = nullptr;
+    if (max_M < 1 || max_K <= 0 || max_N <= 0 || (max_K % kGroup) != 0 || (max_N % kStripRows) != 0)
+        return FDQP_ERR_SHAPE;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+        cudaGetLastError();
+        return FDQP_ERR_CUDA;
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return FDQP_ERR_CUDA;
+    if (prop.major != 10) return FDQP_ERR_ARCH;  // sm_100a code only; no other path exists
+    DeviceGuard guard(device);
+    if (!guard.ok) return FDQP_ERR_CUDA;
+    fdqp_ctx* ctx = new (std::nothrow) fdqp_ctx();
+    if (!ctx) return FDQP_ERR_NOMEM;
+    ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->smem_optin = (int)prop.sharedMemPerBlockOptin;
+    ctx->max_M = max_M;
+    ctx->max_K = max_K;
+    ctx->max_N = max_N;
+    const int64_t S = max_N / kStripRows;
+    const size_t slot = sizeof(float) * kStripRows * kMaxTokens;
+    cudaError_t e;
+    fdqp_status st = FDQP_OK;
+    do {
+        if ((e = cudaMalloc(&ctx->ws_edge, slot * 2 * (size_t)ctx->sm_count * kMaxCtasPerSm))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMalloc(&ctx->ws_full, slot * (size_t)kMaxSplit * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMalloc(&ctx->tickets, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMemset(ctx->tickets, 0, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaHostAlloc(&ctx->status_host, sizeof(int), cudaHostAllocMapped))) { st = cuda_fail(nullptr, e, ""); break; }
+        *ctx->status_host = 0;
+        if ((e = cudaHostGetDevicePointer(&ctx->status_dev, ctx->status_host, 0))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = gemv_set_smem_limit(ctx->smem_optin))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaDeviceSynchronize())) { st = cuda_fail(nullptr, e, ""); break; }
+    } while (false);
+    if (st != FDQP_OK) {
+        fdqp_destroy(ctx);
+        return st;
+    }
+    *out = ctx;
+    return FDQP_OK;
+}
+
+extern "C" fdqp_status fdqp_destroy(fdqp_ctx* ctx) {
+    if (!ctx) return FDQP_OK;
+    DeviceGuard guard(ctx->device);
+    if (ctx->ws_edge) cudaFree(ctx->ws_edge);
+    if (ctx->ws_full) cudaFree(ctx->ws_full);
+    if (ctx->tickets) cudaFree(ctx->tickets);
+    if (ctx->x_stage) cudaFree(ctx->x_stage);
+    if (ctx->y_stage) cudaFree(ctx->y_stage);
+    if (ctx->status_host) cudaFreeHost(ctx->status_host);
+    cudaGetLastError();
+    delete ctx;
+    return FDQP_OK;
+}
+
+extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, float* y, int64_t M, int64_t K,
+                                int64_t N, void* cuda_stream) {
+    if (!ctx || !x_bf16 || !W_q4nx || !y) return FDQP_ERR_ARG;
+    fdqp_status st = check_shape(ctx, M, K, N);
+    if (st != FDQP_OK) return st;
+    if (!aligned16(x_bf16) || !aligned16(W_q4nx) || !aligned16(y)) return FDQP_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FDQP_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint8_t* W = static_cast<const uint8_t*>(W_q4nx);
+    const uint16_t* x = static_cast<const uint16_t*>(x_bf16);
+    cudaError_t e;
+    if (ctx->p_path == 1) {
+        if ((e = plain_launch(W, x, y, (int)M, (int)K, (int)N, stream))) return cuda_fail(ctx, e, "plain kernel launch");
+        ctx->launches += 1;
+        return FDQP_OK;
+    }
+    // Token rows are processed eight at a time by the streaming GEMV kernel.
+    for (int64_t m0 = 0; m0 < M; m0 += kMaxTokens) {
+        const int mc = (int)((M - m0) < kMaxTokens ? (M - m0) : kMaxTokens);
+        GemvPlan plan;
+        int cw = 0;
+        if (!plan_gemv(ctx, mc, (int)K, (int)N, &cw, &plan)) return FDQP_ERR_SIZE;
+        plan.W = W;
+        plan.x = x + m0 * K;
+        plan.y = y + m0 * N;
+        if ((e = gemv_launch(plan, cw, stream))) return cuda_fail(ctx, e, "gemv kernel launch");
+        ctx->launches += 1;
+    }
+    return FDQP_OK;
+}
+
+extern "C" fdqp_status fdqp_run_host(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,
+                                     int64_t M, int64_t K, int64_t N, void* cuda_stream) {
+    if (!ctx || !x_host_bf16 || !W_q4nx || !y_host) return FDQP_ERR_ARG;
+    fdqp_status st = check_shape(ctx, M, K, N);
+    if (st != FDQP_OK) return st;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FDQP_ERR_CUDA;
+    cudaError_t e;
+    if (!ctx->x_stage) {
+        if ((e = cudaMalloc(&ctx->x_stage, (size_t)ctx->max_M * ctx->max_K * 2))) return cuda_fail(ctx, e, "x staging");
+        if ((e = cudaMalloc(&ctx->y_stage, (size_t)ctx->max_M * ctx->max_N * 4))) return cuda_fail(ctx, e, "y staging");
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if ((e = cudaMemcpyAsync(ctx->x_stage, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, stream)))
+        return cuda_fail(ctx, e, "x copy");
+    st = fdqp_run(ctx, ctx->x_stage, W_q4nx, ctx->y_stage, M, K, N, cuda_stream);
+    if (st != FDQP_OK) return st;
+    if ((e = cudaMemcpyAsync(y_host, ctx->y_stage, (size_t)M * N * 4, cudaMemcpyDeviceToHost, stream)))
+        return cuda_fail(ctx, e, "y copy");
+    if ((e = cudaStreamSynchronize(stream))) return cuda_fail(ctx, e, "stream sync");
+    return fdqp_last_status(ctx);
+}
+
+extern "C" fdqp_status fdqp_dequant(fdqp_ctx* ctx, const void* W_q4nx, void* out, int out_is_bf16, int64_t K, int64_t N,
+                                    void* cuda_stream) {
+    if (!ctx || !W_q4nx || !out || (out_is_bf16 != 0 && out_is_bf16 != 1)) return FDQP_ERR_ARG;
+    fdqp_status st = check_shape(ctx, 1, K, N);
+    if (st != FDQP_OK) return st;
+    if (!aligned16(W_q4nx) || !aligned16(out)) return FDQP_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FDQP_ERR_CUDA;
+    cudaError_t e = dequant_launch(static_cast<const uint8_t*>(W_q4nx), out, out_is_bf16 != 0, (int)K, (int)N,
+                                   static_cast<cudaStream_t>(cuda_stream));
+    if (e) return cuda_fail(ctx, e, "dequant kernel launch");
+    ctx->launches += 1;
+    return FDQP_OK;
+}
+
+extern "C" fdqp_status fdqp_last_status(fdqp_ctx* ctx) {
+    if (!ctx) return FDQP_ERR_ARG;
+    const int v = *static_cast<volatile int*>(ctx->status_host);
+    return v == 0 ? FDQP_OK : static_cast<fdqp_status>(v);
+}
+
+extern "C" const char* fdqp_last_cuda_error(fdqp_ctx* ctx) { return ctx ? ctx->last_err.c_str() : ""; }
+
+extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t value) {
+    if (!ctx || !key) return FDQP_ERR_ARG;
+    const int64_t v = value < 0 ? -1 : value;
+    if (!std::strcmp(key, "path")) {
+        if (v > 1) return FDQP_ERR_ARG;
+        ctx->p_path = v;
+    } else if (!std::strcmp(key, "ctas_per_sm")) {
+        if (v == 0 || v > kMaxCtasPerSm) return FDQP_ERR_ARG;
+        ctx->p_ctas_per_sm = v;
+    } else if (!std::strcmp(key, "consumer_warps")) {
+        if (v != -1 && v != 8 && v != 16) return FDQP_ERR_ARG;
+        ctx->p_cw = v;
+    } else if (!std::strcmp(key, "stages")) {
+        if (v == 0 || v == 1) return FDQP_ERR_ARG;
+        ctx->p_stages = v;
+    } else if (!std::strcmp(key, "split_k")) {
+        if (v != -1 && v != 1 && v != 2 && v != 4) return FDQP_ERR_ARG;
+        ctx->p_split_k = v;
+    } else if (!std::strcmp(key, "l2_evict_first")) {
+        if (v > 1) return FDQP_ERR_ARG;
+        ctx->p_evict = v;
+    } else {
+        return FDQP_ERR_ARG;
+    }
+    return FDQP_OK;
+}
+
+extern "C" int64_t fdqp_launch_count(fdqp_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N, char* buf, size_t buf_bytes) {
+    if (!ctx || !buf || buf_bytes == 0) return FDQP_ERR_ARG;
+    fdqp_status st = check_shape(ctx, M, K, N);
+    if (st != FDQP_OK) return st;
+    if (ctx->p_path == 1) {
+        std::snprintf(buf, buf_bytes, "fdqp_plain_kernel grid=(%lld,%lld) block=128", (long long)((N / 32 + 3) / 4),
+                      (long long)((M + 7) / 8));
+        return FDQP_OK;
+    }
+    GemvPlan plan;
+    int cw = 0;
+    const int mc = (int)(M < kMaxTokens ? M : kMaxTokens);
+    if (!plan_gemv(ctx, mc, (int)K, (int)N, &cw, &plan)) return FDQP_ERR_SIZE;
+    std::snprintf(buf, buf_bytes,
+                  "fdqp_gemv_kernel<%d,%d> launches=%lld grid=%d block=%d smem=%u stages=%d split_k=%d ctas_per_slice=%d "
+                  "evict_first=%d",
+                  cw, mc == 1 ? 1 : 2, (long long)((M + kMaxTokens - 1) / kMaxTokens), plan.Z * plan.Gz, (cw + 2) * 32,
+                  plan.smem_bytes, plan.nstage, plan.Z, plan.Gz, plan.evict_first);
+    return FDQP_OK;
+}

@@ -1,0 +1,41 @@
+// Launch plan of the streaming GEMV kernels: the quantities the host fixes per call and the
+// kernel re-derives per CTA.  Plain data, shared by the host dispatcher and the device code.
+#pragma once
+#include <stdint.h>
+
+namespace fdqp {
+
+constexpr int kStripRows = 32;      // output features per strip
+constexpr int kGroup = 32;          // quantisation group along K
+constexpr int kBlockK = 256;        // input features per full Q4NX block
+constexpr int kBlockBytes = 5120;   // bytes of a full block (Sec. "Dequantization Engine")
+constexpr int kGroupBytes = 640;    // bytes a block spends per group: 512 codes + 64 scales + 64 offsets
+constexpr int kMaxTokens = 8;       // token rows one GEMV launch handles
+constexpr int kMaxSplit = 4;        // K slices
+constexpr int kMaxCtasPerSm = 2;
+
+struct GemvPlan {
+    const uint8_t* W;     // device, packed Q4NX
+    const uint16_t* x;    // device, [M][K] bf16 bits
+    float* y;             // device, [M][N]
+    float* ws_edge;       // device, [grid][2][32*kMaxTokens] partial sums of strips shared between CTAs
+    float* ws_full;       // device, [Z][S][32*kMaxTokens] partial sums of whole strip-slices (Z > 1)
+    int* tickets;         // device, [S] arrival counters, zero between launches
+    int* status;          // host-mapped sticky status word
+    int M, K, N;
+    int S;                // strips = N / 32
+    int nb;               // blocks per strip = ceil(K / 256)
+    int Z;                // K slices
+    int nbz;              // blocks per slice = ceil(nb / Z); every slice is non-empty
+    int Gz;               // CTAs per slice; grid = Z * Gz
+    int nstage;           // ring depth in blocks
+    int evict_first;      // weight copies carry an evict-first L2 hint
+    uint32_t off_xs;      // shared-memory offsets (bytes)
+    uint32_t off_zero;
+    uint32_t off_xsum;
+    uint32_t off_part;
+    uint32_t off_bar;
+    uint32_t smem_bytes;
+};
+
+}  // namespace fdqp

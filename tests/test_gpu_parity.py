@@ -1,0 +1,235 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs -- element by element at sizes that span several tiles and ragged tails, bit-for-bit where
+the arithmetic is exact, and on the full workload shapes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2602_06063_b200 as fd
+import synthgen
+from gpu_common import (ABS_TOL, MAX_K, MAX_M, MAX_N, REL_TOL, Case, assert_close, dev_bytes, exact_regime_weights,
+                        exact_regime_x)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    h = fd.fdqp_create(0, MAX_M, MAX_K, MAX_N)
+    yield h
+    torch.cuda.synchronize()
+    fd.fdqp_destroy(h)
+
+
+@pytest.fixture()
+def fresh(ctx):
+    """The shared context with every launch parameter back to automatic."""
+    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first"):
+        fd.fdqp_set_param(ctx, key, -1)
+    yield ctx
+    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first"):
+        fd.fdqp_set_param(ctx, key, -1)
+
+
+# ------------------------------------------------------------------ dequantisation engine: bit-exact
+
+@pytest.mark.parametrize("K,N", [(32, 32), (288, 64), (1152, 96), (2560, 256)])
+def test_dequant_bit_exact(fresh, K, N):
+    case = Case(K, N, 1, seed=900 + K)
+    w32, w16 = oracle.dequant(case.w.codes, case.w.scales, case.w.offsets)
+    out32 = torch.empty((K, N), dtype=torch.float32, device="cuda")
+    out16 = torch.empty((K, N), dtype=torch.bfloat16, device="cuda")
+    fd.fdqp_dequant(fresh, case.W_dev, out32, False, K, N)
+    fd.fdqp_dequant(fresh, case.W_dev, out16, True, K, N)
+    torch.cuda.synchronize()
+    assert np.array_equal(out32.cpu().numpy().view(np.uint32), w32.view(np.uint32))
+    assert np.array_equal(out16.view(torch.int16).cpu().numpy().view(np.uint16), w16)
+
+
+def test_dequant_bit_exact_extreme_scales(fresh):
+    # scales and offsets over the whole finite bf16 range, subnormals included (nothing may flush to zero)
+    K, N = 512, 64
+    r = synthgen.u64(77, 0, 2 * N * (K // 32)).reshape(2, N, K // 32)
+    bits = ((r >> np.uint64(48)) & np.uint64(0xFFFF)).astype(np.uint16)
+    finite = (bits & 0x7F80) != 0x7F80
+    bits = np.where(finite, bits, bits & 0x807F).astype(np.uint16)
+    # keep exponents below 2^100 so that d*15 + m cannot overflow
+    bits = np.where((bits & 0x7F80) > (227 << 7), bits & 0x80FF | (100 << 7), bits).astype(np.uint16)
+    w = synthgen.weights(78, K, N)
+    w.scales[:], w.offsets[:] = bits[0], bits[1]
+    case = Case(K, N, 1, seed=78, weights=w)
+    w32, w16 = oracle.dequant(w.codes, w.scales, w.offsets)
+    out32 = torch.empty((K, N), dtype=torch.float32, device="cuda")
+    out16 = torch.empty((K, N), dtype=torch.bfloat16, device="cuda")
+    fd.fdqp_dequant(fresh, case.W_dev, out32, False, K, N)
+    fd.fdqp_dequant(fresh, case.W_dev, out16, True, K, N)
+    torch.cuda.synchronize()
+    assert np.array_equal(out32.cpu().numpy().view(np.uint32), w32.view(np.uint32))
+    assert np.array_equal(out16.view(torch.int16).cpu().numpy().view(np.uint16), w16)
+
+
+# ------------------------------------------------------------------ projection: element by element
+
+SMALL = [  # (K, N, M): tiny, tails (K % 256 != 0), several strips, several blocks, every M of the GEMV family, M >= 9
+    (32, 32, 1), (64, 64, 2), (288, 32, 1), (544, 96, 3), (1152, 6912, 1), (2560, 1024, 1), (2560, 2048, 8),
+    (2048, 2560, 5), (4096, 4736, 4), (10240, 2560, 1), (3840, 1280, 7), (1024, 512, 9), (1056, 320, 20),
+]
+
+
+@pytest.mark.parametrize("K,N,M", SMALL)
+@pytest.mark.parametrize("path", [0, 1])
+def test_projection_matches_oracle(fresh, K, N, M, path):
+    fd.fdqp_set_param(fresh, "path", path)
+    case = Case(K, N, M, seed=1000 + K + N + M)
+    y = case.run(fresh)
+    y_ref, a_ref = case.reference()
+    assert_close(y, y_ref, a_ref, f"K={K} N={N} M={M} path={path}")
+
+
+@pytest.mark.parametrize("K,N,M", [(64, 64, 2), (1152, 96, 1), (4096, 1024, 8), (2560, 4736, 3), (21504, 64, 1)])
+def test_exact_arithmetic_regime_is_bit_exact(fresh, K, N, M):
+    # d = 2^-3, m in {-1,0,1}, x in {-2..2}: every partial sum is a multiple of 2^-3 far below 2^24, so any
+    # summation order is exact in fp32 and the result must equal the oracle bit for bit.
+    case = Case(K, N, M, seed=0, weights=exact_regime_weights(31 + K, K, N), x=exact_regime_x(32 + K, M, K))
+    y_ref, _ = case.reference()
+    for path in (0, 1):
+        fd.fdqp_set_param(fresh, "path", path)
+        y = case.run(fresh)
+        assert np.array_equal(y.astype(np.float64), y_ref), f"path {path}"
+
+
+def test_worked_examples_on_gpu(fresh):
+    # E1/E2: K = N = 32, code = (k + 3n) mod 16, d = 0.5, m = -1; x = 1 -> 88; x = e_5 -> 0.5*((5+3n)%16) - 1
+    n, k = np.arange(32)[:, None], np.arange(32)[None, :]
+    w = synthgen.Q4NXWeights(((k + 3 * n) % 16).astype(np.uint8), np.full((32, 1), 0x3F00, np.uint16),
+                             np.full((32, 1), 0xBF80, np.uint16))
+    ones = synthgen.bf16_bits(np.ones((1, 32), np.float32))
+    assert np.all(Case(32, 32, 1, 0, weights=w, x=ones).run(fresh) == 88.0)
+    e5 = synthgen.bf16_bits(np.eye(32, dtype=np.float32)[5:6])
+    y = Case(32, 32, 1, 0, weights=w, x=e5).run(fresh)
+    assert list(y[0, :6]) == [1.5, 3.0, 4.5, 6.0, -0.5, 1.0]
+    # E3: K = N = 64, M = 2 (and the same rows padded to M = 9), all values dyadic
+    K = N = 64
+    n, k, g = np.arange(N)[:, None], np.arange(K)[None, :], np.arange(2)[None, :]
+    w = synthgen.Q4NXWeights(((7 * k + 3 * n) % 16).astype(np.uint8),
+                             synthgen.bf16_bits((2.0 ** -(1.0 + g) + 0 * n).astype(np.float32)),
+                             synthgen.bf16_bits(((n - 32) / 16.0 + g).astype(np.float32)))
+    m_idx = np.arange(9)[:, None]
+    xf = (((k + m_idx) % 5) - 2).astype(np.float32)
+    for M in (2, 9):
+        y = Case(K, N, M, 0, weights=w, x=synthgen.bf16_bits(xf[:M])).run(fresh)
+        assert y[0, 0] == 10.25 and y[0, 1] == -1.625 and y[0, 31] == -5.875 and y[0, 32] == 6.25
+        assert y[0, 63] == -9.875 and y[1, 0] == -9.5 and y[1, 17] == -6.625 and y[1, 63] == -6.375
+        assert y[0].sum() == -532 and y[1].sum() == 308
+
+
+def test_one_hot_reads_out_dequantised_rows(fresh):
+    K, N = 544, 64
+    case = Case(K, N, 8, seed=55)
+    w32, _ = oracle.dequant(case.w.codes, case.w.scales, case.w.offsets)
+    ks = [0, 31, 32, 255, 256, 300, 511, 543]
+    x = np.zeros((8, K), np.float32)
+    for i, kk in enumerate(ks):
+        x[i, kk] = 1.0
+    y = Case(K, N, 8, 0, weights=case.w, x=synthgen.bf16_bits(x)).run(fresh)
+    want = w32[ks].astype(np.float64)
+    assert np.all(np.abs(y - want) <= REL_TOL * np.abs(want) + ABS_TOL)
+    # (the GEMV forms d*S + (m - 128 d)*X with several roundings, so this read-out is close, not bit-equal;
+    # the bit-exact statement of Eq. 3 is fdqp_dequant's)
+
+
+def test_zero_and_offsets_only(fresh):
+    K, N, M = 1152, 64, 4
+    case = Case(K, N, M, seed=66)
+    zero = synthgen.Q4NXWeights(np.zeros_like(case.w.codes), case.w.scales, np.zeros_like(case.w.offsets))
+    assert np.all(Case(K, N, M, 0, weights=zero, x=case.x).run(fresh) == 0)
+    off = synthgen.Q4NXWeights(np.zeros_like(case.w.codes), case.w.scales, case.w.offsets)
+    c = Case(K, N, M, 0, weights=off, x=case.x)
+    y_ref, a_ref = c.reference()
+    assert_close(c.run(fresh), y_ref, a_ref, "offsets only")
+
+
+def test_reruns_are_bit_identical_and_scaling_by_two_commutes(fresh):
+    for K, N, M in [(21504, 5376, 4), (2560, 10240, 1)]:
+        case = Case(K, N, M, seed=70 + M, amp=K ** -0.5)
+        y1 = case.run(fresh)
+        y2 = case.run(fresh)
+        assert np.array_equal(y1.view(np.uint32), y2.view(np.uint32))
+        x2 = synthgen.bf16_bits(2 * synthgen.bf16_to_f32(case.x))
+        y3 = Case(K, N, M, 0, weights=case.w, x=x2).run(fresh)
+        assert np.array_equal(y3, 2 * y1)
+
+
+def test_batched_rows_match_single_row_calls(fresh):
+    K, N, M = 3840, 2048, 8
+    case = Case(K, N, M, seed=81)
+    y = case.run(fresh)
+    y_ref, a_ref = case.reference()
+    for m in (0, 3, 7):
+        xm = dev_bytes(case.x[m:m + 1])
+        y1 = case.run(fresh, M=1, x_dev=xm)
+        assert_close(y1, y_ref[m:m + 1], a_ref[m:m + 1], f"row {m}")
+        assert np.all(np.abs(y1[0] - y[m]) <= 2 * (REL_TOL * a_ref[m] + ABS_TOL))
+
+
+@pytest.mark.parametrize("key,values", [("split_k", [1, 2, 4]), ("consumer_warps", [8, 16]), ("ctas_per_sm", [1, 2]),
+                                        ("stages", [2, 3, 7]), ("l2_evict_first", [0, 1])])
+def test_launch_parameters_do_not_change_results(fresh, key, values):
+    K, N, M = 4352, 2080, 3   # 17 blocks per strip, 65 strips: ragged against every split and grid
+    case = Case(K, N, M, seed=90)
+    y_ref, a_ref = case.reference()
+    exact = Case(K, N, M, 0, weights=exact_regime_weights(91, K, N), x=exact_regime_x(92, M, K))
+    e_ref, _ = exact.reference()
+    for v in values:
+        fd.fdqp_set_param(fresh, key, v)
+        assert_close(case.run(fresh), y_ref, a_ref, f"{key}={v}")
+        assert np.array_equal(exact.run(fresh).astype(np.float64), e_ref), f"{key}={v}"
+
+
+def test_output_is_fully_overwritten_and_nothing_else(fresh):
+    K, N, M = 2560, 1024, 3
+    case = Case(K, N, M, seed=95)
+    buf = torch.full((M * N + 512,), 12345.0, dtype=torch.float32, device="cuda")
+    y = buf[256:256 + M * N]
+    fd.fdqp_run(fresh, case.x_dev, case.W_dev, y, M, K, N)
+    torch.cuda.synchronize()
+    host = buf.cpu().numpy()
+    assert np.all(host[:256] == 12345.0) and np.all(host[256 + M * N:] == 12345.0)
+    y_ref, a_ref = case.reference()
+    assert_close(host[256:256 + M * N].reshape(M, N), y_ref, a_ref, "guarded output")
+
+
+def test_argument_errors_launch_nothing(fresh):
+    K, N, M = 256, 64, 1
+    case = Case(K, N, M, seed=96)
+    y = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+    lib = fd.load_library()
+    before = fd.fdqp_launch_count(fresh)
+    s = torch.cuda.current_stream().cuda_stream
+    xp, wp, yp = case.x_dev.data_ptr(), case.W_dev.data_ptr(), y.data_ptr()
+    assert lib.fdqp_run(fresh, None, wp, yp, M, K, N, s) == 1
+    assert lib.fdqp_run(fresh, xp, wp, yp, 0, K, N, s) == 2
+    assert lib.fdqp_run(fresh, xp, wp, yp, M, K + 16, N, s) == 2
+    assert lib.fdqp_run(fresh, xp, wp, yp, M, K, N + 16, s) == 2
+    assert lib.fdqp_run(fresh, xp + 2, wp, yp, M, K, N, s) == 3
+    assert lib.fdqp_run(fresh, xp, wp + 8, yp, M, K, N, s) == 3
+    assert lib.fdqp_run(fresh, xp, wp, yp + 4, M, K, N, s) == 3
+    assert lib.fdqp_run(fresh, xp, wp, yp, MAX_M + 1, K, N, s) == 4
+    assert lib.fdqp_run(fresh, xp, wp, yp, M, MAX_K + 32, N, s) == 4
+    assert lib.fdqp_dequant(fresh, wp, yp, 2, K, N, s) == 1
+    assert lib.fdqp_set_param(fresh, b"no_such_key", 1) == 1
+    assert lib.fdqp_set_param(fresh, b"split_k", 3) == 1
+    assert fd.fdqp_launch_count(fresh) == before
+    assert "fdqp_gemv_kernel" in fd.fdqp_describe(fresh, 1, 2560, 10240)
+
+
+def test_run_host_roundtrip(fresh):
+    K, N, M = 2560, 2048, 2
+    case = Case(K, N, M, seed=97)
+    x_host = torch.from_numpy(case.x.view(np.int16)).pin_memory()
+    y_host = torch.empty((M, N), dtype=torch.float32).pin_memory()
+    fd.fdqp_run_host(fresh, x_host, case.W_dev, y_host, M, K, N)
+    y_ref, a_ref = case.reference()
+    assert_close(y_host.numpy(), y_ref, a_ref, "run_host")
+    assert np.array_equal(y_host.numpy(), case.run(fresh))
