@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of the FusedDQP hot path on B200.
+
+A step is one Gemma3-4B decoder layer at M = 1: the seven Q4NX projections q, k, v, o, gate, up, down
+(59.1 MB of packed weights) on seeded synthetic inputs.  Several distinct copies of the layer's weights are
+resident in HBM and the steps rotate through them, so every timed step streams its weights from HBM and not
+from L2.  The metric is the achieved bandwidth over the algorithmic bytes of the step
+(0.625*K*N + 2*M*K + 4*M*N per projection); decode tokens/s (projections only: 34 layers + LM head) is
+reported beside it.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  With --impl reference the CPU oracle is timed instead, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import synthgen  # noqa: E402
+
+METRIC = "fused Q4NX dequant-GEMV achieved HBM GB/s & % of peak; decode tokens/s (1 GPU)"
+WORKLOAD = "Gemma3-4B decoder layer at M=1: q,k,v,o,gate,up,down Q4NX group-32 projections (seeds 1-7)"
+L2_BYTES = 126e6
+LAYER_COPIES = 8            # distinct weight sets resident in HBM (8 x 59 MB = 472 MB >> L2)
+NOMINAL_HBM_GBS = 8000.0
+
+
+def alg_bytes(M, K, N):
+    return 0.625 * K * N + 2 * M * K + 4 * M * N
+
+
+def layer_bytes(M=1):
+    return sum(alg_bytes(M, K, N) for _, K, N, _ in synthgen.GEMMA3_4B_LAYER)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons in the background during the timed region."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+                power.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------- reference arm
+
+def run_reference(args, rank, world):
+    """Times the CPU oracle (as it stands) on the host cores: each step is one pass of the decoder layer's
+    seven projections at M = 1 over the same seeded inputs, all output columns, OpenMP over columns."""
+    if rank != 0:
+        return
+    import oracle
+    cores = min(oracle.max_threads(), os.cpu_count() or 1)
+    layer = [(name, K, N, synthgen.weights(seed, K, N), synthgen.activations(seed, 1, K))
+             for name, K, N, seed in synthgen.GEMMA3_4B_LAYER]
+
+    def one_pass():
+        for _, K, N, w, x in layer:
+            oracle.project(x, w.codes, w.scales, w.offsets, nthreads=cores)
+
+    for _ in range(args.warmup):
+        one_pass()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one_pass()
+    dt = time.perf_counter() - t0
+    gbs = layer_bytes() * args.steps / dt / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "note": "CPU oracle (fp64, plain C, OpenMP over output columns)"},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                         "sample": "whole layer, all 7 projections, all outputs, per step"},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------- our arm
+
+def run_ours(args, rank, local_rank, world):
+    import torch
+
+    import paper_2602_06063_b200 as fd
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the FusedDQP library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peaks, peak_kind = measured_peaks()
+    M = 1
+    shapes = synthgen.GEMMA3_4B_LAYER
+    max_K = max(K for _, K, _, _ in shapes)
+    _, hk, hn, hseed = synthgen.GEMMA3_4B_LM_HEAD
+    ctx = fd.fdqp_create(local_rank, 8, max(max_K, hk), max(max(N for _, _, N, _ in shapes), hn))
+    if args.param:
+        for kv in args.param:
+            key, val = kv.split("=")
+            fd.fdqp_set_param(ctx, key, int(val))
+
+    # ---- resident inputs: LAYER_COPIES distinct weight sets, one x and one y per projection
+    copies = []
+    host_layer0 = None
+    for c in range(LAYER_COPIES):
+        layer = []
+        for name, K, N, seed in shapes:
+            w = synthgen.weights(seed + 1000 * c, K, N)
+            packed = fd.q4nx_pack(w.codes, w.scales, w.offsets)
+            layer.append(torch.from_numpy(packed).cuda())
+            if c == 0:
+                host_layer0 = host_layer0 or []
+                host_layer0.append(w)
+        copies.append(layer)
+    xs_host = [synthgen.activations(seed, M, K) for _, K, _, seed in shapes]
+    xs = [torch.from_numpy(x.view(np.int16)).cuda() for x in xs_host]
+    ys = [torch.empty((M, N), dtype=torch.float32, device="cuda") for _, _, N, _ in shapes]
+    stream = torch.cuda.Stream()
+    sraw = stream.cuda_stream
+
+    def enqueue_layer(c):
+        for i, (_, K, N, _) in enumerate(shapes):
+            fd.fdqp_run(ctx, xs[i], copies[c][i], ys[i], M, K, N, sraw)
+
+    # one CUDA graph per weight copy: the seven launches of a step replay without per-launch host cost
+    graphs = None
+    if args.graph:
+        graphs = []
+        with torch.cuda.stream(stream):
+            enqueue_layer(0)
+        stream.synchronize()
+        for c in range(LAYER_COPIES):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                enqueue_layer(c)
+            graphs.append(g)
+
+    def step(i):
+        c = i % LAYER_COPIES
+        if graphs is not None:
+            with torch.cuda.stream(stream):
+                graphs[c].replay()
+        else:
+            enqueue_layer(c)
+
+    for i in range(args.warmup):
+        step(i)
+    stream.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches_before = fd.fdqp_launch_count(ctx)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(args.warmup + i)
+    ev1.record(stream)
+    stream.synchronize()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    kernels_per_step = len(shapes)
+    launches = kernels_per_step * args.steps
+    if graphs is None:
+        assert fd.fdqp_launch_count(ctx) - launches_before == launches
+    clocks = sampler.stop() if rank == 0 else None
+    if fd.fdqp_last_status(ctx) != 0:
+        raise SystemExit("bench.py: a kernel reported " + fd.fdqp_status_string(fd.fdqp_last_status(ctx)))
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # ---- end to end: host x in, host y out, through fdqp_run_host (pinned buffers), every step
+    xs_pin = [torch.from_numpy(x.view(np.int16)).pin_memory() for x in xs_host]
+    ys_pin = [torch.empty((M, N), dtype=torch.float32).pin_memory() for _, _, N, _ in shapes]
+    e2e_steps = max(3, min(args.steps, 200))
+
+    def e2e_step(i):
+        c = i % LAYER_COPIES
+        for j, (_, K, N, _) in enumerate(shapes):
+            fd.fdqp_run_host(ctx, xs_pin[j], copies[c][j], ys_pin[j], M, K, N, sraw)
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        e2e_step(3 + i)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+
+    # ---- LM head (M = 1) for the tokens/s figure: 34 layers + head, projections only
+    head_ms = None
+    if rank == 0 and not args.no_head:
+        hw = synthgen.weights(hseed, hk, hn)
+        hW = torch.from_numpy(fd.q4nx_pack(hw.codes, hw.scales, hw.offsets)).cuda()
+        del hw
+        hx = torch.from_numpy(synthgen.activations(hseed, 1, hk).view(np.int16)).cuda()
+        hy = torch.empty((1, hn), dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            fd.fdqp_run(ctx, hx, hW, hy, 1, hk, hn, sraw)
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record(stream)
+        for _ in range(10):
+            fd.fdqp_run(ctx, hx, hW, hy, 1, hk, hn, sraw)
+        h1.record(stream)
+        stream.synchronize()
+        head_ms = h0.elapsed_time(h1) / 10
+
+    # ---- CPU baseline: the oracle on the host cores, one pass over the same layer (rank 0, N = 1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        import oracle
+        cores = min(oracle.max_threads(), os.cpu_count() or 1)
+        t0 = time.perf_counter()
+        passes = 0
+        while passes < 1 or (time.perf_counter() - t0 < 10 and passes < 50):
+            for w, x in zip(host_layer0, xs_host):
+                oracle.project(x, w.codes, w.scales, w.offsets, nthreads=cores)
+            passes += 1
+        dt = time.perf_counter() - t0
+        cpu = {"value": layer_bytes(M) * passes / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+               "sample": f"{passes} pass(es) of the whole layer (7 projections, all outputs), {dt:.1f} s"}
+
+    if rank == 0:
+        step_bytes = layer_bytes(M)
+        gbs = step_bytes * args.steps * world / (ms * 1e-3) / 1e9
+        per_launch_us = ms * 1e3 / launches
+        achieved = (step_bytes / kernels_per_step) / (per_launch_us * 1e-6) / 1e9
+        layer_ms = ms / args.steps
+        line = {
+            "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": layer_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "M": M, "bytes_per_step": step_bytes, "cuda_graph": bool(graphs),
+                       "l2": f"inputs larger than L2: steps rotate over {LAYER_COPIES} distinct weight sets "
+                             f"({LAYER_COPIES * step_bytes / 1e6:.0f} MB)",
+                       "multi_gpu": "independent replicas, no collective",
+                       "launch": fd.fdqp_describe(ctx, 1, 2560, 10240)},
+            "frac_of_nominal_8TBps": gbs / world / NOMINAL_HBM_GBS,
+            "decode_tokens_per_s": (1e3 / (synthgen.GEMMA3_4B_LAYERS * layer_ms + head_ms)) if head_ms else None,
+            "lm_head_ms": head_ms,
+            "lm_head_gbs": (alg_bytes(1, hk, hn) / (head_ms * 1e-3) / 1e9) if head_ms else None,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_kind": peak_kind,
+                         "kernel": "fdqp_gemv_kernel", "launch_us": per_launch_us},
+            "cpu_baseline": cpu,
+            "e2e": {"value": step_bytes * e2e_steps * world / e2e_s / 1e9, "unit": "GB/s",
+                    "h2d_bytes_per_step": sum(2 * M * K for _, K, _, _ in shapes),
+                    "d2h_bytes_per_step": sum(4 * M * N for _, _, N, _ in shapes), "ms_per_step": e2e_s / e2e_steps * 1e3},
+            "gpu_launches": launches,
+            "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    fd.fdqp_destroy(ctx)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--graph", type=int, default=1, help="replay each step from a CUDA graph (default 1)")
+    ap.add_argument("--param", action="append", help="library launch parameter key=value (repeatable)")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-head", action="store_true", help="skip the LM-head timing")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        if args.steps == 400 and args.warmup == 20:
+            args.steps, args.warmup = 5, 1
+        run_reference(args, rank, world)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+    run_ours(args, rank, local_rank, world)
+
+
+if __name__ == "__main__":
+    main()

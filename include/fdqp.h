@@ -163,9 +163,10 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "path"          0 = dispatch on M (default), 1 = force the plain CUDA-core kernel
  *   "ctas_per_sm"   persistent CTAs per SM for the GEMV kernels (1 or 2; 2 implies 8 consumer warps)
  *   "consumer_warps" 8 or 16 consumer warps per CTA
- *   "stages"        shared-memory ring depth in Q4NX blocks
+ *   "stages"        shared-memory ring depth in stages (a stage holds consumer_warps / 4 Q4NX blocks)
  *   "split_k"       number of K slices (1, 2 or 4)
  *   "l2_evict_first" 1 = weight copies carry an evict-first L2 hint
+ *   "debug"         measurement aid: 1 = the GEMV consumers skip the arithmetic (y is then undefined)
  * Unknown key or unusable value: FDQP_ERR_ARG.  Meant for benchmarks and tests. */
 FDQP_API fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t value);
 

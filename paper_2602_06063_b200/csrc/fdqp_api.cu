@@ -35,7 +35,7 @@ struct fdqp_ctx {
     int64_t launches = 0;
     std::string last_err;
     // overrides (-1 = automatic)
-    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1;
+    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1;
 };
 
 namespace {
@@ -101,27 +101,29 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     int Gz = grid / Z;
     if (Gz < 1) Gz = 1;
     p->Gz = Gz;
-    // shared-memory carve-up
+    // shared-memory carve-up: ring of stages (cw / 4 blocks each), staged x, per-group sums, partial rows, barriers
+    const uint32_t stage_bytes = (uint32_t)(cw / 4) * kBlockBytes;
     const uint32_t tiles = (uint32_t)nbz * 8u;
     const uint32_t xs_bytes = tiles * 64u * (uint32_t)M;
-    const uint32_t xsum_bytes = tiles * kMaxTokens * 4u;
+    const uint32_t xsum_bytes = tiles * (M == 1 ? 8u : 64u);
     const uint32_t part_bytes = 2u * (uint32_t)cw * kStripRows * (uint32_t)M * 4u;
     const uint32_t fixed = round_up(xs_bytes, 128) + 128 + round_up(xsum_bytes, 128) + round_up(part_bytes, 128) +
                            (2u * kMaxStages + 4u) * 8u + 128u;
     const uint32_t per_cta = (uint32_t)ctx->smem_optin / (uint32_t)ctas_per_sm - (ctas_per_sm > 1 ? 1024u : 0u);
-    if (fixed + 2u * kBlockBytes > per_cta) return false;
-    int nstage = (int)((per_cta - fixed) / kBlockBytes);
+    if (fixed + 2u * stage_bytes > per_cta) return false;
+    int nstage = (int)((per_cta - fixed) / stage_bytes);
     if (nstage > kMaxStages) nstage = kMaxStages;
     if (ctx->p_stages > 0 && ctx->p_stages < nstage) nstage = (int)ctx->p_stages;
-    if (nstage < cw / 8) return false;
+    if (nstage < 2) return false;
     p->nstage = nstage;
-    p->off_xs = (uint32_t)nstage * kBlockBytes;
+    p->off_xs = (uint32_t)nstage * stage_bytes;
     p->off_zero = p->off_xs + round_up(xs_bytes, 128);
     p->off_xsum = p->off_zero + 128;
     p->off_part = p->off_xsum + round_up(xsum_bytes, 128);
     p->off_bar = p->off_part + round_up(part_bytes, 128);
     p->smem_bytes = p->off_bar + (2u * (uint32_t)nstage + 4u) * 8u;
     p->evict_first = ctx->p_evict >= 0 ? (ctx->p_evict != 0) : 1;
+    p->debug = ctx->p_debug > 0 ? (int)ctx->p_debug : 0;
     p->ws_edge = ctx->ws_edge;
     p->ws_full = ctx->ws_full;
     p->tickets = ctx->tickets;
@@ -306,6 +308,8 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
     } else if (!std::strcmp(key, "l2_evict_first")) {
         if (v > 1) return FDQP_ERR_ARG;
         ctx->p_evict = v;
+    } else if (!std::strcmp(key, "debug")) {
+        ctx->p_debug = v;
     } else {
         return FDQP_ERR_ARG;
     }

@@ -8,15 +8,15 @@
 // instruction (mma.sync m16n8k16): A = 16 output rows x 16 k of codes, B = 16 k x 8 token columns of
 // x, fp32 accumulate.  Codes are turned into bf16 with one logic op per pair
 //     ((word >> 4i) & 0x000F000F) | 0x43004300  ->  bf16x2 (128 + q_i, 128 + q_{i+4})
-// (exact), the +128 is folded into the offset term (m - 128 d) * sum_k x_k, and the order of k inside
-// a group is a free permutation as long as x is staged with the same one.
+// (exact); the +128 is cancelled by starting the accumulator at -128 * sum_k x_k, and the order of k
+// inside a group is a free permutation as long as x is staged with the same one.
 //
 // Data movement.  The packed matrix is strip-major (32 output rows x all of K contiguous), so every
-// CTA streams one contiguous byte range of HBM exactly once: a producer thread issues one 1-D bulk
-// async copy per Q4NX block (<= 5120 bytes) into a shared-memory ring guarded by mbarriers; each of
-// the 8 consumer warps of a warp group owns one 32 x 32 group-tile of the block.  x (the CTA's K
-// slice, all tokens) is staged once per CTA in the fragment order the MMA wants, together with the
-// per-group sums of x.
+// CTA streams one contiguous byte range of HBM exactly once.  The producer warp issues one 1-D bulk
+// async copy per Q4NX block (<= 5120 bytes), several lanes at a time, into a shared-memory ring of
+// multi-block stages guarded by mbarriers; every consumer warp owns the same 32 x 32 group-tile of
+// two blocks of a stage.  x (the CTA's K slice, all tokens) is staged once per CTA in the fragment
+// order the MMA wants, together with the per-group sums of x.
 //
 // Work split.  The (K-slice, strip, block) space is cut into equal contiguous ranges, one per
 // persistent CTA, so all SMs stream the same number of bytes whatever N and K are.  A strip whose
@@ -45,10 +45,79 @@ __device__ __forceinline__ float* piece_slot(const GemvPlan& p, int z, int64_t c
     return p.ws_edge + (((int64_t)z * p.Gz + ci) * 2 + which) * (kStripRows * kMaxTokens);
 }
 
+// Registers of one 32 x 32 group-tile in flight.
+struct TileRegs {
+    uint32_t c[4];   // code words: word q of rows g, g+8, g+16, g+24
+    uint32_t so[4];  // (d[g], d[g+8]), (d[g+16], d[g+24]), (m[g], m[g+8]), (m[g+16], m[g+24]) as bf16 pairs
+    uint4 xb;        // B fragments of the two k16 steps
+    float xs[4];     // sum of x over the group for tokens 2q, 2q+1, and -128 times it
+    float d0[4], d1[4];
+};
+
+#define FDQP_UNPACK(w, sh) ((((w) >> (sh)) & 0x000F000Fu) | 0x43004300u)
+
+template <int NT>
+__device__ __forceinline__ void tile_load(TileRegs& t, uint32_t code_addr, uint32_t so_addr, uint32_t x_addr,
+                                          uint32_t xsum_addr) {
+    ldmatrix_x4(t.c, code_addr);
+    ldmatrix_x4_trans(t.so, so_addr);
+    t.xb = lds128(x_addr);
+    if (NT == 1) {
+        const float2 v = lds64f(xsum_addr);  // {X, -128 X} of token 2q
+        t.xs[0] = v.x;
+        t.xs[1] = 0.f;
+        t.xs[2] = v.y;
+        t.xs[3] = 0.f;
+    } else {
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                     : "=f"(t.xs[0]), "=f"(t.xs[1]), "=f"(t.xs[2]), "=f"(t.xs[3])
+                     : "r"(xsum_addr));  // {X0, X1, -128 X0, -128 X1}
+    }
+}
+
+__device__ __forceinline__ void tile_mma(TileRegs& t) {
+    const float cinit[4] = {t.xs[2], t.xs[3], t.xs[2], t.xs[3]};  // -128 * sum x cancels the code bias
+    {
+        const uint32_t lo = t.c[0], hi = t.c[1];
+        mma_bf16_16816(t.d0, FDQP_UNPACK(lo, 0), FDQP_UNPACK(hi, 0), FDQP_UNPACK(lo, 4), FDQP_UNPACK(hi, 4), t.xb.x,
+                       t.xb.y, cinit);
+        mma_bf16_16816(t.d0, FDQP_UNPACK(lo, 8), FDQP_UNPACK(hi, 8), FDQP_UNPACK(lo, 12), FDQP_UNPACK(hi, 12), t.xb.z,
+                       t.xb.w, t.d0);
+    }
+    {
+        const uint32_t lo = t.c[2], hi = t.c[3];
+        mma_bf16_16816(t.d1, FDQP_UNPACK(lo, 0), FDQP_UNPACK(hi, 0), FDQP_UNPACK(lo, 4), FDQP_UNPACK(hi, 4), t.xb.x,
+                       t.xb.y, cinit);
+        mma_bf16_16816(t.d1, FDQP_UNPACK(lo, 8), FDQP_UNPACK(hi, 8), FDQP_UNPACK(lo, 12), FDQP_UNPACK(hi, 12), t.xb.z,
+                       t.xb.w, t.d1);
+    }
+}
+
+// acc[row][tok] += d * (sum_k q_k x_k) + m * (sum_k x_k), in fp32 (Eq. 3 applied per group)
+template <int NT>
+__device__ __forceinline__ void tile_scale(const TileRegs& t, float (&acc)[4][NT]) {
+    const float dsc[4] = {bf16_lo_to_f32(t.so[0]), bf16_hi_to_f32(t.so[0]), bf16_lo_to_f32(t.so[1]),
+                          bf16_hi_to_f32(t.so[1])};
+    const float mof[4] = {bf16_lo_to_f32(t.so[2]), bf16_hi_to_f32(t.so[2]), bf16_lo_to_f32(t.so[3]),
+                          bf16_hi_to_f32(t.so[3])};
+    const float dd[4][2] = {{t.d0[0], t.d0[1]}, {t.d0[2], t.d0[3]}, {t.d1[0], t.d1[1]}, {t.d1[2], t.d1[3]}};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+            acc[i][j] = fmaf(dsc[i], dd[i][j], acc[i][j]);
+            acc[i][j] = fmaf(mof[i], t.xs[j], acc[i][j]);
+        }
+}
+
+// CW consumer warps (8 or 16); NT token columns kept per lane (1 when M == 1, else 2).
+// A ring stage holds CB = CW / 4 blocks; warp w owns group-tile (w & 7) of blocks 2*(w >> 3) and
+// 2*(w >> 3) + 1 of every stage.
 template <int CW, int NT>
 __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __grid_constant__ GemvPlan p) {
     extern __shared__ __align__(128) uint8_t smem[];
-    constexpr int NBP = CW / 8;  // blocks in flight per CTA step: one per warp group
+    constexpr int CB = CW / 4;
+    constexpr uint32_t kStageBytes = CB * kBlockBytes;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int M = p.M, K = p.K;
 
@@ -60,74 +129,102 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
     const int64_t a = range_begin(ci, p.Gz, T), e = range_begin(ci + 1, p.Gz, T);
     const int nblk = (int)(e - a);
     if (nblk <= 0) return;
+    const int64_t s_first = a / len;
+    const int bl_first = (int)(a - s_first * len);           // block index inside the slice of the CTA's first block
+    const int npieces = (int)((e - 1) / len - s_first) + 1;  // strips this CTA touches
+    const int nchunk = (nblk + CB - 1) / CB;
 
     const uint32_t ring = smem_u32(smem);
     const uint32_t xs = ring + p.off_xs, zero_slot = ring + p.off_zero, xsum = ring + p.off_xsum;
     const uint32_t part = ring + p.off_part, bars = ring + p.off_bar;
     const int nstage = p.nstage;
-    auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (nstage + s); };
-    auto red_full = [&](int par) { return bars + 8u * (2 * nstage + par); };
-    auto red_empty = [&](int par) { return bars + 8u * (2 * nstage + 2 + par); };
+    const uint32_t full0 = bars, empty0 = bars + 8u * nstage;
+    const uint32_t red_full0 = bars + 16u * nstage, red_empty0 = red_full0 + 16u;
 
-    if (tid == 0) {
-        for (int s = 0; s < nstage; ++s) {
-            mbar_init(full_bar(s), 1);
-            mbar_init(empty_bar(s), 8);
-        }
-        for (int par = 0; par < 2; ++par) {
-            mbar_init(red_full(par), CW);
-            mbar_init(red_empty(par), 1);
-        }
-        mbar_fence_init();
+    for (int s = tid; s < nstage; s += blockDim.x) {
+        mbar_init(full0 + 8u * s, 1);
+        mbar_init(empty0 + 8u * s, CW);
     }
+    if (tid < 2) {
+        mbar_init(red_full0 + 8u * tid, CW);
+        mbar_init(red_empty0 + 8u * tid, 1);
+    }
+    mbar_fence_init();
     __syncthreads();
 
     const int groups_total = K / kGroup;
     const int64_t strip_bytes = (int64_t)kGroupBytes * groups_total;
-    auto block_groups = [&](int b) {
-        const int rest = groups_total - 8 * b;
-        return rest < 8 ? rest : 8;
-    };
 
-    // ---- producer state (warp CW, lane 0) and first fills: start the HBM stream before staging x
-    const bool is_producer = (warp == CW) && (lane == 0);
-    int64_t prod_s = 0;
-    int prod_bl = 0, prod_i = 0, prod_stage = 0;
-    uint64_t policy = 0;
-    if (is_producer) {
+    if (warp == CW) {
+        // =============================== producer ================================================
+        // Lane j < CB copies block j of every stage; lane 0 owns the barrier traffic.
+        uint64_t policy = 0;
         if (p.evict_first) policy = l2_policy_evict_first();
-        prod_s = a / len;
-        prod_bl = (int)(a - prod_s * len);
-        const int first = nblk < nstage ? nblk : nstage;
-        for (; prod_i < first; ++prod_i) {
-            const int b = b_first + prod_bl;
-            const uint32_t bytes = (uint32_t)(kGroupBytes * block_groups(b));
-            const uint8_t* src = p.W + prod_s * strip_bytes + (int64_t)b * kBlockBytes;
-            mbar_arrive_expect_tx(full_bar(prod_stage), bytes);
-            if (p.evict_first)
-                bulk_g2s_hint(ring + prod_stage * kBlockBytes, src, bytes, full_bar(prod_stage), policy);
-            else
-                bulk_g2s(ring + prod_stage * kBlockBytes, src, bytes, full_bar(prod_stage));
-            if (++prod_bl == len) { prod_bl = 0; ++prod_s; }
-            if (++prod_stage == nstage) prod_stage = 0;
+        int64_t ps = s_first;
+        int pbl = bl_first + lane;  // only meaningful for lane < CB
+        while (pbl >= len) { pbl -= len; ++ps; }
+        int stage = 0;
+        uint32_t phase = 0;  // parity of the stage's previous use
+        bool alive = true;
+        int c = 0;
+        for (; c < nchunk && alive; ++c) {
+            if (c >= nstage) {
+                int ok = 1;
+                if (lane == 0) ok = mbar_wait(empty0 + 8u * stage, phase ^ 1u, p.status) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { alive = false; break; }
+            }
+            const int i = c * CB + lane;
+            uint32_t bytes = 0;
+            if (lane < CB && i < nblk) {
+                const int rest = groups_total - 8 * (b_first + pbl);
+                bytes = (uint32_t)kGroupBytes * (uint32_t)(rest < 8 ? rest : 8);
+            }
+            const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+            if (lane == 0) mbar_arrive_expect_tx(full0 + 8u * stage, total);
+            __syncwarp();
+            if (bytes) {
+                const uint8_t* src = p.W + ps * strip_bytes + (int64_t)(b_first + pbl) * kBlockBytes;
+                const uint32_t dst = ring + stage * kStageBytes + lane * kBlockBytes;
+                if (p.evict_first)
+                    bulk_g2s_hint(dst, src, bytes, full0 + 8u * stage, policy);
+                else
+                    bulk_g2s(dst, src, bytes, full0 + 8u * stage);
+            }
+            pbl += CB;
+            while (pbl >= len) { pbl -= len; ++ps; }
+            if (++stage == nstage) { stage = 0; phase ^= 1u; }
         }
+        // Do not leave while a copy into this CTA's shared memory may still be in flight.
+        if (lane == 0) {
+            const int issued = c;
+            const int from = issued > nstage ? issued - nstage : 0;
+            for (int k = from; k < issued; ++k)
+                if (!mbar_wait(full0 + 8u * (k % nstage), (k / nstage) & 1, p.status)) break;
+        }
+        return;
     }
 
-    // ---- stage this CTA's K slice of x: fragment order for the MMA, plus per-group sums
+    // ---- consumers and reducer: stage this CTA's K slice of x (fragment order + per-group sums)
     {
+        const int nthr = (CW + 1) * 32;
+        const int t2 = warp < CW ? tid : tid - 32;  // skip the producer warp's ids
         const int kbeg = b_first * kBlockK;
         const int kend_full = (b_first + len) * kBlockK;
         const int kend = kend_full < K ? kend_full : K;
         const int ntiles = (kend - kbeg) / kGroup;
         uint8_t* xs_g = smem + p.off_xs;
         float* xsum_g = reinterpret_cast<float*>(smem + p.off_xsum);
-        for (int i = tid; i < ntiles * kMaxTokens; i += blockDim.x)
-            if ((i & 7) >= M) xsum_g[i] = 0.f;
-        if (tid < 16) reinterpret_cast<uint32_t*>(smem + p.off_zero)[tid] = 0u;
+        const int xsum_stride = (NT == 1) ? 2 : 4 * 4;  // floats per tile: {X,-128X} or 4 quads of {X0,X1,-128X0,-128X1}
+        if (NT == 2)
+            for (int i = t2; i < ntiles * 16; i += nthr) {
+                const int tok = ((i >> 2) & 3) * 2 + (i & 1);  // slot i holds token 2q + (i & 1), q = (i >> 2) & 3
+                if (tok >= M) xsum_g[i] = 0.f;
+            }
+        if (t2 < 16) reinterpret_cast<uint32_t*>(smem + p.off_zero)[t2] = 0u;
         const int items = ntiles * M * 4;
-        for (int base = 0; base < items; base += blockDim.x) {
-            const int idx = base + tid;
+        for (int base = 0; base < items; base += nthr) {
+            const int idx = base + t2;
             const bool valid = idx < items;
             float psum = 0.f;
             const int q = idx & 3, tm = idx >> 2;
@@ -146,25 +243,35 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
             }
             psum += __shfl_xor_sync(0xffffffffu, psum, 1);
             psum += __shfl_xor_sync(0xffffffffu, psum, 2);
-            if (valid && q == 0) xsum_g[tile * kMaxTokens + tok] = psum;
+            if (valid && q == 0) {
+                if (NT == 1) {
+                    xsum_g[tile * 2] = psum;
+                    xsum_g[tile * 2 + 1] = -128.f * psum;
+                } else {
+                    float* dst = xsum_g + tile * xsum_stride + (tok >> 1) * 4 + (tok & 1);
+                    dst[0] = psum;
+                    dst[2] = -128.f * psum;
+                }
+            }
         }
+        asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
     }
-    __syncthreads();
 
     if (warp < CW) {
         // =============================== consumers ===============================================
-        const int wg = warp >> 3, tw = warp & 7;
+        const int tw = warp & 7, j0 = (warp >> 3) * 2;
         const int g = lane >> 2, q = lane & 3;
         const uint32_t x_lane = (g < M) ? xs + g * 64 + q * 16 : zero_slot;
         const uint32_t x_stride = (g < M) ? (uint32_t)M * 64u : 0u;
-        const uint32_t xsum_lane = xsum + q * 8;
+        const uint32_t xsum_lane = (NT == 1) ? xsum : xsum + q * 16;
+        const uint32_t xsum_stride = (NT == 1) ? 8u : 64u;
         // ldmatrix source rows: codes = row `lane` of the tile; scales/offsets = the four 16-byte
         // chunks of this tile's scale words and of its offset words, duplicated so that after the
         // transposed load every lane of a quad holds (d[g], d[g+8]), (d[g+16], d[g+24]), (m..), (m..)
         const uint32_t code_lane = tw * 512 + lane * 16;
         const int mat = lane >> 3;
         const uint32_t so_chunk = tw * 64 + (((mat & 1) * 2 + (lane & 1)) * 16);
-        const bool so_is_offset = mat >= 2;
+        const uint32_t so_sect = mat >= 2 ? 576u : 512u;  // offsets section follows the scales section
 
         float acc[4][NT];
 #pragma unroll
@@ -172,78 +279,12 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
 #pragma unroll
             for (int j = 0; j < NT; ++j) acc[i][j] = 0.f;
 
-        int i_rel = wg;                 // index of this group's next block relative to `a`
-        int stage = wg % nstage;        // its ring stage
-        uint32_t phase = (wg / nstage) & 1;
         int piece = 0;
         bool alive = true;
-        int64_t pa = a;
-        while (pa < e && alive) {
-            const int64_t s = pa / len;
-            const int64_t unit_end = (s + 1) * len;
-            const int64_t pe = unit_end < e ? unit_end : e;
-            int bl = (int)(a + i_rel - s * len);  // block index inside the slice for i_rel (valid when inside piece)
-            const int i_end = (int)(pe - a);
-            for (; i_rel < i_end; i_rel += NBP, bl += NBP) {
-                const int b = b_first + bl;
-                const int jb = block_groups(b);
-                if (!mbar_wait(full_bar(stage), phase, p.status)) { alive = false; break; }
-                if (tw < jb) {
-                    const uint32_t sbase = ring + stage * kBlockBytes;
-                    uint32_t c[4], so[4];
-                    ldmatrix_x4(c, sbase + code_lane);
-                    ldmatrix_x4_trans(so, sbase + (so_is_offset ? 576u : 512u) * jb + so_chunk);
-                    const int tile = bl * 8 + tw;
-                    const uint4 xb = lds128(x_lane + tile * x_stride);
-                    const float2 xs2 = lds64f(xsum_lane + tile * (kMaxTokens * 4));
-                    const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
-                    float d0[4], d1[4];
-                    {
-                        const uint32_t lo = c[0], hi = c[1];
-                        mma_bf16_16816(d0, (lo & 0x000F000Fu) | 0x43004300u, (hi & 0x000F000Fu) | 0x43004300u,
-                                       ((lo >> 4) & 0x000F000Fu) | 0x43004300u, ((hi >> 4) & 0x000F000Fu) | 0x43004300u,
-                                       xb.x, xb.y, zero4);
-                        mma_bf16_16816(d0, ((lo >> 8) & 0x000F000Fu) | 0x43004300u,
-                                       ((hi >> 8) & 0x000F000Fu) | 0x43004300u,
-                                       ((lo >> 12) & 0x000F000Fu) | 0x43004300u,
-                                       ((hi >> 12) & 0x000F000Fu) | 0x43004300u, xb.z, xb.w, d0);
-                    }
-                    {
-                        const uint32_t lo = c[2], hi = c[3];
-                        mma_bf16_16816(d1, (lo & 0x000F000Fu) | 0x43004300u, (hi & 0x000F000Fu) | 0x43004300u,
-                                       ((lo >> 4) & 0x000F000Fu) | 0x43004300u, ((hi >> 4) & 0x000F000Fu) | 0x43004300u,
-                                       xb.x, xb.y, zero4);
-                        mma_bf16_16816(d1, ((lo >> 8) & 0x000F000Fu) | 0x43004300u,
-                                       ((hi >> 8) & 0x000F000Fu) | 0x43004300u,
-                                       ((lo >> 12) & 0x000F000Fu) | 0x43004300u,
-                                       ((hi >> 12) & 0x000F000Fu) | 0x43004300u, xb.z, xb.w, d1);
-                    }
-                    // per-group scale and offset, fp32: rows g, g+8, g+16, g+24
-                    const float dsc[4] = {bf16_lo_to_f32(so[0]), bf16_hi_to_f32(so[0]), bf16_lo_to_f32(so[1]),
-                                          bf16_hi_to_f32(so[1])};
-                    const float mof[4] = {bf16_lo_to_f32(so[2]), bf16_hi_to_f32(so[2]), bf16_lo_to_f32(so[3]),
-                                          bf16_hi_to_f32(so[3])};
-                    const float dd[4][2] = {{d0[0], d0[1]}, {d0[2], d0[3]}, {d1[0], d1[1]}, {d1[2], d1[3]}};
-                    const float xsv[2] = {xs2.x, xs2.y};
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float cc = fmaf(dsc[i], -128.f, mof[i]);  // offset with the +128 code bias folded in
-#pragma unroll
-                        for (int j = 0; j < NT; ++j) {
-                            acc[i][j] = fmaf(dsc[i], dd[i][j], acc[i][j]);
-                            acc[i][j] = fmaf(cc, xsv[j], acc[i][j]);
-                        }
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty_bar(stage));
-                stage += NBP;
-                if (stage >= nstage) { stage -= nstage; phase ^= 1u; }
-            }
-            if (!alive) break;
-            // ---- end of this strip piece: hand the warp's partial rows to the reducer warp
+        // hand the warp's partial rows of the current strip piece to the reducer warp
+        auto flush = [&]() {
             const int par = piece & 1;
-            if (piece >= 2 && !mbar_wait(red_empty(par), ((piece >> 1) - 1) & 1, p.status)) { alive = false; break; }
+            if (piece >= 2 && !mbar_wait(red_empty0 + 8u * par, ((piece >> 1) - 1) & 1, p.status)) alive = false;
             const uint32_t slot = part + (uint32_t)((par * CW + warp) * kStripRows * M) * 4u;
 #pragma unroll
             for (int i = 0; i < 4; ++i)
@@ -257,49 +298,69 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
                     acc[i][j] = 0.f;
                 }
             __syncwarp();
-            if (lane == 0) mbar_arrive(red_full(par));
+            if (lane == 0) mbar_arrive(red_full0 + 8u * par);
             ++piece;
-            pa = pe;
-        }
-    } else if (warp == CW) {
-        // =============================== producer ================================================
-        if (lane == 0) {
-            bool alive = true;
-            for (; prod_i < nblk && alive; ++prod_i) {
-                // the stage was last used by block prod_i - nstage; wait until its 8 warps released it
-                if (!mbar_wait(empty_bar(prod_stage), ((prod_i / nstage) - 1) & 1, p.status)) { alive = false; break; }
-                const int b = b_first + prod_bl;
-                const uint32_t bytes = (uint32_t)(kGroupBytes * block_groups(b));
-                const uint8_t* src = p.W + prod_s * strip_bytes + (int64_t)b * kBlockBytes;
-                mbar_arrive_expect_tx(full_bar(prod_stage), bytes);
-                if (p.evict_first)
-                    bulk_g2s_hint(ring + prod_stage * kBlockBytes, src, bytes, full_bar(prod_stage), policy);
-                else
-                    bulk_g2s(ring + prod_stage * kBlockBytes, src, bytes, full_bar(prod_stage));
-                if (++prod_bl == len) { prod_bl = 0; ++prod_s; }
-                if (++prod_stage == nstage) prod_stage = 0;
+        };
+
+        int unit_first = -bl_first;          // index (relative to the CTA's first block) of block 0 of the current strip
+        int unit_next = unit_first + len;    // ... and of the next strip
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int c = 0; c < nchunk && alive; ++c) {
+            if (!mbar_wait(full0 + 8u * stage, phase, p.status)) { alive = false; break; }
+            const uint32_t sbase = ring + stage * kStageBytes + j0 * kBlockBytes;
+            const int i0 = c * CB + j0, i1 = i0 + 1;
+            // block index inside the slice (for the staged x) and group count of both blocks
+            int bl0 = i0 - unit_first, bl1;
+            while (bl0 >= len) bl0 -= len;
+            bl1 = bl0 + 1;
+            if (bl1 >= len) bl1 -= len;
+            const int r0 = groups_total - 8 * (b_first + bl0), r1 = groups_total - 8 * (b_first + bl1);
+            const int jb0 = r0 < 8 ? r0 : 8, jb1 = r1 < 8 ? r1 : 8;
+            const bool work = !(p.debug & 1);
+            const bool act0 = work && (i0 < nblk) && (tw < jb0), act1 = work && (i1 < nblk) && (tw < jb1);
+            TileRegs ta, tb;
+            if (act0) {
+                const int tile = bl0 * 8 + tw;
+                tile_load<NT>(ta, sbase + code_lane, sbase + so_sect * jb0 + so_chunk, x_lane + tile * x_stride,
+                              xsum_lane + tile * xsum_stride);
             }
-            // Do not leave while a copy into this CTA's shared memory may still be in flight.
-            const int issued = prod_i;
-            const int from = issued > nstage ? issued - nstage : 0;
-            for (int i = from; i < issued; ++i)
-                if (!mbar_wait(full_bar(i % nstage), (i / nstage) & 1, p.status)) break;
+            if (act1) {
+                const int tile = bl1 * 8 + tw;
+                tile_load<NT>(tb, sbase + kBlockBytes + code_lane, sbase + kBlockBytes + so_sect * jb1 + so_chunk,
+                              x_lane + tile * x_stride, xsum_lane + tile * xsum_stride);
+            }
+            if (act0) tile_mma(ta);
+            if (act1) tile_mma(tb);
+            // all shared-memory reads of this stage are done: release it before the fp32 epilogue
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8u * stage);
+            if (i0 < nblk) {
+                while (i0 >= unit_next && alive) { flush(); unit_first = unit_next; unit_next += len; }
+                if (act0) tile_scale<NT>(ta, acc);
+            }
+            if (i1 < nblk) {
+                while (i1 >= unit_next && alive) { flush(); unit_first = unit_next; unit_next += len; }
+                if (act1) tile_scale<NT>(tb, acc);
+            }
+            if (++stage == nstage) { stage = 0; phase ^= 1u; }
         }
+        while (piece < npieces && alive) flush();
     } else {
         // =============================== reducer =================================================
-        int piece = 0;
         int64_t pa = a;
-        while (pa < e) {
-            const int64_t s = pa / len;
+        for (int piece = 0; piece < npieces; ++piece) {
+            const int64_t s = s_first + piece;
             const int64_t unit_begin = s * len, unit_end = unit_begin + len;
             const int64_t pe = unit_end < e ? unit_end : e;
             const int par = piece & 1;
-            if (!mbar_wait(red_full(par), (piece >> 1) & 1, p.status)) break;
+            if (!mbar_wait(red_full0 + 8u * par, (piece >> 1) & 1, p.status)) break;
             float v[kMaxTokens];
 #pragma unroll
             for (int t = 0; t < kMaxTokens; ++t) {
                 v[t] = 0.f;
                 if (t < M) {
+#pragma unroll
                     for (int w = 0; w < CW; ++w) {
                         float f;
                         asm volatile("ld.shared.f32 %0, [%1];"
@@ -311,7 +372,7 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(red_empty(par));
+            if (lane == 0) mbar_arrive(red_empty0 + 8u * par);
 
             const bool whole_unit = (pa == unit_begin) && (pe == unit_end);
             float* yrow = p.y + s * kStripRows + lane;
@@ -359,7 +420,6 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
                     if (lane == 0) p.tickets[s] = 0;  // ready for the next launch on this stream
                 }
             }
-            ++piece;
             pa = pe;
         }
     }

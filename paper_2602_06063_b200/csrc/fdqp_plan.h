@@ -28,8 +28,9 @@ struct GemvPlan {
     int Z;                // K slices
     int nbz;              // blocks per slice = ceil(nb / Z); every slice is non-empty
     int Gz;               // CTAs per slice; grid = Z * Gz
-    int nstage;           // ring depth in blocks
+    int nstage;           // ring depth in stages of (consumer warps / 4) blocks
     int evict_first;      // weight copies carry an evict-first L2 hint
+    int debug;            // measurement aid: bit 0 = consumers skip the arithmetic (results are then undefined)
     uint32_t off_xs;      // shared-memory offsets (bytes)
     uint32_t off_zero;
     uint32_t off_xsum;

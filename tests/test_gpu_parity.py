@@ -143,7 +143,10 @@ def test_zero_and_offsets_only(fresh):
     K, N, M = 1152, 64, 4
     case = Case(K, N, M, seed=66)
     zero = synthgen.Q4NXWeights(np.zeros_like(case.w.codes), case.w.scales, np.zeros_like(case.w.offsets))
-    assert np.all(Case(K, N, M, 0, weights=zero, x=case.x).run(fresh) == 0)
+    # codes 0 and offsets 0 with non-zero scales: every w_hat is 0, the bound collapses to its absolute term
+    assert np.all(np.abs(Case(K, N, M, 0, weights=zero, x=case.x).run(fresh)) <= ABS_TOL)
+    dead = synthgen.Q4NXWeights(zero.codes, np.zeros_like(case.w.scales), zero.offsets)
+    assert np.all(Case(K, N, M, 0, weights=dead, x=case.x).run(fresh) == 0)
     off = synthgen.Q4NXWeights(np.zeros_like(case.w.codes), case.w.scales, case.w.offsets)
     c = Case(K, N, M, 0, weights=off, x=case.x)
     y_ref, a_ref = c.reference()
