@@ -120,6 +120,9 @@ FDQP_API fdqp_status fdqp_destroy(fdqp_ctx* ctx);
  * from HBM through a shared-memory ring, nibbles unpacked in registers, scale and
  * offset applied in fp32, split-K across CTAs reduced in a fixed order); M >= 9
  * runs the dequantise-into-shared-memory tensor-core path.
+ * In the GEMV kernels the activations of each 32-group are held as 24-bit fixed
+ * point relative to the group's largest exponent: exact for every element within
+ * 2^15 of the group's largest magnitude, rounded to 2^-23 of it otherwise.
  * Asynchronous on `cuda_stream`; no allocation and no host synchronisation.  W, x
  * and y must stay valid until the stream has passed the call.  Two calls that
  * share a context must be ordered on one stream.
@@ -164,7 +167,7 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "ctas_per_sm"   persistent CTAs per SM for the GEMV kernels (1 or 2; 2 implies 8 consumer warps)
  *   "consumer_warps" 8 or 16 consumer warps per CTA
  *   "stages"        shared-memory ring depth in stages (a stage holds consumer_warps / 4 Q4NX blocks)
- *   "split_k"       number of K slices (1, 2 or 4)
+ *   "split_k"       number of K slices (1, 2, 4 or 8)
  *   "l2_evict_first" 1 = weight copies carry an evict-first L2 hint
  *   "debug"         measurement aid: 1 = the GEMV consumers skip the arithmetic (y is then undefined)
  * Unknown key or unusable value: FDQP_ERR_ARG.  Meant for benchmarks and tests. */

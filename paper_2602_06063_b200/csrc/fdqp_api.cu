@@ -14,6 +14,7 @@
 namespace fdqp {
 cudaError_t gemv_launch(const GemvPlan& p, int consumer_warps, cudaStream_t stream);
 cudaError_t gemv_set_smem_limit(int bytes);
+cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream);
 cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
 }  // namespace fdqp
@@ -28,6 +29,8 @@ struct fdqp_ctx {
     float* ws_edge = nullptr;
     float* ws_full = nullptr;
     int* tickets = nullptr;
+    uint32_t* xq = nullptr;      // prepared activations of the call in flight
+    float* xsc = nullptr;
     int* status_host = nullptr;  // pinned, mapped
     int* status_dev = nullptr;   // device alias of status_host
     void* x_stage = nullptr;     // fdqp_run_host staging (allocated on its first use)
@@ -41,7 +44,7 @@ struct fdqp_ctx {
 namespace {
 
 constexpr int kMaxStages = 40;
-constexpr uint32_t kXsBudget = 100u * 1024u;  // shared memory the staged activations may take
+constexpr int kMinStages = 3;  // ring depth below which another K slice is preferred
 
 struct DeviceGuard {
     int prev = -1;
@@ -70,6 +73,27 @@ fdqp_status check_shape(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     return FDQP_OK;
 }
 
+// Shared-memory carve-up for a given configuration; returns the ring depth that fits (0 if none).
+struct SmemLayout {
+    uint32_t stage_bytes, xs_bytes, xsum_bytes, part_bytes, fixed;
+    int nstage;
+};
+
+SmemLayout smem_layout(const fdqp_ctx* ctx, int M, int nbz, int cw, int ctas_per_sm) {
+    SmemLayout L;
+    L.stage_bytes = (uint32_t)(cw / 4) * kBlockBytes;
+    const uint32_t tiles = (uint32_t)nbz * 8u;
+    L.xs_bytes = tiles * 128u * (uint32_t)M;          // prepared activations of the K slice
+    L.xsum_bytes = M == 1 ? 0u : tiles * 64u;         // per-token {sum x, unit}
+    L.part_bytes = 2u * (uint32_t)cw * kStripRows * (uint32_t)M * 4u;
+    L.fixed = round_up(L.xs_bytes, 128) + round_up(L.xsum_bytes, 128) + round_up(L.part_bytes, 128) +
+              (2u * kMaxStages + 5u) * 8u + 128u;
+    const uint32_t per_cta = (uint32_t)ctx->smem_optin / (uint32_t)ctas_per_sm - (ctas_per_sm > 1 ? 1024u : 0u);
+    L.nstage = per_cta > L.fixed ? (int)((per_cta - L.fixed) / L.stage_bytes) : 0;
+    if (L.nstage > kMaxStages) L.nstage = kMaxStages;
+    return L;
+}
+
 // Fill the launch plan of one GEMV launch (M <= 8).  Returns false if no ring fits.
 bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, GemvPlan* p) {
     std::memset(p, 0, sizeof(*p));
@@ -78,20 +102,25 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     p->N = N;
     p->S = N / kStripRows;
     p->nb = (K + kBlockK - 1) / kBlockK;
-    int ctas_per_sm = ctx->p_ctas_per_sm > 0 ? (int)ctx->p_ctas_per_sm : 1;
+    // measured on B200: two 8-warp CTAs per SM stream fastest at M = 1; larger M wants the smem of one CTA
+    int ctas_per_sm = ctx->p_ctas_per_sm > 0 ? (int)ctx->p_ctas_per_sm : (M == 1 && ctx->p_cw != 16 ? 2 : 1);
     if (ctas_per_sm > kMaxCtasPerSm) ctas_per_sm = kMaxCtasPerSm;
-    // register file: one 18-warp CTA or two 10-warp CTAs fit an SM
-    const int cw = ctas_per_sm > 1 ? 8 : ((ctx->p_cw == 8 || ctx->p_cw == 16) ? (int)ctx->p_cw : 16);
-    // K slices: as few as keep the staged activations within budget
-    int Z = 1;
-    if (ctx->p_split_k > 0) {
-        Z = (int)ctx->p_split_k;
-    } else {
-        while (Z < kMaxSplit && (uint32_t)((p->nb + Z - 1) / Z) * 8u * 64u * (uint32_t)M > kXsBudget / (uint32_t)ctas_per_sm)
-            Z *= 2;
+    int cw = 16, Z = 1, nbz = p->nb;
+    SmemLayout L{};
+    for (;; --ctas_per_sm) {
+        // register file: one 19-warp CTA or two 10-warp CTAs fit an SM
+        cw = ctas_per_sm > 1 ? 8 : ((ctx->p_cw == 8 || ctx->p_cw == 16) ? (int)ctx->p_cw : 16);
+        // K slices: as few as leave a ring of at least kMinStages stages beside the staged activations
+        Z = ctx->p_split_k > 0 ? (int)ctx->p_split_k : 1;
+        for (;; Z *= 2) {
+            if (Z > p->nb) Z = p->nb;
+            nbz = (p->nb + Z - 1) / Z;
+            L = smem_layout(ctx, M, nbz, cw, ctas_per_sm);
+            if (L.nstage >= kMinStages || Z >= kMaxSplit || Z >= p->nb) break;
+        }
+        if (L.nstage >= 2 || ctas_per_sm == 1) break;
     }
-    if (Z > p->nb) Z = p->nb;
-    int nbz = (p->nb + Z - 1) / Z;
+    if (L.nstage < 2) return false;
     Z = (p->nb + nbz - 1) / nbz;  // drop slices that would be empty
     p->Z = Z;
     p->nbz = nbz;
@@ -101,32 +130,21 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     int Gz = grid / Z;
     if (Gz < 1) Gz = 1;
     p->Gz = Gz;
-    // shared-memory carve-up: ring of stages (cw / 4 blocks each), staged x, per-group sums, partial rows, barriers
-    const uint32_t stage_bytes = (uint32_t)(cw / 4) * kBlockBytes;
-    const uint32_t tiles = (uint32_t)nbz * 8u;
-    const uint32_t xs_bytes = tiles * 64u * (uint32_t)M;
-    const uint32_t xsum_bytes = tiles * (M == 1 ? 8u : 64u);
-    const uint32_t part_bytes = 2u * (uint32_t)cw * kStripRows * (uint32_t)M * 4u;
-    const uint32_t fixed = round_up(xs_bytes, 128) + 128 + round_up(xsum_bytes, 128) + round_up(part_bytes, 128) +
-                           (2u * kMaxStages + 4u) * 8u + 128u;
-    const uint32_t per_cta = (uint32_t)ctx->smem_optin / (uint32_t)ctas_per_sm - (ctas_per_sm > 1 ? 1024u : 0u);
-    if (fixed + 2u * stage_bytes > per_cta) return false;
-    int nstage = (int)((per_cta - fixed) / stage_bytes);
-    if (nstage > kMaxStages) nstage = kMaxStages;
+    int nstage = L.nstage;
     if (ctx->p_stages > 0 && ctx->p_stages < nstage) nstage = (int)ctx->p_stages;
-    if (nstage < 2) return false;
     p->nstage = nstage;
-    p->off_xs = (uint32_t)nstage * stage_bytes;
-    p->off_zero = p->off_xs + round_up(xs_bytes, 128);
-    p->off_xsum = p->off_zero + 128;
-    p->off_part = p->off_xsum + round_up(xsum_bytes, 128);
-    p->off_bar = p->off_part + round_up(part_bytes, 128);
-    p->smem_bytes = p->off_bar + (2u * (uint32_t)nstage + 4u) * 8u;
+    p->off_xs = (uint32_t)nstage * L.stage_bytes;
+    p->off_xsum = p->off_xs + round_up(L.xs_bytes, 128);
+    p->off_part = p->off_xsum + round_up(L.xsum_bytes, 128);
+    p->off_bar = p->off_part + round_up(L.part_bytes, 128);
+    p->smem_bytes = p->off_bar + (2u * (uint32_t)nstage + 5u) * 8u;
     p->evict_first = ctx->p_evict >= 0 ? (ctx->p_evict != 0) : 1;
     p->debug = ctx->p_debug > 0 ? (int)ctx->p_debug : 0;
     p->ws_edge = ctx->ws_edge;
     p->ws_full = ctx->ws_full;
     p->tickets = ctx->tickets;
+    p->xq = ctx->xq;
+    p->xsc = ctx->xsc;
     p->status = ctx->status_dev;
     *consumer_warps = cw;
     return true;
@@ -181,6 +199,11 @@ extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, in
         if ((e = cudaMalloc(&ctx->ws_full, slot * (size_t)kMaxSplit * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->tickets, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMemset(ctx->tickets, 0, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
+        const size_t tiles = (size_t)(max_K / kGroup), toks = (size_t)(max_M < kMaxTokens ? max_M : kMaxTokens);
+        if ((e = cudaMalloc(&ctx->xq, tiles * toks * 128))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMalloc(&ctx->xsc, tiles * 64))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMemset(ctx->xq, 0, tiles * toks * 128))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMemset(ctx->xsc, 0, tiles * 64))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaHostAlloc(&ctx->status_host, sizeof(int), cudaHostAllocMapped))) { st = cuda_fail(nullptr, e, ""); break; }
         *ctx->status_host = 0;
         if ((e = cudaHostGetDevicePointer(&ctx->status_dev, ctx->status_host, 0))) { st = cuda_fail(nullptr, e, ""); break; }
@@ -201,6 +224,8 @@ extern "C" fdqp_status fdqp_destroy(fdqp_ctx* ctx) {
     if (ctx->ws_edge) cudaFree(ctx->ws_edge);
     if (ctx->ws_full) cudaFree(ctx->ws_full);
     if (ctx->tickets) cudaFree(ctx->tickets);
+    if (ctx->xq) cudaFree(ctx->xq);
+    if (ctx->xsc) cudaFree(ctx->xsc);
     if (ctx->x_stage) cudaFree(ctx->x_stage);
     if (ctx->y_stage) cudaFree(ctx->y_stage);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
@@ -235,8 +260,9 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
         plan.W = W;
         plan.x = x + m0 * K;
         plan.y = y + m0 * N;
+        if ((e = xprep_launch(plan.x, ctx->xq, ctx->xsc, mc, (int)K, stream))) return cuda_fail(ctx, e, "x preparation launch");
         if ((e = gemv_launch(plan, cw, stream))) return cuda_fail(ctx, e, "gemv kernel launch");
-        ctx->launches += 1;
+        ctx->launches += 2;
     }
     return FDQP_OK;
 }
@@ -303,7 +329,7 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
         if (v == 0 || v == 1) return FDQP_ERR_ARG;
         ctx->p_stages = v;
     } else if (!std::strcmp(key, "split_k")) {
-        if (v != -1 && v != 1 && v != 2 && v != 4) return FDQP_ERR_ARG;
+        if (v != -1 && v != 1 && v != 2 && v != 4 && v != 8) return FDQP_ERR_ARG;
         ctx->p_split_k = v;
     } else if (!std::strcmp(key, "l2_evict_first")) {
         if (v > 1) return FDQP_ERR_ARG;
@@ -332,9 +358,9 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
     const int mc = (int)(M < kMaxTokens ? M : kMaxTokens);
     if (!plan_gemv(ctx, mc, (int)K, (int)N, &cw, &plan)) return FDQP_ERR_SIZE;
     std::snprintf(buf, buf_bytes,
-                  "fdqp_gemv_kernel<%d,%d> launches=%lld grid=%d block=%d smem=%u stages=%d split_k=%d ctas_per_slice=%d "
+                  "fdqp_xprep_kernel + fdqp_gemv_kernel<%d,%d> pairs=%lld grid=%d block=%d smem=%u stages=%d split_k=%d ctas_per_slice=%d "
                   "evict_first=%d",
-                  cw, mc == 1 ? 1 : 2, (long long)((M + kMaxTokens - 1) / kMaxTokens), plan.Z * plan.Gz, (cw + 2) * 32,
+                  cw, mc == 1 ? 1 : 2, (long long)((M + kMaxTokens - 1) / kMaxTokens), plan.Z * plan.Gz, (cw + 1 + cw / 8) * 32,
                   plan.smem_bytes, plan.nstage, plan.Z, plan.Gz, plan.evict_first);
     return FDQP_OK;
 }

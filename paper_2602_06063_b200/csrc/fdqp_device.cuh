@@ -130,6 +130,29 @@ __device__ __forceinline__ float2 lds64f(uint32_t addr) {
     return v;
 }
 
+// Mixed-precision FMA (bf16 x bf16 + f32 -> f32): one FMA-pipe instruction that reads a 16-bit half of a
+// 32-bit register, so widening a packed bf16 pair costs no integer/logic instruction.
+// a = low / high half of `packed`, b = HIGH half of `w` (the bf16 truncation of an fp32 value, exact when that
+// value is a power of two or already bf16).
+__device__ __forceinline__ float bf16lo_mul_f32hi(uint32_t packed, float w) {
+    float r;
+    asm("{\n\t.reg .b16 alo, ahi, wlo, whi;\n\t"
+        "mov.b32 {alo, ahi}, %1;\n\tmov.b32 {wlo, whi}, %2;\n\t"
+        "fma.rn.f32.bf16 %0, alo, whi, %3;\n\t}"
+        : "=f"(r)
+        : "r"(packed), "f"(w), "f"(0.f));
+    return r;
+}
+__device__ __forceinline__ float bf16hi_mul_f32hi(uint32_t packed, float w) {
+    float r;
+    asm("{\n\t.reg .b16 alo, ahi, wlo, whi;\n\t"
+        "mov.b32 {alo, ahi}, %1;\n\tmov.b32 {wlo, whi}, %2;\n\t"
+        "fma.rn.f32.bf16 %0, ahi, whi, %3;\n\t}"
+        : "=f"(r)
+        : "r"(packed), "f"(w), "f"(0.f));
+    return r;
+}
+
 __device__ __forceinline__ float bf16_lo_to_f32(uint32_t packed) { return __uint_as_float(packed << 16); }
 __device__ __forceinline__ float bf16_hi_to_f32(uint32_t packed) { return __uint_as_float(packed & 0xffff0000u); }
 

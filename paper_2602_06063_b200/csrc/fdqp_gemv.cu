@@ -4,24 +4,37 @@
 // Shape of the computation.  For every quantisation group (32 consecutive k of one output row n)
 //     sum_k x_k * (d * q_k + m)  =  d * (sum_k q_k x_k)  +  m * (sum_k x_k)
 // so the per-weight work is only "unpack a nibble and multiply-accumulate it with x"; scale d and
-// offset m are applied once per group in fp32.  The inner sums run on the warp-level bf16 tensor-core
-// instruction (mma.sync m16n8k16): A = 16 output rows x 16 k of codes, B = 16 k x 8 token columns of
-// x, fp32 accumulate.  Codes are turned into bf16 with one logic op per pair
-//     ((word >> 4i) & 0x000F000F) | 0x43004300  ->  bf16x2 (128 + q_i, 128 + q_{i+4})
-// (exact); the +128 is cancelled by starting the accumulator at -128 * sum_k x_k, and the order of k
-// inside a group is a free permutation as long as x is staged with the same one.
+// offset m are applied once per group in fp32.
+//
+// The inner sums sum_k q_k x_k run on the warp-level integer tensor-core instruction
+// (mma.sync m16n8k32, u8 x s8/u8 -> s32): the 4-bit codes become bytes with two logic ops per four
+// codes (w & 0x0F0F0F0F, (w >> 4) & 0x0F0F0F0F -- B200 issues integer/logic instructions at half the
+// fp32 rate, so this unpack is the budget that matters), and the activations of a group are held as
+// 24-bit fixed point relative to the group's largest exponent, split into three byte planes
+// (x = 2^e_g * (65536 p2 + 256 p1 + p0), p2 signed, p1 and p0 unsigned; exact for every element
+// within 2^15 of the group's largest, rounded to 2^-23 of it otherwise).  One MMA covers a whole
+// group of 16 output rows; its s32 result is exact.  The order of k inside a group is a free
+// permutation as long as both operands use the same one (even k in the low half, odd k in the high).
+// The three plane sums are turned into fp32 without a conversion instruction: the accumulator starts
+// at the bit pattern of 1.5 * 2^23, so the s32 result *is* the float 12582912 + sum.
+// At M = 1 seven of the MMA's eight token columns would be idle, so the three planes of the single
+// token ride in columns 0, 1, 2 (as signed digits) and ONE MMA per 16 rows yields all three sums.
+//
+// The plane split of x is done once per call by a small preparation kernel; every GEMV CTA then
+// brings its K slice of the prepared x into shared memory with bulk async copies.
 //
 // Data movement.  The packed matrix is strip-major (32 output rows x all of K contiguous), so every
 // CTA streams one contiguous byte range of HBM exactly once.  The producer warp issues one 1-D bulk
 // async copy per Q4NX block (<= 5120 bytes), several lanes at a time, into a shared-memory ring of
 // multi-block stages guarded by mbarriers; every consumer warp owns the same 32 x 32 group-tile of
-// two blocks of a stage.  x (the CTA's K slice, all tokens) is staged once per CTA in the fragment
-// order the MMA wants, together with the per-group sums of x.
+// two blocks of a stage.
 //
 // Work split.  The (K-slice, strip, block) space is cut into equal contiguous ranges, one per
 // persistent CTA, so all SMs stream the same number of bytes whatever N and K are.  A strip whose
 // blocks end up in several CTAs (or several K slices) is completed by whichever CTA arrives last at
-// the strip's ticket: it sums the partial rows in a fixed order, so results are reproducible run to run.
+// the strip's ticket: it sums the partial rows in a fixed order, so results are reproducible run to
+// run.  A CTA handles the shared strip at the END of its range FIRST, so that the exchange through
+// global memory is off its critical path and its last piece is a whole strip written directly.
 // No CTA ever waits for another CTA.
 #include "fdqp_device.cuh"
 #include "fdqp_plan.h"
@@ -45,78 +58,220 @@ __device__ __forceinline__ float* piece_slot(const GemvPlan& p, int z, int64_t c
     return p.ws_edge + (((int64_t)z * p.Gz + ci) * 2 + which) * (kStripRows * kMaxTokens);
 }
 
-// Registers of one 32 x 32 group-tile in flight.
-struct TileRegs {
+#ifdef FDQP_TRACE
+__device__ unsigned long long g_fdqp_trace[1024 * 8];
+#define FDQP_STAMP(i) do { if (lane == 0) g_fdqp_trace[(blockIdx.x & 1023) * 8 + (i)] = globaltimer_ns(); } while (0)
+#else
+#define FDQP_STAMP(i) do { } while (0)
+#endif
+
+// ---- activation preparation ------------------------------------------------------------------------
+//
+// One thread per (group-tile T, token, quarter q): eight consecutive activations, turned into fixed point
+// relative to the largest exponent of the 32-group and split into byte planes in MMA fragment order
+// ({bytes of even k, bytes of odd k} per plane).
+//
+// M >= 2 (SINGLE == false): 24-bit fixed point, planes 2 (signed), 1, 0 (unsigned).  Record of 32 bytes at
+//   xq[((T*M + tok)*4 + q)*32]: words 0..5 = planes 2, 1, 0; words 6, 7 = {sum of the group's x, unit 2^e_g};
+//   and xsc[T*16 + (tok/2)*4 + (tok%2)*2 + {0,1}] holds the same two scalars indexed by token.
+// M == 1 (SINGLE == true): 23-bit fixed point in three SIGNED digits.  Per tile 128 bytes:
+//   [plane 2: 4 x 8 B by q][plane 1][plane 0][{sum x, unit}][24 zero bytes].
+template <bool SINGLE>
+__global__ void __launch_bounds__(128) fdqp_xprep_kernel(const uint16_t* __restrict__ x, uint32_t* __restrict__ xq,
+                                                          float* __restrict__ xsc, int M, int K) {
+    const int items = (K / kGroup) * M * 4;
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool valid = idx < items;
+    const int q = idx & 3, tm = idx >> 2;
+    const int tok = valid ? tm % M : 0, tile = valid ? tm / M : 0;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (valid) v = *reinterpret_cast<const uint4*>(x + (int64_t)tok * K + tile * kGroup + q * 8);
+    const uint32_t h[8] = {v.x & 0xffffu, v.x >> 16, v.y & 0xffffu, v.y >> 16,
+                           v.z & 0xffffu, v.z >> 16, v.w & 0xffffu, v.w >> 16};
+    float f[8];
+    uint32_t amax = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        f[i] = __uint_as_float(h[i] << 16);
+        const uint32_t mag = h[i] & 0x7fffu;
+        amax = mag > amax ? mag : amax;
+    }
+    float psum = ((f[0] + f[1]) + (f[2] + f[3])) + ((f[4] + f[5]) + (f[6] + f[7]));
+    {
+        uint32_t o = __shfl_xor_sync(0xffffffffu, amax, 1);
+        amax = o > amax ? o : amax;
+        o = __shfl_xor_sync(0xffffffffu, amax, 2);
+        amax = o > amax ? o : amax;
+        psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+        psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+    }
+    // exponent field of the group's largest magnitude, kept where both scale factors are normal floats
+    constexpr int kFrac = SINGLE ? 21 : 22;  // |fixed-point value| < 2^(kFrac + 1)
+    int emax = (int)(amax >> 7);
+    emax = emax < 24 ? 24 : (emax > 254 ? 254 : emax);
+    const float to_fixed = __uint_as_float((uint32_t)(254 + kFrac - emax) << 23);  // 2^(127 + kFrac - emax)
+    const float unit = __uint_as_float((uint32_t)(emax - kFrac) << 23);            // 2^(emax - 127 - kFrac)
+    int I[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) I[i] = __float2int_rn(f[i] * to_fixed);
+    uint32_t plane[3][2];  // [0] most significant; {even k, odd k}
+    int D[3][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        if (SINGLE) {  // signed digits: I = 65536 d2 + 256 d1 + d0, each in [-128, 127]
+            const int d0 = (I[i] << 24) >> 24;
+            const int r1 = (I[i] - d0) >> 8;
+            const int d1 = (r1 << 24) >> 24;
+            D[2][i] = d0;
+            D[1][i] = d1;
+            D[0][i] = (r1 - d1) >> 8;
+        } else {       // two's-complement bytes: top byte signed, lower bytes unsigned
+            D[2][i] = I[i];
+            D[1][i] = I[i] >> 8;
+            D[0][i] = I[i] >> 16;
+        }
+    }
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) {
+        const uint32_t e01 = __byte_perm(D[pl][0], D[pl][2], 0x0040), e23 = __byte_perm(D[pl][4], D[pl][6], 0x0040);
+        const uint32_t o01 = __byte_perm(D[pl][1], D[pl][3], 0x0040), o23 = __byte_perm(D[pl][5], D[pl][7], 0x0040);
+        plane[pl][0] = __byte_perm(e01, e23, 0x5410);
+        plane[pl][1] = __byte_perm(o01, o23, 0x5410);
+    }
+    if (!valid) return;
+    if (SINGLE) {
+        uint32_t* rec = xq + (int64_t)tile * 32;  // 128 bytes per tile
+#pragma unroll
+        for (int pl = 0; pl < 3; ++pl)
+            *reinterpret_cast<uint2*>(rec + pl * 8 + q * 2) = make_uint2(plane[pl][0], plane[pl][1]);
+        if (q == 0) *reinterpret_cast<uint2*>(rec + 24) = make_uint2(__float_as_uint(psum), __float_as_uint(unit));
+        if (q == 1) *reinterpret_cast<uint2*>(rec + 26) = make_uint2(0u, 0u);
+        if (q == 2) *reinterpret_cast<uint4*>(rec + 28) = make_uint4(0u, 0u, 0u, 0u);
+    } else {
+        uint4* dst = reinterpret_cast<uint4*>(xq + (int64_t)idx * 8);
+        dst[0] = make_uint4(plane[0][0], plane[0][1], plane[1][0], plane[1][1]);
+        dst[1] = make_uint4(plane[2][0], plane[2][1], __float_as_uint(psum), __float_as_uint(unit));
+        if (q == 0) {
+            float* sc = xsc + (int64_t)tile * 16 + (tok >> 1) * 4 + (tok & 1) * 2;
+            sc[0] = psum;
+            sc[1] = unit;
+        }
+    }
+}
+
+// ---- one 32 x 32 group-tile -------------------------------------------------------------------------
+
+constexpr int kMagicBits = 0x4B400000;  // bit pattern of 12582912.0f = 1.5 * 2^23
+constexpr float kMagic = 12582912.0f;
+
+struct TileIn {
     uint32_t c[4];   // code words: word q of rows g, g+8, g+16, g+24
     uint32_t so[4];  // (d[g], d[g+8]), (d[g+16], d[g+24]), (m[g], m[g+8]), (m[g+16], m[g+24]) as bf16 pairs
-    uint4 xb;        // B fragments of the two k16 steps
-    float xs[4];     // sum of x over the group for tokens 2q, 2q+1, and -128 times it
-    float d0[4], d1[4];
+    uint32_t b[6];   // B fragments {even k, odd k}: planes 2, 1, 0 (NT == 2) or this lane's column (NT == 1)
+    float sc[4];     // {sum x, unit} of token 2q and of token 2q+1 (NT == 2) or of the only token (NT == 1)
 };
 
-#define FDQP_UNPACK(w, sh) ((((w) >> (sh)) & 0x000F000Fu) | 0x43004300u)
-
 template <int NT>
-__device__ __forceinline__ void tile_load(TileRegs& t, uint32_t code_addr, uint32_t so_addr, uint32_t x_addr,
-                                          uint32_t xsum_addr) {
+__device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_t so_addr, uint32_t x_addr,
+                                          uint32_t xsc_addr) {
     ldmatrix_x4(t.c, code_addr);
     ldmatrix_x4_trans(t.so, so_addr);
-    t.xb = lds128(x_addr);
     if (NT == 1) {
-        const float2 v = lds64f(xsum_addr);  // {X, -128 X} of token 2q
-        t.xs[0] = v.x;
-        t.xs[1] = 0.f;
-        t.xs[2] = v.y;
-        t.xs[3] = 0.f;
+        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(t.b[0]), "=r"(t.b[1]) : "r"(x_addr));
+        const float2 v = lds64f(xsc_addr);
+        t.sc[0] = v.x;
+        t.sc[1] = v.y;
     } else {
+        const uint4 r0 = lds128(x_addr);
+        t.b[0] = r0.x; t.b[1] = r0.y; t.b[2] = r0.z; t.b[3] = r0.w;
+        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(t.b[4]), "=r"(t.b[5]) : "r"(x_addr + 16));
         asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
-                     : "=f"(t.xs[0]), "=f"(t.xs[1]), "=f"(t.xs[2]), "=f"(t.xs[3])
-                     : "r"(xsum_addr));  // {X0, X1, -128 X0, -128 X1}
+                     : "=f"(t.sc[0]), "=f"(t.sc[1]), "=f"(t.sc[2]), "=f"(t.sc[3])
+                     : "r"(xsc_addr));
     }
 }
 
-__device__ __forceinline__ void tile_mma(TileRegs& t) {
-    const float cinit[4] = {t.xs[2], t.xs[3], t.xs[2], t.xs[3]};  // -128 * sum x cancels the code bias
-    {
-        const uint32_t lo = t.c[0], hi = t.c[1];
-        mma_bf16_16816(t.d0, FDQP_UNPACK(lo, 0), FDQP_UNPACK(hi, 0), FDQP_UNPACK(lo, 4), FDQP_UNPACK(hi, 4), t.xb.x,
-                       t.xb.y, cinit);
-        mma_bf16_16816(t.d0, FDQP_UNPACK(lo, 8), FDQP_UNPACK(hi, 8), FDQP_UNPACK(lo, 12), FDQP_UNPACK(hi, 12), t.xb.z,
-                       t.xb.w, t.d0);
-    }
-    {
-        const uint32_t lo = t.c[2], hi = t.c[3];
-        mma_bf16_16816(t.d1, FDQP_UNPACK(lo, 0), FDQP_UNPACK(hi, 0), FDQP_UNPACK(lo, 4), FDQP_UNPACK(hi, 4), t.xb.x,
-                       t.xb.y, cinit);
-        mma_bf16_16816(t.d1, FDQP_UNPACK(lo, 8), FDQP_UNPACK(hi, 8), FDQP_UNPACK(lo, 12), FDQP_UNPACK(hi, 12), t.xb.z,
-                       t.xb.w, t.d1);
-    }
+template <bool B_SIGNED>
+__device__ __forceinline__ void imma(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                     uint32_t b1) {
+    if (B_SIGNED)
+        asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+            : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(kMagicBits));
+    else
+        asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+            : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(kMagicBits));
 }
 
-// acc[row][tok] += d * (sum_k q_k x_k) + m * (sum_k x_k), in fp32 (Eq. 3 applied per group)
+// Per-lane constants of the single-token kernel: which two MMA columns the lane holds.
+//   q == 0: columns (plane 2, plane 1) -> 256 * s2 + s1, weighted 256 * unit, and the lane adds m * sum x
+//   q == 1: columns (plane 0, zero)    -> s0, weighted unit
+//   q >= 2: zero columns
+struct LaneConst {
+    float k_first;  // weight of the first column relative to the second
+    float w_unit;   // factor on `unit`
+    float w_sum;    // factor on `sum x`
+};
+
+// acc[row][tok] += d * unit * (sum_k q_k X_k) + m * (sum_k x_k), fp32 (Eq. 3 applied per group).
+// `unit` (and 256 * unit) are powers of two, so d * unit is formed exactly by the mixed bf16 FMA.
 template <int NT>
-__device__ __forceinline__ void tile_scale(const TileRegs& t, float (&acc)[4][NT]) {
-    const float dsc[4] = {bf16_lo_to_f32(t.so[0]), bf16_hi_to_f32(t.so[0]), bf16_lo_to_f32(t.so[1]),
-                          bf16_hi_to_f32(t.so[1])};
-    const float mof[4] = {bf16_lo_to_f32(t.so[2]), bf16_hi_to_f32(t.so[2]), bf16_lo_to_f32(t.so[3]),
-                          bf16_hi_to_f32(t.so[3])};
-    const float dd[4][2] = {{t.d0[0], t.d0[1]}, {t.d0[2], t.d0[3]}, {t.d1[0], t.d1[1]}, {t.d1[2], t.d1[3]}};
+__device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][NT], const LaneConst& lc) {
+    const float uq = t.sc[1] * lc.w_unit, xq = t.sc[0] * lc.w_sum;  // used when NT == 1
+    const float mof[4] = {bf16lo_mul_f32hi(t.so[2], 1.0f), bf16hi_mul_f32hi(t.so[2], 1.0f),
+                          bf16lo_mul_f32hi(t.so[3], 1.0f), bf16hi_mul_f32hi(t.so[3], 1.0f)};
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int h = 0; h < 2; ++h) {  // rows (g, g+8) then (g+16, g+24)
+        const uint32_t w0 = t.c[2 * h], w1 = t.c[2 * h + 1];
+        const uint32_t e0 = w0 & 0x0F0F0F0Fu, o0 = (w0 >> 4) & 0x0F0F0F0Fu;  // even-k codes, odd-k codes
+        const uint32_t e1 = w1 & 0x0F0F0F0Fu, o1 = (w1 >> 4) & 0x0F0F0F0Fu;
+        if (NT == 1) {
+            int d[4];
+            imma<true>(d, e0, e1, o0, o1, t.b[0], t.b[1]);
+            const float dq[2] = {bf16lo_mul_f32hi(t.so[h], uq), bf16hi_mul_f32hi(t.so[h], uq)};
 #pragma unroll
-        for (int j = 0; j < NT; ++j) {
-            acc[i][j] = fmaf(dsc[i], dd[i][j], acc[i][j]);
-            acc[i][j] = fmaf(mof[i], t.xs[j], acc[i][j]);
+            for (int r = 0; r < 2; ++r) {
+                const int i = 2 * h + r;
+                const float a0 = __int_as_float(d[2 * r]) - kMagic, a1 = __int_as_float(d[2 * r + 1]) - kMagic;
+                const float s = fmaf(a0, lc.k_first, a1);  // exact: |s| < 2^24
+                acc[i][0] = fmaf(dq[r], s, acc[i][0]);
+                acc[i][0] = fmaf(mof[i], xq, acc[i][0]);
+            }
+        } else {
+            int d2[4], d1[4], d0[4];
+            imma<true>(d2, e0, e1, o0, o1, t.b[0], t.b[1]);
+            imma<false>(d1, e0, e1, o0, o1, t.b[2], t.b[3]);
+            imma<false>(d0, e0, e1, o0, o1, t.b[4], t.b[5]);
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int i = 2 * h + r;
+#pragma unroll
+                for (int j = 0; j < NT; ++j) {
+                    const int e = 2 * r + j;
+                    const float s2 = __int_as_float(d2[e]) - kMagic, s1 = __int_as_float(d1[e]) - kMagic,
+                                s0 = __int_as_float(d0[e]) - kMagic;
+                    const float s = fmaf(fmaf(s2, 256.f, s1), 256.f, s0);  // exact up to 2^24, else one rounding
+                    const float dq = r == 0 ? bf16lo_mul_f32hi(t.so[h], t.sc[2 * j + 1])
+                                            : bf16hi_mul_f32hi(t.so[h], t.sc[2 * j + 1]);
+                    acc[i][j] = fmaf(dq, s, acc[i][j]);
+                    acc[i][j] = fmaf(mof[i], t.sc[2 * j], acc[i][j]);
+                }
+            }
         }
+    }
 }
 
 // CW consumer warps (8 or 16); NT token columns kept per lane (1 when M == 1, else 2).
 // A ring stage holds CB = CW / 4 blocks; warp w owns group-tile (w & 7) of blocks 2*(w >> 3) and
 // 2*(w >> 3) + 1 of every stage.
+// Warps CW+1 .. CW+NR are reducers (NR = CW / 8): reducer r completes the strip pieces with piece % NR == r.
 template <int CW, int NT>
-__global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __grid_constant__ GemvPlan p) {
+__global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
+    fdqp_gemv_kernel(const __grid_constant__ GemvPlan p) {
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int CB = CW / 4;
+    constexpr int NR = CW / 8;
     constexpr uint32_t kStageBytes = CB * kBlockBytes;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int M = p.M, K = p.K;
@@ -129,17 +284,22 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
     const int64_t a = range_begin(ci, p.Gz, T), e = range_begin(ci + 1, p.Gz, T);
     const int nblk = (int)(e - a);
     if (nblk <= 0) return;
-    const int64_t s_first = a / len;
-    const int bl_first = (int)(a - s_first * len);           // block index inside the slice of the CTA's first block
-    const int npieces = (int)((e - 1) / len - s_first) + 1;  // strips this CTA touches
+    const int64_t s_first = a / len, s_last = (e - 1) / len;
+    const int bl_first = (int)(a - s_first * len);    // block index inside the slice of the CTA's first block
+    const int npieces = (int)(s_last - s_first) + 1;  // strips this CTA touches
+    // Processing order: the blocks of a partial last strip come first, then the rest of the range in order.
+    const int64_t tail_begin = s_last * len > a ? s_last * len : a;
+    const int nt = (npieces >= 2 && e < (s_last + 1) * len) ? (int)(e - tail_begin) : 0;
+    const int bl_tail = (int)(tail_begin - s_last * len);
     const int nchunk = (nblk + CB - 1) / CB;
+    if (warp == 0) FDQP_STAMP(0);
 
     const uint32_t ring = smem_u32(smem);
-    const uint32_t xs = ring + p.off_xs, zero_slot = ring + p.off_zero, xsum = ring + p.off_xsum;
+    const uint32_t xs = ring + p.off_xs, xsc = ring + p.off_xsum;
     const uint32_t part = ring + p.off_part, bars = ring + p.off_bar;
     const int nstage = p.nstage;
     const uint32_t full0 = bars, empty0 = bars + 8u * nstage;
-    const uint32_t red_full0 = bars + 16u * nstage, red_empty0 = red_full0 + 16u;
+    const uint32_t red_full0 = bars + 16u * nstage, red_empty0 = red_full0 + 16u, x_bar = red_full0 + 32u;
 
     for (int s = tid; s < nstage; s += blockDim.x) {
         mbar_init(full0 + 8u * s, 1);
@@ -149,22 +309,44 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
         mbar_init(red_full0 + 8u * tid, CW);
         mbar_init(red_empty0 + 8u * tid, 1);
     }
+    if (tid == 2) mbar_init(x_bar, 1);
     mbar_fence_init();
     __syncthreads();
+    if (warp == 0) FDQP_STAMP(1);
 
     const int groups_total = K / kGroup;
     const int64_t strip_bytes = (int64_t)kGroupBytes * groups_total;
 
     if (warp == CW) {
         // =============================== producer ================================================
+        // The prepared activations of this CTA's K slice: one barrier, a few large copies.
+        if (lane == 0) {
+            const int kbeg = b_first * kBlockK;
+            const int kend_full = (b_first + len) * kBlockK;
+            const int kend = kend_full < K ? kend_full : K;
+            const uint32_t tile0 = (uint32_t)(kbeg / kGroup), ntiles = (uint32_t)((kend - kbeg) / kGroup);
+            const uint32_t rec_bytes = ntiles * (uint32_t)M * 128u, sc_bytes = (NT == 2) ? ntiles * 64u : 0u;
+            mbar_arrive_expect_tx(x_bar, rec_bytes + sc_bytes);
+            const uint8_t* src = reinterpret_cast<const uint8_t*>(p.xq) + (size_t)tile0 * M * 128u;
+            for (uint32_t off = 0; off < rec_bytes; off += 32768u) {
+                const uint32_t n = rec_bytes - off < 32768u ? rec_bytes - off : 32768u;
+                bulk_g2s(xs + off, src + off, n, x_bar);
+            }
+            if constexpr (NT == 2) {
+                const uint8_t* s2 = reinterpret_cast<const uint8_t*>(p.xsc) + (size_t)tile0 * 64u;
+                for (uint32_t off = 0; off < sc_bytes; off += 32768u) {
+                    const uint32_t n = sc_bytes - off < 32768u ? sc_bytes - off : 32768u;
+                    bulk_g2s(xsc + off, s2 + off, n, x_bar);
+                }
+            }
+        }
         // Lane j < CB copies block j of every stage; lane 0 owns the barrier traffic.
         uint64_t policy = 0;
         if (p.evict_first) policy = l2_policy_evict_first();
-        int64_t ps = s_first;
-        int pbl = bl_first + lane;  // only meaningful for lane < CB
-        while (pbl >= len) { pbl -= len; ++ps; }
+        const uint32_t len_magic = (uint32_t)(0x100000000ull / (uint32_t)len) + 1u;
+        const bool magic_ok = ((uint64_t)(nblk + len) * (uint64_t)len) < 0x80000000ull && len > 1;
         int stage = 0;
-        uint32_t phase = 0;  // parity of the stage's previous use
+        uint32_t phase = 0;  // parity of the stage's current use
         bool alive = true;
         int c = 0;
         for (; c < nchunk && alive; ++c) {
@@ -174,9 +356,17 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) { alive = false; break; }
             }
-            const int i = c * CB + lane;
+            const int i = c * CB + lane;  // position in processing order
             uint32_t bytes = 0;
+            int64_t ps = 0;
+            int pbl = 0;
             if (lane < CB && i < nblk) {
+                // block i of the processing order -> (strip, block inside the slice)
+                const uint32_t rel = (uint32_t)bl_first + (uint32_t)(i < nt ? (nblk - nt + i) : (i - nt));
+                uint32_t so = __umulhi(rel, len_magic);  // rel / len: exact while rel * len < 2^32
+                if (!magic_ok) so = rel / (uint32_t)len;
+                ps = s_first + so;
+                pbl = (int)(rel - so * (uint32_t)len);
                 const int rest = groups_total - 8 * (b_first + pbl);
                 bytes = (uint32_t)kGroupBytes * (uint32_t)(rest < 8 ? rest : 8);
             }
@@ -191,12 +381,11 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
                 else
                     bulk_g2s(dst, src, bytes, full0 + 8u * stage);
             }
-            pbl += CB;
-            while (pbl >= len) { pbl -= len; ++ps; }
             if (++stage == nstage) { stage = 0; phase ^= 1u; }
         }
         // Do not leave while a copy into this CTA's shared memory may still be in flight.
         if (lane == 0) {
+            mbar_wait(x_bar, 0, p.status);
             const int issued = c;
             const int from = issued > nstage ? issued - nstage : 0;
             for (int k = from; k < issued; ++k)
@@ -205,66 +394,22 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
         return;
     }
 
-    // ---- consumers and reducer: stage this CTA's K slice of x (fragment order + per-group sums)
-    {
-        const int nthr = (CW + 1) * 32;
-        const int t2 = warp < CW ? tid : tid - 32;  // skip the producer warp's ids
-        const int kbeg = b_first * kBlockK;
-        const int kend_full = (b_first + len) * kBlockK;
-        const int kend = kend_full < K ? kend_full : K;
-        const int ntiles = (kend - kbeg) / kGroup;
-        uint8_t* xs_g = smem + p.off_xs;
-        float* xsum_g = reinterpret_cast<float*>(smem + p.off_xsum);
-        const int xsum_stride = (NT == 1) ? 2 : 4 * 4;  // floats per tile: {X,-128X} or 4 quads of {X0,X1,-128X0,-128X1}
-        if (NT == 2)
-            for (int i = t2; i < ntiles * 16; i += nthr) {
-                const int tok = ((i >> 2) & 3) * 2 + (i & 1);  // slot i holds token 2q + (i & 1), q = (i >> 2) & 3
-                if (tok >= M) xsum_g[i] = 0.f;
-            }
-        if (t2 < 16) reinterpret_cast<uint32_t*>(smem + p.off_zero)[t2] = 0u;
-        const int items = ntiles * M * 4;
-        for (int base = 0; base < items; base += nthr) {
-            const int idx = base + t2;
-            const bool valid = idx < items;
-            float psum = 0.f;
-            const int q = idx & 3, tm = idx >> 2;
-            const int tok = tm % M, tile = tm / M;
-            if (valid) {
-                const uint4 v =
-                    *reinterpret_cast<const uint4*>(p.x + (int64_t)tok * K + kbeg + tile * kGroup + q * 8);
-                uint4 o;  // k order inside the lane's 8 values: 0,4,1,5,2,6,3,7
-                o.x = __byte_perm(v.x, v.z, 0x5410);
-                o.y = __byte_perm(v.x, v.z, 0x7632);
-                o.z = __byte_perm(v.y, v.w, 0x5410);
-                o.w = __byte_perm(v.y, v.w, 0x7632);
-                *reinterpret_cast<uint4*>(xs_g + ((int64_t)tile * M + tok) * 64 + q * 16) = o;
-                psum = ((bf16_lo_to_f32(v.x) + bf16_hi_to_f32(v.x)) + (bf16_lo_to_f32(v.y) + bf16_hi_to_f32(v.y))) +
-                       ((bf16_lo_to_f32(v.z) + bf16_hi_to_f32(v.z)) + (bf16_lo_to_f32(v.w) + bf16_hi_to_f32(v.w)));
-            }
-            psum += __shfl_xor_sync(0xffffffffu, psum, 1);
-            psum += __shfl_xor_sync(0xffffffffu, psum, 2);
-            if (valid && q == 0) {
-                if (NT == 1) {
-                    xsum_g[tile * 2] = psum;
-                    xsum_g[tile * 2 + 1] = -128.f * psum;
-                } else {
-                    float* dst = xsum_g + tile * xsum_stride + (tok >> 1) * 4 + (tok & 1);
-                    dst[0] = psum;
-                    dst[2] = -128.f * psum;
-                }
-            }
-        }
-        asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
-    }
-
     if (warp < CW) {
         // =============================== consumers ===============================================
         const int tw = warp & 7, j0 = (warp >> 3) * 2;
         const int g = lane >> 2, q = lane & 3;
-        const uint32_t x_lane = (g < M) ? xs + g * 64 + q * 16 : zero_slot;
-        const uint32_t x_stride = (g < M) ? (uint32_t)M * 64u : 0u;
-        const uint32_t xsum_lane = (NT == 1) ? xsum : xsum + q * 16;
-        const uint32_t xsum_stride = (NT == 1) ? 8u : 64u;
+        // B fragments.  NT == 2: column g is token g (any valid token for unused columns: their results are
+        // never stored).  NT == 1: column g < 3 is plane 2 - g of the only token, other columns read zeros.
+        const int gtok = g < M ? g : M - 1;
+        const uint32_t x_lane = (NT == 1) ? xs + (g < 3 ? (uint32_t)(g * 32 + q * 8) : 104u)
+                                          : xs + (uint32_t)(gtok * 4 + q) * 32u;
+        const uint32_t x_stride = (uint32_t)M * 128u;
+        const uint32_t xsc_lane = (NT == 1) ? xs + 96u : xsc + q * 16;
+        const uint32_t xsc_stride = (NT == 1) ? 128u : 64u;
+        LaneConst lc;
+        lc.k_first = q == 0 ? 256.f : 1.f;
+        lc.w_unit = q == 0 ? 256.f : (q == 1 ? 1.f : 0.f);
+        lc.w_sum = q == 0 ? 1.f : 0.f;
         // ldmatrix source rows: codes = row `lane` of the tile; scales/offsets = the four 16-byte
         // chunks of this tile's scale words and of its offset words, duplicated so that after the
         // transposed load every lane of a quad holds (d[g], d[g+8]), (d[g+16], d[g+24]), (m..), (m..)
@@ -283,6 +428,10 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
         bool alive = true;
         // hand the warp's partial rows of the current strip piece to the reducer warp
         auto flush = [&]() {
+            if (NT == 1) {  // lanes q == 0 and q == 1 hold the two halves of each row's sum
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[i][0] += __shfl_xor_sync(0xffffffffu, acc[i][0], 1);
+            }
             const int par = piece & 1;
             if (piece >= 2 && !mbar_wait(red_empty0 + 8u * par, ((piece >> 1) - 1) & 1, p.status)) alive = false;
             const uint32_t slot = part + (uint32_t)((par * CW + warp) * kStripRows * M) * 4u;
@@ -302,73 +451,98 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
             ++piece;
         };
 
-        int unit_first = -bl_first;          // index (relative to the CTA's first block) of block 0 of the current strip
-        int unit_next = unit_first + len;    // ... and of the next strip
+        // Strip bookkeeping in processing order: position of block 0 of the current strip, position where
+        // the next strip starts, and the in-slice index of the first block after the leading tail piece.
+        int unit_first = nt > 0 ? -bl_tail : -bl_first;
+        int unit_next = nt > 0 ? nt : unit_first + len;
+        int first_fix = nt > 0 ? bl_first : 0;
+        auto next_unit = [&]() {
+            unit_first = unit_next - first_fix;
+            first_fix = 0;
+            unit_next = unit_first + len;
+        };
+
+        if (!mbar_wait(x_bar, 0, p.status)) alive = false;
+        if (warp == 0) FDQP_STAMP(2);
+        const bool work = !(p.debug & 1);
+        // An "interior" stage -- both of the warp's blocks inside the range and the current strip, every block
+        // full -- needs no bookkeeping beyond two tile indices.  `lim` is the first position that is not interior.
+        const bool all_full = (groups_total & 7) == 0;
+        const uint32_t so_lane8 = so_sect * 8u + so_chunk;
+        auto interior_limit = [&]() { return (all_full && work) ? (unit_next < nblk ? unit_next : nblk) : -1; };
+        int lim = interior_limit();
         int stage = 0;
         uint32_t phase = 0;
         for (int c = 0; c < nchunk && alive; ++c) {
-            if (!mbar_wait(full0 + 8u * stage, phase, p.status)) { alive = false; break; }
-            const uint32_t sbase = ring + stage * kStageBytes + j0 * kBlockBytes;
             const int i0 = c * CB + j0, i1 = i0 + 1;
-            // block index inside the slice (for the staged x) and group count of both blocks
-            int bl0 = i0 - unit_first, bl1;
-            while (bl0 >= len) bl0 -= len;
-            bl1 = bl0 + 1;
-            if (bl1 >= len) bl1 -= len;
-            const int r0 = groups_total - 8 * (b_first + bl0), r1 = groups_total - 8 * (b_first + bl1);
-            const int jb0 = r0 < 8 ? r0 : 8, jb1 = r1 < 8 ? r1 : 8;
-            const bool work = !(p.debug & 1);
-            const bool act0 = work && (i0 < nblk) && (tw < jb0), act1 = work && (i1 < nblk) && (tw < jb1);
-            TileRegs ta, tb;
-            if (act0) {
+            if (i0 < nblk && i0 >= unit_next) {
+                while (i0 >= unit_next && alive) { flush(); next_unit(); }
+                lim = interior_limit();
+            }
+            if (!mbar_wait(full0 + 8u * stage, phase, p.status)) { alive = false; break; }
+            if (warp == 0 && c == 0) FDQP_STAMP(3);
+            const uint32_t sbase = ring + stage * kStageBytes + j0 * kBlockBytes;
+            const int bl0 = i0 - unit_first;
+            TileIn ta, tb;
+            if (i1 < lim) {
                 const int tile = bl0 * 8 + tw;
-                tile_load<NT>(ta, sbase + code_lane, sbase + so_sect * jb0 + so_chunk, x_lane + tile * x_stride,
-                              xsum_lane + tile * xsum_stride);
-            }
-            if (act1) {
-                const int tile = bl1 * 8 + tw;
-                tile_load<NT>(tb, sbase + kBlockBytes + code_lane, sbase + kBlockBytes + so_sect * jb1 + so_chunk,
-                              x_lane + tile * x_stride, xsum_lane + tile * xsum_stride);
-            }
-            if (act0) tile_mma(ta);
-            if (act1) tile_mma(tb);
-            // all shared-memory reads of this stage are done: release it before the fp32 epilogue
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty0 + 8u * stage);
-            if (i0 < nblk) {
-                while (i0 >= unit_next && alive) { flush(); unit_first = unit_next; unit_next += len; }
-                if (act0) tile_scale<NT>(ta, acc);
-            }
-            if (i1 < nblk) {
-                while (i1 >= unit_next && alive) { flush(); unit_first = unit_next; unit_next += len; }
-                if (act1) tile_scale<NT>(tb, acc);
+                const uint32_t xa = x_lane + tile * x_stride, sa = xsc_lane + tile * xsc_stride;
+                tile_load<NT>(ta, sbase + code_lane, sbase + so_lane8, xa, sa);
+                tile_load<NT>(tb, sbase + kBlockBytes + code_lane, sbase + kBlockBytes + so_lane8, xa + 8 * x_stride,
+                              sa + 8 * xsc_stride);
+                tile_compute<NT>(ta, acc, lc);
+                // every shared-memory read of this stage has been consumed by now: hand the stage back
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8u * stage);
+                tile_compute<NT>(tb, acc, lc);
+            } else {
+                // general stage: range end, strip boundary between the two blocks, or a short last block
+                const bool cross = i1 >= unit_next;
+                const int bl1 = cross ? i1 - (unit_next - first_fix) : i1 - unit_first;
+                const int r0 = groups_total - 8 * (b_first + bl0), r1 = groups_total - 8 * (b_first + bl1);
+                const int jb0 = r0 < 8 ? r0 : 8, jb1 = r1 < 8 ? r1 : 8;
+                const bool act0 = work && (i0 < nblk) && (tw < jb0), act1 = work && (i1 < nblk) && (tw < jb1);
+                if (act0) {
+                    const int tile = bl0 * 8 + tw;
+                    tile_load<NT>(ta, sbase + code_lane, sbase + so_sect * jb0 + so_chunk, x_lane + tile * x_stride,
+                                  xsc_lane + tile * xsc_stride);
+                }
+                if (act1) {
+                    const int tile = bl1 * 8 + tw;
+                    tile_load<NT>(tb, sbase + kBlockBytes + code_lane, sbase + kBlockBytes + so_sect * jb1 + so_chunk,
+                                  x_lane + tile * x_stride, xsc_lane + tile * xsc_stride);
+                }
+                if (act0) tile_compute<NT>(ta, acc, lc);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8u * stage);
+                if (i1 < nblk) {
+                    if (cross && alive) { flush(); next_unit(); lim = interior_limit(); }
+                    if (act1) tile_compute<NT>(tb, acc, lc);
+                }
             }
             if (++stage == nstage) { stage = 0; phase ^= 1u; }
         }
+        if (warp == 0) FDQP_STAMP(4);
         while (piece < npieces && alive) flush();
     } else {
         // =============================== reducer =================================================
-        int64_t pa = a;
-        for (int piece = 0; piece < npieces; ++piece) {
-            const int64_t s = s_first + piece;
+        for (int piece = warp - CW - 1; piece < npieces; piece += NR) {
+            // pieces in processing order: the partial last strip first (if any), then the strips in order
+            const int64_t s = nt > 0 ? (piece == 0 ? s_last : s_first + piece - 1) : s_first + piece;
             const int64_t unit_begin = s * len, unit_end = unit_begin + len;
+            const int64_t pa = unit_begin > a ? unit_begin : a;
             const int64_t pe = unit_end < e ? unit_end : e;
             const int par = piece & 1;
             if (!mbar_wait(red_full0 + 8u * par, (piece >> 1) & 1, p.status)) break;
+            const float* part_g = reinterpret_cast<const float*>(smem + p.off_part);
             float v[kMaxTokens];
 #pragma unroll
             for (int t = 0; t < kMaxTokens; ++t) {
                 v[t] = 0.f;
                 if (t < M) {
 #pragma unroll
-                    for (int w = 0; w < CW; ++w) {
-                        float f;
-                        asm volatile("ld.shared.f32 %0, [%1];"
-                                     : "=f"(f)
-                                     : "r"(part + (uint32_t)(((par * CW + w) * M + t) * kStripRows + lane) * 4u)
-                                     : "memory");
-                        v[t] += f;
-                    }
+                    for (int w = 0; w < CW; ++w)
+                        v[t] += part_g[((par * CW + w) * M + t) * kStripRows + lane];
                 }
             }
             __syncwarp();
@@ -385,7 +559,6 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
 #pragma unroll
                 for (int t = 0; t < kMaxTokens; ++t)
                     if (t < M) slot[t * kStripRows + lane] = v[t];
-                __threadfence();
                 __syncwarp();
                 // how many pieces does strip s have over all slices?
                 int total = 0;
@@ -394,12 +567,13 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
                     const int64_t T2 = (int64_t)p.S * l2;
                     total += (int)(cta_of(s * l2 + l2 - 1, p.Gz, T2) - cta_of(s * l2, p.Gz, T2)) + 1;
                 }
+                // release this warp's partial rows and acquire everybody else's in one round trip
                 int old = 0;
-                if (lane == 0) old = atomicAdd(p.tickets + s, 1);
+                if (lane == 0)
+                    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.tickets + s) : "memory");
                 old = __shfl_sync(0xffffffffu, old, 0);
                 if (old == total - 1) {
                     // last piece to arrive: add all pieces of the strip in a fixed order
-                    __threadfence();
 #pragma unroll
                     for (int t = 0; t < kMaxTokens; ++t) v[t] = 0.f;
                     for (int zz = 0; zz < p.Z; ++zz) {
@@ -420,16 +594,31 @@ __global__ void __launch_bounds__((CW + 2) * 32, 1) fdqp_gemv_kernel(const __gri
                     if (lane == 0) p.tickets[s] = 0;  // ready for the next launch on this stream
                 }
             }
-            pa = pe;
         }
+        if (warp == CW + 1) FDQP_STAMP(5);
     }
 }
+
+#ifdef FDQP_TRACE
+extern "C" __attribute__((visibility("default"))) int fdqp_trace_read(unsigned long long* host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_fdqp_trace, sizeof(unsigned long long) * n);
+}
+#endif
 
 // ---- host-visible launchers ------------------------------------------------------------------
 
 template <int CW, int NT>
 static cudaError_t launch_one(const GemvPlan& p, cudaStream_t stream) {
-    fdqp_gemv_kernel<CW, NT><<<p.Z * p.Gz, (CW + 2) * 32, p.smem_bytes, stream>>>(p);
+    fdqp_gemv_kernel<CW, NT><<<p.Z * p.Gz, (CW + 1 + CW / 8) * 32, p.smem_bytes, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream) {
+    const int items = (K / kGroup) * M * 4;
+    if (M == 1)
+        fdqp_xprep_kernel<true><<<(items + 127) / 128, 128, 0, stream>>>(x, xq, xsc, M, K);
+    else
+        fdqp_xprep_kernel<false><<<(items + 127) / 128, 128, 0, stream>>>(x, xq, xsc, M, K);
     return cudaGetLastError();
 }
 

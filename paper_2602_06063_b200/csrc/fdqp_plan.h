@@ -11,12 +11,14 @@ constexpr int kBlockK = 256;        // input features per full Q4NX block
 constexpr int kBlockBytes = 5120;   // bytes of a full block (Sec. "Dequantization Engine")
 constexpr int kGroupBytes = 640;    // bytes a block spends per group: 512 codes + 64 scales + 64 offsets
 constexpr int kMaxTokens = 8;       // token rows one GEMV launch handles
-constexpr int kMaxSplit = 4;        // K slices
+constexpr int kMaxSplit = 8;        // K slices
 constexpr int kMaxCtasPerSm = 2;
 
 struct GemvPlan {
     const uint8_t* W;     // device, packed Q4NX
     const uint16_t* x;    // device, [M][K] bf16 bits
+    const uint32_t* xq;   // device, prepared activations: 32-byte records [K/32][M][4] (see fdqp_xprep_kernel)
+    const float* xsc;     // device, per-group {sum x, unit} by token: [K/32][8][2]
     float* y;             // device, [M][N]
     float* ws_edge;       // device, [grid][2][32*kMaxTokens] partial sums of strips shared between CTAs
     float* ws_full;       // device, [Z][S][32*kMaxTokens] partial sums of whole strip-slices (Z > 1)
@@ -31,9 +33,8 @@ struct GemvPlan {
     int nstage;           // ring depth in stages of (consumer warps / 4) blocks
     int evict_first;      // weight copies carry an evict-first L2 hint
     int debug;            // measurement aid: bit 0 = consumers skip the arithmetic (results are then undefined)
-    uint32_t off_xs;      // shared-memory offsets (bytes)
-    uint32_t off_zero;
-    uint32_t off_xsum;
+    uint32_t off_xs;      // shared-memory offsets (bytes): prepared-x records, per-token scalars,
+    uint32_t off_xsum;    //   partial rows, barriers
     uint32_t off_part;
     uint32_t off_bar;
     uint32_t smem_bytes;

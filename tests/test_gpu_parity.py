@@ -143,10 +143,8 @@ def test_zero_and_offsets_only(fresh):
     K, N, M = 1152, 64, 4
     case = Case(K, N, M, seed=66)
     zero = synthgen.Q4NXWeights(np.zeros_like(case.w.codes), case.w.scales, np.zeros_like(case.w.offsets))
-    # codes 0 and offsets 0 with non-zero scales: every w_hat is 0, the bound collapses to its absolute term
-    assert np.all(np.abs(Case(K, N, M, 0, weights=zero, x=case.x).run(fresh)) <= ABS_TOL)
-    dead = synthgen.Q4NXWeights(zero.codes, np.zeros_like(case.w.scales), zero.offsets)
-    assert np.all(Case(K, N, M, 0, weights=dead, x=case.x).run(fresh) == 0)
+    # codes 0 and offsets 0 (scales left non-zero): every w_hat is 0 and so is every output, exactly
+    assert np.all(Case(K, N, M, 0, weights=zero, x=case.x).run(fresh) == 0)
     off = synthgen.Q4NXWeights(np.zeros_like(case.w.codes), case.w.scales, case.w.offsets)
     c = Case(K, N, M, 0, weights=off, x=case.x)
     y_ref, a_ref = c.reference()
@@ -176,7 +174,7 @@ def test_batched_rows_match_single_row_calls(fresh):
         assert np.all(np.abs(y1[0] - y[m]) <= 2 * (REL_TOL * a_ref[m] + ABS_TOL))
 
 
-@pytest.mark.parametrize("key,values", [("split_k", [1, 2, 4]), ("consumer_warps", [8, 16]), ("ctas_per_sm", [1, 2]),
+@pytest.mark.parametrize("key,values", [("split_k", [1, 2, 4, 8]), ("consumer_warps", [8, 16]), ("ctas_per_sm", [1, 2]),
                                         ("stages", [2, 3, 7]), ("l2_evict_first", [0, 1])])
 def test_launch_parameters_do_not_change_results(fresh, key, values):
     K, N, M = 4352, 2080, 3   # 17 blocks per strip, 65 strips: ragged against every split and grid
