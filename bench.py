@@ -2,9 +2,11 @@
 """Benchmark of the FusedDQP hot path on B200.
 
 A step is one Gemma3-4B decoder layer at M = 1: the seven Q4NX projections q, k, v, o, gate, up, down
-(59.1 MB of packed weights) on seeded synthetic inputs.  Several distinct copies of the layer's weights are
-resident in HBM and the steps rotate through them, so every timed step streams its weights from HBM and not
-from L2.  The metric is the achieved bandwidth over the algorithmic bytes of the step
+(59.1 MB of packed weights) on seeded synthetic inputs.  Projections that share their input are launched
+together -- q|k|v and gate|up are concatenated along N, which in the strip-major Q4NX container is plain
+concatenation of the packed bytes -- so a step is four fdqp_run calls (--fuse 0 runs the seven one by one).
+Several distinct copies of the layer's weights are resident in HBM and the steps rotate through them, so every
+timed step streams its weights from HBM and not from L2.  The metric is the achieved bandwidth over the algorithmic bytes of the step
 (0.625*K*N + 2*M*K + 4*M*N per projection); decode tokens/s (projections only: 34 layers + LM head) is
 reported beside it.
 
@@ -165,8 +167,13 @@ def run_ours(args, rank, local_rank, world):
 
     peaks, peak_kind = measured_peaks()
     M = 1
-    shapes = synthgen.GEMMA3_4B_LAYER
+    layer_shapes = synthgen.GEMMA3_4B_LAYER
+    # launch groups: projections sharing their input run as one call on weights concatenated along N
+    groups = [["q", "k", "v"], ["o"], ["gate", "up"], ["down"]] if args.fuse else [[n] for n, _, _, _ in layer_shapes]
+    by_name = {n: (K, N, seed) for n, K, N, seed in layer_shapes}
+    shapes = [("|".join(g), by_name[g[0]][0], sum(by_name[n][1] for n in g), by_name[g[0]][2]) for g in groups]
     max_K = max(K for _, K, _, _ in shapes)
+    step_bytes_layer = layer_bytes(M)
     _, hk, hn, hseed = synthgen.GEMMA3_4B_LM_HEAD
     ctx = fd.fdqp_create(local_rank, 8, max(max_K, hk), max(max(N for _, _, N, _ in shapes), hn))
     if args.param:
@@ -179,13 +186,16 @@ def run_ours(args, rank, local_rank, world):
     host_layer0 = None
     for c in range(LAYER_COPIES):
         layer = []
-        for name, K, N, seed in shapes:
-            w = synthgen.weights(seed + 1000 * c, K, N)
-            packed = fd.q4nx_pack(w.codes, w.scales, w.offsets)
-            layer.append(torch.from_numpy(packed).cuda())
-            if c == 0:
-                host_layer0 = host_layer0 or []
-                host_layer0.append(w)
+        for g in groups:
+            parts = []
+            for name in g:
+                K, N, seed = by_name[name]
+                w = synthgen.weights(seed + 1000 * c, K, N)
+                parts.append(fd.q4nx_pack(w.codes, w.scales, w.offsets))
+                if c == 0:
+                    host_layer0 = host_layer0 or []
+                    host_layer0.append((w, synthgen.activations(by_name[g[0]][2], M, K)))
+            layer.append(torch.from_numpy(np.concatenate(parts)).cuda())
         copies.append(layer)
     xs_host = [synthgen.activations(seed, M, K) for _, K, _, seed in shapes]
     xs = [torch.from_numpy(x.view(np.int16)).cuda() for x in xs_host]
@@ -197,8 +207,11 @@ def run_ours(args, rank, local_rank, world):
         for i, (_, K, N, _) in enumerate(shapes):
             fd.fdqp_run(ctx, xs[i], copies[c][i], ys[i], M, K, N, sraw)
 
-    # one CUDA graph per weight copy: the seven launches of a step replay without per-launch host cost
+    # CUDA graphs: a decode step of the real model is 34 such layers back to back, so the layers are captured
+    # LAYER_COPIES at a time (one pass over all resident weight copies per graph); single-layer graphs cover the
+    # remainder when the step count is not a multiple of LAYER_COPIES.
     graphs = None
+    pass_graph = None
     if args.graph:
         graphs = []
         with torch.cuda.stream(stream):
@@ -209,17 +222,35 @@ def run_ours(args, rank, local_rank, world):
             with torch.cuda.graph(g, stream=stream):
                 enqueue_layer(c)
             graphs.append(g)
+        pass_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(pass_graph, stream=stream):
+            for c in range(LAYER_COPIES):
+                enqueue_layer(c)
+
+    def run_steps(first, count):
+        """Enqueue `count` consecutive steps starting at step index `first`."""
+        i = first
+        end = first + count
+        while i < end:
+            c = i % LAYER_COPIES
+            if pass_graph is not None and c == 0 and end - i >= LAYER_COPIES:
+                with torch.cuda.stream(stream):
+                    pass_graph.replay()
+                i += LAYER_COPIES
+            elif graphs is not None:
+                with torch.cuda.stream(stream):
+                    graphs[c].replay()
+                i += 1
+            else:
+                enqueue_layer(c)
+                i += 1
 
     def step(i):
-        c = i % LAYER_COPIES
-        if graphs is not None:
-            with torch.cuda.stream(stream):
-                graphs[c].replay()
-        else:
-            enqueue_layer(c)
+        run_steps(i, 1)
 
-    for i in range(args.warmup):
-        step(i)
+    run_steps(0, args.warmup)
+    first_timed = -(-args.warmup // LAYER_COPIES) * LAYER_COPIES   # start the timed region on a pass boundary
+    run_steps(args.warmup, first_timed - args.warmup)
     stream.synchronize()
 
     sampler = ClockSampler(local_rank)
@@ -230,13 +261,13 @@ def run_ours(args, rank, local_rank, world):
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     ev0.record(stream)
-    for i in range(args.steps):
-        step(args.warmup + i)
+    run_steps(first_timed, args.steps)
     ev1.record(stream)
     stream.synchronize()
     barrier()
     ms = ev0.elapsed_time(ev1)
-    kernels_per_step = len(shapes)
+    calls_per_step = len(shapes)
+    kernels_per_step = 2 * calls_per_step        # each call = activation preparation kernel + GEMV kernel
     launches = kernels_per_step * args.steps
     if graphs is None:
         assert fd.fdqp_launch_count(ctx) - launches_before == launches
@@ -297,7 +328,7 @@ def run_ours(args, rank, local_rank, world):
         t0 = time.perf_counter()
         passes = 0
         while passes < 1 or (time.perf_counter() - t0 < 10 and passes < 50):
-            for w, x in zip(host_layer0, xs_host):
+            for w, x in host_layer0:
                 oracle.project(x, w.codes, w.scales, w.offsets, nthreads=cores)
             passes += 1
         dt = time.perf_counter() - t0
@@ -305,16 +336,17 @@ def run_ours(args, rank, local_rank, world):
                "sample": f"{passes} pass(es) of the whole layer (7 projections, all outputs), {dt:.1f} s"}
 
     if rank == 0:
-        step_bytes = layer_bytes(M)
+        step_bytes = step_bytes_layer
         gbs = step_bytes * args.steps * world / (ms * 1e-3) / 1e9
-        per_launch_us = ms * 1e3 / launches
-        achieved = (step_bytes / kernels_per_step) / (per_launch_us * 1e-6) / 1e9
+        per_launch_us = ms * 1e3 / (calls_per_step * args.steps)   # one GEMV launch incl. its preparation kernel
+        achieved = (step_bytes / calls_per_step) / (per_launch_us * 1e-6) / 1e9
         layer_ms = ms / args.steps
         line = {
             "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": layer_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": {"workload": WORKLOAD, "M": M, "bytes_per_step": step_bytes, "cuda_graph": bool(graphs),
+            "config": {"workload": WORKLOAD, "M": M, "bytes_per_step": step_bytes, "cuda_graph": (f"{LAYER_COPIES} steps per graph" if graphs else False),
+                       "calls_per_step": [name for name, _, _, _ in shapes],
                        "l2": f"inputs larger than L2: steps rotate over {LAYER_COPIES} distinct weight sets "
                              f"({LAYER_COPIES * step_bytes / 1e6:.0f} MB)",
                        "multi_gpu": "independent replicas, no collective",
@@ -346,6 +378,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--graph", type=int, default=1, help="replay each step from a CUDA graph (default 1)")
+    ap.add_argument("--fuse", type=int, default=1, help="run q|k|v and gate|up as one call each (default 1)")
     ap.add_argument("--param", action="append", help="library launch parameter key=value (repeatable)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-head", action="store_true", help="skip the LM-head timing")

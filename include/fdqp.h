@@ -169,6 +169,8 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "stages"        shared-memory ring depth in stages (a stage holds consumer_warps / 4 Q4NX blocks)
  *   "split_k"       number of K slices (1, 2, 4 or 8)
  *   "l2_evict_first" 1 = weight copies carry an evict-first L2 hint
+ *   "strip_aligned" 1 = CTA work ranges are cut at strip boundaries, 0 = equal block counts per CTA
+ *   "prep_inline"   1 = every GEMV CTA prepares its slice of x itself, 0 = a preparation kernel runs first
  *   "debug"         measurement aid: 1 = the GEMV consumers skip the arithmetic (y is then undefined)
  * Unknown key or unusable value: FDQP_ERR_ARG.  Meant for benchmarks and tests. */
 FDQP_API fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t value);

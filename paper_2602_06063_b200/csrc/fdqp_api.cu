@@ -38,12 +38,13 @@ struct fdqp_ctx {
     int64_t launches = 0;
     std::string last_err;
     // overrides (-1 = automatic)
-    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1;
+    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1, p_prep = -1, p_aligned = -1;
 };
 
 namespace {
 
 constexpr int kMaxStages = 40;
+constexpr double kTwoCtaBytes = 48e6;
 constexpr int kMinStages = 3;  // ring depth below which another K slice is preferred
 
 struct DeviceGuard {
@@ -102,8 +103,11 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     p->N = N;
     p->S = N / kStripRows;
     p->nb = (K + kBlockK - 1) / kBlockK;
-    // measured on B200: two 8-warp CTAs per SM stream fastest at M = 1; larger M wants the smem of one CTA
-    int ctas_per_sm = ctx->p_ctas_per_sm > 0 ? (int)ctx->p_ctas_per_sm : (M == 1 && ctx->p_cw != 16 ? 2 : 1);
+    // measured on B200: two 8-warp CTAs per SM stream fastest at M = 1 once the matrix is large; small matrices and
+    // larger M do better with one 16-warp CTA (one start-up per SM, all of its shared memory)
+    const double packed_bytes = 0.625 * (double)K * (double)N;
+    int ctas_per_sm = ctx->p_ctas_per_sm > 0 ? (int)ctx->p_ctas_per_sm
+                                             : (M == 1 && ctx->p_cw != 16 && packed_bytes >= kTwoCtaBytes ? 2 : 1);
     if (ctas_per_sm > kMaxCtasPerSm) ctas_per_sm = kMaxCtasPerSm;
     int cw = 16, Z = 1, nbz = p->nb;
     SmemLayout L{};
@@ -129,6 +133,20 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     if (grid > total_blocks) grid = (int)total_blocks;
     int Gz = grid / Z;
     if (Gz < 1) Gz = 1;
+    // Equal block counts per CTA keep every SM streaming, but a strip shared by two CTAs is finished through
+    // global memory (~2 us on the critical path unless the CTA also owns whole strips to do afterwards).  Cutting at
+    // strip boundaries avoids that at the price of imbalance.  Estimate both (us) and take the cheaper.
+    {
+        const double t_block = 0.125 * ctas_per_sm;  // one 5 KB block at an SM's share of HBM bandwidth
+        const int64_t blocks_bal = (total_blocks / Z + Gz - 1) / Gz;
+        const double cost_bal = blocks_bal * t_block + (blocks_bal >= 2 * (int64_t)nbz ? 0.6 : 2.0);
+        const int Ga = Gz < p->S ? Gz : p->S;
+        const int64_t blocks_al = (int64_t)((p->S + Ga - 1) / Ga) * nbz;
+        const double cost_al = blocks_al * t_block + (Z > 1 ? 2.0 : 0.4);
+        const bool aligned = ctx->p_aligned >= 0 ? ctx->p_aligned != 0 : cost_al < cost_bal;
+        p->strip_aligned = aligned ? 1 : 0;
+        if (aligned) Gz = Ga;
+    }
     p->Gz = Gz;
     int nstage = L.nstage;
     if (ctx->p_stages > 0 && ctx->p_stages < nstage) nstage = (int)ctx->p_stages;
@@ -140,6 +158,8 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     p->smem_bytes = p->off_bar + (2u * (uint32_t)nstage + 5u) * 8u;
     p->evict_first = ctx->p_evict >= 0 ? (ctx->p_evict != 0) : 1;
     p->debug = ctx->p_debug > 0 ? (int)ctx->p_debug : 0;
+    // work items (8 activations each) per CTA if x is prepared in-kernel; beyond this a preparation kernel is cheaper
+    p->prep_inline = ctx->p_prep >= 0 ? (int)(ctx->p_prep != 0) : ((int64_t)nbz * 8 * M * 4 <= (int64_t)cw * 32);
     p->ws_edge = ctx->ws_edge;
     p->ws_full = ctx->ws_full;
     p->tickets = ctx->tickets;
@@ -260,9 +280,13 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
         plan.W = W;
         plan.x = x + m0 * K;
         plan.y = y + m0 * N;
-        if ((e = xprep_launch(plan.x, ctx->xq, ctx->xsc, mc, (int)K, stream))) return cuda_fail(ctx, e, "x preparation launch");
+        if (!plan.prep_inline) {
+            if ((e = xprep_launch(plan.x, ctx->xq, ctx->xsc, mc, (int)K, stream)))
+                return cuda_fail(ctx, e, "x preparation launch");
+            ctx->launches += 1;
+        }
         if ((e = gemv_launch(plan, cw, stream))) return cuda_fail(ctx, e, "gemv kernel launch");
-        ctx->launches += 2;
+        ctx->launches += 1;
     }
     return FDQP_OK;
 }
@@ -336,6 +360,12 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
         ctx->p_evict = v;
     } else if (!std::strcmp(key, "debug")) {
         ctx->p_debug = v;
+    } else if (!std::strcmp(key, "strip_aligned")) {
+        if (v > 1) return FDQP_ERR_ARG;
+        ctx->p_aligned = v;
+    } else if (!std::strcmp(key, "prep_inline")) {
+        if (v > 1) return FDQP_ERR_ARG;
+        ctx->p_prep = v;
     } else {
         return FDQP_ERR_ARG;
     }
@@ -358,9 +388,9 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
     const int mc = (int)(M < kMaxTokens ? M : kMaxTokens);
     if (!plan_gemv(ctx, mc, (int)K, (int)N, &cw, &plan)) return FDQP_ERR_SIZE;
     std::snprintf(buf, buf_bytes,
-                  "fdqp_xprep_kernel + fdqp_gemv_kernel<%d,%d> pairs=%lld grid=%d block=%d smem=%u stages=%d split_k=%d ctas_per_slice=%d "
-                  "evict_first=%d",
-                  cw, mc == 1 ? 1 : 2, (long long)((M + kMaxTokens - 1) / kMaxTokens), plan.Z * plan.Gz, (cw + 1 + cw / 8) * 32,
-                  plan.smem_bytes, plan.nstage, plan.Z, plan.Gz, plan.evict_first);
+                  "%sfdqp_gemv_kernel<%d,%d> calls=%lld grid=%d block=%d smem=%u stages=%d split_k=%d ctas_per_slice=%d "
+                  "evict_first=%d strip_aligned=%d",
+                  plan.prep_inline ? "" : "fdqp_xprep_kernel + ", cw, mc == 1 ? 1 : 2, (long long)((M + kMaxTokens - 1) / kMaxTokens), plan.Z * plan.Gz, (cw + 1 + cw / 8) * 32,
+                  plan.smem_bytes, plan.nstage, plan.Z, plan.Gz, plan.evict_first, plan.strip_aligned);
     return FDQP_OK;
 }

@@ -76,16 +76,17 @@ __device__ unsigned long long g_fdqp_trace[1024 * 8];
 //   and xsc[T*16 + (tok/2)*4 + (tok%2)*2 + {0,1}] holds the same two scalars indexed by token.
 // M == 1 (SINGLE == true): 23-bit fixed point in three SIGNED digits.  Per tile 128 bytes:
 //   [plane 2: 4 x 8 B by q][plane 1][plane 0][{sum x, unit}][24 zero bytes].
-template <bool SINGLE>
-__global__ void __launch_bounds__(128) fdqp_xprep_kernel(const uint16_t* __restrict__ x, uint32_t* __restrict__ xq,
-                                                          float* __restrict__ xsc, int M, int K) {
-    const int items = (K / kGroup) * M * 4;
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    const bool valid = idx < items;
-    const int q = idx & 3, tm = idx >> 2;
-    const int tok = valid ? tm % M : 0, tile = valid ? tm / M : 0;
+// `tile` is the group-tile index in x, `slot` the tile's index in the destination (global: the same; shared
+// memory: relative to the CTA's K slice).  Must be called by whole quads (the four q of a (tile, token)).
+__device__ __forceinline__ uint4 xprep_load(const uint16_t* __restrict__ x, int K, int tile, int tok, int q, bool valid) {
     uint4 v = make_uint4(0, 0, 0, 0);
     if (valid) v = *reinterpret_cast<const uint4*>(x + (int64_t)tok * K + tile * kGroup + q * 8);
+    return v;
+}
+
+template <bool SINGLE>
+__device__ __forceinline__ void xprep_item(const uint4 v, int M, int slot, int tok, int q, bool valid,
+                                           uint32_t* __restrict__ xq, float* __restrict__ xsc) {
     const uint32_t h[8] = {v.x & 0xffffu, v.x >> 16, v.y & 0xffffu, v.y >> 16,
                            v.z & 0xffffu, v.z >> 16, v.w & 0xffffu, v.w >> 16};
     float f[8];
@@ -140,7 +141,7 @@ __global__ void __launch_bounds__(128) fdqp_xprep_kernel(const uint16_t* __restr
     }
     if (!valid) return;
     if (SINGLE) {
-        uint32_t* rec = xq + (int64_t)tile * 32;  // 128 bytes per tile
+        uint32_t* rec = xq + (int64_t)slot * 32;  // 128 bytes per tile
 #pragma unroll
         for (int pl = 0; pl < 3; ++pl)
             *reinterpret_cast<uint2*>(rec + pl * 8 + q * 2) = make_uint2(plane[pl][0], plane[pl][1]);
@@ -148,15 +149,31 @@ __global__ void __launch_bounds__(128) fdqp_xprep_kernel(const uint16_t* __restr
         if (q == 1) *reinterpret_cast<uint2*>(rec + 26) = make_uint2(0u, 0u);
         if (q == 2) *reinterpret_cast<uint4*>(rec + 28) = make_uint4(0u, 0u, 0u, 0u);
     } else {
-        uint4* dst = reinterpret_cast<uint4*>(xq + (int64_t)idx * 8);
+        uint4* dst = reinterpret_cast<uint4*>(xq + ((int64_t)(slot * M + tok) * 4 + q) * 8);
         dst[0] = make_uint4(plane[0][0], plane[0][1], plane[1][0], plane[1][1]);
         dst[1] = make_uint4(plane[2][0], plane[2][1], __float_as_uint(psum), __float_as_uint(unit));
         if (q == 0) {
-            float* sc = xsc + (int64_t)tile * 16 + (tok >> 1) * 4 + (tok & 1) * 2;
+            float* sc = xsc + (int64_t)slot * 16 + (tok >> 1) * 4 + (tok & 1) * 2;
             sc[0] = psum;
             sc[1] = unit;
         }
     }
+}
+
+// Stand-alone preparation of a whole x, for calls whose K slice is too large to prepare inside every GEMV CTA.
+template <bool SINGLE>
+__global__ void __launch_bounds__(128) fdqp_xprep_kernel(const uint16_t* __restrict__ x, uint32_t* __restrict__ xq,
+                                                          float* __restrict__ xsc, int M, int K) {
+    // The GEMV kernel that follows is launched with programmatic stream serialisation: it may start now and
+    // stream weights; it waits (griddepcontrol.wait) before touching what this kernel writes.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // x may be the previous launch's output
+    const int items = (K / kGroup) * M * 4;
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool valid = idx < items;
+    const int q = idx & 3, tm = idx >> 2;
+    const int tok = valid ? tm % M : 0, tile = valid ? tm / M : 0;
+    xprep_item<SINGLE>(xprep_load(x, K, tile, tok, q, valid), M, tile, tok, q, valid, xq, xsc);
 }
 
 // ---- one 32 x 32 group-tile -------------------------------------------------------------------------
@@ -281,7 +298,9 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
     const int b_first = z * p.nbz;
     const int len = slice_len(p, z);
     const int64_t T = (int64_t)p.S * len;
-    const int64_t a = range_begin(ci, p.Gz, T), e = range_begin(ci + 1, p.Gz, T);
+    // contiguous range of the slice's blocks: equal block counts, or whole strips when the plan asks for that
+    const int64_t a = p.strip_aligned ? range_begin(ci, p.Gz, p.S) * len : range_begin(ci, p.Gz, T);
+    const int64_t e = p.strip_aligned ? range_begin(ci + 1, p.Gz, p.S) * len : range_begin(ci + 1, p.Gz, T);
     const int nblk = (int)(e - a);
     if (nblk <= 0) return;
     const int64_t s_first = a / len, s_last = (e - 1) / len;
@@ -313,33 +332,15 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
     mbar_fence_init();
     __syncthreads();
     if (warp == 0) FDQP_STAMP(1);
+    // The next launch in the stream may begin as soon as SM slots free up: it streams weights (which nothing in this
+    // library writes) and waits for this grid to complete before it touches activations, outputs or workspace.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const int groups_total = K / kGroup;
     const int64_t strip_bytes = (int64_t)kGroupBytes * groups_total;
 
     if (warp == CW) {
         // =============================== producer ================================================
-        // The prepared activations of this CTA's K slice: one barrier, a few large copies.
-        if (lane == 0) {
-            const int kbeg = b_first * kBlockK;
-            const int kend_full = (b_first + len) * kBlockK;
-            const int kend = kend_full < K ? kend_full : K;
-            const uint32_t tile0 = (uint32_t)(kbeg / kGroup), ntiles = (uint32_t)((kend - kbeg) / kGroup);
-            const uint32_t rec_bytes = ntiles * (uint32_t)M * 128u, sc_bytes = (NT == 2) ? ntiles * 64u : 0u;
-            mbar_arrive_expect_tx(x_bar, rec_bytes + sc_bytes);
-            const uint8_t* src = reinterpret_cast<const uint8_t*>(p.xq) + (size_t)tile0 * M * 128u;
-            for (uint32_t off = 0; off < rec_bytes; off += 32768u) {
-                const uint32_t n = rec_bytes - off < 32768u ? rec_bytes - off : 32768u;
-                bulk_g2s(xs + off, src + off, n, x_bar);
-            }
-            if constexpr (NT == 2) {
-                const uint8_t* s2 = reinterpret_cast<const uint8_t*>(p.xsc) + (size_t)tile0 * 64u;
-                for (uint32_t off = 0; off < sc_bytes; off += 32768u) {
-                    const uint32_t n = sc_bytes - off < 32768u ? sc_bytes - off : 32768u;
-                    bulk_g2s(xsc + off, s2 + off, n, x_bar);
-                }
-            }
-        }
         // Lane j < CB copies block j of every stage; lane 0 owns the barrier traffic.
         uint64_t policy = 0;
         if (p.evict_first) policy = l2_policy_evict_first();
@@ -385,7 +386,7 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         }
         // Do not leave while a copy into this CTA's shared memory may still be in flight.
         if (lane == 0) {
-            mbar_wait(x_bar, 0, p.status);
+            if (!p.prep_inline) mbar_wait(x_bar, 0, p.status);
             const int issued = c;
             const int from = issued > nstage ? issued - nstage : 0;
             for (int k = from; k < issued; ++k)
@@ -462,7 +463,41 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             unit_next = unit_first + len;
         };
 
-        if (!mbar_wait(x_bar, 0, p.status)) alive = false;
+        // Everything up to here touched only this CTA's shared memory.  x may come from the previous launch.
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (p.prep_inline) {
+            // prepare this CTA's K slice of x straight into shared memory (cheap, and the first weights are still
+            // on their way from HBM)
+            const int kbeg = b_first * kBlockK;
+            const int kend_full = (b_first + len) * kBlockK;
+            const int tile0 = kbeg / kGroup, ntiles = ((kend_full < K ? kend_full : K) - kbeg) / kGroup;
+            const int items = ntiles * M * 4;
+            uint32_t* xs_g = reinterpret_cast<uint32_t*>(smem + p.off_xs);
+            float* xsc_g = reinterpret_cast<float*>(smem + p.off_xsum);
+            constexpr int kBatch = 8;  // loads in flight per thread: one trip to L2 / HBM for typical decode shapes
+            for (int base = 0; base < items; base += kBatch * CW * 32) {
+                uint4 v[kBatch];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int idx = base + u * CW * 32 + tid;
+                    const bool valid = idx < items;
+                    const int tm = idx >> 2;
+                    v[u] = xprep_load(p.x, K, tile0 + (valid ? tm / M : 0), valid ? tm % M : 0, idx & 3, valid);
+                }
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int idx = base + u * CW * 32 + tid;
+                    if (base + u * CW * 32 < items) {  // warp-uniform: whole quads run the shuffles together
+                        const bool valid = idx < items;
+                        const int tm = idx >> 2;
+                        xprep_item<NT == 1>(v[u], M, valid ? tm / M : 0, valid ? tm % M : 0, idx & 3, valid, xs_g, xsc_g);
+                    }
+                }
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(CW * 32) : "memory");
+        } else if (!mbar_wait(x_bar, 0, p.status)) {
+            alive = false;
+        }
         if (warp == 0) FDQP_STAMP(2);
         const bool work = !(p.debug & 1);
         // An "interior" stage -- both of the warp's blocks inside the range and the current strip, every block
@@ -526,6 +561,29 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         while (piece < npieces && alive) flush();
     } else {
         // =============================== reducer =================================================
+        // The prepared activations of this CTA's K slice: one barrier, a few large copies.  They are written by
+        // the preparation kernel this launch may overlap with, hence the dependency wait first.
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // before any global write of this grid
+        if (warp == CW + 1 && lane == 0 && !p.prep_inline) {
+            const int kbeg = b_first * kBlockK;
+            const int kend_full = (b_first + len) * kBlockK;
+            const int kend = kend_full < K ? kend_full : K;
+            const uint32_t tile0 = (uint32_t)(kbeg / kGroup), ntiles = (uint32_t)((kend - kbeg) / kGroup);
+            const uint32_t rec_bytes = ntiles * (uint32_t)M * 128u, sc_bytes = (NT == 2) ? ntiles * 64u : 0u;
+            mbar_arrive_expect_tx(x_bar, rec_bytes + sc_bytes);
+            const uint8_t* src = reinterpret_cast<const uint8_t*>(p.xq) + (size_t)tile0 * M * 128u;
+            for (uint32_t off = 0; off < rec_bytes; off += 32768u) {
+                const uint32_t n = rec_bytes - off < 32768u ? rec_bytes - off : 32768u;
+                bulk_g2s(xs + off, src + off, n, x_bar);
+            }
+            if constexpr (NT == 2) {
+                const uint8_t* s2 = reinterpret_cast<const uint8_t*>(p.xsc) + (size_t)tile0 * 64u;
+                for (uint32_t off = 0; off < sc_bytes; off += 32768u) {
+                    const uint32_t n = sc_bytes - off < 32768u ? sc_bytes - off : 32768u;
+                    bulk_g2s(xsc + off, s2 + off, n, x_bar);
+                }
+            }
+        }
         for (int piece = warp - CW - 1; piece < npieces; piece += NR) {
             // pieces in processing order: the partial last strip first (if any), then the strips in order
             const int64_t s = nt > 0 ? (piece == 0 ? s_last : s_first + piece - 1) : s_first + piece;
@@ -561,11 +619,14 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                     if (t < M) slot[t * kStripRows + lane] = v[t];
                 __syncwarp();
                 // how many pieces does strip s have over all slices?
-                int total = 0;
-                for (int zz = 0; zz < p.Z; ++zz) {
-                    const int l2 = slice_len(p, zz);
-                    const int64_t T2 = (int64_t)p.S * l2;
-                    total += (int)(cta_of(s * l2 + l2 - 1, p.Gz, T2) - cta_of(s * l2, p.Gz, T2)) + 1;
+                int total = p.Z;  // strip-aligned ranges: one whole piece per slice
+                if (!p.strip_aligned) {
+                    total = 0;
+                    for (int zz = 0; zz < p.Z; ++zz) {
+                        const int l2 = slice_len(p, zz);
+                        const int64_t T2 = (int64_t)p.S * l2;
+                        total += (int)(cta_of(s * l2 + l2 - 1, p.Gz, T2) - cta_of(s * l2, p.Gz, T2)) + 1;
+                    }
                 }
                 // release this warp's partial rows and acquire everybody else's in one round trip
                 int old = 0;
@@ -580,7 +641,8 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                         const int l2 = slice_len(p, zz);
                         const int64_t T2 = (int64_t)p.S * l2;
                         const int64_t u0 = s * l2;
-                        const int64_t cf = cta_of(u0, p.Gz, T2), cl = cta_of(u0 + l2 - 1, p.Gz, T2);
+                        const int64_t cf = p.strip_aligned ? 0 : cta_of(u0, p.Gz, T2);
+                        const int64_t cl = p.strip_aligned ? 0 : cta_of(u0 + l2 - 1, p.Gz, T2);
                         for (int64_t c2 = cf; c2 <= cl; ++c2) {
                             const float* src = piece_slot(p, zz, c2, s, u0, cf == cl, range_begin(c2, p.Gz, T2));
 #pragma unroll
@@ -609,17 +671,32 @@ extern "C" __attribute__((visibility("default"))) int fdqp_trace_read(unsigned l
 
 template <int CW, int NT>
 static cudaError_t launch_one(const GemvPlan& p, cudaStream_t stream) {
-    fdqp_gemv_kernel<CW, NT><<<p.Z * p.Gz, (CW + 1 + CW / 8) * 32, p.smem_bytes, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.Z * p.Gz));
+    cfg.blockDim = dim3((unsigned)((CW + 1 + CW / 8) * 32));
+    cfg.dynamicSmemBytes = p.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may overlap the preparation kernel before it
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<CW, NT>, p);
 }
 
 cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream) {
     const int items = (K / kGroup) * M * 4;
-    if (M == 1)
-        fdqp_xprep_kernel<true><<<(items + 127) / 128, 128, 0, stream>>>(x, xq, xsc, M, K);
-    else
-        fdqp_xprep_kernel<false><<<(items + 127) / 128, 128, 0, stream>>>(x, xq, xsc, M, K);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((items + 127) / 128));
+    cfg.blockDim = dim3(128);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return M == 1 ? cudaLaunchKernelEx(&cfg, fdqp_xprep_kernel<true>, x, xq, xsc, M, K)
+                  : cudaLaunchKernelEx(&cfg, fdqp_xprep_kernel<false>, x, xq, xsc, M, K);
 }
 
 cudaError_t gemv_launch(const GemvPlan& p, int consumer_warps, cudaStream_t stream) {
