@@ -139,6 +139,26 @@ FDQP_API fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W_q
 FDQP_API fdqp_status fdqp_run_host(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,
                           int64_t M, int64_t K, int64_t N, void* cuda_stream);
 
+/* The same projection for callers that must not allocate device memory at the time of the call -- a server that
+ * gave all device memory to its own pool at start-up, a real-time loop that cannot take the device-wide
+ * synchronisation an allocation may bring, a plug-in that may not allocate after initialisation.  (The paper has no
+ * counterpart: this is a packaging of fdqp_run's GEMV kernel, not another operation.)
+ *   x_bf16, W_q4nx, y   device pointers, 16-byte aligned, as for fdqp_run; runs on the CURRENT device
+ *   limits              M <= 8; N <= 262144; and the prepared activations must fit shared memory without
+ *                       splitting K (about M*K <= 32768, e.g. K <= 3840 at M = 8); beyond them FDQP_ERR_SIZE
+ * It takes no context and calls no cudaMalloc / cudaFree or any other allocating routine.  Its scratch -- the
+ * partial-row slots of strips shared between CTAs, their arrival counters, a status word -- is a 688,384-byte
+ * array inside the library image, resident on every device that loads the library until the process exits.
+ * The first call on a device looks up the device's limits and the array's device address; make that first call
+ * before any stream capture.  Every call clears the arrival counters it is going to use (a cudaMemsetAsync on
+ * the stream) and then launches the kernel; the rest of the array keeps the previous call's contents.
+ * All calls on a device share the one array: calls whose kernels could overlap on the GPU (different streams,
+ * no dependency between them) race and give wrong results -- keep them on one stream or order them.
+ * Asynchronous on `cuda_stream`.  Errors (nothing is launched): FDQP_ERR_ARG, FDQP_ERR_SHAPE, FDQP_ERR_ALIGN,
+ * FDQP_ERR_SIZE, FDQP_ERR_ARCH, FDQP_ERR_CUDA. */
+FDQP_API fdqp_status fdqp_run_noalloc(const void* x_bf16, const void* W_q4nx, float* y, int64_t M, int64_t K,
+                                      int64_t N, void* cuda_stream);
+
 /* ---- the dequantisation engine (Sec. "Dequantization Engine", Eq. 3) ------- */
 
 /* Write the dequantised matrix w_hat[k][n] to `out` (device, [K][N] row-major,

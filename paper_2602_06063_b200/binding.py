@@ -24,7 +24,7 @@ STATUS = {
 EXPORTS = [
     "q4nx_packed_bytes", "q4nx_pack", "q4nx_unpack", "fdqp_create", "fdqp_destroy", "fdqp_run", "fdqp_run_host",
     "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
-    "fdqp_launch_count", "fdqp_describe",
+    "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc",
 ]
 
 
@@ -63,6 +63,8 @@ def load_library():
     lib.fdqp_run.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_run_host.restype = ci
     lib.fdqp_run_host.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.fdqp_run_noalloc.restype = ci
+    lib.fdqp_run_noalloc.argtypes = [vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_dequant.restype = ci
     lib.fdqp_dequant.argtypes = [vp, vp, vp, ci, i64, i64, vp]
     lib.fdqp_last_status.restype = ci
@@ -169,6 +171,13 @@ def fdqp_run_host(ctx: int, x_host_bf16, W_q4nx, y_host, M: int, K: int, N: int,
     """x, y: HOST buffers (numpy or pinned torch); W: device.  Returns after y_host is filled."""
     _check(load_library().fdqp_run_host(ctx, _addr(x_host_bf16), _addr(W_q4nx), _addr(y_host), M, K, N,
                                         _stream(stream)), "fdqp_run_host", ctx)
+
+
+def fdqp_run_noalloc(x_bf16, W_q4nx, y, M: int, K: int, N: int, stream=None) -> None:
+    """fdqp_run for callers that cannot allocate: no context, scratch lives in the library image (see fdqp.h).
+    Runs on the current device; all calls share one scratch array, so keep them ordered on a stream."""
+    _check(load_library().fdqp_run_noalloc(_addr(x_bf16), _addr(W_q4nx), _addr(y), M, K, N, _stream(stream)),
+           "fdqp_run_noalloc")
 
 
 def fdqp_dequant(ctx: int, W_q4nx, out, out_is_bf16: bool, K: int, N: int, stream=None) -> None:

@@ -5,6 +5,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 
@@ -392,5 +393,97 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
                   "evict_first=%d strip_aligned=%d",
                   plan.prep_inline ? "" : "fdqp_xprep_kernel + ", cw, mc == 1 ? 1 : 2, (long long)((M + kMaxTokens - 1) / kMaxTokens), plan.Z * plan.Gz, (cw + 1 + cw / 8) * 32,
                   plan.smem_bytes, plan.nstage, plan.Z, plan.Gz, plan.evict_first, plan.strip_aligned);
+    return FDQP_OK;
+}
+
+// ---- projection without any allocation -------------------------------------------------------------------------
+//
+// fdqp_run_noalloc serves callers that must not allocate device memory when they run a projection: a server that
+// handed all device memory to its own pool at start-up, a real-time loop that cannot afford the device-wide
+// synchronisation an allocation may imply, a plug-in that is forbidden to allocate after initialisation.  It is the
+// streaming GEMV kernel with its scratch -- the partial-row slots of strips shared between CTAs, the strips' arrival
+// counters and the status word -- in a fixed array that is part of the loaded library image.
+
+namespace {
+
+constexpr int kNoAllocMaxCtas = 320;                  // partial-row slots: two per persistent CTA
+constexpr int64_t kNoAllocMaxN = 262144;              // arrival counters: one per 32-row strip
+constexpr size_t kNoAllocEdgeBytes = (size_t)kNoAllocMaxCtas * 2 * kStripRows * kMaxTokens * sizeof(float);
+constexpr size_t kNoAllocTicketBytes = (size_t)(kNoAllocMaxN / kStripRows) * sizeof(int);
+constexpr size_t kNoAllocScratchBytes = kNoAllocEdgeBytes + kNoAllocTicketBytes + 256;  // + status word
+
+struct NoAllocDevice {
+    bool ready = false;
+    unsigned char* scratch = nullptr;  // device address of g_noalloc_scratch on this device
+    int sm_count = 0;
+    int smem_optin = 0;
+};
+
+constexpr int kNoAllocMaxDevices = 64;
+NoAllocDevice g_noalloc_devices[kNoAllocMaxDevices];
+std::mutex g_noalloc_mutex;
+
+}  // namespace
+
+// 688,384 bytes, held by every device that loads the library until the process exits.  In host code this name is
+// only a handle for the runtime; the device address comes from cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+extern "C" fdqp_status fdqp_run_noalloc(const void* x_bf16, const void* W_q4nx, float* y, int64_t M, int64_t K, int64_t N,
+                                        void* cuda_stream) {
+    if (!x_bf16 || !W_q4nx || !y) return FDQP_ERR_ARG;
+    if (M < 1 || K <= 0 || N <= 0 || (K % kGroup) != 0 || (N % kStripRows) != 0) return FDQP_ERR_SHAPE;
+    if (M > kMaxTokens || N > kNoAllocMaxN) return FDQP_ERR_SIZE;
+    if (!aligned16(x_bf16) || !aligned16(W_q4nx) || !aligned16(y)) return FDQP_ERR_ALIGN;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoAllocMaxDevices) {
+        cudaGetLastError();
+        return FDQP_ERR_CUDA;
+    }
+    NoAllocDevice info;
+    {
+        // First call on this device: look the device up and resolve the scratch array's address, with the device current.
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        NoAllocDevice& d = g_noalloc_devices[dev];
+        if (!d.ready) {
+            int major = 0;
+            if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return FDQP_ERR_CUDA;
+            if (major != 10) return FDQP_ERR_ARCH;
+            if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+                cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+                return FDQP_ERR_CUDA;
+            if (gemv_set_smem_limit(d.smem_optin) != cudaSuccess) { cudaGetLastError(); return FDQP_ERR_CUDA; }
+            void* ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) { cudaGetLastError(); return FDQP_ERR_CUDA; }
+            d.scratch = static_cast<unsigned char*>(ptr);
+            d.ready = true;
+        }
+        info = d;
+    }
+    // Plan with the ordinary planner on a stack context: no K split (its workspace would not be modest) and the
+    // activations prepared inside the kernel (no staging buffer).
+    fdqp_ctx tmp;
+    tmp.device = dev;
+    tmp.sm_count = info.sm_count;
+    tmp.smem_optin = info.smem_optin;
+    tmp.max_M = kMaxTokens;
+    tmp.max_K = K;
+    tmp.max_N = kNoAllocMaxN;
+    tmp.p_split_k = 1;
+    tmp.p_prep = 1;
+    tmp.ws_edge = reinterpret_cast<float*>(info.scratch);
+    tmp.tickets = reinterpret_cast<int*>(info.scratch + kNoAllocEdgeBytes);
+    tmp.status_dev = reinterpret_cast<int*>(info.scratch + kNoAllocEdgeBytes + kNoAllocTicketBytes);
+    GemvPlan plan;
+    int cw = 0;
+    if (!plan_gemv(&tmp, (int)M, (int)K, (int)N, &cw, &plan)) return FDQP_ERR_SIZE;  // the K slice of x must fit shared memory
+    if (plan.Z != 1 || plan.Z * plan.Gz > kNoAllocMaxCtas) return FDQP_ERR_SIZE;
+    plan.W = static_cast<const uint8_t*>(W_q4nx);
+    plan.x = static_cast<const uint16_t*>(x_bf16);
+    plan.y = y;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // The array keeps whatever the last call left: the arrival counters must start at zero.
+    if (cudaMemsetAsync(plan.tickets, 0, sizeof(int) * (size_t)plan.S, stream) != cudaSuccess) { cudaGetLastError(); return FDQP_ERR_CUDA; }
+    if (gemv_launch(plan, cw, stream) != cudaSuccess) { cudaGetLastError(); return FDQP_ERR_CUDA; }
     return FDQP_OK;
 }
