@@ -145,6 +145,53 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------------------------- one shape
+
+def run_shape(args):
+    """Times ONE projection shape (--shape K,N,M): the per-kernel view used for the roofline tables in profiles/.
+    Weights are a seeded 4096-column matrix tiled along N (strip-major makes that byte concatenation); enough distinct
+    copies are rotated to keep every launch's weights out of L2."""
+    import torch
+
+    import paper_2602_06063_b200 as fd
+
+    K, N, M = (int(v) for v in args.shape.split(","))
+    torch.cuda.set_device(0)
+    peaks, peak_kind = measured_peaks()
+    ctx = fd.fdqp_create(0, max(M, 8), K, N)
+    for kv in args.param or []:
+        key, val = kv.split("=")
+        fd.fdqp_set_param(ctx, key, int(val))
+    nb = min(N, 4096)
+    w = synthgen.weights(5, K, nb)
+    tile = fd.q4nx_pack(w.codes, w.scales, w.offsets)
+    packed = np.tile(tile, -(-N // nb))[:fd.q4nx_packed_bytes(K, N)]
+    base = torch.from_numpy(np.ascontiguousarray(packed)).cuda()
+    ncopies = max(1, int(np.ceil(4 * L2_BYTES / base.numel()))) if not args.same_weights else 1
+    copies = [base] + [base.clone() for _ in range(ncopies - 1)]
+    x = torch.from_numpy(synthgen.activations(1, M, K).view(np.int16)).cuda()
+    y = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    sraw = stream.cuda_stream
+    for i in range(max(3, args.warmup)):
+        fd.fdqp_run(ctx, x, copies[i % ncopies], y, M, K, N, sraw)
+    stream.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        fd.fdqp_run(ctx, x, copies[i % ncopies], y, M, K, N, sraw)
+    e1.record(stream)
+    stream.synchronize()
+    assert fd.fdqp_last_status(ctx) == 0
+    us = e0.elapsed_time(e1) * 1e3 / args.steps
+    gbs = alg_bytes(M, K, N) / us / 1e3
+    print(json.dumps({"shape": {"K": K, "N": N, "M": M}, "us_per_call": us, "GBps": gbs,
+                      "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
+                      "peak_kind": peak_kind, "weight_copies": ncopies, "steps": args.steps,
+                      "launch": fd.fdqp_describe(ctx, M, K, N)}), flush=True)
+    fd.fdqp_destroy(ctx)
+
+
 # ----------------------------------------------------------------------------------------------- our arm
 
 def run_ours(args, rank, local_rank, world):
@@ -380,6 +427,8 @@ def main():
     ap.add_argument("--graph", type=int, default=1, help="replay each step from a CUDA graph (default 1)")
     ap.add_argument("--fuse", type=int, default=1, help="run q|k|v and gate|up as one call each (default 1)")
     ap.add_argument("--param", action="append", help="library launch parameter key=value (repeatable)")
+    ap.add_argument("--shape", help="K,N,M: time this one projection shape instead of the layer workload")
+    ap.add_argument("--same-weights", action="store_true", help="with --shape: reuse one weight buffer (for ncu captures)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-head", action="store_true", help="skip the LM-head timing")
     args = ap.parse_args()
@@ -393,6 +442,11 @@ def main():
         return
     if args.warmup < 3:
         args.warmup = 3
+    if args.shape:
+        if args.steps == 400:
+            args.steps = 50
+        run_shape(args)
+        return
     run_ours(args, rank, local_rank, world)
 
 
