@@ -403,7 +403,10 @@ def run_ours(args, rank, local_rank, world):
             "lm_head_ms": head_ms,
             "lm_head_gbs": (alg_bytes(1, hk, hn) / (head_ms * 1e-3) / 1e9) if head_ms else None,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_kind": peak_kind,
+                         "frac": achieved / peaks["hbm_gbs"],
+                         # ncu, K=2560 N=98304 M=1 (profiles/gemv_m1_k2560_n98304.md): dram read+write = 1.023 x the
+                         # algorithmic bytes; traffic grows in proportion to 0.625*K*N, so scale to this call size
+                         "traffic": 1.023 * step_bytes / calls_per_step, "peak_kind": peak_kind + " copy bandwidth",
                          "kernel": "fdqp_gemv_kernel", "launch_us": per_launch_us},
             "cpu_baseline": cpu,
             "e2e": {"value": step_bytes * e2e_steps * world / e2e_s / 1e9, "unit": "GB/s",
