@@ -183,7 +183,8 @@ FDQP_API const char* fdqp_last_cuda_error(fdqp_ctx* ctx);
 FDQP_API const char* fdqp_status_string(fdqp_status s);
 
 /* Override a launch parameter; value < 0 restores the built-in choice.  Keys:
- *   "path"          0 = dispatch on M (default), 1 = force the plain CUDA-core kernel
+ *   "path"          0 = dispatch on M (default), 1 = force the plain CUDA-core kernel,
+ *                   2 = run M >= 9 through the GEMV kernel eight token rows at a time
  *   "ctas_per_sm"   persistent CTAs per SM for the GEMV kernels (1 or 2; 2 implies 8 consumer warps)
  *   "consumer_warps" 8 or 16 consumer warps per CTA
  *   "stages"        shared-memory ring depth in stages (a stage holds consumer_warps / 4 Q4NX blocks)

@@ -17,6 +17,9 @@ cudaError_t gemv_launch(const GemvPlan& p, int consumer_warps, cudaStream_t stre
 cudaError_t gemv_set_smem_limit(int bytes);
 cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream);
 cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
+cudaError_t prefill_set_smem_limit();
+cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, int* status, int M, int K, int N,
+                           cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
 }  // namespace fdqp
 
@@ -229,6 +232,7 @@ extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, in
         *ctx->status_host = 0;
         if ((e = cudaHostGetDevicePointer(&ctx->status_dev, ctx->status_host, 0))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = gemv_set_smem_limit(ctx->smem_optin))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = prefill_set_smem_limit())) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaDeviceSynchronize())) { st = cuda_fail(nullptr, e, ""); break; }
     } while (false);
     if (st != FDQP_OK) {
@@ -269,6 +273,13 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
     cudaError_t e;
     if (ctx->p_path == 1) {
         if ((e = plain_launch(W, x, y, (int)M, (int)K, (int)N, stream))) return cuda_fail(ctx, e, "plain kernel launch");
+        ctx->launches += 1;
+        return FDQP_OK;
+    }
+    if (M > kMaxTokens && ctx->p_path != 2) {
+        // prefill-sized M: dequantise into shared memory, contract with tcgen05 (accumulators in TMEM)
+        if ((e = prefill_launch(W, x, y, ctx->status_dev, (int)M, (int)K, (int)N, stream)))
+            return cuda_fail(ctx, e, "prefill kernel launch");
         ctx->launches += 1;
         return FDQP_OK;
     }
@@ -342,7 +353,7 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
     if (!ctx || !key) return FDQP_ERR_ARG;
     const int64_t v = value < 0 ? -1 : value;
     if (!std::strcmp(key, "path")) {
-        if (v > 1) return FDQP_ERR_ARG;
+        if (v > 2) return FDQP_ERR_ARG;
         ctx->p_path = v;
     } else if (!std::strcmp(key, "ctas_per_sm")) {
         if (v == 0 || v > kMaxCtasPerSm) return FDQP_ERR_ARG;
@@ -382,6 +393,11 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
     if (ctx->p_path == 1) {
         std::snprintf(buf, buf_bytes, "fdqp_plain_kernel grid=(%lld,%lld) block=128", (long long)((N / 32 + 3) / 4),
                       (long long)((M + 7) / 8));
+        return FDQP_OK;
+    }
+    if (M > kMaxTokens && ctx->p_path != 2) {
+        std::snprintf(buf, buf_bytes, "fdqp_prefill_kernel grid=%lld block=320 tile=256x256 stages=3 tmem_cols=512",
+                      (long long)(((N + 255) / 256) * ((M + 255) / 256)));
         return FDQP_OK;
     }
     GemvPlan plan;

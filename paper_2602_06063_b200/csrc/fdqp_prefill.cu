@@ -1,0 +1,374 @@
+// Prefill-sized projection (M >= 9 token rows): dequantise Q4NX blocks into shared memory and contract on the
+// 5th-generation tensor cores (tcgen05.mma, accumulators in TMEM).
+//
+// The paper's prefill path dequantises a Q4NX block to bf16, writes it to DRAM and runs a tiled bf16 GEMM on it
+// (Sec. "Dequantization Engine", Sec. "Tiling-based MM").  Here the DRAM round trip is removed: the dequantised tile
+// only ever exists in shared memory, in the layout the tensor core reads.
+//
+// One CTA computes a 256 (output features) x 256 (tokens) tile of y:
+//   D[n][tok] = sum_k w16[k][n] * x[tok][k],   w16 = RNE_bf16( RN_fp32(d * q + m) )      (Eq. 3, then Eq. 14)
+//   - UMMA shape 128 x N_inst x 16 (kind::f16, bf16 inputs, fp32 accumulate), two accumulators (rows 0..127 and
+//     128..255 of the tile) of 256 TMEM columns each = all 512 columns;
+//   - A = dequantised weights, [256 rows][64 k] bf16 per pipeline stage, K-major, 128-byte swizzle, written by eight
+//     dequantisation warps (one 32-row strip each) with plain shared-memory stores;
+//   - B = x, [256 tokens][64 k] bf16 per stage, K-major, 128-byte swizzle, loaded by TMA (2-D tiled copy, no
+//     multicast); rows beyond M and columns beyond K are zero-filled by the copy engine;
+//   - one elected thread issues the MMAs; tcgen05.commit hands stages back and announces the finished accumulators;
+//   - epilogue: the eight dequantisation warps read TMEM (tcgen05.ld 32x32b) and store fp32 y, 128 contiguous bytes
+//     per warp store.
+// Every wait is bounded; TMEM is released on every path.
+#include <cuda.h>
+
+#include "fdqp_device.cuh"
+#include "fdqp_plan.h"
+
+namespace fdqp {
+
+constexpr int kPfRows = 256;      // output features per CTA tile
+constexpr int kPfToks = 256;      // tokens per CTA tile
+constexpr int kPfK = 64;          // k per pipeline stage (one 128-byte swizzle row of bf16)
+constexpr int kPfStages = 3;
+constexpr uint32_t kPfABytes = kPfRows * kPfK * 2;  // 32 KB
+constexpr uint32_t kPfBBytes = kPfToks * kPfK * 2;  // 32 KB
+constexpr uint32_t kPfStageBytes = kPfABytes + kPfBBytes;
+constexpr int kPfDequantWarps = 8;
+constexpr int kPfThreads = (2 + kPfDequantWarps) * 32;  // warp 0: TMA + TMEM owner, warp 1: MMA issuer
+constexpr uint32_t kPfTmemCols = 512;
+constexpr uint32_t kPfSmemBytes = kPfStages * kPfStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+struct PrefillParams {
+    const uint8_t* W;
+    float* y;
+    int* status;
+    int M, K, N;
+};
+
+// ---- tcgen05 wrappers -----------------------------------------------------------------------------------------
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem desc] * B[smem desc]; issued by one thread for the whole CTA.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive on `bar` once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);  // start address
+    d |= (uint64_t)1 << 16;                        // leading-dimension byte offset (unused for this layout)
+    d |= (uint64_t)(1024 >> 4) << 32;              // stride-dimension byte offset: next 8-row group
+    d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                        // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = n_inst.
+__device__ __forceinline__ uint32_t umma_idesc(uint32_t n_inst) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((n_inst >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,"
+        "%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// ---- dequantisation of one (strip, group) into the swizzled A tile ---------------------------------------------------
+
+struct GroupRegs {
+    uint4 codes;      // this lane's row: 32 codes of the group
+    uint32_t d_bits;  // bf16 scale in the low half
+    uint32_t m_bits;  // bf16 offset in the low half
+    bool valid;
+};
+
+__device__ __forceinline__ GroupRegs group_load(const uint8_t* __restrict__ W, int K, int64_t strip, int g, int lane,
+                                                bool strip_ok) {
+    GroupRegs r;
+    const int groups = K / kGroup;
+    r.valid = strip_ok && g < groups;
+    r.codes = make_uint4(0, 0, 0, 0);
+    r.d_bits = 0;
+    r.m_bits = 0;
+    if (r.valid) {
+        const int b = g >> 3, t = g & 7;
+        const int rest = groups - 8 * b;
+        const int jb = rest < 8 ? rest : 8;
+        const uint8_t* blk = W + strip * ((int64_t)kGroupBytes * groups) + (int64_t)b * kBlockBytes;
+        r.codes = __ldg(reinterpret_cast<const uint4*>(blk + t * 512 + lane * 16));
+        r.d_bits = __ldg(reinterpret_cast<const unsigned short*>(blk + 512 * jb + 2 * (t * 32 + lane)));
+        r.m_bits = __ldg(reinterpret_cast<const unsigned short*>(blk + 576 * jb + 2 * (t * 32 + lane)));
+    }
+    return r;
+}
+
+// (low | high) half of a packed bf16 pair times bf16 d plus fp32 m, rounded once to fp32: exactly Eq. 3, because the
+// product of an integer code <= 15 and a bf16 scale is exact inside the fused multiply-add.
+__device__ __forceinline__ float dequant_lo(uint32_t q2, uint32_t d_bits, float m) {
+    float r;
+    asm("{\n\t.reg .b16 qlo, qhi, dlo, dhi;\n\tmov.b32 {qlo, qhi}, %1;\n\tmov.b32 {dlo, dhi}, %2;\n\t"
+        "fma.rn.f32.bf16 %0, qlo, dlo, %3;\n\t}"
+        : "=f"(r) : "r"(q2), "r"(d_bits), "f"(m));
+    return r;
+}
+__device__ __forceinline__ float dequant_hi(uint32_t q2, uint32_t d_bits, float m) {
+    float r;
+    asm("{\n\t.reg .b16 qlo, qhi, dlo, dhi;\n\tmov.b32 {qlo, qhi}, %1;\n\tmov.b32 {dlo, dhi}, %2;\n\t"
+        "fma.rn.f32.bf16 %0, qhi, dlo, %3;\n\t}"
+        : "=f"(r) : "r"(q2), "r"(d_bits), "f"(m));
+    return r;
+}
+
+// Writes row (strip_local*32 + lane), k in [32*gl, 32*gl + 32) of the A tile: w16 = RNE_bf16(RN_fp32(d*q + m)).
+// Codes become bf16 pairs with one logic op per pair ((w >> 4i) & 0x000F000F | 0x43004300 = (128+q_i, 128+q_{i+4}));
+// the bias is removed exactly by a packed bf16 subtract; no integer-to-float conversion instruction is used.
+__device__ __forceinline__ void group_store(uint8_t* a_tile, const GroupRegs& r, int strip_local, int gl, int lane) {
+    const int row = strip_local * 32 + lane;
+    uint8_t* row_base = a_tile + (row >> 3) * 1024 + (row & 7) * 128;
+    const float m = __uint_as_float(r.m_bits << 16);
+    const uint32_t words[4] = {r.codes.x, r.codes.y, r.codes.z, r.codes.w};
+#pragma unroll
+    for (int wi = 0; wi < 4; ++wi) {  // 8 codes -> one 16-byte chunk
+        const uint32_t w = words[wi];
+        float f[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t q2 = ((w >> (4 * i)) & 0x000F000Fu) | 0x43004300u;  // bf16x2 (128 + q_i, 128 + q_{i+4})
+            asm("sub.bf16x2 %0, %0, %1;" : "+r"(q2) : "r"(0x43004300u));  // exact: (q_i, q_{i+4})
+            f[i] = dequant_lo(q2, r.d_bits, m);
+            f[i + 4] = dequant_hi(q2, r.d_bits, m);
+        }
+        uint32_t out[4];
+#pragma unroll
+        for (int pq = 0; pq < 4; ++pq) {
+            uint32_t packed;
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(packed) : "f"(f[2 * pq + 1]), "f"(f[2 * pq]));  // {hi, lo}
+            out[pq] = r.valid ? packed : 0u;
+        }
+        const int chunk = gl * 4 + wi;  // 16-byte chunk index inside the 128-byte row
+        *reinterpret_cast<uint4*>(row_base + ((chunk ^ (row & 7)) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
+    }
+}
+
+// ---- the kernel -------------------------------------------------------------------------------------------------------
+
+__global__ void __launch_bounds__(kPfThreads, 1)
+    fdqp_prefill_kernel(const __grid_constant__ CUtensorMap x_map, const PrefillParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // tiles must start on a 1024-byte boundary (swizzle atom)
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t bars = base + kPfStages * kPfStageBytes;
+    // barriers: full_a[s], full_b[s], empty[s], acc_done; then the TMEM base address slot
+    auto full_a = [&](int s) { return bars + 8u * s; };
+    auto full_b = [&](int s) { return bars + 8u * (kPfStages + s); };
+    auto empty = [&](int s) { return bars + 8u * (2 * kPfStages + s); };
+    const uint32_t acc_done = bars + 8u * (3 * kPfStages);
+    const uint32_t tmem_slot = acc_done + 8u;
+    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(smem + kPfStages * kPfStageBytes + 8 * (3 * kPfStages + 1));
+
+    const int tok_tiles = (p.M + kPfToks - 1) / kPfToks;
+    const int n_tile = blockIdx.x / tok_tiles, tok_tile = blockIdx.x % tok_tiles;  // token tiles of one n-tile adjacent
+    const int n0 = n_tile * kPfRows, tok0 = tok_tile * kPfToks;
+    const int toks = (p.M - tok0) < kPfToks ? (p.M - tok0) : kPfToks;
+    const uint32_t n_inst = (uint32_t)((toks + 15) & ~15);
+    const int ksteps = (p.K + kPfK - 1) / kPfK;
+
+    if (tid == 0) {
+        for (int s = 0; s < kPfStages; ++s) {
+            mbar_init(full_a(s), kPfDequantWarps);
+            mbar_init(full_b(s), 1);
+            mbar_init(empty(s), 1);
+        }
+        mbar_init(acc_done, 1);
+        mbar_fence_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(tmem_slot, kPfTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot_g;
+    bool ok = true;
+
+    if (warp == 0) {
+        // =============================== TMA producer: x tiles ==============================================
+        if (lane == 0) {
+            for (int i = 0; i < ksteps && ok; ++i) {
+                const int s = i % kPfStages;
+                if (i >= kPfStages) ok = mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status);
+                if (!ok) break;
+                mbar_arrive_expect_tx(full_b(s), kPfBBytes);
+                tma_load_2d(base + s * kPfStageBytes + kPfABytes, &x_map, i * kPfK, tok0, full_b(s));
+            }
+        }
+    } else if (warp == 1) {
+        // =============================== MMA issuer =========================================================
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc(n_inst);
+            for (int i = 0; i < ksteps && ok; ++i) {
+                const int s = i % kPfStages;
+                const uint32_t ph = (i / kPfStages) & 1;
+                ok = mbar_wait(full_a(s), ph, p.status) && mbar_wait(full_b(s), ph, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = base + s * kPfStageBytes, b_addr = a_addr + kPfABytes;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const uint64_t adesc = umma_smem_desc(a_addr + half * (kPfABytes / 2));
+                    const uint64_t bdesc = umma_smem_desc(b_addr);
+#pragma unroll
+                    for (int k4 = 0; k4 < kPfK / 16; ++k4)  // 32 bytes (16 bf16) further along the swizzled row
+                        umma_bf16(tmem_base + half * 256, adesc + 2 * k4, bdesc + 2 * k4, idesc, (i | k4) != 0);
+                }
+                umma_commit(empty(s));  // the stage may be refilled once these MMAs have read it
+            }
+            umma_commit(acc_done);
+        }
+    } else {
+        // =============================== dequantisation warps ================================================
+        const int dw = warp - 2;  // strip of the tile this warp owns
+        const int64_t strip = (int64_t)n_tile * (kPfRows / 32) + dw;
+        const bool strip_ok = strip < p.N / kStripRows;
+        // software pipeline: the loads of the next stage are in flight while this one is converted
+        GroupRegs g0 = group_load(p.W, p.K, strip, 0, lane, strip_ok), g1 = group_load(p.W, p.K, strip, 1, lane, strip_ok);
+        for (int i = 0; i < ksteps && ok; ++i) {
+            const int s = i % kPfStages;
+            GroupRegs n0r, n1r;
+            if (i + 1 < ksteps) {
+                n0r = group_load(p.W, p.K, strip, 2 * (i + 1), lane, strip_ok);
+                n1r = group_load(p.W, p.K, strip, 2 * (i + 1) + 1, lane, strip_ok);
+            } else {
+                n0r = g0;
+                n1r = g1;
+            }
+            if (i >= kPfStages) ok = mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status);
+            if (!ok) break;
+            uint8_t* a_tile = smem + s * kPfStageBytes;
+            group_store(a_tile, g0, dw, 0, lane);
+            group_store(a_tile, g1, dw, 1, lane);
+            // make the generic-proxy stores visible to the tensor core's (async-proxy) reads, then signal
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full_a(s));
+            g0 = n0r;
+            g1 = n1r;
+        }
+        // =============================== epilogue: TMEM -> y =================================================
+        if (ok) ok = mbar_wait(acc_done, 0, p.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+            tc_fence_after();
+            const int quarter = warp & 3;        // TMEM lanes this warp may read
+            const int half = dw >> 2;            // which accumulator: warps 2..5 -> 0, 6..9 -> 1 ... by construction below
+            // warps 2,3,4,5 have quarters 2,3,0,1 and warps 6,7,8,9 have quarters 2,3,0,1: every (half, quarter) once
+            const int n = n0 + half * 128 + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 256);
+            for (int c = 0; c < (int)n_inst; c += 32) {
+                uint32_t v[32];
+                tmem_ld_32cols(taddr + c, v);
+                if (n < p.N) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (c + j < toks) p.y[(int64_t)(tok0 + c + j) * p.N + n] = __uint_as_float(v[j]);
+                }
+            }
+        }
+    }
+    // =============================== teardown: every path releases TMEM =====================================
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kPfTmemCols);
+    }
+}
+
+// ---- host side ----------------------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+cudaError_t prefill_set_smem_limit() {
+    return cudaFuncSetAttribute(fdqp_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPfSmemBytes);
+}
+
+// x: [M][K] bf16 row-major (device).  Returns cudaErrorNotSupported if the tensor map cannot be built.
+cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, int* status, int M, int K, int N,
+                           cudaStream_t stream) {
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return cudaErrorNotSupported;
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};      // innermost first
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};              // bytes between token rows
+    const cuuint32_t box[2] = {(cuuint32_t)kPfK, (cuuint32_t)kPfToks};
+    const cuuint32_t elem[2] = {1, 1};
+    if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t*>(x), dims, strides, box, elem,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    PrefillParams p;
+    p.W = W;
+    p.y = y;
+    p.status = status;
+    p.M = M;
+    p.K = K;
+    p.N = N;
+    const int n_tiles = (N + kPfRows - 1) / kPfRows, tok_tiles = (M + kPfToks - 1) / kPfToks;
+    fdqp_prefill_kernel<<<n_tiles * tok_tiles, kPfThreads, kPfSmemBytes, stream>>>(map, p);
+    return cudaGetLastError();
+}
+
+}  // namespace fdqp

@@ -99,6 +99,43 @@ def test_exact_arithmetic_regime_is_bit_exact(fresh, K, N, M):
         assert np.array_equal(y.astype(np.float64), y_ref), f"path {path}"
 
 
+PREFILL = [(64, 32, 9), (1024, 512, 9), (1056, 320, 20), (2560, 1024, 100), (512, 288, 300), (4096, 768, 512)]
+
+
+@pytest.mark.parametrize("K,N,M", PREFILL)
+def test_prefill_tensor_path_matches_oracle(fresh, K, N, M):
+    # M >= 9: dequantise-into-shared-memory + tcgen05 path.  Ragged token tiles, a K that is not a multiple of
+    # the 64-wide pipeline step, N that is not a multiple of the 256-row tile, more than one token tile.
+    case = Case(K, N, M, seed=2000 + K + N + M)
+    assert "fdqp_prefill_kernel" in fd.fdqp_describe(fresh, M, K, N)
+    y = case.run(fresh)
+    y_ref, a_ref = case.reference()
+    assert_close(y, y_ref, a_ref, f"prefill K={K} N={N} M={M}")
+    # the same rows through the GEMV kernel, eight at a time: both are within the bound of the oracle
+    fd.fdqp_set_param(fresh, "path", 2)
+    assert "fdqp_gemv_kernel" in fd.fdqp_describe(fresh, M, K, N)
+    assert_close(case.run(fresh), y_ref, a_ref, f"gemv-chunked K={K} N={N} M={M}")
+
+
+def test_prefill_exact_cases(fresh):
+    # (i) exact-arithmetic regime: weights are bf16-exact, every fp32 sum is exact -> bit-equal to the oracle
+    K, N, M = 1152, 288, 40
+    case = Case(K, N, M, seed=0, weights=exact_regime_weights(71, K, N), x=exact_regime_x(72, M, K))
+    y_ref, _ = case.reference()
+    assert np.array_equal(case.run(fresh).astype(np.float64), y_ref)
+    # (ii) one-hot activations read out rows of the bf16-rounded dequantised matrix, bit for bit
+    K, N, M = 544, 96, 16
+    c2 = Case(K, N, M, seed=73)
+    _, w16 = oracle.dequant(c2.w.codes, c2.w.scales, c2.w.offsets)
+    ks = [0, 31, 32, 63, 64, 255, 256, 300, 511, 512, 543, 7, 100, 200, 400, 500]
+    x = np.zeros((M, K), np.float32)
+    for i, kk in enumerate(ks):
+        x[i, kk] = 1.0
+    y = Case(K, N, M, 0, weights=c2.w, x=synthgen.bf16_bits(x)).run(fresh)
+    assert np.array_equal(y.view(np.uint32) >> 16, w16[ks].astype(np.uint32))
+    assert np.all((y.view(np.uint32) & 0xFFFF) == 0)
+
+
 def test_worked_examples_on_gpu(fresh):
     # E1/E2: K = N = 32, code = (k + 3n) mod 16, d = 0.5, m = -1; x = 1 -> 88; x = e_5 -> 0.5*((5+3n)%16) - 1
     n, k = np.arange(32)[:, None], np.arange(32)[None, :]
