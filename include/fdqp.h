@@ -119,7 +119,9 @@ FDQP_API fdqp_status fdqp_destroy(fdqp_ctx* ctx);
  * Dispatch: M = 1 and 2..8 run the streaming GEMV kernels (weights fetched once
  * from HBM through a shared-memory ring, nibbles unpacked in registers, scale and
  * offset applied in fp32, split-K across CTAs reduced in a fixed order); M >= 9
- * runs the dequantise-into-shared-memory tensor-core path.
+ * runs the dequantise-into-shared-memory tensor-core path (tcgen05, accumulators
+ * in TMEM) when its 256 x 256 output tiles can fill at least half of the SMs or
+ * M > 128, and otherwise the GEMV kernel eight token rows at a time.
  * In the GEMV kernels the activations of each 32-group are held as 24-bit fixed
  * point relative to the group's largest exponent: exact for every element within
  * 2^15 of the group's largest magnitude, rounded to 2^-23 of it otherwise.
@@ -184,7 +186,8 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
 
 /* Override a launch parameter; value < 0 restores the built-in choice.  Keys:
  *   "path"          0 = dispatch on M (default), 1 = force the plain CUDA-core kernel,
- *                   2 = run M >= 9 through the GEMV kernel eight token rows at a time
+ *                   2 = run M >= 9 through the GEMV kernel eight token rows at a time,
+ *                   3 = run every M >= 9 through the tensor-core prefill kernel
  *   "ctas_per_sm"   persistent CTAs per SM for the GEMV kernels (1 or 2; 2 implies 8 consumer warps)
  *   "consumer_warps" 8 or 16 consumer warps per CTA
  *   "stages"        shared-memory ring depth in stages (a stage holds consumer_warps / 4 Q4NX blocks)

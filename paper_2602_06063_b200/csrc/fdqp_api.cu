@@ -78,6 +78,15 @@ fdqp_status check_shape(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     return FDQP_OK;
 }
 
+// M >= 9 goes to the tensor-core kernel when its 256 x 256 tiles can occupy at least half of the SMs or the token
+// count is large; a few tiles with few tokens are faster through the GEMV kernel, eight token rows at a time.
+bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t N) {
+    if (M <= kMaxTokens || ctx->p_path == 2) return false;
+    if (ctx->p_path == 3) return true;
+    const int64_t tiles = ((N + 255) / 256) * ((M + 255) / 256);
+    return tiles * 2 >= ctx->sm_count || M > 128;
+}
+
 // Shared-memory carve-up for a given configuration; returns the ring depth that fits (0 if none).
 struct SmemLayout {
     uint32_t stage_bytes, xs_bytes, xsum_bytes, part_bytes, fixed;
@@ -276,7 +285,7 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
         ctx->launches += 1;
         return FDQP_OK;
     }
-    if (M > kMaxTokens && ctx->p_path != 2) {
+    if (use_prefill(ctx, M, N)) {
         // prefill-sized M: dequantise into shared memory, contract with tcgen05 (accumulators in TMEM)
         if ((e = prefill_launch(W, x, y, ctx->status_dev, (int)M, (int)K, (int)N, stream)))
             return cuda_fail(ctx, e, "prefill kernel launch");
@@ -353,7 +362,7 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
     if (!ctx || !key) return FDQP_ERR_ARG;
     const int64_t v = value < 0 ? -1 : value;
     if (!std::strcmp(key, "path")) {
-        if (v > 2) return FDQP_ERR_ARG;
+        if (v > 3) return FDQP_ERR_ARG;
         ctx->p_path = v;
     } else if (!std::strcmp(key, "ctas_per_sm")) {
         if (v == 0 || v > kMaxCtasPerSm) return FDQP_ERR_ARG;
@@ -395,7 +404,7 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
                       (long long)((M + 7) / 8));
         return FDQP_OK;
     }
-    if (M > kMaxTokens && ctx->p_path != 2) {
+    if (use_prefill(ctx, M, N)) {
         std::snprintf(buf, buf_bytes, "fdqp_prefill_kernel grid=%lld block=320 tile=256x256 stages=3 tmem_cols=512",
                       (long long)(((N + 255) / 256) * ((M + 255) / 256)));
         return FDQP_OK;

@@ -157,9 +157,11 @@ __device__ __forceinline__ float dequant_hi(uint32_t q2, uint32_t d_bits, float 
 // Writes row (strip_local*32 + lane), k in [32*gl, 32*gl + 32) of the A tile: w16 = RNE_bf16(RN_fp32(d*q + m)).
 // Codes become bf16 pairs with one logic op per pair ((w >> 4i) & 0x000F000F | 0x43004300 = (128+q_i, 128+q_{i+4}));
 // the bias is removed exactly by a packed bf16 subtract; no integer-to-float conversion instruction is used.
+// An absent group arrives with codes, d and m all zero and therefore writes zeros.
 __device__ __forceinline__ void group_store(uint8_t* a_tile, const GroupRegs& r, int strip_local, int gl, int lane) {
     const int row = strip_local * 32 + lane;
     uint8_t* row_base = a_tile + (row >> 3) * 1024 + (row & 7) * 128;
+    const uint32_t r7s = (uint32_t)(row & 7) << 4;
     const float m = __uint_as_float(r.m_bits << 16);
     const uint32_t words[4] = {r.codes.x, r.codes.y, r.codes.z, r.codes.w};
 #pragma unroll
@@ -173,15 +175,13 @@ __device__ __forceinline__ void group_store(uint8_t* a_tile, const GroupRegs& r,
             f[i] = dequant_lo(q2, r.d_bits, m);
             f[i + 4] = dequant_hi(q2, r.d_bits, m);
         }
-        uint32_t out[4];
-#pragma unroll
-        for (int pq = 0; pq < 4; ++pq) {
-            uint32_t packed;
-            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(packed) : "f"(f[2 * pq + 1]), "f"(f[2 * pq]));  // {hi, lo}
-            out[pq] = r.valid ? packed : 0u;
-        }
-        const int chunk = gl * 4 + wi;  // 16-byte chunk index inside the 128-byte row
-        *reinterpret_cast<uint4*>(row_base + ((chunk ^ (row & 7)) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
+        uint4 out;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out.x) : "f"(f[1]), "f"(f[0]));  // {hi, lo}
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out.y) : "f"(f[3]), "f"(f[2]));
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out.z) : "f"(f[5]), "f"(f[4]));
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out.w) : "f"(f[7]), "f"(f[6]));
+        // 16-byte chunk (gl*4 + wi) of the 128-byte row, at its swizzled position
+        *reinterpret_cast<uint4*>(row_base + ((uint32_t)((gl * 4 + wi) << 4) ^ r7s)) = out;
     }
 }
 

@@ -107,6 +107,7 @@ def test_prefill_tensor_path_matches_oracle(fresh, K, N, M):
     # M >= 9: dequantise-into-shared-memory + tcgen05 path.  Ragged token tiles, a K that is not a multiple of
     # the 64-wide pipeline step, N that is not a multiple of the 256-row tile, more than one token tile.
     case = Case(K, N, M, seed=2000 + K + N + M)
+    fd.fdqp_set_param(fresh, "path", 3)
     assert "fdqp_prefill_kernel" in fd.fdqp_describe(fresh, M, K, N)
     y = case.run(fresh)
     y_ref, a_ref = case.reference()
@@ -120,6 +121,7 @@ def test_prefill_tensor_path_matches_oracle(fresh, K, N, M):
 def test_prefill_exact_cases(fresh):
     # (i) exact-arithmetic regime: weights are bf16-exact, every fp32 sum is exact -> bit-equal to the oracle
     K, N, M = 1152, 288, 40
+    fd.fdqp_set_param(fresh, "path", 3)
     case = Case(K, N, M, seed=0, weights=exact_regime_weights(71, K, N), x=exact_regime_x(72, M, K))
     y_ref, _ = case.reference()
     assert np.array_equal(case.run(fresh).astype(np.float64), y_ref)
@@ -154,7 +156,8 @@ def test_worked_examples_on_gpu(fresh):
                              synthgen.bf16_bits(((n - 32) / 16.0 + g).astype(np.float32)))
     m_idx = np.arange(9)[:, None]
     xf = (((k + m_idx) % 5) - 2).astype(np.float32)
-    for M in (2, 9):
+    for M, path in ((2, 0), (9, 2), (9, 3)):
+        fd.fdqp_set_param(fresh, "path", path)
         y = Case(K, N, M, 0, weights=w, x=synthgen.bf16_bits(xf[:M])).run(fresh)
         assert y[0, 0] == 10.25 and y[0, 1] == -1.625 and y[0, 31] == -5.875 and y[0, 32] == 6.25
         assert y[0, 63] == -9.875 and y[1, 0] == -9.5 and y[1, 17] == -6.625 and y[1, 63] == -6.375
