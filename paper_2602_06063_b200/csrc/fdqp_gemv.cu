@@ -186,19 +186,26 @@ struct TileIn {
     uint32_t so[4];  // (d[g], d[g+8]), (d[g+16], d[g+24]), (m[g], m[g+8]), (m[g+16], m[g+24]) as bf16 pairs
     uint32_t b[6];   // B fragments {even k, odd k}: planes 2, 1, 0 (NT == 2) or this lane's column (NT == 1)
     float sc[4];     // {sum x, unit} of token 2q and of token 2q+1 (NT == 2) or of the only token (NT == 1)
+    uint32_t m_row;  // NT == 1: bf16 offset of row `lane` (low half)
 };
 
+// NT == 1: so_addr addresses the scale chunks only (lanes 0..15 matter) and m_addr this lane's own offset word.
 template <int NT>
-__device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_t so_addr, uint32_t x_addr,
+__device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_t so_addr, uint32_t m_addr, uint32_t x_addr,
                                           uint32_t xsc_addr) {
     ldmatrix_x4(t.c, code_addr);
-    ldmatrix_x4_trans(t.so, so_addr);
     if (NT == 1) {
+        uint32_t dd[2];
+        ldmatrix_x2_trans(dd, so_addr);
+        t.so[0] = dd[0];
+        t.so[1] = dd[1];
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(t.m_row) : "r"(m_addr));
         asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(t.b[0]), "=r"(t.b[1]) : "r"(x_addr));
         const float2 v = lds64f(xsc_addr);
         t.sc[0] = v.x;
         t.sc[1] = v.y;
     } else {
+        ldmatrix_x4_trans(t.so, so_addr);
         const uint4 r0 = lds128(x_addr);
         t.b[0] = r0.x; t.b[1] = r0.y; t.b[2] = r0.z; t.b[3] = r0.w;
         asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(t.b[4]), "=r"(t.b[5]) : "r"(x_addr + 16));
@@ -210,7 +217,8 @@ __device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_
 
 template <bool B_SIGNED>
 __device__ __forceinline__ void imma(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                     uint32_t b1) {
+                                     uint32_t b1, int c = kMagicBits) {
+    const int kMagicBits = c;  // accumulator start value (shadows the constant on purpose)
     if (B_SIGNED)
         asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
             : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
@@ -226,16 +234,35 @@ __device__ __forceinline__ void imma(int (&d)[4], uint32_t a0, uint32_t a1, uint
 //   q == 1: columns (plane 0, zero)    -> s0, weighted unit
 //   q >= 2: zero columns
 struct LaneConst {
-    float k_first;  // weight of the first column relative to the second
+    int k_first;    // weight of the first column relative to the second (256 or 1)
     float w_unit;   // factor on `unit`
-    float w_sum;    // factor on `sum x`
 };
 
 // acc[row][tok] += d * unit * (sum_k q_k X_k) + m * (sum_k x_k), fp32 (Eq. 3 applied per group).
 // `unit` (and 256 * unit) are powers of two, so d * unit is formed exactly by the mixed bf16 FMA.
+// acc_m (NT == 1 only): this lane's row (row = lane) of sum_g m_g * X_g; the offset term does not need the MMA layout.
 template <int NT>
-__device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][NT], const LaneConst& lc) {
-    const float uq = t.sc[1] * lc.w_unit, xq = t.sc[0] * lc.w_sum;  // used when NT == 1
+__device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][NT], float& acc_m, const LaneConst& lc) {
+    if (NT == 1) {
+        const float uq = t.sc[1] * lc.w_unit;
+        acc_m = fmaf(bf16lo_mul_f32hi(t.m_row, 1.0f), t.sc[0], acc_m);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {  // rows (g, g+8) then (g+16, g+24)
+            const uint32_t w0 = t.c[2 * h], w1 = t.c[2 * h + 1];
+            const uint32_t e0 = w0 & 0x0F0F0F0Fu, o0 = (w0 >> 4) & 0x0F0F0F0Fu;  // even-k codes, odd-k codes
+            const uint32_t e1 = w1 & 0x0F0F0F0Fu, o1 = (w1 >> 4) & 0x0F0F0F0Fu;
+            int d[4];
+            imma<true>(d, e0, e1, o0, o1, t.b[0], t.b[1], 0);
+            const float dq[2] = {bf16lo_mul_f32hi(t.so[h], uq), bf16hi_mul_f32hi(t.so[h], uq)};
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                // the lane's two columns combined in integers (exact, |.| < 2^24), one conversion
+                const float s = __int2float_rn(d[2 * r] * lc.k_first + d[2 * r + 1]);
+                acc[2 * h + r][0] = fmaf(dq[r], s, acc[2 * h + r][0]);
+            }
+        }
+        return;
+    }
     const float mof[4] = {bf16lo_mul_f32hi(t.so[2], 1.0f), bf16hi_mul_f32hi(t.so[2], 1.0f),
                           bf16lo_mul_f32hi(t.so[3], 1.0f), bf16hi_mul_f32hi(t.so[3], 1.0f)};
 #pragma unroll
@@ -243,37 +270,23 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][NT
         const uint32_t w0 = t.c[2 * h], w1 = t.c[2 * h + 1];
         const uint32_t e0 = w0 & 0x0F0F0F0Fu, o0 = (w0 >> 4) & 0x0F0F0F0Fu;  // even-k codes, odd-k codes
         const uint32_t e1 = w1 & 0x0F0F0F0Fu, o1 = (w1 >> 4) & 0x0F0F0F0Fu;
-        if (NT == 1) {
-            int d[4];
-            imma<true>(d, e0, e1, o0, o1, t.b[0], t.b[1]);
-            const float dq[2] = {bf16lo_mul_f32hi(t.so[h], uq), bf16hi_mul_f32hi(t.so[h], uq)};
+        int d2[4], d1[4], d0[4];
+        imma<true>(d2, e0, e1, o0, o1, t.b[0], t.b[1]);
+        imma<false>(d1, e0, e1, o0, o1, t.b[2], t.b[3]);
+        imma<false>(d0, e0, e1, o0, o1, t.b[4], t.b[5]);
 #pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const int i = 2 * h + r;
-                const float a0 = __int_as_float(d[2 * r]) - kMagic, a1 = __int_as_float(d[2 * r + 1]) - kMagic;
-                const float s = fmaf(a0, lc.k_first, a1);  // exact: |s| < 2^24
-                acc[i][0] = fmaf(dq[r], s, acc[i][0]);
-                acc[i][0] = fmaf(mof[i], xq, acc[i][0]);
-            }
-        } else {
-            int d2[4], d1[4], d0[4];
-            imma<true>(d2, e0, e1, o0, o1, t.b[0], t.b[1]);
-            imma<false>(d1, e0, e1, o0, o1, t.b[2], t.b[3]);
-            imma<false>(d0, e0, e1, o0, o1, t.b[4], t.b[5]);
+        for (int r = 0; r < 2; ++r) {
+            const int i = 2 * h + r;
 #pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const int i = 2 * h + r;
-#pragma unroll
-                for (int j = 0; j < NT; ++j) {
-                    const int e = 2 * r + j;
-                    const float s2 = __int_as_float(d2[e]) - kMagic, s1 = __int_as_float(d1[e]) - kMagic,
-                                s0 = __int_as_float(d0[e]) - kMagic;
-                    const float s = fmaf(fmaf(s2, 256.f, s1), 256.f, s0);  // exact up to 2^24, else one rounding
-                    const float dq = r == 0 ? bf16lo_mul_f32hi(t.so[h], t.sc[2 * j + 1])
-                                            : bf16hi_mul_f32hi(t.so[h], t.sc[2 * j + 1]);
-                    acc[i][j] = fmaf(dq, s, acc[i][j]);
-                    acc[i][j] = fmaf(mof[i], t.sc[2 * j], acc[i][j]);
-                }
+            for (int j = 0; j < NT; ++j) {
+                const int e = 2 * r + j;
+                const float s2 = __int_as_float(d2[e]) - kMagic, s1 = __int_as_float(d1[e]) - kMagic,
+                            s0 = __int_as_float(d0[e]) - kMagic;
+                const float s = fmaf(fmaf(s2, 256.f, s1), 256.f, s0);  // exact up to 2^24, else one rounding
+                const float dq = r == 0 ? bf16lo_mul_f32hi(t.so[h], t.sc[2 * j + 1])
+                                        : bf16hi_mul_f32hi(t.so[h], t.sc[2 * j + 1]);
+                acc[i][j] = fmaf(dq, s, acc[i][j]);
+                acc[i][j] = fmaf(mof[i], t.sc[2 * j], acc[i][j]);
             }
         }
     }
@@ -408,16 +421,17 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         const uint32_t xsc_lane = (NT == 1) ? xs + 96u : xsc + q * 16;
         const uint32_t xsc_stride = (NT == 1) ? 128u : 64u;
         LaneConst lc;
-        lc.k_first = q == 0 ? 256.f : 1.f;
+        lc.k_first = q == 0 ? 256 : 1;
         lc.w_unit = q == 0 ? 256.f : (q == 1 ? 1.f : 0.f);
-        lc.w_sum = q == 0 ? 1.f : 0.f;
+        float acc_m = 0.f;  // NT == 1: offset term of row `lane`
         // ldmatrix source rows: codes = row `lane` of the tile; scales/offsets = the four 16-byte
         // chunks of this tile's scale words and of its offset words, duplicated so that after the
         // transposed load every lane of a quad holds (d[g], d[g+8]), (d[g+16], d[g+24]), (m..), (m..)
         const uint32_t code_lane = tw * 512 + lane * 16;
         const int mat = lane >> 3;
         const uint32_t so_chunk = tw * 64 + (((mat & 1) * 2 + (lane & 1)) * 16);
-        const uint32_t so_sect = mat >= 2 ? 576u : 512u;  // offsets section follows the scales section
+        const uint32_t so_sect = (NT == 2 && mat >= 2) ? 576u : 512u;  // offsets section follows the scales section
+        const uint32_t m_lane = tw * 64 + lane * 2;                      // NT == 1: this lane's own offset word
 
         float acc[4][NT];
 #pragma unroll
@@ -429,9 +443,13 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         bool alive = true;
         // hand the warp's partial rows of the current strip piece to the reducer warp
         auto flush = [&]() {
-            if (NT == 1) {  // lanes q == 0 and q == 1 hold the two halves of each row's sum
+            if (NT == 1) {  // lanes q == 0 and q == 1 hold the two halves of each row's sum; lane r holds row r's offsets
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[i][0] += __shfl_xor_sync(0xffffffffu, acc[i][0], 1);
+                for (int i = 0; i < 4; ++i) {
+                    acc[i][0] += __shfl_xor_sync(0xffffffffu, acc[i][0], 1);
+                    acc[i][0] += __shfl_sync(0xffffffffu, acc_m, g + 8 * i);
+                }
+                acc_m = 0.f;
             }
             const int par = piece & 1;
             if (piece >= 2 && !mbar_wait(red_empty0 + 8u * par, ((piece >> 1) - 1) & 1, p.status)) alive = false;
@@ -522,14 +540,14 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             if (i1 < lim) {
                 const int tile = bl0 * 8 + tw;
                 const uint32_t xa = x_lane + tile * x_stride, sa = xsc_lane + tile * xsc_stride;
-                tile_load<NT>(ta, sbase + code_lane, sbase + so_lane8, xa, sa);
-                tile_load<NT>(tb, sbase + kBlockBytes + code_lane, sbase + kBlockBytes + so_lane8, xa + 8 * x_stride,
-                              sa + 8 * xsc_stride);
-                tile_compute<NT>(ta, acc, lc);
+                tile_load<NT>(ta, sbase + code_lane, sbase + so_lane8, sbase + 576u * 8u + m_lane, xa, sa);
+                tile_load<NT>(tb, sbase + kBlockBytes + code_lane, sbase + kBlockBytes + so_lane8,
+                              sbase + kBlockBytes + 576u * 8u + m_lane, xa + 8 * x_stride, sa + 8 * xsc_stride);
+                tile_compute<NT>(ta, acc, acc_m, lc);
                 // every shared-memory read of this stage has been consumed by now: hand the stage back
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8u * stage);
-                tile_compute<NT>(tb, acc, lc);
+                tile_compute<NT>(tb, acc, acc_m, lc);
             } else {
                 // general stage: range end, strip boundary between the two blocks, or a short last block
                 const bool cross = i1 >= unit_next;
@@ -539,20 +557,21 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                 const bool act0 = work && (i0 < nblk) && (tw < jb0), act1 = work && (i1 < nblk) && (tw < jb1);
                 if (act0) {
                     const int tile = bl0 * 8 + tw;
-                    tile_load<NT>(ta, sbase + code_lane, sbase + so_sect * jb0 + so_chunk, x_lane + tile * x_stride,
-                                  xsc_lane + tile * xsc_stride);
+                    tile_load<NT>(ta, sbase + code_lane, sbase + so_sect * jb0 + so_chunk, sbase + 576u * jb0 + m_lane,
+                                  x_lane + tile * x_stride, xsc_lane + tile * xsc_stride);
                 }
                 if (act1) {
                     const int tile = bl1 * 8 + tw;
                     tile_load<NT>(tb, sbase + kBlockBytes + code_lane, sbase + kBlockBytes + so_sect * jb1 + so_chunk,
-                                  x_lane + tile * x_stride, xsc_lane + tile * xsc_stride);
+                                  sbase + kBlockBytes + 576u * jb1 + m_lane, x_lane + tile * x_stride,
+                                  xsc_lane + tile * xsc_stride);
                 }
-                if (act0) tile_compute<NT>(ta, acc, lc);
+                if (act0) tile_compute<NT>(ta, acc, acc_m, lc);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8u * stage);
                 if (i1 < nblk) {
                     if (cross && alive) { flush(); next_unit(); lim = interior_limit(); }
-                    if (act1) tile_compute<NT>(tb, acc, lc);
+                    if (act1) tile_compute<NT>(tb, acc, acc_m, lc);
                 }
             }
             if (++stage == nstage) { stage = 0; phase ^= 1u; }
