@@ -42,7 +42,7 @@ struct fdqp_ctx {
     int64_t launches = 0;
     std::string last_err;
     // overrides (-1 = automatic)
-    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1, p_prep = -1, p_aligned = -1;
+    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1, p_prep = -1, p_aligned = -1, p_bpw = -1;
 };
 
 namespace {
@@ -93,9 +93,9 @@ struct SmemLayout {
     int nstage;
 };
 
-SmemLayout smem_layout(const fdqp_ctx* ctx, int M, int nbz, int cw, int ctas_per_sm) {
+SmemLayout smem_layout(const fdqp_ctx* ctx, int M, int nbz, int cw, int ctas_per_sm, int bpw) {
     SmemLayout L;
-    L.stage_bytes = (uint32_t)(cw / 4) * kBlockBytes;
+    L.stage_bytes = (uint32_t)(cw / 8) * (uint32_t)bpw * kBlockBytes;
     const uint32_t tiles = (uint32_t)nbz * 8u;
     L.xs_bytes = tiles * 128u * (uint32_t)M;          // prepared activations of the K slice
     L.xsum_bytes = M == 1 ? 0u : tiles * 64u;         // per-token {sum x, unit}
@@ -122,7 +122,7 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     int ctas_per_sm = ctx->p_ctas_per_sm > 0 ? (int)ctx->p_ctas_per_sm
                                              : (M == 1 && ctx->p_cw != 16 && packed_bytes >= kTwoCtaBytes ? 2 : 1);
     if (ctas_per_sm > kMaxCtasPerSm) ctas_per_sm = kMaxCtasPerSm;
-    int cw = 16, Z = 1, nbz = p->nb;
+    int cw = 16, Z = 1, nbz = p->nb, bpw = 2;
     SmemLayout L{};
     for (;; --ctas_per_sm) {
         // register file: one 19-warp CTA or two 10-warp CTAs fit an SM
@@ -132,7 +132,11 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
         for (;; Z *= 2) {
             if (Z > p->nb) Z = p->nb;
             nbz = (p->nb + Z - 1) / Z;
-            L = smem_layout(ctx, M, nbz, cw, ctas_per_sm);
+            // four blocks per warp per stage halve the barrier traffic per tile; worth it once a CTA streams many blocks
+            const int64_t blocks_per_cta = (int64_t)p->S * p->nb / ((int64_t)ctx->sm_count * ctas_per_sm);
+            bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (M == 1 && blocks_per_cta >= 32 ? 4 : 2);
+            if (M != 1) bpw = 2;
+            L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw);
             if (L.nstage >= kMinStages || Z >= kMaxSplit || Z >= p->nb) break;
         }
         if (L.nstage >= 2 || ctas_per_sm == 1) break;
@@ -164,6 +168,7 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     int nstage = L.nstage;
     if (ctx->p_stages > 0 && ctx->p_stages < nstage) nstage = (int)ctx->p_stages;
     p->nstage = nstage;
+    p->bpw = bpw;
     p->off_xs = (uint32_t)nstage * L.stage_bytes;
     p->off_xsum = p->off_xs + round_up(L.xs_bytes, 128);
     p->off_part = p->off_xsum + round_up(L.xsum_bytes, 128);
@@ -381,6 +386,9 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
         ctx->p_evict = v;
     } else if (!std::strcmp(key, "debug")) {
         ctx->p_debug = v;
+    } else if (!std::strcmp(key, "blocks_per_warp")) {
+        if (v != -1 && v != 2 && v != 4) return FDQP_ERR_ARG;
+        ctx->p_bpw = v;
     } else if (!std::strcmp(key, "strip_aligned")) {
         if (v > 1) return FDQP_ERR_ARG;
         ctx->p_aligned = v;
@@ -415,9 +423,9 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
     if (!plan_gemv(ctx, mc, (int)K, (int)N, &cw, &plan)) return FDQP_ERR_SIZE;
     std::snprintf(buf, buf_bytes,
                   "%sfdqp_gemv_kernel<%d,%d> calls=%lld grid=%d block=%d smem=%u stages=%d split_k=%d ctas_per_slice=%d "
-                  "evict_first=%d strip_aligned=%d",
+                  "evict_first=%d strip_aligned=%d blocks_per_warp=%d",
                   plan.prep_inline ? "" : "fdqp_xprep_kernel + ", cw, mc == 1 ? 1 : 2, (long long)((M + kMaxTokens - 1) / kMaxTokens), plan.Z * plan.Gz, (cw + 1 + cw / 8) * 32,
-                  plan.smem_bytes, plan.nstage, plan.Z, plan.Gz, plan.evict_first, plan.strip_aligned);
+                  plan.smem_bytes, plan.nstage, plan.Z, plan.Gz, plan.evict_first, plan.strip_aligned, plan.bpw);
     return FDQP_OK;
 }
 

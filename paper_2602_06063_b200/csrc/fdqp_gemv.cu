@@ -293,14 +293,14 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][NT
 }
 
 // CW consumer warps (8 or 16); NT token columns kept per lane (1 when M == 1, else 2).
-// A ring stage holds CB = CW / 4 blocks; warp w owns group-tile (w & 7) of blocks 2*(w >> 3) and
-// 2*(w >> 3) + 1 of every stage.
+// A ring stage holds CB = (CW / 8) * BPW blocks; warp w owns group-tile (w & 7) of the BPW (2 or 4) consecutive
+// blocks starting at BPW * (w >> 3) of every stage.  More blocks per stage = fewer barrier round trips per tile.
 // Warps CW+1 .. CW+NR are reducers (NR = CW / 8): reducer r completes the strip pieces with piece % NR == r.
-template <int CW, int NT>
+template <int CW, int NT, int BPW>
 __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
     fdqp_gemv_kernel(const __grid_constant__ GemvPlan p) {
     extern __shared__ __align__(128) uint8_t smem[];
-    constexpr int CB = CW / 4;
+    constexpr int CB = (CW / 8) * BPW;
     constexpr int NR = CW / 8;
     constexpr uint32_t kStageBytes = CB * kBlockBytes;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -410,7 +410,7 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
 
     if (warp < CW) {
         // =============================== consumers ===============================================
-        const int tw = warp & 7, j0 = (warp >> 3) * 2;
+        const int tw = warp & 7, j0 = (warp >> 3) * BPW;
         const int g = lane >> 2, q = lane & 3;
         // B fragments.  NT == 2: column g is token g (any valid token for unused columns: their results are
         // never stored).  NT == 1: column g < 3 is plane 2 - g of the only token, other columns read zeros.
@@ -527,7 +527,7 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         int stage = 0;
         uint32_t phase = 0;
         for (int c = 0; c < nchunk && alive; ++c) {
-            const int i0 = c * CB + j0, i1 = i0 + 1;
+            const int i0 = c * CB + j0;
             if (i0 < nblk && i0 >= unit_next) {
                 while (i0 >= unit_next && alive) { flush(); next_unit(); }
                 lim = interior_limit();
@@ -535,44 +535,49 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             if (!mbar_wait(full0 + 8u * stage, phase, p.status)) { alive = false; break; }
             if (warp == 0 && c == 0) FDQP_STAMP(3);
             const uint32_t sbase = ring + stage * kStageBytes + j0 * kBlockBytes;
-            const int bl0 = i0 - unit_first;
-            TileIn ta, tb;
-            if (i1 < lim) {
-                const int tile = bl0 * 8 + tw;
+            if (i0 + BPW - 1 < lim) {
+                const int tile = (i0 - unit_first) * 8 + tw;
                 const uint32_t xa = x_lane + tile * x_stride, sa = xsc_lane + tile * xsc_stride;
-                tile_load<NT>(ta, sbase + code_lane, sbase + so_lane8, sbase + 576u * 8u + m_lane, xa, sa);
-                tile_load<NT>(tb, sbase + kBlockBytes + code_lane, sbase + kBlockBytes + so_lane8,
-                              sbase + kBlockBytes + 576u * 8u + m_lane, xa + 8 * x_stride, sa + 8 * xsc_stride);
-                tile_compute<NT>(ta, acc, acc_m, lc);
-                // every shared-memory read of this stage has been consumed by now: hand the stage back
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8u * stage);
-                tile_compute<NT>(tb, acc, acc_m, lc);
+#pragma unroll
+                for (int pr = 0; pr < BPW / 2; ++pr) {  // two tiles in flight at a time
+                    const uint32_t sb = sbase + pr * 2 * kBlockBytes;
+                    TileIn ta, tb;
+                    tile_load<NT>(ta, sb + code_lane, sb + so_lane8, sb + 576u * 8u + m_lane, xa + (16 * pr) * x_stride,
+                                  sa + (16 * pr) * xsc_stride);
+                    tile_load<NT>(tb, sb + kBlockBytes + code_lane, sb + kBlockBytes + so_lane8,
+                                  sb + kBlockBytes + 576u * 8u + m_lane, xa + (16 * pr + 8) * x_stride,
+                                  sa + (16 * pr + 8) * xsc_stride);
+                    tile_compute<NT>(ta, acc, acc_m, lc);
+                    if (pr == BPW / 2 - 1) {
+                        // every shared-memory read of this stage has been issued and consumed in order: hand it back
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(empty0 + 8u * stage);
+                    }
+                    tile_compute<NT>(tb, acc, acc_m, lc);
+                }
             } else {
-                // general stage: range end, strip boundary between the two blocks, or a short last block
-                const bool cross = i1 >= unit_next;
-                const int bl1 = cross ? i1 - (unit_next - first_fix) : i1 - unit_first;
-                const int r0 = groups_total - 8 * (b_first + bl0), r1 = groups_total - 8 * (b_first + bl1);
-                const int jb0 = r0 < 8 ? r0 : 8, jb1 = r1 < 8 ? r1 : 8;
-                const bool act0 = work && (i0 < nblk) && (tw < jb0), act1 = work && (i1 < nblk) && (tw < jb1);
-                if (act0) {
-                    const int tile = bl0 * 8 + tw;
-                    tile_load<NT>(ta, sbase + code_lane, sbase + so_sect * jb0 + so_chunk, sbase + 576u * jb0 + m_lane,
-                                  x_lane + tile * x_stride, xsc_lane + tile * xsc_stride);
+                // general stage (range end, strip boundary, short last block): one block at a time
+                for (int jj = 0; jj < BPW; ++jj) {
+                    const int i = i0 + jj;
+                    if (i >= nblk) break;
+                    if (i >= unit_next) {
+                        while (i >= unit_next && alive) { flush(); next_unit(); }
+                        lim = interior_limit();
+                    }
+                    const int bl = i - unit_first;
+                    const int rest = groups_total - 8 * (b_first + bl);
+                    const int jb = rest < 8 ? rest : 8;
+                    if (work && tw < jb) {
+                        const uint32_t sb = sbase + jj * kBlockBytes;
+                        const int tile = bl * 8 + tw;
+                        TileIn ta;
+                        tile_load<NT>(ta, sb + code_lane, sb + so_sect * jb + so_chunk, sb + 576u * jb + m_lane,
+                                      x_lane + tile * x_stride, xsc_lane + tile * xsc_stride);
+                        tile_compute<NT>(ta, acc, acc_m, lc);
+                    }
                 }
-                if (act1) {
-                    const int tile = bl1 * 8 + tw;
-                    tile_load<NT>(tb, sbase + kBlockBytes + code_lane, sbase + kBlockBytes + so_sect * jb1 + so_chunk,
-                                  sbase + kBlockBytes + 576u * jb1 + m_lane, x_lane + tile * x_stride,
-                                  xsc_lane + tile * xsc_stride);
-                }
-                if (act0) tile_compute<NT>(ta, acc, acc_m, lc);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8u * stage);
-                if (i1 < nblk) {
-                    if (cross && alive) { flush(); next_unit(); lim = interior_limit(); }
-                    if (act1) tile_compute<NT>(tb, acc, acc_m, lc);
-                }
             }
             if (++stage == nstage) { stage = 0; phase ^= 1u; }
         }
@@ -688,7 +693,7 @@ extern "C" __attribute__((visibility("default"))) int fdqp_trace_read(unsigned l
 
 // ---- host-visible launchers ------------------------------------------------------------------
 
-template <int CW, int NT>
+template <int CW, int NT, int BPW>
 static cudaError_t launch_one(const GemvPlan& p, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.Z * p.Gz));
@@ -696,11 +701,11 @@ static cudaError_t launch_one(const GemvPlan& p, cudaStream_t stream) {
     cfg.dynamicSmemBytes = p.smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may overlap the preparation kernel before it
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may overlap the launch before it (see the kernel)
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<CW, NT>, p);
+    return cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<CW, NT, BPW>, p);
 }
 
 cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream) {
@@ -718,17 +723,24 @@ cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int
                   : cudaLaunchKernelEx(&cfg, fdqp_xprep_kernel<false>, x, xq, xsc, M, K);
 }
 
+// consumer_warps: 8 or 16; p.bpw (blocks per warp per stage): 2, or 4 at M == 1
 cudaError_t gemv_launch(const GemvPlan& p, int consumer_warps, cudaStream_t stream) {
-    if (consumer_warps == 16) return p.M == 1 ? launch_one<16, 1>(p, stream) : launch_one<16, 2>(p, stream);
-    return p.M == 1 ? launch_one<8, 1>(p, stream) : launch_one<8, 2>(p, stream);
+    if (p.M == 1) {
+        if (consumer_warps == 16) return p.bpw == 4 ? launch_one<16, 1, 4>(p, stream) : launch_one<16, 1, 2>(p, stream);
+        return p.bpw == 4 ? launch_one<8, 1, 4>(p, stream) : launch_one<8, 1, 2>(p, stream);
+    }
+    return consumer_warps == 16 ? launch_one<16, 2, 2>(p, stream) : launch_one<8, 2, 2>(p, stream);
 }
 
 cudaError_t gemv_set_smem_limit(int bytes) {
     cudaError_t e;
-    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
-    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
-    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
-    return cudaFuncSetAttribute(fdqp_gemv_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    const cudaFuncAttribute a = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 1, 2>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 1, 4>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 1, 2>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 1, 4>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 2, 2>, a, bytes))) return e;
+    return cudaFuncSetAttribute(fdqp_gemv_kernel<16, 2, 2>, a, bytes);
 }
 
 }  // namespace fdqp

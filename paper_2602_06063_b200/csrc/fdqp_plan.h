@@ -30,7 +30,8 @@ struct GemvPlan {
     int Z;                // K slices
     int nbz;              // blocks per slice = ceil(nb / Z); every slice is non-empty
     int Gz;               // CTAs per slice; grid = Z * Gz
-    int nstage;           // ring depth in stages of (consumer warps / 4) blocks
+    int nstage;           // ring depth in stages of (consumer warps / 8) * bpw blocks
+    int bpw;              // blocks each consumer warp handles per stage (2 or 4)
     int evict_first;      // weight copies carry an evict-first L2 hint
     int strip_aligned;    // 1: CTA ranges are cut at strip boundaries (no strip is shared between CTAs of a slice)
     int prep_inline;      // 1: every CTA prepares its K slice of x itself; 0: a preparation kernel ran before

@@ -25,10 +25,10 @@ def ctx():
 @pytest.fixture()
 def fresh(ctx):
     """The shared context with every launch parameter back to automatic."""
-    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned"):
+    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp"):
         fd.fdqp_set_param(ctx, key, -1)
     yield ctx
-    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned"):
+    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp"):
         fd.fdqp_set_param(ctx, key, -1)
 
 
@@ -215,7 +215,7 @@ def test_batched_rows_match_single_row_calls(fresh):
 
 
 @pytest.mark.parametrize("key,values", [("split_k", [1, 2, 4, 8]), ("consumer_warps", [8, 16]), ("ctas_per_sm", [1, 2]),
-                                        ("stages", [2, 3, 7]), ("l2_evict_first", [0, 1]), ("prep_inline", [0, 1]), ("strip_aligned", [0, 1])])
+                                        ("stages", [2, 3, 7]), ("l2_evict_first", [0, 1]), ("prep_inline", [0, 1]), ("strip_aligned", [0, 1]), ("blocks_per_warp", [2, 4])])
 def test_launch_parameters_do_not_change_results(fresh, key, values):
     K, N, M = 4352, 2080, 3   # 17 blocks per strip, 65 strips: ragged against every split and grid
     case = Case(K, N, M, seed=90)
