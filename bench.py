@@ -257,6 +257,11 @@ def run_ours(args, rank, local_rank, world):
     # CUDA graphs: a decode step of the real model is 34 such layers back to back, so the layers are captured
     # LAYER_COPIES at a time (one pass over all resident weight copies per graph); single-layer graphs cover the
     # remainder when the step count is not a multiple of LAYER_COPIES.
+    # kernels one step launches (activation preparation and split-K sum kernels included, when the plan uses them)
+    count0 = fd.fdqp_launch_count(ctx)
+    enqueue_layer(0)
+    torch.cuda.synchronize()
+    kernels_per_step = fd.fdqp_launch_count(ctx) - count0
     graphs = None
     pass_graph = None
     if args.graph:
@@ -314,7 +319,6 @@ def run_ours(args, rank, local_rank, world):
     barrier()
     ms = ev0.elapsed_time(ev1)
     calls_per_step = len(shapes)
-    kernels_per_step = 2 * calls_per_step        # each call = activation preparation kernel + GEMV kernel
     launches = kernels_per_step * args.steps
     if graphs is None:
         assert fd.fdqp_launch_count(ctx) - launches_before == launches

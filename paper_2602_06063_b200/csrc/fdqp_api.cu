@@ -15,6 +15,7 @@
 namespace fdqp {
 cudaError_t gemv_launch(const GemvPlan& p, int consumer_warps, cudaStream_t stream);
 cudaError_t gemv_set_smem_limit(int bytes);
+cudaError_t splitk_sum_launch(const float* ws, float* y, int Z, int S, int M, int N, cudaStream_t stream);
 cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream);
 cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
 cudaError_t prefill_set_smem_limit();
@@ -160,7 +161,9 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
         const int Ga = Gz < p->S ? Gz : p->S;
         const int64_t blocks_al = (int64_t)((p->S + Ga - 1) / Ga) * nbz;
         const double cost_al = blocks_al * t_block + (Z > 1 ? 2.0 : 0.4);
-        const bool aligned = ctx->p_aligned >= 0 ? ctx->p_aligned != 0 : cost_al < cost_bal;
+        // K slices are always strip-aligned: every (slice, strip) then has one owner and the slices are added by a
+        // second small kernel instead of through arrival counters
+        const bool aligned = Z > 1 || (ctx->p_aligned >= 0 ? ctx->p_aligned != 0 : cost_al < cost_bal);
         p->strip_aligned = aligned ? 1 : 0;
         if (aligned) Gz = Ga;
     }
@@ -313,6 +316,11 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
         }
         if ((e = gemv_launch(plan, cw, stream))) return cuda_fail(ctx, e, "gemv kernel launch");
         ctx->launches += 1;
+        if (plan.Z > 1) {
+            if ((e = splitk_sum_launch(ctx->ws_full, plan.y, plan.Z, plan.S, mc, (int)N, stream)))
+                return cuda_fail(ctx, e, "split-K sum launch");
+            ctx->launches += 1;
+        }
     }
     return FDQP_OK;
 }

@@ -12,11 +12,10 @@
 // fp32 rate, so this unpack is the budget that matters), and the activations of a group are held as
 // 24-bit fixed point relative to the group's largest exponent, split into three byte planes
 // (x = 2^e_g * (65536 p2 + 256 p1 + p0), p2 signed, p1 and p0 unsigned; exact for every element
-// within 2^15 of the group's largest, rounded to 2^-23 of it otherwise).  One MMA covers a whole
+// within 2^14 of the group's largest, rounded to 2^-22 of it otherwise).  One MMA covers a whole
 // group of 16 output rows; its s32 result is exact.  The order of k inside a group is a free
 // permutation as long as both operands use the same one (even k in the low half, odd k in the high).
-// The three plane sums are turned into fp32 without a conversion instruction: the accumulator starts
-// at the bit pattern of 1.5 * 2^23, so the s32 result *is* the float 12582912 + sum.
+// The plane sums are recombined in int32 (they fit) and converted to fp32 once per value.
 // At M = 1 seven of the MMA's eight token columns would be idle, so the three planes of the single
 // token ride in columns 0, 1, 2 (as signed digits) and ONE MMA per 16 rows yields all three sums.
 //
@@ -107,7 +106,7 @@ __device__ __forceinline__ void xprep_item(const uint4 v, int M, int slot, int t
         psum += __shfl_xor_sync(0xffffffffu, psum, 2);
     }
     // exponent field of the group's largest magnitude, kept where both scale factors are normal floats
-    constexpr int kFrac = SINGLE ? 21 : 22;  // |fixed-point value| < 2^(kFrac + 1)
+    constexpr int kFrac = 21;  // |fixed-point value| < 2^22: the plane sums of a group recombine inside an int32
     int emax = (int)(amax >> 7);
     emax = emax < 24 ? 24 : (emax > 254 ? 254 : emax);
     const float to_fixed = __uint_as_float((uint32_t)(254 + kFrac - emax) << 23);  // 2^(127 + kFrac - emax)
@@ -178,8 +177,6 @@ __global__ void __launch_bounds__(128) fdqp_xprep_kernel(const uint16_t* __restr
 
 // ---- one 32 x 32 group-tile -------------------------------------------------------------------------
 
-constexpr int kMagicBits = 0x4B400000;  // bit pattern of 12582912.0f = 1.5 * 2^23
-constexpr float kMagic = 12582912.0f;
 
 struct TileIn {
     uint32_t c[4];   // code words: word q of rows g, g+8, g+16, g+24
@@ -217,16 +214,16 @@ __device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_
 
 template <bool B_SIGNED>
 __device__ __forceinline__ void imma(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                     uint32_t b1, int c = kMagicBits) {
-    const int kMagicBits = c;  // accumulator start value (shadows the constant on purpose)
+                                     uint32_t b1) {
+    const int zero = 0;  // accumulator start value
     if (B_SIGNED)
         asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
             : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
-            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(kMagicBits));
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(zero));
     else
         asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
             : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
-            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(kMagicBits));
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(zero));
 }
 
 // Per-lane constants of the single-token kernel: which two MMA columns the lane holds.
@@ -252,7 +249,7 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][NT
             const uint32_t e0 = w0 & 0x0F0F0F0Fu, o0 = (w0 >> 4) & 0x0F0F0F0Fu;  // even-k codes, odd-k codes
             const uint32_t e1 = w1 & 0x0F0F0F0Fu, o1 = (w1 >> 4) & 0x0F0F0F0Fu;
             int d[4];
-            imma<true>(d, e0, e1, o0, o1, t.b[0], t.b[1], 0);
+            imma<true>(d, e0, e1, o0, o1, t.b[0], t.b[1]);
             const float dq[2] = {bf16lo_mul_f32hi(t.so[h], uq), bf16hi_mul_f32hi(t.so[h], uq)};
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
@@ -280,9 +277,8 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][NT
 #pragma unroll
             for (int j = 0; j < NT; ++j) {
                 const int e = 2 * r + j;
-                const float s2 = __int_as_float(d2[e]) - kMagic, s1 = __int_as_float(d1[e]) - kMagic,
-                            s0 = __int_as_float(d0[e]) - kMagic;
-                const float s = fmaf(fmaf(s2, 256.f, s1), 256.f, s0);  // exact up to 2^24, else one rounding
+                // planes recombined in integers (|.| < 2^31), then one conversion (exact below 2^24, else one rounding)
+                const float s = __int2float_rn((d2[e] * 256 + d1[e]) * 256 + d0[e]);
                 const float dq = r == 0 ? bf16lo_mul_f32hi(t.so[h], t.sc[2 * j + 1])
                                         : bf16hi_mul_f32hi(t.so[h], t.sc[2 * j + 1]);
                 acc[i][j] = fmaf(dq, s, acc[i][j]);
@@ -632,7 +628,14 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
 
             const bool whole_unit = (pa == unit_begin) && (pe == unit_end);
             float* yrow = p.y + s * kStripRows + lane;
-            if (whole_unit && p.Z == 1) {
+            if (p.Z > 1) {
+                // K slices: ranges are strip-aligned, every (slice, strip) has one owner; the slices are added by
+                // fdqp_splitk_sum_kernel after this grid (fixed order, no arrival counters)
+                float* slot = p.ws_full + ((int64_t)z * p.S + s) * (kStripRows * kMaxTokens);
+#pragma unroll
+                for (int t = 0; t < kMaxTokens; ++t)
+                    if (t < M) slot[t * kStripRows + lane] = v[t];
+            } else if (whole_unit) {
 #pragma unroll
                 for (int t = 0; t < kMaxTokens; ++t)
                     if (t < M) yrow[(int64_t)t * p.N] = v[t];
@@ -685,6 +688,21 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
     }
 }
 
+// Second phase of a K-split projection: y[tok][n] = sum over slices z (ascending) of the slice partials.
+// ws is [Z][S][kMaxTokens][32]; one thread per (tok, n).
+__global__ void __launch_bounds__(256) fdqp_splitk_sum_kernel(const float* __restrict__ ws, float* __restrict__ y, int Z, int S,
+                                                               int M, int N) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the GEMV grid's partials
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (int64_t)M * N) return;
+    const int tok = (int)(idx / N), n = (int)(idx - (int64_t)tok * N);
+    const int s = n >> 5, r = n & 31;
+    float acc = 0.f;
+    for (int z = 0; z < Z; ++z) acc += ws[(((int64_t)z * S + s) * kMaxTokens + tok) * kStripRows + r];
+    y[idx] = acc;
+}
+
 #ifdef FDQP_TRACE
 extern "C" __attribute__((visibility("default"))) int fdqp_trace_read(unsigned long long* host, int n) {
     return (int)cudaMemcpyFromSymbol(host, g_fdqp_trace, sizeof(unsigned long long) * n);
@@ -721,6 +739,19 @@ cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int
     cfg.numAttrs = 1;
     return M == 1 ? cudaLaunchKernelEx(&cfg, fdqp_xprep_kernel<true>, x, xq, xsc, M, K)
                   : cudaLaunchKernelEx(&cfg, fdqp_xprep_kernel<false>, x, xq, xsc, M, K);
+}
+
+cudaError_t splitk_sum_launch(const float* ws, float* y, int Z, int S, int M, int N, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(((int64_t)M * N + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fdqp_splitk_sum_kernel, ws, y, Z, S, M, N);
 }
 
 // consumer_warps: 8 or 16; p.bpw (blocks per warp per stage): 2, or 4 at M == 1
