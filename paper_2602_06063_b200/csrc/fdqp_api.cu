@@ -99,7 +99,7 @@ SmemLayout smem_layout(const fdqp_ctx* ctx, int M, int nbz, int cw, int ctas_per
     L.stage_bytes = (uint32_t)(cw / 8) * (uint32_t)bpw * kBlockBytes;
     const uint32_t tiles = (uint32_t)nbz * 8u;
     L.xs_bytes = tiles * 128u * (uint32_t)M;          // prepared activations of the K slice
-    L.xsum_bytes = M == 1 ? 0u : tiles * 64u;         // per-token {sum x, unit}
+    L.xsum_bytes = M <= kColsMaxTokens ? 0u : tiles * 64u;         // per-token {sum x, unit} (plane mode only)
     L.part_bytes = 2u * (uint32_t)cw * kStripRows * (uint32_t)M * 4u;
     L.fixed = round_up(L.xs_bytes, 128) + round_up(L.xsum_bytes, 128) + round_up(L.part_bytes, 128) +
               (2u * kMaxStages + 5u) * 8u + 128u;
@@ -314,6 +314,12 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
                 return cuda_fail(ctx, e, "x preparation launch");
             ctx->launches += 1;
         }
+#ifdef FDQP_TRACE
+        {
+            static int trace_seq = 0;  // trace builds only: launch slot of the per-CTA timeline
+            plan.debug |= (trace_seq++ & 31) << 8;
+        }
+#endif
         if ((e = gemv_launch(plan, cw, stream))) return cuda_fail(ctx, e, "gemv kernel launch");
         ctx->launches += 1;
         if (plan.Z > 1) {
@@ -432,7 +438,7 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
     std::snprintf(buf, buf_bytes,
                   "%sfdqp_gemv_kernel<%d,%d> calls=%lld grid=%d block=%d smem=%u stages=%d split_k=%d ctas_per_slice=%d "
                   "evict_first=%d strip_aligned=%d blocks_per_warp=%d",
-                  plan.prep_inline ? "" : "fdqp_xprep_kernel + ", cw, mc == 1 ? 1 : 2, (long long)((M + kMaxTokens - 1) / kMaxTokens), plan.Z * plan.Gz, (cw + 1 + cw / 8) * 32,
+                  plan.prep_inline ? "" : "fdqp_xprep_kernel + ", cw, mc == 1 ? 1 : (mc > kColsMaxTokens ? 2 : (mc == 2 ? 3 : 1)), (long long)((M + kMaxTokens - 1) / kMaxTokens), plan.Z * plan.Gz, (cw + 1 + cw / 8) * 32,
                   plan.smem_bytes, plan.nstage, plan.Z, plan.Gz, plan.evict_first, plan.strip_aligned, plan.bpw);
     return FDQP_OK;
 }

@@ -16,8 +16,10 @@
 // group of 16 output rows; its s32 result is exact.  The order of k inside a group is a free
 // permutation as long as both operands use the same one (even k in the low half, odd k in the high).
 // The plane sums are recombined in int32 (they fit) and converted to fp32 once per value.
-// At M = 1 seven of the MMA's eight token columns would be idle, so the three planes of the single
-// token ride in columns 0, 1, 2 (as signed digits) and ONE MMA per 16 rows yields all three sums.
+// For M <= 4 most of the MMA's eight token columns would be idle, so the three planes of a token ride in
+// three columns (as signed digits; column 3 / 7 is zero): one MMA per 16 rows yields all three plane sums
+// of up to TWO tokens (kernel modes: 1 = one token, 3 = two tokens).  Mode 2 (M = 3..8) issues one MMA per plane
+// with the eight tokens as columns; measured on B200 it beats two column-mode MMAs from M = 3 on.
 //
 // The plane split of x is done once per call by a small preparation kernel; every GEMV CTA then
 // brings its K slice of the prepared x into shared memory with bulk async copies.
@@ -58,8 +60,9 @@ __device__ __forceinline__ float* piece_slot(const GemvPlan& p, int z, int64_t c
 }
 
 #ifdef FDQP_TRACE
-__device__ unsigned long long g_fdqp_trace[1024 * 8];
-#define FDQP_STAMP(i) do { if (lane == 0) g_fdqp_trace[(blockIdx.x & 1023) * 8 + (i)] = globaltimer_ns(); } while (0)
+// 32 launch slots (plan.debug bits 8..12) x 256 CTAs x 16 stamps
+__device__ unsigned long long g_fdqp_trace[32 * 256 * 16];
+#define FDQP_STAMP(i) do { if (lane == 0) g_fdqp_trace[(((p.debug >> 8) & 31) * 256 + (blockIdx.x & 255)) * 16 + (i)] = globaltimer_ns(); } while (0)
 #else
 #define FDQP_STAMP(i) do { } while (0)
 #endif
@@ -70,11 +73,12 @@ __device__ unsigned long long g_fdqp_trace[1024 * 8];
 // relative to the largest exponent of the 32-group and split into byte planes in MMA fragment order
 // ({bytes of even k, bytes of odd k} per plane).
 //
-// M >= 2 (SINGLE == false): 24-bit fixed point, planes 2 (signed), 1, 0 (unsigned).  Record of 32 bytes at
+// M >= 3 (SINGLE == false): 23-bit fixed point, planes 2 (signed), 1, 0 (unsigned).  Record of 32 bytes at
 //   xq[((T*M + tok)*4 + q)*32]: words 0..5 = planes 2, 1, 0; words 6, 7 = {sum of the group's x, unit 2^e_g};
 //   and xsc[T*16 + (tok/2)*4 + (tok%2)*2 + {0,1}] holds the same two scalars indexed by token.
-// M == 1 (SINGLE == true): 23-bit fixed point in three SIGNED digits.  Per tile 128 bytes:
-//   [plane 2: 4 x 8 B by q][plane 1][plane 0][{sum x, unit}][24 zero bytes].
+// M <= 2 (SINGLE == true, "column" layout): 23-bit fixed point in three SIGNED digits.  Per (tile, token) 128 bytes:
+//   [plane 2: 4 x 8 B by q][plane 1][plane 0][{sum x, unit}][8 zero bytes][16 bytes: see next line];
+//   the last 16 bytes of TOKEN 0's record start with the group sums of x of tokens 0 and 1 of that tile.
 // `tile` is the group-tile index in x, `slot` the tile's index in the destination (global: the same; shared
 // memory: relative to the CTA's K slice).  Must be called by whole quads (the four q of a (tile, token)).
 __device__ __forceinline__ uint4 xprep_load(const uint16_t* __restrict__ x, int K, int tile, int tok, int q, bool valid) {
@@ -140,13 +144,13 @@ __device__ __forceinline__ void xprep_item(const uint4 v, int M, int slot, int t
     }
     if (!valid) return;
     if (SINGLE) {
-        uint32_t* rec = xq + (int64_t)slot * 32;  // 128 bytes per tile
+        uint32_t* rec = xq + ((int64_t)slot * M + tok) * 32;  // 128 bytes per (tile, token)
 #pragma unroll
         for (int pl = 0; pl < 3; ++pl)
             *reinterpret_cast<uint2*>(rec + pl * 8 + q * 2) = make_uint2(plane[pl][0], plane[pl][1]);
         if (q == 0) *reinterpret_cast<uint2*>(rec + 24) = make_uint2(__float_as_uint(psum), __float_as_uint(unit));
         if (q == 1) *reinterpret_cast<uint2*>(rec + 26) = make_uint2(0u, 0u);
-        if (q == 2) *reinterpret_cast<uint4*>(rec + 28) = make_uint4(0u, 0u, 0u, 0u);
+        if (q == 2) xq[(int64_t)slot * M * 32 + 28 + tok] = __float_as_uint(psum);
     } else {
         uint4* dst = reinterpret_cast<uint4*>(xq + ((int64_t)(slot * M + tok) * 4 + q) * 8);
         dst[0] = make_uint4(plane[0][0], plane[0][1], plane[1][0], plane[1][1]);
@@ -178,37 +182,63 @@ __global__ void __launch_bounds__(128) fdqp_xprep_kernel(const uint16_t* __restr
 // ---- one 32 x 32 group-tile -------------------------------------------------------------------------
 
 
-struct TileIn {
-    uint32_t c[4];   // code words: word q of rows g, g+8, g+16, g+24
-    uint32_t so[4];  // (d[g], d[g+8]), (d[g+16], d[g+24]), (m[g], m[g+8]), (m[g+16], m[g+24]) as bf16 pairs
-    uint32_t b[6];   // B fragments {even k, odd k}: planes 2, 1, 0 (NT == 2) or this lane's column (NT == 1)
-    float sc[4];     // {sum x, unit} of token 2q and of token 2q+1 (NT == 2) or of the only token (NT == 1)
-    uint32_t m_row;  // NT == 1: bf16 offset of row `lane` (low half)
+// Kernel modes (see the header comment): derived constants.
+template <int MODE>
+struct ModeTraits {
+    static constexpr bool kCols = MODE != 2;     // planes as MMA columns (M <= kColsMaxTokens)
+    static constexpr int kAcc = kCols ? 1 : 2;   // accumulator columns per lane
+    static constexpr bool kXRow = MODE == 3;     // offset term needs the sums of x of both tokens
+    static constexpr int kAccM = MODE == 3 ? 2 : 1;
 };
 
-// NT == 1: so_addr addresses the scale chunks only (lanes 0..15 matter) and m_addr this lane's own offset word.
-template <int NT>
-__device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_t so_addr, uint32_t m_addr, uint32_t x_addr,
-                                          uint32_t xsc_addr) {
+struct TileIn {
+    uint32_t c[4];   // code words: word q of rows g, g+8, g+16, g+24
+    uint32_t so[4];  // column modes: (d[g], d[g+8]), (d[g+16], d[g+24]); mode 2 also (m[g], m[g+8]), (m[g+16], m[g+24])
+    uint32_t b[6];   // B fragments {even k, odd k}: mode 2: planes 2, 1, 0; column modes: this lane's column
+    float sc[4];     // mode 2: {sum x, unit} of tokens 2q, 2q+1; column modes: {sum x, unit} of the lane's token
+    float xrow[2];   // mode 3: sum of x of tokens 0, 1 for this group
+    uint32_t m_row;  // column modes: bf16 offset of row `lane` (low half)
+};
+
+// Per-lane pieces of the shared-memory addresses of the prepared activations.
+struct LaneAddr {
+    uint32_t xs, x_stride;   // base and bytes per tile of the prepared-x records
+    uint32_t xb_off;         // column modes: this lane's B column inside the tile
+    uint32_t sc_off;         // column modes: {sum x, unit} of the token whose columns this lane accumulates
+    uint32_t x_lane, xsc_lane;  // mode 2: this lane's record / scalar quad inside tile 0
+};
+
+// Column modes: so_addr addresses the scale chunks only (lanes 0..15 matter); m_addr is this lane's own offset word.
+template <int MODE>
+__device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_t so_addr, uint32_t m_addr, int tile,
+                                          const LaneAddr& la) {
+    using T = ModeTraits<MODE>;
     ldmatrix_x4(t.c, code_addr);
-    if (NT == 1) {
+    if (T::kCols) {
         uint32_t dd[2];
         ldmatrix_x2_trans(dd, so_addr);
         t.so[0] = dd[0];
         t.so[1] = dd[1];
         asm volatile("ld.shared.u16 %0, [%1];" : "=r"(t.m_row) : "r"(m_addr));
-        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(t.b[0]), "=r"(t.b[1]) : "r"(x_addr));
-        const float2 v = lds64f(xsc_addr);
+        const uint32_t tb = la.xs + (uint32_t)tile * la.x_stride;
+        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(t.b[0]), "=r"(t.b[1]) : "r"(tb + la.xb_off));
+        const float2 v = lds64f(tb + la.sc_off);
         t.sc[0] = v.x;
         t.sc[1] = v.y;
+        if (T::kXRow) {
+            const float2 xr = lds64f(tb + 112u);
+            t.xrow[0] = xr.x;
+            t.xrow[1] = xr.y;
+        }
     } else {
         ldmatrix_x4_trans(t.so, so_addr);
+        const uint32_t x_addr = la.x_lane + (uint32_t)tile * la.x_stride;
         const uint4 r0 = lds128(x_addr);
         t.b[0] = r0.x; t.b[1] = r0.y; t.b[2] = r0.z; t.b[3] = r0.w;
         asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(t.b[4]), "=r"(t.b[5]) : "r"(x_addr + 16));
         asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
                      : "=f"(t.sc[0]), "=f"(t.sc[1]), "=f"(t.sc[2]), "=f"(t.sc[3])
-                     : "r"(xsc_addr));
+                     : "r"(la.xsc_lane + (uint32_t)tile * 64u));
     }
 }
 
@@ -226,23 +256,30 @@ __device__ __forceinline__ void imma(int (&d)[4], uint32_t a0, uint32_t a1, uint
             : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(zero));
 }
 
-// Per-lane constants of the single-token kernel: which two MMA columns the lane holds.
-//   q == 0: columns (plane 2, plane 1) -> 256 * s2 + s1, weighted 256 * unit, and the lane adds m * sum x
-//   q == 1: columns (plane 0, zero)    -> s0, weighted unit
-//   q >= 2: zero columns
+// Per-lane constants of the column modes: which two MMA columns the lane holds.  Columns 4*(tok%2) + {0,1,2} are
+// planes 2, 1, 0 of token tok (of the pair), column 3 / 7 is zero; lane q holds columns 2q, 2q+1:
+//   q even: (plane 2, plane 1) -> 256 * s2 + s1, weighted 256 * unit;   q odd: (plane 0, zero) -> s0, weighted unit.
 struct LaneConst {
-    int k_first;    // weight of the first column relative to the second (256 or 1)
-    float w_unit;   // factor on `unit`
+    int k_first;       // weight of the first column relative to the second (256 or 1)
+    float w_unit;      // factor on `unit` (0 when the lane's token does not exist)
 };
 
-// acc[row][tok] += d * unit * (sum_k q_k X_k) + m * (sum_k x_k), fp32 (Eq. 3 applied per group).
+// acc[row][.] += d * unit * (sum_k q_k X_k) + m * (sum_k x_k), fp32 (Eq. 3 applied per group).
 // `unit` (and 256 * unit) are powers of two, so d * unit is formed exactly by the mixed bf16 FMA.
-// acc_m (NT == 1 only): this lane's row (row = lane) of sum_g m_g * X_g; the offset term does not need the MMA layout.
-template <int NT>
-__device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][NT], float& acc_m, const LaneConst& lc) {
-    if (NT == 1) {
+// Column modes keep the offset term sum_g m_g * X_g in a lane-per-row layout (acc_m[tok], row = lane).
+template <int MODE>
+__device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][ModeTraits<MODE>::kAcc],
+                                             float (&acc_m)[ModeTraits<MODE>::kAccM], const LaneConst& lc) {
+    using T = ModeTraits<MODE>;
+    if (T::kCols) {
+        const float mw = bf16lo_mul_f32hi(t.m_row, 1.0f);
+        if (T::kXRow) {
+#pragma unroll
+            for (int tk = 0; tk < T::kAccM; ++tk) acc_m[tk] = fmaf(mw, t.xrow[tk], acc_m[tk]);
+        } else {
+            acc_m[0] = fmaf(mw, t.sc[0], acc_m[0]);
+        }
         const float uq = t.sc[1] * lc.w_unit;
-        acc_m = fmaf(bf16lo_mul_f32hi(t.m_row, 1.0f), t.sc[0], acc_m);
 #pragma unroll
         for (int h = 0; h < 2; ++h) {  // rows (g, g+8) then (g+16, g+24)
             const uint32_t w0 = t.c[2 * h], w1 = t.c[2 * h + 1];
@@ -275,7 +312,7 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][NT
         for (int r = 0; r < 2; ++r) {
             const int i = 2 * h + r;
 #pragma unroll
-            for (int j = 0; j < NT; ++j) {
+            for (int j = 0; j < 2; ++j) {
                 const int e = 2 * r + j;
                 // planes recombined in integers (|.| < 2^31), then one conversion (exact below 2^24, else one rounding)
                 const float s = __int2float_rn((d2[e] * 256 + d1[e]) * 256 + d0[e]);
@@ -288,19 +325,21 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][NT
     }
 }
 
-// CW consumer warps (8 or 16); NT token columns kept per lane (1 when M == 1, else 2).
+// CW consumer warps (8 or 16); MODE as above (1: M = 1, 3: M = 2, 2: M = 3..8).
 // A ring stage holds CB = (CW / 8) * BPW blocks; warp w owns group-tile (w & 7) of the BPW (2 or 4) consecutive
 // blocks starting at BPW * (w >> 3) of every stage.  More blocks per stage = fewer barrier round trips per tile.
 // Warps CW+1 .. CW+NR are reducers (NR = CW / 8): reducer r completes the strip pieces with piece % NR == r.
-template <int CW, int NT, int BPW>
+template <int CW, int MODE, int BPW>
 __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
     fdqp_gemv_kernel(const __grid_constant__ GemvPlan p) {
     extern __shared__ __align__(128) uint8_t smem[];
+    using MT = ModeTraits<MODE>;
+    constexpr int NT = MT::kAcc;
     constexpr int CB = (CW / 8) * BPW;
     constexpr int NR = CW / 8;
     constexpr uint32_t kStageBytes = CB * kBlockBytes;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int M = p.M, K = p.K;
+    const int M = MODE == 1 ? 1 : (MODE == 3 ? 2 : p.M), K = p.K;  // compile-time in the column modes
 
     const int z = blockIdx.x / p.Gz;
     const int64_t ci = blockIdx.x % p.Gz;
@@ -408,26 +447,35 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         // =============================== consumers ===============================================
         const int tw = warp & 7, j0 = (warp >> 3) * BPW;
         const int g = lane >> 2, q = lane & 3;
-        // B fragments.  NT == 2: column g is token g (any valid token for unused columns: their results are
-        // never stored).  NT == 1: column g < 3 is plane 2 - g of the only token, other columns read zeros.
-        const int gtok = g < M ? g : M - 1;
-        const uint32_t x_lane = (NT == 1) ? xs + (g < 3 ? (uint32_t)(g * 32 + q * 8) : 104u)
-                                          : xs + (uint32_t)(gtok * 4 + q) * 32u;
-        const uint32_t x_stride = (uint32_t)M * 128u;
-        const uint32_t xsc_lane = (NT == 1) ? xs + 96u : xsc + q * 16;
-        const uint32_t xsc_stride = (NT == 1) ? 128u : 64u;
+        // B fragments.  Mode 2: column g is token g (any valid token for unused columns: their results are never
+        // stored).  Column modes: column g is plane 2 - g%4 of token g/4 (zeros for g%4 == 3 and for a token that
+        // does not exist); this lane accumulates the columns of token q/2.
+        LaneAddr la;
         LaneConst lc;
-        lc.k_first = q == 0 ? 256 : 1;
-        lc.w_unit = q == 0 ? 256.f : (q == 1 ? 1.f : 0.f);
-        float acc_m = 0.f;  // NT == 1: offset term of row `lane`
+        la.xs = xs;
+        la.x_stride = (uint32_t)M * 128u;
+        {
+            const int gtok = g < M ? g : M - 1;
+            la.x_lane = xs + (uint32_t)(gtok * 4 + q) * 32u;
+            la.xsc_lane = xsc + q * 16;
+            lc.k_first = (q & 1) ? 1 : 256;
+            const int tok_b = g >> 2, pl = g & 3;
+            la.xb_off = (tok_b < M && pl < 3) ? (uint32_t)(tok_b * 128 + pl * 32 + q * 8) : 104u;
+            const int tok_d = q >> 1;
+            la.sc_off = (uint32_t)((tok_d < M ? tok_d : 0) * 128 + 96);
+            lc.w_unit = tok_d < M ? ((q & 1) ? 1.f : 256.f) : 0.f;
+        }
+        float acc_m[MT::kAccM];  // column modes: offset term of row `lane`, per token
+#pragma unroll
+        for (int tk = 0; tk < MT::kAccM; ++tk) acc_m[tk] = 0.f;
         // ldmatrix source rows: codes = row `lane` of the tile; scales/offsets = the four 16-byte
         // chunks of this tile's scale words and of its offset words, duplicated so that after the
         // transposed load every lane of a quad holds (d[g], d[g+8]), (d[g+16], d[g+24]), (m..), (m..)
         const uint32_t code_lane = tw * 512 + lane * 16;
         const int mat = lane >> 3;
         const uint32_t so_chunk = tw * 64 + (((mat & 1) * 2 + (lane & 1)) * 16);
-        const uint32_t so_sect = (NT == 2 && mat >= 2) ? 576u : 512u;  // offsets section follows the scales section
-        const uint32_t m_lane = tw * 64 + lane * 2;                      // NT == 1: this lane's own offset word
+        const uint32_t so_sect = (!MT::kCols && mat >= 2) ? 576u : 512u;  // offsets section follows the scales section
+        const uint32_t m_lane = tw * 64 + lane * 2;                         // column modes: this lane's own offset word
 
         float acc[4][NT];
 #pragma unroll
@@ -439,13 +487,17 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         bool alive = true;
         // hand the warp's partial rows of the current strip piece to the reducer warp
         auto flush = [&]() {
-            if (NT == 1) {  // lanes q == 0 and q == 1 hold the two halves of each row's sum; lane r holds row r's offsets
+            if (MT::kCols) {
+                // lanes q and q^1 hold the two halves of each row's sum for token q/2; lane r holds row r's offset terms
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     acc[i][0] += __shfl_xor_sync(0xffffffffu, acc[i][0], 1);
-                    acc[i][0] += __shfl_sync(0xffffffffu, acc_m, g + 8 * i);
+                    const float m0 = __shfl_sync(0xffffffffu, acc_m[0], g + 8 * i);
+                    const float m1 = MT::kAccM == 1 ? 0.f : __shfl_sync(0xffffffffu, acc_m[MT::kAccM - 1], g + 8 * i);
+                    acc[i][0] += (q >> 1) ? m1 : m0;
                 }
-                acc_m = 0.f;
+#pragma unroll
+                for (int tk = 0; tk < MT::kAccM; ++tk) acc_m[tk] = 0.f;
             }
             const int par = piece & 1;
             if (piece >= 2 && !mbar_wait(red_empty0 + 8u * par, ((piece >> 1) - 1) & 1, p.status)) alive = false;
@@ -454,8 +506,9 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int j = 0; j < NT; ++j) {
-                    const int tok = 2 * q + j;
-                    if (tok < M)
+                    // column modes: the accumulator is token q/2, complete in the lanes with even q
+                    const int tok = MT::kCols ? (q >> 1) : 2 * q + j;
+                    if (tok < M && (!MT::kCols || (q & 1) == 0))
                         asm volatile("st.shared.f32 [%0], %1;" ::"r"(slot + (uint32_t)(tok * kStripRows + g + 8 * i) * 4u),
                                      "f"(acc[i][j])
                                      : "memory");
@@ -479,6 +532,7 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
 
         // Everything up to here touched only this CTA's shared memory.  x may come from the previous launch.
         asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (warp == 0) FDQP_STAMP(6);
         if (p.prep_inline) {
             // prepare this CTA's K slice of x straight into shared memory (cheap, and the first weights are still
             // on their way from HBM)
@@ -498,16 +552,21 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                     const int tm = idx >> 2;
                     v[u] = xprep_load(p.x, K, tile0 + (valid ? tm / M : 0), valid ? tm % M : 0, idx & 3, valid);
                 }
+#ifdef FDQP_TRACE
+                asm volatile("" ::"r"(v[0].x), "r"(v[kBatch - 1].x));
+                if (warp == 0 && base == 0) FDQP_STAMP(8);
+#endif
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
                     const int idx = base + u * CW * 32 + tid;
                     if (base + u * CW * 32 < items) {  // warp-uniform: whole quads run the shuffles together
                         const bool valid = idx < items;
                         const int tm = idx >> 2;
-                        xprep_item<NT == 1>(v[u], M, valid ? tm / M : 0, valid ? tm % M : 0, idx & 3, valid, xs_g, xsc_g);
+                        xprep_item<MT::kCols>(v[u], M, valid ? tm / M : 0, valid ? tm % M : 0, idx & 3, valid, xs_g, xsc_g);
                     }
                 }
             }
+            if (warp == 0) FDQP_STAMP(9);
             asm volatile("bar.sync 1, %0;" ::"n"(CW * 32) : "memory");
         } else if (!mbar_wait(x_bar, 0, p.status)) {
             alive = false;
@@ -533,23 +592,20 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             const uint32_t sbase = ring + stage * kStageBytes + j0 * kBlockBytes;
             if (i0 + BPW - 1 < lim) {
                 const int tile = (i0 - unit_first) * 8 + tw;
-                const uint32_t xa = x_lane + tile * x_stride, sa = xsc_lane + tile * xsc_stride;
 #pragma unroll
                 for (int pr = 0; pr < BPW / 2; ++pr) {  // two tiles in flight at a time
                     const uint32_t sb = sbase + pr * 2 * kBlockBytes;
                     TileIn ta, tb;
-                    tile_load<NT>(ta, sb + code_lane, sb + so_lane8, sb + 576u * 8u + m_lane, xa + (16 * pr) * x_stride,
-                                  sa + (16 * pr) * xsc_stride);
-                    tile_load<NT>(tb, sb + kBlockBytes + code_lane, sb + kBlockBytes + so_lane8,
-                                  sb + kBlockBytes + 576u * 8u + m_lane, xa + (16 * pr + 8) * x_stride,
-                                  sa + (16 * pr + 8) * xsc_stride);
-                    tile_compute<NT>(ta, acc, acc_m, lc);
+                    tile_load<MODE>(ta, sb + code_lane, sb + so_lane8, sb + 576u * 8u + m_lane, tile + 16 * pr, la);
+                    tile_load<MODE>(tb, sb + kBlockBytes + code_lane, sb + kBlockBytes + so_lane8,
+                                    sb + kBlockBytes + 576u * 8u + m_lane, tile + 16 * pr + 8, la);
+                    tile_compute<MODE>(ta, acc, acc_m, lc);
                     if (pr == BPW / 2 - 1) {
                         // every shared-memory read of this stage has been issued and consumed in order: hand it back
                         __syncwarp();
                         if (lane == 0) mbar_arrive(empty0 + 8u * stage);
                     }
-                    tile_compute<NT>(tb, acc, acc_m, lc);
+                    tile_compute<MODE>(tb, acc, acc_m, lc);
                 }
             } else {
                 // general stage (range end, strip boundary, short last block): one block at a time
@@ -567,9 +623,8 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                         const uint32_t sb = sbase + jj * kBlockBytes;
                         const int tile = bl * 8 + tw;
                         TileIn ta;
-                        tile_load<NT>(ta, sb + code_lane, sb + so_sect * jb + so_chunk, sb + 576u * jb + m_lane,
-                                      x_lane + tile * x_stride, xsc_lane + tile * xsc_stride);
-                        tile_compute<NT>(ta, acc, acc_m, lc);
+                        tile_load<MODE>(ta, sb + code_lane, sb + so_sect * jb + so_chunk, sb + 576u * jb + m_lane, tile, la);
+                        tile_compute<MODE>(ta, acc, acc_m, lc);
                     }
                 }
                 __syncwarp();
@@ -584,19 +639,22 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         // The prepared activations of this CTA's K slice: one barrier, a few large copies.  They are written by
         // the preparation kernel this launch may overlap with, hence the dependency wait first.
         asm volatile("griddepcontrol.wait;" ::: "memory");  // before any global write of this grid
+#ifdef FDQP_TRACE
+        if (warp == CW + 1) { mbar_wait(full0, 0, p.status); FDQP_STAMP(7); }
+#endif
         if (warp == CW + 1 && lane == 0 && !p.prep_inline) {
             const int kbeg = b_first * kBlockK;
             const int kend_full = (b_first + len) * kBlockK;
             const int kend = kend_full < K ? kend_full : K;
             const uint32_t tile0 = (uint32_t)(kbeg / kGroup), ntiles = (uint32_t)((kend - kbeg) / kGroup);
-            const uint32_t rec_bytes = ntiles * (uint32_t)M * 128u, sc_bytes = (NT == 2) ? ntiles * 64u : 0u;
+            const uint32_t rec_bytes = ntiles * (uint32_t)M * 128u, sc_bytes = MT::kCols ? 0u : ntiles * 64u;
             mbar_arrive_expect_tx(x_bar, rec_bytes + sc_bytes);
             const uint8_t* src = reinterpret_cast<const uint8_t*>(p.xq) + (size_t)tile0 * M * 128u;
             for (uint32_t off = 0; off < rec_bytes; off += 32768u) {
                 const uint32_t n = rec_bytes - off < 32768u ? rec_bytes - off : 32768u;
                 bulk_g2s(xs + off, src + off, n, x_bar);
             }
-            if constexpr (NT == 2) {
+            if constexpr (!MT::kCols) {
                 const uint8_t* s2 = reinterpret_cast<const uint8_t*>(p.xsc) + (size_t)tile0 * 64u;
                 for (uint32_t off = 0; off < sc_bytes; off += 32768u) {
                     const uint32_t n = sc_bytes - off < 32768u ? sc_bytes - off : 32768u;
@@ -711,7 +769,7 @@ extern "C" __attribute__((visibility("default"))) int fdqp_trace_read(unsigned l
 
 // ---- host-visible launchers ------------------------------------------------------------------
 
-template <int CW, int NT, int BPW>
+template <int CW, int MODE, int BPW>
 static cudaError_t launch_one(const GemvPlan& p, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.Z * p.Gz));
@@ -723,7 +781,7 @@ static cudaError_t launch_one(const GemvPlan& p, cudaStream_t stream) {
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<CW, NT, BPW>, p);
+    return cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<CW, MODE, BPW>, p);
 }
 
 cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream) {
@@ -737,7 +795,7 @@ cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return M == 1 ? cudaLaunchKernelEx(&cfg, fdqp_xprep_kernel<true>, x, xq, xsc, M, K)
+    return M <= kColsMaxTokens ? cudaLaunchKernelEx(&cfg, fdqp_xprep_kernel<true>, x, xq, xsc, M, K)
                   : cudaLaunchKernelEx(&cfg, fdqp_xprep_kernel<false>, x, xq, xsc, M, K);
 }
 
@@ -754,13 +812,15 @@ cudaError_t splitk_sum_launch(const float* ws, float* y, int Z, int S, int M, in
     return cudaLaunchKernelEx(&cfg, fdqp_splitk_sum_kernel, ws, y, Z, S, M, N);
 }
 
-// consumer_warps: 8 or 16; p.bpw (blocks per warp per stage): 2, or 4 at M == 1
+// consumer_warps: 8 or 16; p.bpw (blocks per warp per stage): 2, or 4 at M == 1.  Kernel mode by M (see the header).
 cudaError_t gemv_launch(const GemvPlan& p, int consumer_warps, cudaStream_t stream) {
+    const bool w16 = consumer_warps == 16;
     if (p.M == 1) {
-        if (consumer_warps == 16) return p.bpw == 4 ? launch_one<16, 1, 4>(p, stream) : launch_one<16, 1, 2>(p, stream);
+        if (w16) return p.bpw == 4 ? launch_one<16, 1, 4>(p, stream) : launch_one<16, 1, 2>(p, stream);
         return p.bpw == 4 ? launch_one<8, 1, 4>(p, stream) : launch_one<8, 1, 2>(p, stream);
     }
-    return consumer_warps == 16 ? launch_one<16, 2, 2>(p, stream) : launch_one<8, 2, 2>(p, stream);
+    if (p.M > kColsMaxTokens) return w16 ? launch_one<16, 2, 2>(p, stream) : launch_one<8, 2, 2>(p, stream);
+    return w16 ? launch_one<16, 3, 2>(p, stream) : launch_one<8, 3, 2>(p, stream);
 }
 
 cudaError_t gemv_set_smem_limit(int bytes) {
@@ -770,6 +830,8 @@ cudaError_t gemv_set_smem_limit(int bytes) {
     if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 1, 4>, a, bytes))) return e;
     if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 1, 2>, a, bytes))) return e;
     if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 1, 4>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 3, 2>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 3, 2>, a, bytes))) return e;
     if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 2, 2>, a, bytes))) return e;
     return cudaFuncSetAttribute(fdqp_gemv_kernel<16, 2, 2>, a, bytes);
 }

@@ -11,6 +11,8 @@ constexpr int kBlockK = 256;        // input features per full Q4NX block
 constexpr int kBlockBytes = 5120;   // bytes of a full block (Sec. "Dequantization Engine")
 constexpr int kGroupBytes = 640;    // bytes a block spends per group: 512 codes + 64 scales + 64 offsets
 constexpr int kMaxTokens = 8;       // token rows one GEMV launch handles
+// Up to this many tokens the GEMV lays the byte planes of a token out as MMA columns; above it, one MMA per plane.
+constexpr int kColsMaxTokens = 2;
 constexpr int kMaxSplit = 8;        // K slices
 constexpr int kMaxCtasPerSm = 2;
 
