@@ -42,9 +42,20 @@
 
 namespace fdqp {
 
-__device__ __forceinline__ int64_t range_begin(int64_t ci, int64_t G, int64_t T) { return (ci * T) / G; }
+// 32-bit arithmetic is exact (and an order of magnitude cheaper than a 64-bit division) while (G + 1)(T + 1) < 2^32.
+__device__ __forceinline__ bool fits32(int64_t G, int64_t T) { return (((uint64_t)(G + 1) * (uint64_t)(T + 1)) >> 32) == 0; }
+__device__ __forceinline__ int64_t div_floor(int64_t a, int64_t b, bool small) {
+    return small ? (int64_t)((uint32_t)a / (uint32_t)b) : a / b;
+}
+__device__ __forceinline__ int64_t range_begin(int64_t ci, int64_t G, int64_t T) {
+    if (fits32(G, T)) return (int64_t)(((uint32_t)ci * (uint32_t)T) / (uint32_t)G);
+    return (ci * T) / G;
+}
 // index of the CTA whose range [range_begin(ci), range_begin(ci+1)) contains L
-__device__ __forceinline__ int64_t cta_of(int64_t L, int64_t G, int64_t T) { return ((L + 1) * G - 1) / T; }
+__device__ __forceinline__ int64_t cta_of(int64_t L, int64_t G, int64_t T) {
+    if (fits32(G, T)) return (int64_t)((((uint32_t)L + 1u) * (uint32_t)G - 1u) / (uint32_t)T);
+    return ((L + 1) * G - 1) / T;
+}
 
 __device__ __forceinline__ int slice_len(const GemvPlan& p, int z) {
     const int rest = p.nb - z * p.nbz;
@@ -90,55 +101,43 @@ __device__ __forceinline__ uint4 xprep_load(const uint16_t* __restrict__ x, int 
 template <bool SINGLE>
 __device__ __forceinline__ void xprep_item(const uint4 v, int M, int slot, int tok, int q, bool valid,
                                            uint32_t* __restrict__ xq, float* __restrict__ xsc) {
-    const uint32_t h[8] = {v.x & 0xffffu, v.x >> 16, v.y & 0xffffu, v.y >> 16,
-                           v.z & 0xffffu, v.z >> 16, v.w & 0xffffu, v.w >> 16};
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     float f[8];
-    uint32_t amax = 0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        f[i] = __uint_as_float(h[i] << 16);
-        const uint32_t mag = h[i] & 0x7fffu;
-        amax = mag > amax ? mag : amax;
+    for (int i = 0; i < 4; ++i) {
+        f[2 * i] = __uint_as_float(w[i] << 16);
+        f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
     }
+    float amax = fmaxf(fmaxf(fmaxf(fabsf(f[0]), fabsf(f[1])), fmaxf(fabsf(f[2]), fabsf(f[3]))),
+                       fmaxf(fmaxf(fabsf(f[4]), fabsf(f[5])), fmaxf(fabsf(f[6]), fabsf(f[7]))));
     float psum = ((f[0] + f[1]) + (f[2] + f[3])) + ((f[4] + f[5]) + (f[6] + f[7]));
-    {
-        uint32_t o = __shfl_xor_sync(0xffffffffu, amax, 1);
-        amax = o > amax ? o : amax;
-        o = __shfl_xor_sync(0xffffffffu, amax, 2);
-        amax = o > amax ? o : amax;
-        psum += __shfl_xor_sync(0xffffffffu, psum, 1);
-        psum += __shfl_xor_sync(0xffffffffu, psum, 2);
-    }
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+    psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+    psum += __shfl_xor_sync(0xffffffffu, psum, 2);
     // exponent field of the group's largest magnitude, kept where both scale factors are normal floats
-    constexpr int kFrac = 21;  // |fixed-point value| < 2^22: the plane sums of a group recombine inside an int32
-    int emax = (int)(amax >> 7);
+    constexpr int kFrac = 21;  // |fixed-point value| <= 2^22: the plane sums of a group recombine inside an int32
+    int emax = (int)(__float_as_uint(amax) >> 23);
     emax = emax < 24 ? 24 : (emax > 254 ? 254 : emax);
     const float to_fixed = __uint_as_float((uint32_t)(254 + kFrac - emax) << 23);  // 2^(127 + kFrac - emax)
     const float unit = __uint_as_float((uint32_t)(emax - kFrac) << 23);            // 2^(emax - 127 - kFrac)
-    int I[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) I[i] = __float2int_rn(f[i] * to_fixed);
-    uint32_t plane[3][2];  // [0] most significant; {even k, odd k}
-    int D[3][8];
+    // Round to the nearest integer I (ties to even) by adding 1.5 * 2^23: the sum's low mantissa bits are 2^22 + I.
+    // Column layout: bytes 0..2 of (I + 0x808080) ^ 0x808080 are the signed digits of I in base 256
+    // (I = 65536 d2 + 256 d1 + d0, each in [-128, 127]); plane layout: the two's-complement bytes of I themselves
+    // (top byte signed, lower bytes unsigned).
+    constexpr uint32_t kMagicBits = 0x4B400000u;  // bits of 12582912.0f
+    uint32_t J[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        if (SINGLE) {  // signed digits: I = 65536 d2 + 256 d1 + d0, each in [-128, 127]
-            const int d0 = (I[i] << 24) >> 24;
-            const int r1 = (I[i] - d0) >> 8;
-            const int d1 = (r1 << 24) >> 24;
-            D[2][i] = d0;
-            D[1][i] = d1;
-            D[0][i] = (r1 - d1) >> 8;
-        } else {       // two's-complement bytes: top byte signed, lower bytes unsigned
-            D[2][i] = I[i];
-            D[1][i] = I[i] >> 8;
-            D[0][i] = I[i] >> 16;
-        }
+        const uint32_t bits = __float_as_uint(fmaf(f[i], to_fixed, 12582912.0f));
+        J[i] = SINGLE ? ((bits - (kMagicBits - 0x00808080u)) ^ 0x00808080u) : (bits - kMagicBits);
     }
+    uint32_t plane[3][2];  // [0] most significant; {even k, odd k}
 #pragma unroll
     for (int pl = 0; pl < 3; ++pl) {
-        const uint32_t e01 = __byte_perm(D[pl][0], D[pl][2], 0x0040), e23 = __byte_perm(D[pl][4], D[pl][6], 0x0040);
-        const uint32_t o01 = __byte_perm(D[pl][1], D[pl][3], 0x0040), o23 = __byte_perm(D[pl][5], D[pl][7], 0x0040);
+        const uint32_t sel = (uint32_t)(2 - pl) | ((uint32_t)(6 - pl) << 4);  // byte 2 - pl of both operands
+        const uint32_t e01 = __byte_perm(J[0], J[2], sel), e23 = __byte_perm(J[4], J[6], sel);
+        const uint32_t o01 = __byte_perm(J[1], J[3], sel), o23 = __byte_perm(J[5], J[7], sel);
         plane[pl][0] = __byte_perm(e01, e23, 0x5410);
         plane[pl][1] = __byte_perm(o01, o23, 0x5410);
     }
@@ -351,7 +350,8 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
     const int64_t e = p.strip_aligned ? range_begin(ci + 1, p.Gz, p.S) * len : range_begin(ci + 1, p.Gz, T);
     const int nblk = (int)(e - a);
     if (nblk <= 0) return;
-    const int64_t s_first = a / len, s_last = (e - 1) / len;
+    const bool small = fits32(p.Gz, T);
+    const int64_t s_first = div_floor(a, len, small), s_last = div_floor(e - 1, len, small);
     const int bl_first = (int)(a - s_first * len);    // block index inside the slice of the CTA's first block
     const int npieces = (int)(s_last - s_first) + 1;  // strips this CTA touches
     // Processing order: the blocks of a partial last strip come first, then the rest of the range in order.
