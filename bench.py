@@ -177,10 +177,24 @@ def run_shape(args):
         fd.fdqp_run(ctx, x, copies[i % ncopies], y, M, K, N, sraw)
     stream.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(args.steps):
-        fd.fdqp_run(ctx, x, copies[i % ncopies], y, M, K, N, sraw)
-    e1.record(stream)
+    if args.graph and not args.same_weights:
+        # the timed launches replayed from one CUDA graph, so that the host's launch cost is not what is measured
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(args.steps):
+                fd.fdqp_run(ctx, x, copies[i % ncopies], y, M, K, N, sraw)
+        with torch.cuda.stream(stream):
+            g.replay()
+        stream.synchronize()
+        e0.record(stream)
+        with torch.cuda.stream(stream):
+            g.replay()
+        e1.record(stream)
+    else:
+        e0.record(stream)
+        for i in range(args.steps):
+            fd.fdqp_run(ctx, x, copies[i % ncopies], y, M, K, N, sraw)
+        e1.record(stream)
     stream.synchronize()
     assert fd.fdqp_last_status(ctx) == 0
     us = e0.elapsed_time(e1) * 1e3 / args.steps
@@ -188,6 +202,7 @@ def run_shape(args):
     print(json.dumps({"shape": {"K": K, "N": N, "M": M}, "us_per_call": us, "GBps": gbs,
                       "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
                       "peak_kind": peak_kind, "weight_copies": ncopies, "steps": args.steps,
+                      "graph": bool(args.graph and not args.same_weights),
                       "launch": fd.fdqp_describe(ctx, M, K, N)}), flush=True)
     fd.fdqp_destroy(ctx)
 
