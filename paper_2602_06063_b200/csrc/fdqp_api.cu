@@ -19,7 +19,7 @@ cudaError_t splitk_sum_launch(const float* ws, float* y, int Z, int S, int M, in
 cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream);
 cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
 cudaError_t prefill_set_smem_limit();
-cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, int* status, int M, int K, int N,
+cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, int* status, int M, int K, int N, int pair,
                            cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
 }  // namespace fdqp
@@ -43,7 +43,7 @@ struct fdqp_ctx {
     int64_t launches = 0;
     std::string last_err;
     // overrides (-1 = automatic)
-    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1, p_prep = -1, p_aligned = -1, p_bpw = -1;
+    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1, p_prep = -1, p_aligned = -1, p_bpw = -1, p_pair = -1;
 };
 
 namespace {
@@ -81,6 +81,9 @@ fdqp_status check_shape(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
 
 // M >= 9 goes to the tensor-core kernel when its 256 x 256 tiles can occupy at least half of the SMs or the token
 // count is large; a few tiles with few tokens are faster through the GEMV kernel, eight token rows at a time.
+// More than 256 token rows: a pair of SMs works on a 256 x 512 tile (every converted weight serves 512 tokens).
+bool use_pair(const fdqp_ctx* ctx, int64_t M) { return ctx->p_pair >= 0 ? ctx->p_pair != 0 : M > 256; }
+
 bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t N) {
     if (M <= kMaxTokens || ctx->p_path == 2) return false;
     if (ctx->p_path == 3) return true;
@@ -295,7 +298,7 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
     }
     if (use_prefill(ctx, M, N)) {
         // prefill-sized M: dequantise into shared memory, contract with tcgen05 (accumulators in TMEM)
-        if ((e = prefill_launch(W, x, y, ctx->status_dev, (int)M, (int)K, (int)N, stream)))
+        if ((e = prefill_launch(W, x, y, ctx->status_dev, (int)M, (int)K, (int)N, use_pair(ctx, M) ? 1 : 0, stream)))
             return cuda_fail(ctx, e, "prefill kernel launch");
         ctx->launches += 1;
         return FDQP_OK;
@@ -395,6 +398,9 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
     } else if (!std::strcmp(key, "split_k")) {
         if (v != -1 && v != 1 && v != 2 && v != 4 && v != 8) return FDQP_ERR_ARG;
         ctx->p_split_k = v;
+    } else if (!std::strcmp(key, "prefill_pair")) {
+        if (v > 1) return FDQP_ERR_ARG;
+        ctx->p_pair = v;
     } else if (!std::strcmp(key, "l2_evict_first")) {
         if (v > 1) return FDQP_ERR_ARG;
         ctx->p_evict = v;
@@ -427,8 +433,13 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
         return FDQP_OK;
     }
     if (use_prefill(ctx, M, N)) {
-        std::snprintf(buf, buf_bytes, "fdqp_prefill_kernel grid=%lld block=320 tile=256x256 stages=3 tmem_cols=512",
-                      (long long)(((N + 255) / 256) * ((M + 255) / 256)));
+        if (use_pair(ctx, M))
+            std::snprintf(buf, buf_bytes,
+                          "fdqp_prefill_pair_kernel grid=%lld cluster=2 block=320 tile=256x512 per pair stages=4 tmem_cols=512",
+                          (long long)(2 * ((N + 255) / 256) * ((M + 511) / 512)));
+        else
+            std::snprintf(buf, buf_bytes, "fdqp_prefill_kernel grid=%lld block=320 tile=256x256 stages=3 tmem_cols=512",
+                          (long long)(((N + 255) / 256) * ((M + 255) / 256)));
         return FDQP_OK;
     }
     GemvPlan plan;

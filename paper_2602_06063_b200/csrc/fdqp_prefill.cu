@@ -158,9 +158,9 @@ __device__ __forceinline__ float dequant_hi(uint32_t q2, uint32_t d_bits, float 
 // Codes become bf16 pairs with one logic op per pair ((w >> 4i) & 0x000F000F | 0x43004300 = (128+q_i, 128+q_{i+4}));
 // the bias is removed exactly by a packed bf16 subtract; no integer-to-float conversion instruction is used.
 // An absent group arrives with codes, d and m all zero and therefore writes zeros.
-__device__ __forceinline__ void group_store(uint8_t* a_tile, const GroupRegs& r, int strip_local, int gl, int lane) {
+__device__ __forceinline__ void group_store(uint32_t a_tile, const GroupRegs& r, int strip_local, int gl, int lane) {
     const int row = strip_local * 32 + lane;
-    uint8_t* row_base = a_tile + (row >> 3) * 1024 + (row & 7) * 128;
+    const uint32_t row_base = a_tile + (uint32_t)((row >> 3) * 1024 + (row & 7) * 128);
     const uint32_t r7s = (uint32_t)(row & 7) << 4;
     const float m = __uint_as_float(r.m_bits << 16);
     const uint32_t words[4] = {r.codes.x, r.codes.y, r.codes.z, r.codes.w};
@@ -175,13 +175,15 @@ __device__ __forceinline__ void group_store(uint8_t* a_tile, const GroupRegs& r,
             f[i] = dequant_lo(q2, r.d_bits, m);
             f[i + 4] = dequant_hi(q2, r.d_bits, m);
         }
-        uint4 out;
-        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out.x) : "f"(f[1]), "f"(f[0]));  // {hi, lo}
-        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out.y) : "f"(f[3]), "f"(f[2]));
-        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out.z) : "f"(f[5]), "f"(f[4]));
-        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out.w) : "f"(f[7]), "f"(f[6]));
+        uint32_t o0, o1, o2, o3;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o0) : "f"(f[1]), "f"(f[0]));  // {hi, lo}
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o1) : "f"(f[3]), "f"(f[2]));
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o2) : "f"(f[5]), "f"(f[4]));
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o3) : "f"(f[7]), "f"(f[6]));
         // 16-byte chunk (gl*4 + wi) of the 128-byte row, at its swizzled position
-        *reinterpret_cast<uint4*>(row_base + ((uint32_t)((gl * 4 + wi) << 4) ^ r7s)) = out;
+        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(row_base + (((uint32_t)(gl * 4 + wi) << 4) ^ r7s)),
+                     "r"(o0), "r"(o1), "r"(o2), "r"(o3)
+                     : "memory");
     }
 }
 
@@ -283,7 +285,7 @@ __global__ void __launch_bounds__(kPfThreads, 1)
             }
             if (i >= kPfStages) ok = mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status);
             if (!ok) break;
-            uint8_t* a_tile = smem + s * kPfStageBytes;
+            const uint32_t a_tile = base + s * kPfStageBytes;
             group_store(a_tile, g0, dw, 0, lane);
             group_store(a_tile, g1, dw, 1, lane);
             // make the generic-proxy stores visible to the tensor core's (async-proxy) reads, then signal
@@ -323,6 +325,233 @@ __global__ void __launch_bounds__(kPfThreads, 1)
     }
 }
 
+// ---- the two-SM kernel (M > 256) ----------------------------------------------------------------------------------
+//
+// A cluster of two CTAs computes a 256 (output features) x 512 (tokens) tile with tcgen05.mma.cta_group::2: each CTA
+// dequantises ITS 128 rows (16 KB per 64-k stage) and loads ITS half of the tokens of each MMA (2 x 128 tokens, 32 KB
+// per stage); the tensor cores of the pair read both CTAs' shared memory, so every converted weight serves 512 tokens
+// and every loaded activation serves 256 rows.  Accumulators: 128 lanes x 512 columns of each CTA's TMEM (rows of that
+// CTA, all 512 tokens).  CTA 0 of the pair issues the MMAs; stage barriers it waits on live in CTA 0 and are signalled
+// by both CTAs; tcgen05.commit releases the stage in both CTAs at once.
+
+constexpr int kP2Rows = 128;      // output features per CTA (256 per pair)
+constexpr int kP2Toks = 512;      // tokens per pair tile
+constexpr int kP2TokBox = 128;    // tokens per CTA per MMA
+constexpr int kP2Stages = 4;
+constexpr uint32_t kP2ABytes = kP2Rows * kPfK * 2;        // 16 KB
+constexpr uint32_t kP2BBoxBytes = kP2TokBox * kPfK * 2;   // 16 KB
+constexpr uint32_t kP2StageBytes = kP2ABytes + 2 * kP2BBoxBytes;  // 48 KB
+constexpr uint32_t kP2SmemBytes = kP2Stages * kP2StageBytes + 1024 + 256;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address of the same shared-memory offset in CTA `rank` of the cluster (shared::cluster window).
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Arrive on a barrier of another CTA of the cluster.  The data this signals was written to the issuing CTA's own shared
+// memory and already made visible to the async proxy (the tensor cores) by fence.proxy.async; a cluster-scope release
+// here would add a full memory barrier per warp per stage (measured: the dominant stall).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Bounded wait whose success also orders the other CTA's writes before this thread's later operations.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, int* status) {
+    const unsigned long long t0 = globaltimer_ns();
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if ((it & 63u) == 63u && globaltimer_ns() - t0 > kWaitLimitNs) {
+            atomicExch(status, kStatusTimeout);
+            __threadfence_system();
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma2_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                           uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive on the barrier at this offset in BOTH CTAs once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
+    asm volatile(
+        "{\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}"
+        ::"r"(bar)
+        : "memory");
+}
+// This CTA's box of x into its own shared memory; the bytes are counted on CTA 0's barrier.
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar_cta0) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cta0), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+__global__ void __launch_bounds__(kPfThreads, 1)
+    fdqp_prefill_pair_kernel(const __grid_constant__ CUtensorMap x_map, const PrefillParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;  // same offset in both CTAs (same kernel, same dynamic size)
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t bars = base + kP2Stages * kP2StageBytes;
+    auto full_a = [&](int s) { return bars + 8u * s; };                      // used in CTA 0: 16 warp arrivals
+    auto full_b = [&](int s) { return bars + 8u * (kP2Stages + s); };        // used in CTA 0: 1 arrival + 64 KB
+    auto empty = [&](int s) { return bars + 8u * (2 * kP2Stages + s); };     // each CTA its own, signalled by commit
+    const uint32_t acc_done = bars + 8u * (3 * kP2Stages);
+    const uint32_t tmem_slot = acc_done + 8u;
+    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(smem + kP2Stages * kP2StageBytes + 8 * (3 * kP2Stages + 1));
+
+    const uint32_t rank = cluster_ctarank();
+    const int pair = blockIdx.x >> 1;
+    const int tok_tiles = (p.M + kP2Toks - 1) / kP2Toks;
+    const int n_tile = pair / tok_tiles, tok_tile = pair % tok_tiles;
+    const int n0 = n_tile * (2 * kP2Rows) + (int)rank * kP2Rows, tok0 = tok_tile * kP2Toks;
+    const int ksteps = (p.K + kPfK - 1) / kPfK;
+
+    if (tid == 0) {
+        for (int s = 0; s < kP2Stages; ++s) {
+            mbar_init(full_a(s), 2 * kPfDequantWarps);
+            mbar_init(full_b(s), 1);
+            mbar_init(empty(s), 1);
+        }
+        mbar_init(acc_done, 1);
+        mbar_fence_init();
+    }
+    if (warp == 0) {
+        tmem_alloc2(tmem_slot, kPfTmemCols);
+        tmem_relinquish2();
+    }
+    tc_fence_before();
+    cluster_sync_all();  // barriers of both CTAs initialised, TMEM allocated in both
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot_g;
+    bool ok = true;
+
+    if (warp == 0) {
+        // =============================== TMA producer: this CTA's token boxes ================================
+        if (lane == 0) {
+            for (int i = 0; i < ksteps && ok; ++i) {
+                const int s = i % kP2Stages;
+                if (i >= kP2Stages) ok = mbar_wait(empty(s), ((i / kP2Stages) - 1) & 1, p.status);
+                if (!ok) break;
+                if (rank == 0) mbar_arrive_expect_tx(full_b(s), 4 * kP2BBoxBytes);  // both CTAs' boxes
+                const uint32_t bar0 = mapa_shared(full_b(s), 0);
+                const uint32_t b_addr = base + s * kP2StageBytes + kP2ABytes;
+#pragma unroll
+                for (int j = 0; j < 2; ++j)  // MMA j covers tokens [256 j, 256 j + 256): this CTA's 128 of them
+                    tma2_load_2d(b_addr + j * kP2BBoxBytes, &x_map, i * kPfK, tok0 + j * 256 + (int)rank * kP2TokBox, bar0);
+            }
+        }
+    } else if (warp == 1) {
+        // =============================== MMA issuer (CTA 0 only) ============================================
+        if (lane == 0 && rank == 0) {
+            // kind::f16: D fp32, A and B bf16, both K-major, M = 256 over the pair, N = 256
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
+            for (int i = 0; i < ksteps && ok; ++i) {
+                const int s = i % kP2Stages;
+                const uint32_t ph = (i / kP2Stages) & 1;
+                ok = mbar_wait_cluster(full_a(s), ph, p.status) && mbar_wait_cluster(full_b(s), ph, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = base + s * kP2StageBytes, b_addr = a_addr + kP2ABytes;
+                const uint64_t adesc = umma_smem_desc(a_addr);
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const uint64_t bdesc = umma_smem_desc(b_addr + j * kP2BBoxBytes);
+#pragma unroll
+                    for (int k4 = 0; k4 < kPfK / 16; ++k4)
+                        umma2_bf16(tmem_base + j * 256, adesc + 2 * k4, bdesc + 2 * k4, idesc, (i | k4) != 0);
+                }
+                umma2_commit_both(empty(s));
+            }
+            umma2_commit_both(acc_done);
+        }
+    } else {
+        // =============================== dequantisation warps ================================================
+        const int dw = warp - 2;
+        const int sl = dw >> 1, gl = dw & 1;  // strip of this CTA's 128 rows, group of the 64-k stage
+        const int64_t strip = (int64_t)(n0 / kStripRows) + sl;
+        const bool strip_ok = strip < p.N / kStripRows;
+        // software pipeline: the loads of the next three stages are in flight while this one is converted (a stage
+        // lasts well under a microsecond here, less than one trip to L2 / HBM); groups past K load as zeros
+        GroupRegs g0 = group_load(p.W, p.K, strip, gl, lane, strip_ok);
+        GroupRegs g1 = group_load(p.W, p.K, strip, 2 + gl, lane, strip_ok);
+        GroupRegs g2 = group_load(p.W, p.K, strip, 4 + gl, lane, strip_ok);
+        const uint32_t full_a0 = mapa_shared(full_a(0), 0);
+        for (int i = 0; i < ksteps && ok; ++i) {
+            const int s = i % kP2Stages;
+            const GroupRegs g3 = group_load(p.W, p.K, strip, 2 * (i + 3) + gl, lane, strip_ok);
+            if (i >= kP2Stages) ok = mbar_wait(empty(s), ((i / kP2Stages) - 1) & 1, p.status);
+            if (!ok) break;
+            group_store(base + s * kP2StageBytes, g0, sl, gl, lane);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(full_a0 + 8u * s);
+            g0 = g1;
+            g1 = g2;
+            g2 = g3;
+        }
+        // =============================== epilogue: this CTA's TMEM -> y ======================================
+        if (ok) ok = mbar_wait(acc_done, 0, p.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+            tc_fence_after();
+            const int quarter = warp & 3;   // TMEM lanes this warp may read
+            const int chalf = dw >> 2;      // columns [256 chalf, 256 chalf + 256): every (quarter, half) once
+            const int n = n0 + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(chalf * 256);
+            const int toks = p.M - tok0 - chalf * 256;  // tokens of this column half that exist
+            for (int c = 0; c < 256 && c < toks; c += 32) {
+                uint32_t v[32];
+                tmem_ld_32cols(taddr + c, v);
+                if (n < p.N) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (c + j < toks) p.y[(int64_t)(tok0 + chalf * 256 + c + j) * p.N + n] = __uint_as_float(v[j]);
+                }
+            }
+        }
+    }
+    // =============================== teardown: every path of both CTAs releases TMEM =========================
+    tc_fence_before();
+    cluster_sync_all();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc2(tmem_base, kPfTmemCols);
+    }
+}
+
 // ---- host side ----------------------------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -342,18 +571,21 @@ static EncodeTiledFn encode_tiled_fn() {
 }
 
 cudaError_t prefill_set_smem_limit() {
-    return cudaFuncSetAttribute(fdqp_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPfSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(fdqp_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPfSmemBytes);
+    if (e) return e;
+    return cudaFuncSetAttribute(fdqp_prefill_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kP2SmemBytes);
 }
 
 // x: [M][K] bf16 row-major (device).  Returns cudaErrorNotSupported if the tensor map cannot be built.
-cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, int* status, int M, int K, int N,
+// pair != 0: the two-SM kernel (256 x 512 tiles per CTA pair), meant for M > 256.
+cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, int* status, int M, int K, int N, int pair,
                            cudaStream_t stream) {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};      // innermost first
     const cuuint64_t strides[1] = {(cuuint64_t)K * 2};              // bytes between token rows
-    const cuuint32_t box[2] = {(cuuint32_t)kPfK, (cuuint32_t)kPfToks};
+    const cuuint32_t box[2] = {(cuuint32_t)kPfK, (cuuint32_t)(pair ? kP2TokBox : kPfToks)};
     const cuuint32_t elem[2] = {1, 1};
     if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t*>(x), dims, strides, box, elem,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -366,6 +598,22 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, int* s
     p.M = M;
     p.K = K;
     p.N = N;
+    if (pair) {
+        const int n_tiles = (N + 2 * kP2Rows - 1) / (2 * kP2Rows), tok_tiles = (M + kP2Toks - 1) / kP2Toks;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(2 * n_tiles * tok_tiles));
+        cfg.blockDim = dim3((unsigned)kPfThreads);
+        cfg.dynamicSmemBytes = kP2SmemBytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, fdqp_prefill_pair_kernel, map, p);
+    }
     const int n_tiles = (N + kPfRows - 1) / kPfRows, tok_tiles = (M + kPfToks - 1) / kPfToks;
     fdqp_prefill_kernel<<<n_tiles * tok_tiles, kPfThreads, kPfSmemBytes, stream>>>(map, p);
     return cudaGetLastError();

@@ -25,10 +25,10 @@ def ctx():
 @pytest.fixture()
 def fresh(ctx):
     """The shared context with every launch parameter back to automatic."""
-    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp"):
+    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp", "prefill_pair"):
         fd.fdqp_set_param(ctx, key, -1)
     yield ctx
-    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp"):
+    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp", "prefill_pair"):
         fd.fdqp_set_param(ctx, key, -1)
 
 
@@ -99,7 +99,8 @@ def test_exact_arithmetic_regime_is_bit_exact(fresh, K, N, M):
         assert np.array_equal(y.astype(np.float64), y_ref), f"path {path}"
 
 
-PREFILL = [(64, 32, 9), (1024, 512, 9), (1056, 320, 20), (2560, 1024, 100), (512, 288, 300), (4096, 768, 512)]
+PREFILL = [(64, 32, 9), (1024, 512, 9), (1056, 320, 20), (2560, 1024, 100), (512, 288, 300), (4096, 768, 512),
+           (1056, 320, 257), (544, 1056, 511)]
 
 
 @pytest.mark.parametrize("K,N,M", PREFILL)
@@ -108,10 +109,15 @@ def test_prefill_tensor_path_matches_oracle(fresh, K, N, M):
     # the 64-wide pipeline step, N that is not a multiple of the 256-row tile, more than one token tile.
     case = Case(K, N, M, seed=2000 + K + N + M)
     fd.fdqp_set_param(fresh, "path", 3)
-    assert "fdqp_prefill_kernel" in fd.fdqp_describe(fresh, M, K, N)
+    assert ("fdqp_prefill_pair_kernel" if M > 256 else "fdqp_prefill_kernel") in fd.fdqp_describe(fresh, M, K, N)
     y = case.run(fresh)
     y_ref, a_ref = case.reference()
     assert_close(y, y_ref, a_ref, f"prefill K={K} N={N} M={M}")
+    # the other tensor-core kernel (two-SM 256 x 512 tile <-> one-SM 256 x 256 tile) on the same inputs
+    fd.fdqp_set_param(fresh, "prefill_pair", 0 if M > 256 else 1)
+    assert ("fdqp_prefill_kernel" if M > 256 else "fdqp_prefill_pair_kernel") in fd.fdqp_describe(fresh, M, K, N)
+    assert_close(case.run(fresh), y_ref, a_ref, f"prefill (other tile) K={K} N={N} M={M}")
+    fd.fdqp_set_param(fresh, "prefill_pair", -1)
     # the same rows through the GEMV kernel, eight at a time: both are within the bound of the oracle
     fd.fdqp_set_param(fresh, "path", 2)
     assert "fdqp_gemv_kernel" in fd.fdqp_describe(fresh, M, K, N)
