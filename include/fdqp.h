@@ -141,6 +141,17 @@ FDQP_API fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W_q
 FDQP_API fdqp_status fdqp_run_host(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,
                           int64_t M, int64_t K, int64_t N, void* cuda_stream);
 
+/* fdqp_run_host without the final synchronisation: the copy of x, the projection
+ * and the copy of y are enqueued on `cuda_stream` and the call returns.  x_host and
+ * y_host (host; pinned memory for the copies to be asynchronous) must stay valid
+ * and untouched until the stream has passed the call; y_host holds the result once
+ * the caller has synchronised the stream, after which fdqp_last_status tells whether
+ * a kernel gave up.  Several calls may be queued on one stream (they share the
+ * context's staging buffers in stream order); calls on different streams must not
+ * share a context.  Errors as fdqp_run. */
+FDQP_API fdqp_status fdqp_run_host_async(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,
+                                int64_t M, int64_t K, int64_t N, void* cuda_stream);
+
 /* The same projection for callers that must not allocate device memory at the time of the call -- a server that
  * gave all device memory to its own pool at start-up, a real-time loop that cannot take the device-wide
  * synchronisation an allocation may bring, a plug-in that may not allocate after initialisation.  (The paper has no

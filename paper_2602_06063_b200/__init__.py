@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     fdqp_launch_count,
     fdqp_run,
     fdqp_run_host,
+    fdqp_run_host_async,
     fdqp_run_noalloc,
     fdqp_set_param,
     fdqp_status_string,

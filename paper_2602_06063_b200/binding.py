@@ -23,6 +23,7 @@ STATUS = {
 
 EXPORTS = [
     "q4nx_packed_bytes", "q4nx_pack", "q4nx_unpack", "fdqp_create", "fdqp_destroy", "fdqp_run", "fdqp_run_host",
+    "fdqp_run_host_async",
     "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
     "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc",
 ]
@@ -63,6 +64,8 @@ def load_library():
     lib.fdqp_run.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_run_host.restype = ci
     lib.fdqp_run_host.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.fdqp_run_host_async.restype = ci
+    lib.fdqp_run_host_async.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_run_noalloc.restype = ci
     lib.fdqp_run_noalloc.argtypes = [vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_dequant.restype = ci
@@ -171,6 +174,12 @@ def fdqp_run_host(ctx: int, x_host_bf16, W_q4nx, y_host, M: int, K: int, N: int,
     """x, y: HOST buffers (numpy or pinned torch); W: device.  Returns after y_host is filled."""
     _check(load_library().fdqp_run_host(ctx, _addr(x_host_bf16), _addr(W_q4nx), _addr(y_host), M, K, N,
                                         _stream(stream)), "fdqp_run_host", ctx)
+
+
+def fdqp_run_host_async(ctx: int, x_host_bf16, W_q4nx, y_host, M: int, K: int, N: int, stream=None) -> None:
+    """fdqp_run_host without the final synchronisation: y_host is valid once the caller has synchronised the stream."""
+    _check(load_library().fdqp_run_host_async(ctx, _addr(x_host_bf16), _addr(W_q4nx), _addr(y_host), M, K, N,
+                                              _stream(stream)), "fdqp_run_host_async", ctx)
 
 
 def fdqp_run_noalloc(x_bf16, W_q4nx, y, M: int, K: int, N: int, stream=None) -> None:

@@ -334,8 +334,8 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
     return FDQP_OK;
 }
 
-extern "C" fdqp_status fdqp_run_host(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,
-                                     int64_t M, int64_t K, int64_t N, void* cuda_stream) {
+extern "C" fdqp_status fdqp_run_host_async(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,
+                                           int64_t M, int64_t K, int64_t N, void* cuda_stream) {
     if (!ctx || !x_host_bf16 || !W_q4nx || !y_host) return FDQP_ERR_ARG;
     fdqp_status st = check_shape(ctx, M, K, N);
     if (st != FDQP_OK) return st;
@@ -353,7 +353,15 @@ extern "C" fdqp_status fdqp_run_host(fdqp_ctx* ctx, const void* x_host_bf16, con
     if (st != FDQP_OK) return st;
     if ((e = cudaMemcpyAsync(y_host, ctx->y_stage, (size_t)M * N * 4, cudaMemcpyDeviceToHost, stream)))
         return cuda_fail(ctx, e, "y copy");
-    if ((e = cudaStreamSynchronize(stream))) return cuda_fail(ctx, e, "stream sync");
+    return FDQP_OK;
+}
+
+extern "C" fdqp_status fdqp_run_host(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,
+                                     int64_t M, int64_t K, int64_t N, void* cuda_stream) {
+    const fdqp_status st = fdqp_run_host_async(ctx, x_host_bf16, W_q4nx, y_host, M, K, N, cuda_stream);
+    if (st != FDQP_OK) return st;
+    const cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream));
+    if (e) return cuda_fail(ctx, e, "stream sync");
     return fdqp_last_status(ctx);
 }
 

@@ -280,3 +280,12 @@ def test_run_host_roundtrip(fresh):
     y_ref, a_ref = case.reference()
     assert_close(y_host.numpy(), y_ref, a_ref, "run_host")
     assert np.array_equal(y_host.numpy(), case.run(fresh))
+    # the asynchronous form: two calls queued on one stream, results valid after the caller's synchronisation
+    y2 = torch.zeros((M, N), dtype=torch.float32).pin_memory()
+    y3 = torch.zeros((1, N), dtype=torch.float32).pin_memory()
+    fd.fdqp_run_host_async(fresh, x_host, case.W_dev, y2, M, K, N)
+    fd.fdqp_run_host_async(fresh, x_host[:1], case.W_dev, y3, 1, K, N)
+    torch.cuda.synchronize()
+    assert fd.fdqp_last_status(fresh) == 0
+    assert np.array_equal(y2.numpy(), y_host.numpy())
+    assert_close(y3.numpy(), y_ref[:1], a_ref[:1], "run_host_async M=1")
