@@ -438,6 +438,12 @@ __global__ void __launch_bounds__(kPfThreads, 1)
     const int n_tile = pair / tok_tiles, tok_tile = pair % tok_tiles;
     const int n0 = n_tile * (2 * kP2Rows) + (int)rank * kP2Rows, tok0 = tok_tile * kP2Toks;
     const int ksteps = (p.K + kPfK - 1) / kPfK;
+    // tokens of the two MMAs of a k-step, rounded up to the instruction's granularity (16); the second MMA is dropped
+    // when the tile has no more than 256 tokens.  Each CTA supplies half of an MMA's tokens.
+    const int rem = p.M - tok0;
+    const int n_mma0 = rem >= 256 ? 256 : ((rem + 15) & ~15);
+    const int n_mma1 = rem <= 256 ? 0 : (rem - 256 >= 256 ? 256 : ((rem - 256 + 15) & ~15));
+    const int n_mmas = n_mma1 > 0 ? 2 : 1;
 
     if (tid == 0) {
         for (int s = 0; s < kP2Stages; ++s) {
@@ -465,19 +471,22 @@ __global__ void __launch_bounds__(kPfThreads, 1)
                 const int s = i % kP2Stages;
                 if (i >= kP2Stages) ok = mbar_wait(empty(s), ((i / kP2Stages) - 1) & 1, p.status);
                 if (!ok) break;
-                if (rank == 0) mbar_arrive_expect_tx(full_b(s), 4 * kP2BBoxBytes);  // both CTAs' boxes
+                if (rank == 0) mbar_arrive_expect_tx(full_b(s), 2 * n_mmas * kP2BBoxBytes);  // both CTAs' boxes
                 const uint32_t bar0 = mapa_shared(full_b(s), 0);
                 const uint32_t b_addr = base + s * kP2StageBytes + kP2ABytes;
-#pragma unroll
-                for (int j = 0; j < 2; ++j)  // MMA j covers tokens [256 j, 256 j + 256): this CTA's 128 of them
-                    tma2_load_2d(b_addr + j * kP2BBoxBytes, &x_map, i * kPfK, tok0 + j * 256 + (int)rank * kP2TokBox, bar0);
+                // MMA j covers tokens [256 j, 256 j + n_j): this CTA supplies n_j / 2 of them (a full 128-token box is
+                // copied; what the MMA does not read is ignored, what lies beyond M arrives as zeros)
+                tma2_load_2d(b_addr, &x_map, i * kPfK, tok0 + (int)rank * (n_mma0 / 2), bar0);
+                if (n_mmas == 2)
+                    tma2_load_2d(b_addr + kP2BBoxBytes, &x_map, i * kPfK, tok0 + 256 + (int)rank * (n_mma1 / 2), bar0);
             }
         }
     } else if (warp == 1) {
         // =============================== MMA issuer (CTA 0 only) ============================================
         if (lane == 0 && rank == 0) {
-            // kind::f16: D fp32, A and B bf16, both K-major, M = 256 over the pair, N = 256
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
+            // kind::f16: D fp32, A and B bf16, both K-major, M = 256 over the pair, N = tokens of the MMA
+            const uint32_t idesc_mn = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 4) << 24);
+            const uint32_t idesc[2] = {idesc_mn | ((uint32_t)(n_mma0 >> 3) << 17), idesc_mn | ((uint32_t)(n_mma1 >> 3) << 17)};
             for (int i = 0; i < ksteps && ok; ++i) {
                 const int s = i % kP2Stages;
                 const uint32_t ph = (i / kP2Stages) & 1;
@@ -488,10 +497,12 @@ __global__ void __launch_bounds__(kPfThreads, 1)
                 const uint64_t adesc = umma_smem_desc(a_addr);
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
-                    const uint64_t bdesc = umma_smem_desc(b_addr + j * kP2BBoxBytes);
+                    if (j < n_mmas) {
+                        const uint64_t bdesc = umma_smem_desc(b_addr + j * kP2BBoxBytes);
 #pragma unroll
-                    for (int k4 = 0; k4 < kPfK / 16; ++k4)
-                        umma2_bf16(tmem_base + j * 256, adesc + 2 * k4, bdesc + 2 * k4, idesc, (i | k4) != 0);
+                        for (int k4 = 0; k4 < kPfK / 16; ++k4)
+                            umma2_bf16(tmem_base + j * 256, adesc + 2 * k4, bdesc + 2 * k4, idesc[j], (i | k4) != 0);
+                    }
                 }
                 umma2_commit_both(empty(s));
             }

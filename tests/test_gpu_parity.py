@@ -100,7 +100,7 @@ def test_exact_arithmetic_regime_is_bit_exact(fresh, K, N, M):
 
 
 PREFILL = [(64, 32, 9), (1024, 512, 9), (1056, 320, 20), (2560, 1024, 100), (512, 288, 300), (4096, 768, 512),
-           (1056, 320, 257), (544, 1056, 511)]
+           (1056, 320, 257), (544, 1056, 511), (512, 512, 272), (512, 512, 400)]
 
 
 @pytest.mark.parametrize("K,N,M", PREFILL)
