@@ -110,6 +110,23 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+# ----------------------------------------------------------------------------------------------- rank plumbing
+
+def max_over_ranks(value, dist, device):
+    """The slowest rank's figure: a whole-job time is the maximum over ranks (replicas do not talk otherwise)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(bytes_per_step, steps, world, ms):
+    """Aggregate over all replicas: every rank moved bytes_per_step * steps in the (max-over-ranks) time ms."""
+    return bytes_per_step * steps * world / (ms * 1e-3) / 1e9
+
+
 # ----------------------------------------------------------------------------------------------- reference arm
 
 def run_reference(args, rank, world):
@@ -340,10 +357,7 @@ def run_ours(args, rank, local_rank, world):
     clocks = sampler.stop() if rank == 0 else None
     if fd.fdqp_last_status(ctx) != 0:
         raise SystemExit("bench.py: a kernel reported " + fd.fdqp_status_string(fd.fdqp_last_status(ctx)))
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, "cuda")
 
     # ---- end to end: host x in, host y out, through fdqp_run_host_async (pinned buffers) + one stream sync, every step
     xs_pin = [torch.from_numpy(x.view(np.int16)).pin_memory() for x in xs_host]
@@ -364,10 +378,7 @@ def run_ours(args, rank, local_rank, world):
         e2e_step(3 + i)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s, dist, "cuda")
 
     # ---- LM head (M = 1) for the tokens/s figure: 34 layers + head, projections only
     head_ms = None
@@ -432,7 +443,7 @@ def run_ours(args, rank, local_rank, world):
 
     if rank == 0:
         step_bytes = step_bytes_layer
-        gbs = step_bytes * args.steps * world / (ms * 1e-3) / 1e9
+        gbs = whole_job_gbs(step_bytes, args.steps, world, ms)
         per_launch_us = ms * 1e3 / (calls_per_step * args.steps)   # one GEMV launch incl. its preparation kernel
         achieved = (step_bytes / calls_per_step) / (per_launch_us * 1e-6) / 1e9
         layer_ms = ms / args.steps
@@ -458,7 +469,7 @@ def run_ours(args, rank, local_rank, world):
                          "kernel": "fdqp_gemv_kernel", "launch_us": per_launch_us},
             "prefill_lm_head": prefill,
             "cpu_baseline": cpu,
-            "e2e": {"value": step_bytes * e2e_steps * world / e2e_s / 1e9, "unit": "GB/s",
+            "e2e": {"value": whole_job_gbs(step_bytes, e2e_steps, world, e2e_s * 1e3), "unit": "GB/s",
                     "h2d_bytes_per_step": sum(2 * M * K for _, K, _, _ in shapes),
                     "d2h_bytes_per_step": sum(4 * M * N for _, _, N, _ in shapes), "ms_per_step": e2e_s / e2e_steps * 1e3},
             "gpu_launches": launches,
