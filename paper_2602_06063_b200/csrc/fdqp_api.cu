@@ -138,9 +138,13 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
             nbz = (p->nb + Z - 1) / Z;
             // four blocks per warp per stage halve the barrier traffic per tile; worth it once a CTA streams many blocks
             const int64_t blocks_per_cta = (int64_t)p->S * p->nb / ((int64_t)ctx->sm_count * ctas_per_sm);
-            bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (M == 1 && blocks_per_cta >= 64 ? 4 : 2);
-            if (M != 1) bpw = 2;
+            // (measured: pays up to M = 4, never when the larger stage would force a K split)
+            bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (M <= 4 && blocks_per_cta >= 64 ? 4 : 2);
             L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw);
+            if (bpw == 4 && ctx->p_bpw != 4 && M > 1 && L.nstage < kMinStages) {
+                bpw = 2;
+                L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw);
+            }
             if (L.nstage >= kMinStages || Z >= kMaxSplit || Z >= p->nb) break;
         }
         if (L.nstage >= 2 || ctas_per_sm == 1) break;

@@ -812,28 +812,37 @@ cudaError_t splitk_sum_launch(const float* ws, float* y, int Z, int S, int M, in
     return cudaLaunchKernelEx(&cfg, fdqp_splitk_sum_kernel, ws, y, Z, S, M, N);
 }
 
-// consumer_warps: 8 or 16; p.bpw (blocks per warp per stage): 2, or 4 at M == 1.  Kernel mode by M (see the header).
+// consumer_warps: 8 or 16; p.bpw (blocks per warp per stage): 2 or 4.  Kernel mode by M (see the header).
 cudaError_t gemv_launch(const GemvPlan& p, int consumer_warps, cudaStream_t stream) {
-    const bool w16 = consumer_warps == 16;
+    const bool w16 = consumer_warps == 16, b4 = p.bpw == 4;
     if (p.M == 1) {
-        if (w16) return p.bpw == 4 ? launch_one<16, 1, 4>(p, stream) : launch_one<16, 1, 2>(p, stream);
-        return p.bpw == 4 ? launch_one<8, 1, 4>(p, stream) : launch_one<8, 1, 2>(p, stream);
+        if (w16) return b4 ? launch_one<16, 1, 4>(p, stream) : launch_one<16, 1, 2>(p, stream);
+        return b4 ? launch_one<8, 1, 4>(p, stream) : launch_one<8, 1, 2>(p, stream);
     }
-    if (p.M > kColsMaxTokens) return w16 ? launch_one<16, 2, 2>(p, stream) : launch_one<8, 2, 2>(p, stream);
-    return w16 ? launch_one<16, 3, 2>(p, stream) : launch_one<8, 3, 2>(p, stream);
+    if (p.M > kColsMaxTokens) {
+        if (w16) return b4 ? launch_one<16, 2, 4>(p, stream) : launch_one<16, 2, 2>(p, stream);
+        return b4 ? launch_one<8, 2, 4>(p, stream) : launch_one<8, 2, 2>(p, stream);
+    }
+    if (w16) return b4 ? launch_one<16, 3, 4>(p, stream) : launch_one<16, 3, 2>(p, stream);
+    return b4 ? launch_one<8, 3, 4>(p, stream) : launch_one<8, 3, 2>(p, stream);
+}
+
+template <int CW, int MODE>
+static cudaError_t set_smem_limit_mode(int bytes) {
+    const cudaFuncAttribute a = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    cudaError_t e = cudaFuncSetAttribute(fdqp_gemv_kernel<CW, MODE, 2>, a, bytes);
+    if (e) return e;
+    return cudaFuncSetAttribute(fdqp_gemv_kernel<CW, MODE, 4>, a, bytes);
 }
 
 cudaError_t gemv_set_smem_limit(int bytes) {
     cudaError_t e;
-    const cudaFuncAttribute a = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 1, 2>, a, bytes))) return e;
-    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 1, 4>, a, bytes))) return e;
-    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 1, 2>, a, bytes))) return e;
-    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 1, 4>, a, bytes))) return e;
-    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 3, 2>, a, bytes))) return e;
-    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 3, 2>, a, bytes))) return e;
-    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<8, 2, 2>, a, bytes))) return e;
-    return cudaFuncSetAttribute(fdqp_gemv_kernel<16, 2, 2>, a, bytes);
+    if ((e = set_smem_limit_mode<8, 1>(bytes))) return e;
+    if ((e = set_smem_limit_mode<16, 1>(bytes))) return e;
+    if ((e = set_smem_limit_mode<8, 2>(bytes))) return e;
+    if ((e = set_smem_limit_mode<16, 2>(bytes))) return e;
+    if ((e = set_smem_limit_mode<8, 3>(bytes))) return e;
+    return set_smem_limit_mode<16, 3>(bytes);
 }
 
 }  // namespace fdqp
