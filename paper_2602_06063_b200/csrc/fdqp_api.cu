@@ -103,7 +103,7 @@ SmemLayout smem_layout(const fdqp_ctx* ctx, int M, int nbz, int cw, int ctas_per
     const uint32_t tiles = (uint32_t)nbz * 8u;
     L.xs_bytes = tiles * 128u * (uint32_t)M;          // prepared activations of the K slice
     L.xsum_bytes = M <= kColsMaxTokens ? 0u : tiles * 64u;         // per-token {sum x, unit} (plane mode only)
-    L.part_bytes = 2u * (uint32_t)cw * kStripRows * (uint32_t)M * 4u;
+    L.part_bytes = 2u * (uint32_t)cw * kStripRows * (uint32_t)M * 4u * (M <= kColsMaxTokens ? (uint32_t)kColsPartTerms : 1u);
     L.fixed = round_up(L.xs_bytes, 128) + round_up(L.xsum_bytes, 128) + round_up(L.part_bytes, 128) +
               (2u * kMaxStages + 5u) * 8u + 128u;
     const uint32_t per_cta = (uint32_t)ctx->smem_optin / (uint32_t)ctas_per_sm - (ctas_per_sm > 1 ? 1024u : 0u);

@@ -487,33 +487,42 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         bool alive = true;
         // hand the warp's partial rows of the current strip piece to the reducer warp
         auto flush = [&]() {
-            if (MT::kCols) {
-                // lanes q and q^1 hold the two halves of each row's sum for token q/2; lane r holds row r's offset terms
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    acc[i][0] += __shfl_xor_sync(0xffffffffu, acc[i][0], 1);
-                    const float m0 = __shfl_sync(0xffffffffu, acc_m[0], g + 8 * i);
-                    const float m1 = MT::kAccM == 1 ? 0.f : __shfl_sync(0xffffffffu, acc_m[MT::kAccM - 1], g + 8 * i);
-                    acc[i][0] += (q >> 1) ? m1 : m0;
-                }
-#pragma unroll
-                for (int tk = 0; tk < MT::kAccM; ++tk) acc_m[tk] = 0.f;
-            }
             const int par = piece & 1;
             if (piece >= 2 && !mbar_wait(red_empty0 + 8u * par, ((piece >> 1) - 1) & 1, p.status)) alive = false;
-            const uint32_t slot = part + (uint32_t)((par * CW + warp) * kStripRows * M) * 4u;
+            constexpr int PT = MT::kCols ? kColsPartTerms : 1;
+            const uint32_t slot = part + (uint32_t)((par * CW + warp) * PT * kStripRows * M) * 4u;
+            if (MT::kCols) {
+                // Lanes q and q^1 hold the two column halves of each row's sum for token q/2, lane r holds row r's
+                // offset terms: all three go to the reducer as they are ([term][token][row]); it adds them.
+                const int tok = q >> 1;
+                if (tok < M) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < NT; ++j) {
-                    // column modes: the accumulator is token q/2, complete in the lanes with even q
-                    const int tok = MT::kCols ? (q >> 1) : 2 * q + j;
-                    if (tok < M && (!MT::kCols || (q & 1) == 0))
-                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(slot + (uint32_t)(tok * kStripRows + g + 8 * i) * 4u),
-                                     "f"(acc[i][j])
+                    for (int i = 0; i < 4; ++i)
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(slot + (uint32_t)((((q & 1) * M + tok) * kStripRows) + g + 8 * i) * 4u),
+                                     "f"(acc[i][0])
                                      : "memory");
-                    acc[i][j] = 0.f;
                 }
+#pragma unroll
+                for (int tk = 0; tk < MT::kAccM; ++tk) {
+                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(slot + (uint32_t)((2 * M + tk) * kStripRows + lane) * 4u), "f"(acc_m[tk])
+                                 : "memory");
+                    acc_m[tk] = 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[i][0] = 0.f;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < NT; ++j) {
+                        const int tok = 2 * q + j;
+                        if (tok < M)
+                            asm volatile("st.shared.f32 [%0], %1;" ::"r"(slot + (uint32_t)(tok * kStripRows + g + 8 * i) * 4u),
+                                         "f"(acc[i][j])
+                                         : "memory");
+                        acc[i][j] = 0.f;
+                    }
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(red_full0 + 8u * par);
             ++piece;
@@ -676,9 +685,12 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             for (int t = 0; t < kMaxTokens; ++t) {
                 v[t] = 0.f;
                 if (t < M) {
+                    constexpr int PT = MT::kCols ? kColsPartTerms : 1;
 #pragma unroll
                     for (int w = 0; w < CW; ++w)
-                        v[t] += part_g[((par * CW + w) * M + t) * kStripRows + lane];
+#pragma unroll
+                        for (int h = 0; h < PT; ++h)
+                            v[t] += part_g[(((par * CW + w) * PT + h) * M + t) * kStripRows + lane];
                 }
             }
             __syncwarp();

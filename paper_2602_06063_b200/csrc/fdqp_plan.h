@@ -13,6 +13,8 @@ constexpr int kGroupBytes = 640;    // bytes a block spends per group: 512 codes
 constexpr int kMaxTokens = 8;       // token rows one GEMV launch handles
 // Up to this many tokens the GEMV lays the byte planes of a token out as MMA columns; above it, one MMA per plane.
 constexpr int kColsMaxTokens = 2;
+// Column modes hand three partial terms per (row, token) to the reducer (two column halves + the offset term).
+constexpr int kColsPartTerms = 3;
 constexpr int kMaxSplit = 8;        // K slices
 constexpr int kMaxCtasPerSm = 2;
 
