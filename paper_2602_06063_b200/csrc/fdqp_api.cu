@@ -79,16 +79,26 @@ fdqp_status check_shape(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     return FDQP_OK;
 }
 
-// M >= 9 goes to the tensor-core kernel when its 256 x 256 tiles can occupy at least half of the SMs or the token
-// count is large; a few tiles with few tokens are faster through the GEMV kernel, eight token rows at a time.
 // More than 256 token rows: a pair of SMs works on a 256 x 512 tile (every converted weight serves 512 tokens).
 bool use_pair(const fdqp_ctx* ctx, int64_t M) { return ctx->p_pair >= 0 ? ctx->p_pair != 0 : M > 256; }
 
-bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t N) {
+// M >= 9: the tensor-core kernels, or the GEMV kernel eight token rows at a time -- whichever a small cost model
+// (microseconds, constants measured on B200) says is faster.
+//   GEMV: every 8-row chunk streams the whole matrix at about 3 TB/s plus a fixed ~5 us.
+//   Tensor-core kernels: limited by converting the weights, ~0.9 us per 64-wide k-step per wave of tiles, whatever M is;
+//   measured 1.45x slower while the whole of x is smaller than 128 KB.
+bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     if (M <= kMaxTokens || ctx->p_path == 2) return false;
     if (ctx->p_path == 3) return true;
-    const int64_t tiles = ((N + 255) / 256) * ((M + 255) / 256);
-    return tiles * 2 >= ctx->sm_count || M > 128;
+    const double chunks = (double)((M + kMaxTokens - 1) / kMaxTokens);
+    const double t_gemv = chunks * (5.0 + 0.625 * (double)K * (double)N / 3.0e6);
+    const bool pair = use_pair(ctx, M);
+    const int64_t tiles = ((N + 255) / 256) * (pair ? (M + 511) / 512 : (M + 255) / 256);
+    const int64_t slots = pair ? ctx->sm_count / 2 : ctx->sm_count;
+    const double waves = (double)((tiles + slots - 1) / slots);
+    double t_tensor = 5.0 + waves * (double)((K + 63) / 64) * 0.9;
+    if (M * K < 65536) t_tensor *= 1.45;
+    return t_tensor < t_gemv;
 }
 
 // Shared-memory carve-up for a given configuration; returns the ring depth that fits (0 if none).
@@ -300,7 +310,7 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
         ctx->launches += 1;
         return FDQP_OK;
     }
-    if (use_prefill(ctx, M, N)) {
+    if (use_prefill(ctx, M, K, N)) {
         // prefill-sized M: dequantise into shared memory, contract with tcgen05 (accumulators in TMEM)
         if ((e = prefill_launch(W, x, y, ctx->status_dev, (int)M, (int)K, (int)N, use_pair(ctx, M) ? 1 : 0, stream)))
             return cuda_fail(ctx, e, "prefill kernel launch");
@@ -444,7 +454,7 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
                       (long long)((M + 7) / 8));
         return FDQP_OK;
     }
-    if (use_prefill(ctx, M, N)) {
+    if (use_prefill(ctx, M, K, N)) {
         if (use_pair(ctx, M))
             std::snprintf(buf, buf_bytes,
                           "fdqp_prefill_pair_kernel grid=%lld cluster=2 block=320 tile=256x512 per pair stages=4 tmem_cols=512",
