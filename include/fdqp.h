@@ -99,8 +99,10 @@ FDQP_API fdqp_status q4nx_unpack(const void* packed, int64_t K, int64_t N, uint8
 /* ---- context --------------------------------------------------------------- */
 
 /* Create a context on CUDA device `device` for projections up to max_M x max_K x
- * max_N.  Allocates (device) the split-K workspace, its arrival counters, and the
- * staging buffers of fdqp_run_host; reads the SM count and shared-memory limits.
+ * max_N.  Allocates (device) the split-K workspace and its arrival counters, and, when
+ * max_M > 8, up to 128 MB for the partial results of K-split tensor-core calls; the
+ * staging buffers of fdqp_run_host are allocated by its first call.  Reads the SM count
+ * and shared-memory limits.
  * A context serves one stream at a time: its workspace is not re-entrant.
  * Errors: FDQP_ERR_ARG (null), FDQP_ERR_SHAPE, FDQP_ERR_ARCH (not sm_100),
  * FDQP_ERR_CUDA, FDQP_ERR_NOMEM.  On error *ctx is NULL. */
@@ -207,6 +209,8 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "l2_evict_first" 1 = weight copies carry an evict-first L2 hint
  *   "strip_aligned" 1 = CTA work ranges are cut at strip boundaries, 0 = equal block counts per CTA
  *   "prep_inline"   1 = every GEMV CTA prepares its slice of x itself, 0 = a preparation kernel runs first
+ *   "prefill_split_k" 1..8 K slices for the tensor-core kernels (their partial results are added by a second
+ *                   kernel); default: as many as fill the SMs when a shape has few output tiles
  *   "prefill_pair"  1 = prefill-sized calls use the two-SM kernel (256 x 512 tile per CTA pair), 0 = the one-SM kernel
  *                   (256 x 256 tile); default: two-SM kernel when M > 256
  *   "debug"         measurement aid: 1 = the GEMV consumers skip the arithmetic (y is then undefined)

@@ -19,7 +19,8 @@ cudaError_t splitk_sum_launch(const float* ws, float* y, int Z, int S, int M, in
 cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream);
 cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
 cudaError_t prefill_set_smem_limit();
-cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, int* status, int M, int K, int N, int pair,
+cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, float* ws, int* status, int M, int K, int N, int pair,
+                           int Z,
                            cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
 }  // namespace fdqp
@@ -33,6 +34,8 @@ struct fdqp_ctx {
     int64_t max_M = 0, max_K = 0, max_N = 0;
     float* ws_edge = nullptr;
     float* ws_full = nullptr;
+    float* pf_ws = nullptr;      // partial results of K-split tensor-core calls
+    size_t pf_ws_bytes = 0;
     int* tickets = nullptr;
     uint32_t* xq = nullptr;      // prepared activations of the call in flight
     float* xsc = nullptr;
@@ -43,13 +46,14 @@ struct fdqp_ctx {
     int64_t launches = 0;
     std::string last_err;
     // overrides (-1 = automatic)
-    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1, p_prep = -1, p_aligned = -1, p_bpw = -1, p_pair = -1;
+    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1, p_prep = -1, p_aligned = -1, p_bpw = -1, p_pair = -1, p_pf_split = -1;
 };
 
 namespace {
 
 constexpr int kMaxStages = 40;
 constexpr double kTwoCtaBytes = 256e6;
+constexpr size_t kPrefillWsCap = 128u << 20;  // bytes of partial results a context keeps for K-split tensor-core calls
 constexpr int kMinStages = 3;  // ring depth below which another K slice is preferred
 
 struct DeviceGuard {
@@ -82,6 +86,22 @@ fdqp_status check_shape(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
 // More than 256 token rows: a pair of SMs works on a 256 x 512 tile (every converted weight serves 512 tokens).
 bool use_pair(const fdqp_ctx* ctx, int64_t M) { return ctx->p_pair >= 0 ? ctx->p_pair != 0 : M > 256; }
 
+// K slices of a tensor-core call: as many as fill one wave of SMs (or SM pairs), while every slice keeps at least eight
+// 64-wide k-steps and the partial results fit the context's workspace.
+int prefill_slices(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
+    const bool pair = use_pair(ctx, M);
+    const int64_t tiles = ((N + 255) / 256) * (pair ? (M + 511) / 512 : (M + 255) / 256);
+    const int64_t slots = pair ? ctx->sm_count / 2 : ctx->sm_count;
+    const int64_t ksteps = (K + 63) / 64;
+    int64_t Z = slots / tiles;
+    if (ctx->p_pf_split > 0) Z = ctx->p_pf_split;
+    if (Z > kMaxSplit) Z = kMaxSplit;
+    if (Z > ksteps / 8) Z = ksteps / 8;
+    const int64_t fit = (int64_t)(ctx->pf_ws_bytes / ((size_t)M * (size_t)N * 4));
+    if (Z > fit) Z = fit;
+    return Z < 1 ? 1 : (int)Z;
+}
+
 // M >= 9: the tensor-core kernels, or the GEMV kernel eight token rows at a time -- whichever a small cost model
 // (microseconds, constants measured on B200) says is faster.
 //   GEMV: every 8-row chunk streams the whole matrix at about 3 TB/s plus a fixed ~5 us.
@@ -95,8 +115,10 @@ bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     const bool pair = use_pair(ctx, M);
     const int64_t tiles = ((N + 255) / 256) * (pair ? (M + 511) / 512 : (M + 255) / 256);
     const int64_t slots = pair ? ctx->sm_count / 2 : ctx->sm_count;
-    const double waves = (double)((tiles + slots - 1) / slots);
-    double t_tensor = 5.0 + waves * (double)((K + 63) / 64) * 0.9;
+    const int Z = prefill_slices(ctx, M, K, N);
+    const double waves = (double)((tiles * Z + slots - 1) / slots);
+    double t_tensor = 5.0 + waves * (double)(((K + 63) / 64 + Z - 1) / Z) * 0.9;
+    if (Z > 1) t_tensor += 3.0 + (double)(Z + 1) * (double)M * (double)N * 4.0 / 5.0e6;  // partial results out and back
     if (M * K < 65536) t_tensor *= 1.45;
     return t_tensor < t_gemv;
 }
@@ -256,6 +278,12 @@ extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, in
         if ((e = cudaMalloc(&ctx->ws_edge, slot * 2 * (size_t)ctx->sm_count * kMaxCtasPerSm))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->ws_full, slot * (size_t)kMaxSplit * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->tickets, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
+        if (max_M > kMaxTokens) {
+            // K-split tensor-core calls (shapes with few output tiles): up to kMaxSplit partial results, capped
+            const size_t want = (size_t)kMaxSplit * (size_t)max_M * (size_t)max_N * 4;
+            ctx->pf_ws_bytes = want < kPrefillWsCap ? want : kPrefillWsCap;
+            if ((e = cudaMalloc(&ctx->pf_ws, ctx->pf_ws_bytes))) { st = cuda_fail(nullptr, e, ""); break; }
+        }
         if ((e = cudaMemset(ctx->tickets, 0, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
         const size_t tiles = (size_t)(max_K / kGroup), toks = (size_t)(max_M < kMaxTokens ? max_M : kMaxTokens);
         if ((e = cudaMalloc(&ctx->xq, tiles * toks * 128))) { st = cuda_fail(nullptr, e, ""); break; }
@@ -282,6 +310,7 @@ extern "C" fdqp_status fdqp_destroy(fdqp_ctx* ctx) {
     DeviceGuard guard(ctx->device);
     if (ctx->ws_edge) cudaFree(ctx->ws_edge);
     if (ctx->ws_full) cudaFree(ctx->ws_full);
+    if (ctx->pf_ws) cudaFree(ctx->pf_ws);
     if (ctx->tickets) cudaFree(ctx->tickets);
     if (ctx->xq) cudaFree(ctx->xq);
     if (ctx->xsc) cudaFree(ctx->xsc);
@@ -312,9 +341,10 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
     }
     if (use_prefill(ctx, M, K, N)) {
         // prefill-sized M: dequantise into shared memory, contract with tcgen05 (accumulators in TMEM)
-        if ((e = prefill_launch(W, x, y, ctx->status_dev, (int)M, (int)K, (int)N, use_pair(ctx, M) ? 1 : 0, stream)))
+        if ((e = prefill_launch(W, x, y, ctx->pf_ws, ctx->status_dev, (int)M, (int)K, (int)N, use_pair(ctx, M) ? 1 : 0,
+                                prefill_slices(ctx, M, K, N), stream)))
             return cuda_fail(ctx, e, "prefill kernel launch");
-        ctx->launches += 1;
+        ctx->launches += prefill_slices(ctx, M, K, N) > 1 ? 2 : 1;
         return FDQP_OK;
     }
     // Token rows are processed eight at a time by the streaming GEMV kernel.
@@ -420,6 +450,9 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
     } else if (!std::strcmp(key, "split_k")) {
         if (v != -1 && v != 1 && v != 2 && v != 4 && v != 8) return FDQP_ERR_ARG;
         ctx->p_split_k = v;
+    } else if (!std::strcmp(key, "prefill_split_k")) {
+        if (v == 0 || v > kMaxSplit) return FDQP_ERR_ARG;
+        ctx->p_pf_split = v;
     } else if (!std::strcmp(key, "prefill_pair")) {
         if (v > 1) return FDQP_ERR_ARG;
         ctx->p_pair = v;
@@ -455,13 +488,16 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
         return FDQP_OK;
     }
     if (use_prefill(ctx, M, K, N)) {
+        const int Z = prefill_slices(ctx, M, K, N);
         if (use_pair(ctx, M))
             std::snprintf(buf, buf_bytes,
-                          "fdqp_prefill_pair_kernel grid=%lld cluster=2 block=320 tile=256x512 per pair stages=4 tmem_cols=512",
-                          (long long)(2 * ((N + 255) / 256) * ((M + 511) / 512)));
+                          "fdqp_prefill_pair_kernel grid=%lld cluster=2 block=320 tile=256x512 per pair stages=4 tmem_cols=512 "
+                          "split_k=%d%s",
+                          (long long)(2 * ((N + 255) / 256) * ((M + 511) / 512) * Z), Z, Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
         else
-            std::snprintf(buf, buf_bytes, "fdqp_prefill_kernel grid=%lld block=320 tile=256x256 stages=3 tmem_cols=512",
-                          (long long)(((N + 255) / 256) * ((M + 255) / 256)));
+            std::snprintf(buf, buf_bytes,
+                          "fdqp_prefill_kernel grid=%lld block=320 tile=256x256 stages=3 tmem_cols=512 split_k=%d%s",
+                          (long long)(((N + 255) / 256) * ((M + 255) / 256) * Z), Z, Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
         return FDQP_OK;
     }
     GemvPlan plan;

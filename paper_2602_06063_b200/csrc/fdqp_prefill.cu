@@ -38,9 +38,11 @@ constexpr uint32_t kPfSmemBytes = kPfStages * kPfStageBytes + 1024 /*alignment s
 
 struct PrefillParams {
     const uint8_t* W;
-    float* y;
+    float* y;       // [M][N] result, or (Z > 1) Z partial results of that shape, one per K slice
     int* status;
     int M, K, N;
+    int Z;          // K slices; slice z covers k-steps [z * ksteps_z, (z + 1) * ksteps_z)
+    int ksteps_z;   // 64-wide k-steps per slice
 };
 
 // ---- tcgen05 wrappers -----------------------------------------------------------------------------------------
@@ -207,11 +209,15 @@ __global__ void __launch_bounds__(kPfThreads, 1)
     volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(smem + kPfStages * kPfStageBytes + 8 * (3 * kPfStages + 1));
 
     const int tok_tiles = (p.M + kPfToks - 1) / kPfToks;
-    const int n_tile = blockIdx.x / tok_tiles, tok_tile = blockIdx.x % tok_tiles;  // token tiles of one n-tile adjacent
+    const int tile_id = blockIdx.x / p.Z, z = blockIdx.x % p.Z;                    // K slices of one tile adjacent
+    const int n_tile = tile_id / tok_tiles, tok_tile = tile_id % tok_tiles;        // token tiles of one n-tile adjacent
     const int n0 = n_tile * kPfRows, tok0 = tok_tile * kPfToks;
     const int toks = (p.M - tok0) < kPfToks ? (p.M - tok0) : kPfToks;
     const uint32_t n_inst = (uint32_t)((toks + 15) & ~15);
-    const int ksteps = (p.K + kPfK - 1) / kPfK;
+    const int ksteps_all = (p.K + kPfK - 1) / kPfK;
+    const int ks0 = z * p.ksteps_z;                                                // first k-step of this slice
+    const int ksteps = (ksteps_all - ks0) < p.ksteps_z ? (ksteps_all - ks0) : p.ksteps_z;
+    float* const yout = p.y + (int64_t)z * p.M * p.N;
 
     if (tid == 0) {
         for (int s = 0; s < kPfStages; ++s) {
@@ -240,7 +246,7 @@ __global__ void __launch_bounds__(kPfThreads, 1)
                 if (i >= kPfStages) ok = mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status);
                 if (!ok) break;
                 mbar_arrive_expect_tx(full_b(s), kPfBBytes);
-                tma_load_2d(base + s * kPfStageBytes + kPfABytes, &x_map, i * kPfK, tok0, full_b(s));
+                tma_load_2d(base + s * kPfStageBytes + kPfABytes, &x_map, (ks0 + i) * kPfK, tok0, full_b(s));
             }
         }
     } else if (warp == 1) {
@@ -272,13 +278,14 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         const int64_t strip = (int64_t)n_tile * (kPfRows / 32) + dw;
         const bool strip_ok = strip < p.N / kStripRows;
         // software pipeline: the loads of the next stage are in flight while this one is converted
-        GroupRegs g0 = group_load(p.W, p.K, strip, 0, lane, strip_ok), g1 = group_load(p.W, p.K, strip, 1, lane, strip_ok);
+        GroupRegs g0 = group_load(p.W, p.K, strip, 2 * ks0, lane, strip_ok);
+        GroupRegs g1 = group_load(p.W, p.K, strip, 2 * ks0 + 1, lane, strip_ok);
         for (int i = 0; i < ksteps && ok; ++i) {
             const int s = i % kPfStages;
             GroupRegs n0r, n1r;
             if (i + 1 < ksteps) {
-                n0r = group_load(p.W, p.K, strip, 2 * (i + 1), lane, strip_ok);
-                n1r = group_load(p.W, p.K, strip, 2 * (i + 1) + 1, lane, strip_ok);
+                n0r = group_load(p.W, p.K, strip, 2 * (ks0 + i + 1), lane, strip_ok);
+                n1r = group_load(p.W, p.K, strip, 2 * (ks0 + i + 1) + 1, lane, strip_ok);
             } else {
                 n0r = g0;
                 n1r = g1;
@@ -305,14 +312,17 @@ __global__ void __launch_bounds__(kPfThreads, 1)
             // warps 2,3,4,5 have quarters 2,3,0,1 and warps 6,7,8,9 have quarters 2,3,0,1: every (half, quarter) once
             const int n = n0 + half * 128 + quarter * 32 + lane;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 256);
+            const int64_t ldy = p.N;
+            float* yrow = yout + (int64_t)tok0 * ldy + n;  // token row of column 0
             for (int c = 0; c < (int)n_inst; c += 32) {
                 uint32_t v[32];
                 tmem_ld_32cols(taddr + c, v);
                 if (n < p.N) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if (c + j < toks) p.y[(int64_t)(tok0 + c + j) * p.N + n] = __uint_as_float(v[j]);
+                        if (c + j < toks) yrow[j * ldy] = __uint_as_float(v[j]);
                 }
+                yrow += 32 * ldy;
             }
         }
     }
@@ -435,9 +445,13 @@ __global__ void __launch_bounds__(kPfThreads, 1)
     const uint32_t rank = cluster_ctarank();
     const int pair = blockIdx.x >> 1;
     const int tok_tiles = (p.M + kP2Toks - 1) / kP2Toks;
-    const int n_tile = pair / tok_tiles, tok_tile = pair % tok_tiles;
+    const int tile_id = pair / p.Z, z = pair % p.Z;
+    const int n_tile = tile_id / tok_tiles, tok_tile = tile_id % tok_tiles;
     const int n0 = n_tile * (2 * kP2Rows) + (int)rank * kP2Rows, tok0 = tok_tile * kP2Toks;
-    const int ksteps = (p.K + kPfK - 1) / kPfK;
+    const int ksteps_all = (p.K + kPfK - 1) / kPfK;
+    const int ks0 = z * p.ksteps_z;
+    const int ksteps = (ksteps_all - ks0) < p.ksteps_z ? (ksteps_all - ks0) : p.ksteps_z;
+    float* const yout = p.y + (int64_t)z * p.M * p.N;
     // tokens of the two MMAs of a k-step, rounded up to the instruction's granularity (16); the second MMA is dropped
     // when the tile has no more than 256 tokens.  Each CTA supplies half of an MMA's tokens.
     const int rem = p.M - tok0;
@@ -476,9 +490,9 @@ __global__ void __launch_bounds__(kPfThreads, 1)
                 const uint32_t b_addr = base + s * kP2StageBytes + kP2ABytes;
                 // MMA j covers tokens [256 j, 256 j + n_j): this CTA supplies n_j / 2 of them (a full 128-token box is
                 // copied; what the MMA does not read is ignored, what lies beyond M arrives as zeros)
-                tma2_load_2d(b_addr, &x_map, i * kPfK, tok0 + (int)rank * (n_mma0 / 2), bar0);
+                tma2_load_2d(b_addr, &x_map, (ks0 + i) * kPfK, tok0 + (int)rank * (n_mma0 / 2), bar0);
                 if (n_mmas == 2)
-                    tma2_load_2d(b_addr + kP2BBoxBytes, &x_map, i * kPfK, tok0 + 256 + (int)rank * (n_mma1 / 2), bar0);
+                    tma2_load_2d(b_addr + kP2BBoxBytes, &x_map, (ks0 + i) * kPfK, tok0 + 256 + (int)rank * (n_mma1 / 2), bar0);
             }
         }
     } else if (warp == 1) {
@@ -516,13 +530,14 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         const bool strip_ok = strip < p.N / kStripRows;
         // software pipeline: the loads of the next three stages are in flight while this one is converted (a stage
         // lasts well under a microsecond here, less than one trip to L2 / HBM); groups past K load as zeros
-        GroupRegs g0 = group_load(p.W, p.K, strip, gl, lane, strip_ok);
-        GroupRegs g1 = group_load(p.W, p.K, strip, 2 + gl, lane, strip_ok);
-        GroupRegs g2 = group_load(p.W, p.K, strip, 4 + gl, lane, strip_ok);
+        const int gbase = 2 * ks0 + gl;  // this warp's group in k-step i of the slice: gbase + 2 i
+        GroupRegs g0 = group_load(p.W, p.K, strip, gbase, lane, strip_ok);
+        GroupRegs g1 = group_load(p.W, p.K, strip, gbase + 2, lane, strip_ok);
+        GroupRegs g2 = group_load(p.W, p.K, strip, gbase + 4, lane, strip_ok);
         const uint32_t full_a0 = mapa_shared(full_a(0), 0);
         for (int i = 0; i < ksteps && ok; ++i) {
             const int s = i % kP2Stages;
-            const GroupRegs g3 = group_load(p.W, p.K, strip, 2 * (i + 3) + gl, lane, strip_ok);
+            const GroupRegs g3 = group_load(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
             if (i >= kP2Stages) ok = mbar_wait(empty(s), ((i / kP2Stages) - 1) & 1, p.status);
             if (!ok) break;
             group_store(base + s * kP2StageBytes, g0, sl, gl, lane);
@@ -543,14 +558,17 @@ __global__ void __launch_bounds__(kPfThreads, 1)
             const int n = n0 + quarter * 32 + lane;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(chalf * 256);
             const int toks = p.M - tok0 - chalf * 256;  // tokens of this column half that exist
+            const int64_t ldy = p.N;
+            float* yrow = yout + (int64_t)(tok0 + chalf * 256) * ldy + n;  // token row of column 0 of this half
             for (int c = 0; c < 256 && c < toks; c += 32) {
                 uint32_t v[32];
                 tmem_ld_32cols(taddr + c, v);
                 if (n < p.N) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if (c + j < toks) p.y[(int64_t)(tok0 + chalf * 256 + c + j) * p.N + n] = __uint_as_float(v[j]);
+                        if (c + j < toks) yrow[j * ldy] = __uint_as_float(v[j]);
                 }
+                yrow += 32 * ldy;
             }
         }
     }
@@ -561,6 +579,22 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         tc_fence_after();
         tmem_dealloc2(tmem_base, kPfTmemCols);
     }
+}
+
+// Second phase of a K-split call: y = sum over slices z (ascending) of the partial results; four outputs per thread.
+__global__ void __launch_bounds__(256) fdqp_prefill_sum_kernel(const float4* __restrict__ ws, float4* __restrict__ y, int Z,
+                                                                int64_t quads) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= quads) return;
+    float4 acc = ws[i];
+    for (int z = 1; z < Z; ++z) {
+        const float4 v = ws[(int64_t)z * quads + i];
+        acc.x += v.x;
+        acc.y += v.y;
+        acc.z += v.z;
+        acc.w += v.w;
+    }
+    y[i] = acc;
 }
 
 // ---- host side ----------------------------------------------------------------------------------------------------
@@ -589,8 +623,10 @@ cudaError_t prefill_set_smem_limit() {
 
 // x: [M][K] bf16 row-major (device).  Returns cudaErrorNotSupported if the tensor map cannot be built.
 // pair != 0: the two-SM kernel (256 x 512 tiles per CTA pair), meant for M > 256.
-cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, int* status, int M, int K, int N, int pair,
-                           cudaStream_t stream) {
+// Z > 1: K is cut into Z slices (tiles x Z CTAs or CTA pairs), their partial results go to `ws` ([Z][M][N] floats) and a
+// second kernel adds them in slice order into y.  For shapes with too few tiles to fill the GPU.
+cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, float* ws, int* status, int M, int K, int N, int pair,
+                           int Z, cudaStream_t stream) {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     CUtensorMap map;
@@ -603,16 +639,22 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, int* s
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
     PrefillParams p;
+    const int ksteps_all = (K + kPfK - 1) / kPfK;
+    if (Z < 1 || Z > ksteps_all || !ws) Z = 1;
     p.W = W;
-    p.y = y;
+    p.y = Z > 1 ? ws : y;
     p.status = status;
     p.M = M;
     p.K = K;
     p.N = N;
+    p.ksteps_z = (ksteps_all + Z - 1) / Z;
+    p.Z = (ksteps_all + p.ksteps_z - 1) / p.ksteps_z;  // no empty slice
+    Z = p.Z;
+    cudaError_t err;
     if (pair) {
         const int n_tiles = (N + 2 * kP2Rows - 1) / (2 * kP2Rows), tok_tiles = (M + kP2Toks - 1) / kP2Toks;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(2 * n_tiles * tok_tiles));
+        cfg.gridDim = dim3((unsigned)(2 * n_tiles * tok_tiles * Z));
         cfg.blockDim = dim3((unsigned)kPfThreads);
         cfg.dynamicSmemBytes = kP2SmemBytes;
         cfg.stream = stream;
@@ -623,10 +665,16 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, int* s
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, fdqp_prefill_pair_kernel, map, p);
+        err = cudaLaunchKernelEx(&cfg, fdqp_prefill_pair_kernel, map, p);
+    } else {
+        const int n_tiles = (N + kPfRows - 1) / kPfRows, tok_tiles = (M + kPfToks - 1) / kPfToks;
+        fdqp_prefill_kernel<<<n_tiles * tok_tiles * Z, kPfThreads, kPfSmemBytes, stream>>>(map, p);
+        err = cudaGetLastError();
     }
-    const int n_tiles = (N + kPfRows - 1) / kPfRows, tok_tiles = (M + kPfToks - 1) / kPfToks;
-    fdqp_prefill_kernel<<<n_tiles * tok_tiles, kPfThreads, kPfSmemBytes, stream>>>(map, p);
+    if (err != cudaSuccess || Z == 1) return err;
+    const int64_t quads = (int64_t)M * N / 4;  // N is a multiple of 32
+    fdqp_prefill_sum_kernel<<<(unsigned)((quads + 255) / 256), 256, 0, stream>>>(reinterpret_cast<const float4*>(ws),
+                                                                                reinterpret_cast<float4*>(y), Z, quads);
     return cudaGetLastError();
 }
 

@@ -25,10 +25,10 @@ def ctx():
 @pytest.fixture()
 def fresh(ctx):
     """The shared context with every launch parameter back to automatic."""
-    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp", "prefill_pair"):
+    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp", "prefill_pair", "prefill_split_k"):
         fd.fdqp_set_param(ctx, key, -1)
     yield ctx
-    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp", "prefill_pair"):
+    for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp", "prefill_pair", "prefill_split_k"):
         fd.fdqp_set_param(ctx, key, -1)
 
 
@@ -122,6 +122,25 @@ def test_prefill_tensor_path_matches_oracle(fresh, K, N, M):
     fd.fdqp_set_param(fresh, "path", 2)
     assert "fdqp_gemv_kernel" in fd.fdqp_describe(fresh, M, K, N)
     assert_close(case.run(fresh), y_ref, a_ref, f"gemv-chunked K={K} N={N} M={M}")
+
+
+@pytest.mark.parametrize("K,N,M,Z", [(2048, 256, 64, 4), (2112, 544, 300, 3), (4096, 288, 512, 8), (1024, 32, 40, 2)])
+def test_prefill_k_slices(fresh, K, N, M, Z):
+    # few output tiles: K is cut into slices whose partial results a second kernel adds in slice order
+    case = Case(K, N, M, seed=3000 + K + N + M)
+    fd.fdqp_set_param(fresh, "path", 3)
+    y_ref, a_ref = case.reference()
+    auto = fd.fdqp_describe(fresh, M, K, N)
+    assert "split_k=" in auto and "split_k=1" not in auto      # such shapes are split without being asked
+    y_auto = case.run(fresh)
+    assert_close(y_auto, y_ref, a_ref, f"prefill auto split K={K} N={N} M={M}")
+    fd.fdqp_set_param(fresh, "prefill_split_k", Z)
+    assert f"split_k={Z}" in fd.fdqp_describe(fresh, M, K, N)
+    y_z = case.run(fresh)
+    assert_close(y_z, y_ref, a_ref, f"prefill split_k={Z} K={K} N={N} M={M}")
+    assert np.array_equal(y_z, case.run(fresh))                 # fixed summation order: reruns are bit-identical
+    fd.fdqp_set_param(fresh, "prefill_split_k", 1)
+    assert_close(case.run(fresh), y_ref, a_ref, f"prefill unsplit K={K} N={N} M={M}")
 
 
 def test_prefill_exact_cases(fresh):
