@@ -278,29 +278,28 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         const int64_t strip = (int64_t)n_tile * (kPfRows / 32) + dw;
         const bool strip_ok = strip < p.N / kStripRows;
         // software pipeline: the loads of the next stage are in flight while this one is converted
-        GroupRegs g0 = group_load(p.W, p.K, strip, 2 * ks0, lane, strip_ok);
-        GroupRegs g1 = group_load(p.W, p.K, strip, 2 * ks0 + 1, lane, strip_ok);
+        // the loads of the next two stages are in flight while this one is converted (a stage lasts about as long as
+        // one trip to HBM); groups past K load as zeros
+        const int g00 = 2 * ks0;
+        GroupRegs a0 = group_load(p.W, p.K, strip, g00, lane, strip_ok), a1 = group_load(p.W, p.K, strip, g00 + 1, lane, strip_ok);
+        GroupRegs b0 = group_load(p.W, p.K, strip, g00 + 2, lane, strip_ok), b1 = group_load(p.W, p.K, strip, g00 + 3, lane, strip_ok);
         for (int i = 0; i < ksteps && ok; ++i) {
             const int s = i % kPfStages;
-            GroupRegs n0r, n1r;
-            if (i + 1 < ksteps) {
-                n0r = group_load(p.W, p.K, strip, 2 * (ks0 + i + 1), lane, strip_ok);
-                n1r = group_load(p.W, p.K, strip, 2 * (ks0 + i + 1) + 1, lane, strip_ok);
-            } else {
-                n0r = g0;
-                n1r = g1;
-            }
+            const GroupRegs c0 = group_load(p.W, p.K, strip, g00 + 2 * (i + 2), lane, strip_ok);
+            const GroupRegs c1 = group_load(p.W, p.K, strip, g00 + 2 * (i + 2) + 1, lane, strip_ok);
             if (i >= kPfStages) ok = mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status);
             if (!ok) break;
             const uint32_t a_tile = base + s * kPfStageBytes;
-            group_store(a_tile, g0, dw, 0, lane);
-            group_store(a_tile, g1, dw, 1, lane);
+            group_store(a_tile, a0, dw, 0, lane);
+            group_store(a_tile, a1, dw, 1, lane);
             // make the generic-proxy stores visible to the tensor core's (async-proxy) reads, then signal
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(full_a(s));
-            g0 = n0r;
-            g1 = n1r;
+            a0 = b0;
+            a1 = b1;
+            b0 = c0;
+            b1 = c1;
         }
         // =============================== epilogue: TMEM -> y =================================================
         if (ok) ok = mbar_wait(acc_done, 0, p.status);
