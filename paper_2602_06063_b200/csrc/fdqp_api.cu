@@ -496,7 +496,7 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
                           (long long)(2 * ((N + 255) / 256) * ((M + 511) / 512) * Z), Z, Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
         else
             std::snprintf(buf, buf_bytes,
-                          "fdqp_prefill_kernel grid=%lld block=320 tile=256x256 stages=3 tmem_cols=512 split_k=%d%s",
+                          "fdqp_prefill_kernel grid=%lld block=576 tile=256x256 stages=3 tmem_cols=512 split_k=%d%s",
                           (long long)(((N + 255) / 256) * ((M + 255) / 256) * Z), Z, Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
         return FDQP_OK;
     }

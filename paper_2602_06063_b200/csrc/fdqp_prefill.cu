@@ -31,8 +31,10 @@ constexpr int kPfStages = 3;
 constexpr uint32_t kPfABytes = kPfRows * kPfK * 2;  // 32 KB
 constexpr uint32_t kPfBBytes = kPfToks * kPfK * 2;  // 32 KB
 constexpr uint32_t kPfStageBytes = kPfABytes + kPfBBytes;
-constexpr int kPfDequantWarps = 8;
+constexpr int kPfDequantWarps = 8;   // two-SM kernel: one (strip, group) of the CTA's 128 rows each
 constexpr int kPfThreads = (2 + kPfDequantWarps) * 32;  // warp 0: TMA + TMEM owner, warp 1: MMA issuer
+constexpr int kPf1DequantWarps = 16;  // one-SM kernel: one (strip, group) of the CTA's 256 rows each
+constexpr int kPf1Threads = (2 + kPf1DequantWarps) * 32;
 constexpr uint32_t kPfTmemCols = 512;
 constexpr uint32_t kPfSmemBytes = kPfStages * kPfStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
@@ -191,7 +193,7 @@ __device__ __forceinline__ void group_store(uint32_t a_tile, const GroupRegs& r,
 
 // ---- the kernel -------------------------------------------------------------------------------------------------------
 
-__global__ void __launch_bounds__(kPfThreads, 1)
+__global__ void __launch_bounds__(kPf1Threads, 1)
     fdqp_prefill_kernel(const __grid_constant__ CUtensorMap x_map, const PrefillParams p) {
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -221,7 +223,7 @@ __global__ void __launch_bounds__(kPfThreads, 1)
 
     if (tid == 0) {
         for (int s = 0; s < kPfStages; ++s) {
-            mbar_init(full_a(s), kPfDequantWarps);
+            mbar_init(full_a(s), kPf1DequantWarps);
             mbar_init(full_b(s), 1);
             mbar_init(empty(s), 1);
         }
@@ -274,32 +276,29 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         }
     } else {
         // =============================== dequantisation warps ================================================
-        const int dw = warp - 2;  // strip of the tile this warp owns
-        const int64_t strip = (int64_t)n_tile * (kPfRows / 32) + dw;
+        const int dw = warp - 2;
+        const int sl = dw >> 1, gl = dw & 1;  // strip of the tile and group of the 64-k stage this warp converts
+        const int64_t strip = (int64_t)n_tile * (kPfRows / 32) + sl;
         const bool strip_ok = strip < p.N / kStripRows;
-        // software pipeline: the loads of the next stage are in flight while this one is converted
-        // the loads of the next two stages are in flight while this one is converted (a stage lasts about as long as
-        // one trip to HBM); groups past K load as zeros
-        const int g00 = 2 * ks0;
-        GroupRegs a0 = group_load(p.W, p.K, strip, g00, lane, strip_ok), a1 = group_load(p.W, p.K, strip, g00 + 1, lane, strip_ok);
-        GroupRegs b0 = group_load(p.W, p.K, strip, g00 + 2, lane, strip_ok), b1 = group_load(p.W, p.K, strip, g00 + 3, lane, strip_ok);
+        // the loads of the next three stages are in flight while this one is converted (a stage lasts about as long
+        // as one trip to HBM); groups past K load as zeros
+        const int gbase = 2 * ks0 + gl;  // this warp's group in k-step i of the slice: gbase + 2 i
+        GroupRegs g0 = group_load(p.W, p.K, strip, gbase, lane, strip_ok);
+        GroupRegs g1 = group_load(p.W, p.K, strip, gbase + 2, lane, strip_ok);
+        GroupRegs g2 = group_load(p.W, p.K, strip, gbase + 4, lane, strip_ok);
         for (int i = 0; i < ksteps && ok; ++i) {
             const int s = i % kPfStages;
-            const GroupRegs c0 = group_load(p.W, p.K, strip, g00 + 2 * (i + 2), lane, strip_ok);
-            const GroupRegs c1 = group_load(p.W, p.K, strip, g00 + 2 * (i + 2) + 1, lane, strip_ok);
+            const GroupRegs g3 = group_load(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
             if (i >= kPfStages) ok = mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status);
             if (!ok) break;
-            const uint32_t a_tile = base + s * kPfStageBytes;
-            group_store(a_tile, a0, dw, 0, lane);
-            group_store(a_tile, a1, dw, 1, lane);
+            group_store(base + s * kPfStageBytes, g0, sl, gl, lane);
             // make the generic-proxy stores visible to the tensor core's (async-proxy) reads, then signal
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(full_a(s));
-            a0 = b0;
-            a1 = b1;
-            b0 = c0;
-            b1 = c1;
+            g0 = g1;
+            g1 = g2;
+            g2 = g3;
         }
         // =============================== epilogue: TMEM -> y =================================================
         if (ok) ok = mbar_wait(acc_done, 0, p.status);
@@ -307,19 +306,21 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         if (ok) {
             tc_fence_after();
             const int quarter = warp & 3;        // TMEM lanes this warp may read
-            const int half = dw >> 2;            // which accumulator: warps 2..5 -> 0, 6..9 -> 1 ... by construction below
-            // warps 2,3,4,5 have quarters 2,3,0,1 and warps 6,7,8,9 have quarters 2,3,0,1: every (half, quarter) once
+            // the four warps of a quarter (dw = quarter', quarter' + 4, + 8, + 12) take (accumulator, column half)
+            const int half = (dw >> 2) & 1, chalf = dw >> 3;
             const int n = n0 + half * 128 + quarter * 32 + lane;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 256);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 256 + chalf * 128);
+            const int c_end = ((int)n_inst < chalf * 128 + 128 ? (int)n_inst : chalf * 128 + 128) - chalf * 128;
             const int64_t ldy = p.N;
-            float* yrow = yout + (int64_t)tok0 * ldy + n;  // token row of column 0
-            for (int c = 0; c < (int)n_inst; c += 32) {
+            float* yrow = yout + (int64_t)(tok0 + chalf * 128) * ldy + n;  // token row of this warp's column 0
+            const int toks_h = toks - chalf * 128;                          // tokens of this column half that exist
+            for (int c = 0; c < c_end; c += 32) {
                 uint32_t v[32];
                 tmem_ld_32cols(taddr + c, v);
                 if (n < p.N) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if (c + j < toks) yrow[j * ldy] = __uint_as_float(v[j]);
+                        if (c + j < toks_h) yrow[j * ldy] = __uint_as_float(v[j]);
                 }
                 yrow += 32 * ldy;
             }
@@ -667,7 +668,7 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, float*
         err = cudaLaunchKernelEx(&cfg, fdqp_prefill_pair_kernel, map, p);
     } else {
         const int n_tiles = (N + kPfRows - 1) / kPfRows, tok_tiles = (M + kPfToks - 1) / kPfToks;
-        fdqp_prefill_kernel<<<n_tiles * tok_tiles * Z, kPfThreads, kPfSmemBytes, stream>>>(map, p);
+        fdqp_prefill_kernel<<<n_tiles * tok_tiles * Z, kPf1Threads, kPfSmemBytes, stream>>>(map, p);
         err = cudaGetLastError();
     }
     if (err != cudaSuccess || Z == 1) return err;
