@@ -121,12 +121,15 @@ FDQP_API fdqp_status fdqp_destroy(fdqp_ctx* ctx);
  * Dispatch: M = 1 and 2..8 run the streaming GEMV kernels (weights fetched once
  * from HBM through a shared-memory ring, nibbles unpacked in registers, scale and
  * offset applied in fp32, split-K across CTAs reduced in a fixed order); M >= 9
- * runs the dequantise-into-shared-memory tensor-core path (tcgen05, accumulators
- * in TMEM) when its 256 x 256 output tiles can fill at least half of the SMs or
- * M > 128, and otherwise the GEMV kernel eight token rows at a time.
- * In the GEMV kernels the activations of each 32-group are held as 24-bit fixed
- * point relative to the group's largest exponent: exact for every element within
- * 2^15 of the group's largest magnitude, rounded to 2^-23 of it otherwise.
+ * runs either the dequantise-into-shared-memory tensor-core path (tcgen05,
+ * accumulators in TMEM; a one-SM kernel up to 256 token rows, a two-SM kernel
+ * above; K cut into slices when a shape has few output tiles) or the GEMV kernel
+ * eight token rows at a time, whichever a small cost model expects to be faster
+ * (GEMV chunks up to about 16-24 rows, or more when N is small).
+ * In the GEMV kernels the activations of each 32-group are held as fixed point
+ * relative to the group's largest exponent (22 fraction bits below it): exact for
+ * every element within 2^14 of the group's largest magnitude, rounded to 2^-22 of
+ * that magnitude otherwise.
  * Asynchronous on `cuda_stream`; no allocation and no host synchronisation.  W, x
  * and y must stay valid until the stream has passed the call.  Two calls that
  * share a context must be ordered on one stream.

@@ -10,31 +10,33 @@
 // (mma.sync m16n8k32, u8 x s8/u8 -> s32): the 4-bit codes become bytes with two logic ops per four
 // codes (w & 0x0F0F0F0F, (w >> 4) & 0x0F0F0F0F -- B200 issues integer/logic instructions at half the
 // fp32 rate, so this unpack is the budget that matters), and the activations of a group are held as
-// 24-bit fixed point relative to the group's largest exponent, split into three byte planes
+// fixed point relative to the group's largest exponent (|value| <= 2^22), split into three byte planes
 // (x = 2^e_g * (65536 p2 + 256 p1 + p0), p2 signed, p1 and p0 unsigned; exact for every element
 // within 2^14 of the group's largest, rounded to 2^-22 of it otherwise).  One MMA covers a whole
 // group of 16 output rows; its s32 result is exact.  The order of k inside a group is a free
 // permutation as long as both operands use the same one (even k in the low half, odd k in the high).
 // The plane sums are recombined in int32 (they fit) and converted to fp32 once per value.
-// For M <= 4 most of the MMA's eight token columns would be idle, so the three planes of a token ride in
+// For M <= 2 most of the MMA's eight token columns would be idle, so the three planes of a token ride in
 // three columns (as signed digits; column 3 / 7 is zero): one MMA per 16 rows yields all three plane sums
 // of up to TWO tokens (kernel modes: 1 = one token, 3 = two tokens).  Mode 2 (M = 3..8) issues one MMA per plane
 // with the eight tokens as columns; measured on B200 it beats two column-mode MMAs from M = 3 on.
 //
-// The plane split of x is done once per call by a small preparation kernel; every GEMV CTA then
-// brings its K slice of the prepared x into shared memory with bulk async copies.
+// The plane split of x is done by every GEMV CTA itself when its K slice is short (one work item per
+// consumer thread at most), else once per call by a small preparation kernel, after which every GEMV
+// CTA brings its K slice of the prepared x into shared memory with bulk async copies.
 //
 // Data movement.  The packed matrix is strip-major (32 output rows x all of K contiguous), so every
 // CTA streams one contiguous byte range of HBM exactly once.  The producer warp issues one 1-D bulk
 // async copy per Q4NX block (<= 5120 bytes), several lanes at a time, into a shared-memory ring of
 // multi-block stages guarded by mbarriers; every consumer warp owns the same 32 x 32 group-tile of
-// two blocks of a stage.
+// two or four blocks of a stage.
 //
 // Work split.  The (K-slice, strip, block) space is cut into equal contiguous ranges, one per
 // persistent CTA, so all SMs stream the same number of bytes whatever N and K are.  A strip whose
 // blocks end up in several CTAs (or several K slices) is completed by whichever CTA arrives last at
 // the strip's ticket: it sums the partial rows in a fixed order, so results are reproducible run to
-// run.  A CTA handles the shared strip at the END of its range FIRST, so that the exchange through
+// run (K slices, used only when the prepared x of the whole K would not fit beside the ring, are
+// strip-aligned and added by fdqp_splitk_sum_kernel instead).  A CTA handles the shared strip at the END of its range FIRST, so that the exchange through
 // global memory is off its critical path and its last piece is a whole strip written directly.
 // No CTA ever waits for another CTA.
 #include "fdqp_device.cuh"
