@@ -19,9 +19,8 @@ cudaError_t splitk_sum_launch(const float* ws, float* y, int Z, int S, int M, in
 cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream);
 cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
 cudaError_t prefill_set_smem_limit();
-cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, float* ws, int* status, int M, int K, int N, int pair,
-                           int Z,
-                           cudaStream_t stream);
+cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, float* ws, int* status, int M,
+                           int K, int N, int pair, int Z, cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
 }  // namespace fdqp
 
@@ -35,6 +34,7 @@ struct fdqp_ctx {
     float* ws_edge = nullptr;
     float* ws_full = nullptr;
     float* pf_ws = nullptr;      // partial results of K-split tensor-core calls
+    uint8_t* x_spread = nullptr; // small x copied with its rows further apart (see kSpreadBelowBytes)
     size_t pf_ws_bytes = 0;
     int* tickets = nullptr;
     uint32_t* xq = nullptr;      // prepared activations of the call in flight
@@ -53,6 +53,12 @@ namespace {
 
 constexpr int kMaxStages = 40;
 constexpr double kTwoCtaBytes = 256e6;
+// Measured on B200: while all of x is smaller than 128 KB, the tensor-core kernels (every CTA re-reads the same few rows
+// of x by TMA at every k-step) run 1.45x slower; with the same rows placed further apart, so that they cover at least
+// 256 KB of addresses, the slow-down is gone.  Such an x is therefore copied into a spread-out staging buffer first.
+constexpr int64_t kSpreadBelowBytes = 128 << 10;
+constexpr int64_t kSpreadToBytes = 256 << 10;
+constexpr size_t kSpreadBufBytes = (size_t)kSpreadToBytes + 256 * 128;  // row distance rounds up to 128 bytes, M <= 256 here
 constexpr size_t kPrefillWsCap = 128u << 20;  // bytes of partial results a context keeps for K-split tensor-core calls
 constexpr int kMinStages = 3;  // ring depth below which another K slice is preferred
 
@@ -104,22 +110,24 @@ int prefill_slices(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
 
 // M >= 9: the tensor-core kernels, or the GEMV kernel eight token rows at a time -- whichever a small cost model
 // (microseconds, constants measured on B200) says is faster.
-//   GEMV: every 8-row chunk streams the whole matrix at about 3 TB/s plus a fixed ~5 us.
-//   Tensor-core kernels: limited by converting the weights, ~0.9 us per 64-wide k-step per wave of tiles, whatever M is;
-//   measured 1.45x slower while the whole of x is smaller than 128 KB.
+//   GEMV: every chunk streams the whole matrix, at about 5.5 TB/s for 1-2 rows, 3.9 for 3-4, 3.2 for 5-8, plus ~5 us.
+//   Tensor-core kernels: limited by converting the weights: per wave of tiles and 64-wide k-step ~0.78 us (one-SM
+//   kernel) or ~0.95 us (two-SM kernel, which also has twice the tokens' MMAs to issue), whatever M is.
 bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     if (M <= kMaxTokens || ctx->p_path == 2) return false;
     if (ctx->p_path == 3) return true;
-    const double chunks = (double)((M + kMaxTokens - 1) / kMaxTokens);
-    const double t_gemv = chunks * (5.0 + 0.625 * (double)K * (double)N / 3.0e6);
+    const double mb = 0.625 * (double)K * (double)N / 1.0e6;  // packed weights, bytes per microsecond = TB/s * 1e6
+    const int64_t last = M % kMaxTokens;                       // rows of the ragged last chunk (0: none)
+    const double last_rate = last <= 2 ? 5.5 : (last <= 4 ? 3.9 : 3.2);
+    const double t_gemv = (double)(M / kMaxTokens) * (5.0 + mb / 3.2) + (last ? 5.0 + mb / last_rate : 0.0);
     const bool pair = use_pair(ctx, M);
     const int64_t tiles = ((N + 255) / 256) * (pair ? (M + 511) / 512 : (M + 255) / 256);
     const int64_t slots = pair ? ctx->sm_count / 2 : ctx->sm_count;
     const int Z = prefill_slices(ctx, M, K, N);
     const double waves = (double)((tiles * Z + slots - 1) / slots);
-    double t_tensor = 5.0 + waves * (double)(((K + 63) / 64 + Z - 1) / Z) * 0.9;
+    double t_tensor = 5.0 + waves * (double)(((K + 63) / 64 + Z - 1) / Z) * (pair ? 0.95 : 0.78);
     if (Z > 1) t_tensor += 3.0 + (double)(Z + 1) * (double)M * (double)N * 4.0 / 5.0e6;  // partial results out and back
-    if (M * K < 65536) t_tensor *= 1.45;
+    if (M * K * 2 < kSpreadBelowBytes) t_tensor += 3.0;                                   // the spreading copy
     return t_tensor < t_gemv;
 }
 
@@ -283,6 +291,7 @@ extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, in
             const size_t want = (size_t)kMaxSplit * (size_t)max_M * (size_t)max_N * 4;
             ctx->pf_ws_bytes = want < kPrefillWsCap ? want : kPrefillWsCap;
             if ((e = cudaMalloc(&ctx->pf_ws, ctx->pf_ws_bytes))) { st = cuda_fail(nullptr, e, ""); break; }
+            if ((e = cudaMalloc(&ctx->x_spread, kSpreadBufBytes))) { st = cuda_fail(nullptr, e, ""); break; }
         }
         if ((e = cudaMemset(ctx->tickets, 0, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
         const size_t tiles = (size_t)(max_K / kGroup), toks = (size_t)(max_M < kMaxTokens ? max_M : kMaxTokens);
@@ -311,6 +320,7 @@ extern "C" fdqp_status fdqp_destroy(fdqp_ctx* ctx) {
     if (ctx->ws_edge) cudaFree(ctx->ws_edge);
     if (ctx->ws_full) cudaFree(ctx->ws_full);
     if (ctx->pf_ws) cudaFree(ctx->pf_ws);
+    if (ctx->x_spread) cudaFree(ctx->x_spread);
     if (ctx->tickets) cudaFree(ctx->tickets);
     if (ctx->xq) cudaFree(ctx->xq);
     if (ctx->xsc) cudaFree(ctx->xsc);
@@ -341,8 +351,17 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
     }
     if (use_prefill(ctx, M, K, N)) {
         // prefill-sized M: dequantise into shared memory, contract with tcgen05 (accumulators in TMEM)
-        if ((e = prefill_launch(W, x, y, ctx->pf_ws, ctx->status_dev, (int)M, (int)K, (int)N, use_pair(ctx, M) ? 1 : 0,
-                                prefill_slices(ctx, M, K, N), stream)))
+        const uint16_t* xt = x;
+        int64_t x_row_bytes = K * 2;
+        if (M * K * 2 < kSpreadBelowBytes && ctx->x_spread) {
+            x_row_bytes = ((kSpreadToBytes + M - 1) / M + 127) / 128 * 128;
+            if ((e = cudaMemcpy2DAsync(ctx->x_spread, (size_t)x_row_bytes, x, (size_t)K * 2, (size_t)K * 2, (size_t)M,
+                                       cudaMemcpyDeviceToDevice, stream)))
+                return cuda_fail(ctx, e, "x spreading copy");
+            xt = reinterpret_cast<const uint16_t*>(ctx->x_spread);
+        }
+        if ((e = prefill_launch(W, xt, x_row_bytes, y, ctx->pf_ws, ctx->status_dev, (int)M, (int)K, (int)N,
+                                use_pair(ctx, M) ? 1 : 0, prefill_slices(ctx, M, K, N), stream)))
             return cuda_fail(ctx, e, "prefill kernel launch");
         ctx->launches += prefill_slices(ctx, M, K, N) > 1 ? 2 : 1;
         return FDQP_OK;

@@ -625,13 +625,14 @@ cudaError_t prefill_set_smem_limit() {
 // pair != 0: the two-SM kernel (256 x 512 tiles per CTA pair), meant for M > 256.
 // Z > 1: K is cut into Z slices (tiles x Z CTAs or CTA pairs), their partial results go to `ws` ([Z][M][N] floats) and a
 // second kernel adds them in slice order into y.  For shapes with too few tiles to fill the GPU.
-cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, float* y, float* ws, int* status, int M, int K, int N, int pair,
-                           int Z, cudaStream_t stream) {
+// x_row_bytes: distance between token rows of x (K * 2 for a dense [M][K] array; a multiple of 16).
+cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, float* ws, int* status, int M,
+                           int K, int N, int pair, int Z, cudaStream_t stream) {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};      // innermost first
-    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};              // bytes between token rows
+    const cuuint64_t strides[1] = {(cuuint64_t)x_row_bytes};        // bytes between token rows
     const cuuint32_t box[2] = {(cuuint32_t)kPfK, (cuuint32_t)(pair ? kP2TokBox : kPfToks)};
     const cuuint32_t elem[2] = {1, 1};
     if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t*>(x), dims, strides, box, elem,
