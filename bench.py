@@ -73,7 +73,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -484,8 +484,8 @@ def run_ours(args, rank, local_rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=8000)
+    ap.add_argument("--warmup", type=int, default=40)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--graph", type=int, default=1, help="replay each step from a CUDA graph (default 1)")
     ap.add_argument("--fuse", type=int, default=1, help="run q|k|v and gate|up as one call each (default 1)")
@@ -499,14 +499,14 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
-        if args.steps == 400 and args.warmup == 20:
+        if args.steps == 8000 and args.warmup == 40:
             args.steps, args.warmup = 5, 1
         run_reference(args, rank, world)
         return
     if args.warmup < 3:
         args.warmup = 3
     if args.shape:
-        if args.steps == 400:
+        if args.steps == 8000:
             args.steps = 50
         run_shape(args)
         return
