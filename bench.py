@@ -398,6 +398,49 @@ def run_ours(args, rank, local_rank, world):
         stream.synchronize()
         head_ms = h0.elapsed_time(h1) / 10
 
+    # ---- the same projections at M = 8 (batched decode): one graph pass over the weight copies, LM head directly
+    batch8 = None
+    if rank == 0 and not args.no_head:
+        M8 = 8
+        xs8 = [torch.from_numpy(synthgen.activations(seed, M8, K).view(np.int16)).cuda() for _, K, _, seed in shapes]
+        ys8 = [torch.empty((M8, N), dtype=torch.float32, device="cuda") for _, _, N, _ in shapes]
+
+        def enqueue_layer8(c):
+            for i, (_, K, N, _) in enumerate(shapes):
+                fd.fdqp_run(ctx, xs8[i], copies[c][i], ys8[i], M8, K, N, sraw)
+
+        with torch.cuda.stream(stream):
+            enqueue_layer8(0)
+        stream.synchronize()
+        g8 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g8, stream=stream):
+            for c in range(LAYER_COPIES):
+                enqueue_layer8(c)
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                g8.replay()
+            b0.record(stream)
+            for _ in range(20):
+                g8.replay()
+            b1.record(stream)
+        stream.synchronize()
+        layer8_ms = b0.elapsed_time(b1) / (20 * LAYER_COPIES)
+        hx8 = torch.from_numpy(synthgen.activations(hseed, M8, hk).view(np.int16)).cuda()
+        hy8 = torch.empty((M8, hn), dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            fd.fdqp_run(ctx, hx8, hW, hy8, M8, hk, hn, sraw)
+        b0.record(stream)
+        for _ in range(10):
+            fd.fdqp_run(ctx, hx8, hW, hy8, M8, hk, hn, sraw)
+        b1.record(stream)
+        stream.synchronize()
+        head8_ms = b0.elapsed_time(b1) / 10
+        batch8 = {"M": M8, "layer_ms": layer8_ms, "lm_head_ms": head8_ms,
+                  "layer_gbs": layer_bytes(M8) / (layer8_ms * 1e-3) / 1e9,
+                  "decode_tokens_per_s": M8 * 1e3 / (synthgen.GEMMA3_4B_LAYERS * layer8_ms + head8_ms)}
+        del xs8, ys8, hx8, hy8
+
     # ---- LM head at a prefill chunk (M = 512, BASELINE configs[4]): the tensor-core path, against the tensor roofline
     prefill = None
     if rank == 0 and not args.no_head:
@@ -467,6 +510,7 @@ def run_ours(args, rank, local_rank, world):
                          # algorithmic bytes; traffic grows in proportion to 0.625*K*N, so scale to this call size
                          "traffic": 1.024 * step_bytes / calls_per_step, "peak_kind": peak_kind + " copy bandwidth",
                          "kernel": "fdqp_gemv_kernel", "launch_us": per_launch_us},
+            "batched_decode": batch8,
             "prefill_lm_head": prefill,
             "cpu_baseline": cpu,
             "e2e": {"value": whole_job_gbs(step_bytes, e2e_steps, world, e2e_s * 1e3), "unit": "GB/s",
