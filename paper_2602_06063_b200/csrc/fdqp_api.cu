@@ -52,7 +52,6 @@ struct fdqp_ctx {
 namespace {
 
 constexpr int kMaxStages = 40;
-constexpr double kTwoCtaBytes = 256e6;
 // Measured on B200: while all of x is smaller than 128 KB, the tensor-core kernels (every CTA re-reads the same few rows
 // of x by TMA at every k-step) run 1.45x slower; with the same rows placed further apart, so that they cover at least
 // 256 KB of addresses, the slow-down is gone.  Such an x is therefore copied into a spread-out staging buffer first.
@@ -160,11 +159,9 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     p->N = N;
     p->S = N / kStripRows;
     p->nb = (K + kBlockK - 1) / kBlockK;
-    // measured on B200: one 19-warp CTA per SM (one start-up per SM, all of its shared memory) is the better shape
-    // except for very large matrices at M = 1, where two 10-warp CTAs per SM stream ~2 % faster
-    const double packed_bytes = 0.625 * (double)K * (double)N;
-    int ctas_per_sm = ctx->p_ctas_per_sm > 0 ? (int)ctx->p_ctas_per_sm
-                                             : (M == 1 && ctx->p_cw != 16 && packed_bytes >= kTwoCtaBytes ? 2 : 1);
+    // measured on B200: one 19-warp CTA per SM (one start-up per SM, all of its shared memory) is the better shape at
+    // every size; two 10-warp CTAs per SM remain available as a launch parameter
+    int ctas_per_sm = ctx->p_ctas_per_sm > 0 ? (int)ctx->p_ctas_per_sm : 1;
     if (ctas_per_sm > kMaxCtasPerSm) ctas_per_sm = kMaxCtasPerSm;
     int cw = 16, Z = 1, nbz = p->nb, bpw = 2;
     SmemLayout L{};
@@ -204,7 +201,9 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     {
         const double t_block = 0.125 * ctas_per_sm;  // one 5 KB block at an SM's share of HBM bandwidth
         const int64_t blocks_bal = (total_blocks / Z + Gz - 1) / Gz;
-        const double cost_bal = blocks_bal * t_block + (blocks_bal >= 2 * (int64_t)nbz ? 0.6 : 2.0);
+        // (measured: ranges cut inside strips also stream ~4 % slower up to M = 4 -- strip boundaries then fall at odd
+        // places inside the stages, and more stages take the bookkeeping path)
+        const double cost_bal = blocks_bal * t_block * (M <= 4 ? 1.04 : 1.0) + (blocks_bal >= 2 * (int64_t)nbz ? 0.6 : 2.0);
         const int Ga = Gz < p->S ? Gz : p->S;
         const int64_t blocks_al = (int64_t)((p->S + Ga - 1) / Ga) * nbz;
         const double cost_al = blocks_al * t_block + (Z > 1 ? 2.0 : 0.4);
