@@ -618,8 +618,38 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                     }
                     tile_compute<MODE>(tb, acc, acc_m, lc);
                 }
+            } else if (all_full && work && i0 + BPW <= nblk && unit_next > i0 && unit_next - first_fix + len >= i0 + BPW) {
+                // exactly one strip boundary inside the warp's blocks, every block full and inside the range: the blocks
+                // before it, the hand-off of the finished strip piece, the blocks after it -- two tiles in flight
+                // wherever two neighbours are on the same side
+                const int pb = unit_next - i0;  // first block of the next strip piece, 1 .. BPW - 1
+#pragma unroll 1
+                for (int jj = 0; jj < BPW;) {
+                    if (jj == pb) {
+                        flush();
+                        next_unit();
+                        lim = interior_limit();
+                    }
+                    const uint32_t sb = sbase + jj * kBlockBytes;
+                    const int tile = (i0 + jj - unit_first) * 8 + tw;
+                    TileIn ta;
+                    tile_load<MODE>(ta, sb + code_lane, sb + so_lane8, sb + 576u * 8u + m_lane, tile, la);
+                    if (jj + 1 < BPW && jj + 1 != pb) {
+                        TileIn tb;
+                        tile_load<MODE>(tb, sb + kBlockBytes + code_lane, sb + kBlockBytes + so_lane8,
+                                        sb + kBlockBytes + 576u * 8u + m_lane, tile + 8, la);
+                        tile_compute<MODE>(ta, acc, acc_m, lc);
+                        tile_compute<MODE>(tb, acc, acc_m, lc);
+                        jj += 2;
+                    } else {
+                        tile_compute<MODE>(ta, acc, acc_m, lc);
+                        jj += 1;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8u * stage);
             } else {
-                // general stage (range end, strip boundary, short last block): one block at a time
+                // general stage (range end, several boundaries, short last block): one block at a time
                 for (int jj = 0; jj < BPW; ++jj) {
                     const int i = i0 + jj;
                     if (i >= nblk) break;
