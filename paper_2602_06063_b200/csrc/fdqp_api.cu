@@ -173,10 +173,10 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
         for (;; Z *= 2) {
             if (Z > p->nb) Z = p->nb;
             nbz = (p->nb + Z - 1) / Z;
-            // four blocks per warp per stage halve the barrier traffic per tile; worth it once a CTA streams many blocks
+            // four blocks per warp per stage halve the barrier traffic per tile
             const int64_t blocks_per_cta = (int64_t)p->S * p->nb / ((int64_t)ctx->sm_count * ctas_per_sm);
             // (measured: pays up to M = 4, never when the larger stage would force a K split)
-            bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (M <= 4 && blocks_per_cta >= 64 ? 4 : 2);
+            bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (M <= 4 && blocks_per_cta >= 4 ? 4 : 2);
             L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw);
             if (bpw == 4 && ctx->p_bpw != 4 && M > 1 && L.nstage < kMinStages) {
                 bpw = 2;
