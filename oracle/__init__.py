@@ -50,6 +50,10 @@ def _load():
         lib.oracle_project.argtypes = [p, p, p, p, i64, i64, i64, i64, i64, ci, ci, p, p]
         lib.oracle_project_packed.restype = ci
         lib.oracle_project_packed.argtypes = [p, p, i64, i64, i64, i64, i64, ci, ci, p, p]
+        lib.oracle_gelu_tanh.restype = ctypes.c_double
+        lib.oracle_gelu_tanh.argtypes = [ctypes.c_double]
+        lib.oracle_geglu.restype = ci
+        lib.oracle_geglu.argtypes = [p, i64, i64, p, p]
         lib.oracle_max_threads.restype = ci
         _lib = lib
     return _lib
@@ -141,3 +145,21 @@ def project_packed(x_bf16, packed, K: int, N: int, n0: int = 0, n1: int | None =
     if rc != 0:
         raise ValueError(f"oracle_project_packed failed ({rc})")
     return y, a
+
+
+def gelu_tanh(g: float) -> float:
+    """GELU, tanh form (the reading taken for the paper's "GeLU activation with MUL")."""
+    return float(_load().oracle_gelu_tanh(float(g)))
+
+
+def geglu(y):
+    """Gated GELU of a fused gate|up projection y [M, N] (per 32-row strip: rows 0..15 gate, 16..31 up):
+    (out [M, N/2] fp64, out_bf16 [M, N/2] uint16 = RNE bf16 of the fp32 rounding)."""
+    y = _c(y, np.float64)
+    M, N = y.shape
+    out = np.empty((M, N // 2), np.float64)
+    out16 = np.empty((M, N // 2), np.uint16)
+    rc = _load().oracle_geglu(_ptr(y), M, N, _ptr(out), _ptr(out16))
+    if rc != 0:
+        raise ValueError(f"oracle_geglu failed ({rc})")
+    return out, out16

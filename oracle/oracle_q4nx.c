@@ -37,6 +37,10 @@
  * widened bf16 scale/offset; w16 is the round-to-nearest-even bf16 of w32.
  * The projection accumulates (double)x * (double)w32 sequentially in k.
  *
+ * Gated GELU epilogue (a next step beyond the paper's FusedDQP, which leaves the activation to a separate kernel):
+ * oracle_gelu_tanh / oracle_geglu below; pinned against the error-function form, symmetry, limits and a
+ * pairing case with exact products.
+ *
  * Pins (tests/test_oracle_pins.py): the paper's 5120-byte block, hand-written
  * byte dumps, closed-form worked examples, exact rational evaluation of eq. 3
  * over all codes, an independent fp64 matmul, and invariants.  Parity with
@@ -218,6 +222,33 @@ int oracle_project_packed(const uint16_t *x_bf16, const uint8_t *packed, int64_t
             if (abs_sum) abs_sum[m * W + (n - n0)] = aacc;
         }
     }
+    return 0;
+}
+
+/* ---- gated GELU on a fused gate|up projection (next-step epilogue) ------ */
+
+/* GELU in its tanh form, 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3))).  The paper names "GeLU activation with
+ * MUL" as the operation that follows the gate and up projections (Sec. on the decoder mapping) without giving the
+ * formula; the tanh form is this build's reading (it is the form Gemma's published configuration selects). */
+double oracle_gelu_tanh(double g) {
+    const double c = 0.79788456080286535588; /* sqrt(2 / pi) */
+    return 0.5 * g * (1.0 + tanh(c * (g + 0.044715 * g * g * g)));
+}
+
+/* y is [M][N] with N a multiple of 32: in every 32-row strip, rows 0..15 are gate features and rows 16..31 the up
+ * features of the same 16 outputs.  out[m][16 j + r] = gelu(y[m][32 j + r]) * y[m][32 j + 16 + r]  ([M][N/2], fp64);
+ * out_bf16, if not NULL, receives the round-to-nearest-even bf16 of the fp32 rounding of that value. */
+int oracle_geglu(const double *y, int64_t M, int64_t N, double *out, uint16_t *out_bf16) {
+    if (!y || !out || M < 1 || N < 32 || (N % 32) != 0) return 1;
+    const int64_t H = N / 2;
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t j = 0; j < N / 32; ++j)
+            for (int64_t r = 0; r < 16; ++r) {
+                const double g = y[m * N + 32 * j + r], u = y[m * N + 32 * j + 16 + r];
+                const double v = oracle_gelu_tanh(g) * u;
+                out[m * H + 16 * j + r] = v;
+                if (out_bf16) out_bf16[m * H + 16 * j + r] = fp32_to_bf16_rne((float)v);
+            }
     return 0;
 }
 

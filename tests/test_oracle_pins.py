@@ -331,3 +331,47 @@ def test_invariants_linearity_and_rows():
     # each row of a batched call equals the single-row call; rows are not mixed up or transposed
     yb, _ = oracle.project(synthgen.bf16_bits(np.concatenate([x1, x2])), w.codes, w.scales, w.offsets)
     assert np.array_equal(yb[0], y1[0]) and np.array_equal(yb[1], y2[0])
+
+
+# ---- gated GELU epilogue (next step beyond FusedDQP) ---------------------------------------------------------------
+
+def test_gelu_tanh_against_the_error_function_form_and_limits():
+    import math
+
+    # the tanh form approximates x * Phi(x) (library erf) to within 1e-3 everywhere
+    worst = 0.0
+    for i in range(-1200, 1201):
+        x = i / 200.0
+        exact = 0.5 * x * (1.0 + math.erf(x / math.sqrt(2.0)))
+        worst = max(worst, abs(oracle.gelu_tanh(x) - exact))
+    assert worst < 1e-3
+    assert worst > 1e-5                                  # ... and is not secretly the erf form
+    assert oracle.gelu_tanh(0.0) == 0.0
+    assert oracle.gelu_tanh(30.0) == 30.0                # tanh saturates: identity for large arguments
+    assert abs(oracle.gelu_tanh(-30.0)) < 1e-300
+    for x in (0.1, 0.7, 1.0, 2.5, 5.0):                  # gelu(x) - gelu(-x) = x for any odd inner function
+        assert abs(oracle.gelu_tanh(x) - oracle.gelu_tanh(-x) - x) < 1e-15
+    # widely tabulated values of the tanh form, four digits
+    for x, v in ((1.0, 0.8412), (2.0, 1.9546), (-1.0, -0.1588), (3.0, 2.9964)):
+        assert abs(oracle.gelu_tanh(x) - v) < 5e-5
+
+
+def test_geglu_pairs_rows_r_and_r_plus_16_of_each_strip():
+    # arguments >= 20 make the tanh exactly 1, so gelu(g) = g and every output is an exact integer product that
+    # names the two rows it came from
+    M, N = 2, 96
+    y = np.array([[20.0 + n + 1000.0 * m for n in range(N)] for m in range(M)])
+    out, out16 = oracle.geglu(y)
+    assert out.shape == (M, N // 2)
+    for m in range(M):
+        for j in range(N // 32):
+            for r in range(16):
+                g, u = y[m, 32 * j + r], y[m, 32 * j + 16 + r]
+                assert out[m, 16 * j + r] == g * u
+    # bf16 output: round-to-nearest-even of the fp32 value, checked with integer arithmetic on the bits
+    f32 = out.astype(np.float32).view(np.uint32).astype(np.uint64)
+    expect = ((f32 + 0x7FFF + ((f32 >> 16) & 1)) >> 16).astype(np.uint16)
+    assert np.array_equal(out16, expect)
+    # a gate of zero silences its output whatever the up value is
+    y[:, 0] = 0.0
+    assert np.all(oracle.geglu(y)[0][:, 0] == 0.0)
