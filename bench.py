@@ -187,11 +187,19 @@ def run_shape(args):
     ncopies = max(1, int(np.ceil(4 * L2_BYTES / base.numel()))) if not args.same_weights else 1
     copies = [base] + [base.clone() for _ in range(ncopies - 1)]
     x = torch.from_numpy(synthgen.activations(1, M, K).view(np.int16)).cuda()
-    y = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    epi = {"none": fd.EPI_NONE, "bf16": fd.EPI_BF16, "geglu": fd.EPI_GEGLU_BF16}[args.epilogue]
+    if epi == fd.EPI_NONE:
+        y = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    else:
+        y = torch.empty((M, N // 2 if epi == fd.EPI_GEGLU_BF16 else N), dtype=torch.bfloat16, device="cuda")
     stream = torch.cuda.Stream()
     sraw = stream.cuda_stream
+
+    def launch(W):
+        fd.fdqp_run_epilogue(ctx, x, W, y, epi, M, K, N, sraw)
+
     for i in range(max(3, args.warmup)):
-        fd.fdqp_run(ctx, x, copies[i % ncopies], y, M, K, N, sraw)
+        launch(copies[i % ncopies])
     stream.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if args.graph and not args.same_weights:
@@ -199,7 +207,7 @@ def run_shape(args):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=stream):
             for i in range(args.steps):
-                fd.fdqp_run(ctx, x, copies[i % ncopies], y, M, K, N, sraw)
+                launch(copies[i % ncopies])
         with torch.cuda.stream(stream):
             g.replay()
         stream.synchronize()
@@ -210,7 +218,7 @@ def run_shape(args):
     else:
         e0.record(stream)
         for i in range(args.steps):
-            fd.fdqp_run(ctx, x, copies[i % ncopies], y, M, K, N, sraw)
+            launch(copies[i % ncopies])
         e1.record(stream)
     stream.synchronize()
     assert fd.fdqp_last_status(ctx) == 0
@@ -219,7 +227,7 @@ def run_shape(args):
     print(json.dumps({"shape": {"K": K, "N": N, "M": M}, "us_per_call": us, "GBps": gbs,
                       "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
                       "peak_kind": peak_kind, "weight_copies": ncopies, "steps": args.steps,
-                      "graph": bool(args.graph and not args.same_weights),
+                      "graph": bool(args.graph and not args.same_weights), "epilogue": args.epilogue,
                       "launch": fd.fdqp_describe(ctx, M, K, N)}), flush=True)
     fd.fdqp_destroy(ctx)
 
@@ -536,6 +544,8 @@ def main():
     ap.add_argument("--param", action="append", help="library launch parameter key=value (repeatable)")
     ap.add_argument("--shape", help="K,N,M: time this one projection shape instead of the layer workload")
     ap.add_argument("--same-weights", action="store_true", help="with --shape: reuse one weight buffer (for ncu captures)")
+    ap.add_argument("--epilogue", default="none", choices=["none", "bf16", "geglu"],
+                    help="with --shape: fused store-side epilogue (geglu: gate and up rows interleaved 16 by 16 along N)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-head", action="store_true", help="skip the LM-head timing")
     args = ap.parse_args()

@@ -138,6 +138,31 @@ FDQP_API fdqp_status fdqp_destroy(fdqp_ctx* ctx);
 FDQP_API fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, float* y, int64_t M, int64_t K,
                      int64_t N, void* cuda_stream);
 
+/* Epilogues of fdqp_run_epilogue. */
+typedef enum {
+    FDQP_EPI_NONE = 0,       /* out = y, fp32 [M][N]: the same as fdqp_run */
+    FDQP_EPI_BF16 = 1,       /* out = y rounded to nearest-even bf16, [M][N] */
+    FDQP_EPI_GEGLU_BF16 = 2  /* out = gelu(gate) * up as bf16, [M][N/2] (see below) */
+} fdqp_epilogue;
+
+/* The projection followed, in the same kernels, by the step that comes after it in a
+ * decoder layer.  The paper runs "GeLU activation with MUL" as a kernel of its own
+ * after the gate and up projections (its section on mapping the decoder) and gives
+ * no formula; this entry point fuses it into the projection's store, with GELU in
+ * its tanh form 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3))), evaluated in fp32
+ * on the fp32 projection results.
+ *   FDQP_EPI_GEGLU_BF16: W holds the gate and up matrices fused along N with their
+ *   rows interleaved sixteen by sixteen: rows 32j .. 32j+15 of W are gate features
+ *   16j .. 16j+15, rows 32j+16 .. 32j+31 are the up features of the same outputs
+ *   (a row order for the caller to apply before q4nx_pack).  Output value
+ *   out[m][16j + r] = bf16(gelu(y[m][32j + r]) * y[m][32j + 16 + r]), r = 0..15.
+ *   out     device, 16-byte aligned; fp32 or bf16 as the epilogue says; fully overwritten
+ * Everything else (arguments, dispatch, asynchrony, errors) as fdqp_run; additionally
+ * FDQP_ERR_ARG for an unknown epilogue, or for a bf16 epilogue while the "path"
+ * parameter selects the plain self-check kernel. */
+FDQP_API fdqp_status fdqp_run_epilogue(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, void* out, int epilogue,
+                              int64_t M, int64_t K, int64_t N, void* cuda_stream);
+
 /* Same projection with HOST activations and result: copies x (host, [M][K] bf16)
  * to the context's device staging buffer, runs fdqp_run, copies y back to `y_host`
  * (host, [M][N] fp32) and synchronises the stream before returning.  W stays a

@@ -12,7 +12,11 @@ from .binding import (  # noqa: F401
     fdqp_last_cuda_error,
     fdqp_last_status,
     fdqp_launch_count,
+    EPI_BF16,
+    EPI_GEGLU_BF16,
+    EPI_NONE,
     fdqp_run,
+    fdqp_run_epilogue,
     fdqp_run_host,
     fdqp_run_host_async,
     fdqp_run_noalloc,

@@ -23,7 +23,7 @@ STATUS = {
 
 EXPORTS = [
     "q4nx_packed_bytes", "q4nx_pack", "q4nx_unpack", "fdqp_create", "fdqp_destroy", "fdqp_run", "fdqp_run_host",
-    "fdqp_run_host_async",
+    "fdqp_run_host_async", "fdqp_run_epilogue",
     "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
     "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc",
 ]
@@ -64,6 +64,8 @@ def load_library():
     lib.fdqp_run.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_run_host.restype = ci
     lib.fdqp_run_host.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.fdqp_run_epilogue.restype = ci
+    lib.fdqp_run_epilogue.argtypes = [vp, vp, vp, vp, ci, i64, i64, i64, vp]
     lib.fdqp_run_host_async.restype = ci
     lib.fdqp_run_host_async.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_run_noalloc.restype = ci
@@ -168,6 +170,16 @@ def fdqp_run(ctx: int, x_bf16, W_q4nx, y, M: int, K: int, N: int, stream=None) -
     """x, W, y: device tensors (or addresses).  Asynchronous on `stream`."""
     _check(load_library().fdqp_run(ctx, _addr(x_bf16), _addr(W_q4nx), _addr(y), M, K, N, _stream(stream)),
            "fdqp_run", ctx)
+
+
+EPI_NONE, EPI_BF16, EPI_GEGLU_BF16 = 0, 1, 2
+
+
+def fdqp_run_epilogue(ctx: int, x_bf16, W_q4nx, out, epilogue: int, M: int, K: int, N: int, stream=None) -> None:
+    """fdqp_run with the store-side epilogue fused in: EPI_NONE (fp32 [M, N]), EPI_BF16 (bf16 [M, N]) or
+    EPI_GEGLU_BF16 (bf16 [M, N/2]; gate and up rows interleaved sixteen by sixteen in W, see fdqp.h)."""
+    _check(load_library().fdqp_run_epilogue(ctx, _addr(x_bf16), _addr(W_q4nx), _addr(out), int(epilogue), M, K, N,
+                                            _stream(stream)), "fdqp_run_epilogue", ctx)
 
 
 def fdqp_run_host(ctx: int, x_host_bf16, W_q4nx, y_host, M: int, K: int, N: int, stream=None) -> None:

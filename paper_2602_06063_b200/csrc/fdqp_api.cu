@@ -15,12 +15,13 @@
 namespace fdqp {
 cudaError_t gemv_launch(const GemvPlan& p, int consumer_warps, cudaStream_t stream);
 cudaError_t gemv_set_smem_limit(int bytes);
-cudaError_t splitk_sum_launch(const float* ws, float* y, int Z, int S, int M, int N, cudaStream_t stream);
+cudaError_t splitk_sum_launch(const float* ws, float* y, uint16_t* y16, int epi, int Z, int S, int M, int N,
+                              cudaStream_t stream);
 cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream);
 cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
 cudaError_t prefill_set_smem_limit();
-cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, float* ws, int* status, int M,
-                           int K, int N, int pair, int Z, cudaStream_t stream);
+cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, uint16_t* y16, int epi, float* ws,
+                           int* status, int M, int K, int N, int pair, int Z, cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
 }  // namespace fdqp
 
@@ -331,12 +332,21 @@ extern "C" fdqp_status fdqp_destroy(fdqp_ctx* ctx) {
     return FDQP_OK;
 }
 
-extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, float* y, int64_t M, int64_t K,
-                                int64_t N, void* cuda_stream) {
-    if (!ctx || !x_bf16 || !W_q4nx || !y) return FDQP_ERR_ARG;
+namespace {
+
+// The projection with its epilogue: `out` is fp32 [M][N] (kEpiNone), bf16 [M][N] (kEpiBf16) or bf16 [M][N/2]
+// (kEpiGegluBf16).
+fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, void* out, int epi, int64_t M, int64_t K,
+                     int64_t N, void* cuda_stream) {
+    if (!ctx || !x_bf16 || !W_q4nx || !out) return FDQP_ERR_ARG;
+    if (epi != kEpiNone && epi != kEpiBf16 && epi != kEpiGegluBf16) return FDQP_ERR_ARG;
     fdqp_status st = check_shape(ctx, M, K, N);
     if (st != FDQP_OK) return st;
-    if (!aligned16(x_bf16) || !aligned16(W_q4nx) || !aligned16(y)) return FDQP_ERR_ALIGN;
+    if (!aligned16(x_bf16) || !aligned16(W_q4nx) || !aligned16(out)) return FDQP_ERR_ALIGN;
+    if (epi != kEpiNone && ctx->p_path == 1) return FDQP_ERR_ARG;  // the plain self-check kernel writes fp32 only
+    float* y = epi == kEpiNone ? static_cast<float*>(out) : nullptr;
+    uint16_t* y16 = epi == kEpiNone ? nullptr : static_cast<uint16_t*>(out);
+    const int64_t n_out = epi == kEpiGegluBf16 ? N / 2 : N;  // output values per token row
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FDQP_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -359,7 +369,7 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
                 return cuda_fail(ctx, e, "x spreading copy");
             xt = reinterpret_cast<const uint16_t*>(ctx->x_spread);
         }
-        if ((e = prefill_launch(W, xt, x_row_bytes, y, ctx->pf_ws, ctx->status_dev, (int)M, (int)K, (int)N,
+        if ((e = prefill_launch(W, xt, x_row_bytes, y, y16, epi, ctx->pf_ws, ctx->status_dev, (int)M, (int)K, (int)N,
                                 use_pair(ctx, M) ? 1 : 0, prefill_slices(ctx, M, K, N), stream)))
             return cuda_fail(ctx, e, "prefill kernel launch");
         ctx->launches += prefill_slices(ctx, M, K, N) > 1 ? 2 : 1;
@@ -373,7 +383,9 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
         if (!plan_gemv(ctx, mc, (int)K, (int)N, &cw, &plan)) return FDQP_ERR_SIZE;
         plan.W = W;
         plan.x = x + m0 * K;
-        plan.y = y + m0 * N;
+        plan.y = y ? y + m0 * N : nullptr;
+        plan.y16 = y16 ? y16 + m0 * n_out : nullptr;
+        plan.epi = epi;
         if (!plan.prep_inline) {
             if ((e = xprep_launch(plan.x, ctx->xq, ctx->xsc, mc, (int)K, stream)))
                 return cuda_fail(ctx, e, "x preparation launch");
@@ -388,12 +400,24 @@ extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W
         if ((e = gemv_launch(plan, cw, stream))) return cuda_fail(ctx, e, "gemv kernel launch");
         ctx->launches += 1;
         if (plan.Z > 1) {
-            if ((e = splitk_sum_launch(ctx->ws_full, plan.y, plan.Z, plan.S, mc, (int)N, stream)))
+            if ((e = splitk_sum_launch(ctx->ws_full, plan.y, plan.y16, epi, plan.Z, plan.S, mc, (int)N, stream)))
                 return cuda_fail(ctx, e, "split-K sum launch");
             ctx->launches += 1;
         }
     }
     return FDQP_OK;
+}
+
+}  // namespace
+
+extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, float* y, int64_t M, int64_t K,
+                                int64_t N, void* cuda_stream) {
+    return run_impl(ctx, x_bf16, W_q4nx, y, kEpiNone, M, K, N, cuda_stream);
+}
+
+extern "C" fdqp_status fdqp_run_epilogue(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, void* out, int epilogue,
+                                         int64_t M, int64_t K, int64_t N, void* cuda_stream) {
+    return run_impl(ctx, x_bf16, W_q4nx, out, epilogue, M, K, N, cuda_stream);
 }
 
 extern "C" fdqp_status fdqp_run_host_async(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,

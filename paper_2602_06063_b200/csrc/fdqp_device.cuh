@@ -157,6 +157,38 @@ __device__ __forceinline__ float bf16hi_mul_f32hi(uint32_t packed, float w) {
     return r;
 }
 
+// Round-to-nearest-even bf16 bits of an fp32 (one conversion instruction).
+__device__ __forceinline__ uint16_t f32_to_bf16_rne(float f) {
+    uint16_t r;
+    asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(r) : "f"(f));
+    return r;
+}
+
+// GELU, tanh form: 0.5 g (1 + tanh(z)), z = sqrt(2/pi) (g + 0.044715 g^3), written as g / (1 + exp(-2 z)): the same
+// function, two fast-math instructions instead of a tanh call; saturates to g and to -0 exactly.
+__device__ __forceinline__ float gelu_tanh(float g) {
+    const float z2 = 1.5957691216057308f * (g + 0.044715f * g * g * g);  // 2 z
+    return __fdividef(g, 1.0f + __expf(-z2));
+}
+
+// The stored bits of one finished value under a bf16 epilogue; `up` is the partner row's value (gated GELU only).
+__device__ __forceinline__ uint16_t epilogue_bf16(int epi, float v, float up) {
+    return f32_to_bf16_rne(epi == 1 ? v : gelu_tanh(v) * up);
+}
+
+// One finished output value per lane: row `lane` of 32-row strip s, token row t.  All 32 lanes must call it together.
+__device__ __forceinline__ void store_output(float* y, uint16_t* y16, int epi, int64_t N, int64_t s, int lane, int t,
+                                             float v) {
+    if (epi == 0) {
+        y[(int64_t)t * N + s * 32 + lane] = v;
+    } else if (epi == 1) {
+        y16[(int64_t)t * N + s * 32 + lane] = epilogue_bf16(1, v, 0.f);
+    } else {
+        const float up = __shfl_xor_sync(0xffffffffu, v, 16);
+        if (lane < 16) y16[(int64_t)t * (N / 2) + s * 16 + lane] = epilogue_bf16(2, v, up);
+    }
+}
+
 __device__ __forceinline__ float bf16_lo_to_f32(uint32_t packed) { return __uint_as_float(packed << 16); }
 __device__ __forceinline__ float bf16_hi_to_f32(uint32_t packed) { return __uint_as_float(packed & 0xffff0000u); }
 

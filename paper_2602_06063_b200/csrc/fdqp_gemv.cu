@@ -326,11 +326,12 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][Mo
     }
 }
 
-// CW consumer warps (8 or 16); MODE as above (1: M = 1, 3: M = 2, 2: M = 3..8).
+// CW consumer warps (8 or 16); MODE as above (1: M = 1, 3: M = 2, 2: M = 3..8); EPI: built with the bf16 epilogues
+// (the fp32-only build keeps its stores free of the epilogue's branches).
 // A ring stage holds CB = (CW / 8) * BPW blocks; warp w owns group-tile (w & 7) of the BPW (2 or 4) consecutive
 // blocks starting at BPW * (w >> 3) of every stage.  More blocks per stage = fewer barrier round trips per tile.
 // Warps CW+1 .. CW+NR are reducers (NR = CW / 8): reducer r completes the strip pieces with piece % NR == r.
-template <int CW, int MODE, int BPW>
+template <int CW, int MODE, int BPW, bool EPI>
 __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
     fdqp_gemv_kernel(const __grid_constant__ GemvPlan p) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -729,7 +730,6 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             if (lane == 0) mbar_arrive(red_empty0 + 8u * par);
 
             const bool whole_unit = (pa == unit_begin) && (pe == unit_end);
-            float* yrow = p.y + s * kStripRows + lane;
             if (p.Z > 1) {
                 // K slices: ranges are strip-aligned, every (slice, strip) has one owner; the slices are added by
                 // fdqp_splitk_sum_kernel after this grid (fixed order, no arrival counters)
@@ -738,9 +738,16 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                 for (int t = 0; t < kMaxTokens; ++t)
                     if (t < M) slot[t * kStripRows + lane] = v[t];
             } else if (whole_unit) {
+                if (!EPI) {  // EPI: the bf16 / gated-GELU epilogues are compiled in (plan.epi says which)
+                    float* yrow = p.y + s * kStripRows + lane;
 #pragma unroll
-                for (int t = 0; t < kMaxTokens; ++t)
-                    if (t < M) yrow[(int64_t)t * p.N] = v[t];
+                    for (int t = 0; t < kMaxTokens; ++t)
+                        if (t < M) yrow[(int64_t)t * p.N] = v[t];
+                } else {
+#pragma unroll
+                    for (int t = 0; t < kMaxTokens; ++t)
+                        if (t < M) store_output(p.y, p.y16, p.epi, p.N, s, lane, t, v[t]);
+                }
             } else {
                 float* slot = piece_slot(p, z, ci, s, unit_begin, whole_unit, a);
 #pragma unroll
@@ -779,9 +786,16 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                                 if (t < M) v[t] += __ldcg(src + t * kStripRows + lane);
                         }
                     }
+                    if (!EPI) {  // EPI: the bf16 / gated-GELU epilogues are compiled in (plan.epi says which)
+                        float* yrow = p.y + s * kStripRows + lane;
 #pragma unroll
-                    for (int t = 0; t < kMaxTokens; ++t)
-                        if (t < M) yrow[(int64_t)t * p.N] = v[t];
+                        for (int t = 0; t < kMaxTokens; ++t)
+                            if (t < M) yrow[(int64_t)t * p.N] = v[t];
+                    } else {
+#pragma unroll
+                        for (int t = 0; t < kMaxTokens; ++t)
+                            if (t < M) store_output(p.y, p.y16, p.epi, p.N, s, lane, t, v[t]);
+                    }
                     if (lane == 0) p.tickets[s] = 0;  // ready for the next launch on this stream
                 }
             }
@@ -792,17 +806,18 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
 
 // Second phase of a K-split projection: y[tok][n] = sum over slices z (ascending) of the slice partials.
 // ws is [Z][S][kMaxTokens][32]; one thread per (tok, n).
-__global__ void __launch_bounds__(256) fdqp_splitk_sum_kernel(const float* __restrict__ ws, float* __restrict__ y, int Z, int S,
-                                                               int M, int N) {
+__global__ void __launch_bounds__(256) fdqp_splitk_sum_kernel(const float* __restrict__ ws, float* __restrict__ y,
+                                                               uint16_t* __restrict__ y16, int epi, int Z, int S, int M, int N) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");  // the GEMV grid's partials
+    // whole warps stay together (store_output shuffles): M * N is a multiple of 32
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (int64_t)M * N) return;
     const int tok = (int)(idx / N), n = (int)(idx - (int64_t)tok * N);
     const int s = n >> 5, r = n & 31;
     float acc = 0.f;
     for (int z = 0; z < Z; ++z) acc += ws[(((int64_t)z * S + s) * kMaxTokens + tok) * kStripRows + r];
-    y[idx] = acc;
+    store_output(y, y16, epi, N, s, r, tok, acc);
 }
 
 #ifdef FDQP_TRACE
@@ -825,7 +840,8 @@ static cudaError_t launch_one(const GemvPlan& p, cudaStream_t stream) {
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<CW, MODE, BPW>, p);
+    return p.epi == kEpiNone ? cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<CW, MODE, BPW, false>, p)
+                             : cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<CW, MODE, BPW, true>, p);
 }
 
 cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream) {
@@ -843,7 +859,8 @@ cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int
                   : cudaLaunchKernelEx(&cfg, fdqp_xprep_kernel<false>, x, xq, xsc, M, K);
 }
 
-cudaError_t splitk_sum_launch(const float* ws, float* y, int Z, int S, int M, int N, cudaStream_t stream) {
+cudaError_t splitk_sum_launch(const float* ws, float* y, uint16_t* y16, int epi, int Z, int S, int M, int N,
+                              cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(((int64_t)M * N + 255) / 256));
     cfg.blockDim = dim3(256);
@@ -853,7 +870,7 @@ cudaError_t splitk_sum_launch(const float* ws, float* y, int Z, int S, int M, in
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fdqp_splitk_sum_kernel, ws, y, Z, S, M, N);
+    return cudaLaunchKernelEx(&cfg, fdqp_splitk_sum_kernel, ws, y, y16, epi, Z, S, M, N);
 }
 
 // consumer_warps: 8 or 16; p.bpw (blocks per warp per stage): 2 or 4.  Kernel mode by M (see the header).
@@ -874,9 +891,11 @@ cudaError_t gemv_launch(const GemvPlan& p, int consumer_warps, cudaStream_t stre
 template <int CW, int MODE>
 static cudaError_t set_smem_limit_mode(int bytes) {
     const cudaFuncAttribute a = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    cudaError_t e = cudaFuncSetAttribute(fdqp_gemv_kernel<CW, MODE, 2>, a, bytes);
-    if (e) return e;
-    return cudaFuncSetAttribute(fdqp_gemv_kernel<CW, MODE, 4>, a, bytes);
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<CW, MODE, 2, false>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<CW, MODE, 4, false>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<CW, MODE, 2, true>, a, bytes))) return e;
+    return cudaFuncSetAttribute(fdqp_gemv_kernel<CW, MODE, 4, true>, a, bytes);
 }
 
 cudaError_t gemv_set_smem_limit(int bytes) {

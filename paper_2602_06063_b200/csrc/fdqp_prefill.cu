@@ -43,6 +43,8 @@ struct PrefillParams {
     float* y;       // [M][N] result, or (Z > 1) Z partial results of that shape, one per K slice
     int* status;
     int M, K, N;
+    uint16_t* y16;  // bf16 output of the epilogues other than kEpiNone (Z == 1 only; K-split calls leave it to the sum)
+    int epi;
     int Z;          // K slices; slice z covers k-steps [z * ksteps_z, (z + 1) * ksteps_z)
     int ksteps_z;   // 64-wide k-steps per slice
 };
@@ -191,6 +193,28 @@ __device__ __forceinline__ void group_store(uint32_t a_tile, const GroupRegs& r,
     }
 }
 
+// ---- bf16 epilogues: the tile goes through shared memory so that global memory sees whole 128-byte lines --------------
+//
+// A thread owns one output feature (a TMEM lane) and many tokens, so 2-byte results written straight to y would reach
+// memory as 64- or 32-byte pieces of a line per store (measured: twice the time of the fp32 store for half the bytes).
+// The warps therefore write their results into the pipeline's shared memory (free once the accumulators are final) as a
+// [token][column] bf16 tile, and then copy it out row by row, 16 bytes per lane.
+
+// Copies rows [0, toks) of a [toks][cols] bf16 tile at shared address `stage` (cols * 2 in {128, 256, 512} bytes) to
+// dst[t * ld16 + 0 .. valid_cols); warp wi of nwarps, 16-byte chunks, whole warps.
+__device__ __forceinline__ void stage_copy_out(uint32_t stage, uint16_t* dst, int64_t ld16, int toks, int cols,
+                                               int valid_cols, int wi, int nwarps, int lane) {
+    const int cpr = cols / 8;   // 16-byte chunks per tile row: 8, 16 or 32
+    const int rpi = 32 / cpr;   // tile rows one warp moves per step
+    const int chunk = lane % cpr;
+    for (int t = wi * rpi + lane / cpr; t < toks; t += nwarps * rpi) {
+        if (chunk * 8 < valid_cols) {
+            const uint4 v = lds128(stage + (uint32_t)(t * cols + chunk * 8) * 2u);
+            *reinterpret_cast<uint4*>(dst + (int64_t)t * ld16 + chunk * 8) = v;
+        }
+    }
+}
+
 // ---- the kernel -------------------------------------------------------------------------------------------------------
 
 __global__ void __launch_bounds__(kPf1Threads, 1)
@@ -208,6 +232,7 @@ __global__ void __launch_bounds__(kPf1Threads, 1)
     auto empty = [&](int s) { return bars + 8u * (2 * kPfStages + s); };
     const uint32_t acc_done = bars + 8u * (3 * kPfStages);
     const uint32_t tmem_slot = acc_done + 8u;
+    const uint32_t staged = tmem_slot + 8u;  // bf16 epilogues: every epilogue warp has written its part of the tile
     volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(smem + kPfStages * kPfStageBytes + 8 * (3 * kPfStages + 1));
 
     const int tok_tiles = (p.M + kPfToks - 1) / kPfToks;
@@ -228,6 +253,7 @@ __global__ void __launch_bounds__(kPf1Threads, 1)
             mbar_init(empty(s), 1);
         }
         mbar_init(acc_done, 1);
+        mbar_init(staged, kPf1DequantWarps);
         mbar_fence_init();
     }
     if (warp == 0) {
@@ -303,26 +329,66 @@ __global__ void __launch_bounds__(kPf1Threads, 1)
         // =============================== epilogue: TMEM -> y =================================================
         if (ok) ok = mbar_wait(acc_done, 0, p.status);
         ok = __all_sync(0xffffffffu, ok);
+        const bool via_smem = p.epi != kEpiNone && p.Z == 1;  // bf16 epilogues (a K-split call leaves them to the sum)
+        const bool geglu = p.epi == kEpiGegluBf16;
+        const int cols = geglu ? kPfRows / 2 : kPfRows;       // bf16 values per token row of the staged tile
         if (ok) {
             tc_fence_after();
             const int quarter = warp & 3;        // TMEM lanes this warp may read
             // the four warps of a quarter (dw = quarter', quarter' + 4, + 8, + 12) take (accumulator, column half)
             const int half = (dw >> 2) & 1, chalf = dw >> 3;
-            const int n = n0 + half * 128 + quarter * 32 + lane;
+            const int n_local = half * 128 + quarter * 32 + lane;
+            const int n = n0 + n_local;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 256 + chalf * 128);
             const int c_end = ((int)n_inst < chalf * 128 + 128 ? (int)n_inst : chalf * 128 + 128) - chalf * 128;
             const int64_t ldy = p.N;
             float* yrow = yout + (int64_t)(tok0 + chalf * 128) * ldy + n;  // token row of this warp's column 0
             const int toks_h = toks - chalf * 128;                          // tokens of this column half that exist
+            // staged tile: this lane's column, and the first token row of this warp
+            const uint32_t scol = base + (uint32_t)((chalf * 128) * cols + (geglu ? (n_local >> 5) * 16 + (lane & 15) : n_local)) * 2u;
             for (int c = 0; c < c_end; c += 32) {
                 uint32_t v[32];
                 tmem_ld_32cols(taddr + c, v);
-                if (n < p.N) {
+                if (!via_smem) {
+                    if (n < p.N) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (c + j < toks_h) yrow[j * ldy] = __uint_as_float(v[j]);
+                        for (int j = 0; j < 32; ++j)
+                            if (c + j < toks_h) yrow[j * ldy] = __uint_as_float(v[j]);
+                    }
+                    yrow += 32 * ldy;
+                } else {
+                    if (!geglu) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(scol + (uint32_t)((c + j) * cols) * 2u),
+                                         "h"(f32_to_bf16_rne(__uint_as_float(v[j])))
+                                         : "memory");
+                    } else {
+                        // lanes 0..15 hold gate rows, lanes 16..31 the up rows of the same outputs: the low half finishes
+                        // the even tokens, the high half the odd ones -- one exchange per token pair, every lane busy
+                        const bool low = lane < 16;
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj) {
+                            const float a = __uint_as_float(v[2 * jj]), b = __uint_as_float(v[2 * jj + 1]);
+                            const float got = __shfl_xor_sync(0xffffffffu, low ? b : a, 16);
+                            const float gate = low ? a : got, up = low ? got : b;
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(scol + (uint32_t)((c + 2 * jj + (low ? 0 : 1)) * cols) * 2u),
+                                         "h"(f32_to_bf16_rne(gelu_tanh(gate) * up))
+                                         : "memory");
+                        }
+                    }
                 }
-                yrow += 32 * ldy;
+            }
+        }
+        if (via_smem) {
+            // every warp arrives (also one that gave up), then the tile leaves shared memory in whole lines
+            __syncwarp();
+            if (lane == 0) mbar_arrive(staged);
+            if (ok && mbar_wait(staged, 0, p.status)) {
+                const int64_t ld16 = geglu ? p.N / 2 : p.N;
+                const int col0 = geglu ? n0 / 2 : n0;
+                const int valid = (int)((ld16 - col0) < cols ? (ld16 - col0) : cols);
+                stage_copy_out(base, p.y16 + (int64_t)tok0 * ld16 + col0, ld16, toks, cols, valid, dw, kPf1DequantWarps, lane);
             }
         }
     }
@@ -440,6 +506,7 @@ __global__ void __launch_bounds__(kPfThreads, 1)
     auto empty = [&](int s) { return bars + 8u * (2 * kP2Stages + s); };     // each CTA its own, signalled by commit
     const uint32_t acc_done = bars + 8u * (3 * kP2Stages);
     const uint32_t tmem_slot = acc_done + 8u;
+    const uint32_t staged = tmem_slot + 8u;  // bf16 epilogues: every epilogue warp has written its part of the tile
     volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(smem + kP2Stages * kP2StageBytes + 8 * (3 * kP2Stages + 1));
 
     const uint32_t rank = cluster_ctarank();
@@ -466,6 +533,7 @@ __global__ void __launch_bounds__(kPfThreads, 1)
             mbar_init(empty(s), 1);
         }
         mbar_init(acc_done, 1);
+        mbar_init(staged, kPfDequantWarps);
         mbar_fence_init();
     }
     if (warp == 0) {
@@ -551,24 +619,63 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         // =============================== epilogue: this CTA's TMEM -> y ======================================
         if (ok) ok = mbar_wait(acc_done, 0, p.status);
         ok = __all_sync(0xffffffffu, ok);
+        const bool via_smem = p.epi != kEpiNone && p.Z == 1;  // bf16 epilogues (a K-split call leaves them to the sum)
+        const bool geglu = p.epi == kEpiGegluBf16;
+        const int cols = geglu ? kP2Rows / 2 : kP2Rows;       // bf16 values per token row of the staged tile
+        const int toks_all = (p.M - tok0) < kP2Toks ? (p.M - tok0) : kP2Toks;
         if (ok) {
             tc_fence_after();
             const int quarter = warp & 3;   // TMEM lanes this warp may read
             const int chalf = dw >> 2;      // columns [256 chalf, 256 chalf + 256): every (quarter, half) once
-            const int n = n0 + quarter * 32 + lane;
+            const int n_local = quarter * 32 + lane;
+            const int n = n0 + n_local;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(chalf * 256);
             const int toks = p.M - tok0 - chalf * 256;  // tokens of this column half that exist
             const int64_t ldy = p.N;
             float* yrow = yout + (int64_t)(tok0 + chalf * 256) * ldy + n;  // token row of column 0 of this half
+            const uint32_t scol = base + (uint32_t)((chalf * 256) * cols + (geglu ? (n_local >> 5) * 16 + (lane & 15) : n_local)) * 2u;
             for (int c = 0; c < 256 && c < toks; c += 32) {
                 uint32_t v[32];
                 tmem_ld_32cols(taddr + c, v);
-                if (n < p.N) {
+                if (!via_smem) {
+                    if (n < p.N) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (c + j < toks) yrow[j * ldy] = __uint_as_float(v[j]);
+                        for (int j = 0; j < 32; ++j)
+                            if (c + j < toks) yrow[j * ldy] = __uint_as_float(v[j]);
+                    }
+                    yrow += 32 * ldy;
+                } else {
+                    if (!geglu) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(scol + (uint32_t)((c + j) * cols) * 2u),
+                                         "h"(f32_to_bf16_rne(__uint_as_float(v[j])))
+                                         : "memory");
+                    } else {
+                        // lanes 0..15 hold gate rows, lanes 16..31 the up rows of the same outputs: the low half finishes
+                        // the even tokens, the high half the odd ones -- one exchange per token pair, every lane busy
+                        const bool low = lane < 16;
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj) {
+                            const float a = __uint_as_float(v[2 * jj]), b = __uint_as_float(v[2 * jj + 1]);
+                            const float got = __shfl_xor_sync(0xffffffffu, low ? b : a, 16);
+                            const float gate = low ? a : got, up = low ? got : b;
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(scol + (uint32_t)((c + 2 * jj + (low ? 0 : 1)) * cols) * 2u),
+                                         "h"(f32_to_bf16_rne(gelu_tanh(gate) * up))
+                                         : "memory");
+                        }
+                    }
                 }
-                yrow += 32 * ldy;
+            }
+        }
+        if (via_smem) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(staged);
+            if (ok && mbar_wait(staged, 0, p.status)) {
+                const int64_t ld16 = geglu ? p.N / 2 : p.N;
+                const int col0 = geglu ? n0 / 2 : n0;
+                const int valid = (int)((ld16 - col0) < cols ? (ld16 - col0) : cols);
+                stage_copy_out(base, p.y16 + (int64_t)tok0 * ld16 + col0, ld16, toks_all, cols, valid, dw, kPfDequantWarps, lane);
             }
         }
     }
@@ -595,6 +702,18 @@ __global__ void __launch_bounds__(256) fdqp_prefill_sum_kernel(const float4* __r
         acc.w += v.w;
     }
     y[i] = acc;
+}
+
+// The same for the bf16 / gated-GELU epilogues: one output value per thread, whole warps on one (token, strip).
+__global__ void __launch_bounds__(256) fdqp_prefill_sum_epi_kernel(const float* __restrict__ ws, uint16_t* __restrict__ y16,
+                                                                    int epi, int Z, int M, int N) {
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t total = (int64_t)M * N;  // a multiple of 32
+    if (idx >= total) return;
+    float acc = ws[idx];
+    for (int z = 1; z < Z; ++z) acc += ws[(int64_t)z * total + idx];
+    const int tok = (int)(idx / N), n = (int)(idx - (int64_t)tok * N);
+    store_output(nullptr, y16, epi, N, n >> 5, n & 31, tok, acc);
 }
 
 // ---- host side ----------------------------------------------------------------------------------------------------
@@ -626,8 +745,9 @@ cudaError_t prefill_set_smem_limit() {
 // Z > 1: K is cut into Z slices (tiles x Z CTAs or CTA pairs), their partial results go to `ws` ([Z][M][N] floats) and a
 // second kernel adds them in slice order into y.  For shapes with too few tiles to fill the GPU.
 // x_row_bytes: distance between token rows of x (K * 2 for a dense [M][K] array; a multiple of 16).
-cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, float* ws, int* status, int M,
-                           int K, int N, int pair, int Z, cudaStream_t stream) {
+// epi: kEpiNone writes fp32 y; the other epilogues write bf16 to y16 (see fdqp_plan.h).
+cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, uint16_t* y16, int epi, float* ws,
+                           int* status, int M, int K, int N, int pair, int Z, cudaStream_t stream) {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     CUtensorMap map;
@@ -644,6 +764,8 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_by
     if (Z < 1 || Z > ksteps_all || !ws) Z = 1;
     p.W = W;
     p.y = Z > 1 ? ws : y;
+    p.y16 = y16;
+    p.epi = epi;
     p.status = status;
     p.M = M;
     p.K = K;
@@ -673,6 +795,11 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_by
         err = cudaGetLastError();
     }
     if (err != cudaSuccess || Z == 1) return err;
+    if (epi != kEpiNone) {
+        const int64_t total = (int64_t)M * N;
+        fdqp_prefill_sum_epi_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(ws, y16, epi, Z, M, N);
+        return cudaGetLastError();
+    }
     const int64_t quads = (int64_t)M * N / 4;  // N is a multiple of 32
     fdqp_prefill_sum_kernel<<<(unsigned)((quads + 255) / 256), 256, 0, stream>>>(reinterpret_cast<const float4*>(ws),
                                                                                 reinterpret_cast<float4*>(y), Z, quads);

@@ -1,0 +1,140 @@
+"""GPU parity of the fused store-side epilogues (bf16 output, gated GELU on a fused gate|up projection) against the
+CPU oracle, through the C ABI, on every kernel family the projection dispatches to."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2602_06063_b200 as fd
+import synthgen
+from gpu_common import ABS_TOL, MAX_K, MAX_M, MAX_N, REL_TOL, Case
+
+pytestmark = pytest.mark.gpu
+
+PARAMS = ("path", "split_k", "prefill_pair", "prefill_split_k", "strip_aligned", "blocks_per_warp")
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    h = fd.fdqp_create(0, MAX_M, MAX_K, MAX_N)
+    yield h
+    torch.cuda.synchronize()
+    fd.fdqp_destroy(h)
+
+
+@pytest.fixture()
+def fresh(ctx):
+    for key in PARAMS:
+        fd.fdqp_set_param(ctx, key, -1)
+    yield ctx
+    for key in PARAMS:
+        fd.fdqp_set_param(ctx, key, -1)
+
+
+def bf16_rne_bits(f32: np.ndarray) -> np.ndarray:
+    u = f32.astype(np.float32).view(np.uint32).astype(np.uint64)
+    return ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+
+
+def run_epilogue(ctx, case, epi, M=None):
+    M = case.M if M is None else M
+    n_out = case.N // 2 if epi == fd.EPI_GEGLU_BF16 else case.N
+    out = torch.full((M, n_out), -1, dtype=torch.int16, device="cuda")
+    fd.fdqp_run_epilogue(ctx, case.x_dev, case.W_dev, out, epi, M, case.K, case.N)
+    torch.cuda.synchronize()
+    assert fd.fdqp_last_status(ctx) == 0
+    return out.cpu().numpy().view(np.uint16)
+
+
+def geglu_bound(y_ref, a_ref):
+    """Per-output bound on |out - out_ref| that follows from the projection's acceptance bound: the gate and the up
+    value may each be off by tol = REL_TOL * A + ABS_TOL; |gelu'| <= 1.13; then one bf16 rounding (2^-8 relative,
+    which also covers the fp32 evaluation of tanh)."""
+    M, N = y_ref.shape
+    tol = REL_TOL * a_ref + ABS_TOL
+    yv = y_ref.reshape(M, N // 32, 2, 16)
+    tv = tol.reshape(M, N // 32, 2, 16)
+    g, u, tg, tu = yv[:, :, 0], yv[:, :, 1], tv[:, :, 0], tv[:, :, 1]
+    gelu_g = np.vectorize(oracle.gelu_tanh)(g)
+    out = gelu_g * u
+    bound = 1.13 * tg * (np.abs(u) + tu) + np.abs(gelu_g) * tu + np.abs(out) * 2.0 ** -8 + 1e-6
+    return bound.reshape(M, N // 2)
+
+
+# (K, N, M, launch parameters): every kernel family and reduction path
+CASES = [
+    (1152, 288, 1, {}),                                  # GEMV, one token, tail block
+    (2560, 2048, 2, {}),                                 # GEMV, two tokens
+    (1024, 512, 5, {}),                                  # GEMV, plane mode
+    (4096, 4736, 8, {"strip_aligned": 0}),               # strips shared between CTAs (arrival counters)
+    (10240, 320, 3, {"split_k": 4}),                     # K slices + sum kernel
+    (1056, 320, 20, {"path": 2}),                        # GEMV eight rows at a time
+    (1056, 320, 40, {"path": 3}),                        # one-SM tensor-core kernel
+    (2048, 256, 64, {"path": 3, "prefill_split_k": 4}),  # ... with K slices + sum kernel
+    (544, 1056, 300, {"path": 3}),                       # two-SM tensor-core kernel, ragged tokens
+    (4096, 288, 512, {"path": 3, "prefill_split_k": 3}),
+]
+
+
+@pytest.mark.parametrize("K,N,M,params", CASES)
+def test_bf16_epilogue_is_the_rounded_fp32_result(fresh, K, N, M, params):
+    case = Case(K, N, M, seed=4000 + K + N + M)
+    for k, v in params.items():
+        fd.fdqp_set_param(fresh, k, v)
+    y = case.run(fresh)                                   # fp32 through the same kernels
+    out = run_epilogue(fresh, case, fd.EPI_BF16)
+    assert np.array_equal(out, bf16_rne_bits(y))          # same arithmetic, one extra rounding: bit for bit
+    # and EPI_NONE is fdqp_run
+    o32 = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    fd.fdqp_run_epilogue(fresh, case.x_dev, case.W_dev, o32, fd.EPI_NONE, M, K, N)
+    torch.cuda.synchronize()
+    assert np.array_equal(o32.cpu().numpy(), y)
+
+
+@pytest.mark.parametrize("K,N,M,params", CASES)
+def test_geglu_epilogue_matches_oracle(fresh, K, N, M, params):
+    case = Case(K, N, M, seed=5000 + K + N + M)
+    for k, v in params.items():
+        fd.fdqp_set_param(fresh, k, v)
+    out = synthgen.bf16_to_f32(run_epilogue(fresh, case, fd.EPI_GEGLU_BF16)).astype(np.float64)
+    y_ref, a_ref = case.reference()
+    out_ref, _ = oracle.geglu(y_ref)
+    err = np.abs(out - out_ref)
+    bound = geglu_bound(y_ref, a_ref)
+    assert np.all(np.isfinite(out))
+    bad = err > bound
+    assert not bad.any(), f"{bad.sum()} of {bad.size} outside the bound, first {np.argwhere(bad)[0]}"
+
+
+@pytest.mark.parametrize("M,params", [(1, {}), (2, {}), (6, {"strip_aligned": 0}), (8, {"split_k": 2}), (24, {"path": 3}),
+                                      (300, {"path": 3})])
+def test_geglu_pairing_exact(fresh, M, params):
+    # d = 2^-3, m = 1, x = 1: every y is an exact dyadic >= K, where gelu(g) = g in fp32 (tanh saturates), so the
+    # output is exactly the bf16 of the exact product of rows r and r + 16 of each strip, as the oracle computes it
+    K, N = 128, 576
+    r = synthgen.u64(77, 0, N * K).reshape(N, K)
+    w = synthgen.Q4NXWeights((r >> np.uint64(60)).astype(np.uint8), np.full((N, K // 32), 0x3E00, np.uint16),
+                             np.full((N, K // 32), 0x3F80, np.uint16))
+    x = np.full((M, K), 0x3F80, np.uint16)
+    x[:, ::3] = 0x4000                                    # some activations are 2
+    case = Case(K, N, M, seed=0, weights=w, x=x)
+    for k, v in params.items():
+        fd.fdqp_set_param(fresh, k, v)
+    y_ref, _ = case.reference()
+    assert y_ref.min() >= K
+    _, out16_ref = oracle.geglu(y_ref)
+    assert np.array_equal(run_epilogue(fresh, case, fd.EPI_GEGLU_BF16), out16_ref)
+
+
+def test_epilogue_argument_errors(fresh):
+    case = Case(256, 64, 1, seed=9)
+    out = torch.empty((1, 64), dtype=torch.int16, device="cuda")
+    lib = fd.load_library()
+    s = torch.cuda.current_stream().cuda_stream
+    args = (fresh, case.x_dev.data_ptr(), case.W_dev.data_ptr(), out.data_ptr())
+    assert lib.fdqp_run_epilogue(*args, 3, 1, 256, 64, s) == 1       # unknown epilogue
+    assert lib.fdqp_run_epilogue(*args[:3], None, 1, 1, 256, 64, s) == 1
+    fd.fdqp_set_param(fresh, "path", 1)
+    assert lib.fdqp_run_epilogue(*args, 1, 1, 256, 64, s) == 1       # the plain self-check kernel is fp32-only
+    assert lib.fdqp_run_epilogue(*args, 0, 1, 256, 64, s) == 0
+    torch.cuda.synchronize()
