@@ -146,7 +146,7 @@ typedef enum {
 } fdqp_epilogue;
 
 /* The projection followed, in the same kernels, by the step that comes after it in a
- * decoder layer.  The paper runs "GeLU activation with MUL" as a kernel of its own
+ * decoder layer.  The paper runs the GELU-and-multiply step as a kernel of its own
  * after the gate and up projections (its section on mapping the decoder) and gives
  * no formula; this entry point fuses it into the projection's store, with GELU in
  * its tanh form 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3))), evaluated in fp32

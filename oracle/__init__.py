@@ -148,7 +148,7 @@ def project_packed(x_bf16, packed, K: int, N: int, n0: int = 0, n1: int | None =
 
 
 def gelu_tanh(g: float) -> float:
-    """GELU, tanh form (the reading taken for the paper's "GeLU activation with MUL")."""
+    """GELU, tanh form (the reading taken for the GELU-and-multiply step the paper places after the gate and up projections)."""
     return float(_load().oracle_gelu_tanh(float(g)))
 
 

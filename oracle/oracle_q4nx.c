@@ -227,9 +227,9 @@ int oracle_project_packed(const uint16_t *x_bf16, const uint8_t *packed, int64_t
 
 /* ---- gated GELU on a fused gate|up projection (next-step epilogue) ------ */
 
-/* GELU in its tanh form, 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3))).  The paper names "GeLU activation with
- * MUL" as the operation that follows the gate and up projections (Sec. on the decoder mapping) without giving the
- * formula; the tanh form is this build's reading (it is the form Gemma's published configuration selects). */
+/* GELU in its tanh form, 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3))).  The paper places a GELU-and-multiply step
+ * after the gate and up projections (its section on mapping the decoder) without giving the formula; the tanh form is
+ * this build's reading (it is the form Gemma's published configuration selects). */
 double oracle_gelu_tanh(double g) {
     const double c = 0.79788456080286535588; /* sqrt(2 / pi) */
     return 0.5 * g * (1.0 + tanh(c * (g + 0.044715 * g * g * g)));
