@@ -138,3 +138,19 @@ def test_epilogue_argument_errors(fresh):
     assert lib.fdqp_run_epilogue(*args, 1, 1, 256, 64, s) == 1       # the plain self-check kernel is fp32-only
     assert lib.fdqp_run_epilogue(*args, 0, 1, 256, 64, s) == 0
     torch.cuda.synchronize()
+
+
+def test_gemma3_12b_gate_up_gated_gelu_full_size(ctx):
+    # the fused gate|up projection of the 12B model at its full size, decode batch sizes, default launch plan; the
+    # fused matrix's rows are read as interleaved gate / up rows (sixteen by sixteen per strip)
+    for key in PARAMS:
+        fd.fdqp_set_param(ctx, key, -1)
+    _, K, N, seed = synthgen.GEMMA3_12B_GATE_UP
+    case = Case(K, N, 8, seed)
+    y_ref, a_ref = case.reference()
+    out_ref, _ = oracle.geglu(y_ref)
+    bound = geglu_bound(y_ref, a_ref)
+    for M in (1, 2, 4, 8):
+        out = synthgen.bf16_to_f32(run_epilogue(ctx, case, fd.EPI_GEGLU_BF16, M=M)).astype(np.float64)
+        assert np.all(np.isfinite(out))
+        assert np.all(np.abs(out - out_ref[:M]) <= bound[:M]), f"12B gate|up gated GELU M={M}"
