@@ -54,6 +54,8 @@ def _load():
         lib.oracle_gelu_tanh.argtypes = [ctypes.c_double]
         lib.oracle_geglu.restype = ci
         lib.oracle_geglu.argtypes = [p, i64, i64, p, p]
+        lib.oracle_rmsnorm.restype = ci
+        lib.oracle_rmsnorm.argtypes = [p, p, ctypes.c_double, i64, i64, p]
         lib.oracle_max_threads.restype = ci
         _lib = lib
     return _lib
@@ -163,3 +165,17 @@ def geglu(y):
     if rc != 0:
         raise ValueError(f"oracle_geglu failed ({rc})")
     return out, out16
+
+
+def rmsnorm(x_bf16, gamma_bf16, eps: float):
+    """RMS normalisation with scale (1 + gamma): bf16 bits [M, K] in, bf16 bits [M, K] out."""
+    x_bf16 = _c(x_bf16, np.uint16)
+    gamma_bf16 = _c(gamma_bf16, np.uint16)
+    M, K = x_bf16.shape
+    if gamma_bf16.shape != (K,):
+        raise ValueError("gamma must be [K]")
+    out = np.empty((M, K), np.uint16)
+    rc = _load().oracle_rmsnorm(_ptr(x_bf16), _ptr(gamma_bf16), float(eps), M, K, _ptr(out))
+    if rc != 0:
+        raise ValueError(f"oracle_rmsnorm failed ({rc})")
+    return out

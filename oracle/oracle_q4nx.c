@@ -37,9 +37,9 @@
  * widened bf16 scale/offset; w16 is the round-to-nearest-even bf16 of w32.
  * The projection accumulates (double)x * (double)w32 sequentially in k.
  *
- * Gated GELU epilogue (a next step beyond the paper's FusedDQP, which leaves the activation to a separate kernel):
- * oracle_gelu_tanh / oracle_geglu below; pinned against the error-function form, symmetry, limits and a
- * pairing case with exact products.
+ * RMS normalisation prologue and gated GELU epilogue (next steps beyond the paper's FusedDQP, which leaves both to
+ * separate kernels): oracle_rmsnorm, oracle_gelu_tanh / oracle_geglu below; pinned by closed-form rows, invariances,
+ * the error-function form, symmetry, limits and a pairing case with exact products.
  *
  * Pins (tests/test_oracle_pins.py): the paper's 5120-byte block, hand-written
  * byte dumps, closed-form worked examples, exact rational evaluation of eq. 3
@@ -249,6 +249,30 @@ int oracle_geglu(const double *y, int64_t M, int64_t N, double *out, uint16_t *o
                 out[m * H + 16 * j + r] = v;
                 if (out_bf16) out_bf16[m * H + 16 * j + r] = fp32_to_bf16_rne((float)v);
             }
+    return 0;
+}
+
+/* ---- RMS normalisation ahead of a projection (next-step prologue) -------- */
+
+/* out[m][k] = bf16( x[m][k] * r_m * (1 + gamma[k]) ),  r_m = 1 / sqrt(mean_k x[m][k]^2 + eps), evaluated in fp64 and
+ * rounded fp64 -> fp32 -> bf16 (nearest-even), the way the model family's reference normalisation hands bf16
+ * activations to the projection that follows it.  The paper lists RMS normalisation among the vector kernels between
+ * projections without a formula; this is the form Gemma's published code uses (scale = 1 + weight). */
+int oracle_rmsnorm(const uint16_t *x_bf16, const uint16_t *gamma_bf16, double eps, int64_t M, int64_t K,
+                   uint16_t *out_bf16) {
+    if (!x_bf16 || !gamma_bf16 || !out_bf16 || M < 1 || K < 1) return 1;
+    for (int64_t m = 0; m < M; ++m) {
+        double ss = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            const double v = bf16_bits_to_double(x_bf16[m * K + k]);
+            ss += v * v;
+        }
+        const double r = 1.0 / sqrt(ss / (double)K + eps);
+        for (int64_t k = 0; k < K; ++k) {
+            const double v = bf16_bits_to_double(x_bf16[m * K + k]) * r * (1.0 + bf16_bits_to_double(gamma_bf16[k]));
+            out_bf16[m * K + k] = fp32_to_bf16_rne((float)v);
+        }
+    }
     return 0;
 }
 

@@ -375,3 +375,48 @@ def test_geglu_pairs_rows_r_and_r_plus_16_of_each_strip():
     # a gate of zero silences its output whatever the up value is
     y[:, 0] = 0.0
     assert np.all(oracle.geglu(y)[0][:, 0] == 0.0)
+
+
+# ---- RMS normalisation prologue (next step beyond FusedDQP) ---------------------------------------------------------
+
+def _bf(vals):
+    return synthgen.bf16_bits(np.asarray(vals, np.float32))
+
+
+def test_rmsnorm_hand_case_invariances_and_unit_power():
+    import math
+
+    K = 32
+    x = np.zeros((1, K), np.float32)
+    x[0, 0], x[0, 1] = 3.0, 4.0                       # mean square = 25 / 32, r = sqrt(32) / 5
+    zero = _bf(np.zeros(K))
+    out = synthgen.bf16_to_f32(oracle.rmsnorm(_bf(x), zero, 0.0))
+    r = math.sqrt(32.0) / 5.0
+    assert abs(out[0, 0] - 3.0 * r) <= 2.0 ** -8 * 3.0 * r and abs(out[0, 1] - 4.0 * r) <= 2.0 ** -8 * 4.0 * r
+    assert np.all(out[0, 2:] == 0.0)
+    assert out[0, 0] == synthgen.bf16_to_f32(_bf([3.0 * r]))[0]          # exactly the nearest bf16
+    # a constant row normalises to +-1 whatever its magnitude; with eps it is 1 / sqrt(1 + eps / c^2)
+    for c in (0.5, -7.0, 1000.0):
+        o = synthgen.bf16_to_f32(oracle.rmsnorm(_bf(np.full((1, K), c)), zero, 0.0))
+        assert np.all(o == math.copysign(1.0, c))
+    o = synthgen.bf16_to_f32(oracle.rmsnorm(_bf(np.full((1, K), 2.0)), zero, 12.0))   # 1 / sqrt(1 + 12/4) = 0.5
+    assert np.all(o == 0.5)
+    # power-of-two rescaling of the input changes nothing when eps = 0; gamma = 1 doubles every output exactly
+    xs = synthgen.activations(3, 4, 256)
+    a = oracle.rmsnorm(xs, _bf(np.zeros(256)), 0.0)
+    x4 = _bf(synthgen.bf16_to_f32(xs) * 4.0)
+    assert np.array_equal(oracle.rmsnorm(x4, _bf(np.zeros(256)), 0.0), a)
+    b = oracle.rmsnorm(xs, _bf(np.ones(256)), 0.0)
+    assert np.array_equal(synthgen.bf16_to_f32(b), 2.0 * synthgen.bf16_to_f32(a))
+    # unit mean square of the output (gamma = 0, tiny eps) up to the bf16 rounding of each element
+    o = synthgen.bf16_to_f32(oracle.rmsnorm(xs, _bf(np.zeros(256)), 1e-12)).astype(np.float64)
+    assert np.all(np.abs((o * o).mean(axis=1) - 1.0) < 2.0 ** -7)
+    # every row has its own r: rows normalised together equal rows normalised one by one
+    for m in range(4):
+        assert np.array_equal(oracle.rmsnorm(xs[m:m + 1], _bf(np.zeros(256)), 1e-6), oracle.rmsnorm(xs, _bf(np.zeros(256)), 1e-6)[m:m + 1])
+    # gamma is indexed by k: a one-hot gamma touches exactly its own column
+    g = np.zeros(256, np.float32)
+    g[17] = 1.0
+    c = synthgen.bf16_to_f32(oracle.rmsnorm(xs, _bf(g), 0.0))
+    a32 = synthgen.bf16_to_f32(a)
+    assert np.array_equal(np.delete(c, 17, axis=1), np.delete(a32, 17, axis=1)) and np.array_equal(c[:, 17], 2.0 * a32[:, 17])
