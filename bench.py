@@ -195,8 +195,13 @@ def run_shape(args):
     stream = torch.cuda.Stream()
     sraw = stream.cuda_stream
 
+    gamma = torch.zeros(K, dtype=torch.int16, device="cuda")
+
     def launch(W):
-        fd.fdqp_run_epilogue(ctx, x, W, y, epi, M, K, N, sraw)
+        if args.rmsnorm:
+            fd.fdqp_run_rmsnorm_epilogue(ctx, x, gamma, 1e-6, W, y, epi, M, K, N, sraw)
+        else:
+            fd.fdqp_run_epilogue(ctx, x, W, y, epi, M, K, N, sraw)
 
     for i in range(max(3, args.warmup)):
         launch(copies[i % ncopies])
@@ -227,7 +232,7 @@ def run_shape(args):
     print(json.dumps({"shape": {"K": K, "N": N, "M": M}, "us_per_call": us, "GBps": gbs,
                       "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
                       "peak_kind": peak_kind, "weight_copies": ncopies, "steps": args.steps,
-                      "graph": bool(args.graph and not args.same_weights), "epilogue": args.epilogue,
+                      "graph": bool(args.graph and not args.same_weights), "epilogue": args.epilogue, "rmsnorm": bool(args.rmsnorm),
                       "launch": fd.fdqp_describe(ctx, M, K, N)}), flush=True)
     fd.fdqp_destroy(ctx)
 
@@ -544,6 +549,7 @@ def main():
     ap.add_argument("--param", action="append", help="library launch parameter key=value (repeatable)")
     ap.add_argument("--shape", help="K,N,M: time this one projection shape instead of the layer workload")
     ap.add_argument("--same-weights", action="store_true", help="with --shape: reuse one weight buffer (for ncu captures)")
+    ap.add_argument("--rmsnorm", action="store_true", help="with --shape: RMS-normalise x first (fused where possible)")
     ap.add_argument("--epilogue", default="none", choices=["none", "bf16", "geglu"],
                     help="with --shape: fused store-side epilogue (geglu: gate and up rows interleaved 16 by 16 along N)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")

@@ -163,6 +163,22 @@ typedef enum {
 FDQP_API fdqp_status fdqp_run_epilogue(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, void* out, int epilogue,
                               int64_t M, int64_t K, int64_t N, void* cuda_stream);
 
+/* fdqp_run_epilogue preceded, in the same launch where possible, by the RMS
+ * normalisation that comes before a projection in a decoder layer (the paper runs
+ * it as a vector kernel of its own and gives no formula; this is the form with
+ * scale 1 + weight, evaluated in fp32 and handed on as bf16):
+ *   x_n[m][k] = bf16( x[m][k] * rsqrt(mean_k x[m][k]^2 + eps) * (1 + gamma[k]) ),
+ *   out = epilogue( x_n * dequant(W) ).
+ *   gamma_bf16  device, [K] bf16, 16-byte aligned; eps >= 0
+ * The normalisation is fused into the GEMV kernel's activation preparation when the
+ * call is a single GEMV launch that prepares the whole row of x inside every CTA
+ * (about M * K <= 4096, e.g. every K = 2560 projection at M = 1); otherwise a small
+ * kernel writes x_n to a staging buffer of the context first.  x is not modified.
+ * Everything else as fdqp_run_epilogue; FDQP_ERR_ARG also for a null gamma or eps < 0. */
+FDQP_API fdqp_status fdqp_run_rmsnorm_epilogue(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, float eps,
+                                      const void* W_q4nx, void* out, int epilogue, int64_t M, int64_t K, int64_t N,
+                                      void* cuda_stream);
+
 /* Same projection with HOST activations and result: copies x (host, [M][K] bf16)
  * to the context's device staging buffer, runs fdqp_run, copies y back to `y_host`
  * (host, [M][N] fp32) and synchronises the stream before returning.  W stays a

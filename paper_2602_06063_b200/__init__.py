@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     EPI_NONE,
     fdqp_run,
     fdqp_run_epilogue,
+    fdqp_run_rmsnorm_epilogue,
     fdqp_run_host,
     fdqp_run_host_async,
     fdqp_run_noalloc,

@@ -23,7 +23,7 @@ STATUS = {
 
 EXPORTS = [
     "q4nx_packed_bytes", "q4nx_pack", "q4nx_unpack", "fdqp_create", "fdqp_destroy", "fdqp_run", "fdqp_run_host",
-    "fdqp_run_host_async", "fdqp_run_epilogue",
+    "fdqp_run_host_async", "fdqp_run_epilogue", "fdqp_run_rmsnorm_epilogue",
     "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
     "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc",
 ]
@@ -66,6 +66,8 @@ def load_library():
     lib.fdqp_run_host.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_run_epilogue.restype = ci
     lib.fdqp_run_epilogue.argtypes = [vp, vp, vp, vp, ci, i64, i64, i64, vp]
+    lib.fdqp_run_rmsnorm_epilogue.restype = ci
+    lib.fdqp_run_rmsnorm_epilogue.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp, ci, i64, i64, i64, vp]
     lib.fdqp_run_host_async.restype = ci
     lib.fdqp_run_host_async.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_run_noalloc.restype = ci
@@ -180,6 +182,14 @@ def fdqp_run_epilogue(ctx: int, x_bf16, W_q4nx, out, epilogue: int, M: int, K: i
     EPI_GEGLU_BF16 (bf16 [M, N/2]; gate and up rows interleaved sixteen by sixteen in W, see fdqp.h)."""
     _check(load_library().fdqp_run_epilogue(ctx, _addr(x_bf16), _addr(W_q4nx), _addr(out), int(epilogue), M, K, N,
                                             _stream(stream)), "fdqp_run_epilogue", ctx)
+
+
+def fdqp_run_rmsnorm_epilogue(ctx: int, x_bf16, gamma_bf16, eps: float, W_q4nx, out, epilogue: int, M: int, K: int,
+                              N: int, stream=None) -> None:
+    """fdqp_run_epilogue on x RMS-normalised with scale (1 + gamma) (fused into the launch where possible, see fdqp.h)."""
+    _check(load_library().fdqp_run_rmsnorm_epilogue(ctx, _addr(x_bf16), _addr(gamma_bf16), float(eps), _addr(W_q4nx),
+                                                    _addr(out), int(epilogue), M, K, N, _stream(stream)),
+           "fdqp_run_rmsnorm_epilogue", ctx)
 
 
 def fdqp_run_host(ctx: int, x_host_bf16, W_q4nx, y_host, M: int, K: int, N: int, stream=None) -> None:

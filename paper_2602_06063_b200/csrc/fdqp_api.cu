@@ -22,6 +22,8 @@ cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, in
 cudaError_t prefill_set_smem_limit();
 cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, uint16_t* y16, int epi, float* ws,
                            int* status, int M, int K, int N, int pair, int Z, cudaStream_t stream);
+cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* gamma, float eps, uint16_t* out, int M, int K,
+                           cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
 }  // namespace fdqp
 
@@ -35,6 +37,7 @@ struct fdqp_ctx {
     float* ws_edge = nullptr;
     float* ws_full = nullptr;
     float* pf_ws = nullptr;      // partial results of K-split tensor-core calls
+    uint16_t* x_norm = nullptr;  // normalised activations of calls whose RMS normalisation cannot be fused (max_M x max_K)
     uint8_t* x_spread = nullptr; // small x copied with its rows further apart (see kSpreadBelowBytes)
     size_t pf_ws_bytes = 0;
     int* tickets = nullptr;
@@ -145,7 +148,7 @@ SmemLayout smem_layout(const fdqp_ctx* ctx, int M, int nbz, int cw, int ctas_per
     L.xsum_bytes = M <= kColsMaxTokens ? 0u : tiles * 64u;         // per-token {sum x, unit} (plane mode only)
     L.part_bytes = 2u * (uint32_t)cw * kStripRows * (uint32_t)M * 4u * (M <= kColsMaxTokens ? (uint32_t)kColsPartTerms : 1u);
     L.fixed = round_up(L.xs_bytes, 128) + round_up(L.xsum_bytes, 128) + round_up(L.part_bytes, 128) +
-              (2u * kMaxStages + 5u) * 8u + 128u;
+              (2u * kMaxStages + 6u) * 8u + 512u + 128u;
     const uint32_t per_cta = (uint32_t)ctx->smem_optin / (uint32_t)ctas_per_sm - (ctas_per_sm > 1 ? 1024u : 0u);
     L.nstage = per_cta > L.fixed ? (int)((per_cta - L.fixed) / L.stage_bytes) : 0;
     if (L.nstage > kMaxStages) L.nstage = kMaxStages;
@@ -223,7 +226,7 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     p->off_xsum = p->off_xs + round_up(L.xs_bytes, 128);
     p->off_part = p->off_xsum + round_up(L.xsum_bytes, 128);
     p->off_bar = p->off_part + round_up(L.part_bytes, 128);
-    p->smem_bytes = p->off_bar + (2u * (uint32_t)nstage + 5u) * 8u;
+    p->smem_bytes = p->off_bar + (2u * (uint32_t)nstage + 6u) * 8u + 512u;  // barriers, then the fused normalisation's sums
     p->evict_first = ctx->p_evict >= 0 ? (ctx->p_evict != 0) : 1;
     p->debug = ctx->p_debug > 0 ? (int)ctx->p_debug : 0;
     // work items (8 activations each) per CTA if x is prepared in-kernel; beyond this a preparation kernel is cheaper
@@ -286,6 +289,7 @@ extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, in
         if ((e = cudaMalloc(&ctx->ws_edge, slot * 2 * (size_t)ctx->sm_count * kMaxCtasPerSm))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->ws_full, slot * (size_t)kMaxSplit * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->tickets, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMalloc(&ctx->x_norm, (size_t)max_M * (size_t)max_K * 2))) { st = cuda_fail(nullptr, e, ""); break; }
         if (max_M > kMaxTokens) {
             // K-split tensor-core calls (shapes with few output tiles): up to kMaxSplit partial results, capped
             const size_t want = (size_t)kMaxSplit * (size_t)max_M * (size_t)max_N * 4;
@@ -321,6 +325,7 @@ extern "C" fdqp_status fdqp_destroy(fdqp_ctx* ctx) {
     if (ctx->ws_full) cudaFree(ctx->ws_full);
     if (ctx->pf_ws) cudaFree(ctx->pf_ws);
     if (ctx->x_spread) cudaFree(ctx->x_spread);
+    if (ctx->x_norm) cudaFree(ctx->x_norm);
     if (ctx->tickets) cudaFree(ctx->tickets);
     if (ctx->xq) cudaFree(ctx->xq);
     if (ctx->xsc) cudaFree(ctx->xsc);
@@ -336,14 +341,18 @@ namespace {
 
 // The projection with its epilogue: `out` is fp32 [M][N] (kEpiNone), bf16 [M][N] (kEpiBf16) or bf16 [M][N/2]
 // (kEpiGegluBf16).
-fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, void* out, int epi, int64_t M, int64_t K,
-                     int64_t N, void* cuda_stream) {
+// gamma != nullptr: x is RMS-normalised first, x <- bf16(x * rsqrt(mean_k x^2 + eps) * (1 + gamma)) per token row --
+// inside the GEMV kernel's activation preparation when that runs in-kernel on the whole row, else by a kernel of its own.
+fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, float eps, const void* W_q4nx, void* out,
+                     int epi, int64_t M, int64_t K, int64_t N, void* cuda_stream) {
     if (!ctx || !x_bf16 || !W_q4nx || !out) return FDQP_ERR_ARG;
+    if (gamma_bf16 && !aligned16(gamma_bf16)) return FDQP_ERR_ALIGN;
+    if (gamma_bf16 && !(eps >= 0.f)) return FDQP_ERR_ARG;
     if (epi != kEpiNone && epi != kEpiBf16 && epi != kEpiGegluBf16) return FDQP_ERR_ARG;
     fdqp_status st = check_shape(ctx, M, K, N);
     if (st != FDQP_OK) return st;
     if (!aligned16(x_bf16) || !aligned16(W_q4nx) || !aligned16(out)) return FDQP_ERR_ALIGN;
-    if (epi != kEpiNone && ctx->p_path == 1) return FDQP_ERR_ARG;  // the plain self-check kernel writes fp32 only
+    if ((epi != kEpiNone || gamma_bf16) && ctx->p_path == 1) return FDQP_ERR_ARG;  // the plain self-check kernel does neither
     float* y = epi == kEpiNone ? static_cast<float*>(out) : nullptr;
     uint16_t* y16 = epi == kEpiNone ? nullptr : static_cast<uint16_t*>(out);
     const int64_t n_out = epi == kEpiGegluBf16 ? N / 2 : N;  // output values per token row
@@ -352,7 +361,22 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, void
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const uint8_t* W = static_cast<const uint8_t*>(W_q4nx);
     const uint16_t* x = static_cast<const uint16_t*>(x_bf16);
+    const uint16_t* gamma = static_cast<const uint16_t*>(gamma_bf16);
     cudaError_t e;
+    bool fuse_norm = false;
+    if (gamma) {
+        // fused when the call is one GEMV launch that prepares the whole row of x inside every CTA
+        GemvPlan probe;
+        int cw = 0;
+        fuse_norm = M <= kMaxTokens && !use_prefill(ctx, M, K, N) && plan_gemv(ctx, (int)M, (int)K, (int)N, &cw, &probe) &&
+                    probe.prep_inline && probe.Z == 1 && (K / kGroup) * M * 4 <= (int64_t)cw * 32;
+        if (!fuse_norm) {
+            if ((e = rmsnorm_launch(x, gamma, eps, ctx->x_norm, (int)M, (int)K, stream)))
+                return cuda_fail(ctx, e, "RMS normalisation launch");
+            ctx->launches += 1;
+            x = ctx->x_norm;
+        }
+    }
     if (ctx->p_path == 1) {
         if ((e = plain_launch(W, x, y, (int)M, (int)K, (int)N, stream))) return cuda_fail(ctx, e, "plain kernel launch");
         ctx->launches += 1;
@@ -386,6 +410,11 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, void
         plan.y = y ? y + m0 * N : nullptr;
         plan.y16 = y16 ? y16 + m0 * n_out : nullptr;
         plan.epi = epi;
+        if (fuse_norm) {
+            plan.norm = 1;
+            plan.gamma = gamma;
+            plan.eps = eps;
+        }
         if (!plan.prep_inline) {
             if ((e = xprep_launch(plan.x, ctx->xq, ctx->xsc, mc, (int)K, stream)))
                 return cuda_fail(ctx, e, "x preparation launch");
@@ -412,12 +441,19 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, void
 
 extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, float* y, int64_t M, int64_t K,
                                 int64_t N, void* cuda_stream) {
-    return run_impl(ctx, x_bf16, W_q4nx, y, kEpiNone, M, K, N, cuda_stream);
+    return run_impl(ctx, x_bf16, nullptr, 0.f, W_q4nx, y, kEpiNone, M, K, N, cuda_stream);
 }
 
 extern "C" fdqp_status fdqp_run_epilogue(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, void* out, int epilogue,
                                          int64_t M, int64_t K, int64_t N, void* cuda_stream) {
-    return run_impl(ctx, x_bf16, W_q4nx, out, epilogue, M, K, N, cuda_stream);
+    return run_impl(ctx, x_bf16, nullptr, 0.f, W_q4nx, out, epilogue, M, K, N, cuda_stream);
+}
+
+extern "C" fdqp_status fdqp_run_rmsnorm_epilogue(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, float eps,
+                                                 const void* W_q4nx, void* out, int epilogue, int64_t M, int64_t K, int64_t N,
+                                                 void* cuda_stream) {
+    if (!gamma_bf16) return FDQP_ERR_ARG;
+    return run_impl(ctx, x_bf16, gamma_bf16, eps, W_q4nx, out, epilogue, M, K, N, cuda_stream);
 }
 
 extern "C" fdqp_status fdqp_run_host_async(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,

@@ -327,7 +327,7 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][Mo
 }
 
 // CW consumer warps (8 or 16); MODE as above (1: M = 1, 3: M = 2, 2: M = 3..8); EPI: built with the bf16 epilogues
-// (the fp32-only build keeps its stores free of the epilogue's branches).
+// and the fused RMS normalisation (the plain build keeps its stores and its preparation free of their branches).
 // A ring stage holds CB = (CW / 8) * BPW blocks; warp w owns group-tile (w & 7) of the BPW (2 or 4) consecutive
 // blocks starting at BPW * (w >> 3) of every stage.  More blocks per stage = fewer barrier round trips per tile.
 // Warps CW+1 .. CW+NR are reducers (NR = CW / 8): reducer r completes the strip pieces with piece % NR == r.
@@ -380,6 +380,8 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         mbar_init(red_empty0 + 8u * tid, 1);
     }
     if (tid == 2) mbar_init(x_bar, 1);
+    // fused RMS normalisation: one sum of squares per (group-tile, token) quad, up to 128 of them
+    float* const norm_q = reinterpret_cast<float*>(smem + p.off_bar + (2u * (uint32_t)nstage + 6u) * 8u);
     mbar_fence_init();
     __syncthreads();
     if (warp == 0) FDQP_STAMP(1);
@@ -568,6 +570,43 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                 asm volatile("" ::"r"(v[0].x), "r"(v[kBatch - 1].x));
                 if (warp == 0 && base == 0) FDQP_STAMP(8);
 #endif
+                if (EPI && p.norm) {
+                    // RMS normalisation in place (the plan guarantees one item per thread at most and the whole row in
+                    // this CTA): sum of squares per token over all quads, then x <- bf16(x * r * (1 + gamma))
+                    const bool valid = tid < items;
+                    const int tm = tid >> 2, tok = valid ? tm % M : 0, tile = valid ? tm / M : 0;
+                    const uint4 gm = xprep_load(p.gamma, K, tile0 + tile, 0, tid & 3, valid);
+                    const uint32_t xw[4] = {v[0].x, v[0].y, v[0].z, v[0].w}, gw[4] = {gm.x, gm.y, gm.z, gm.w};
+                    float f[8], ss = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        f[2 * i] = __uint_as_float(xw[i] << 16);
+                        f[2 * i + 1] = __uint_as_float(xw[i] & 0xffff0000u);
+                        ss = fmaf(f[2 * i], f[2 * i], ss);
+                        ss = fmaf(f[2 * i + 1], f[2 * i + 1], ss);
+                    }
+                    ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+                    ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+                    if (valid && (tid & 3) == 0) norm_q[tm] = ss;  // tm = tile * M + tok
+                    asm volatile("bar.sync 1, %0;" ::"n"(CW * 32) : "memory");
+                    // the row's quads in a fixed order (four interleaved chains): the same sum in every thread and run
+                    float t4[4] = {0.f, 0.f, 0.f, 0.f};
+                    int t2 = 0;
+                    for (; t2 + 4 <= ntiles; t2 += 4) {
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) t4[c4] += norm_q[(t2 + c4) * M + tok];
+                    }
+                    for (; t2 < ntiles; ++t2) t4[0] += norm_q[t2 * M + tok];
+                    const float tot = (t4[0] + t4[1]) + (t4[2] + t4[3]);
+                    const float r = rsqrtf(tot / (float)K + p.eps);
+                    uint32_t o[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float g0 = 1.0f + __uint_as_float(gw[i] << 16), g1 = 1.0f + __uint_as_float(gw[i] & 0xffff0000u);
+                        o[i] = (uint32_t)f32_to_bf16_rne(f[2 * i] * r * g0) | ((uint32_t)f32_to_bf16_rne(f[2 * i + 1] * r * g1) << 16);
+                    }
+                    v[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                }
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
                     const int idx = base + u * CW * 32 + tid;
@@ -826,6 +865,63 @@ extern "C" __attribute__((visibility("default"))) int fdqp_trace_read(unsigned l
 }
 #endif
 
+// RMS normalisation on its own (the calls whose activation preparation does not happen inside a GEMV CTA): one CTA per
+// token row, out[m][k] = bf16(x * rsqrt(mean(x^2) + eps) * (1 + gamma[k])).
+__global__ void __launch_bounds__(256) fdqp_rmsnorm_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
+                                                            float eps, uint16_t* __restrict__ out, int K) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // x may be the previous launch's output
+    __shared__ float part[8];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint16_t* xr = x + (int64_t)blockIdx.x * K;
+    uint16_t* orow = out + (int64_t)blockIdx.x * K;
+    float ss = 0.f;
+    for (int k = tid * 8; k < K; k += 256 * 8) {  // K is a multiple of 32
+        const uint4 w = *reinterpret_cast<const uint4*>(xr + k);
+        const uint32_t xw[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float a = __uint_as_float(xw[i] << 16), b = __uint_as_float(xw[i] & 0xffff0000u);
+            ss = fmaf(a, a, ss);
+            ss = fmaf(b, b, ss);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if (lane == 0) part[warp] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += part[w];
+    const float r = rsqrtf(tot / (float)K + eps);
+    for (int k = tid * 8; k < K; k += 256 * 8) {
+        const uint4 w = *reinterpret_cast<const uint4*>(xr + k), g = *reinterpret_cast<const uint4*>(gamma + k);
+        const uint32_t xw[4] = {w.x, w.y, w.z, w.w}, gw[4] = {g.x, g.y, g.z, g.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float a = __uint_as_float(xw[i] << 16), b = __uint_as_float(xw[i] & 0xffff0000u);
+            const float g0 = 1.0f + __uint_as_float(gw[i] << 16), g1 = 1.0f + __uint_as_float(gw[i] & 0xffff0000u);
+            o[i] = (uint32_t)f32_to_bf16_rne(a * r * g0) | ((uint32_t)f32_to_bf16_rne(b * r * g1) << 16);
+        }
+        *reinterpret_cast<uint4*>(orow + k) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* gamma, float eps, uint16_t* out, int M, int K,
+                           cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)M);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fdqp_rmsnorm_kernel, x, gamma, eps, out, K);
+}
+
 // ---- host-visible launchers ------------------------------------------------------------------
 
 template <int CW, int MODE, int BPW>
@@ -840,7 +936,7 @@ static cudaError_t launch_one(const GemvPlan& p, cudaStream_t stream) {
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return p.epi == kEpiNone ? cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<CW, MODE, BPW, false>, p)
+    return (p.epi == kEpiNone && !p.norm) ? cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<CW, MODE, BPW, false>, p)
                              : cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<CW, MODE, BPW, true>, p);
 }
 

@@ -30,6 +30,9 @@ struct GemvPlan {
     float* y;            // fp32 output (epilogue kEpiNone)
     uint16_t* y16;       // bf16 output (other epilogues)
     int epi;
+    const uint16_t* gamma;  // RMS normalisation of x fused into the in-kernel activation preparation (norm != 0):
+    float eps;              //   x <- bf16(x * rsqrt(mean(x^2) + eps) * (1 + gamma)), per token row
+    int norm;
             // device, [M][N]
     float* ws_edge;       // device, [grid][2][32*kMaxTokens] partial sums of strips shared between CTAs
     float* ws_full;       // device, [Z][S][32*kMaxTokens] partial sums of whole strip-slices (Z > 1)

@@ -154,3 +154,79 @@ def test_gemma3_12b_gate_up_gated_gelu_full_size(ctx):
         out = synthgen.bf16_to_f32(run_epilogue(ctx, case, fd.EPI_GEGLU_BF16, M=M)).astype(np.float64)
         assert np.all(np.isfinite(out))
         assert np.all(np.abs(out - out_ref[:M]) <= bound[:M]), f"12B gate|up gated GELU M={M}"
+
+
+# ---- RMS normalisation ahead of the projection ----------------------------------------------------------------------
+
+def run_norm(ctx, case, gamma_dev, eps, epi, M=None):
+    M = case.M if M is None else M
+    n_out = case.N // 2 if epi == fd.EPI_GEGLU_BF16 else case.N
+    dt = torch.float32 if epi == fd.EPI_NONE else torch.int16
+    out = torch.zeros((M, n_out), dtype=dt, device="cuda")
+    fd.fdqp_run_rmsnorm_epilogue(ctx, case.x_dev, gamma_dev, eps, case.W_dev, out, epi, M, case.K, case.N)
+    torch.cuda.synchronize()
+    assert fd.fdqp_last_status(ctx) == 0
+    return out.cpu().numpy()
+
+
+# (K, N, M, launch parameters, launches expected for the call)
+NORM_CASES = [
+    (2560, 2048, 1, {}, 1),                # fused into the GEMV launch
+    (1152, 288, 3, {}, 1),                 # fused, three token rows, tail block
+    (2560, 512, 2, {}, 3),                 # too many items for in-kernel preparation: norm kernel + preparation + GEMV
+    (10240, 320, 1, {}, 3),
+    (1056, 320, 20, {"path": 2}, 7),       # norm kernel, then three GEMV chunks with their preparation
+    (1056, 320, 40, {"path": 3}, 3),       # norm kernel + tensor-core kernel (K slices) + its sum kernel
+    (544, 1056, 300, {"path": 3}, 2),
+]
+
+
+@pytest.mark.parametrize("K,N,M,params,launches", NORM_CASES)
+def test_rmsnorm_then_projection_matches_oracle(fresh, K, N, M, params, launches):
+    case = Case(K, N, M, seed=6000 + K + N + M, amp=3.0)
+    gamma = synthgen.bf16_bits((0.25 * synthgen.bf16_to_f32(synthgen.activations(6100 + K, 1, K))[0]).astype(np.float32))
+    gamma_dev = torch.from_numpy(gamma.view(np.int16)).cuda()
+    eps = 1e-6
+    for k, v in params.items():
+        fd.fdqp_set_param(fresh, k, v)
+    before = fd.fdqp_launch_count(fresh)
+    y = run_norm(fresh, case, gamma_dev, eps, fd.EPI_NONE)
+    assert fd.fdqp_launch_count(fresh) - before == launches
+    x_n = oracle.rmsnorm(case.x, gamma, eps)
+    y_ref, a_ref = oracle.project(x_n, case.w.codes, case.w.scales, case.w.offsets, nthreads=8)
+    err = np.abs(y.astype(np.float64) - y_ref)
+    assert np.all(np.isfinite(y)) and np.all(err <= REL_TOL * a_ref + ABS_TOL)
+    # together with the gated GELU epilogue
+    out = synthgen.bf16_to_f32(run_norm(fresh, case, gamma_dev, eps, fd.EPI_GEGLU_BF16).view(np.uint16)).astype(np.float64)
+    out_ref, _ = oracle.geglu(y_ref)
+    assert np.all(np.abs(out - out_ref) <= geglu_bound(y_ref, a_ref))
+
+
+@pytest.mark.parametrize("K,N,M,params", [(2560, 1024, 1, {}), (2560, 512, 2, {}), (512, 288, 40, {"path": 3})])
+def test_rmsnorm_of_constant_rows_is_exact(fresh, K, N, M, params):
+    # a row of constant magnitude normalises to +-1 exactly (gamma = 0), whatever the magnitude: the result must be
+    # bit-equal to the plain projection of that +-1 row
+    case = Case(K, N, M, seed=61)
+    signs = np.where(synthgen.bf16_to_f32(case.x) >= 0, 1.0, -1.0).astype(np.float32)
+    mags = np.array([0.37, 5.0, 1000.0, 0.002] * ((M + 3) // 4), np.float32)[:M, None]
+    scaled = Case(K, N, M, seed=61, weights=case.w, x=synthgen.bf16_bits(signs * mags))
+    unit = Case(K, N, M, seed=61, weights=case.w, x=synthgen.bf16_bits(signs))
+    for k, v in params.items():
+        fd.fdqp_set_param(fresh, k, v)
+    gamma_dev = torch.zeros(K, dtype=torch.int16, device="cuda")
+    assert np.array_equal(run_norm(fresh, scaled, gamma_dev, 0.0, fd.EPI_NONE), unit.run(fresh))
+
+
+def test_rmsnorm_argument_errors(fresh):
+    case = Case(256, 64, 1, seed=9)
+    out = torch.empty((1, 64), dtype=torch.float32, device="cuda")
+    g = torch.zeros(256 + 8, dtype=torch.int16, device="cuda")
+    lib = fd.load_library()
+    s = torch.cuda.current_stream().cuda_stream
+    a = (fresh, case.x_dev.data_ptr())
+    b = (case.W_dev.data_ptr(), out.data_ptr(), 0, 1, 256, 64, s)
+    assert lib.fdqp_run_rmsnorm_epilogue(*a, None, 1e-6, *b) == 1                  # null gamma
+    assert lib.fdqp_run_rmsnorm_epilogue(*a, g.data_ptr() + 2, 1e-6, *b) == 3      # misaligned gamma
+    assert lib.fdqp_run_rmsnorm_epilogue(*a, g.data_ptr(), -1.0, *b) == 1          # negative eps
+    assert lib.fdqp_run_rmsnorm_epilogue(*a, g.data_ptr(), 1e-6, *b) == 0
+    torch.cuda.synchronize()
