@@ -56,6 +56,8 @@ def _load():
         lib.oracle_geglu.argtypes = [p, i64, i64, p, p]
         lib.oracle_rmsnorm.restype = ci
         lib.oracle_rmsnorm.argtypes = [p, p, ctypes.c_double, i64, i64, p]
+        lib.oracle_decode_attention.restype = ci
+        lib.oracle_decode_attention.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, ctypes.c_double, p, p]
         lib.oracle_max_threads.restype = ci
         _lib = lib
     return _lib
@@ -179,3 +181,22 @@ def rmsnorm(x_bf16, gamma_bf16, eps: float):
     if rc != 0:
         raise ValueError(f"oracle_rmsnorm failed ({rc})")
     return out
+
+
+def decode_attention(q, K, V, L: int, window: int = 0, scale: float = 1.0):
+    """Attention of one new token over a KV cache (the paper's decoding-step attention; grouped queries, optional
+    sliding window): q [H, d], K and V [G, pitch, d] bf16 bits -> (out [H, d] fp64, sum_j p_j |v_j| [H, d] fp64)."""
+    q = _c(q, np.uint16)
+    K = _c(K, np.uint16)
+    V = _c(V, np.uint16)
+    H, d = q.shape
+    G, pitch, d2 = K.shape
+    if d2 != d or V.shape != K.shape:
+        raise ValueError("K and V must be [G, pitch, d] with q's d")
+    out = np.empty((H, d), np.float64)
+    absw = np.empty((H, d), np.float64)
+    rc = _load().oracle_decode_attention(_ptr(q), _ptr(K), _ptr(V), H, G, d, L, pitch, window, float(scale), _ptr(out),
+                                         _ptr(absw))
+    if rc != 0:
+        raise ValueError(f"oracle_decode_attention failed ({rc})")
+    return out, absw

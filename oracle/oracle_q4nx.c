@@ -40,6 +40,8 @@
  * RMS normalisation prologue and gated GELU epilogue (next steps beyond the paper's FusedDQP, which leaves both to
  * separate kernels): oracle_rmsnorm, oracle_gelu_tanh / oracle_geglu below; pinned by closed-form rows, invariances,
  * the error-function form, symmetry, limits and a pairing case with exact products.
+ * Decode attention over a KV cache (the paper's second decode kernel, FlowKV, computes it chunk by chunk):
+ * oracle_decode_attention is the plain softmax-weighted sum; pinned by closed forms and invariances.
  *
  * Pins (tests/test_oracle_pins.py): the paper's 5120-byte block, hand-written
  * byte dumps, closed-form worked examples, exact rational evaluation of eq. 3
@@ -49,6 +51,7 @@
  */
 #include <stddef.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 #include <math.h>
 #ifdef _OPENMP
@@ -273,6 +276,55 @@ int oracle_rmsnorm(const uint16_t *x_bf16, const uint16_t *gamma_bf16, double ep
             out_bf16[m * K + k] = fp32_to_bf16_rne((float)v);
         }
     }
+    return 0;
+}
+
+/* ---- decode attention over a KV cache (next step: the other memory-bound half of decode) -------------------------- */
+
+/* The paper's attention at decoding step t (its equation for causal attention during decoding): the new token's query
+ * attends to the keys of all earlier positions and itself,
+ *     o = sum_j softmax_j(scale * q . k_j) v_j ,
+ * in a local layer only to the last `window` positions; with grouped-query attention query head h reads KV head
+ * h / (H / G).  (The paper omits the scale "for simplicity"; it is an argument here.)  This is that definition written
+ * out in fp64: scores, their maximum, exponentials, the sum, the weighted sum -- no chunking.
+ *   q    [H][d]         bf16 bits
+ *   K, V [G][pitch][d]  bf16 bits; positions 0 .. L-1 of every head are valid
+ *   window <= 0 or >= L: all L positions; else positions L - window .. L - 1
+ *   out  [H][d] fp64;  absw (may be NULL) [H][d] = sum_j p_j |v_j|, the scale of the result's rounding error */
+int oracle_decode_attention(const uint16_t *q, const uint16_t *K, const uint16_t *V, int64_t H, int64_t G, int64_t d,
+                            int64_t L, int64_t pitch, int64_t window, double scale, double *out, double *absw) {
+    if (!q || !K || !V || !out || H < 1 || G < 1 || (H % G) != 0 || d < 1 || L < 1 || pitch < L) return 1;
+    const int64_t j0 = (window > 0 && window < L) ? L - window : 0;
+    const int64_t n = L - j0;
+    double *s = (double *)malloc((size_t)n * sizeof(double));
+    if (!s) return 2;
+    for (int64_t h = 0; h < H; ++h) {
+        const int64_t g = h / (H / G);
+        const uint16_t *Kg = K + g * pitch * d, *Vg = V + g * pitch * d;
+        double smax = -INFINITY;
+        for (int64_t j = 0; j < n; ++j) {
+            double acc = 0.0;
+            for (int64_t i = 0; i < d; ++i) acc += bf16_bits_to_double(q[h * d + i]) * bf16_bits_to_double(Kg[(j0 + j) * d + i]);
+            s[j] = scale * acc;
+            if (s[j] > smax) smax = s[j];
+        }
+        double denom = 0.0;
+        for (int64_t j = 0; j < n; ++j) {
+            s[j] = exp(s[j] - smax);
+            denom += s[j];
+        }
+        for (int64_t i = 0; i < d; ++i) {
+            double acc = 0.0, aacc = 0.0;
+            for (int64_t j = 0; j < n; ++j) {
+                const double v = bf16_bits_to_double(Vg[(j0 + j) * d + i]);
+                acc += s[j] * v;
+                aacc += s[j] * fabs(v);
+            }
+            out[h * d + i] = acc / denom;
+            if (absw) absw[h * d + i] = aacc / denom;
+        }
+    }
+    free(s);
     return 0;
 }
 

@@ -420,3 +420,67 @@ def test_rmsnorm_hand_case_invariances_and_unit_power():
     c = synthgen.bf16_to_f32(oracle.rmsnorm(xs, _bf(g), 0.0))
     a32 = synthgen.bf16_to_f32(a)
     assert np.array_equal(np.delete(c, 17, axis=1), np.delete(a32, 17, axis=1)) and np.array_equal(c[:, 17], 2.0 * a32[:, 17])
+
+
+# ---- decode attention over a KV cache (next step: the paper's second decode kernel) ---------------------------------
+
+def test_decode_attention_closed_forms_and_invariances():
+    import math
+
+    d, G, H, pitch = 8, 2, 4, 16
+    rng = np.random.default_rng(5)
+
+    def bf(a):
+        return synthgen.bf16_bits(np.asarray(a, np.float32))
+
+    # two positions, scores 0 and ln 3 -> weights 1/4 and 3/4 (q = e0, k0 = 0, k1 = ln3 * e0 is not bf16-exact, so use
+    # scale: q . k1 = 1 and scale = ln 3)
+    q = np.zeros((H, d), np.float32)
+    q[:, 0] = 1.0
+    K = np.zeros((G, pitch, d), np.float32)
+    V = np.zeros((G, pitch, d), np.float32)
+    K[:, 1, 0] = 1.0
+    V[0, 0], V[0, 1] = 4.0, 8.0
+    V[1, 0], V[1, 1] = -4.0, 16.0
+    out, absw = oracle.decode_attention(bf(q), bf(K), bf(V), L=2, scale=math.log(3.0))
+    assert np.allclose(out[0], 0.25 * 4.0 + 0.75 * 8.0, rtol=0, atol=1e-14)
+    assert np.allclose(out[2], 0.25 * -4.0 + 0.75 * 16.0, rtol=0, atol=1e-14)       # heads 2, 3 read KV head 1
+    assert np.array_equal(out[0], out[1]) and np.array_equal(out[2], out[3])
+    assert np.allclose(absw[2], 0.25 * 4.0 + 0.75 * 16.0, rtol=0, atol=1e-14)
+    # equal keys -> uniform weights -> the mean of the values; a query of zero does the same
+    L = 11
+    K = np.tile(rng.standard_normal((G, 1, d)).astype(np.float32), (1, pitch, 1))
+    V = rng.standard_normal((G, pitch, d)).astype(np.float32)
+    q = rng.standard_normal((H, d)).astype(np.float32)
+    Vb = synthgen.bf16_to_f32(bf(V)).astype(np.float64)
+    out, _ = oracle.decode_attention(bf(q), bf(K), bf(V), L=L, scale=0.3)
+    for h in range(H):
+        assert np.allclose(out[h], Vb[h // 2, :L].mean(axis=0), rtol=0, atol=1e-13)
+    K = rng.standard_normal((G, pitch, d)).astype(np.float32)
+    out0, _ = oracle.decode_attention(bf(np.zeros((H, d))), bf(K), bf(V), L=L)
+    assert np.allclose(out0[3], Vb[1, :L].mean(axis=0), rtol=0, atol=1e-13)
+    # the window keeps the last `window` positions: same as attention over a cache that only holds those
+    full, _ = oracle.decode_attention(bf(q), bf(K), bf(V), L=L, window=4, scale=0.5)
+    cut, _ = oracle.decode_attention(bf(q), bf(K[:, L - 4:L]), bf(V[:, L - 4:L]), L=4, scale=0.5)
+    assert np.array_equal(full, cut)
+    same, _ = oracle.decode_attention(bf(q), bf(K), bf(V), L=L, window=L + 5, scale=0.5)
+    allp, _ = oracle.decode_attention(bf(q), bf(K), bf(V), L=L, window=0, scale=0.5)
+    assert np.array_equal(same, allp)
+    # positions beyond L are never read
+    K2, V2 = K.copy(), V.copy()
+    K2[:, L:], V2[:, L:] = 1e30, -1e30
+    assert np.array_equal(oracle.decode_attention(bf(q), bf(K2), bf(V2), L=L, scale=0.5)[0], allp)
+    # a dominant score selects its value; an independent numpy softmax agrees everywhere
+    Kb = synthgen.bf16_to_f32(bf(K)).astype(np.float64)
+    qb = synthgen.bf16_to_f32(bf(q)).astype(np.float64)
+    for h in range(H):
+        s = 0.5 * Kb[h // 2, :L] @ qb[h]
+        p = np.exp(s - s.max())
+        p /= p.sum()
+        assert np.allclose(allp[h], p @ Vb[h // 2, :L], rtol=1e-13, atol=1e-14)
+    big = np.zeros((H, d), np.float32)
+    big[:, 1] = 64.0
+    Kd = np.zeros((G, pitch, d), np.float32)
+    Kd[:, 7, 1] = 8.0
+    sel, _ = oracle.decode_attention(bf(big), bf(Kd), bf(V), L=L)
+    assert np.allclose(sel[0], Vb[0, 7], rtol=0, atol=1e-12)
