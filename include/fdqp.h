@@ -179,6 +179,28 @@ FDQP_API fdqp_status fdqp_run_rmsnorm_epilogue(fdqp_ctx* ctx, const void* x_bf16
                                       const void* W_q4nx, void* out, int epilogue, int64_t M, int64_t K, int64_t N,
                                       void* cuda_stream);
 
+/* Decode attention over a KV cache (the paper's FlowKV, and FlowKV-SWA for local
+ * layers): the attention of ONE new token at decoding step L,
+ *     out[h] = sum_j softmax_j( scale * q[h] . K[g][j] ) V[g][j],   g = h / (H / G),
+ * over positions j = 0 .. L-1, or only the last `window` of them (window > 0 and
+ * < L: sliding-window attention); evaluated chunk by chunk with a running maximum
+ * and a running sum, K and V each read once.  (The paper's equation for the
+ * decoding step omits the scale; it is an argument here.)
+ *   q_bf16  device, [H][d] bf16
+ *   K_bf16, V_bf16  device, [G][pitch][d] bf16: position j of KV head g at
+ *           (g * pitch + j) * d; pitch >= L is the cache's capacity in positions
+ *   out     device, [H][d] fp32, fully overwritten
+ *   H % G == 0, H / G <= 8, H <= 64, d in {128, 256}; all pointers 16-byte aligned
+ * Probabilities pass through bf16 before they weight the values (tensor-core
+ * operand); bound against an fp64 evaluation, per element:
+ *     |out - ref| <= 6e-3 * sum_j p_j |V[g][j]| + 1e-5.
+ * Asynchronous on `cuda_stream`; no allocation; uses the context's workspace, so
+ * calls sharing a context must be ordered on one stream.
+ * Errors: FDQP_ERR_ARG, FDQP_ERR_SHAPE, FDQP_ERR_SIZE, FDQP_ERR_ALIGN, FDQP_ERR_CUDA. */
+FDQP_API fdqp_status fdqp_flowkv_decode(fdqp_ctx* ctx, const void* q_bf16, const void* K_bf16, const void* V_bf16, float* out,
+                               int64_t H, int64_t G, int64_t d, int64_t L, int64_t pitch, int64_t window, float scale,
+                               void* cuda_stream);
+
 /* Same projection with HOST activations and result: copies x (host, [M][K] bf16)
  * to the context's device staging buffer, runs fdqp_run, copies y back to `y_host`
  * (host, [M][N] fp32) and synchronises the stream before returning.  W stays a

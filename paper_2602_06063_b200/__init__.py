@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     fdqp_dequant,
     fdqp_describe,
     fdqp_destroy,
+    fdqp_flowkv_decode,
     fdqp_last_cuda_error,
     fdqp_last_status,
     fdqp_launch_count,

@@ -23,7 +23,7 @@ STATUS = {
 
 EXPORTS = [
     "q4nx_packed_bytes", "q4nx_pack", "q4nx_unpack", "fdqp_create", "fdqp_destroy", "fdqp_run", "fdqp_run_host",
-    "fdqp_run_host_async", "fdqp_run_epilogue", "fdqp_run_rmsnorm_epilogue",
+    "fdqp_run_host_async", "fdqp_run_epilogue", "fdqp_run_rmsnorm_epilogue", "fdqp_flowkv_decode",
     "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
     "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc",
 ]
@@ -68,6 +68,8 @@ def load_library():
     lib.fdqp_run_epilogue.argtypes = [vp, vp, vp, vp, ci, i64, i64, i64, vp]
     lib.fdqp_run_rmsnorm_epilogue.restype = ci
     lib.fdqp_run_rmsnorm_epilogue.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp, ci, i64, i64, i64, vp]
+    lib.fdqp_flowkv_decode.restype = ci
+    lib.fdqp_flowkv_decode.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, ctypes.c_float, vp]
     lib.fdqp_run_host_async.restype = ci
     lib.fdqp_run_host_async.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_run_noalloc.restype = ci
@@ -190,6 +192,14 @@ def fdqp_run_rmsnorm_epilogue(ctx: int, x_bf16, gamma_bf16, eps: float, W_q4nx, 
     _check(load_library().fdqp_run_rmsnorm_epilogue(ctx, _addr(x_bf16), _addr(gamma_bf16), float(eps), _addr(W_q4nx),
                                                     _addr(out), int(epilogue), M, K, N, _stream(stream)),
            "fdqp_run_rmsnorm_epilogue", ctx)
+
+
+def fdqp_flowkv_decode(ctx: int, q_bf16, K_bf16, V_bf16, out, H: int, G: int, d: int, L: int, pitch: int, window: int,
+                       scale: float, stream=None) -> None:
+    """Attention of one new token over a KV cache (q [H, d], K and V [G, pitch, d] bf16 on the device -> out [H, d]
+    fp32); window > 0 restricts it to the last `window` positions."""
+    _check(load_library().fdqp_flowkv_decode(ctx, _addr(q_bf16), _addr(K_bf16), _addr(V_bf16), _addr(out), H, G, d, L,
+                                             pitch, window, float(scale), _stream(stream)), "fdqp_flowkv_decode", ctx)
 
 
 def fdqp_run_host(ctx: int, x_host_bf16, W_q4nx, y_host, M: int, K: int, N: int, stream=None) -> None:

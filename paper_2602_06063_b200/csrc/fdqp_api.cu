@@ -24,6 +24,8 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_by
                            int* status, int M, int K, int N, int pair, int Z, cudaStream_t stream);
 cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* gamma, float eps, uint16_t* out, int M, int K,
                            cudaStream_t stream);
+cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* V, float* out, float* ws, int max_splits, int H,
+                          int G, int d, int L, int pitch, int window, float scale, int sm_count, cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
 }  // namespace fdqp
 
@@ -37,6 +39,7 @@ struct fdqp_ctx {
     float* ws_edge = nullptr;
     float* ws_full = nullptr;
     float* pf_ws = nullptr;      // partial results of K-split tensor-core calls
+    float* kv_ws = nullptr;      // decode attention: per (query head, split) partial results
     uint16_t* x_norm = nullptr;  // normalised activations of calls whose RMS normalisation cannot be fused (max_M x max_K)
     uint8_t* x_spread = nullptr; // small x copied with its rows further apart (see kSpreadBelowBytes)
     size_t pf_ws_bytes = 0;
@@ -62,6 +65,7 @@ constexpr int kMaxStages = 40;
 constexpr int64_t kSpreadBelowBytes = 128 << 10;
 constexpr int64_t kSpreadToBytes = 256 << 10;
 constexpr size_t kSpreadBufBytes = (size_t)kSpreadToBytes + 256 * 128;  // row distance rounds up to 128 bytes, M <= 256 here
+constexpr int kKvMaxHeads = 64, kKvMaxSplits = 148, kKvMaxDim = 256;  // decode attention workspace
 constexpr size_t kPrefillWsCap = 128u << 20;  // bytes of partial results a context keeps for K-split tensor-core calls
 constexpr int kMinStages = 3;  // ring depth below which another K slice is preferred
 
@@ -289,6 +293,7 @@ extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, in
         if ((e = cudaMalloc(&ctx->ws_edge, slot * 2 * (size_t)ctx->sm_count * kMaxCtasPerSm))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->ws_full, slot * (size_t)kMaxSplit * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->tickets, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMalloc(&ctx->kv_ws, (size_t)kKvMaxHeads * kKvMaxSplits * (kKvMaxDim + 2) * 4))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->x_norm, (size_t)max_M * (size_t)max_K * 2))) { st = cuda_fail(nullptr, e, ""); break; }
         if (max_M > kMaxTokens) {
             // K-split tensor-core calls (shapes with few output tiles): up to kMaxSplit partial results, capped
@@ -326,6 +331,7 @@ extern "C" fdqp_status fdqp_destroy(fdqp_ctx* ctx) {
     if (ctx->pf_ws) cudaFree(ctx->pf_ws);
     if (ctx->x_spread) cudaFree(ctx->x_spread);
     if (ctx->x_norm) cudaFree(ctx->x_norm);
+    if (ctx->kv_ws) cudaFree(ctx->kv_ws);
     if (ctx->tickets) cudaFree(ctx->tickets);
     if (ctx->xq) cudaFree(ctx->xq);
     if (ctx->xsc) cudaFree(ctx->xsc);
@@ -454,6 +460,24 @@ extern "C" fdqp_status fdqp_run_rmsnorm_epilogue(fdqp_ctx* ctx, const void* x_bf
                                                  void* cuda_stream) {
     if (!gamma_bf16) return FDQP_ERR_ARG;
     return run_impl(ctx, x_bf16, gamma_bf16, eps, W_q4nx, out, epilogue, M, K, N, cuda_stream);
+}
+
+extern "C" fdqp_status fdqp_flowkv_decode(fdqp_ctx* ctx, const void* q_bf16, const void* K_bf16, const void* V_bf16, float* out,
+                                          int64_t H, int64_t G, int64_t d, int64_t L, int64_t pitch, int64_t window,
+                                          float scale, void* cuda_stream) {
+    if (!ctx || !q_bf16 || !K_bf16 || !V_bf16 || !out) return FDQP_ERR_ARG;
+    if (H < 1 || G < 1 || (H % G) != 0 || H / G > 8 || (d != 128 && d != 256) || L < 1 || pitch < L) return FDQP_ERR_SHAPE;
+    if (H > kKvMaxHeads || pitch > (int64_t)1 << 30) return FDQP_ERR_SIZE;
+    if (!aligned16(q_bf16) || !aligned16(K_bf16) || !aligned16(V_bf16) || !aligned16(out)) return FDQP_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FDQP_ERR_CUDA;
+    const cudaError_t e = flowkv_launch(static_cast<const uint16_t*>(q_bf16), static_cast<const uint16_t*>(K_bf16),
+                                        static_cast<const uint16_t*>(V_bf16), out, ctx->kv_ws, kKvMaxSplits, (int)H, (int)G, (int)d,
+                                        (int)L, (int)pitch, (int)window, scale, ctx->sm_count,
+                                        static_cast<cudaStream_t>(cuda_stream));
+    if (e) return cuda_fail(ctx, e, "decode attention launch");
+    ctx->launches += 2;
+    return FDQP_OK;
 }
 
 extern "C" fdqp_status fdqp_run_host_async(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,
