@@ -237,6 +237,61 @@ def run_shape(args):
     fd.fdqp_destroy(ctx)
 
 
+# ----------------------------------------------------------------------------------------------- decode attention
+
+def run_flowkv(args):
+    """Times the decode attention (--flowkv H,G,d,L,window): one new token against a cache of L positions.  Enough
+    distinct caches are rotated to keep every launch's keys and values out of L2.  Algorithmic bytes per call: the
+    attended positions of K and V, 2 * G * n * d * 2 (q and out are negligible)."""
+    import torch
+
+    import paper_2602_06063_b200 as fd
+
+    H, G, d, L, window = (int(v) for v in args.flowkv.split(","))
+    torch.cuda.set_device(0)
+    peaks, peak_kind = measured_peaks()
+    ctx = fd.fdqp_create(0, 8, 256, 256)
+    n = window if 0 < window < L else L
+    cache_bytes = 2 * G * L * d * 2
+    ncopies = max(1, int(np.ceil(4 * L2_BYTES / cache_bytes)))
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    caches = [(torch.randn((G, L, d), device="cuda", generator=gen).to(torch.bfloat16),
+               torch.randn((G, L, d), device="cuda", generator=gen).to(torch.bfloat16)) for _ in range(ncopies)]
+    q = torch.randn((H, d), device="cuda", generator=gen).to(torch.bfloat16)
+    out = torch.empty((H, d), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    sraw = stream.cuda_stream
+    scale = d ** -0.5
+
+    def launch(i):
+        Kc, Vc = caches[i % ncopies]
+        fd.fdqp_flowkv_decode(ctx, q, Kc, Vc, out, H, G, d, L, L, window, scale, sraw)
+
+    for i in range(3):
+        launch(i)
+    stream.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        for i in range(args.steps):
+            launch(i)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        g.replay()
+        e0.record(stream)
+        g.replay()
+        e1.record(stream)
+    stream.synchronize()
+    assert fd.fdqp_last_status(ctx) == 0
+    us = e0.elapsed_time(e1) * 1e3 / args.steps
+    alg = 2.0 * G * n * d * 2
+    gbs = alg / us / 1e3
+    print(json.dumps({"flowkv": {"H": H, "G": G, "d": d, "L": L, "window": window}, "us_per_call": us, "GBps": gbs,
+                      "attended_bytes": alg, "frac_of_measured_peak": gbs / peaks["hbm_gbs"],
+                      "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS, "peak_kind": peak_kind, "cache_copies": ncopies,
+                      "steps": args.steps}), flush=True)
+    fd.fdqp_destroy(ctx)
+
+
 # ----------------------------------------------------------------------------------------------- our arm
 
 def run_ours(args, rank, local_rank, world):
@@ -549,6 +604,7 @@ def main():
     ap.add_argument("--param", action="append", help="library launch parameter key=value (repeatable)")
     ap.add_argument("--shape", help="K,N,M: time this one projection shape instead of the layer workload")
     ap.add_argument("--same-weights", action="store_true", help="with --shape: reuse one weight buffer (for ncu captures)")
+    ap.add_argument("--flowkv", help="H,G,d,L,window: time the decode attention over a KV cache instead of a projection")
     ap.add_argument("--rmsnorm", action="store_true", help="with --shape: RMS-normalise x first (fused where possible)")
     ap.add_argument("--epilogue", default="none", choices=["none", "bf16", "geglu"],
                     help="with --shape: fused store-side epilogue (geglu: gate and up rows interleaved 16 by 16 along N)")
@@ -565,6 +621,11 @@ def main():
         return
     if args.warmup < 3:
         args.warmup = 3
+    if args.flowkv:
+        if args.steps == 8000:
+            args.steps = 50
+        run_flowkv(args)
+        return
     if args.shape:
         if args.steps == 8000:
             args.steps = 50

@@ -23,6 +23,7 @@ constexpr int kKvWarps = 4;
 constexpr int kKvTile = 16;     // positions per warp tile
 constexpr int kKvStages = 3;
 constexpr int kKvMaxGroup = 8;  // query heads per KV head
+constexpr int kKvMaxSplitsDev = 160;  // upper bound of the split count the merge kernel handles (a multiple of 32)
 
 struct FlowKvParams {
     const uint16_t* q;  // [H][d]
@@ -60,6 +61,10 @@ __global__ void __launch_bounds__(kKvWarps * 32, 1) flowkv_decode_kernel(const F
     constexpr int kStageBytes = 2 * kTileBytes;              // K tile then V tile
     constexpr int kCopies = kKvTile * kChunksPerRow / 32;    // 16-byte copies per lane per tile and matrix
     extern __shared__ __align__(128) uint8_t smem[];
+    // Launched with programmatic stream serialisation: the next launch may be set up while this grid runs; this grid
+    // touches nothing (q, the cache and the workspace may all come from earlier launches) before those have completed.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g4 = lane >> 2, q4 = lane & 3;
     const int split = blockIdx.x, kvh = blockIdx.y;
@@ -239,18 +244,42 @@ __global__ void __launch_bounds__(kKvWarps * 32, 1) flowkv_decode_kernel(const F
 // out[h][i] = sum_s O_s[i] 2^(m_s - m*) / sum_s l_s 2^(m_s - m*), splits in order; one block per query head.
 template <int D>
 __global__ void __launch_bounds__(D) flowkv_merge_kernel(const float* __restrict__ ws, float* __restrict__ out, int splits) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int h = blockIdx.x, i = threadIdx.x;
     const float* base = ws + (size_t)h * splits * (D + 2);
-    float m = -INFINITY;
-    for (int s = 0; s < splits; ++s) m = fmaxf(m, base[(size_t)s * (D + 2) + D]);
-    float acc = 0.f, l = 0.f;
-    for (int s = 0; s < splits; ++s) {
-        const float* ps = base + (size_t)s * (D + 2);
-        const float f = ps[D] == -INFINITY ? 0.f : exp2f(ps[D] - m);
-        acc += ps[i] * f;
-        l += ps[D + 1] * f;
+    __shared__ float factor[kKvMaxSplitsDev];  // 2^(m_s - m*) per split
+    __shared__ float l_total;
+    if (i < 32) {  // warp 0: the splits' statistics, a few per lane, all loads independent
+        constexpr int kPer = kKvMaxSplitsDev / 32;
+        float ms[kPer], ls[kPer];
+        float m = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < kPer; ++k) {
+            const int s = i + 32 * k;
+            ms[k] = s < splits ? base[(size_t)s * (D + 2) + D] : -INFINITY;
+            ls[k] = s < splits ? base[(size_t)s * (D + 2) + D + 1] : 0.f;
+            m = fmaxf(m, ms[k]);
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        float l = 0.f;
+#pragma unroll
+        for (int k = 0; k < kPer; ++k) {
+            const int s = i + 32 * k;
+            const float f = ms[k] == -INFINITY ? 0.f : exp2f(ms[k] - m);
+            if (s < splits) factor[s] = f;
+            l += ls[k] * f;
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+        if (i == 0) l_total = l;
     }
-    out[(size_t)h * D + i] = acc / l;
+    __syncthreads();
+    float acc = 0.f;
+#pragma unroll 8
+    for (int s = 0; s < splits; ++s) acc += base[(size_t)s * (D + 2) + i] * factor[s];
+    out[(size_t)h * D + i] = acc / l_total;
 }
 
 // ---- host side ------------------------------------------------------------------------------------------------------
@@ -266,13 +295,26 @@ static cudaError_t flowkv_launch_d(const FlowKvParams& p, float* out, cudaStream
         if ((e = cudaFuncSetAttribute(flowkv_decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem))) return e;
         attr_set = true;
     }
-    flowkv_decode_kernel<D><<<dim3((unsigned)p.splits, (unsigned)p.G), kKvWarps * 32, kSmem, stream>>>(p);
-    if ((e = cudaGetLastError())) return e;
-    flowkv_merge_kernel<D><<<(unsigned)p.H, D, 0, stream>>>(p.ws, out, p.splits);
-    return cudaGetLastError();
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.splits, (unsigned)p.G);
+    cfg.blockDim = dim3(kKvWarps * 32);
+    cfg.dynamicSmemBytes = kSmem;
+    cfg.stream = stream;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if ((e = cudaLaunchKernelEx(&cfg, flowkv_decode_kernel<D>, p))) return e;
+    cfg.gridDim = dim3((unsigned)p.H);
+    cfg.blockDim = dim3(D);
+    cfg.dynamicSmemBytes = 0;
+    const float* ws = p.ws;
+    const int splits = p.splits;
+    return cudaLaunchKernelEx(&cfg, flowkv_merge_kernel<D>, ws, out, splits);
 }
 
-// Returns the number of splits used (>= 1) through *splits_out; ws must hold H * max_splits * (d + 2) floats.
+// ws must hold H * max_splits * (d + 2) floats; max_splits <= kKvMaxSplitsDev.
 cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* V, float* out, float* ws, int max_splits, int H,
                           int G, int d, int L, int pitch, int window, float scale, int sm_count, cudaStream_t stream) {
     FlowKvParams p;
@@ -293,6 +335,7 @@ cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* 
     int chunk = ((n + want - 1) / want + gran - 1) / gran * gran;
     p.chunk = chunk;
     p.splits = (n + chunk - 1) / chunk;
+    if (p.splits > kKvMaxSplitsDev) return cudaErrorInvalidValue;
     p.scale_log2e = scale * 1.4426950408889634f;
     if (d == 256) return flowkv_launch_d<256>(p, out, stream);
     if (d == 128) return flowkv_launch_d<128>(p, out, stream);
