@@ -293,7 +293,7 @@ extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, in
         if ((e = cudaMalloc(&ctx->ws_edge, slot * 2 * (size_t)ctx->sm_count * kMaxCtasPerSm))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->ws_full, slot * (size_t)kMaxSplit * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->tickets, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
-        if ((e = cudaMalloc(&ctx->kv_ws, (size_t)kKvMaxHeads * kKvMaxSplits * (kKvMaxDim + 2) * 4))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMalloc(&ctx->kv_ws, (size_t)kKvMaxHeads * kKvMaxSplits * (kKvMaxDim + 4) * 4))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->x_norm, (size_t)max_M * (size_t)max_K * 2))) { st = cuda_fail(nullptr, e, ""); break; }
         if (max_M > kMaxTokens) {
             // K-split tensor-core calls (shapes with few output tiles): up to kMaxSplit partial results, capped

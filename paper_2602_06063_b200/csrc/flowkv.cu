@@ -23,13 +23,14 @@ constexpr int kKvWarps = 4;
 constexpr int kKvTile = 16;     // positions per warp tile
 constexpr int kKvStages = 3;
 constexpr int kKvMaxGroup = 8;  // query heads per KV head
+constexpr int kKvMergeThreads = 1024;
 constexpr int kKvMaxSplitsDev = 160;  // upper bound of the split count the merge kernel handles (a multiple of 32)
 
 struct FlowKvParams {
     const uint16_t* q;  // [H][d]
     const uint16_t* K;  // [G][pitch][d]
     const uint16_t* V;
-    float* ws;          // [H][splits][d + 2]: partial O (unnormalised), running maximum, running sum
+    float* ws;          // [H][splits][d + 4]: partial O (unnormalised), running maximum, running sum, 2 unused
     int H, G, L, pitch;
     int j0;             // first position attended to (0, or L - window)
     int chunk;          // positions per split (a multiple of kKvWarps * kKvTile)
@@ -232,7 +233,7 @@ __global__ void __launch_bounds__(kKvWarps * 32, 1) flowkv_decode_kernel(const F
             acc += part[(size_t)(w * kKvMaxGroup + h) * D + i] * f;
             l += stats[(w * kKvMaxGroup + h) * 2 + 1] * f;
         }
-        float* dst = p.ws + ((size_t)(kvh * R + h) * p.splits + split) * (D + 2);
+        float* dst = p.ws + ((size_t)(kvh * R + h) * p.splits + split) * (D + 4);
         dst[i] = acc;
         if (i == 0) {
             dst[D] = m;
@@ -241,15 +242,17 @@ __global__ void __launch_bounds__(kKvWarps * 32, 1) flowkv_decode_kernel(const F
     }
 }
 
-// out[h][i] = sum_s O_s[i] 2^(m_s - m*) / sum_s l_s 2^(m_s - m*), splits in order; one block per query head.
+// out[h][i] = sum_s O_s[i] 2^(m_s - m*) / sum_s l_s 2^(m_s - m*) in a fixed order; one block per query head.
 template <int D>
-__global__ void __launch_bounds__(D) flowkv_merge_kernel(const float* __restrict__ ws, float* __restrict__ out, int splits) {
+__global__ void __launch_bounds__(kKvMergeThreads) flowkv_merge_kernel(const float* __restrict__ ws, float* __restrict__ out, int splits) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int h = blockIdx.x, i = threadIdx.x;
-    const float* base = ws + (size_t)h * splits * (D + 2);
+    const float* base = ws + (size_t)h * splits * (D + 4);
     __shared__ float factor[kKvMaxSplitsDev];  // 2^(m_s - m*) per split
     __shared__ float l_total;
+    constexpr int kCols = D / 4, kParts = kKvMergeThreads / kCols;
+    __shared__ float4 partial[kParts][kCols];
     if (i < 32) {  // warp 0: the splits' statistics, a few per lane, all loads independent
         constexpr int kPer = kKvMaxSplitsDev / 32;
         float ms[kPer], ls[kPer];
@@ -257,8 +260,8 @@ __global__ void __launch_bounds__(D) flowkv_merge_kernel(const float* __restrict
 #pragma unroll
         for (int k = 0; k < kPer; ++k) {
             const int s = i + 32 * k;
-            ms[k] = s < splits ? base[(size_t)s * (D + 2) + D] : -INFINITY;
-            ls[k] = s < splits ? base[(size_t)s * (D + 2) + D + 1] : 0.f;
+            ms[k] = s < splits ? base[(size_t)s * (D + 4) + D] : -INFINITY;
+            ls[k] = s < splits ? base[(size_t)s * (D + 4) + D + 1] : 0.f;
             m = fmaxf(m, ms[k]);
         }
 #pragma unroll
@@ -276,10 +279,34 @@ __global__ void __launch_bounds__(D) flowkv_merge_kernel(const float* __restrict
         if (i == 0) l_total = l;
     }
     __syncthreads();
-    float acc = 0.f;
-#pragma unroll 8
-    for (int s = 0; s < splits; ++s) acc += base[(size_t)s * (D + 2) + i] * factor[s];
-    out[(size_t)h * D + i] = acc / l_total;
+    // the sum over splits: four columns per thread, the splits dealt round-robin to kParts thread groups (all of a
+    // thread's loads are independent), then the groups' sums added in group order
+    const int c = i % kCols, part = i / kCols;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int s = part; s < splits; s += kParts) {
+        const float4 v = *reinterpret_cast<const float4*>(base + (size_t)s * (D + 4) + 4 * c);
+        const float f = factor[s];
+        acc.x += v.x * f;
+        acc.y += v.y * f;
+        acc.z += v.z * f;
+        acc.w += v.w * f;
+    }
+    partial[part][c] = acc;
+    __syncthreads();
+    if (i < kCols) {
+        float4 t = partial[0][i];
+#pragma unroll
+        for (int q = 1; q < kParts; ++q) {
+            const float4 v = partial[q][i];
+            t.x += v.x;
+            t.y += v.y;
+            t.z += v.z;
+            t.w += v.w;
+        }
+        const float l = l_total;
+        *reinterpret_cast<float4*>(out + (size_t)h * D + 4 * i) = make_float4(t.x / l, t.y / l, t.z / l, t.w / l);
+    }
 }
 
 // ---- host side ------------------------------------------------------------------------------------------------------
@@ -307,14 +334,14 @@ static cudaError_t flowkv_launch_d(const FlowKvParams& p, float* out, cudaStream
     cfg.numAttrs = 1;
     if ((e = cudaLaunchKernelEx(&cfg, flowkv_decode_kernel<D>, p))) return e;
     cfg.gridDim = dim3((unsigned)p.H);
-    cfg.blockDim = dim3(D);
+    cfg.blockDim = dim3(kKvMergeThreads);
     cfg.dynamicSmemBytes = 0;
     const float* ws = p.ws;
     const int splits = p.splits;
     return cudaLaunchKernelEx(&cfg, flowkv_merge_kernel<D>, ws, out, splits);
 }
 
-// ws must hold H * max_splits * (d + 2) floats; max_splits <= kKvMaxSplitsDev.
+// ws must hold H * max_splits * (d + 4) floats; max_splits <= kKvMaxSplitsDev.
 cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* V, float* out, float* ws, int max_splits, int H,
                           int G, int d, int L, int pitch, int window, float scale, int sm_count, cudaStream_t stream) {
     FlowKvParams p;
@@ -329,7 +356,10 @@ cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* 
     p.j0 = (window > 0 && window < L) ? L - window : 0;
     const int n = L - p.j0;
     const int gran = kKvWarps * kKvTile;
-    int want = (sm_count + G - 1) / G;  // CTAs over all KV heads ~ one per SM
+    // CTAs over all KV heads: as many as are resident at once (one per SM at d = 256, whose rings take 192 KB; two at
+    // d = 128), never more -- a CTA that has to wait for a free SM would double the time.
+    const int resident = sm_count * (d == 128 ? 2 : 1);
+    int want = resident / G;
     if (want > max_splits) want = max_splits;
     if (want < 1) want = 1;
     int chunk = ((n + want - 1) / want + gran - 1) / gran * gran;
