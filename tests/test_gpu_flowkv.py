@@ -62,6 +62,31 @@ def test_decode_attention_matches_oracle(ctx, H, G, d, L, window, pitch):
     assert not bad.any(), f"{bad.sum()} of {bad.size} outside the bound; worst {(err / (absw + 1e-30)).max():.2e}"
 
 
+# Full-size caches in the launch configurations the benchmark times (one CTA per SM, every split several hundred tiles
+# long): the oracle still evaluates every output (a few GFLOP in fp64).  Inputs from a seeded numpy generator, which is
+# fast enough for 10^8 values; keys get a slowly varying component so that the softmax is not flat over the cache.
+FULL = [(8, 4, 256, 131072, 0), (8, 4, 256, 131072, 1024), (16, 8, 256, 32768 + 17, 0), (32, 16, 128, 65536, 0),
+        (4, 1, 256, 32768, 0)]
+
+
+@pytest.mark.parametrize("H,G,d,L,window", FULL)
+def test_full_size_caches(ctx, H, G, d, L, window):
+    rng = np.random.default_rng(900 + H + L + window)
+    q = synthgen.bf16_bits(rng.standard_normal((H, d), dtype=np.float32))
+    Kf = rng.standard_normal((G, L, d), dtype=np.float32)
+    Kf[:, :, 0] += 6.0 * np.sin(np.arange(L, dtype=np.float32) * 1e-3)[None, :]
+    K = synthgen.bf16_bits(Kf)
+    del Kf
+    V = synthgen.bf16_bits(rng.standard_normal((G, L, d), dtype=np.float32))
+    scale = d ** -0.5
+    out = run(ctx, q, K, V, L, window, scale)
+    ref, absw = oracle.decode_attention(q, K, V, L, window, scale)
+    assert np.all(np.isfinite(out))
+    err = np.abs(out.astype(np.float64) - ref)
+    bad = err > REL * absw + ABS
+    assert not bad.any(), f"{bad.sum()} of {bad.size} outside the bound; worst {(err / (absw + 1e-30)).max():.2e}"
+
+
 def test_peaked_scores_and_large_magnitudes(ctx):
     # a large scale makes the distribution collapse onto few positions (running-maximum updates matter)
     H, G, d, L = 8, 4, 256, 1500

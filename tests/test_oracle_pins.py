@@ -478,6 +478,14 @@ def test_decode_attention_closed_forms_and_invariances():
         p = np.exp(s - s.max())
         p /= p.sum()
         assert np.allclose(allp[h], p @ Vb[h // 2, :L], rtol=1e-13, atol=1e-14)
+    # one position -> its value, whatever the score; any permutation of the attended positions changes nothing
+    one, _ = oracle.decode_attention(bf(q), bf(K), bf(V), L=1, scale=0.5)
+    assert np.array_equal(one[1], Vb[0, 0]) and np.array_equal(one[2], Vb[1, 0])
+    perm = rng.permutation(L)
+    Kp, Vp = K.copy(), V.copy()
+    Kp[:, :L], Vp[:, :L] = K[:, perm], V[:, perm]
+    outp, _ = oracle.decode_attention(bf(q), bf(Kp), bf(Vp), L=L, scale=0.5)
+    assert np.allclose(outp, allp, rtol=1e-13, atol=1e-14)
     big = np.zeros((H, d), np.float32)
     big[:, 1] = 64.0
     Kd = np.zeros((G, pitch, d), np.float32)
