@@ -58,6 +58,14 @@ def _load():
         lib.oracle_rmsnorm.argtypes = [p, p, ctypes.c_double, i64, i64, p]
         lib.oracle_decode_attention.restype = ci
         lib.oracle_decode_attention.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, ctypes.c_double, p, p]
+        lib.oracle_fmt_packed_bytes.restype = ctypes.c_size_t
+        lib.oracle_fmt_packed_bytes.argtypes = [ci, i64, i64]
+        lib.oracle_fmt_unpack.restype = ci
+        lib.oracle_fmt_unpack.argtypes = [ci, p, i64, i64, p, p, p]
+        lib.oracle_fmt_dequant.restype = ci
+        lib.oracle_fmt_dequant.argtypes = [ci, p, p, p, i64, i64, i64, i64, p, p]
+        lib.oracle_fmt_project.restype = ci
+        lib.oracle_fmt_project.argtypes = [ci, p, p, p, p, i64, i64, i64, i64, i64, ci, p, p]
         lib.oracle_max_threads.restype = ci
         _lib = lib
     return _lib
@@ -200,3 +208,68 @@ def decode_attention(q, K, V, L: int, window: int = 0, scale: float = 1.0):
     if rc != 0:
         raise ValueError(f"oracle_decode_attention failed ({rc})")
     return out, absw
+
+
+# ---- format variants of the block container (group sizes 64 / 128, MXFP4) ----------------------------------------
+
+FMT_G64, FMT_G128, FMT_MXFP4 = 1, 2, 3
+FMT_GROUP = {FMT_G64: 64, FMT_G128: 128, FMT_MXFP4: 32}
+
+
+def fmt_packed_bytes(fmt: int, K: int, N: int) -> int:
+    """Size of a packed K x N matrix in a variant format: 4608 (group 64) or 4352 (group 128, MXFP4) bytes per block."""
+    return int(_load().oracle_fmt_packed_bytes(fmt, K, N))
+
+
+def fmt_unpack(fmt: int, packed, K: int, N: int):
+    """Packed bytes -> (codes[N,K] u8, scales[N,K/g] u16, offsets[N,K/g] u16 or None).  MXFP4 scales are the E8M0
+    bytes widened to u16."""
+    packed = _c(packed, np.uint8)
+    if packed.size != fmt_packed_bytes(fmt, K, N) or packed.size == 0:
+        raise ValueError("packed size does not match fmt, K, N")
+    g = FMT_GROUP[fmt]
+    codes = np.empty((N, K), np.uint8)
+    scales = np.empty((N, K // g), np.uint16)
+    offsets = None if fmt == FMT_MXFP4 else np.empty((N, K // g), np.uint16)
+    rc = _load().oracle_fmt_unpack(fmt, _ptr(packed), K, N, _ptr(codes), _ptr(scales),
+                                   None if offsets is None else _ptr(offsets))
+    if rc != 0:
+        raise ValueError(f"oracle_fmt_unpack failed ({rc})")
+    return codes, scales, offsets
+
+
+def fmt_dequant(fmt: int, codes, scales, offsets=None, n0: int = 0, n1: int | None = None):
+    """Eq. 3 with the format's group size, or the MXFP4 element times its power-of-two scale: (w32, w16 bits)."""
+    codes = _c(codes, np.uint8)
+    scales = _c(scales, np.uint16)
+    offsets = None if offsets is None else _c(offsets, np.uint16)
+    N, K = codes.shape
+    n1 = N if n1 is None else n1
+    w32 = np.empty((K, n1 - n0), np.float32)
+    w16 = np.empty((K, n1 - n0), np.uint16)
+    rc = _load().oracle_fmt_dequant(fmt, _ptr(codes), _ptr(scales), None if offsets is None else _ptr(offsets), K, N,
+                                    n0, n1, _ptr(w32), _ptr(w16))
+    if rc != 0:
+        raise ValueError(f"oracle_fmt_dequant failed ({rc})")
+    return w32, w16
+
+
+def fmt_project(fmt: int, x_bf16, codes, scales, offsets=None, n0: int = 0, n1: int | None = None, nthreads: int = 1):
+    """y = x . w32 of the variant format in fp64, k ascending: (y[M, n1-n0], abs_sum[M, n1-n0])."""
+    x_bf16 = _c(x_bf16, np.uint16)
+    codes = _c(codes, np.uint8)
+    scales = _c(scales, np.uint16)
+    offsets = None if offsets is None else _c(offsets, np.uint16)
+    N, K = codes.shape
+    M = x_bf16.shape[0]
+    if x_bf16.shape != (M, K):
+        raise ValueError("x must be [M, K]")
+    n1 = N if n1 is None else n1
+    y = np.empty((M, n1 - n0), np.float64)
+    a = np.empty((M, n1 - n0), np.float64)
+    rc = _load().oracle_fmt_project(fmt, _ptr(x_bf16), _ptr(codes), _ptr(scales),
+                                    None if offsets is None else _ptr(offsets), M, K, N, n0, n1, nthreads, _ptr(y),
+                                    _ptr(a))
+    if rc != 0:
+        raise ValueError(f"oracle_fmt_project failed ({rc})")
+    return y, a

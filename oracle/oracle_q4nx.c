@@ -43,6 +43,12 @@
  * Decode attention over a KV cache (the paper's second decode kernel, FlowKV, computes it chunk by chunk):
  * oracle_decode_attention is the plain softmax-weighted sum; pinned by closed forms and invariances.
  *
+ * Format variants of the block container (next step; the paper calls its dequantisation logic format-agnostic and names
+ * other group sizes and MXFP4 as the formats the container is meant to take): oracle_fmt_* below -- group sizes 64 and
+ * 128 with Eq. 3 unchanged, and MXFP4 (4-bit E2M1 elements, one 8-bit power-of-two scale per 32 elements, as the OCP
+ * Microscaling specification defines them).  Pinned by the bit-field definitions of E2M1 / E8M0, exact rational
+ * evaluation, equivalence with the group-32 routines on duplicated scales, hand-located bytes and a numpy matmul.
+ *
  * Pins (tests/test_oracle_pins.py): the paper's 5120-byte block, hand-written
  * byte dumps, closed-form worked examples, exact rational evaluation of eq. 3
  * over all codes, an independent fp64 matmul, and invariants.  Parity with
@@ -326,6 +332,122 @@ int oracle_decode_attention(const uint16_t *q, const uint16_t *K, const uint16_t
     }
     free(s);
     return 0;
+}
+
+/* ---- format variants of the 32 x 256 block container (next step) ------------------------------------------------ */
+
+/* fmt 1, 2: Eq. 3 with group size 64 / 128 along K (bf16 scale and offset per group).  fmt 3: MXFP4 -- the 4-bit
+ * code is an E2M1 floating-point element (sign, 2 exponent bits, 1 mantissa bit: 0, 0.5, 1, 1.5, 2, 3, 4, 6 and their
+ * negatives), a group of 32 shares one E8M0 scale 2^(e - 127), e = 0..254 (255 is the format's NaN and is rejected);
+ * there is no offset.  K must be a multiple of 256 (whole blocks), N of 32.
+ * Block bytes: [codes 4096, addressed exactly as in the group-32 container][scales][offsets]:
+ *   fmt 1: 4 groups per row and block -> scale u16 at 4096 + 2*(t*32 + r), t = (k % 256) / 64; offsets 256 bytes on;
+ *          block = 4608 bytes (4.5 bits per weight)
+ *   fmt 2: 2 groups -> t = (k % 256) / 128; offsets 128 bytes on; block = 4352 bytes (4.25 bits per weight)
+ *   fmt 3: 8 groups -> scale u8 at 4096 + t*32 + r, t = (k % 256) / 32; block = 4352 bytes (4.25 bits per weight)
+ * Unpacked form: codes[N][K]; scales[N][K/g] as uint16 (bf16 bits; for fmt 3 the E8M0 byte, 0..254); offsets likewise
+ * (ignored for fmt 3). */
+static int fmt_group(int fmt) { return fmt == 1 ? 64 : fmt == 2 ? 128 : fmt == 3 ? 32 : 0; }
+static size_t fmt_block_bytes(int fmt) { return fmt == 1 ? 4608u : (fmt == 2 || fmt == 3) ? 4352u : 0u; }
+
+size_t oracle_fmt_packed_bytes(int fmt, int64_t K, int64_t N) {
+    if (fmt_group(fmt) == 0 || K <= 0 || N <= 0 || (K % 256) != 0 || (N % 32) != 0) return 0;
+    return (size_t)(N / 32) * (size_t)(K / 256) * fmt_block_bytes(fmt);
+}
+
+int oracle_fmt_unpack(int fmt, const uint8_t *packed, int64_t K, int64_t N, uint8_t *codes, uint16_t *scales,
+                      uint16_t *offsets) {
+    if (oracle_fmt_packed_bytes(fmt, K, N) == 0 || !packed || !codes || !scales) return -1;
+    if (fmt != 3 && !offsets) return -1;
+    const int64_t g = fmt_group(fmt), G = K / g, per_block = 256 / g;
+    const size_t bb = fmt_block_bytes(fmt);
+    for (int64_t n = 0; n < N; ++n) {
+        const int64_t s = n / 32, r = n % 32;
+        for (int64_t k = 0; k < K; ++k) {
+            const int64_t b = k / 256, c = k % 256;
+            const uint8_t *blk = packed + ((size_t)s * (size_t)(K / 256) + (size_t)b) * bb;
+            const uint8_t byte = blk[(c / 32) * 512 + r * 16 + (c % 32) / 2];
+            codes[n * K + k] = (c & 1) ? (uint8_t)(byte >> 4) : (uint8_t)(byte & 0x0f);
+            if ((k % g) == 0) {
+                const int64_t t = c / g;
+                if (fmt == 3) {
+                    scales[n * G + k / g] = blk[4096 + t * 32 + r];
+                } else {
+                    scales[n * G + k / g] = read_u16le(blk + 4096 + 2 * (t * 32 + r));
+                    offsets[n * G + k / g] = read_u16le(blk + 4096 + 64 * per_block + 2 * (t * 32 + r));
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+/* E2M1 element of code q (bit 3 sign, bits 2..1 exponent E, bit 0 mantissa M): E = 0 is subnormal, M / 2; otherwise
+ * 2^(E-1) (1 + M/2). */
+static double e2m1_value(unsigned q) {
+    static const double mag[8] = {0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0};
+    return (q & 8u) ? -mag[q & 7u] : mag[q & 7u];
+}
+
+/* One dequantised weight, rounded once to fp32.  fmt 3: element times 2^(e-127), exact in double. */
+static int fmt_dequant_one(int fmt, uint16_t d_bits, uint16_t m_bits, unsigned q, float *w) {
+    if (q > 15u) return -2;
+    if (fmt == 3) {
+        if (d_bits > 254u) return -3;
+        *w = (float)ldexp(e2m1_value(q), (int)d_bits - 127);
+        return 0;
+    }
+    *w = dequant_one(d_bits, m_bits, q);
+    return 0;
+}
+
+/* w32 / w16: [K][n1-n0], as oracle_dequant. */
+int oracle_fmt_dequant(int fmt, const uint8_t *codes, const uint16_t *scales, const uint16_t *offsets, int64_t K,
+                       int64_t N, int64_t n0, int64_t n1, float *w32, uint16_t *w16) {
+    if (oracle_fmt_packed_bytes(fmt, K, N) == 0 || !codes || !scales || (fmt != 3 && !offsets)) return -1;
+    if (n0 < 0 || n1 > N || n0 > n1) return -1;
+    const int64_t g = fmt_group(fmt), G = K / g, W = n1 - n0;
+    for (int64_t n = n0; n < n1; ++n) {
+        for (int64_t k = 0; k < K; ++k) {
+            float w;
+            int rc = fmt_dequant_one(fmt, scales[n * G + k / g], fmt == 3 ? 0 : offsets[n * G + k / g], codes[n * K + k], &w);
+            if (rc) return rc;
+            if (w32) w32[k * W + (n - n0)] = w;
+            if (w16) w16[k * W + (n - n0)] = fp32_to_bf16_rne(w);
+        }
+    }
+    return 0;
+}
+
+/* y[m][n - n0] = sum_k x[m][k] * w32[k][n], fp64, k ascending; abs_sum as oracle_project. */
+int oracle_fmt_project(int fmt, const uint16_t *x_bf16, const uint8_t *codes, const uint16_t *scales,
+                       const uint16_t *offsets, int64_t M, int64_t K, int64_t N, int64_t n0, int64_t n1, int nthreads,
+                       double *y, double *abs_sum) {
+    if (oracle_fmt_packed_bytes(fmt, K, N) == 0 || M < 1 || !x_bf16 || !codes || !scales || (fmt != 3 && !offsets) || !y)
+        return -1;
+    if (n0 < 0 || n1 > N || n0 > n1) return -1;
+    const int64_t g = fmt_group(fmt), G = K / g, W = n1 - n0;
+    int bad = 0;
+    (void)nthreads;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(static) num_threads(nthreads > 0 ? nthreads : 1) reduction(| : bad)
+#endif
+    for (int64_t n = n0; n < n1; ++n) {
+        for (int64_t m = 0; m < M; ++m) {
+            double acc = 0.0, aacc = 0.0;
+            for (int64_t k = 0; k < K; ++k) {
+                float w = 0.f;
+                if (fmt_dequant_one(fmt, scales[n * G + k / g], fmt == 3 ? 0 : offsets[n * G + k / g], codes[n * K + k], &w))
+                    bad = 1;
+                double p = bf16_bits_to_double(x_bf16[m * K + k]) * (double)w;
+                acc += p;
+                aacc += fabs(p);
+            }
+            y[m * W + (n - n0)] = acc;
+            if (abs_sum) abs_sum[m * W + (n - n0)] = aacc;
+        }
+    }
+    return bad ? -2 : 0;
 }
 
 int oracle_max_threads(void) {

@@ -84,6 +84,30 @@ def weights(seed: int, K: int, N: int, sigma_d: float = 0.02, sigma_m: float = 0
     return Q4NXWeights(codes, scales, offsets)
 
 
+FMT_Q4NX, FMT_G64, FMT_G128, FMT_MXFP4 = 0, 1, 2, 3
+FMT_GROUP = {FMT_Q4NX: 32, FMT_G64: 64, FMT_G128: 128, FMT_MXFP4: 32}
+
+
+def weights_fmt(seed: int, K: int, N: int, fmt: int) -> Q4NXWeights:
+    """Content for a format variant of the container.  Group sizes 64 / 128: the Q4NX recipe with one scale and one
+    offset per larger group.  MXFP4: codes uniform 0..15 (E2M1 elements), `scales` holds the E8M0 exponent bytes
+    (uniform 118..122, i.e. scales 2^-9 .. 2^-5: weights of a few hundredths like the Q4NX recipe's) widened to uint16;
+    `offsets` is None."""
+    assert K % 256 == 0 and N % 32 == 0
+    g = FMT_GROUP[fmt]
+    lib = _load()
+    codes = np.empty((N, K), np.uint8)
+    lib.synth_codes(seed, codes.size, ctypes.c_void_p(codes.ctypes.data))
+    if fmt == FMT_MXFP4:
+        e = (118 + u64(seed, 7, N * (K // g)) % np.uint64(5)).astype(np.uint16).reshape(N, K // g)
+        return Q4NXWeights(codes, e, None)
+    scales = np.empty((N, K // g), np.uint16)
+    offsets = np.empty((N, K // g), np.uint16)
+    lib.synth_scales(seed, scales.size, 0.02, ctypes.c_void_p(scales.ctypes.data))
+    lib.synth_offsets(seed, offsets.size, 0.01, ctypes.c_void_p(offsets.ctypes.data))
+    return Q4NXWeights(codes, scales, offsets)
+
+
 def activations(seed: int, M: int, K: int, amp: float = 1.0) -> np.ndarray:
     """x[M, K] as bf16 bits, bf16(amp * N(0, 1))."""
     x = np.empty((M, K), np.uint16)
