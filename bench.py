@@ -180,9 +180,15 @@ def run_shape(args):
         key, val = kv.split("=")
         fd.fdqp_set_param(ctx, key, int(val))
     nb = min(N, 4096)
-    w = synthgen.weights(5, K, nb)
-    tile = fd.q4nx_pack(w.codes, w.scales, w.offsets)
-    packed = np.tile(tile, -(-N // nb))[:fd.q4nx_packed_bytes(K, N)]
+    fmt = {"q4nx": fd.FMT_Q4NX, "g64": fd.FMT_G64, "g128": fd.FMT_G128, "mxfp4": fd.FMT_MXFP4}[args.format]
+    if fmt == fd.FMT_Q4NX:
+        w = synthgen.weights(5, K, nb)
+        tile = fd.q4nx_pack(w.codes, w.scales, w.offsets)
+    else:
+        w = synthgen.weights_fmt(5, K, nb, fmt)
+        tile = fd.q4nx_pack_fmt(fmt, w.codes, w.scales, w.offsets)
+    packed_bytes = fd.q4nx_packed_bytes_fmt(fmt, K, N)
+    packed = np.tile(tile, -(-N // nb))[:packed_bytes]
     base = torch.from_numpy(np.ascontiguousarray(packed)).cuda()
     ncopies = max(1, int(np.ceil(4 * L2_BYTES / base.numel()))) if not args.same_weights else 1
     copies = [base] + [base.clone() for _ in range(ncopies - 1)]
@@ -198,7 +204,9 @@ def run_shape(args):
     gamma = torch.zeros(K, dtype=torch.int16, device="cuda")
 
     def launch(W):
-        if args.rmsnorm:
+        if fmt != fd.FMT_Q4NX:
+            fd.fdqp_run_fmt(ctx, fmt, x, W, y, M, K, N, sraw)
+        elif args.rmsnorm:
             fd.fdqp_run_rmsnorm_epilogue(ctx, x, gamma, 1e-6, W, y, epi, M, K, N, sraw)
         else:
             fd.fdqp_run_epilogue(ctx, x, W, y, epi, M, K, N, sraw)
@@ -228,8 +236,8 @@ def run_shape(args):
     stream.synchronize()
     assert fd.fdqp_last_status(ctx) == 0
     us = e0.elapsed_time(e1) * 1e3 / args.steps
-    gbs = alg_bytes(M, K, N) / us / 1e3
-    print(json.dumps({"shape": {"K": K, "N": N, "M": M}, "us_per_call": us, "GBps": gbs,
+    gbs = (alg_bytes(M, K, N) - 0.625 * K * N + packed_bytes) / us / 1e3  # the format's own bytes per weight
+    print(json.dumps({"shape": {"K": K, "N": N, "M": M}, "format": args.format, "us_per_call": us, "GBps": gbs,
                       "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
                       "peak_kind": peak_kind, "weight_copies": ncopies, "steps": args.steps,
                       "graph": bool(args.graph and not args.same_weights), "epilogue": args.epilogue, "rmsnorm": bool(args.rmsnorm),
@@ -608,6 +616,8 @@ def main():
     ap.add_argument("--rmsnorm", action="store_true", help="with --shape: RMS-normalise x first (fused where possible)")
     ap.add_argument("--epilogue", default="none", choices=["none", "bf16", "geglu"],
                     help="with --shape: fused store-side epilogue (geglu: gate and up rows interleaved 16 by 16 along N)")
+    ap.add_argument("--format", default="q4nx", choices=["q4nx", "g64", "g128", "mxfp4"],
+                    help="with --shape: format variant of the block container (group 64 / 128, MXFP4)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-head", action="store_true", help="skip the LM-head timing")
     args = ap.parse_args()

@@ -96,6 +96,40 @@ FDQP_API fdqp_status q4nx_pack(const uint8_t* codes, const uint16_t* scales_bf16
 FDQP_API fdqp_status q4nx_unpack(const void* packed, int64_t K, int64_t N, uint8_t* codes, uint16_t* scales_bf16,
                         uint16_t* offsets_bf16);
 
+/* ---- format variants of the block container ---------------------------------- */
+
+/* The paper describes its dequantisation logic as format-agnostic and the block
+ * container as able to take other group sizes and MXFP4.  Every variant keeps the
+ * 32 x 256 block and its 4096-byte code section (addressed exactly as in Q4NX);
+ * the metadata that follows differs.  With r = n % 32 and c = k % 256:
+ *   FDQP_FMT_Q4NX  : the container above (group 32, 5120-byte blocks)
+ *   FDQP_FMT_G64   : Eq. 3 with one bf16 scale and offset per 64 inputs:
+ *                    scale u16 at 4096 + 2*((c/64)*32 + r), offsets 256 bytes
+ *                    further on; 4608-byte blocks (4.5 bits per weight)
+ *   FDQP_FMT_G128  : one per 128 inputs: scale at 4096 + 2*((c/128)*32 + r),
+ *                    offsets 128 bytes on; 4352-byte blocks (4.25 bits)
+ *   FDQP_FMT_MXFP4 : the code is an E2M1 element (bit 3 sign, bits 2..1 exponent,
+ *                    bit 0 mantissa: 0, 0.5, 1, 1.5, 2, 3, 4, 6 and negatives), a
+ *                    group of 32 shares the E8M0 scale 2^(e-127), e = 0..254, one
+ *                    byte at 4096 + (c/32)*32 + r; no offsets; 4352-byte blocks.
+ *                    w_hat = element * 2^(e-127), exact in fp32.
+ * The variants need K % 256 == 0 and N % 32 == 0 (whole blocks). */
+typedef enum { FDQP_FMT_Q4NX = 0, FDQP_FMT_G64 = 1, FDQP_FMT_G128 = 2, FDQP_FMT_MXFP4 = 3 } fdqp_format;
+
+/* Bytes of a packed K x N matrix in `format`; 0 for a shape the format cannot hold. */
+FDQP_API size_t q4nx_packed_bytes_fmt(int format, int64_t K, int64_t N);
+
+/* q4nx_pack / q4nx_unpack for any format.  With g the format's group size:
+ *   codes    host, [N][K], one code per byte, 0..15
+ *   scales   host, [N][K/g]: raw bf16 bits (uint16) for the Eq. 3 formats, the E8M0
+ *            byte (uint8, 255 = NaN is refused with FDQP_ERR_ARG) for MXFP4
+ *   offsets_bf16  host, [N][K/g] raw bf16 bits; ignored (may be null) for MXFP4
+ * Errors as q4nx_pack. */
+FDQP_API fdqp_status q4nx_pack_fmt(int format, const uint8_t* codes, const void* scales, const uint16_t* offsets_bf16,
+                          int64_t K, int64_t N, void* out, size_t out_bytes);
+FDQP_API fdqp_status q4nx_unpack_fmt(int format, const void* packed, int64_t K, int64_t N, uint8_t* codes, void* scales,
+                            uint16_t* offsets_bf16);
+
 /* ---- context --------------------------------------------------------------- */
 
 /* Create a context on CUDA device `device` for projections up to max_M x max_K x
@@ -247,6 +281,20 @@ FDQP_API fdqp_status fdqp_run_noalloc(const void* x_bf16, const void* W_q4nx, fl
  * Bit-exact by definition (one rounding to fp32).  Asynchronous on the stream. */
 FDQP_API fdqp_status fdqp_dequant(fdqp_ctx* ctx, const void* W_q4nx, void* out, int out_is_bf16, int64_t K, int64_t N,
                          void* cuda_stream);
+
+/* fdqp_run and fdqp_dequant for a matrix packed in `format` (fdqp_format).  Same
+ * arguments, results, acceptance bound (dequantised values bit-exact; y within
+ * 2e-3 * sum_k |x_k w_hat_k| + 1e-5 of the fp64 product), asynchrony and errors as
+ * fdqp_run / fdqp_dequant; FDQP_FMT_Q4NX is exactly those calls.  The variants run
+ * on the streaming GEMV kernels for every M (rows beyond eight in further launches
+ * of eight); there is no tensor-core path for them.  In the projection an MXFP4
+ * scale byte of 0 (2^-127, below 1e-38) counts as a scale of zero; the
+ * dequantisation engine returns it exactly.  FDQP_ERR_ARG for an unknown
+ * format, FDQP_ERR_SHAPE when K is not a multiple of 256. */
+FDQP_API fdqp_status fdqp_run_fmt(fdqp_ctx* ctx, int format, const void* x_bf16, const void* W_packed, float* y, int64_t M,
+                         int64_t K, int64_t N, void* cuda_stream);
+FDQP_API fdqp_status fdqp_dequant_fmt(fdqp_ctx* ctx, int format, const void* W_packed, void* out, int out_is_bf16, int64_t K,
+                             int64_t N, void* cuda_stream);
 
 /* ---- status, tuning, introspection ---------------------------------------- */
 

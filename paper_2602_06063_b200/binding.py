@@ -25,7 +25,8 @@ EXPORTS = [
     "q4nx_packed_bytes", "q4nx_pack", "q4nx_unpack", "fdqp_create", "fdqp_destroy", "fdqp_run", "fdqp_run_host",
     "fdqp_run_host_async", "fdqp_run_epilogue", "fdqp_run_rmsnorm_epilogue", "fdqp_flowkv_decode",
     "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
-    "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc",
+    "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc", "q4nx_packed_bytes_fmt", "q4nx_pack_fmt",
+    "q4nx_unpack_fmt", "fdqp_run_fmt", "fdqp_dequant_fmt",
 ]
 
 
@@ -56,6 +57,16 @@ def load_library():
     lib.q4nx_pack.argtypes = [vp, vp, vp, i64, i64, vp, sz]
     lib.q4nx_unpack.restype = ci
     lib.q4nx_unpack.argtypes = [vp, i64, i64, vp, vp, vp]
+    lib.q4nx_packed_bytes_fmt.restype = sz
+    lib.q4nx_packed_bytes_fmt.argtypes = [ci, i64, i64]
+    lib.q4nx_pack_fmt.restype = ci
+    lib.q4nx_pack_fmt.argtypes = [ci, vp, vp, vp, i64, i64, vp, sz]
+    lib.q4nx_unpack_fmt.restype = ci
+    lib.q4nx_unpack_fmt.argtypes = [ci, vp, i64, i64, vp, vp, vp]
+    lib.fdqp_run_fmt.restype = ci
+    lib.fdqp_run_fmt.argtypes = [vp, ci, vp, vp, vp, i64, i64, i64, vp]
+    lib.fdqp_dequant_fmt.restype = ci
+    lib.fdqp_dequant_fmt.argtypes = [vp, ci, vp, vp, ci, i64, i64, vp]
     lib.fdqp_create.restype = ci
     lib.fdqp_create.argtypes = [ctypes.POINTER(vp), ci, i64, i64, i64]
     lib.fdqp_destroy.restype = ci
@@ -224,6 +235,65 @@ def fdqp_run_noalloc(x_bf16, W_q4nx, y, M: int, K: int, N: int, stream=None) -> 
 def fdqp_dequant(ctx: int, W_q4nx, out, out_is_bf16: bool, K: int, N: int, stream=None) -> None:
     _check(load_library().fdqp_dequant(ctx, _addr(W_q4nx), _addr(out), int(out_is_bf16), K, N, _stream(stream)),
            "fdqp_dequant", ctx)
+
+
+FMT_Q4NX, FMT_G64, FMT_G128, FMT_MXFP4 = 0, 1, 2, 3
+_FMT_GROUP = {FMT_Q4NX: 32, FMT_G64: 64, FMT_G128: 128, FMT_MXFP4: 32}
+
+
+def q4nx_packed_bytes_fmt(fmt: int, K: int, N: int) -> int:
+    return int(load_library().q4nx_packed_bytes_fmt(int(fmt), K, N))
+
+
+def q4nx_pack_fmt(fmt: int, codes: np.ndarray, scales: np.ndarray, offsets_bf16=None) -> np.ndarray:
+    """codes[N,K] u8; scales[N,K/g]: bf16 bits (u16), or for FMT_MXFP4 the E8M0 bytes (any integer dtype, 0..254);
+    offsets[N,K/g] bf16 bits (None for FMT_MXFP4) -> packed bytes (host numpy)."""
+    if fmt not in _FMT_GROUP:
+        raise FdqpError(1, "q4nx_pack_fmt")
+    g = _FMT_GROUP[fmt]
+    codes = np.ascontiguousarray(codes, np.uint8)
+    N, K = codes.shape
+    mx = fmt == FMT_MXFP4
+    if mx and (np.asarray(scales).max(initial=0) > 255 or np.asarray(scales).min(initial=0) < 0):
+        raise FdqpError(1, "q4nx_pack_fmt", "E8M0 scales are bytes")
+    scales = np.ascontiguousarray(scales, np.uint8 if mx else np.uint16)
+    offs = None if mx else np.ascontiguousarray(offsets_bf16, np.uint16)
+    size = q4nx_packed_bytes_fmt(fmt, K, N)
+    if size == 0:
+        raise FdqpError(2, "q4nx_pack_fmt")
+    if scales.shape != (N, K // g) or (offs is not None and offs.shape != (N, K // g)):
+        raise FdqpError(2, "q4nx_pack_fmt", "scales/offsets must be [N, K/g]")
+    out = np.empty(size, np.uint8)
+    _check(load_library().q4nx_pack_fmt(int(fmt), codes.ctypes.data, scales.ctypes.data,
+                                        None if offs is None else offs.ctypes.data, K, N, out.ctypes.data, out.size),
+           "q4nx_pack_fmt")
+    return out
+
+
+def q4nx_unpack_fmt(fmt: int, packed: np.ndarray, K: int, N: int):
+    """-> (codes[N,K] u8, scales[N,K/g] (u16 bf16 bits, or u8 E8M0 bytes for FMT_MXFP4), offsets or None)."""
+    packed = np.ascontiguousarray(packed, np.uint8)
+    if fmt not in _FMT_GROUP or q4nx_packed_bytes_fmt(fmt, K, N) == 0 or packed.size != q4nx_packed_bytes_fmt(fmt, K, N):
+        raise FdqpError(2, "q4nx_unpack_fmt")
+    g = _FMT_GROUP[fmt]
+    mx = fmt == FMT_MXFP4
+    codes = np.empty((N, K), np.uint8)
+    scales = np.empty((N, K // g), np.uint8 if mx else np.uint16)
+    offs = None if mx else np.empty((N, K // g), np.uint16)
+    _check(load_library().q4nx_unpack_fmt(int(fmt), packed.ctypes.data, K, N, codes.ctypes.data, scales.ctypes.data,
+                                          None if offs is None else offs.ctypes.data), "q4nx_unpack_fmt")
+    return codes, scales, offs
+
+
+def fdqp_run_fmt(ctx: int, fmt: int, x_bf16, W_packed, y, M: int, K: int, N: int, stream=None) -> None:
+    """fdqp_run for a matrix packed in a format variant (FMT_G64, FMT_G128, FMT_MXFP4; FMT_Q4NX = fdqp_run)."""
+    _check(load_library().fdqp_run_fmt(ctx, int(fmt), _addr(x_bf16), _addr(W_packed), _addr(y), M, K, N, _stream(stream)),
+           "fdqp_run_fmt", ctx)
+
+
+def fdqp_dequant_fmt(ctx: int, fmt: int, W_packed, out, out_is_bf16: bool, K: int, N: int, stream=None) -> None:
+    _check(load_library().fdqp_dequant_fmt(ctx, int(fmt), _addr(W_packed), _addr(out), int(out_is_bf16), K, N,
+                                           _stream(stream)), "fdqp_dequant_fmt", ctx)
 
 
 def fdqp_last_status(ctx: int) -> int:

@@ -10,6 +10,7 @@
 #include <string>
 
 #include "fdqp.h"
+#include "fdqp_format.h"
 #include "fdqp_plan.h"
 
 namespace fdqp {
@@ -19,6 +20,7 @@ cudaError_t splitk_sum_launch(const float* ws, float* y, uint16_t* y16, int epi,
                               cudaStream_t stream);
 cudaError_t xprep_launch(const uint16_t* x, uint32_t* xq, float* xsc, int M, int K, cudaStream_t stream);
 cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
+cudaError_t dequant_fmt_launch(int fmt, const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
 cudaError_t prefill_set_smem_limit();
 cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, uint16_t* y16, int epi, float* ws,
                            int* status, int M, int K, int N, int pair, int Z, cudaStream_t stream);
@@ -144,9 +146,9 @@ struct SmemLayout {
     int nstage;
 };
 
-SmemLayout smem_layout(const fdqp_ctx* ctx, int M, int nbz, int cw, int ctas_per_sm, int bpw) {
+SmemLayout smem_layout(const fdqp_ctx* ctx, int M, int nbz, int cw, int ctas_per_sm, int bpw, int fmt) {
     SmemLayout L;
-    L.stage_bytes = (uint32_t)(cw / 8) * (uint32_t)bpw * kBlockBytes;
+    L.stage_bytes = (uint32_t)(cw / 8) * (uint32_t)bpw * (uint32_t)fmt_block_bytes(fmt);
     const uint32_t tiles = (uint32_t)nbz * 8u;
     L.xs_bytes = tiles * 128u * (uint32_t)M;          // prepared activations of the K slice
     L.xsum_bytes = M <= kColsMaxTokens ? 0u : tiles * 64u;         // per-token {sum x, unit} (plane mode only)
@@ -160,8 +162,9 @@ SmemLayout smem_layout(const fdqp_ctx* ctx, int M, int nbz, int cw, int ctas_per
 }
 
 // Fill the launch plan of one GEMV launch (M <= 8).  Returns false if no ring fits.
-bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, GemvPlan* p) {
+bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, GemvPlan* p, int fmt = kFmtQ4nx) {
     std::memset(p, 0, sizeof(*p));
+    p->fmt = fmt;
     p->M = M;
     p->K = K;
     p->N = N;
@@ -171,11 +174,13 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     // every size; two 10-warp CTAs per SM remain available as a launch parameter
     int ctas_per_sm = ctx->p_ctas_per_sm > 0 ? (int)ctx->p_ctas_per_sm : 1;
     if (ctas_per_sm > kMaxCtasPerSm) ctas_per_sm = kMaxCtasPerSm;
+    if (fmt != kFmtQ4nx) ctas_per_sm = 1;  // the variants are built for the 16-consumer-warp shape only
     int cw = 16, Z = 1, nbz = p->nb, bpw = 2;
     SmemLayout L{};
     for (;; --ctas_per_sm) {
         // register file: one 19-warp CTA or two 10-warp CTAs fit an SM
         cw = ctas_per_sm > 1 ? 8 : ((ctx->p_cw == 8 || ctx->p_cw == 16) ? (int)ctx->p_cw : 16);
+        if (fmt != kFmtQ4nx) cw = 16;
         // K slices: as few as leave a ring of at least kMinStages stages beside the staged activations
         Z = ctx->p_split_k > 0 ? (int)ctx->p_split_k : 1;
         for (;; Z *= 2) {
@@ -185,10 +190,10 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
             const int64_t blocks_per_cta = (int64_t)p->S * p->nb / ((int64_t)ctx->sm_count * ctas_per_sm);
             // (measured: pays up to M = 4, never when the larger stage would force a K split)
             bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (M <= 4 && blocks_per_cta >= 4 ? 4 : 2);
-            L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw);
+            L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw, fmt);
             if (bpw == 4 && ctx->p_bpw != 4 && M > 1 && L.nstage < kMinStages) {
                 bpw = 2;
-                L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw);
+                L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw, fmt);
             }
             if (L.nstage >= kMinStages || Z >= kMaxSplit || Z >= p->nb) break;
         }
@@ -350,15 +355,18 @@ namespace {
 // gamma != nullptr: x is RMS-normalised first, x <- bf16(x * rsqrt(mean_k x^2 + eps) * (1 + gamma)) per token row --
 // inside the GEMV kernel's activation preparation when that runs in-kernel on the whole row, else by a kernel of its own.
 fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, float eps, const void* W_q4nx, void* out,
-                     int epi, int64_t M, int64_t K, int64_t N, void* cuda_stream) {
+                     int epi, int64_t M, int64_t K, int64_t N, void* cuda_stream, int fmt = kFmtQ4nx) {
     if (!ctx || !x_bf16 || !W_q4nx || !out) return FDQP_ERR_ARG;
+    if (fmt < 0 || fmt >= kFmtCount) return FDQP_ERR_ARG;
+    if (fmt != kFmtQ4nx && (K % kBlockK) != 0) return FDQP_ERR_SHAPE;           // the variants hold whole blocks only
+    if (fmt != kFmtQ4nx && (epi != kEpiNone || gamma_bf16)) return FDQP_ERR_ARG;  // ... and have the fp32 store only
     if (gamma_bf16 && !aligned16(gamma_bf16)) return FDQP_ERR_ALIGN;
     if (gamma_bf16 && !(eps >= 0.f)) return FDQP_ERR_ARG;
     if (epi != kEpiNone && epi != kEpiBf16 && epi != kEpiGegluBf16) return FDQP_ERR_ARG;
     fdqp_status st = check_shape(ctx, M, K, N);
     if (st != FDQP_OK) return st;
     if (!aligned16(x_bf16) || !aligned16(W_q4nx) || !aligned16(out)) return FDQP_ERR_ALIGN;
-    if ((epi != kEpiNone || gamma_bf16) && ctx->p_path == 1) return FDQP_ERR_ARG;  // the plain self-check kernel does neither
+    if ((epi != kEpiNone || gamma_bf16 || fmt != kFmtQ4nx) && ctx->p_path == 1) return FDQP_ERR_ARG;  // the plain self-check kernel does none of these
     float* y = epi == kEpiNone ? static_cast<float*>(out) : nullptr;
     uint16_t* y16 = epi == kEpiNone ? nullptr : static_cast<uint16_t*>(out);
     const int64_t n_out = epi == kEpiGegluBf16 ? N / 2 : N;  // output values per token row
@@ -388,7 +396,7 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
         ctx->launches += 1;
         return FDQP_OK;
     }
-    if (use_prefill(ctx, M, K, N)) {
+    if (fmt == kFmtQ4nx && use_prefill(ctx, M, K, N)) {
         // prefill-sized M: dequantise into shared memory, contract with tcgen05 (accumulators in TMEM)
         const uint16_t* xt = x;
         int64_t x_row_bytes = K * 2;
@@ -410,7 +418,7 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
         const int mc = (int)((M - m0) < kMaxTokens ? (M - m0) : kMaxTokens);
         GemvPlan plan;
         int cw = 0;
-        if (!plan_gemv(ctx, mc, (int)K, (int)N, &cw, &plan)) return FDQP_ERR_SIZE;
+        if (!plan_gemv(ctx, mc, (int)K, (int)N, &cw, &plan, fmt)) return FDQP_ERR_SIZE;
         plan.W = W;
         plan.x = x + m0 * K;
         plan.y = y ? y + m0 * N : nullptr;
@@ -448,6 +456,11 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
 extern "C" fdqp_status fdqp_run(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, float* y, int64_t M, int64_t K,
                                 int64_t N, void* cuda_stream) {
     return run_impl(ctx, x_bf16, nullptr, 0.f, W_q4nx, y, kEpiNone, M, K, N, cuda_stream);
+}
+
+extern "C" fdqp_status fdqp_run_fmt(fdqp_ctx* ctx, int format, const void* x_bf16, const void* W_packed, float* y, int64_t M,
+                                    int64_t K, int64_t N, void* cuda_stream) {
+    return run_impl(ctx, x_bf16, nullptr, 0.f, W_packed, y, kEpiNone, M, K, N, cuda_stream, format);
 }
 
 extern "C" fdqp_status fdqp_run_epilogue(fdqp_ctx* ctx, const void* x_bf16, const void* W_q4nx, void* out, int epilogue,
@@ -521,6 +534,24 @@ extern "C" fdqp_status fdqp_dequant(fdqp_ctx* ctx, const void* W_q4nx, void* out
     if (!guard.ok) return FDQP_ERR_CUDA;
     cudaError_t e = dequant_launch(static_cast<const uint8_t*>(W_q4nx), out, out_is_bf16 != 0, (int)K, (int)N,
                                    static_cast<cudaStream_t>(cuda_stream));
+    if (e) return cuda_fail(ctx, e, "dequant kernel launch");
+    ctx->launches += 1;
+    return FDQP_OK;
+}
+
+extern "C" fdqp_status fdqp_dequant_fmt(fdqp_ctx* ctx, int format, const void* W_packed, void* out, int out_is_bf16,
+                                        int64_t K, int64_t N, void* cuda_stream) {
+    if (format == kFmtQ4nx) return fdqp_dequant(ctx, W_packed, out, out_is_bf16, K, N, cuda_stream);
+    if (!ctx || !W_packed || !out || (out_is_bf16 != 0 && out_is_bf16 != 1) || format < 0 || format >= kFmtCount)
+        return FDQP_ERR_ARG;
+    fdqp_status st = check_shape(ctx, 1, K, N);
+    if (st != FDQP_OK) return st;
+    if ((K % kBlockK) != 0) return FDQP_ERR_SHAPE;
+    if (!aligned16(W_packed) || !aligned16(out)) return FDQP_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FDQP_ERR_CUDA;
+    cudaError_t e = dequant_fmt_launch(format, static_cast<const uint8_t*>(W_packed), out, out_is_bf16 != 0, (int)K, (int)N,
+                                       static_cast<cudaStream_t>(cuda_stream));
     if (e) return cuda_fail(ctx, e, "dequant kernel launch");
     ctx->launches += 1;
     return FDQP_OK;

@@ -40,6 +40,7 @@
 // global memory is off its critical path and its last piece is a whole strip written directly.
 // No CTA ever waits for another CTA.
 #include "fdqp_device.cuh"
+#include "fdqp_format.h"
 #include "fdqp_plan.h"
 
 namespace fdqp {
@@ -210,17 +211,46 @@ struct LaneAddr {
 };
 
 // Column modes: so_addr addresses the scale chunks only (lanes 0..15 matter); m_addr is this lane's own offset word.
-template <int MODE>
+// MXFP4: so_addr is the byte address of row g's scale of this tile, m_addr that of row `lane`'s; so[0..3] then hold,
+// as fp32 bits, the scales 2^(e-127) of rows g, g+8, g+16, g+24 (a scale byte of 0, i.e. 2^-127, counts as 0 here),
+// m_row that of row `lane`; the B fragments are re-ordered to the natural k order the element look-up produces.
+__device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+// {even k, odd k} byte order of a B fragment pair -> {k 0..3, k 4..7}
+__device__ __forceinline__ void mx_natural_order(uint32_t& b0, uint32_t& b1) {
+    const uint32_t e = b0, o = b1;
+    b0 = prmt(e, o, 0x5140u);
+    b1 = prmt(e, o, 0x7362u);
+}
+
+template <int MODE, int FMT = kFmtQ4nx>
 __device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_t so_addr, uint32_t m_addr, int tile,
                                           const LaneAddr& la) {
     using T = ModeTraits<MODE>;
+    constexpr bool kMx = FmtTraits<FMT>::kMx;
     ldmatrix_x4(t.c, code_addr);
+    if (kMx) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) t.so[k] = lds_u8(so_addr + 8u * k) << 23;
+    }
     if (T::kCols) {
-        uint32_t dd[2];
-        ldmatrix_x2_trans(dd, so_addr);
-        t.so[0] = dd[0];
-        t.so[1] = dd[1];
-        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(t.m_row) : "r"(m_addr));
+        if (kMx) {
+            t.m_row = lds_u8(m_addr) << 23;
+        } else {
+            uint32_t dd[2];
+            ldmatrix_x2_trans(dd, so_addr);
+            t.so[0] = dd[0];
+            t.so[1] = dd[1];
+            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(t.m_row) : "r"(m_addr));
+        }
         const uint32_t tb = la.xs + (uint32_t)tile * la.x_stride;
         asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(t.b[0]), "=r"(t.b[1]) : "r"(tb + la.xb_off));
         const float2 v = lds64f(tb + la.sc_off);
@@ -231,8 +261,9 @@ __device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_
             t.xrow[0] = xr.x;
             t.xrow[1] = xr.y;
         }
+        if (kMx) mx_natural_order(t.b[0], t.b[1]);
     } else {
-        ldmatrix_x4_trans(t.so, so_addr);
+        if (!kMx) ldmatrix_x4_trans(t.so, so_addr);
         const uint32_t x_addr = la.x_lane + (uint32_t)tile * la.x_stride;
         const uint4 r0 = lds128(x_addr);
         t.b[0] = r0.x; t.b[1] = r0.y; t.b[2] = r0.z; t.b[3] = r0.w;
@@ -240,7 +271,47 @@ __device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_
         asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
                      : "=f"(t.sc[0]), "=f"(t.sc[1]), "=f"(t.sc[2]), "=f"(t.sc[3])
                      : "r"(la.xsc_lane + (uint32_t)tile * 64u));
+        if (kMx) {
+            mx_natural_order(t.b[0], t.b[1]);
+            mx_natural_order(t.b[2], t.b[3]);
+            mx_natural_order(t.b[4], t.b[5]);
+        }
     }
+}
+
+// Eight E2M1 codes of a word -> the unsigned bytes 2v + 12 (0 .. 24) of k 0..3 and k 4..7.  A 16-entry table as two
+// byte permutes: a selector nibble with bit 3 set returns the selected byte's sign fill, which is 0 for these bytes, so
+// the table of the non-negative codes answers only codes 0..7 and, with bit 3 flipped, that of the negative codes only
+// codes 8..15.
+// The two answers are disjoint (one of them is 0 in every byte), so they are not merged: each goes through the MMA and
+// the accumulator adds them.
+struct MxBytes {
+    uint32_t pos_lo, pos_hi, neg_lo, neg_hi;
+};
+__device__ __forceinline__ MxBytes mx_codes_to_bytes(uint32_t w) {
+    constexpr uint32_t kPos0 = 0x0F0E0D0Cu, kPos1 = 0x18141210u;  // 12 + {0, 1, 2, 3, 4, 6, 8, 12}
+    constexpr uint32_t kNeg0 = 0x090A0B0Cu, kNeg1 = 0x00040608u;  // 12 - {0, 1, 2, 3, 4, 6, 8, 12}
+    const uint32_t wn = w ^ 0x88888888u;
+    MxBytes r;
+    r.pos_lo = prmt(kPos0, kPos1, w);
+    r.neg_lo = prmt(kNeg0, kNeg1, wn);
+    r.pos_hi = prmt(kPos0, kPos1, w >> 16);
+    r.neg_hi = prmt(kNeg0, kNeg1, wn >> 16);
+    return r;
+}
+
+// d += A . B (same shapes and types as imma below)
+template <bool B_SIGNED>
+__device__ __forceinline__ void imma_acc(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+    if (B_SIGNED)
+        asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 template <bool B_SIGNED>
@@ -268,27 +339,37 @@ struct LaneConst {
 // acc[row][.] += d * unit * (sum_k q_k X_k) + m * (sum_k x_k), fp32 (Eq. 3 applied per group).
 // `unit` (and 256 * unit) are powers of two, so d * unit is formed exactly by the mixed bf16 FMA.
 // Column modes keep the offset term sum_g m_g * X_g in a lane-per-row layout (acc_m[tok], row = lane).
-template <int MODE>
+// MXFP4 (FMT): the element bytes 2v + 12 take the codes' place, half the power-of-two scale takes d's, and -12 times
+// that takes m's.
+template <int MODE, int FMT = kFmtQ4nx>
 __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][ModeTraits<MODE>::kAcc],
                                              float (&acc_m)[ModeTraits<MODE>::kAccM], const LaneConst& lc) {
     using T = ModeTraits<MODE>;
+    constexpr bool kMx = FmtTraits<FMT>::kMx;
     if (T::kCols) {
-        const float mw = bf16lo_mul_f32hi(t.m_row, 1.0f);
+        const float mw = kMx ? -0.5f * (float)kMxBias * __uint_as_float(t.m_row) : bf16lo_mul_f32hi(t.m_row, 1.0f);
         if (T::kXRow) {
 #pragma unroll
             for (int tk = 0; tk < T::kAccM; ++tk) acc_m[tk] = fmaf(mw, t.xrow[tk], acc_m[tk]);
         } else {
             acc_m[0] = fmaf(mw, t.sc[0], acc_m[0]);
         }
-        const float uq = t.sc[1] * lc.w_unit;
+        const float uq = t.sc[1] * lc.w_unit;  // (MXFP4: w_unit carries the 1/2 of the elements' integer form)
 #pragma unroll
         for (int h = 0; h < 2; ++h) {  // rows (g, g+8) then (g+16, g+24)
             const uint32_t w0 = t.c[2 * h], w1 = t.c[2 * h + 1];
-            const uint32_t e0 = w0 & 0x0F0F0F0Fu, o0 = (w0 >> 4) & 0x0F0F0F0Fu;  // even-k codes, odd-k codes
-            const uint32_t e1 = w1 & 0x0F0F0F0Fu, o1 = (w1 >> 4) & 0x0F0F0F0Fu;
             int d[4];
-            imma<true>(d, e0, e1, o0, o1, t.b[0], t.b[1]);
-            const float dq[2] = {bf16lo_mul_f32hi(t.so[h], uq), bf16hi_mul_f32hi(t.so[h], uq)};
+            if (kMx) {
+                const MxBytes m0 = mx_codes_to_bytes(w0), m1 = mx_codes_to_bytes(w1);  // lo: k 0..3, hi: k 4..7
+                imma<true>(d, m0.pos_lo, m1.pos_lo, m0.pos_hi, m1.pos_hi, t.b[0], t.b[1]);
+                imma_acc<true>(d, m0.neg_lo, m1.neg_lo, m0.neg_hi, m1.neg_hi, t.b[0], t.b[1]);
+            } else {
+                const uint32_t e0 = w0 & 0x0F0F0F0Fu, o0 = (w0 >> 4) & 0x0F0F0F0Fu;  // even-k codes, odd-k codes
+                const uint32_t e1 = w1 & 0x0F0F0F0Fu, o1 = (w1 >> 4) & 0x0F0F0F0Fu;
+                imma<true>(d, e0, e1, o0, o1, t.b[0], t.b[1]);
+            }
+            const float dq[2] = {kMx ? __uint_as_float(t.so[2 * h]) * uq : bf16lo_mul_f32hi(t.so[h], uq),
+                                 kMx ? __uint_as_float(t.so[2 * h + 1]) * uq : bf16hi_mul_f32hi(t.so[h], uq)};
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 // the lane's two columns combined in integers (exact, |.| < 2^24), one conversion
@@ -298,17 +379,31 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][Mo
         }
         return;
     }
-    const float mof[4] = {bf16lo_mul_f32hi(t.so[2], 1.0f), bf16hi_mul_f32hi(t.so[2], 1.0f),
-                          bf16lo_mul_f32hi(t.so[3], 1.0f), bf16hi_mul_f32hi(t.so[3], 1.0f)};
+    constexpr float kMxOff = -0.5f * (float)kMxBias;
+    const float mof[4] = {kMx ? kMxOff * __uint_as_float(t.so[0]) : bf16lo_mul_f32hi(t.so[2], 1.0f),
+                          kMx ? kMxOff * __uint_as_float(t.so[1]) : bf16hi_mul_f32hi(t.so[2], 1.0f),
+                          kMx ? kMxOff * __uint_as_float(t.so[2]) : bf16lo_mul_f32hi(t.so[3], 1.0f),
+                          kMx ? kMxOff * __uint_as_float(t.so[3]) : bf16hi_mul_f32hi(t.so[3], 1.0f)};
+    const float half_unit[2] = {0.5f * t.sc[1], 0.5f * t.sc[3]};  // MXFP4: the 1/2 of the elements' integer form
 #pragma unroll
     for (int h = 0; h < 2; ++h) {  // rows (g, g+8) then (g+16, g+24)
         const uint32_t w0 = t.c[2 * h], w1 = t.c[2 * h + 1];
-        const uint32_t e0 = w0 & 0x0F0F0F0Fu, o0 = (w0 >> 4) & 0x0F0F0F0Fu;  // even-k codes, odd-k codes
-        const uint32_t e1 = w1 & 0x0F0F0F0Fu, o1 = (w1 >> 4) & 0x0F0F0F0Fu;
         int d2[4], d1[4], d0[4];
-        imma<true>(d2, e0, e1, o0, o1, t.b[0], t.b[1]);
-        imma<false>(d1, e0, e1, o0, o1, t.b[2], t.b[3]);
-        imma<false>(d0, e0, e1, o0, o1, t.b[4], t.b[5]);
+        if (kMx) {
+            // three planes share the A operand: merging the two answers (four ORs) is cheaper than six more MMAs
+            const MxBytes m0 = mx_codes_to_bytes(w0), m1 = mx_codes_to_bytes(w1);  // lo: k 0..3, hi: k 4..7
+            const uint32_t e0 = m0.pos_lo | m0.neg_lo, o0 = m0.pos_hi | m0.neg_hi;
+            const uint32_t e1 = m1.pos_lo | m1.neg_lo, o1 = m1.pos_hi | m1.neg_hi;
+            imma<true>(d2, e0, e1, o0, o1, t.b[0], t.b[1]);
+            imma<false>(d1, e0, e1, o0, o1, t.b[2], t.b[3]);
+            imma<false>(d0, e0, e1, o0, o1, t.b[4], t.b[5]);
+        } else {
+            const uint32_t e0 = w0 & 0x0F0F0F0Fu, o0 = (w0 >> 4) & 0x0F0F0F0Fu;  // even-k codes, odd-k codes
+            const uint32_t e1 = w1 & 0x0F0F0F0Fu, o1 = (w1 >> 4) & 0x0F0F0F0Fu;
+            imma<true>(d2, e0, e1, o0, o1, t.b[0], t.b[1]);
+            imma<false>(d1, e0, e1, o0, o1, t.b[2], t.b[3]);
+            imma<false>(d0, e0, e1, o0, o1, t.b[4], t.b[5]);
+        }
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             const int i = 2 * h + r;
@@ -317,8 +412,9 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][Mo
                 const int e = 2 * r + j;
                 // planes recombined in integers (|.| < 2^31), then one conversion (exact below 2^24, else one rounding)
                 const float s = __int2float_rn((d2[e] * 256 + d1[e]) * 256 + d0[e]);
-                const float dq = r == 0 ? bf16lo_mul_f32hi(t.so[h], t.sc[2 * j + 1])
-                                        : bf16hi_mul_f32hi(t.so[h], t.sc[2 * j + 1]);
+                const float dq = kMx ? __uint_as_float(t.so[i]) * half_unit[j]
+                                     : (r == 0 ? bf16lo_mul_f32hi(t.so[h], t.sc[2 * j + 1])
+                                               : bf16hi_mul_f32hi(t.so[h], t.sc[2 * j + 1]));
                 acc[i][j] = fmaf(dq, s, acc[i][j]);
                 acc[i][j] = fmaf(mof[i], t.sc[2 * j], acc[i][j]);
             }
@@ -331,15 +427,20 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][Mo
 // A ring stage holds CB = (CW / 8) * BPW blocks; warp w owns group-tile (w & 7) of the BPW (2 or 4) consecutive
 // blocks starting at BPW * (w >> 3) of every stage.  More blocks per stage = fewer barrier round trips per tile.
 // Warps CW+1 .. CW+NR are reducers (NR = CW / 8): reducer r completes the strip pieces with piece % NR == r.
-template <int CW, int MODE, int BPW, bool EPI>
+// FMT: the container's format (fdqp_format.h).  The variants differ in the block size, in where a tile's scale and
+// offset sit (one per 64 or 128 inputs: tiles share them) and, for MXFP4, in how codes and scales become numbers; they
+// hold whole blocks only.
+template <int CW, int MODE, int BPW, bool EPI, int FMT = kFmtQ4nx>
 __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
     fdqp_gemv_kernel(const __grid_constant__ GemvPlan p) {
     extern __shared__ __align__(128) uint8_t smem[];
     using MT = ModeTraits<MODE>;
+    using F = FmtTraits<FMT>;
     constexpr int NT = MT::kAcc;
     constexpr int CB = (CW / 8) * BPW;
     constexpr int NR = CW / 8;
-    constexpr uint32_t kStageBytes = CB * kBlockBytes;
+    constexpr uint32_t kBB = F::kBlock;  // bytes of a full block
+    constexpr uint32_t kStageBytes = CB * kBB;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int M = MODE == 1 ? 1 : (MODE == 3 ? 2 : p.M), K = p.K;  // compile-time in the column modes
 
@@ -390,7 +491,7 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const int groups_total = K / kGroup;
-    const int64_t strip_bytes = (int64_t)kGroupBytes * groups_total;
+    const int64_t strip_bytes = FMT == kFmtQ4nx ? (int64_t)kGroupBytes * groups_total : (int64_t)kBB * (groups_total / 8);
 
     if (warp == CW) {
         // =============================== producer ================================================
@@ -422,14 +523,14 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                 ps = s_first + so;
                 pbl = (int)(rel - so * (uint32_t)len);
                 const int rest = groups_total - 8 * (b_first + pbl);
-                bytes = (uint32_t)kGroupBytes * (uint32_t)(rest < 8 ? rest : 8);
+                bytes = FMT == kFmtQ4nx ? (uint32_t)kGroupBytes * (uint32_t)(rest < 8 ? rest : 8) : kBB;
             }
             const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
             if (lane == 0) mbar_arrive_expect_tx(full0 + 8u * stage, total);
             __syncwarp();
             if (bytes) {
-                const uint8_t* src = p.W + ps * strip_bytes + (int64_t)(b_first + pbl) * kBlockBytes;
-                const uint32_t dst = ring + stage * kStageBytes + lane * kBlockBytes;
+                const uint8_t* src = p.W + ps * strip_bytes + (int64_t)(b_first + pbl) * kBB;
+                const uint32_t dst = ring + stage * kStageBytes + lane * kBB;
                 if (p.evict_first)
                     bulk_g2s_hint(dst, src, bytes, full0 + 8u * stage, policy);
                 else
@@ -468,7 +569,7 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             la.xb_off = (tok_b < M && pl < 3) ? (uint32_t)(tok_b * 128 + pl * 32 + q * 8) : 104u;
             const int tok_d = q >> 1;
             la.sc_off = (uint32_t)((tok_d < M ? tok_d : 0) * 128 + 96);
-            lc.w_unit = tok_d < M ? ((q & 1) ? 1.f : 256.f) : 0.f;
+            lc.w_unit = (tok_d < M ? ((q & 1) ? 1.f : 256.f) : 0.f) * (F::kMx ? 0.5f : 1.f);
         }
         float acc_m[MT::kAccM];  // column modes: offset term of row `lane`, per token
 #pragma unroll
@@ -478,9 +579,13 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         // transposed load every lane of a quad holds (d[g], d[g+8]), (d[g+16], d[g+24]), (m..), (m..)
         const uint32_t code_lane = tw * 512 + lane * 16;
         const int mat = lane >> 3;
-        const uint32_t so_chunk = tw * 64 + (((mat & 1) * 2 + (lane & 1)) * 16);
+        const uint32_t so_chunk = (tw >> F::kShift) * 64 + (((mat & 1) * 2 + (lane & 1)) * 16);
         const uint32_t so_sect = (!MT::kCols && mat >= 2) ? 576u : 512u;  // offsets section follows the scales section
-        const uint32_t m_lane = tw * 64 + lane * 2;                         // column modes: this lane's own offset word
+        const uint32_t m_lane = (tw >> F::kShift) * 64 + lane * 2;         // column modes: this lane's own offset word
+        // the same two addresses inside a full block of the format (MXFP4: scale bytes of row g and of row `lane`)
+        const uint32_t so_full = F::kMx ? (uint32_t)kCodeBytes + tw * 32 + g
+                                        : ((!MT::kCols && mat >= 2) ? (uint32_t)F::kOffSect : (uint32_t)kCodeBytes) + so_chunk;
+        const uint32_t m_full = F::kMx ? (uint32_t)kCodeBytes + tw * 32 + lane : (uint32_t)F::kOffSect + m_lane;
 
         float acc[4][NT];
 #pragma unroll
@@ -627,7 +732,6 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         // An "interior" stage -- both of the warp's blocks inside the range and the current strip, every block
         // full -- needs no bookkeeping beyond two tile indices.  `lim` is the first position that is not interior.
         const bool all_full = (groups_total & 7) == 0;
-        const uint32_t so_lane8 = so_sect * 8u + so_chunk;
         auto interior_limit = [&]() { return (all_full && work) ? (unit_next < nblk ? unit_next : nblk) : -1; };
         int lim = interior_limit();
         int stage = 0;
@@ -640,23 +744,22 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             }
             if (!mbar_wait(full0 + 8u * stage, phase, p.status)) { alive = false; break; }
             if (warp == 0 && c == 0) FDQP_STAMP(3);
-            const uint32_t sbase = ring + stage * kStageBytes + j0 * kBlockBytes;
+            const uint32_t sbase = ring + stage * kStageBytes + j0 * kBB;
             if (i0 + BPW - 1 < lim) {
                 const int tile = (i0 - unit_first) * 8 + tw;
 #pragma unroll
                 for (int pr = 0; pr < BPW / 2; ++pr) {  // two tiles in flight at a time
-                    const uint32_t sb = sbase + pr * 2 * kBlockBytes;
+                    const uint32_t sb = sbase + pr * 2 * kBB;
                     TileIn ta, tb;
-                    tile_load<MODE>(ta, sb + code_lane, sb + so_lane8, sb + 576u * 8u + m_lane, tile + 16 * pr, la);
-                    tile_load<MODE>(tb, sb + kBlockBytes + code_lane, sb + kBlockBytes + so_lane8,
-                                    sb + kBlockBytes + 576u * 8u + m_lane, tile + 16 * pr + 8, la);
-                    tile_compute<MODE>(ta, acc, acc_m, lc);
+                    tile_load<MODE, FMT>(ta, sb + code_lane, sb + so_full, sb + m_full, tile + 16 * pr, la);
+                    tile_load<MODE, FMT>(tb, sb + kBB + code_lane, sb + kBB + so_full, sb + kBB + m_full, tile + 16 * pr + 8, la);
+                    tile_compute<MODE, FMT>(ta, acc, acc_m, lc);
                     if (pr == BPW / 2 - 1) {
                         // every shared-memory read of this stage has been issued and consumed in order: hand it back
                         __syncwarp();
                         if (lane == 0) mbar_arrive(empty0 + 8u * stage);
                     }
-                    tile_compute<MODE>(tb, acc, acc_m, lc);
+                    tile_compute<MODE, FMT>(tb, acc, acc_m, lc);
                 }
             } else if (all_full && work && i0 + BPW <= nblk && unit_next > i0 && unit_next - first_fix + len >= i0 + BPW) {
                 // exactly one strip boundary inside the warp's blocks, every block full and inside the range: the blocks
@@ -670,19 +773,18 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                         next_unit();
                         lim = interior_limit();
                     }
-                    const uint32_t sb = sbase + jj * kBlockBytes;
+                    const uint32_t sb = sbase + jj * kBB;
                     const int tile = (i0 + jj - unit_first) * 8 + tw;
                     TileIn ta;
-                    tile_load<MODE>(ta, sb + code_lane, sb + so_lane8, sb + 576u * 8u + m_lane, tile, la);
+                    tile_load<MODE, FMT>(ta, sb + code_lane, sb + so_full, sb + m_full, tile, la);
                     if (jj + 1 < BPW && jj + 1 != pb) {
                         TileIn tb;
-                        tile_load<MODE>(tb, sb + kBlockBytes + code_lane, sb + kBlockBytes + so_lane8,
-                                        sb + kBlockBytes + 576u * 8u + m_lane, tile + 8, la);
-                        tile_compute<MODE>(ta, acc, acc_m, lc);
-                        tile_compute<MODE>(tb, acc, acc_m, lc);
+                        tile_load<MODE, FMT>(tb, sb + kBB + code_lane, sb + kBB + so_full, sb + kBB + m_full, tile + 8, la);
+                        tile_compute<MODE, FMT>(ta, acc, acc_m, lc);
+                        tile_compute<MODE, FMT>(tb, acc, acc_m, lc);
                         jj += 2;
                     } else {
-                        tile_compute<MODE>(ta, acc, acc_m, lc);
+                        tile_compute<MODE, FMT>(ta, acc, acc_m, lc);
                         jj += 1;
                     }
                 }
@@ -701,11 +803,14 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                     const int rest = groups_total - 8 * (b_first + bl);
                     const int jb = rest < 8 ? rest : 8;
                     if (work && tw < jb) {
-                        const uint32_t sb = sbase + jj * kBlockBytes;
+                        const uint32_t sb = sbase + jj * kBB;
                         const int tile = bl * 8 + tw;
                         TileIn ta;
-                        tile_load<MODE>(ta, sb + code_lane, sb + so_sect * jb + so_chunk, sb + 576u * jb + m_lane, tile, la);
-                        tile_compute<MODE>(ta, acc, acc_m, lc);
+                        if (FMT == kFmtQ4nx)  // the only format with short last blocks
+                            tile_load<MODE, FMT>(ta, sb + code_lane, sb + so_sect * jb + so_chunk, sb + 576u * jb + m_lane, tile, la);
+                        else
+                            tile_load<MODE, FMT>(ta, sb + code_lane, sb + so_full, sb + m_full, tile, la);
+                        tile_compute<MODE, FMT>(ta, acc, acc_m, lc);
                     }
                 }
                 __syncwarp();
@@ -970,7 +1075,38 @@ cudaError_t splitk_sum_launch(const float* ws, float* y, uint16_t* y16, int epi,
 }
 
 // consumer_warps: 8 or 16; p.bpw (blocks per warp per stage): 2 or 4.  Kernel mode by M (see the header).
+// The format variants: 16 consumer warps, fp32 output.
+template <int FMT>
+static cudaError_t launch_fmt(const GemvPlan& p, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.Z * p.Gz));
+    cfg.blockDim = dim3((unsigned)((16 + 1 + 2) * 32));
+    cfg.dynamicSmemBytes = p.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    const bool b4 = p.bpw == 4;
+    if (p.M == 1)
+        return b4 ? cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<16, 1, 4, false, FMT>, p)
+                  : cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<16, 1, 2, false, FMT>, p);
+    if (p.M > kColsMaxTokens)
+        return b4 ? cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<16, 2, 4, false, FMT>, p)
+                  : cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<16, 2, 2, false, FMT>, p);
+    return b4 ? cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<16, 3, 4, false, FMT>, p)
+              : cudaLaunchKernelEx(&cfg, fdqp_gemv_kernel<16, 3, 2, false, FMT>, p);
+}
+
 cudaError_t gemv_launch(const GemvPlan& p, int consumer_warps, cudaStream_t stream) {
+    if (p.fmt != kFmtQ4nx) {
+        if (consumer_warps != 16 || p.epi != kEpiNone || p.norm) return cudaErrorInvalidValue;
+        if (p.fmt == kFmtG64) return launch_fmt<kFmtG64>(p, stream);
+        if (p.fmt == kFmtG128) return launch_fmt<kFmtG128>(p, stream);
+        if (p.fmt == kFmtMxfp4) return launch_fmt<kFmtMxfp4>(p, stream);
+        return cudaErrorInvalidValue;
+    }
     const bool w16 = consumer_warps == 16, b4 = p.bpw == 4;
     if (p.M == 1) {
         if (w16) return b4 ? launch_one<16, 1, 4>(p, stream) : launch_one<16, 1, 2>(p, stream);
@@ -994,8 +1130,23 @@ static cudaError_t set_smem_limit_mode(int bytes) {
     return cudaFuncSetAttribute(fdqp_gemv_kernel<CW, MODE, 4, true>, a, bytes);
 }
 
+template <int FMT>
+static cudaError_t set_smem_limit_fmt(int bytes) {
+    const cudaFuncAttribute a = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 1, 2, false, FMT>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 1, 4, false, FMT>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 2, 2, false, FMT>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 2, 4, false, FMT>, a, bytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_gemv_kernel<16, 3, 2, false, FMT>, a, bytes))) return e;
+    return cudaFuncSetAttribute(fdqp_gemv_kernel<16, 3, 4, false, FMT>, a, bytes);
+}
+
 cudaError_t gemv_set_smem_limit(int bytes) {
     cudaError_t e;
+    if ((e = set_smem_limit_fmt<kFmtG64>(bytes))) return e;
+    if ((e = set_smem_limit_fmt<kFmtG128>(bytes))) return e;
+    if ((e = set_smem_limit_fmt<kFmtMxfp4>(bytes))) return e;
     if ((e = set_smem_limit_mode<8, 1>(bytes))) return e;
     if ((e = set_smem_limit_mode<16, 1>(bytes))) return e;
     if ((e = set_smem_limit_mode<8, 2>(bytes))) return e;

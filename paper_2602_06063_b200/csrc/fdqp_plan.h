@@ -38,6 +38,7 @@ struct GemvPlan {
     float* ws_full;       // device, [Z][S][32*kMaxTokens] partial sums of whole strip-slices (Z > 1)
     int* tickets;         // device, [S] arrival counters, zero between launches
     int* status;          // host-mapped sticky status word
+    int fmt;              // container format (fdqp_format.h); 0 = Q4NX
     int M, K, N;
     int S;                // strips = N / 32
     int nb;               // blocks per strip = ceil(K / 256)

@@ -1,0 +1,154 @@
+"""GPU parity of the format variants of the block container (group sizes 64 / 128, MXFP4) against the CPU oracle:
+the dequantisation engine bit for bit, the projection within the acceptance bound, on every GEMV kernel mode."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2602_06063_b200 as fd
+import synthgen
+from gpu_common import MAX_K, MAX_M, MAX_N, assert_close, dev_bytes
+
+pytestmark = pytest.mark.gpu
+
+FMTS = [fd.FMT_G64, fd.FMT_G128, fd.FMT_MXFP4]
+NAMES = {fd.FMT_G64: "g64", fd.FMT_G128: "g128", fd.FMT_MXFP4: "mxfp4"}
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    h = fd.fdqp_create(0, MAX_M, MAX_K, MAX_N)
+    yield h
+    torch.cuda.synchronize()
+    fd.fdqp_destroy(h)
+
+
+class FmtCase:
+    def __init__(self, fmt, K, N, M, seed, amp=1.0, weights=None):
+        self.fmt, self.K, self.N, self.M = fmt, K, N, M
+        self.w = weights if weights is not None else synthgen.weights_fmt(seed, K, N, fmt)
+        self.x = synthgen.activations(seed + 1, M, K, amp)
+        self.packed = fd.q4nx_pack_fmt(fmt, self.w.codes, self.w.scales, self.w.offsets)
+        self.W_dev = dev_bytes(self.packed)
+        self.x_dev = dev_bytes(self.x)
+
+    def run(self, ctx, M=None):
+        M = self.M if M is None else M
+        y = torch.full((M, self.N), float("nan"), dtype=torch.float32, device="cuda")
+        fd.fdqp_run_fmt(ctx, self.fmt, self.x_dev, self.W_dev, y, M, self.K, self.N)
+        torch.cuda.synchronize()
+        assert fd.fdqp_last_status(ctx) == 0
+        return y.cpu().numpy()
+
+    def reference(self, n0=0, n1=None):
+        return oracle.fmt_project(self.fmt, self.x, self.w.codes, self.w.scales, self.w.offsets, n0=n0, n1=n1,
+                                  nthreads=min(16, oracle.max_threads()))
+
+
+@pytest.mark.parametrize("fmt", FMTS, ids=lambda f: NAMES[f])
+def test_packer_round_trip_and_oracle_reader(fmt):
+    K, N = 768, 96
+    w = synthgen.weights_fmt(40 + fmt, K, N, fmt)
+    packed = fd.q4nx_pack_fmt(fmt, w.codes, w.scales, w.offsets)
+    assert packed.size == oracle.fmt_packed_bytes(fmt, K, N) == fd.q4nx_packed_bytes_fmt(fmt, K, N)
+    c, s, o = oracle.fmt_unpack(fmt, packed, K, N)
+    assert np.array_equal(c, w.codes) and np.array_equal(s, w.scales)
+    assert fmt == fd.FMT_MXFP4 or np.array_equal(o, w.offsets)
+
+
+@pytest.mark.parametrize("fmt", FMTS, ids=lambda f: NAMES[f])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_dequant_engine_is_bit_exact(ctx, fmt, bf16):
+    K, N = 1024, 160
+    w = synthgen.weights_fmt(50 + fmt, K, N, fmt)
+    if fmt == fd.FMT_MXFP4:   # every scale byte the packer accepts, and every code, occur
+        w.scales[:, :] = (np.arange(w.scales.size, dtype=np.uint32) % 255).reshape(w.scales.shape).astype(np.uint16)
+    W_dev = dev_bytes(fd.q4nx_pack_fmt(fmt, w.codes, w.scales, w.offsets))
+    out = torch.empty((K, N), dtype=torch.bfloat16 if bf16 else torch.float32, device="cuda")
+    fd.fdqp_dequant_fmt(ctx, fmt, W_dev, out, bf16, K, N)
+    torch.cuda.synchronize()
+    w32, w16 = oracle.fmt_dequant(fmt, w.codes, w.scales, w.offsets)
+    if bf16:
+        assert np.array_equal(out.view(torch.int16).cpu().numpy().view(np.uint16), w16)
+    else:
+        assert np.array_equal(out.cpu().numpy().view(np.uint32), w32.view(np.uint32))
+
+
+# (K, N, M): one token (planes as columns), two (same, paired), three to eight (one MMA per plane); shapes whose strips
+# split across CTAs, whose K needs slices, and whose ranges are cut at strip boundaries
+SHAPES = [(256, 32, 1), (512, 64, 2), (2560, 4096, 1), (2560, 4096, 2), (2560, 4096, 3), (2560, 4096, 8), (10240, 2560, 1),
+          (10240, 2560, 5), (21504, 320, 1), (21504, 320, 8), (1280, 6912, 4), (3840, 1024, 7), (2560, 8192, 12)]
+
+
+@pytest.mark.parametrize("fmt", FMTS, ids=lambda f: NAMES[f])
+@pytest.mark.parametrize("K,N,M", SHAPES)
+def test_projection_matches_oracle(ctx, fmt, K, N, M):
+    amp = 1.0 / np.sqrt(K) if K > 20000 else 1.0
+    c = FmtCase(fmt, K, N, M, 6000 + K + N + M + fmt, amp)
+    y = c.run(ctx)
+    n1 = min(N, 1024)
+    y_ref, a_ref = c.reference(0, n1)
+    assert_close(y[:, :n1], y_ref, a_ref, f"{NAMES[fmt]} K={K} N={N} M={M}")
+    if N > n1:
+        y_ref, a_ref = c.reference(N - 256, N)
+        assert_close(y[:, N - 256:], y_ref, a_ref, f"{NAMES[fmt]} K={K} N={N} M={M} tail")
+
+
+@pytest.mark.parametrize("fmt", FMTS, ids=lambda f: NAMES[f])
+@pytest.mark.parametrize("M", [1, 2, 6])
+def test_exact_arithmetic_cases_are_bit_equal(ctx, fmt, M):
+    """Power-of-two scales, integer offsets and small integer activations: every partial sum is exact in fp32 in any
+    order, so the kernel must reproduce the oracle's value exactly."""
+    K, N = 1024, 256
+    w = synthgen.weights_fmt(70 + fmt, K, N, fmt)
+    r = synthgen.u64(71 + fmt, 3, w.scales.size).reshape(w.scales.shape)
+    if fmt == fd.FMT_MXFP4:
+        w.scales[:, :] = (124 + r % np.uint64(3)).astype(np.uint16)            # 2^-3 .. 2^-1
+    else:
+        w.scales[:, :] = 0x3E00                                                  # bf16 2^-3
+        w.offsets[:, :] = np.array([0xBF80, 0x0000, 0x3F80], np.uint16)[(r % np.uint64(3)).astype(np.int64)]
+    xi = (synthgen.u64(72 + fmt, 4, M * K).reshape(M, K) % np.uint64(5)).astype(np.float32) - 2.0
+    c = FmtCase(fmt, K, N, M, 0, weights=w)
+    c.x = synthgen.bf16_bits(xi)
+    c.x_dev = dev_bytes(c.x)
+    y = c.run(ctx)
+    y_ref, _ = c.reference()
+    assert np.array_equal(y.astype(np.float64), y_ref)
+
+
+@pytest.mark.parametrize("fmt", FMTS, ids=lambda f: NAMES[f])
+def test_full_size_lm_head_sampled_columns(ctx, fmt):
+    """The 4B LM head shape (K = 2560, N = 262144) in the launch configuration the benchmark times; the oracle checks
+    the first, middle and last 256 columns."""
+    K, N, M = 2560, 262144, 1
+    rng = np.random.default_rng(80 + fmt)
+    g = synthgen.FMT_GROUP[fmt]
+    codes = rng.integers(0, 16, (N, K), dtype=np.uint8)
+    if fmt == fd.FMT_MXFP4:
+        scales = rng.integers(118, 123, (N, K // g)).astype(np.uint16)
+        offsets = None
+    else:
+        scales = synthgen.bf16_bits(np.abs(rng.standard_normal((N, K // g), dtype=np.float32)) * 0.02)
+        offsets = synthgen.bf16_bits(rng.standard_normal((N, K // g), dtype=np.float32) * 0.01)
+    w = synthgen.Q4NXWeights(codes, scales, offsets)
+    c = FmtCase(fmt, K, N, M, 81, weights=w)
+    y = c.run(ctx)
+    for n0 in (0, N // 2 - 128, N - 256):
+        y_ref, a_ref = c.reference(n0, n0 + 256)
+        assert_close(y[:, n0:n0 + 256], y_ref, a_ref, f"{NAMES[fmt]} LM head columns {n0}..")
+
+
+def test_argument_errors(ctx):
+    x = torch.zeros((1, 512), dtype=torch.bfloat16, device="cuda")
+    W = torch.zeros(fd.q4nx_packed_bytes_fmt(fd.FMT_G64, 512, 64), dtype=torch.uint8, device="cuda")
+    y = torch.zeros((1, 64), dtype=torch.float32, device="cuda")
+    with pytest.raises(fd.FdqpError) as e:
+        fd.fdqp_run_fmt(ctx, 7, x, W, y, 1, 512, 64)
+    assert e.value.code == 1
+    with pytest.raises(fd.FdqpError) as e:
+        fd.fdqp_run_fmt(ctx, fd.FMT_MXFP4, x, W, y, 1, 288, 64)     # whole blocks only
+    assert e.value.code == 2
+    assert fd.q4nx_packed_bytes_fmt(fd.FMT_G128, 288, 64) == 0
+    with pytest.raises(fd.FdqpError):
+        fd.q4nx_pack_fmt(fd.FMT_MXFP4, np.zeros((32, 256), np.uint8), np.full((32, 8), 255), None)   # NaN scale
+    torch.cuda.synchronize()
