@@ -288,15 +288,26 @@ __device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_
 struct MxBytes {
     uint32_t pos_lo, pos_hi, neg_lo, neg_hi;
 };
-__device__ __forceinline__ MxBytes mx_codes_to_bytes(uint32_t w) {
-    constexpr uint32_t kPos0 = 0x0F0E0D0Cu, kPos1 = 0x18141210u;  // 12 + {0, 1, 2, 3, 4, 6, 8, 12}
-    constexpr uint32_t kNeg0 = 0x090A0B0Cu, kNeg1 = 0x00040608u;  // 12 - {0, 1, 2, 3, 4, 6, 8, 12}
+// The four table words live in registers for the whole kernel (loaded through an opaque move, so that the compiler
+// does not re-create the constants in front of every permute).
+struct MxTables {
+    uint32_t pos0, pos1, neg0, neg1;
+};
+__device__ __forceinline__ MxTables mx_tables() {
+    MxTables t;
+    asm volatile("mov.b32 %0, 0x0F0E0D0C;" : "=r"(t.pos0));  // 12 + {0, 1, 2, 3}
+    asm volatile("mov.b32 %0, 0x18141210;" : "=r"(t.pos1));  // 12 + {4, 6, 8, 12}
+    asm volatile("mov.b32 %0, 0x090A0B0C;" : "=r"(t.neg0));  // 12 - {0, 1, 2, 3}
+    asm volatile("mov.b32 %0, 0x00040608;" : "=r"(t.neg1));  // 12 - {4, 6, 8, 12}
+    return t;
+}
+__device__ __forceinline__ MxBytes mx_codes_to_bytes(uint32_t w, const MxTables& tb) {
     const uint32_t wn = w ^ 0x88888888u;
     MxBytes r;
-    r.pos_lo = prmt(kPos0, kPos1, w);
-    r.neg_lo = prmt(kNeg0, kNeg1, wn);
-    r.pos_hi = prmt(kPos0, kPos1, w >> 16);
-    r.neg_hi = prmt(kNeg0, kNeg1, wn >> 16);
+    r.pos_lo = prmt(tb.pos0, tb.pos1, w);
+    r.neg_lo = prmt(tb.neg0, tb.neg1, wn);
+    r.pos_hi = prmt(tb.pos0, tb.pos1, w >> 16);
+    r.neg_hi = prmt(tb.neg0, tb.neg1, wn >> 16);
     return r;
 }
 
@@ -334,6 +345,7 @@ __device__ __forceinline__ void imma(int (&d)[4], uint32_t a0, uint32_t a1, uint
 struct LaneConst {
     int k_first;       // weight of the first column relative to the second (256 or 1)
     float w_unit;      // factor on `unit` (0 when the lane's token does not exist)
+    MxTables mx;       // MXFP4 only: the element look-up tables
 };
 
 // acc[row][.] += d * unit * (sum_k q_k X_k) + m * (sum_k x_k), fp32 (Eq. 3 applied per group).
@@ -360,7 +372,7 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][Mo
             const uint32_t w0 = t.c[2 * h], w1 = t.c[2 * h + 1];
             int d[4];
             if (kMx) {
-                const MxBytes m0 = mx_codes_to_bytes(w0), m1 = mx_codes_to_bytes(w1);  // lo: k 0..3, hi: k 4..7
+                const MxBytes m0 = mx_codes_to_bytes(w0, lc.mx), m1 = mx_codes_to_bytes(w1, lc.mx);  // lo: k 0..3, hi: k 4..7
                 imma<true>(d, m0.pos_lo, m1.pos_lo, m0.pos_hi, m1.pos_hi, t.b[0], t.b[1]);
                 imma_acc<true>(d, m0.neg_lo, m1.neg_lo, m0.neg_hi, m1.neg_hi, t.b[0], t.b[1]);
             } else {
@@ -391,7 +403,7 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][Mo
         int d2[4], d1[4], d0[4];
         if (kMx) {
             // three planes share the A operand: merging the two answers (four ORs) is cheaper than six more MMAs
-            const MxBytes m0 = mx_codes_to_bytes(w0), m1 = mx_codes_to_bytes(w1);  // lo: k 0..3, hi: k 4..7
+            const MxBytes m0 = mx_codes_to_bytes(w0, lc.mx), m1 = mx_codes_to_bytes(w1, lc.mx);  // lo: k 0..3, hi: k 4..7
             const uint32_t e0 = m0.pos_lo | m0.neg_lo, o0 = m0.pos_hi | m0.neg_hi;
             const uint32_t e1 = m1.pos_lo | m1.neg_lo, o1 = m1.pos_hi | m1.neg_hi;
             imma<true>(d2, e0, e1, o0, o1, t.b[0], t.b[1]);
@@ -557,7 +569,7 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         // stored).  Column modes: column g is plane 2 - g%4 of token g/4 (zeros for g%4 == 3 and for a token that
         // does not exist); this lane accumulates the columns of token q/2.
         LaneAddr la;
-        LaneConst lc;
+        LaneConst lc{};
         la.xs = xs;
         la.x_stride = (uint32_t)M * 128u;
         {
@@ -570,6 +582,7 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             const int tok_d = q >> 1;
             la.sc_off = (uint32_t)((tok_d < M ? tok_d : 0) * 128 + 96);
             lc.w_unit = (tok_d < M ? ((q & 1) ? 1.f : 256.f) : 0.f) * (F::kMx ? 0.5f : 1.f);
+            if (F::kMx) lc.mx = mx_tables();
         }
         float acc_m[MT::kAccM];  // column modes: offset term of row `lane`, per token
 #pragma unroll
