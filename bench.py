@@ -545,6 +545,64 @@ def run_ours(args, rank, local_rank, world):
         fd.fdqp_destroy(pctx)
         del px, py
 
+    # ---- next steps beside the projection: decode attention over a KV cache, and the format variants of the container
+    attention = None
+    formats = None
+    if rank == 0 and not args.no_head:
+        H, G, d, L = 8, 4, 256, 32768          # Gemma3-4B heads at a 32k context
+        ncache = max(1, int(np.ceil(4 * L2_BYTES / (2 * G * L * d * 2))))
+        gen = torch.Generator(device="cuda").manual_seed(2)
+        caches = [(torch.randn((G, L, d), device="cuda", generator=gen).to(torch.bfloat16),
+                   torch.randn((G, L, d), device="cuda", generator=gen).to(torch.bfloat16)) for _ in range(ncache)]
+        aq = torch.randn((H, d), device="cuda", generator=gen).to(torch.bfloat16)
+        ao = torch.empty((H, d), dtype=torch.float32, device="cuda")
+        attention = {"workload": f"Gemma3-4B decode attention, H={H} G={G} d={d}, L={L}", "bound": "hbm"}
+        for name, window in (("global", 0), ("window_1024", 1024)):
+            reps = 20
+            ga = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(stream):
+                for i in range(3):
+                    fd.fdqp_flowkv_decode(ctx, aq, caches[i % ncache][0], caches[i % ncache][1], ao, H, G, d, L, L, window,
+                                          d ** -0.5, sraw)
+            stream.synchronize()
+            with torch.cuda.graph(ga, stream=stream):
+                for i in range(reps):
+                    fd.fdqp_flowkv_decode(ctx, aq, caches[i % ncache][0], caches[i % ncache][1], ao, H, G, d, L, L, window,
+                                          d ** -0.5, sraw)
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(stream):
+                ga.replay()
+                a0.record(stream)
+                ga.replay()
+                a1.record(stream)
+            stream.synchronize()
+            us = a0.elapsed_time(a1) * 1e3 / reps
+            n_att = window if window else L
+            a_gbs = 2.0 * G * n_att * d * 2 / us / 1e3
+            attention[name] = {"us": us, "gbs": a_gbs, "frac": a_gbs / peaks["hbm_gbs"]}
+            del ga
+        del caches
+        formats = {"workload": f"LM head K={hk} N={hn} at M=1, bytes of the format's own container"}
+        for name, fmt in (("g64", fd.FMT_G64), ("g128", fd.FMT_G128), ("mxfp4", fd.FMT_MXFP4)):
+            fw = synthgen.weights_fmt(hseed, hk, 4096, fmt)
+            tile = fd.q4nx_pack_fmt(fmt, fw.codes, fw.scales, fw.offsets)
+            nbytes = fd.q4nx_packed_bytes_fmt(fmt, hk, hn)
+            fW = torch.from_numpy(np.tile(tile, hn // 4096)[:nbytes].copy()).cuda()
+            for _ in range(3):
+                fd.fdqp_run_fmt(ctx, fmt, hx, fW, hy, 1, hk, hn, sraw)
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            f0.record(stream)
+            for _ in range(10):
+                fd.fdqp_run_fmt(ctx, fmt, hx, fW, hy, 1, hk, hn, sraw)
+            f1.record(stream)
+            stream.synchronize()
+            f_ms = f0.elapsed_time(f1) / 10
+            f_gbs = (nbytes + 2 * hk + 4 * hn) / (f_ms * 1e-3) / 1e9
+            formats[name] = {"ms": f_ms, "gbs": f_gbs, "frac": f_gbs / peaks["hbm_gbs"]}
+            del fW
+        if fd.fdqp_last_status(ctx) != 0:
+            raise SystemExit("bench.py: a kernel reported " + fd.fdqp_status_string(fd.fdqp_last_status(ctx)))
+
     # ---- CPU baseline: the oracle on the host cores, one pass over the same layer (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -588,6 +646,8 @@ def run_ours(args, rank, local_rank, world):
                          "kernel": "fdqp_gemv_kernel", "launch_us": per_launch_us},
             "batched_decode": batch8,
             "prefill_lm_head": prefill,
+            "decode_attention": attention,
+            "format_variants": formats,
             "cpu_baseline": cpu,
             "e2e": {"value": whole_job_gbs(step_bytes, e2e_steps, world, e2e_s * 1e3), "unit": "GB/s",
                     "h2d_bytes_per_step": sum(2 * M * K for _, K, _, _ in shapes),
