@@ -190,7 +190,7 @@ def run_shape(args):
     packed_bytes = fd.q4nx_packed_bytes_fmt(fmt, K, N)
     packed = np.tile(tile, -(-N // nb))[:packed_bytes]
     base = torch.from_numpy(np.ascontiguousarray(packed)).cuda()
-    ncopies = max(1, int(np.ceil(4 * L2_BYTES / base.numel()))) if not args.same_weights else 1
+    ncopies = max(1, int(np.ceil(4 * L2_BYTES / base.numel()))) if not (args.same_weights or args.l2_resident) else 1
     copies = [base] + [base.clone() for _ in range(ncopies - 1)]
     x = torch.from_numpy(synthgen.activations(1, M, K).view(np.int16)).cuda()
     epi = {"none": fd.EPI_NONE, "bf16": fd.EPI_BF16, "geglu": fd.EPI_GEGLU_BF16}[args.epilogue]
@@ -678,6 +678,8 @@ def main():
                     help="with --shape: fused store-side epilogue (geglu: gate and up rows interleaved 16 by 16 along N)")
     ap.add_argument("--format", default="q4nx", choices=["q4nx", "g64", "g128", "mxfp4"],
                     help="with --shape: format variant of the block container (group 64 / 128, MXFP4)")
+    ap.add_argument("--l2-resident", action="store_true",
+                    help="with --shape: one weight copy, graph-replayed (what a call costs when its weights are already in L2)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-head", action="store_true", help="skip the LM-head timing")
     args = ap.parse_args()

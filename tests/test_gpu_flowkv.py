@@ -47,6 +47,7 @@ CASES = [
     (8, 4, 256, 65, 0, 70), (8, 4, 256, 1000, 0, 1024), (8, 4, 256, 4113, 0, 4200), (8, 4, 256, 5000, 1024, 5000),
     (8, 4, 256, 700, 1024, 800), (8, 4, 256, 2049, 1, 2100),
     (32, 16, 128, 777, 0, 800), (16, 2, 128, 3001, 512, 3001), (4, 4, 256, 300, 0, 300), (8, 1, 128, 129, 0, 129),
+    (12, 4, 256, 2500, 0, 2500), (6, 1, 128, 9000, 0, 9000), (20, 4, 128, 1500, 700, 1600), (7, 1, 256, 333, 0, 400),
 ]
 
 
