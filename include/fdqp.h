@@ -285,11 +285,11 @@ FDQP_API fdqp_status fdqp_dequant(fdqp_ctx* ctx, const void* W_q4nx, void* out, 
 /* fdqp_run and fdqp_dequant for a matrix packed in `format` (fdqp_format).  Same
  * arguments, results, acceptance bound (dequantised values bit-exact; y within
  * 2e-3 * sum_k |x_k w_hat_k| + 1e-5 of the fp64 product), asynchrony and errors as
- * fdqp_run / fdqp_dequant; FDQP_FMT_Q4NX is exactly those calls.  The variants run
- * on the streaming GEMV kernels for every M (rows beyond eight in further launches
- * of eight); there is no tensor-core path for them.  In the projection an MXFP4
- * scale byte of 0 (2^-127, below 1e-38) counts as a scale of zero; the
- * dequantisation engine returns it exactly.  FDQP_ERR_ARG for an unknown
+ * fdqp_run / fdqp_dequant; FDQP_FMT_Q4NX is exactly those calls.  Dispatch on M as
+ * in fdqp_run: the streaming GEMV kernels up to eight token rows, the tensor-core
+ * kernels (which dequantise the format into shared memory) above.  In the GEMV
+ * kernels an MXFP4 scale byte of 0 (2^-127, below 1e-38) counts as a scale of zero;
+ * the tensor-core kernels and the dequantisation engine use it exactly.  FDQP_ERR_ARG for an unknown
  * format, FDQP_ERR_SHAPE when K is not a multiple of 256. */
 FDQP_API fdqp_status fdqp_run_fmt(fdqp_ctx* ctx, int format, const void* x_bf16, const void* W_packed, float* y, int64_t M,
                          int64_t K, int64_t N, void* cuda_stream);

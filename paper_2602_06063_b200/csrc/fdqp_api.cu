@@ -23,7 +23,7 @@ cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, in
 cudaError_t dequant_fmt_launch(int fmt, const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
 cudaError_t prefill_set_smem_limit();
 cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, uint16_t* y16, int epi, float* ws,
-                           int* status, int M, int K, int N, int pair, int Z, cudaStream_t stream);
+                           int* status, int M, int K, int N, int pair, int Z, int fmt, cudaStream_t stream);
 cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* gamma, float eps, uint16_t* out, int M, int K,
                            cudaStream_t stream);
 cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* V, float* out, float* ws, int max_splits, int H,
@@ -396,7 +396,7 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
         ctx->launches += 1;
         return FDQP_OK;
     }
-    if (fmt == kFmtQ4nx && use_prefill(ctx, M, K, N)) {
+    if (use_prefill(ctx, M, K, N)) {
         // prefill-sized M: dequantise into shared memory, contract with tcgen05 (accumulators in TMEM)
         const uint16_t* xt = x;
         int64_t x_row_bytes = K * 2;
@@ -408,7 +408,7 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
             xt = reinterpret_cast<const uint16_t*>(ctx->x_spread);
         }
         if ((e = prefill_launch(W, xt, x_row_bytes, y, y16, epi, ctx->pf_ws, ctx->status_dev, (int)M, (int)K, (int)N,
-                                use_pair(ctx, M) ? 1 : 0, prefill_slices(ctx, M, K, N), stream)))
+                                use_pair(ctx, M) ? 1 : 0, prefill_slices(ctx, M, K, N), fmt, stream)))
             return cuda_fail(ctx, e, "prefill kernel launch");
         ctx->launches += prefill_slices(ctx, M, K, N) > 1 ? 2 : 1;
         return FDQP_OK;

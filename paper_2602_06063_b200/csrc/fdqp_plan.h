@@ -11,11 +11,11 @@ constexpr int kBlockK = 256;        // input features per full Q4NX block
 constexpr int kBlockBytes = 5120;   // bytes of a full block (Sec. "Dequantization Engine")
 constexpr int kGroupBytes = 640;    // bytes a block spends per group: 512 codes + 64 scales + 64 offsets
 constexpr int kMaxTokens = 8;       // token rows one GEMV launch handles
-// Up to this many tokens the GEMV lays the byte planes of a token out as MMA columns; above it, one MMA per plane.
 // What a kernel writes for a finished output value (values of fdqp_epilogue in fdqp.h).
 constexpr int kEpiNone = 0;       // fp32 y [M][N]
 constexpr int kEpiBf16 = 1;       // bf16 y [M][N]
 constexpr int kEpiGegluBf16 = 2;  // bf16 [M][N/2]: gelu(row r) * (row r + 16) of every 32-row strip
+// Up to this many tokens the GEMV lays the byte planes of a token out as MMA columns; above it, one MMA per plane.
 constexpr int kColsMaxTokens = 2;
 // Column modes hand three partial terms per (row, token) to the reducer (two column halves + the offset term).
 constexpr int kColsPartTerms = 3;
@@ -27,13 +27,12 @@ struct GemvPlan {
     const uint16_t* x;    // device, [M][K] bf16 bits
     const uint32_t* xq;   // device, prepared activations: 32-byte records [K/32][M][4] (see fdqp_xprep_kernel)
     const float* xsc;     // device, per-group {sum x, unit} by token: [K/32][8][2]
-    float* y;            // fp32 output (epilogue kEpiNone)
-    uint16_t* y16;       // bf16 output (other epilogues)
+    float* y;             // device, fp32 output [M][N] (epilogue kEpiNone)
+    uint16_t* y16;        // device, bf16 output (other epilogues)
     int epi;
     const uint16_t* gamma;  // RMS normalisation of x fused into the in-kernel activation preparation (norm != 0):
     float eps;              //   x <- bf16(x * rsqrt(mean(x^2) + eps) * (1 + gamma)), per token row
     int norm;
-            // device, [M][N]
     float* ws_edge;       // device, [grid][2][32*kMaxTokens] partial sums of strips shared between CTAs
     float* ws_full;       // device, [Z][S][32*kMaxTokens] partial sums of whole strip-slices (Z > 1)
     int* tickets;         // device, [S] arrival counters, zero between launches

@@ -20,6 +20,7 @@
 #include <cuda.h>
 
 #include "fdqp_device.cuh"
+#include "fdqp_format.h"
 #include "fdqp_plan.h"
 
 namespace fdqp {
@@ -118,19 +119,38 @@ __device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&r)[32]
 
 struct GroupRegs {
     uint4 codes;      // this lane's row: 32 codes of the group
-    uint32_t d_bits;  // bf16 scale in the low half
+    uint32_t d_bits;  // bf16 scale in the low half (MXFP4: the E8M0 scale byte)
     uint32_t m_bits;  // bf16 offset in the low half
     bool valid;
 };
 
+// g counts 32-column tiles along K; the format variants (whole blocks only) keep the tile's scale and offset at the
+// index of the larger group it belongs to.
+template <int FMT>
 __device__ __forceinline__ GroupRegs group_load(const uint8_t* __restrict__ W, int K, int64_t strip, int g, int lane,
                                                 bool strip_ok) {
+    using F = FmtTraits<FMT>;
     GroupRegs r;
     const int groups = K / kGroup;
     r.valid = strip_ok && g < groups;
     r.codes = make_uint4(0, 0, 0, 0);
     r.d_bits = 0;
     r.m_bits = 0;
+    if (FMT != kFmtQ4nx) {
+        if (r.valid) {
+            const int b = g >> 3, t = g & 7;
+            const uint8_t* blk = W + (strip * (int64_t)(K / kBlockK) + b) * (int64_t)F::kBlock;
+            r.codes = __ldg(reinterpret_cast<const uint4*>(blk + t * 512 + lane * 16));
+            if (F::kMx) {
+                r.d_bits = __ldg(blk + kCodeBytes + t * 32 + lane);
+            } else {
+                const int at = 2 * ((t >> F::kShift) * 32 + lane);
+                r.d_bits = __ldg(reinterpret_cast<const unsigned short*>(blk + kCodeBytes + at));
+                r.m_bits = __ldg(reinterpret_cast<const unsigned short*>(blk + F::kOffSect + at));
+            }
+        }
+        return r;
+    }
     if (r.valid) {
         const int b = g >> 3, t = g & 7;
         const int rest = groups - 8 * b;
@@ -164,12 +184,50 @@ __device__ __forceinline__ float dequant_hi(uint32_t q2, uint32_t d_bits, float 
 // Codes become bf16 pairs with one logic op per pair ((w >> 4i) & 0x000F000F | 0x43004300 = (128+q_i, 128+q_{i+4}));
 // the bias is removed exactly by a packed bf16 subtract; no integer-to-float conversion instruction is used.
 // An absent group arrives with codes, d and m all zero and therefore writes zeros.
+//
+// MXFP4: every element times its power-of-two scale is a bf16 number, so the tile is exact.  Eight E2M1 codes become
+// bf16 through two byte tables (high and low byte of the magnitude's bf16 pattern, indexed by the code's low three bits
+// with one permute per four codes each), the sign bits are moved to bit 7 of the high bytes by one more permute, the
+// bytes are interleaved into bf16 pairs, and a packed bf16 multiply applies the scale 2^(e-127) (bf16 bits e << 7).
+__device__ __forceinline__ uint32_t pf_prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+template <int FMT>
 __device__ __forceinline__ void group_store(uint32_t a_tile, const GroupRegs& r, int strip_local, int gl, int lane) {
     const int row = strip_local * 32 + lane;
     const uint32_t row_base = a_tile + (uint32_t)((row >> 3) * 1024 + (row & 7) * 128);
     const uint32_t r7s = (uint32_t)(row & 7) << 4;
-    const float m = __uint_as_float(r.m_bits << 16);
     const uint32_t words[4] = {r.codes.x, r.codes.y, r.codes.z, r.codes.w};
+    if (FmtTraits<FMT>::kMx) {
+        constexpr uint32_t kHi0 = 0x3F3F3F00u, kHi1 = 0x40404040u;  // bf16 of 0, .5, 1, 1.5 | 2, 3, 4, 6: high bytes
+        constexpr uint32_t kLo0 = 0xC0800000u, kLo1 = 0xC0804000u;  //                                     low bytes
+        const uint32_t e = r.valid ? r.d_bits : 127u;               // an absent group has zero codes: any scale does
+        const uint32_t sc = e ? e << 7 : 0x0040u;                   // bf16 bits of 2^(e-127)
+        const uint32_t sc2 = sc | (sc << 16);
+#pragma unroll
+        for (int wi = 0; wi < 4; ++wi) {  // 8 codes -> one 16-byte chunk
+            const uint32_t w = words[wi];
+            const uint32_t mag = w & 0x77777777u, w4 = w << 4;
+            uint32_t hi_a = pf_prmt(kHi0, kHi1, mag), lo_a = pf_prmt(kLo0, kLo1, mag);              // codes 0..3
+            uint32_t hi_b = pf_prmt(kHi0, kHi1, mag >> 16), lo_b = pf_prmt(kLo0, kLo1, mag >> 16);  // codes 4..7
+            hi_a |= pf_prmt(w, w4, 0x1504u) & 0x80808080u;  // signs: bit 3 of nibble j -> bit 7 of byte j
+            hi_b |= pf_prmt(w, w4, 0x3726u) & 0x80808080u;
+            uint32_t o0 = pf_prmt(lo_a, hi_a, 0x5140u), o1 = pf_prmt(lo_a, hi_a, 0x7362u);
+            uint32_t o2 = pf_prmt(lo_b, hi_b, 0x5140u), o3 = pf_prmt(lo_b, hi_b, 0x7362u);
+            asm("mul.rn.bf16x2 %0, %0, %1;" : "+r"(o0) : "r"(sc2));
+            asm("mul.rn.bf16x2 %0, %0, %1;" : "+r"(o1) : "r"(sc2));
+            asm("mul.rn.bf16x2 %0, %0, %1;" : "+r"(o2) : "r"(sc2));
+            asm("mul.rn.bf16x2 %0, %0, %1;" : "+r"(o3) : "r"(sc2));
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(row_base + (((uint32_t)(gl * 4 + wi) << 4) ^ r7s)),
+                         "r"(o0), "r"(o1), "r"(o2), "r"(o3)
+                         : "memory");
+        }
+        return;
+    }
+    const float m = __uint_as_float(r.m_bits << 16);
 #pragma unroll
     for (int wi = 0; wi < 4; ++wi) {  // 8 codes -> one 16-byte chunk
         const uint32_t w = words[wi];
@@ -217,6 +275,7 @@ __device__ __forceinline__ void stage_copy_out(uint32_t stage, uint16_t* dst, in
 
 // ---- the kernel -------------------------------------------------------------------------------------------------------
 
+template <int FMT>
 __global__ void __launch_bounds__(kPf1Threads, 1)
     fdqp_prefill_kernel(const __grid_constant__ CUtensorMap x_map, const PrefillParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -309,15 +368,15 @@ __global__ void __launch_bounds__(kPf1Threads, 1)
         // the loads of the next three stages are in flight while this one is converted (a stage lasts about as long
         // as one trip to HBM); groups past K load as zeros
         const int gbase = 2 * ks0 + gl;  // this warp's group in k-step i of the slice: gbase + 2 i
-        GroupRegs g0 = group_load(p.W, p.K, strip, gbase, lane, strip_ok);
-        GroupRegs g1 = group_load(p.W, p.K, strip, gbase + 2, lane, strip_ok);
-        GroupRegs g2 = group_load(p.W, p.K, strip, gbase + 4, lane, strip_ok);
+        GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase, lane, strip_ok);
+        GroupRegs g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2, lane, strip_ok);
+        GroupRegs g2 = group_load<FMT>(p.W, p.K, strip, gbase + 4, lane, strip_ok);
         for (int i = 0; i < ksteps && ok; ++i) {
             const int s = i % kPfStages;
-            const GroupRegs g3 = group_load(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
+            const GroupRegs g3 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
             if (i >= kPfStages) ok = mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status);
             if (!ok) break;
-            group_store(base + s * kPfStageBytes, g0, sl, gl, lane);
+            group_store<FMT>(base + s * kPfStageBytes, g0, sl, gl, lane);
             // make the generic-proxy stores visible to the tensor core's (async-proxy) reads, then signal
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
@@ -493,6 +552,7 @@ __device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap* ma
         : "memory");
 }
 
+template <int FMT>
 __global__ void __launch_bounds__(kPfThreads, 1)
     fdqp_prefill_pair_kernel(const __grid_constant__ CUtensorMap x_map, const PrefillParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -599,16 +659,16 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         // software pipeline: the loads of the next three stages are in flight while this one is converted (a stage
         // lasts well under a microsecond here, less than one trip to L2 / HBM); groups past K load as zeros
         const int gbase = 2 * ks0 + gl;  // this warp's group in k-step i of the slice: gbase + 2 i
-        GroupRegs g0 = group_load(p.W, p.K, strip, gbase, lane, strip_ok);
-        GroupRegs g1 = group_load(p.W, p.K, strip, gbase + 2, lane, strip_ok);
-        GroupRegs g2 = group_load(p.W, p.K, strip, gbase + 4, lane, strip_ok);
+        GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase, lane, strip_ok);
+        GroupRegs g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2, lane, strip_ok);
+        GroupRegs g2 = group_load<FMT>(p.W, p.K, strip, gbase + 4, lane, strip_ok);
         const uint32_t full_a0 = mapa_shared(full_a(0), 0);
         for (int i = 0; i < ksteps && ok; ++i) {
             const int s = i % kP2Stages;
-            const GroupRegs g3 = group_load(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
+            const GroupRegs g3 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
             if (i >= kP2Stages) ok = mbar_wait(empty(s), ((i / kP2Stages) - 1) & 1, p.status);
             if (!ok) break;
-            group_store(base + s * kP2StageBytes, g0, sl, gl, lane);
+            group_store<FMT>(base + s * kP2StageBytes, g0, sl, gl, lane);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(full_a0 + 8u * s);
@@ -734,10 +794,43 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-cudaError_t prefill_set_smem_limit() {
-    cudaError_t e = cudaFuncSetAttribute(fdqp_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPfSmemBytes);
+template <int FMT>
+static cudaError_t prefill_set_smem_limit_fmt() {
+    cudaError_t e = cudaFuncSetAttribute(fdqp_prefill_kernel<FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPfSmemBytes);
     if (e) return e;
-    return cudaFuncSetAttribute(fdqp_prefill_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kP2SmemBytes);
+    return cudaFuncSetAttribute(fdqp_prefill_pair_kernel<FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kP2SmemBytes);
+}
+
+cudaError_t prefill_set_smem_limit() {
+    cudaError_t e;
+    if ((e = prefill_set_smem_limit_fmt<kFmtQ4nx>())) return e;
+    if ((e = prefill_set_smem_limit_fmt<kFmtG64>())) return e;
+    if ((e = prefill_set_smem_limit_fmt<kFmtG128>())) return e;
+    return prefill_set_smem_limit_fmt<kFmtMxfp4>();
+}
+
+template <int FMT>
+static cudaError_t prefill_launch_kernels(const CUtensorMap& map, const PrefillParams& p, int pair, int M, int N, int Z,
+                                          cudaStream_t stream) {
+    if (pair) {
+        const int n_tiles = (N + 2 * kP2Rows - 1) / (2 * kP2Rows), tok_tiles = (M + kP2Toks - 1) / kP2Toks;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(2 * n_tiles * tok_tiles * Z));
+        cfg.blockDim = dim3((unsigned)kPfThreads);
+        cfg.dynamicSmemBytes = kP2SmemBytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, fdqp_prefill_pair_kernel<FMT>, map, p);
+    }
+    const int n_tiles = (N + kPfRows - 1) / kPfRows, tok_tiles = (M + kPfToks - 1) / kPfToks;
+    fdqp_prefill_kernel<FMT><<<n_tiles * tok_tiles * Z, kPf1Threads, kPfSmemBytes, stream>>>(map, p);
+    return cudaGetLastError();
 }
 
 // x: [M][K] bf16 row-major (device).  Returns cudaErrorNotSupported if the tensor map cannot be built.
@@ -746,8 +839,9 @@ cudaError_t prefill_set_smem_limit() {
 // second kernel adds them in slice order into y.  For shapes with too few tiles to fill the GPU.
 // x_row_bytes: distance between token rows of x (K * 2 for a dense [M][K] array; a multiple of 16).
 // epi: kEpiNone writes fp32 y; the other epilogues write bf16 to y16 (see fdqp_plan.h).
+// fmt: the container's format (fdqp_format.h).
 cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, uint16_t* y16, int epi, float* ws,
-                           int* status, int M, int K, int N, int pair, int Z, cudaStream_t stream) {
+                           int* status, int M, int K, int N, int pair, int Z, int fmt, cudaStream_t stream) {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     CUtensorMap map;
@@ -774,25 +868,12 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_by
     p.Z = (ksteps_all + p.ksteps_z - 1) / p.ksteps_z;  // no empty slice
     Z = p.Z;
     cudaError_t err;
-    if (pair) {
-        const int n_tiles = (N + 2 * kP2Rows - 1) / (2 * kP2Rows), tok_tiles = (M + kP2Toks - 1) / kP2Toks;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(2 * n_tiles * tok_tiles * Z));
-        cfg.blockDim = dim3((unsigned)kPfThreads);
-        cfg.dynamicSmemBytes = kP2SmemBytes;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        err = cudaLaunchKernelEx(&cfg, fdqp_prefill_pair_kernel, map, p);
-    } else {
-        const int n_tiles = (N + kPfRows - 1) / kPfRows, tok_tiles = (M + kPfToks - 1) / kPfToks;
-        fdqp_prefill_kernel<<<n_tiles * tok_tiles * Z, kPf1Threads, kPfSmemBytes, stream>>>(map, p);
-        err = cudaGetLastError();
+    switch (fmt) {
+        case kFmtQ4nx: err = prefill_launch_kernels<kFmtQ4nx>(map, p, pair, M, N, Z, stream); break;
+        case kFmtG64: err = prefill_launch_kernels<kFmtG64>(map, p, pair, M, N, Z, stream); break;
+        case kFmtG128: err = prefill_launch_kernels<kFmtG128>(map, p, pair, M, N, Z, stream); break;
+        case kFmtMxfp4: err = prefill_launch_kernels<kFmtMxfp4>(map, p, pair, M, N, Z, stream); break;
+        default: return cudaErrorInvalidValue;
     }
     if (err != cudaSuccess || Z == 1) return err;
     if (epi != kEpiNone) {

@@ -94,6 +94,49 @@ def test_projection_matches_oracle(ctx, fmt, K, N, M):
         assert_close(y[:, N - 256:], y_ref, a_ref, f"{NAMES[fmt]} K={K} N={N} M={M} tail")
 
 
+# Prefill-sized token counts: the tensor-core kernels (one-SM tile up to 256 tokens, SM pairs above; K slices when the
+# tiles are few), which dequantise the format into shared memory.
+PREFILL_SHAPES = [(2560, 4096, 64), (2560, 2048, 300), (3840, 1024, 130), (21504, 320, 40), (1280, 6912, 512), (512, 288, 17)]
+
+
+@pytest.mark.parametrize("fmt", FMTS, ids=lambda f: NAMES[f])
+@pytest.mark.parametrize("K,N,M", PREFILL_SHAPES)
+def test_prefill_sized_projection_matches_oracle(ctx, fmt, K, N, M):
+    amp = 1.0 / np.sqrt(K) if K > 20000 else 1.0
+    c = FmtCase(fmt, K, N, M, 9000 + K + N + M + fmt, amp)
+    fd.fdqp_set_param(ctx, "path", 3)       # the tensor-core kernels whatever the dispatch model would choose
+    try:
+        y = c.run(ctx)
+    finally:
+        fd.fdqp_set_param(ctx, "path", 0)
+    n1 = min(N, 512)
+    y_ref, a_ref = c.reference(0, n1)
+    assert_close(y[:, :n1], y_ref, a_ref, f"{NAMES[fmt]} prefill K={K} N={N} M={M}")
+    if N > n1:
+        y_ref, a_ref = c.reference(N - 128, N)
+        assert_close(y[:, N - 128:], y_ref, a_ref, f"{NAMES[fmt]} prefill K={K} N={N} M={M} tail")
+
+
+def test_mxfp4_prefill_is_exact_on_exact_inputs(ctx):
+    """MXFP4 weights are bf16 numbers, so with small integer activations the tensor-core result is the oracle's."""
+    K, N, M = 1024, 512, 96
+    fmt = fd.FMT_MXFP4
+    w = synthgen.weights_fmt(91, K, N, fmt)
+    r = synthgen.u64(92, 3, w.scales.size).reshape(w.scales.shape)
+    w.scales[:, :] = (124 + r % np.uint64(3)).astype(np.uint16)
+    xi = (synthgen.u64(93, 4, M * K).reshape(M, K) % np.uint64(5)).astype(np.float32) - 2.0
+    c = FmtCase(fmt, K, N, M, 0, weights=w)
+    c.x = synthgen.bf16_bits(xi)
+    c.x_dev = dev_bytes(c.x)
+    fd.fdqp_set_param(ctx, "path", 3)
+    try:
+        y = c.run(ctx)
+    finally:
+        fd.fdqp_set_param(ctx, "path", 0)
+    y_ref, _ = c.reference()
+    assert np.array_equal(y.astype(np.float64), y_ref)
+
+
 @pytest.mark.parametrize("fmt", FMTS, ids=lambda f: NAMES[f])
 @pytest.mark.parametrize("M", [1, 2, 6])
 def test_exact_arithmetic_cases_are_bit_equal(ctx, fmt, M):
