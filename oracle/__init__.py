@@ -56,6 +56,8 @@ def _load():
         lib.oracle_geglu.argtypes = [p, i64, i64, p, p]
         lib.oracle_rmsnorm.restype = ci
         lib.oracle_rmsnorm.argtypes = [p, p, ctypes.c_double, i64, i64, p]
+        lib.oracle_add_residual.restype = ci
+        lib.oracle_add_residual.argtypes = [p, p, i64, i64, p]
         lib.oracle_decode_attention.restype = ci
         lib.oracle_decode_attention.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, ctypes.c_double, p, p]
         lib.oracle_fmt_packed_bytes.restype = ctypes.c_size_t
@@ -189,6 +191,19 @@ def rmsnorm(x_bf16, gamma_bf16, eps: float):
     if rc != 0:
         raise ValueError(f"oracle_rmsnorm failed ({rc})")
     return out
+
+
+def add_residual(x_bf16, r_bf16):
+    """The residual stream ahead of a normalisation: bf16(x + r), one rounding (bf16 bits in, bf16 bits out)."""
+    x_bf16 = _c(x_bf16, np.uint16)
+    r_bf16 = _c(r_bf16, np.uint16)
+    if x_bf16.shape != r_bf16.shape or x_bf16.ndim != 2:
+        raise ValueError("x and r must be [M, K]")
+    h = np.empty_like(x_bf16)
+    rc = _load().oracle_add_residual(_ptr(x_bf16), _ptr(r_bf16), x_bf16.shape[0], x_bf16.shape[1], _ptr(h))
+    if rc != 0:
+        raise ValueError(f"oracle_add_residual failed ({rc})")
+    return h
 
 
 def decode_attention(q, K, V, L: int, window: int = 0, scale: float = 1.0):

@@ -40,6 +40,8 @@
  * RMS normalisation prologue and gated GELU epilogue (next steps beyond the paper's FusedDQP, which leaves both to
  * separate kernels): oracle_rmsnorm, oracle_gelu_tanh / oracle_geglu below; pinned by closed-form rows, invariances,
  * the error-function form, symmetry, limits and a pairing case with exact products.
+ * The residual addition that precedes a normalisation in a decoder layer: oracle_add_residual, bf16(x + r) rounded
+ * once from the exact sum; pinned by hand tie cases and by exact rational sums of random pairs.
  * Decode attention over a KV cache (the paper's second decode kernel, FlowKV, computes it chunk by chunk):
  * oracle_decode_attention is the plain softmax-weighted sum; pinned by closed forms and invariances.
  *
@@ -282,6 +284,39 @@ int oracle_rmsnorm(const uint16_t *x_bf16, const uint16_t *gamma_bf16, double ep
             out_bf16[m * K + k] = fp32_to_bf16_rne((float)v);
         }
     }
+    return 0;
+}
+
+/* ---- residual addition ahead of the normalisation (next-step prologue) -------------------------------------------- */
+
+/* h[m][k] = bf16( x[m][k] + r[m][k] ): the residual stream of a decoder layer, kept in bf16 as every activation in the
+ * paper; the sum of two bf16 numbers is exact in double, so this is one rounding (to nearest, ties to even).  The
+ * normalisation that follows is oracle_rmsnorm on h. */
+static uint16_t double_to_bf16_rne(double v) {
+    /* v is a sum of two bf16 numbers: it has at most ~270 significant bits of span but, being a double already, is
+     * exact; round it to 8 significant bits by integer arithmetic on the scaled value */
+    if (v == 0.0) return (uint16_t)(signbit(v) ? 0x8000u : 0u);
+    if (isnan(v)) return 0x7fc0u;
+    if (isinf(v)) return (uint16_t)(v < 0 ? 0xff80u : 0x7f80u);
+    int e;
+    double m = frexp(fabs(v), &e); /* |v| = m 2^e, m in [0.5, 1) */
+    int ulp_exp = e - 8;           /* 8 significant bits */
+    if (ulp_exp < -133) ulp_exp = -133; /* bf16 subnormals: spacing 2^-133 */
+    double q = ldexp(fabs(v), -ulp_exp); /* exact */
+    double fl = floor(q), frac = q - fl;
+    if (frac > 0.5 || (frac == 0.5 && fmod(fl, 2.0) == 1.0)) fl += 1.0;
+    double r = ldexp(fl, ulp_exp);
+    float f = (float)(v < 0 ? -r : r); /* exact: 8 significant bits; overflow becomes infinity */
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    (void)m;
+    return (uint16_t)(u >> 16);
+}
+
+int oracle_add_residual(const uint16_t *x_bf16, const uint16_t *r_bf16, int64_t M, int64_t K, uint16_t *h_bf16) {
+    if (!x_bf16 || !r_bf16 || !h_bf16 || M < 1 || K < 1) return -1;
+    for (int64_t i = 0; i < M * K; ++i)
+        h_bf16[i] = double_to_bf16_rne(bf16_bits_to_double(x_bf16[i]) + bf16_bits_to_double(r_bf16[i]));
     return 0;
 }
 

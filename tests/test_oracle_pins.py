@@ -492,3 +492,55 @@ def test_decode_attention_closed_forms_and_invariances():
     Kd[:, 7, 1] = 8.0
     sel, _ = oracle.decode_attention(bf(big), bf(Kd), bf(V), L=L)
     assert np.allclose(sel[0], Vb[0, 7], rtol=0, atol=1e-12)
+
+
+def test_add_residual_is_one_rounding_of_the_exact_sum():
+    from fractions import Fraction
+
+    def bf(a):
+        return synthgen.bf16_bits(np.asarray(a, np.float32))
+
+    def frac(bits):
+        return Fraction(float(synthgen.bf16_to_f32(np.array([bits], np.uint16))[0]))
+
+    # hand cases: below half an ulp, a tie to the even neighbour below, a tie to the even neighbour above, cancellation
+    x = bf([[1.0, 1.0, 1.0078125, 3.0, -2.5, 0.0]])
+    r = bf([[2.0 ** -9, 2.0 ** -8, 2.0 ** -8, -3.0, 2.5, 0.0]])
+    h = synthgen.bf16_to_f32(oracle.add_residual(x, r))[0]
+    assert list(h) == [1.0, 1.0, 1.015625, 0.0, 0.0, 0.0]
+    # random pairs, wide exponent gaps and subnormals included: the nearest bf16 to the exact rational sum, found by
+    # comparing the neighbours of a truncated estimate
+    rng = np.random.default_rng(12)
+    n = 4000
+    xb = rng.integers(0, 1 << 16, n).astype(np.uint16)
+    rb = rng.integers(0, 1 << 16, n).astype(np.uint16)
+    expo = lambda b: (b >> 7) & 0xFF
+    keep = (expo(xb) != 255) & (expo(rb) != 255)
+    xb, rb = xb[keep], rb[keep]
+    rb[::3] = (xb[::3] & 0x8000) | np.clip((xb[::3] & 0x7FFF).astype(np.int32) + rng.integers(-300, 300, xb[::3].size), 0, 0x7F7F).astype(np.uint16)
+    got = oracle.add_residual(xb[None, :], rb[None, :])[0]
+    for a, b, g in zip(xb.tolist(), rb.tolist(), got.tolist()):
+        exact = frac(a) + frac(b)
+        if exact == 0:
+            assert g in (0, 0x8000)
+            continue
+        if abs(exact) >= Fraction(2) ** 128:      # beyond the largest finite value by more than half a step
+            assert g == (0xFF80 if exact < 0 else 0x7F80)
+            continue
+        sign = 0x8000 if exact < 0 else 0
+        mag = abs(exact)
+        est = int(np.array([float(mag)], np.float32).view(np.uint32)[0] >> 16)
+        best = None
+        for c in range(max(est - 2, 0), min(est + 3, 0x7F81)):
+            cv = frac(c) if c < 0x7F80 else Fraction(2) ** 128     # infinity stands in as the next step up
+            d = abs(cv - mag)
+            if best is None or d < best[0] or (d == best[0] and c % 2 == 0):
+                best = (d, c)
+        assert g == (sign | best[1]), (hex(a), hex(b), hex(g), hex(sign | best[1]))
+    # identities: adding zero changes nothing, the sum commutes, x + (-x) = 0
+    xs = synthgen.activations(5, 3, 64)
+    zero = np.zeros_like(xs)
+    assert np.array_equal(oracle.add_residual(xs, zero), xs)
+    ys = synthgen.activations(6, 3, 64)
+    assert np.array_equal(oracle.add_residual(xs, ys), oracle.add_residual(ys, xs))
+    assert not np.any(oracle.add_residual(xs, xs ^ 0x8000) & 0x7FFF)
