@@ -202,10 +202,14 @@ def run_shape(args):
     sraw = stream.cuda_stream
 
     gamma = torch.zeros(K, dtype=torch.int16, device="cuda")
+    resid = torch.from_numpy(synthgen.activations(2, M, K).view(np.int16)).cuda()
+    h_out = torch.empty((M, K), dtype=torch.int16, device="cuda")
 
     def launch(W):
         if fmt != fd.FMT_Q4NX:
             fd.fdqp_run_fmt(ctx, fmt, x, W, y, M, K, N, sraw)
+        elif args.rmsnorm and args.residual:
+            fd.fdqp_run_add_rmsnorm_epilogue(ctx, x, resid, h_out, gamma, 1e-6, W, y, epi, M, K, N, sraw)
         elif args.rmsnorm:
             fd.fdqp_run_rmsnorm_epilogue(ctx, x, gamma, 1e-6, W, y, epi, M, K, N, sraw)
         else:
@@ -680,6 +684,8 @@ def main():
                     help="with --shape: format variant of the block container (group 64 / 128, MXFP4)")
     ap.add_argument("--l2-resident", action="store_true",
                     help="with --shape: one weight copy, graph-replayed (what a call costs when its weights are already in L2)")
+    ap.add_argument("--residual", action="store_true",
+                    help="with --shape --rmsnorm: add a residual to x first and write the sum out (fdqp_run_add_rmsnorm_epilogue)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-head", action="store_true", help="skip the LM-head timing")
     args = ap.parse_args()

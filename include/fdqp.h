@@ -213,6 +213,22 @@ FDQP_API fdqp_status fdqp_run_rmsnorm_epilogue(fdqp_ctx* ctx, const void* x_bf16
                                       const void* W_q4nx, void* out, int epilogue, int64_t M, int64_t K, int64_t N,
                                       void* cuda_stream);
 
+/* fdqp_run_rmsnorm_epilogue with the residual addition that precedes the
+ * normalisation in a decoder layer (the paper pairs the two in its vector kernels):
+ *   h[m][k]   = bf16( x[m][k] + residual[m][k] )          one rounding of the exact sum
+ *   x_n[m][k] = bf16( h[m][k] * rsqrt(mean_k h[m][k]^2 + eps) * (1 + gamma[k]) )
+ *   out       = epilogue( x_n * dequant(W) )
+ *   residual_bf16  device, [M][K] bf16, 16-byte aligned
+ *   h_out_bf16     device, [M][K] bf16, 16-byte aligned, or null: receives h (the
+ *                  updated residual stream).  Must not be x or residual themselves:
+ *                  every CTA of the fused launch reads those (FDQP_ERR_ARG).
+ * Fused into the GEMV launch under the same condition as the normalisation alone
+ * (then the grid's first CTA stores h); otherwise the separate normalisation kernel
+ * does the addition.  Everything else as fdqp_run_rmsnorm_epilogue. */
+FDQP_API fdqp_status fdqp_run_add_rmsnorm_epilogue(fdqp_ctx* ctx, const void* x_bf16, const void* residual_bf16,
+                                          void* h_out_bf16, const void* gamma_bf16, float eps, const void* W_q4nx,
+                                          void* out, int epilogue, int64_t M, int64_t K, int64_t N, void* cuda_stream);
+
 /* Decode attention over a KV cache (the paper's FlowKV, and FlowKV-SWA for local
  * layers): the attention of ONE new token at decoding step L,
  *     out[h] = sum_j softmax_j( scale * q[h] . K[g][j] ) V[g][j],   g = h / (H / G),

@@ -26,7 +26,7 @@ EXPORTS = [
     "fdqp_run_host_async", "fdqp_run_epilogue", "fdqp_run_rmsnorm_epilogue", "fdqp_flowkv_decode",
     "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
     "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc", "q4nx_packed_bytes_fmt", "q4nx_pack_fmt",
-    "q4nx_unpack_fmt", "fdqp_run_fmt", "fdqp_dequant_fmt",
+    "q4nx_unpack_fmt", "fdqp_run_fmt", "fdqp_dequant_fmt", "fdqp_run_add_rmsnorm_epilogue",
 ]
 
 
@@ -79,6 +79,8 @@ def load_library():
     lib.fdqp_run_epilogue.argtypes = [vp, vp, vp, vp, ci, i64, i64, i64, vp]
     lib.fdqp_run_rmsnorm_epilogue.restype = ci
     lib.fdqp_run_rmsnorm_epilogue.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp, ci, i64, i64, i64, vp]
+    lib.fdqp_run_add_rmsnorm_epilogue.restype = ci
+    lib.fdqp_run_add_rmsnorm_epilogue.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, ci, i64, i64, i64, vp]
     lib.fdqp_flowkv_decode.restype = ci
     lib.fdqp_flowkv_decode.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, ctypes.c_float, vp]
     lib.fdqp_run_host_async.restype = ci
@@ -203,6 +205,16 @@ def fdqp_run_rmsnorm_epilogue(ctx: int, x_bf16, gamma_bf16, eps: float, W_q4nx, 
     _check(load_library().fdqp_run_rmsnorm_epilogue(ctx, _addr(x_bf16), _addr(gamma_bf16), float(eps), _addr(W_q4nx),
                                                     _addr(out), int(epilogue), M, K, N, _stream(stream)),
            "fdqp_run_rmsnorm_epilogue", ctx)
+
+
+def fdqp_run_add_rmsnorm_epilogue(ctx: int, x_bf16, residual_bf16, h_out_bf16, gamma_bf16, eps: float, W_q4nx, out,
+                                  epilogue: int, M: int, K: int, N: int, stream=None) -> None:
+    """fdqp_run_rmsnorm_epilogue on h = bf16(x + residual); h is also written to h_out_bf16 unless that is None."""
+    _check(load_library().fdqp_run_add_rmsnorm_epilogue(ctx, _addr(x_bf16), _addr(residual_bf16),
+                                                        None if h_out_bf16 is None else _addr(h_out_bf16),
+                                                        _addr(gamma_bf16), float(eps), _addr(W_q4nx), _addr(out),
+                                                        int(epilogue), M, K, N, _stream(stream)),
+           "fdqp_run_add_rmsnorm_epilogue", ctx)
 
 
 def fdqp_flowkv_decode(ctx: int, q_bf16, K_bf16, V_bf16, out, H: int, G: int, d: int, L: int, pitch: int, window: int,

@@ -24,8 +24,8 @@ cudaError_t dequant_fmt_launch(int fmt, const uint8_t* W, void* out, bool out_bf
 cudaError_t prefill_set_smem_limit();
 cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, uint16_t* y16, int epi, float* ws,
                            int* status, int M, int K, int N, int pair, int Z, int fmt, cudaStream_t stream);
-cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* gamma, float eps, uint16_t* out, int M, int K,
-                           cudaStream_t stream);
+cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* residual, uint16_t* h_out, const uint16_t* gamma, float eps,
+                           uint16_t* out, int M, int K, cudaStream_t stream);
 cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* V, float* out, float* ws, int max_splits, int H,
                           int G, int d, int L, int pitch, int window, float scale, int sm_count, cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
@@ -355,8 +355,13 @@ namespace {
 // gamma != nullptr: x is RMS-normalised first, x <- bf16(x * rsqrt(mean_k x^2 + eps) * (1 + gamma)) per token row --
 // inside the GEMV kernel's activation preparation when that runs in-kernel on the whole row, else by a kernel of its own.
 fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, float eps, const void* W_q4nx, void* out,
-                     int epi, int64_t M, int64_t K, int64_t N, void* cuda_stream, int fmt = kFmtQ4nx) {
+                     int epi, int64_t M, int64_t K, int64_t N, void* cuda_stream, int fmt = kFmtQ4nx,
+                     const void* residual_bf16 = nullptr, void* h_out_bf16 = nullptr) {
     if (!ctx || !x_bf16 || !W_q4nx || !out) return FDQP_ERR_ARG;
+    if ((residual_bf16 || h_out_bf16) && !gamma_bf16) return FDQP_ERR_ARG;
+    if (h_out_bf16 && !residual_bf16) return FDQP_ERR_ARG;
+    if (h_out_bf16 && (h_out_bf16 == x_bf16 || h_out_bf16 == residual_bf16)) return FDQP_ERR_ARG;  // read by every CTA
+    if ((residual_bf16 && !aligned16(residual_bf16)) || (h_out_bf16 && !aligned16(h_out_bf16))) return FDQP_ERR_ALIGN;
     if (fmt < 0 || fmt >= kFmtCount) return FDQP_ERR_ARG;
     if (fmt != kFmtQ4nx && (K % kBlockK) != 0) return FDQP_ERR_SHAPE;           // the variants hold whole blocks only
     if (fmt != kFmtQ4nx && (epi != kEpiNone || gamma_bf16)) return FDQP_ERR_ARG;  // ... and have the fp32 store only
@@ -376,6 +381,8 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
     const uint8_t* W = static_cast<const uint8_t*>(W_q4nx);
     const uint16_t* x = static_cast<const uint16_t*>(x_bf16);
     const uint16_t* gamma = static_cast<const uint16_t*>(gamma_bf16);
+    const uint16_t* residual = static_cast<const uint16_t*>(residual_bf16);
+    uint16_t* h_out = static_cast<uint16_t*>(h_out_bf16);
     cudaError_t e;
     bool fuse_norm = false;
     if (gamma) {
@@ -385,7 +392,7 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
         fuse_norm = M <= kMaxTokens && !use_prefill(ctx, M, K, N) && plan_gemv(ctx, (int)M, (int)K, (int)N, &cw, &probe) &&
                     probe.prep_inline && probe.Z == 1 && (K / kGroup) * M * 4 <= (int64_t)cw * 32;
         if (!fuse_norm) {
-            if ((e = rmsnorm_launch(x, gamma, eps, ctx->x_norm, (int)M, (int)K, stream)))
+            if ((e = rmsnorm_launch(x, residual, h_out, gamma, eps, ctx->x_norm, (int)M, (int)K, stream)))
                 return cuda_fail(ctx, e, "RMS normalisation launch");
             ctx->launches += 1;
             x = ctx->x_norm;
@@ -428,6 +435,8 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
             plan.norm = 1;
             plan.gamma = gamma;
             plan.eps = eps;
+            plan.residual = residual;
+            plan.h_out = h_out;
         }
         if (!plan.prep_inline) {
             if ((e = xprep_launch(plan.x, ctx->xq, ctx->xsc, mc, (int)K, stream)))
@@ -473,6 +482,15 @@ extern "C" fdqp_status fdqp_run_rmsnorm_epilogue(fdqp_ctx* ctx, const void* x_bf
                                                  void* cuda_stream) {
     if (!gamma_bf16) return FDQP_ERR_ARG;
     return run_impl(ctx, x_bf16, gamma_bf16, eps, W_q4nx, out, epilogue, M, K, N, cuda_stream);
+}
+
+extern "C" fdqp_status fdqp_run_add_rmsnorm_epilogue(fdqp_ctx* ctx, const void* x_bf16, const void* residual_bf16,
+                                                     void* h_out_bf16, const void* gamma_bf16, float eps, const void* W_q4nx,
+                                                     void* out, int epilogue, int64_t M, int64_t K, int64_t N,
+                                                     void* cuda_stream) {
+    if (!gamma_bf16 || !residual_bf16) return FDQP_ERR_ARG;
+    return run_impl(ctx, x_bf16, gamma_bf16, eps, W_q4nx, out, epilogue, M, K, N, cuda_stream, kFmtQ4nx, residual_bf16,
+                    h_out_bf16);
 }
 
 extern "C" fdqp_status fdqp_flowkv_decode(fdqp_ctx* ctx, const void* q_bf16, const void* K_bf16, const void* V_bf16, float* out,

@@ -101,6 +101,16 @@ __device__ __forceinline__ uint4 xprep_load(const uint16_t* __restrict__ x, int 
     return v;
 }
 
+// Eight bf16 sums, each rounded once from the exact sum (the residual stream of a decoder layer stays in bf16).
+__device__ __forceinline__ uint4 add_bf16x8(uint4 a, uint4 b) {
+    uint4 r;
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r.x) : "r"(a.x), "r"(b.x));
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r.y) : "r"(a.y), "r"(b.y));
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r.z) : "r"(a.z), "r"(b.z));
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r.w) : "r"(a.w), "r"(b.w));
+    return r;
+}
+
 template <bool SINGLE>
 __device__ __forceinline__ void xprep_item(const uint4 v, int M, int slot, int tok, int q, bool valid,
                                            uint32_t* __restrict__ xq, float* __restrict__ xsc) {
@@ -694,6 +704,12 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                     const bool valid = tid < items;
                     const int tm = tid >> 2, tok = valid ? tm % M : 0, tile = valid ? tm / M : 0;
                     const uint4 gm = xprep_load(p.gamma, K, tile0 + tile, 0, tid & 3, valid);
+                    if (p.residual) {
+                        // the residual addition first; every CTA needs the sum, the grid's first CTA also stores it
+                        v[0] = add_bf16x8(v[0], xprep_load(p.residual, K, tile0 + tile, tok, tid & 3, valid));
+                        if (p.h_out && blockIdx.x == 0 && valid)
+                            *reinterpret_cast<uint4*>(p.h_out + (int64_t)tok * K + (tile0 + tile) * kGroup + (tid & 3) * 8) = v[0];
+                    }
                     const uint32_t xw[4] = {v[0].x, v[0].y, v[0].z, v[0].w}, gw[4] = {gm.x, gm.y, gm.z, gm.w};
                     float f[8], ss = 0.f;
 #pragma unroll
@@ -985,17 +1001,24 @@ extern "C" __attribute__((visibility("default"))) int fdqp_trace_read(unsigned l
 
 // RMS normalisation on its own (the calls whose activation preparation does not happen inside a GEMV CTA): one CTA per
 // token row, out[m][k] = bf16(x * rsqrt(mean(x^2) + eps) * (1 + gamma[k])).
-__global__ void __launch_bounds__(256) fdqp_rmsnorm_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
+// residual (may be null): x + residual, rounded once to bf16, is what gets normalised; h_out (may be null) receives it.
+__global__ void __launch_bounds__(256) fdqp_rmsnorm_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ residual,
+                                                            uint16_t* __restrict__ h_out, const uint16_t* __restrict__ gamma,
                                                             float eps, uint16_t* __restrict__ out, int K) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");  // x may be the previous launch's output
     __shared__ float part[8];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint16_t* xr = x + (int64_t)blockIdx.x * K;
+    const uint16_t* rr = residual ? residual + (int64_t)blockIdx.x * K : nullptr;
     uint16_t* orow = out + (int64_t)blockIdx.x * K;
     float ss = 0.f;
     for (int k = tid * 8; k < K; k += 256 * 8) {  // K is a multiple of 32
-        const uint4 w = *reinterpret_cast<const uint4*>(xr + k);
+        uint4 w = *reinterpret_cast<const uint4*>(xr + k);
+        if (rr) {
+            w = add_bf16x8(w, *reinterpret_cast<const uint4*>(rr + k));
+            if (h_out) *reinterpret_cast<uint4*>(h_out + (int64_t)blockIdx.x * K + k) = w;
+        }
         const uint32_t xw[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -1013,7 +1036,9 @@ __global__ void __launch_bounds__(256) fdqp_rmsnorm_kernel(const uint16_t* __res
     for (int w = 0; w < 8; ++w) tot += part[w];
     const float r = rsqrtf(tot / (float)K + eps);
     for (int k = tid * 8; k < K; k += 256 * 8) {
-        const uint4 w = *reinterpret_cast<const uint4*>(xr + k), g = *reinterpret_cast<const uint4*>(gamma + k);
+        uint4 w = *reinterpret_cast<const uint4*>(xr + k);
+        if (rr) w = add_bf16x8(w, *reinterpret_cast<const uint4*>(rr + k));  // the same sum as in the first pass
+        const uint4 g = *reinterpret_cast<const uint4*>(gamma + k);
         const uint32_t xw[4] = {w.x, w.y, w.z, w.w}, gw[4] = {g.x, g.y, g.z, g.w};
         uint32_t o[4];
 #pragma unroll
@@ -1026,8 +1051,8 @@ __global__ void __launch_bounds__(256) fdqp_rmsnorm_kernel(const uint16_t* __res
     }
 }
 
-cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* gamma, float eps, uint16_t* out, int M, int K,
-                           cudaStream_t stream) {
+cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* residual, uint16_t* h_out, const uint16_t* gamma, float eps,
+                           uint16_t* out, int M, int K, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)M);
     cfg.blockDim = dim3(256);
@@ -1037,7 +1062,7 @@ cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* gamma, float eps, 
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fdqp_rmsnorm_kernel, x, gamma, eps, out, K);
+    return cudaLaunchKernelEx(&cfg, fdqp_rmsnorm_kernel, x, residual, h_out, gamma, eps, out, K);
 }
 
 // ---- host-visible launchers ------------------------------------------------------------------

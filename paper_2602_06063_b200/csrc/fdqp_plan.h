@@ -33,6 +33,8 @@ struct GemvPlan {
     const uint16_t* gamma;  // RMS normalisation of x fused into the in-kernel activation preparation (norm != 0):
     float eps;              //   x <- bf16(x * rsqrt(mean(x^2) + eps) * (1 + gamma)), per token row
     int norm;
+    const uint16_t* residual;  // with norm: x + residual (bf16, one rounding) is what gets normalised ...
+    uint16_t* h_out;           // ... and, when not null, is also written here by the grid's first CTA ([M][K] bf16)
     float* ws_edge;       // device, [grid][2][32*kMaxTokens] partial sums of strips shared between CTAs
     float* ws_full;       // device, [Z][S][32*kMaxTokens] partial sums of whole strip-slices (Z > 1)
     int* tickets;         // device, [S] arrival counters, zero between launches

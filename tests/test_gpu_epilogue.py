@@ -230,3 +230,61 @@ def test_rmsnorm_argument_errors(fresh):
     assert lib.fdqp_run_rmsnorm_epilogue(*a, g.data_ptr(), -1.0, *b) == 1          # negative eps
     assert lib.fdqp_run_rmsnorm_epilogue(*a, g.data_ptr(), 1e-6, *b) == 0
     torch.cuda.synchronize()
+
+
+# ---- residual addition + RMS normalisation ahead of the projection ---------------------------------------------------
+
+@pytest.mark.parametrize("K,N,M,params,launches", NORM_CASES)
+def test_residual_add_rmsnorm_then_projection_matches_oracle(fresh, K, N, M, params, launches):
+    case = Case(K, N, M, seed=6500 + K + N + M, amp=2.0)
+    res = synthgen.activations(6600 + K + M, M, K, 1.5)
+    res[0, :8] = case.x[0, :8] ^ 0x8000                          # exact cancellation inside a row
+    gamma = synthgen.bf16_bits((0.25 * synthgen.bf16_to_f32(synthgen.activations(6700 + K, 1, K))[0]).astype(np.float32))
+    gamma_dev = torch.from_numpy(gamma.view(np.int16)).cuda()
+    res_dev = torch.from_numpy(res.view(np.int16)).cuda()
+    h_dev = torch.full((M, K), 0x7FC0, dtype=torch.int16, device="cuda")
+    out = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+    eps = 1e-6
+    for k, v in params.items():
+        fd.fdqp_set_param(fresh, k, v)
+    before = fd.fdqp_launch_count(fresh)
+    fd.fdqp_run_add_rmsnorm_epilogue(fresh, case.x_dev, res_dev, h_dev, gamma_dev, eps, case.W_dev, out, fd.EPI_NONE, M, K, N)
+    torch.cuda.synchronize()
+    assert fd.fdqp_last_status(fresh) == 0
+    assert fd.fdqp_launch_count(fresh) - before == launches      # the addition costs no launch of its own
+    h_ref = oracle.add_residual(case.x, res)
+    assert np.array_equal(h_dev.cpu().numpy().view(np.uint16), h_ref)          # the residual stream, bit for bit
+    x_n = oracle.rmsnorm(h_ref, gamma, eps)
+    y_ref, a_ref = oracle.project(x_n, case.w.codes, case.w.scales, case.w.offsets, nthreads=8)
+    y = out.cpu().numpy()
+    err = np.abs(y.astype(np.float64) - y_ref)
+    assert np.all(np.isfinite(y)) and np.all(err <= REL_TOL * a_ref + ABS_TOL)
+    # without an output for h the projection is the same, bit for bit
+    out2 = torch.zeros_like(out)
+    fd.fdqp_run_add_rmsnorm_epilogue(fresh, case.x_dev, res_dev, None, gamma_dev, eps, case.W_dev, out2, fd.EPI_NONE, M, K, N)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+    # a zero residual is the normalisation alone, bit for bit
+    zero = torch.zeros_like(res_dev)
+    fd.fdqp_run_add_rmsnorm_epilogue(fresh, case.x_dev, zero, None, gamma_dev, eps, case.W_dev, out2, fd.EPI_NONE, M, K, N)
+    torch.cuda.synchronize()
+    assert np.array_equal(out2.cpu().numpy(), run_norm(fresh, case, gamma_dev, eps, fd.EPI_NONE))
+
+
+def test_residual_add_argument_errors(fresh):
+    case = Case(256, 64, 1, seed=9)
+    out = torch.empty((1, 64), dtype=torch.float32, device="cuda")
+    g = torch.zeros(256, dtype=torch.int16, device="cuda")
+    r = torch.zeros(256 + 8, dtype=torch.int16, device="cuda")
+    h = torch.zeros(256, dtype=torch.int16, device="cuda")
+    lib = fd.load_library()
+    s = torch.cuda.current_stream().cuda_stream
+    x = case.x_dev.data_ptr()
+    tail = (case.W_dev.data_ptr(), out.data_ptr(), 0, 1, 256, 64, s)
+    f = lib.fdqp_run_add_rmsnorm_epilogue
+    assert f(fresh, x, None, h.data_ptr(), g.data_ptr(), 1e-6, *tail) == 1                 # null residual
+    assert f(fresh, x, r.data_ptr() + 2, h.data_ptr(), g.data_ptr(), 1e-6, *tail) == 3     # misaligned residual
+    assert f(fresh, x, r.data_ptr(), x, g.data_ptr(), 1e-6, *tail) == 1                    # h aliases x
+    assert f(fresh, x, r.data_ptr(), r.data_ptr(), g.data_ptr(), 1e-6, *tail) == 1         # h aliases the residual
+    assert f(fresh, x, r.data_ptr(), h.data_ptr(), g.data_ptr(), 1e-6, *tail) == 0
+    torch.cuda.synchronize()
