@@ -120,8 +120,9 @@ int prefill_slices(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
 // M >= 9: the tensor-core kernels, or the GEMV kernel eight token rows at a time -- whichever a small cost model
 // (microseconds, constants measured on B200) says is faster.
 //   GEMV: every chunk streams the whole matrix, at about 5.5 TB/s for 1-2 rows, 3.9 for 3-4, 3.2 for 5-8, plus ~5 us.
-//   Tensor-core kernels: limited by converting the weights: per wave of tiles and 64-wide k-step ~0.78 us (one-SM
-//   kernel) or ~0.95 us (two-SM kernel, which also has twice the tokens' MMAs to issue), whatever M is.
+//   Tensor-core kernels: per wave of tiles and 64-wide k-step ~0.72 us (one-SM kernel, 128-row tiles two to an SM, up
+//   to 128 tokens), ~0.78 us (256-row tiles) or ~0.95 us (two-SM kernel, which also has twice the tokens' MMAs to
+//   issue), nearly independent of M.
 bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     if (M <= kMaxTokens || ctx->p_path == 2) return false;
     if (ctx->p_path == 3) return true;
@@ -134,7 +135,7 @@ bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     const int64_t slots = pair ? ctx->sm_count / 2 : ctx->sm_count;
     const int Z = prefill_slices(ctx, M, K, N);
     const double waves = (double)((tiles * Z + slots - 1) / slots);
-    double t_tensor = 5.0 + waves * (double)(((K + 63) / 64 + Z - 1) / Z) * (pair ? 0.95 : 0.78);
+    double t_tensor = 5.0 + waves * (double)(((K + 63) / 64 + Z - 1) / Z) * (pair ? 0.95 : (M <= 128 ? 0.72 : 0.78));
     if (Z > 1) t_tensor += 3.0 + (double)(Z + 1) * (double)M * (double)N * 4.0 / 5.0e6;  // partial results out and back
     if (M * K * 2 < kSpreadBelowBytes) t_tensor += 3.0;                                   // the spreading copy
     return t_tensor < t_gemv;
@@ -645,6 +646,11 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
                           "fdqp_prefill_pair_kernel grid=%lld cluster=2 block=320 tile=256x512 per pair stages=4 tmem_cols=512 "
                           "split_k=%d%s",
                           (long long)(2 * ((N + 255) / 256) * ((M + 511) / 512) * Z), Z, Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
+        else if (M <= 128)
+            std::snprintf(buf, buf_bytes,
+                          "fdqp_prefill_kernel<128> grid=%lld block=320 tile=128x128 two CTAs per SM stages=3 tmem_cols=128 "
+                          "split_k=%d%s",
+                          (long long)(((N + 127) / 128) * Z), Z, Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
         else
             std::snprintf(buf, buf_bytes,
                           "fdqp_prefill_kernel grid=%lld block=576 tile=256x256 stages=3 tmem_cols=512 split_k=%d%s",

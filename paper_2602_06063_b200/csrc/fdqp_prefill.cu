@@ -29,15 +29,24 @@ constexpr int kPfRows = 256;      // output features per CTA tile
 constexpr int kPfToks = 256;      // tokens per CTA tile
 constexpr int kPfK = 64;          // k per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int kPfStages = 3;
-constexpr uint32_t kPfABytes = kPfRows * kPfK * 2;  // 32 KB
-constexpr uint32_t kPfBBytes = kPfToks * kPfK * 2;  // 32 KB
-constexpr uint32_t kPfStageBytes = kPfABytes + kPfBBytes;
 constexpr int kPfDequantWarps = 8;   // two-SM kernel: one (strip, group) of the CTA's 128 rows each
 constexpr int kPfThreads = (2 + kPfDequantWarps) * 32;  // warp 0: TMA + TMEM owner, warp 1: MMA issuer
-constexpr int kPf1DequantWarps = 16;  // one-SM kernel: one (strip, group) of the CTA's 256 rows each
-constexpr int kPf1Threads = (2 + kPf1DequantWarps) * 32;
 constexpr uint32_t kPfTmemCols = 512;
-constexpr uint32_t kPfSmemBytes = kPfStages * kPfStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+// Geometry of the one-SM kernel by tile height (see the kernel).
+template <int ROWS>
+struct Pf1 {
+    static constexpr int kRows = ROWS;
+    static constexpr int kToks = ROWS == 256 ? 256 : 128;             // tokens per CTA tile = rows of the x box
+    static constexpr uint32_t kABytes = ROWS * kPfK * 2;
+    static constexpr uint32_t kBBytes = kToks * kPfK * 2;
+    static constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    static constexpr int kDequantWarps = ROWS / 16;                   // one (strip, group) of the tile each
+    static constexpr int kThreads = (2 + kDequantWarps) * 32;
+    static constexpr uint32_t kTmemCols = ROWS == 256 ? 512 : 128;
+    static constexpr uint32_t kSmemBytes = kPfStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int kCtasPerSm = ROWS == 256 ? 1 : 2;
+};
 
 struct PrefillParams {
     const uint8_t* W;
@@ -275,16 +284,42 @@ __device__ __forceinline__ void stage_copy_out(uint32_t stage, uint16_t* dst, in
 
 // ---- the kernel -------------------------------------------------------------------------------------------------------
 
-template <int FMT>
-__global__ void __launch_bounds__(kPf1Threads, 1)
+#ifdef FDQP_TRACE
+// trace builds only: 16 time stamps / counters for each of the first 512 CTAs of the last launch
+__device__ unsigned long long g_pf_trace[512 * 16];
+#define PF_STAMP(i) do { if (blockIdx.x < 512) g_pf_trace[blockIdx.x * 16 + (i)] = globaltimer_ns(); } while (0)
+#define PF_ADD(i, v) do { if (blockIdx.x < 512) g_pf_trace[blockIdx.x * 16 + (i)] += (v); } while (0)
+#define PF_T0() const unsigned long long pf_t0 = globaltimer_ns()
+#define PF_DT() (globaltimer_ns() - pf_t0)
+extern "C" __attribute__((visibility("default"))) int fdqp_pf_trace_read(unsigned long long* host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_pf_trace, sizeof(unsigned long long) * (size_t)n);
+}
+extern "C" __attribute__((visibility("default"))) int fdqp_pf_trace_clear() {
+    static unsigned long long zeros[512 * 16];
+    return (int)cudaMemcpyToSymbol(g_pf_trace, zeros, sizeof(zeros));
+}
+#else
+#define PF_STAMP(i) do { } while (0)
+#define PF_ADD(i, v) do { } while (0)
+#define PF_T0() do { } while (0)
+#define PF_DT() 0
+#endif
+
+// ROWS: output features per CTA tile.  256: the tile described above, one CTA per SM.  128 (for M <= 128): a 128 x 128
+// tile with half-size stages (16 KB + 16 KB), eight conversion warps and 128 TMEM columns, so that TWO CTAs share an SM:
+// one CTA's start-up, epilogue and stage latencies overlap the other's main loop.
+template <int FMT, int ROWS>
+__global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
     fdqp_prefill_kernel(const __grid_constant__ CUtensorMap x_map, const PrefillParams p) {
+    using P = Pf1<ROWS>;
+    constexpr int CH = P::kToks / 2;  // token columns per epilogue warp of a quarter
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // tiles must start on a 1024-byte boundary (swizzle atom)
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    const uint32_t bars = base + kPfStages * kPfStageBytes;
+    const uint32_t bars = base + kPfStages * P::kStageBytes;
     // barriers: full_a[s], full_b[s], empty[s], acc_done; then the TMEM base address slot
     auto full_a = [&](int s) { return bars + 8u * s; };
     auto full_b = [&](int s) { return bars + 8u * (kPfStages + s); };
@@ -292,31 +327,32 @@ __global__ void __launch_bounds__(kPf1Threads, 1)
     const uint32_t acc_done = bars + 8u * (3 * kPfStages);
     const uint32_t tmem_slot = acc_done + 8u;
     const uint32_t staged = tmem_slot + 8u;  // bf16 epilogues: every epilogue warp has written its part of the tile
-    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(smem + kPfStages * kPfStageBytes + 8 * (3 * kPfStages + 1));
+    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(smem + kPfStages * P::kStageBytes + 8 * (3 * kPfStages + 1));
 
-    const int tok_tiles = (p.M + kPfToks - 1) / kPfToks;
+    const int tok_tiles = (p.M + P::kToks - 1) / P::kToks;
     const int tile_id = blockIdx.x / p.Z, z = blockIdx.x % p.Z;                    // K slices of one tile adjacent
     const int n_tile = tile_id / tok_tiles, tok_tile = tile_id % tok_tiles;        // token tiles of one n-tile adjacent
-    const int n0 = n_tile * kPfRows, tok0 = tok_tile * kPfToks;
-    const int toks = (p.M - tok0) < kPfToks ? (p.M - tok0) : kPfToks;
+    const int n0 = n_tile * P::kRows, tok0 = tok_tile * P::kToks;
+    const int toks = (p.M - tok0) < P::kToks ? (p.M - tok0) : P::kToks;
     const uint32_t n_inst = (uint32_t)((toks + 15) & ~15);
     const int ksteps_all = (p.K + kPfK - 1) / kPfK;
     const int ks0 = z * p.ksteps_z;                                                // first k-step of this slice
     const int ksteps = (ksteps_all - ks0) < p.ksteps_z ? (ksteps_all - ks0) : p.ksteps_z;
     float* const yout = p.y + (int64_t)z * p.M * p.N;
+    if (tid == 0) PF_STAMP(0);
 
     if (tid == 0) {
         for (int s = 0; s < kPfStages; ++s) {
-            mbar_init(full_a(s), kPf1DequantWarps);
+            mbar_init(full_a(s), P::kDequantWarps);
             mbar_init(full_b(s), 1);
             mbar_init(empty(s), 1);
         }
         mbar_init(acc_done, 1);
-        mbar_init(staged, kPf1DequantWarps);
+        mbar_init(staged, P::kDequantWarps);
         mbar_fence_init();
     }
     if (warp == 0) {
-        tmem_alloc(tmem_slot, kPfTmemCols);
+        tmem_alloc(tmem_slot, P::kTmemCols);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -324,6 +360,7 @@ __global__ void __launch_bounds__(kPf1Threads, 1)
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_g;
     bool ok = true;
+    if (tid == 0) PF_STAMP(1);
 
     if (warp == 0) {
         // =============================== TMA producer: x tiles ==============================================
@@ -332,8 +369,8 @@ __global__ void __launch_bounds__(kPf1Threads, 1)
                 const int s = i % kPfStages;
                 if (i >= kPfStages) ok = mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status);
                 if (!ok) break;
-                mbar_arrive_expect_tx(full_b(s), kPfBBytes);
-                tma_load_2d(base + s * kPfStageBytes + kPfABytes, &x_map, (ks0 + i) * kPfK, tok0, full_b(s));
+                mbar_arrive_expect_tx(full_b(s), P::kBBytes);
+                tma_load_2d(base + s * P::kStageBytes + P::kABytes, &x_map, (ks0 + i) * kPfK, tok0, full_b(s));
             }
         }
     } else if (warp == 1) {
@@ -343,68 +380,116 @@ __global__ void __launch_bounds__(kPf1Threads, 1)
             for (int i = 0; i < ksteps && ok; ++i) {
                 const int s = i % kPfStages;
                 const uint32_t ph = (i / kPfStages) & 1;
+#ifdef FDQP_TRACE
+                {
+                    PF_T0();
+                    ok = mbar_wait(full_a(s), ph, p.status);
+                    PF_ADD(12, PF_DT());
+                }
+                {
+                    PF_T0();
+                    ok = ok && mbar_wait(full_b(s), ph, p.status);
+                    PF_ADD(13, PF_DT());
+                }
+                if (i == 0) PF_STAMP(2);
+                if (i == 10) PF_STAMP(3);
+                if (i == 20) PF_STAMP(4);
+                if (i == 30) PF_STAMP(5);
+#else
                 ok = mbar_wait(full_a(s), ph, p.status) && mbar_wait(full_b(s), ph, p.status);
+#endif
                 if (!ok) break;
+#ifdef FDQP_TRACE
+                const unsigned long long pf_m0 = globaltimer_ns();
+#endif
                 tc_fence_after();
-                const uint32_t a_addr = base + s * kPfStageBytes, b_addr = a_addr + kPfABytes;
+                const uint32_t a_addr = base + s * P::kStageBytes, b_addr = a_addr + P::kABytes;
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const uint64_t adesc = umma_smem_desc(a_addr + half * (kPfABytes / 2));
+                for (int half = 0; half < ROWS / 128; ++half) {
+                    const uint64_t adesc = umma_smem_desc(a_addr + half * (128 * kPfK * 2));
                     const uint64_t bdesc = umma_smem_desc(b_addr);
 #pragma unroll
                     for (int k4 = 0; k4 < kPfK / 16; ++k4)  // 32 bytes (16 bf16) further along the swizzled row
                         umma_bf16(tmem_base + half * 256, adesc + 2 * k4, bdesc + 2 * k4, idesc, (i | k4) != 0);
                 }
                 umma_commit(empty(s));  // the stage may be refilled once these MMAs have read it
+#ifdef FDQP_TRACE
+                PF_ADD(14, globaltimer_ns() - pf_m0);
+#endif
             }
+            PF_STAMP(6);
             umma_commit(acc_done);
         }
     } else {
         // =============================== dequantisation warps ================================================
         const int dw = warp - 2;
         const int sl = dw >> 1, gl = dw & 1;  // strip of the tile and group of the 64-k stage this warp converts
-        const int64_t strip = (int64_t)n_tile * (kPfRows / 32) + sl;
+        const int64_t strip = (int64_t)n_tile * (P::kRows / 32) + sl;
         const bool strip_ok = strip < p.N / kStripRows;
         // the loads of the next three stages are in flight while this one is converted (a stage lasts about as long
         // as one trip to HBM); groups past K load as zeros
         const int gbase = 2 * ks0 + gl;  // this warp's group in k-step i of the slice: gbase + 2 i
-        GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase, lane, strip_ok);
-        GroupRegs g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2, lane, strip_ok);
-        GroupRegs g2 = group_load<FMT>(p.W, p.K, strip, gbase + 4, lane, strip_ok);
-        for (int i = 0; i < ksteps && ok; ++i) {
+        // Three register sets, each reloaded right after it has been converted.  (Rotating the sets with moves instead --
+        // g0 = g1; g1 = g2; g2 = just-loaded -- makes the move wait for the load it follows, one trip to memory per k-step.)
+        auto convert_step = [&](int i, const GroupRegs& g) -> bool {
             const int s = i % kPfStages;
-            const GroupRegs g3 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
-            if (i >= kPfStages) ok = mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status);
-            if (!ok) break;
-            group_store<FMT>(base + s * kPfStageBytes, g0, sl, gl, lane);
+#ifdef FDQP_TRACE
+            const unsigned long long pf_w0 = globaltimer_ns();
+#endif
+            if (i >= kPfStages && !mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status)) return false;
+            if (dw == 0 && lane == 0 && i == 0) PF_STAMP(10);
+#ifdef FDQP_TRACE
+            const unsigned long long pf_w1 = globaltimer_ns();
+#endif
+            group_store<FMT>(base + s * P::kStageBytes, g, sl, gl, lane);
             // make the generic-proxy stores visible to the tensor core's (async-proxy) reads, then signal
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(full_a(s));
-            g0 = g1;
-            g1 = g2;
-            g2 = g3;
+#ifdef FDQP_TRACE
+            if (dw == 0 && lane == 0) {
+                PF_ADD(11, pf_w1 - pf_w0);
+                PF_ADD(15, globaltimer_ns() - pf_w1);
+            }
+#endif
+            return true;
+        };
+        GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase, lane, strip_ok);
+        GroupRegs g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2, lane, strip_ok);
+        GroupRegs g2 = group_load<FMT>(p.W, p.K, strip, gbase + 4, lane, strip_ok);
+        for (int i = 0; i < ksteps && ok; i += 3) {
+            ok = convert_step(i, g0);
+            g0 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
+            if (ok && i + 1 < ksteps) {
+                ok = convert_step(i + 1, g1);
+                g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 4), lane, strip_ok);
+            }
+            if (ok && i + 2 < ksteps) {
+                ok = convert_step(i + 2, g2);
+                g2 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 5), lane, strip_ok);
+            }
         }
         // =============================== epilogue: TMEM -> y =================================================
         if (ok) ok = mbar_wait(acc_done, 0, p.status);
         ok = __all_sync(0xffffffffu, ok);
+        if (dw == 0 && lane == 0) PF_STAMP(7);
         const bool via_smem = p.epi != kEpiNone && p.Z == 1;  // bf16 epilogues (a K-split call leaves them to the sum)
         const bool geglu = p.epi == kEpiGegluBf16;
-        const int cols = geglu ? kPfRows / 2 : kPfRows;       // bf16 values per token row of the staged tile
+        const int cols = geglu ? P::kRows / 2 : P::kRows;       // bf16 values per token row of the staged tile
         if (ok) {
             tc_fence_after();
             const int quarter = warp & 3;        // TMEM lanes this warp may read
             // the four warps of a quarter (dw = quarter', quarter' + 4, + 8, + 12) take (accumulator, column half)
-            const int half = (dw >> 2) & 1, chalf = dw >> 3;
+            const int half = ROWS == 256 ? (dw >> 2) & 1 : 0, chalf = ROWS == 256 ? dw >> 3 : dw >> 2;
             const int n_local = half * 128 + quarter * 32 + lane;
             const int n = n0 + n_local;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 256 + chalf * 128);
-            const int c_end = ((int)n_inst < chalf * 128 + 128 ? (int)n_inst : chalf * 128 + 128) - chalf * 128;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 256 + chalf * CH);
+            const int c_end = ((int)n_inst < chalf * CH + CH ? (int)n_inst : chalf * CH + CH) - chalf * CH;
             const int64_t ldy = p.N;
-            float* yrow = yout + (int64_t)(tok0 + chalf * 128) * ldy + n;  // token row of this warp's column 0
-            const int toks_h = toks - chalf * 128;                          // tokens of this column half that exist
+            float* yrow = yout + (int64_t)(tok0 + chalf * CH) * ldy + n;  // token row of this warp's column 0
+            const int toks_h = toks - chalf * CH;                          // tokens of this column half that exist
             // staged tile: this lane's column, and the first token row of this warp
-            const uint32_t scol = base + (uint32_t)((chalf * 128) * cols + (geglu ? (n_local >> 5) * 16 + (lane & 15) : n_local)) * 2u;
+            const uint32_t scol = base + (uint32_t)((chalf * CH) * cols + (geglu ? (n_local >> 5) * 16 + (lane & 15) : n_local)) * 2u;
             for (int c = 0; c < c_end; c += 32) {
                 uint32_t v[32];
                 tmem_ld_32cols(taddr + c, v);
@@ -447,17 +532,19 @@ __global__ void __launch_bounds__(kPf1Threads, 1)
                 const int64_t ld16 = geglu ? p.N / 2 : p.N;
                 const int col0 = geglu ? n0 / 2 : n0;
                 const int valid = (int)((ld16 - col0) < cols ? (ld16 - col0) : cols);
-                stage_copy_out(base, p.y16 + (int64_t)tok0 * ld16 + col0, ld16, toks, cols, valid, dw, kPf1DequantWarps, lane);
+                stage_copy_out(base, p.y16 + (int64_t)tok0 * ld16 + col0, ld16, toks, cols, valid, dw, P::kDequantWarps, lane);
             }
         }
     }
     // =============================== teardown: every path releases TMEM =====================================
+    if (warp == 2 && lane == 0) PF_STAMP(8);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, kPfTmemCols);
+        tmem_dealloc(tmem_base, P::kTmemCols);
     }
+    if (tid == 0) PF_STAMP(9);
 }
 
 // ---- the two-SM kernel (M > 256) ----------------------------------------------------------------------------------
@@ -659,22 +746,31 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         // software pipeline: the loads of the next three stages are in flight while this one is converted (a stage
         // lasts well under a microsecond here, less than one trip to L2 / HBM); groups past K load as zeros
         const int gbase = 2 * ks0 + gl;  // this warp's group in k-step i of the slice: gbase + 2 i
-        GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase, lane, strip_ok);
-        GroupRegs g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2, lane, strip_ok);
-        GroupRegs g2 = group_load<FMT>(p.W, p.K, strip, gbase + 4, lane, strip_ok);
+        // three register sets, each reloaded right after it has been converted (no rotation by moves: see the one-SM kernel)
         const uint32_t full_a0 = mapa_shared(full_a(0), 0);
-        for (int i = 0; i < ksteps && ok; ++i) {
+        auto convert_step = [&](int i, const GroupRegs& g) -> bool {
             const int s = i % kP2Stages;
-            const GroupRegs g3 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
-            if (i >= kP2Stages) ok = mbar_wait(empty(s), ((i / kP2Stages) - 1) & 1, p.status);
-            if (!ok) break;
-            group_store<FMT>(base + s * kP2StageBytes, g0, sl, gl, lane);
+            if (i >= kP2Stages && !mbar_wait(empty(s), ((i / kP2Stages) - 1) & 1, p.status)) return false;
+            group_store<FMT>(base + s * kP2StageBytes, g, sl, gl, lane);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(full_a0 + 8u * s);
-            g0 = g1;
-            g1 = g2;
-            g2 = g3;
+            return true;
+        };
+        GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase, lane, strip_ok);
+        GroupRegs g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2, lane, strip_ok);
+        GroupRegs g2 = group_load<FMT>(p.W, p.K, strip, gbase + 4, lane, strip_ok);
+        for (int i = 0; i < ksteps && ok; i += 3) {
+            ok = convert_step(i, g0);
+            g0 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
+            if (ok && i + 1 < ksteps) {
+                ok = convert_step(i + 1, g1);
+                g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 4), lane, strip_ok);
+            }
+            if (ok && i + 2 < ksteps) {
+                ok = convert_step(i + 2, g2);
+                g2 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 5), lane, strip_ok);
+            }
         }
         // =============================== epilogue: this CTA's TMEM -> y ======================================
         if (ok) ok = mbar_wait(acc_done, 0, p.status);
@@ -796,8 +892,9 @@ static EncodeTiledFn encode_tiled_fn() {
 
 template <int FMT>
 static cudaError_t prefill_set_smem_limit_fmt() {
-    cudaError_t e = cudaFuncSetAttribute(fdqp_prefill_kernel<FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPfSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(fdqp_prefill_kernel<FMT, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Pf1<256>::kSmemBytes);
     if (e) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_prefill_kernel<FMT, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Pf1<128>::kSmemBytes))) return e;
     return cudaFuncSetAttribute(fdqp_prefill_pair_kernel<FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kP2SmemBytes);
 }
 
@@ -828,8 +925,13 @@ static cudaError_t prefill_launch_kernels(const CUtensorMap& map, const PrefillP
         cfg.numAttrs = 1;
         return cudaLaunchKernelEx(&cfg, fdqp_prefill_pair_kernel<FMT>, map, p);
     }
+    if (pair == 0 && M <= Pf1<128>::kToks) {  // small tiles, two CTAs per SM
+        const int n_tiles = (N + 127) / 128;
+        fdqp_prefill_kernel<FMT, 128><<<n_tiles * Z, Pf1<128>::kThreads, Pf1<128>::kSmemBytes, stream>>>(map, p);
+        return cudaGetLastError();
+    }
     const int n_tiles = (N + kPfRows - 1) / kPfRows, tok_tiles = (M + kPfToks - 1) / kPfToks;
-    fdqp_prefill_kernel<FMT><<<n_tiles * tok_tiles * Z, kPf1Threads, kPfSmemBytes, stream>>>(map, p);
+    fdqp_prefill_kernel<FMT, 256><<<n_tiles * tok_tiles * Z, Pf1<256>::kThreads, Pf1<256>::kSmemBytes, stream>>>(map, p);
     return cudaGetLastError();
 }
 
@@ -847,7 +949,7 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_by
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};      // innermost first
     const cuuint64_t strides[1] = {(cuuint64_t)x_row_bytes};        // bytes between token rows
-    const cuuint32_t box[2] = {(cuuint32_t)kPfK, (cuuint32_t)(pair ? kP2TokBox : kPfToks)};
+    const cuuint32_t box[2] = {(cuuint32_t)kPfK, (cuuint32_t)(pair ? kP2TokBox : (M <= Pf1<128>::kToks ? Pf1<128>::kToks : kPfToks))};
     const cuuint32_t elem[2] = {1, 1};
     if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t*>(x), dims, strides, box, elem,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
