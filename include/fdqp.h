@@ -342,7 +342,10 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "prefill_split_k" 1..8 K slices for the tensor-core kernels (their partial results are added by a second
  *                   kernel); default: as many as fill the SMs when a shape has few output tiles
  *   "prefill_pair"  1 = prefill-sized calls use the two-SM kernel (256 x 512 tile per CTA pair), 0 = the one-SM kernel
- *                   (256 x 256 tile); default: two-SM kernel when M > 256
+ *                   (256 x 256 tile; 128 x 128 tiles, two CTAs per SM, up to 128 token rows); default: two-SM kernel
+ *                   when M > 256
+ *   "prefill_a_tmem" one-SM tensor-core kernel up to 128 token rows: 1 (default) = the converted weights are kept in
+ *                   tensor memory and read from there by the MMAs, 0 = in shared memory; same results bit for bit
  *   "debug"         measurement aid: 1 = the GEMV consumers skip the arithmetic (y is then undefined)
  * Unknown key or unusable value: FDQP_ERR_ARG.  Meant for benchmarks and tests. */
 FDQP_API fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t value);

@@ -23,7 +23,7 @@ cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, in
 cudaError_t dequant_fmt_launch(int fmt, const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
 cudaError_t prefill_set_smem_limit();
 cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, uint16_t* y16, int epi, float* ws,
-                           int* status, int M, int K, int N, int pair, int Z, int fmt, cudaStream_t stream);
+                           int* status, int M, int K, int N, int pair, int Z, int fmt, int a_tmem, cudaStream_t stream);
 cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* residual, uint16_t* h_out, const uint16_t* gamma, float eps,
                            uint16_t* out, int M, int K, cudaStream_t stream);
 cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* V, float* out, float* ws, int max_splits, int H,
@@ -56,6 +56,7 @@ struct fdqp_ctx {
     std::string last_err;
     // overrides (-1 = automatic)
     int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1, p_prep = -1, p_aligned = -1, p_bpw = -1, p_pair = -1, p_pf_split = -1;
+    int64_t p_atmem = 1;  // tensor-core kernel up to 128 tokens: keep the converted weights in tensor memory
 };
 
 namespace {
@@ -416,7 +417,7 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
             xt = reinterpret_cast<const uint16_t*>(ctx->x_spread);
         }
         if ((e = prefill_launch(W, xt, x_row_bytes, y, y16, epi, ctx->pf_ws, ctx->status_dev, (int)M, (int)K, (int)N,
-                                use_pair(ctx, M) ? 1 : 0, prefill_slices(ctx, M, K, N), fmt, stream)))
+                                use_pair(ctx, M) ? 1 : 0, prefill_slices(ctx, M, K, N), fmt, ctx->p_atmem != 0 ? 1 : 0, stream)))
             return cuda_fail(ctx, e, "prefill kernel launch");
         ctx->launches += prefill_slices(ctx, M, K, N) > 1 ? 2 : 1;
         return FDQP_OK;
@@ -605,6 +606,9 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
     } else if (!std::strcmp(key, "prefill_split_k")) {
         if (v == 0 || v > kMaxSplit) return FDQP_ERR_ARG;
         ctx->p_pf_split = v;
+    } else if (!std::strcmp(key, "prefill_a_tmem")) {
+        if (v != 0 && v != 1) return FDQP_ERR_ARG;
+        ctx->p_atmem = v;
     } else if (!std::strcmp(key, "prefill_pair")) {
         if (v > 1) return FDQP_ERR_ARG;
         ctx->p_pair = v;
@@ -648,9 +652,10 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
                           (long long)(2 * ((N + 255) / 256) * ((M + 511) / 512) * Z), Z, Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
         else if (M <= 128)
             std::snprintf(buf, buf_bytes,
-                          "fdqp_prefill_kernel<128> grid=%lld block=320 tile=128x128 two CTAs per SM stages=3 tmem_cols=128 "
-                          "split_k=%d%s",
-                          (long long)(((N + 127) / 128) * Z), Z, Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
+                          "fdqp_prefill_kernel<128> grid=%lld block=320 tile=128x128 two CTAs per SM %s split_k=%d%s",
+                          (long long)(((N + 127) / 128) * Z),
+                          ctx->p_atmem ? "weights in TMEM (4 stages) x_stages=6 tmem_cols=256" : "stages=3 tmem_cols=128", Z,
+                          Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
         else
             std::snprintf(buf, buf_bytes,
                           "fdqp_prefill_kernel grid=%lld block=576 tile=256x256 stages=3 tmem_cols=512 split_k=%d%s",

@@ -33,6 +33,7 @@ constexpr int kPfDequantWarps = 8;   // two-SM kernel: one (strip, group) of the
 constexpr int kPfThreads = (2 + kPfDequantWarps) * 32;  // warp 0: TMA + TMEM owner, warp 1: MMA issuer
 constexpr uint32_t kPfTmemCols = 512;
 
+constexpr int kPfTmemAStages = 4, kPfTmemBStages = 6;  // the variant that keeps the weights in tensor memory
 // Geometry of the one-SM kernel by tile height (see the kernel).
 template <int ROWS>
 struct Pf1 {
@@ -46,6 +47,7 @@ struct Pf1 {
     static constexpr uint32_t kTmemCols = ROWS == 256 ? 512 : 128;
     static constexpr uint32_t kSmemBytes = kPfStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
     static constexpr int kCtasPerSm = ROWS == 256 ? 1 : 2;
+    static constexpr uint32_t kSmemBytesTmemA = kPfTmemBStages * kBBytes + 1024 + 256;  // x stages only
 };
 
 struct PrefillParams {
@@ -81,6 +83,24 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+// The same with A taken from tensor memory: lane i of a_tmem = row i of A, one 32-bit column = two consecutive k.
+__device__ __forceinline__ void umma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 16 consecutive 32-bit columns of this thread's TMEM lane (the warp's lane quarter) <- 16 registers.
+__device__ __forceinline__ void tmem_st_16cols(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 // Arrive on `bar` once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -260,6 +280,55 @@ __device__ __forceinline__ void group_store(uint32_t a_tile, const GroupRegs& r,
     }
 }
 
+// The same 32 weights as 16 bf16 pairs in k order in registers (for the kernel that keeps the weights in tensor memory).
+template <int FMT>
+__device__ __forceinline__ void group_convert(const GroupRegs& r, uint32_t (&out)[16]) {
+    const uint32_t words[4] = {r.codes.x, r.codes.y, r.codes.z, r.codes.w};
+    if (FmtTraits<FMT>::kMx) {
+        constexpr uint32_t kHi0 = 0x3F3F3F00u, kHi1 = 0x40404040u, kLo0 = 0xC0800000u, kLo1 = 0xC0804000u;
+        const uint32_t e = r.valid ? r.d_bits : 127u;
+        const uint32_t sc = e ? e << 7 : 0x0040u;
+        const uint32_t sc2 = sc | (sc << 16);
+#pragma unroll
+        for (int wi = 0; wi < 4; ++wi) {
+            const uint32_t w = words[wi];
+            const uint32_t mag = w & 0x77777777u, w4 = w << 4;
+            uint32_t hi_a = pf_prmt(kHi0, kHi1, mag), lo_a = pf_prmt(kLo0, kLo1, mag);
+            uint32_t hi_b = pf_prmt(kHi0, kHi1, mag >> 16), lo_b = pf_prmt(kLo0, kLo1, mag >> 16);
+            hi_a |= pf_prmt(w, w4, 0x1504u) & 0x80808080u;
+            hi_b |= pf_prmt(w, w4, 0x3726u) & 0x80808080u;
+            uint32_t o0 = pf_prmt(lo_a, hi_a, 0x5140u), o1 = pf_prmt(lo_a, hi_a, 0x7362u);
+            uint32_t o2 = pf_prmt(lo_b, hi_b, 0x5140u), o3 = pf_prmt(lo_b, hi_b, 0x7362u);
+            asm("mul.rn.bf16x2 %0, %0, %1;" : "+r"(o0) : "r"(sc2));
+            asm("mul.rn.bf16x2 %0, %0, %1;" : "+r"(o1) : "r"(sc2));
+            asm("mul.rn.bf16x2 %0, %0, %1;" : "+r"(o2) : "r"(sc2));
+            asm("mul.rn.bf16x2 %0, %0, %1;" : "+r"(o3) : "r"(sc2));
+            out[4 * wi] = o0;
+            out[4 * wi + 1] = o1;
+            out[4 * wi + 2] = o2;
+            out[4 * wi + 3] = o3;
+        }
+        return;
+    }
+    const float m = __uint_as_float(r.m_bits << 16);
+#pragma unroll
+    for (int wi = 0; wi < 4; ++wi) {
+        const uint32_t w = words[wi];
+        float f[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t q2 = ((w >> (4 * i)) & 0x000F000Fu) | 0x43004300u;
+            asm("sub.bf16x2 %0, %0, %1;" : "+r"(q2) : "r"(0x43004300u));
+            f[i] = dequant_lo(q2, r.d_bits, m);
+            f[i + 4] = dequant_hi(q2, r.d_bits, m);
+        }
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out[4 * wi]) : "f"(f[1]), "f"(f[0]));
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out[4 * wi + 1]) : "f"(f[3]), "f"(f[2]));
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out[4 * wi + 2]) : "f"(f[5]), "f"(f[4]));
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out[4 * wi + 3]) : "f"(f[7]), "f"(f[6]));
+    }
+}
+
 // ---- bf16 epilogues: the tile goes through shared memory so that global memory sees whole 128-byte lines --------------
 //
 // A thread owns one output feature (a TMEM lane) and many tokens, so 2-byte results written straight to y would reach
@@ -308,26 +377,39 @@ extern "C" __attribute__((visibility("default"))) int fdqp_pf_trace_clear() {
 // ROWS: output features per CTA tile.  256: the tile described above, one CTA per SM.  128 (for M <= 128): a 128 x 128
 // tile with half-size stages (16 KB + 16 KB), eight conversion warps and 128 TMEM columns, so that TWO CTAs share an SM:
 // one CTA's start-up, epilogue and stage latencies overlap the other's main loop.
-template <int FMT, int ROWS>
+// ATMEM (with ROWS = 128 only): the converted weights go to tensor memory (tcgen05.st) instead of shared memory and the
+// MMA takes its A operand from there, which removes the weights' store and re-read from the shared-memory traffic (at
+// <= 128 tokens per MMA that traffic is what the tensor pipe waits for).  Shared memory then holds x stages only (six of
+// them); TMEM holds the accumulators (128 columns) and four weight stages of 32 columns (64 k as bf16 pairs).
+template <int FMT, int ROWS, bool ATMEM = false>
 __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
     fdqp_prefill_kernel(const __grid_constant__ CUtensorMap x_map, const PrefillParams p) {
     using P = Pf1<ROWS>;
+    static_assert(!ATMEM || ROWS == 128, "weights in tensor memory: 128-row tiles only");
     constexpr int CH = P::kToks / 2;  // token columns per epilogue warp of a quarter
+    constexpr int NA = ATMEM ? kPfTmemAStages : kPfStages;    // weight stages
+    constexpr int NB = ATMEM ? kPfTmemBStages : kPfStages;    // x stages
+    constexpr uint32_t kBStride = ATMEM ? P::kBBytes : P::kStageBytes;  // bytes from one x stage to the next
+    constexpr uint32_t kBOff = ATMEM ? 0u : P::kABytes;                  // x tile inside its stage
+    constexpr uint32_t kRing = NB * kBStride;
+    constexpr uint32_t kTmemCols = ATMEM ? 256u : P::kTmemCols;
+    constexpr uint32_t kTmemA = 128;  // ATMEM: first TMEM column of the weight stages
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // tiles must start on a 1024-byte boundary (swizzle atom)
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    const uint32_t bars = base + kPfStages * P::kStageBytes;
-    // barriers: full_a[s], full_b[s], empty[s], acc_done; then the TMEM base address slot
+    const uint32_t bars = base + kRing;
+    // barriers: full_a[NA], full_b[NB], empty_a[NA], empty_b[NB], acc_done; then the TMEM base address slot
     auto full_a = [&](int s) { return bars + 8u * s; };
-    auto full_b = [&](int s) { return bars + 8u * (kPfStages + s); };
-    auto empty = [&](int s) { return bars + 8u * (2 * kPfStages + s); };
-    const uint32_t acc_done = bars + 8u * (3 * kPfStages);
+    auto full_b = [&](int s) { return bars + 8u * (NA + s); };
+    auto empty_a = [&](int s) { return bars + 8u * (NA + NB + s); };
+    auto empty_b = [&](int s) { return bars + 8u * (2 * NA + NB + s); };
+    const uint32_t acc_done = bars + 8u * (2 * NA + 2 * NB);
     const uint32_t tmem_slot = acc_done + 8u;
     const uint32_t staged = tmem_slot + 8u;  // bf16 epilogues: every epilogue warp has written its part of the tile
-    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(smem + kPfStages * P::kStageBytes + 8 * (3 * kPfStages + 1));
+    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(smem + kRing + 8 * (2 * NA + 2 * NB + 1));
 
     const int tok_tiles = (p.M + P::kToks - 1) / P::kToks;
     const int tile_id = blockIdx.x / p.Z, z = blockIdx.x % p.Z;                    // K slices of one tile adjacent
@@ -342,17 +424,20 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
     if (tid == 0) PF_STAMP(0);
 
     if (tid == 0) {
-        for (int s = 0; s < kPfStages; ++s) {
+        for (int s = 0; s < NA; ++s) {
             mbar_init(full_a(s), P::kDequantWarps);
+            mbar_init(empty_a(s), 1);
+        }
+        for (int s = 0; s < NB; ++s) {
             mbar_init(full_b(s), 1);
-            mbar_init(empty(s), 1);
+            mbar_init(empty_b(s), 1);
         }
         mbar_init(acc_done, 1);
         mbar_init(staged, P::kDequantWarps);
         mbar_fence_init();
     }
     if (warp == 0) {
-        tmem_alloc(tmem_slot, P::kTmemCols);
+        tmem_alloc(tmem_slot, kTmemCols);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -366,11 +451,11 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
         // =============================== TMA producer: x tiles ==============================================
         if (lane == 0) {
             for (int i = 0; i < ksteps && ok; ++i) {
-                const int s = i % kPfStages;
-                if (i >= kPfStages) ok = mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status);
+                const int s = i % NB;
+                if (i >= NB) ok = mbar_wait(empty_b(s), ((i / NB) - 1) & 1, p.status);
                 if (!ok) break;
                 mbar_arrive_expect_tx(full_b(s), P::kBBytes);
-                tma_load_2d(base + s * P::kStageBytes + P::kABytes, &x_map, (ks0 + i) * kPfK, tok0, full_b(s));
+                tma_load_2d(base + s * kBStride + kBOff, &x_map, (ks0 + i) * kPfK, tok0, full_b(s));
             }
         }
     } else if (warp == 1) {
@@ -378,17 +463,17 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
         if (lane == 0) {
             const uint32_t idesc = umma_idesc(n_inst);
             for (int i = 0; i < ksteps && ok; ++i) {
-                const int s = i % kPfStages;
-                const uint32_t ph = (i / kPfStages) & 1;
+                const int sa = i % NA, sb = i % NB;
+                const uint32_t pha = (i / NA) & 1, phb = (i / NB) & 1;
 #ifdef FDQP_TRACE
                 {
                     PF_T0();
-                    ok = mbar_wait(full_a(s), ph, p.status);
+                    ok = mbar_wait(full_a(sa), pha, p.status);
                     PF_ADD(12, PF_DT());
                 }
                 {
                     PF_T0();
-                    ok = ok && mbar_wait(full_b(s), ph, p.status);
+                    ok = ok && mbar_wait(full_b(sb), phb, p.status);
                     PF_ADD(13, PF_DT());
                 }
                 if (i == 0) PF_STAMP(2);
@@ -396,23 +481,32 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
                 if (i == 20) PF_STAMP(4);
                 if (i == 30) PF_STAMP(5);
 #else
-                ok = mbar_wait(full_a(s), ph, p.status) && mbar_wait(full_b(s), ph, p.status);
+                ok = mbar_wait(full_a(sa), pha, p.status) && mbar_wait(full_b(sb), phb, p.status);
 #endif
                 if (!ok) break;
 #ifdef FDQP_TRACE
                 const unsigned long long pf_m0 = globaltimer_ns();
 #endif
                 tc_fence_after();
-                const uint32_t a_addr = base + s * P::kStageBytes, b_addr = a_addr + P::kABytes;
-#pragma unroll
-                for (int half = 0; half < ROWS / 128; ++half) {
-                    const uint64_t adesc = umma_smem_desc(a_addr + half * (128 * kPfK * 2));
+                const uint32_t a_addr = base + sa * P::kStageBytes, b_addr = base + sb * kBStride + kBOff;
+                if (ATMEM) {
                     const uint64_t bdesc = umma_smem_desc(b_addr);
 #pragma unroll
-                    for (int k4 = 0; k4 < kPfK / 16; ++k4)  // 32 bytes (16 bf16) further along the swizzled row
-                        umma_bf16(tmem_base + half * 256, adesc + 2 * k4, bdesc + 2 * k4, idesc, (i | k4) != 0);
+                    for (int k4 = 0; k4 < kPfK / 16; ++k4)  // eight TMEM columns (16 bf16) further along the weights' rows
+                        umma_bf16_ta(tmem_base, tmem_base + kTmemA + (uint32_t)(sa * (kPfK / 2) + 8 * k4), bdesc + 2 * k4, idesc,
+                                     (i | k4) != 0);
+                } else {
+#pragma unroll
+                    for (int half = 0; half < ROWS / 128; ++half) {
+                        const uint64_t adesc = umma_smem_desc(a_addr + half * (128 * kPfK * 2));
+                        const uint64_t bdesc = umma_smem_desc(b_addr);
+#pragma unroll
+                        for (int k4 = 0; k4 < kPfK / 16; ++k4)  // 32 bytes (16 bf16) further along the swizzled row
+                            umma_bf16(tmem_base + half * 256, adesc + 2 * k4, bdesc + 2 * k4, idesc, (i | k4) != 0);
+                    }
                 }
-                umma_commit(empty(s));  // the stage may be refilled once these MMAs have read it
+                umma_commit(empty_a(sa));  // the stages may be refilled once these MMAs have read them
+                umma_commit(empty_b(sb));
 #ifdef FDQP_TRACE
                 PF_ADD(14, globaltimer_ns() - pf_m0);
 #endif
@@ -423,7 +517,8 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
     } else {
         // =============================== dequantisation warps ================================================
         const int dw = warp - 2;
-        const int sl = dw >> 1, gl = dw & 1;  // strip of the tile and group of the 64-k stage this warp converts
+        // strip of the tile and group of the 64-k stage this warp converts (ATMEM: the strip is the warp's TMEM lane quarter)
+        const int sl = ATMEM ? (warp & 3) : (dw >> 1), gl = ATMEM ? (dw >> 2) : (dw & 1);
         const int64_t strip = (int64_t)n_tile * (P::kRows / 32) + sl;
         const bool strip_ok = strip < p.N / kStripRows;
         // the loads of the next three stages are in flight while this one is converted (a stage lasts about as long
@@ -432,18 +527,28 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
         // Three register sets, each reloaded right after it has been converted.  (Rotating the sets with moves instead --
         // g0 = g1; g1 = g2; g2 = just-loaded -- makes the move wait for the load it follows, one trip to memory per k-step.)
         auto convert_step = [&](int i, const GroupRegs& g) -> bool {
-            const int s = i % kPfStages;
+            const int s = i % NA;
 #ifdef FDQP_TRACE
             const unsigned long long pf_w0 = globaltimer_ns();
 #endif
-            if (i >= kPfStages && !mbar_wait(empty(s), ((i / kPfStages) - 1) & 1, p.status)) return false;
+            if (i >= NA && !mbar_wait(empty_a(s), ((i / NA) - 1) & 1, p.status)) return false;
             if (dw == 0 && lane == 0 && i == 0) PF_STAMP(10);
 #ifdef FDQP_TRACE
             const unsigned long long pf_w1 = globaltimer_ns();
 #endif
-            group_store<FMT>(base + s * P::kStageBytes, g, sl, gl, lane);
-            // make the generic-proxy stores visible to the tensor core's (async-proxy) reads, then signal
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            if (ATMEM) {
+                // this lane's row of the group, 16 bf16 pairs, into its TMEM lane; ordered against the MMAs that read the
+                // stage before (the barrier wait above) and after (the arrive below) by the tensor-core fences
+                uint32_t wreg[16];
+                group_convert<FMT>(g, wreg);
+                tc_fence_after();
+                tmem_st_16cols(tmem_base + ((uint32_t)(sl * 32) << 16) + kTmemA + (uint32_t)(s * (kPfK / 2) + gl * 16), wreg);
+                tc_fence_before();
+            } else {
+                group_store<FMT>(base + s * P::kStageBytes, g, sl, gl, lane);
+                // make the generic-proxy stores visible to the tensor core's (async-proxy) reads, then signal
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(full_a(s));
 #ifdef FDQP_TRACE
@@ -542,7 +647,7 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
     __syncthreads();
     if (warp == 0) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, P::kTmemCols);
+        tmem_dealloc(tmem_base, kTmemCols);
     }
     if (tid == 0) PF_STAMP(9);
 }
@@ -895,6 +1000,7 @@ static cudaError_t prefill_set_smem_limit_fmt() {
     cudaError_t e = cudaFuncSetAttribute(fdqp_prefill_kernel<FMT, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Pf1<256>::kSmemBytes);
     if (e) return e;
     if ((e = cudaFuncSetAttribute(fdqp_prefill_kernel<FMT, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Pf1<128>::kSmemBytes))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_prefill_kernel<FMT, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Pf1<128>::kSmemBytesTmemA))) return e;
     return cudaFuncSetAttribute(fdqp_prefill_pair_kernel<FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kP2SmemBytes);
 }
 
@@ -907,8 +1013,8 @@ cudaError_t prefill_set_smem_limit() {
 }
 
 template <int FMT>
-static cudaError_t prefill_launch_kernels(const CUtensorMap& map, const PrefillParams& p, int pair, int M, int N, int Z,
-                                          cudaStream_t stream) {
+static cudaError_t prefill_launch_kernels(const CUtensorMap& map, const PrefillParams& p, int pair, int a_tmem, int M, int N,
+                                          int Z, cudaStream_t stream) {
     if (pair) {
         const int n_tiles = (N + 2 * kP2Rows - 1) / (2 * kP2Rows), tok_tiles = (M + kP2Toks - 1) / kP2Toks;
         cudaLaunchConfig_t cfg = {};
@@ -927,7 +1033,10 @@ static cudaError_t prefill_launch_kernels(const CUtensorMap& map, const PrefillP
     }
     if (pair == 0 && M <= Pf1<128>::kToks) {  // small tiles, two CTAs per SM
         const int n_tiles = (N + 127) / 128;
-        fdqp_prefill_kernel<FMT, 128><<<n_tiles * Z, Pf1<128>::kThreads, Pf1<128>::kSmemBytes, stream>>>(map, p);
+        if (a_tmem)
+            fdqp_prefill_kernel<FMT, 128, true><<<n_tiles * Z, Pf1<128>::kThreads, Pf1<128>::kSmemBytesTmemA, stream>>>(map, p);
+        else
+            fdqp_prefill_kernel<FMT, 128><<<n_tiles * Z, Pf1<128>::kThreads, Pf1<128>::kSmemBytes, stream>>>(map, p);
         return cudaGetLastError();
     }
     const int n_tiles = (N + kPfRows - 1) / kPfRows, tok_tiles = (M + kPfToks - 1) / kPfToks;
@@ -943,7 +1052,7 @@ static cudaError_t prefill_launch_kernels(const CUtensorMap& map, const PrefillP
 // epi: kEpiNone writes fp32 y; the other epilogues write bf16 to y16 (see fdqp_plan.h).
 // fmt: the container's format (fdqp_format.h).
 cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, uint16_t* y16, int epi, float* ws,
-                           int* status, int M, int K, int N, int pair, int Z, int fmt, cudaStream_t stream) {
+                           int* status, int M, int K, int N, int pair, int Z, int fmt, int a_tmem, cudaStream_t stream) {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     CUtensorMap map;
@@ -971,10 +1080,10 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_by
     Z = p.Z;
     cudaError_t err;
     switch (fmt) {
-        case kFmtQ4nx: err = prefill_launch_kernels<kFmtQ4nx>(map, p, pair, M, N, Z, stream); break;
-        case kFmtG64: err = prefill_launch_kernels<kFmtG64>(map, p, pair, M, N, Z, stream); break;
-        case kFmtG128: err = prefill_launch_kernels<kFmtG128>(map, p, pair, M, N, Z, stream); break;
-        case kFmtMxfp4: err = prefill_launch_kernels<kFmtMxfp4>(map, p, pair, M, N, Z, stream); break;
+        case kFmtQ4nx: err = prefill_launch_kernels<kFmtQ4nx>(map, p, pair, a_tmem, M, N, Z, stream); break;
+        case kFmtG64: err = prefill_launch_kernels<kFmtG64>(map, p, pair, a_tmem, M, N, Z, stream); break;
+        case kFmtG128: err = prefill_launch_kernels<kFmtG128>(map, p, pair, a_tmem, M, N, Z, stream); break;
+        case kFmtMxfp4: err = prefill_launch_kernels<kFmtMxfp4>(map, p, pair, a_tmem, M, N, Z, stream); break;
         default: return cudaErrorInvalidValue;
     }
     if (err != cudaSuccess || Z == 1) return err;

@@ -118,6 +118,13 @@ def test_prefill_tensor_path_matches_oracle(fresh, K, N, M):
     assert ("fdqp_prefill_kernel" if M > 256 else "fdqp_prefill_pair_kernel") in fd.fdqp_describe(fresh, M, K, N)
     assert_close(case.run(fresh), y_ref, a_ref, f"prefill (other tile) K={K} N={N} M={M}")
     fd.fdqp_set_param(fresh, "prefill_pair", -1)
+    if M <= 128:
+        # up to 128 token rows the converted weights live in tensor memory by default; in shared memory: the same bits
+        assert "weights in TMEM" in fd.fdqp_describe(fresh, M, K, N)
+        fd.fdqp_set_param(fresh, "prefill_a_tmem", 0)
+        assert "weights in TMEM" not in fd.fdqp_describe(fresh, M, K, N)
+        assert np.array_equal(case.run(fresh), y)
+        fd.fdqp_set_param(fresh, "prefill_a_tmem", 1)
     # the same rows through the GEMV kernel, eight at a time: both are within the bound of the oracle
     fd.fdqp_set_param(fresh, "path", 2)
     assert "fdqp_gemv_kernel" in fd.fdqp_describe(fresh, M, K, N)
