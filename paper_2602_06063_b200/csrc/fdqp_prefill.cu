@@ -462,6 +462,9 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
         // =============================== MMA issuer =========================================================
         if (lane == 0) {
             const uint32_t idesc = umma_idesc(n_inst);
+#ifdef FDQP_TRACE
+            unsigned long long tr_wa = 0, tr_wb = 0, tr_is = 0;
+#endif
             for (int i = 0; i < ksteps && ok; ++i) {
                 const int sa = i % NA, sb = i % NB;
                 const uint32_t pha = (i / NA) & 1, phb = (i / NB) & 1;
@@ -469,17 +472,14 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
                 {
                     PF_T0();
                     ok = mbar_wait(full_a(sa), pha, p.status);
-                    PF_ADD(12, PF_DT());
+                    tr_wa += PF_DT();
                 }
                 {
                     PF_T0();
                     ok = ok && mbar_wait(full_b(sb), phb, p.status);
-                    PF_ADD(13, PF_DT());
+                    tr_wb += PF_DT();
                 }
                 if (i == 0) PF_STAMP(2);
-                if (i == 10) PF_STAMP(3);
-                if (i == 20) PF_STAMP(4);
-                if (i == 30) PF_STAMP(5);
 #else
                 ok = mbar_wait(full_a(sa), pha, p.status) && mbar_wait(full_b(sb), phb, p.status);
 #endif
@@ -508,10 +508,15 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
                 umma_commit(empty_a(sa));  // the stages may be refilled once these MMAs have read them
                 umma_commit(empty_b(sb));
 #ifdef FDQP_TRACE
-                PF_ADD(14, globaltimer_ns() - pf_m0);
+                tr_is += globaltimer_ns() - pf_m0;
 #endif
             }
             PF_STAMP(6);
+#ifdef FDQP_TRACE
+            PF_ADD(12, tr_wa);
+            PF_ADD(13, tr_wb);
+            PF_ADD(14, tr_is);
+#endif
             umma_commit(acc_done);
         }
     } else {
@@ -526,6 +531,9 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
         const int gbase = 2 * ks0 + gl;  // this warp's group in k-step i of the slice: gbase + 2 i
         // Three register sets, each reloaded right after it has been converted.  (Rotating the sets with moves instead --
         // g0 = g1; g1 = g2; g2 = just-loaded -- makes the move wait for the load it follows, one trip to memory per k-step.)
+#ifdef FDQP_TRACE
+        unsigned long long tr_wait = 0, tr_conv = 0, tr_st = 0, tr_arr = 0, tr_load = 0;
+#endif
         auto convert_step = [&](int i, const GroupRegs& g) -> bool {
             const int s = i % NA;
 #ifdef FDQP_TRACE
@@ -541,9 +549,18 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
                 // stage before (the barrier wait above) and after (the arrive below) by the tensor-core fences
                 uint32_t wreg[16];
                 group_convert<FMT>(g, wreg);
+#ifdef FDQP_TRACE
+                asm volatile("" ::"r"(wreg[0]), "r"(wreg[15]));
+                const unsigned long long pf_c1 = globaltimer_ns();
+                tr_conv += pf_c1 - pf_w1;
+#endif
                 tc_fence_after();
                 tmem_st_16cols(tmem_base + ((uint32_t)(sl * 32) << 16) + kTmemA + (uint32_t)(s * (kPfK / 2) + gl * 16), wreg);
                 tc_fence_before();
+#ifdef FDQP_TRACE
+                const unsigned long long pf_c2 = globaltimer_ns();
+                tr_st += pf_c2 - pf_c1;
+#endif
             } else {
                 group_store<FMT>(base + s * P::kStageBytes, g, sl, gl, lane);
                 // make the generic-proxy stores visible to the tensor core's (async-proxy) reads, then signal
@@ -552,10 +569,8 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
             __syncwarp();
             if (lane == 0) mbar_arrive(full_a(s));
 #ifdef FDQP_TRACE
-            if (dw == 0 && lane == 0) {
-                PF_ADD(11, pf_w1 - pf_w0);
-                PF_ADD(15, globaltimer_ns() - pf_w1);
-            }
+            tr_wait += pf_w1 - pf_w0;
+            tr_arr += globaltimer_ns() - pf_w1;
 #endif
             return true;
         };
@@ -564,7 +579,13 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
         GroupRegs g2 = group_load<FMT>(p.W, p.K, strip, gbase + 4, lane, strip_ok);
         for (int i = 0; i < ksteps && ok; i += 3) {
             ok = convert_step(i, g0);
+#ifdef FDQP_TRACE
+            const unsigned long long pf_l0 = globaltimer_ns();
+#endif
             g0 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
+#ifdef FDQP_TRACE
+            tr_load += globaltimer_ns() - pf_l0;
+#endif
             if (ok && i + 1 < ksteps) {
                 ok = convert_step(i + 1, g1);
                 g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 4), lane, strip_ok);
@@ -574,6 +595,15 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
                 g2 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 5), lane, strip_ok);
             }
         }
+#ifdef FDQP_TRACE
+        if (dw == 0 && lane == 0) {
+            PF_ADD(11, tr_wait);
+            PF_ADD(3, tr_conv);
+            PF_ADD(4, tr_st);
+            PF_ADD(15, tr_arr);
+            PF_ADD(5, tr_load);
+        }
+#endif
         // =============================== epilogue: TMEM -> y =================================================
         if (ok) ok = mbar_wait(acc_done, 0, p.status);
         ok = __all_sync(0xffffffffu, ok);
