@@ -460,7 +460,10 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
         }
     } else if (warp == 1) {
         // =============================== MMA issuer =========================================================
-        if (lane == 0) {
+        // The whole warp runs the loop on warp-uniform values (so that the descriptors can live in uniform registers,
+        // which is where the tensor-core instructions take them from); lane 0 issues.
+        {
+            const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot_g, 0);
             const uint32_t idesc = umma_idesc(n_inst);
 #ifdef FDQP_TRACE
             unsigned long long tr_wa = 0, tr_wb = 0, tr_is = 0;
@@ -479,16 +482,18 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
                     ok = ok && mbar_wait(full_b(sb), phb, p.status);
                     tr_wb += PF_DT();
                 }
-                if (i == 0) PF_STAMP(2);
+                if (i == 0 && lane == 0) PF_STAMP(2);
 #else
                 ok = mbar_wait(full_a(sa), pha, p.status) && mbar_wait(full_b(sb), phb, p.status);
 #endif
+                ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
 #ifdef FDQP_TRACE
                 const unsigned long long pf_m0 = globaltimer_ns();
 #endif
                 tc_fence_after();
                 const uint32_t a_addr = base + sa * P::kStageBytes, b_addr = base + sb * kBStride + kBOff;
+                if (lane != 0) continue;
                 if (ATMEM) {
                     const uint64_t bdesc = umma_smem_desc(b_addr);
 #pragma unroll
@@ -511,13 +516,15 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
                 tr_is += globaltimer_ns() - pf_m0;
 #endif
             }
-            PF_STAMP(6);
+            if (lane == 0) {
+                PF_STAMP(6);
 #ifdef FDQP_TRACE
-            PF_ADD(12, tr_wa);
-            PF_ADD(13, tr_wb);
-            PF_ADD(14, tr_is);
+                PF_ADD(12, tr_wa);
+                PF_ADD(13, tr_wb);
+                PF_ADD(14, tr_is);
 #endif
-            umma_commit(acc_done);
+                umma_commit(acc_done);
+            }
         }
     } else {
         // =============================== dequantisation warps ================================================
