@@ -56,6 +56,7 @@ struct fdqp_ctx {
     std::string last_err;
     // overrides (-1 = automatic)
     int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1, p_prep = -1, p_aligned = -1, p_bpw = -1, p_pair = -1, p_pf_split = -1;
+    int64_t p_direct_y = 1;  // fdqp_run_host*: small results are stored straight into device-addressable host memory
     int64_t p_atmem = 1;  // tensor-core kernel up to 128 tokens: keep the converted weights in tensor memory
 };
 
@@ -68,6 +69,7 @@ constexpr int kMaxStages = 40;
 constexpr int64_t kSpreadBelowBytes = 128 << 10;
 constexpr int64_t kSpreadToBytes = 256 << 10;
 constexpr size_t kSpreadBufBytes = (size_t)kSpreadToBytes + 256 * 128;  // row distance rounds up to 128 bytes, M <= 256 here
+constexpr size_t kDirectHostBytes = 1u << 20;  // results up to this size go straight to addressable host memory
 constexpr int kKvMaxHeads = 64, kKvMaxSplits = 148, kKvMaxDim = 256;  // decode attention workspace
 constexpr size_t kPrefillWsCap = 128u << 20;  // bytes of partial results a context keeps for K-split tensor-core calls
 constexpr int kMinStages = 3;  // ring depth below which another K slice is preferred
@@ -528,9 +530,21 @@ extern "C" fdqp_status fdqp_run_host_async(fdqp_ctx* ctx, const void* x_host_bf1
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if ((e = cudaMemcpyAsync(ctx->x_stage, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, stream)))
         return cuda_fail(ctx, e, "x copy");
-    st = fdqp_run(ctx, ctx->x_stage, W_q4nx, ctx->y_stage, M, K, N, cuda_stream);
+    // Small results in page-locked host memory that the device can address are stored there by the kernels themselves
+    // (posted writes over the bus, a few microseconds for tens of kilobytes): no copy-out to launch and wait for.
+    // y is write-only for every kernel.  Otherwise: the staging buffer and a copy.
+    float* y_dev = ctx->y_stage;
+    if ((size_t)M * N * 4 <= kDirectHostBytes && ctx->p_direct_y != 0) {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, y_host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer &&
+            aligned16(attr.devicePointer))
+            y_dev = static_cast<float*>(attr.devicePointer);
+        else
+            cudaGetLastError();
+    }
+    st = fdqp_run(ctx, ctx->x_stage, W_q4nx, y_dev, M, K, N, cuda_stream);
     if (st != FDQP_OK) return st;
-    if ((e = cudaMemcpyAsync(y_host, ctx->y_stage, (size_t)M * N * 4, cudaMemcpyDeviceToHost, stream)))
+    if (y_dev == ctx->y_stage && (e = cudaMemcpyAsync(y_host, ctx->y_stage, (size_t)M * N * 4, cudaMemcpyDeviceToHost, stream)))
         return cuda_fail(ctx, e, "y copy");
     return FDQP_OK;
 }
@@ -606,6 +620,9 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
     } else if (!std::strcmp(key, "prefill_split_k")) {
         if (v == 0 || v > kMaxSplit) return FDQP_ERR_ARG;
         ctx->p_pf_split = v;
+    } else if (!std::strcmp(key, "host_direct_y")) {
+        if (v != 0 && v != 1) return FDQP_ERR_ARG;
+        ctx->p_direct_y = v;
     } else if (!std::strcmp(key, "prefill_a_tmem")) {
         if (v != 0 && v != 1) return FDQP_ERR_ARG;
         ctx->p_atmem = v;
