@@ -255,10 +255,11 @@ FDQP_API fdqp_status fdqp_flowkv_decode(fdqp_ctx* ctx, const void* q_bf16, const
  * to the context's device staging buffer, runs fdqp_run, copies y back to `y_host`
  * (host, [M][N] fp32) and synchronises the stream before returning.  W stays a
  * device pointer (weights are resident model state).  Pinned host memory makes
- * the copies asynchronous but is not required.  When y_host is page-locked memory
- * the device can address (e.g. cudaHostAlloc) and the result is at most 1 MiB, the
- * kernels store y there themselves and no copy-out is issued ("host_direct_y"
- * parameter, default 1). */
+ * the copies asynchronous but is not required.  Page-locked buffers the device can
+ * address (e.g. cudaHostAlloc) of at most 1 MiB are used in place ("host_direct_y"
+ * parameter, default 1): the kernels store y there themselves, and up to eight
+ * token rows of x are read from there by the activation-preparation kernel; no
+ * copy is issued for them. */
 FDQP_API fdqp_status fdqp_run_host(fdqp_ctx* ctx, const void* x_host_bf16, const void* W_q4nx, float* y_host,
                           int64_t M, int64_t K, int64_t N, void* cuda_stream);
 
@@ -347,8 +348,8 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "prefill_pair"  1 = prefill-sized calls use the two-SM kernel (256 x 512 tile per CTA pair), 0 = the one-SM kernel
  *                   (256 x 256 tile; 128 x 128 tiles, two CTAs per SM, up to 128 token rows); default: two-SM kernel
  *                   when M > 256
- *   "host_direct_y" fdqp_run_host*: 1 (default) = small results are stored by the kernels straight into
- *                   device-addressable page-locked host memory, 0 = always through the staging buffer and a copy
+ *   "host_direct_y" fdqp_run_host*: 1 (default) = small x and y in device-addressable page-locked host memory are
+ *                   read / written in place by the kernels, 0 = always through the staging buffers and copies
  *   "prefill_a_tmem" one-SM tensor-core kernel up to 128 token rows: 1 (default) = the converted weights are kept in
  *                   tensor memory and read from there by the MMAs, 0 = in shared memory; same results bit for bit
  *   "debug"         measurement aid: 1 = the GEMV consumers skip the arithmetic (y is then undefined)

@@ -528,7 +528,22 @@ extern "C" fdqp_status fdqp_run_host_async(fdqp_ctx* ctx, const void* x_host_bf1
         if ((e = cudaMalloc(&ctx->y_stage, (size_t)ctx->max_M * ctx->max_N * 4))) return cuda_fail(ctx, e, "y staging");
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if ((e = cudaMemcpyAsync(ctx->x_stage, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, stream)))
+    // Decode-sized x in page-locked host memory that the device can address is read from there by the activation
+    // preparation kernel (a few kilobytes over the bus, once), instead of being copied to the device first: the copy
+    // engine's start-up costs more than the kernel.  The GEMV kernels themselves then never touch x.
+    const void* x_dev = ctx->x_stage;
+    bool direct_x = false;
+    if (M <= kMaxTokens && (size_t)M * K * 2 <= kDirectHostBytes && ctx->p_direct_y != 0 && ctx->p_path != 1) {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, x_host_bf16) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer &&
+            aligned16(attr.devicePointer)) {
+            x_dev = attr.devicePointer;
+            direct_x = true;
+        } else {
+            cudaGetLastError();
+        }
+    }
+    if (!direct_x && (e = cudaMemcpyAsync(ctx->x_stage, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, stream)))
         return cuda_fail(ctx, e, "x copy");
     // Small results in page-locked host memory that the device can address are stored there by the kernels themselves
     // (posted writes over the bus, a few microseconds for tens of kilobytes): no copy-out to launch and wait for.
@@ -542,7 +557,10 @@ extern "C" fdqp_status fdqp_run_host_async(fdqp_ctx* ctx, const void* x_host_bf1
         else
             cudaGetLastError();
     }
-    st = fdqp_run(ctx, ctx->x_stage, W_q4nx, y_dev, M, K, N, cuda_stream);
+    const int64_t saved_prep = ctx->p_prep;
+    if (direct_x) ctx->p_prep = 0;  // x is read once, by the preparation kernel
+    st = fdqp_run(ctx, x_dev, W_q4nx, y_dev, M, K, N, cuda_stream);
+    ctx->p_prep = saved_prep;
     if (st != FDQP_OK) return st;
     if (y_dev == ctx->y_stage && (e = cudaMemcpyAsync(y_host, ctx->y_stage, (size_t)M * N * 4, cudaMemcpyDeviceToHost, stream)))
         return cuda_fail(ctx, e, "y copy");

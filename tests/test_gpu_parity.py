@@ -320,18 +320,16 @@ def test_run_host_roundtrip(fresh):
 @pytest.mark.parametrize("K,N,M,params", [(2560, 2048, 1, {}), (21504, 320, 2, {}), (1056, 320, 20, {"path": 3}),
                                           (2560, 4096, 5, {}), (512, 288, 300, {"path": 3})])
 def test_run_host_result_paths_agree(fresh, K, N, M, params):
-    """Pinned (device-addressable) host results are stored by the kernels themselves when small; pageable host memory
-    and the staged route give the same bits, on every kernel family (whole strips, K slices with their sum kernel, the
-    tensor-core kernels)."""
+    """Pinned (device-addressable) host buffers are used in place when small -- x read by the preparation kernel (up to
+    eight token rows), y stored by the kernels themselves; pageable host memory and the staged route give the same bits,
+    on every kernel family (whole strips, K slices with their sum kernel, the tensor-core kernels)."""
     case = Case(K, N, M, seed=980 + K + M, amp=1.0 / np.sqrt(K) if K > 20000 else 1.0)
     for k, v in params.items():
         fd.fdqp_set_param(fresh, k, v)
     ref = case.run(fresh)
     x_pin = torch.from_numpy(case.x.view(np.int16)).pin_memory()
     y_pin = torch.full((M, N), float("nan"), dtype=torch.float32).pin_memory()
-    before = fd.fdqp_launch_count(fresh)
     fd.fdqp_run_host(fresh, x_pin, case.W_dev, y_pin, M, K, N)
-    direct_launches = fd.fdqp_launch_count(fresh) - before
     assert np.array_equal(y_pin.numpy(), ref)
     y_page = torch.full((M, N), float("nan"), dtype=torch.float32)           # pageable: staged, then copied
     fd.fdqp_run_host(fresh, torch.from_numpy(case.x.view(np.int16)), case.W_dev, y_page, M, K, N)
@@ -339,9 +337,7 @@ def test_run_host_result_paths_agree(fresh, K, N, M, params):
     fd.fdqp_set_param(fresh, "host_direct_y", 0)
     try:
         y_staged = torch.full((M, N), float("nan"), dtype=torch.float32).pin_memory()
-        before = fd.fdqp_launch_count(fresh)
         fd.fdqp_run_host(fresh, x_pin, case.W_dev, y_staged, M, K, N)
-        assert fd.fdqp_launch_count(fresh) - before == direct_launches
         assert np.array_equal(y_staged.numpy(), ref)
     finally:
         fd.fdqp_set_param(fresh, "host_direct_y", 1)
