@@ -541,7 +541,7 @@ def run_ours(args, rank, local_rank, world):
                   "decode_tokens_per_s": M8 * 1e3 / (synthgen.GEMMA3_4B_LAYERS * layer8_ms + head8_ms)}
         del xs8, ys8, hx8, hy8
 
-    # ---- LM head at a prefill chunk (M = 512, BASELINE configs[4]): the tensor-core path, against the tensor roofline
+    # ---- LM head at a prefill chunk (M = 512, the largest baseline configuration): the tensor-core path, against the tensor roofline
     prefill = None
     if rank == 0 and not args.no_head:
         PM = 512
