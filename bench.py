@@ -251,6 +251,43 @@ def run_shape(args):
 
 # ----------------------------------------------------------------------------------------------- decode attention
 
+def run_dequant(args):
+    """Times the dequantisation engine (--dequant K,N,bf16|fp32): Q4NX -> dense matrix in HBM.  Algorithmic bytes per
+    weight: 0.625 read + 2 (bf16) or 4 (fp32) written."""
+    import torch
+
+    import paper_2602_06063_b200 as fd
+
+    parts = args.dequant.split(",")
+    K, N, bf16 = int(parts[0]), int(parts[1]), parts[2] == "bf16"
+    torch.cuda.set_device(0)
+    peaks, peak_kind = measured_peaks()
+    ctx = fd.fdqp_create(0, 8, K, N)
+    fmt = {"q4nx": fd.FMT_Q4NX, "g64": fd.FMT_G64, "g128": fd.FMT_G128, "mxfp4": fd.FMT_MXFP4}[args.format]
+    nb = min(N, 4096)
+    w = synthgen.weights_fmt(5, K, nb, fmt) if fmt != fd.FMT_Q4NX else synthgen.weights(5, K, nb)
+    tile = fd.q4nx_pack_fmt(fmt, w.codes, w.scales, w.offsets)
+    nbytes = fd.q4nx_packed_bytes_fmt(fmt, K, N)
+    W = torch.from_numpy(np.tile(tile, -(-N // nb))[:nbytes].copy()).cuda()
+    out = torch.empty((K, N), dtype=torch.bfloat16 if bf16 else torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    sraw = stream.cuda_stream
+    for _ in range(3):
+        fd.fdqp_dequant_fmt(ctx, fmt, W, out, bf16, K, N, sraw)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        fd.fdqp_dequant_fmt(ctx, fmt, W, out, bf16, K, N, sraw)
+    e1.record(stream)
+    stream.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / args.steps
+    alg = nbytes + float(K) * N * (2 if bf16 else 4)
+    gbs = alg / us / 1e3
+    print(json.dumps({"dequant": {"K": K, "N": N, "out": parts[2], "format": args.format}, "us_per_call": us, "GBps": gbs,
+                      "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "peak_kind": peak_kind, "steps": args.steps}), flush=True)
+    fd.fdqp_destroy(ctx)
+
+
 def run_flowkv(args):
     """Times the decode attention (--flowkv H,G,d,L,window): one new token against a cache of L positions.  Enough
     distinct caches are rotated to keep every launch's keys and values out of L2.  Algorithmic bytes per call: the
@@ -699,6 +736,7 @@ def main():
     ap.add_argument("--param", action="append", help="library launch parameter key=value (repeatable)")
     ap.add_argument("--shape", help="K,N,M: time this one projection shape instead of the layer workload")
     ap.add_argument("--same-weights", action="store_true", help="with --shape: reuse one weight buffer (for ncu captures)")
+    ap.add_argument("--dequant", help="K,N,bf16|fp32: time the dequantisation engine (container -> dense matrix) instead")
     ap.add_argument("--flowkv", help="H,G,d,L,window: time the decode attention over a KV cache instead of a projection")
     ap.add_argument("--rmsnorm", action="store_true", help="with --shape: RMS-normalise x first (fused where possible)")
     ap.add_argument("--epilogue", default="none", choices=["none", "bf16", "geglu"],
@@ -722,6 +760,11 @@ def main():
         return
     if args.warmup < 3:
         args.warmup = 3
+    if args.dequant:
+        if args.steps == 8000:
+            args.steps = 10
+        run_dequant(args)
+        return
     if args.flowkv:
         if args.steps == 8000:
             args.steps = 50

@@ -1,51 +1,20 @@
-// Plain CUDA-core kernels: the dequantisation engine (Sec. "Dequantization Engine", Eq. 3) and a
-// straightforward dequantise-then-multiply projection (Eq. 14) that serves as the library's
-// self-check path ("path" = 1).  Neither is tuned; both read the container with plain loads.
+// Plain CUDA-core kernels: the dequantisation engine (Sec. "Dequantization Engine", Eq. 3; bound by its writes) and a
+// straightforward dequantise-then-multiply projection (Eq. 14) that serves as the library's self-check path
+// ("path" = 1; not tuned).  Both read the container with plain loads.
 #include "fdqp_device.cuh"
 #include "fdqp_format.h"
 #include "fdqp_plan.h"
 
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 namespace fdqp {
 
 __device__ __forceinline__ float bf16_bits_to_f32(uint16_t h) { return __uint_as_float(((uint32_t)h) << 16); }
 
-// One warp per (strip, group): lane = output row.  out is [K][N]; the 32 lanes of a warp write 32
-// consecutive n for each k, so every store is one full 128-byte (fp32) or 64-byte (bf16) line.
-template <bool OUT_BF16>
-__global__ void __launch_bounds__(256) fdqp_dequant_kernel(const uint8_t* __restrict__ W, void* __restrict__ out, int K,
-                                                           int N) {
-    const int lane = threadIdx.x & 31;
-    const int groups = K / kGroup;
-    const int64_t unit = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int64_t total = (int64_t)(N / kStripRows) * groups;
-    if (unit >= total) return;
-    const int64_t s = unit / groups;
-    const int gk = (int)(unit % groups);
-    const int b = gk >> 3, t = gk & 7;
-    const int rest = groups - 8 * b;
-    const int jb = rest < 8 ? rest : 8;
-    const uint8_t* blk = W + s * ((int64_t)kGroupBytes * groups) + (int64_t)b * kBlockBytes;
-    const uint4 cv = *reinterpret_cast<const uint4*>(blk + t * 512 + lane * 16);
-    const float d = bf16_bits_to_f32(*reinterpret_cast<const uint16_t*>(blk + 512 * jb + 2 * (t * 32 + lane)));
-    const float m = bf16_bits_to_f32(*reinterpret_cast<const uint16_t*>(blk + 576 * jb + 2 * (t * 32 + lane)));
-    const uint32_t words[4] = {cv.x, cv.y, cv.z, cv.w};
-    const int64_t n = s * kStripRows + lane;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        const float qf = (float)((words[i >> 3] >> (4 * (i & 7))) & 15u);
-        const float w = fmaf(d, qf, m);  // d*q is exact, so this is the single rounding Eq. 3 asks for
-        const int64_t at = (int64_t)(gk * kGroup + i) * N + n;
-        if (OUT_BF16)
-            reinterpret_cast<__nv_bfloat16*>(out)[at] = __float2bfloat16_rn(w);
-        else
-            reinterpret_cast<float*>(out)[at] = w;
-    }
-}
-
-// The same engine for the format variants (whole blocks only): group 64 / 128 read their scale and offset at the larger
-// group's index; MXFP4 multiplies the E2M1 element by its power-of-two scale (exact).
+// Format variants (whole blocks only): group 64 / 128 read their scale and offset at the larger group's index; MXFP4
+// multiplies the E2M1 element by its power-of-two scale (exact).
 __device__ __forceinline__ float e8m0_to_f32(uint32_t e) { return __uint_as_float(e ? e << 23 : 0x00400000u); }  // 2^(e-127)
 __device__ __forceinline__ float e2m1_to_f32(uint32_t q) {
     const uint32_t mag = q & 7u;  // 0, 0.5, 1, 1.5, 2, 3, 4, 6: exponent field mag >> 1, mantissa bit mag & 1
@@ -53,38 +22,70 @@ __device__ __forceinline__ float e2m1_to_f32(uint32_t q) {
     return (q & 8u) ? -v : v;
 }
 
+// The dequantisation engine: a CTA of eight warps dequantises the same 32-wide group of EIGHT consecutive strips (a 32 k x 256 n
+// tile), transposes it through shared memory and writes every k row of the tile as one contiguous run of 256 outputs
+// (512 bytes of bf16, 1 KB of fp32), 16 bytes per lane.  A warp writing its strip directly produces 64-byte pieces (bf16)
+// and measured 62 % of the copy bandwidth; this one is bound by the writes.  Same arithmetic, same bits.
 template <int FMT, bool OUT_BF16>
-__global__ void __launch_bounds__(256) fdqp_dequant_fmt_kernel(const uint8_t* __restrict__ W, void* __restrict__ out, int K,
-                                                               int N) {
+__global__ void __launch_bounds__(256) fdqp_dequant_tile_kernel(const uint8_t* __restrict__ W, void* __restrict__ out, int K,
+                                                                int N) {
     using F = FmtTraits<FMT>;
-    const int lane = threadIdx.x & 31;
-    const int groups = K / kGroup;  // 32-column tiles
-    const int64_t unit = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int64_t total = (int64_t)(N / kStripRows) * groups;
-    if (unit >= total) return;
-    const int64_t s = unit / groups;
-    const int gk = (int)(unit % groups);
-    const int b = gk >> 3, t = gk & 7;
-    const uint8_t* blk = W + (s * (K / kBlockK) + b) * (int64_t)F::kBlock;
-    const uint4 cv = *reinterpret_cast<const uint4*>(blk + t * 512 + lane * 16);
-    float d, m = 0.f;
+    using T = typename std::conditional<OUT_BF16, uint16_t, float>::type;
+    __shared__ __align__(16) T tile[32][256 + (OUT_BF16 ? 8 : 4)];  // [k][n], rows padded against bank conflicts
+    __shared__ float e2m1[16];  // MXFP4: the sixteen element values
     if (F::kMx) {
-        d = e8m0_to_f32(blk[kCodeBytes + t * 32 + lane]);
-    } else {
-        d = bf16_bits_to_f32(*reinterpret_cast<const uint16_t*>(blk + kCodeBytes + 2 * ((t >> F::kShift) * 32 + lane)));
-        m = bf16_bits_to_f32(*reinterpret_cast<const uint16_t*>(blk + F::kOffSect + 2 * ((t >> F::kShift) * 32 + lane)));
+        if (threadIdx.x < 16) e2m1[threadIdx.x] = e2m1_to_f32(threadIdx.x);
+        __syncthreads();
     }
-    const uint32_t words[4] = {cv.x, cv.y, cv.z, cv.w};
-    const int64_t n = s * kStripRows + lane;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int groups = K / kGroup;
+    const int gk = blockIdx.x % groups;                 // consecutive CTAs walk along K: their reads stay inside a block
+    const int64_t s0 = (int64_t)(blockIdx.x / groups) * 8;
+    const int64_t s = s0 + warp;
+    const int strips = N / kStripRows;
+    if (s < strips) {
+        const int b = gk >> 3, t = gk & 7;
+        const uint8_t* blk;
+        float d, m = 0.f;
+        if (FMT == kFmtQ4nx) {
+            const int rest = groups - 8 * b;
+            const int jb = rest < 8 ? rest : 8;
+            blk = W + s * ((int64_t)kGroupBytes * groups) + (int64_t)b * kBlockBytes;
+            d = bf16_bits_to_f32(*reinterpret_cast<const uint16_t*>(blk + 512 * jb + 2 * (t * 32 + lane)));
+            m = bf16_bits_to_f32(*reinterpret_cast<const uint16_t*>(blk + 576 * jb + 2 * (t * 32 + lane)));
+        } else {
+            blk = W + (s * (K / kBlockK) + b) * (int64_t)F::kBlock;
+            if (F::kMx) {
+                d = e8m0_to_f32(blk[kCodeBytes + t * 32 + lane]);
+            } else {
+                d = bf16_bits_to_f32(*reinterpret_cast<const uint16_t*>(blk + kCodeBytes + 2 * ((t >> F::kShift) * 32 + lane)));
+                m = bf16_bits_to_f32(*reinterpret_cast<const uint16_t*>(blk + F::kOffSect + 2 * ((t >> F::kShift) * 32 + lane)));
+            }
+        }
+        const uint4 cv = *reinterpret_cast<const uint4*>(blk + t * 512 + lane * 16);
+        const uint32_t words[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        const uint32_t q = (words[i >> 3] >> (4 * (i & 7))) & 15u;
-        const float w = F::kMx ? e2m1_to_f32(q) * d : fmaf(d, (float)q, m);
-        const int64_t at = (int64_t)(gk * kGroup + i) * N + n;
-        if (OUT_BF16)
-            reinterpret_cast<__nv_bfloat16*>(out)[at] = __float2bfloat16_rn(w);
-        else
-            reinterpret_cast<float*>(out)[at] = w;
+        for (int i = 0; i < 32; ++i) {
+            const uint32_t q = (words[i >> 3] >> (4 * (i & 7))) & 15u;
+            const float w = F::kMx ? e2m1[q] * d : fmaf(d, (float)q, m);  // one rounding (Eq. 3); MXFP4 exact
+            if (OUT_BF16)
+                tile[i][warp * 32 + lane] = (T)__bfloat16_as_ushort(__float2bfloat16_rn(w));
+            else
+                tile[i][warp * 32 + lane] = (T)w;
+        }
+    }
+    __syncthreads();
+    // every k row of the tile: 256 outputs = 32 (bf16) or 64 (fp32) 16-byte pieces
+    constexpr int kPieces = 256 * (int)sizeof(T) / 16;   // per row
+    constexpr int kPer = 16 / (int)sizeof(T);            // outputs per piece
+    const int64_t n0 = s0 * kStripRows;
+    for (int idx = threadIdx.x; idx < 32 * kPieces; idx += 256) {
+        const int row = idx / kPieces, piece = idx % kPieces;
+        const int64_t n = n0 + piece * kPer;
+        if (n < N) {  // N is a multiple of 32, so a piece is entirely inside or outside
+            const uint4 v = *reinterpret_cast<const uint4*>(&tile[row][piece * kPer]);
+            *reinterpret_cast<uint4*>(reinterpret_cast<T*>(out) + (int64_t)(gk * kGroup + row) * N + n) = v;
+        }
     }
 }
 
@@ -123,25 +124,18 @@ __global__ void __launch_bounds__(128) fdqp_plain_kernel(const uint8_t* __restri
         if (tk < mc) y[(int64_t)(m0 + tk) * N + s * kStripRows + lane] = acc[tk];
 }
 
-cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream) {
-    const int64_t units = (int64_t)(N / kStripRows) * (K / kGroup);
-    const unsigned grid = (unsigned)((units + 7) / 8);
+template <int FMT>
+static cudaError_t dequant_fmt_launch_t(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream) {
+    const int64_t ctas = (int64_t)((N / kStripRows + 7) / 8) * (K / kGroup);
     if (out_bf16)
-        fdqp_dequant_kernel<true><<<grid, 256, 0, stream>>>(W, out, K, N);
+        fdqp_dequant_tile_kernel<FMT, true><<<(unsigned)ctas, 256, 0, stream>>>(W, out, K, N);
     else
-        fdqp_dequant_kernel<false><<<grid, 256, 0, stream>>>(W, out, K, N);
+        fdqp_dequant_tile_kernel<FMT, false><<<(unsigned)ctas, 256, 0, stream>>>(W, out, K, N);
     return cudaGetLastError();
 }
 
-template <int FMT>
-static cudaError_t dequant_fmt_launch_t(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream) {
-    const int64_t units = (int64_t)(N / kStripRows) * (K / kGroup);
-    const unsigned grid = (unsigned)((units + 7) / 8);
-    if (out_bf16)
-        fdqp_dequant_fmt_kernel<FMT, true><<<grid, 256, 0, stream>>>(W, out, K, N);
-    else
-        fdqp_dequant_fmt_kernel<FMT, false><<<grid, 256, 0, stream>>>(W, out, K, N);
-    return cudaGetLastError();
+cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream) {
+    return dequant_fmt_launch_t<kFmtQ4nx>(W, out, out_bf16, K, N, stream);
 }
 
 cudaError_t dequant_fmt_launch(int fmt, const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream) {
