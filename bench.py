@@ -609,6 +609,7 @@ def run_ours(args, rank, local_rank, world):
     # ---- next steps beside the projection: decode attention over a KV cache, and the format variants of the container
     attention = None
     formats = None
+    dequant = None
     if rank == 0 and not args.no_head:
         H, G, d, L = 8, 4, 256, 32768          # Gemma3-4B heads at a 32k context
         ncache = max(1, int(np.ceil(4 * L2_BYTES / (2 * G * L * d * 2))))
@@ -661,6 +662,21 @@ def run_ours(args, rank, local_rank, world):
             f_gbs = (nbytes + 2 * hk + 4 * hn) / (f_ms * 1e-3) / 1e9
             formats[name] = {"ms": f_ms, "gbs": f_gbs, "frac": f_gbs / peaks["hbm_gbs"]}
             del fW
+        # the dequantisation engine on the LM head: container -> dense bf16 matrix in HBM (write-bound)
+        dq_out = torch.empty((hk, hn), dtype=torch.bfloat16, device="cuda")
+        for _ in range(2):
+            fd.fdqp_dequant(ctx, hW, dq_out, True, hk, hn, sraw)
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(stream)
+        for _ in range(5):
+            fd.fdqp_dequant(ctx, hW, dq_out, True, hk, hn, sraw)
+        d1.record(stream)
+        stream.synchronize()
+        dq_ms = d0.elapsed_time(d1) / 5
+        dq_gbs = (0.625 + 2.0) * hk * hn / (dq_ms * 1e-3) / 1e9
+        dequant = {"workload": f"LM head K={hk} N={hn} -> bf16 [K][N]", "ms": dq_ms, "gbs": dq_gbs, "bound": "hbm",
+                   "frac": dq_gbs / peaks["hbm_gbs"]}
+        del dq_out
         if fd.fdqp_last_status(ctx) != 0:
             raise SystemExit("bench.py: a kernel reported " + fd.fdqp_status_string(fd.fdqp_last_status(ctx)))
 
@@ -709,6 +725,7 @@ def run_ours(args, rank, local_rank, world):
             "prefill_lm_head": prefill,
             "decode_attention": attention,
             "format_variants": formats,
+            "dequant_engine": dequant,
             "cpu_baseline": cpu,
             "e2e": {"value": whole_job_gbs(step_bytes, e2e_steps, world, e2e_s * 1e3), "unit": "GB/s",
                     "h2d_bytes_per_step": sum(2 * M * K for _, K, _, _ in shapes),
