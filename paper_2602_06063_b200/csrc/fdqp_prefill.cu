@@ -540,6 +540,7 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
         // g0 = g1; g1 = g2; g2 = just-loaded -- makes the move wait for the load it follows, one trip to memory per k-step.)
 #ifdef FDQP_TRACE
         unsigned long long tr_wait = 0, tr_conv = 0, tr_st = 0, tr_arr = 0, tr_load = 0;
+        unsigned long long tr_rt = 0, tr_arrived[4] = {0, 0, 0, 0};  // round trip: arrive on a stage -> the stage seen free again
 #endif
         auto convert_step = [&](int i, const GroupRegs& g) -> bool {
             const int s = i % NA;
@@ -547,9 +548,9 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
             const unsigned long long pf_w0 = globaltimer_ns();
 #endif
             if (i >= NA && !mbar_wait(empty_a(s), ((i / NA) - 1) & 1, p.status)) return false;
-            if (dw == 0 && lane == 0 && i == 0) PF_STAMP(10);
 #ifdef FDQP_TRACE
             const unsigned long long pf_w1 = globaltimer_ns();
+            if (i >= NA) tr_rt += pf_w1 - tr_arrived[i & 3];
 #endif
             if (ATMEM) {
                 // this lane's row of the group, 16 bf16 pairs, into its TMEM lane; ordered against the MMAs that read the
@@ -577,7 +578,8 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
             if (lane == 0) mbar_arrive(full_a(s));
 #ifdef FDQP_TRACE
             tr_wait += pf_w1 - pf_w0;
-            tr_arr += globaltimer_ns() - pf_w1;
+            tr_arrived[i & 3] = globaltimer_ns();
+            tr_arr += tr_arrived[i & 3] - pf_w1;
 #endif
             return true;
         };
@@ -609,6 +611,7 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
             PF_ADD(4, tr_st);
             PF_ADD(15, tr_arr);
             PF_ADD(5, tr_load);
+            PF_ADD(10, tr_rt);
         }
 #endif
         // =============================== epilogue: TMEM -> y =================================================
