@@ -159,7 +159,10 @@ FDQP_API fdqp_status fdqp_destroy(fdqp_ctx* ctx);
  * accumulators in TMEM; a one-SM kernel up to 256 token rows, a two-SM kernel
  * above; K cut into slices when a shape has few output tiles) or the GEMV kernel
  * eight token rows at a time, whichever a small cost model expects to be faster
- * (GEMV chunks up to about 16-24 rows, or more when N is small).
+ * (GEMV chunks up to about 16-24 rows, or more when N is small).  Reductions
+ * shorter than K = 256 always take the GEMV kernels: the tensor-core path
+ * multiplies by bf16-rounded weights, whose rounding errors need a long K to
+ * average out inside the acceptance bound.
  * In the GEMV kernels the activations of each 32-group are held as fixed point
  * relative to the group's largest exponent (22 fraction bits below it): exact for
  * every element within 2^14 of the group's largest magnitude, rounded to 2^-22 of
