@@ -533,10 +533,11 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
         const int sl = ATMEM ? (warp & 3) : (dw >> 1), gl = ATMEM ? (dw >> 2) : (dw & 1);
         const int64_t strip = (int64_t)n_tile * (P::kRows / 32) + sl;
         const bool strip_ok = strip < p.N / kStripRows;
-        // the loads of the next three stages are in flight while this one is converted (a stage lasts about as long
-        // as one trip to HBM); groups past K load as zeros
+        // the loads of the next eight k-steps are in flight while this one is converted: a k-step lasts 0.6-0.7 us and a
+        // load from HBM under this kernel's traffic about as long, with a long tail; three k-steps ahead left the
+        // conversion waiting for its weights (measured: 5-7 % at up to 128 tokens).  Groups past K load as zeros.
         const int gbase = 2 * ks0 + gl;  // this warp's group in k-step i of the slice: gbase + 2 i
-        // Three register sets, each reloaded right after it has been converted.  (Rotating the sets with moves instead --
+        // Eight register sets, each reloaded right after it has been converted.  (Rotating the sets with moves instead --
         // g0 = g1; g1 = g2; g2 = just-loaded -- makes the move wait for the load it follows, one trip to memory per k-step.)
 #ifdef FDQP_TRACE
         unsigned long long tr_wait = 0, tr_conv = 0, tr_st = 0, tr_arr = 0, tr_load = 0;
@@ -583,25 +584,44 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
 #endif
             return true;
         };
-        GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase, lane, strip_ok);
+        GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase + 0, lane, strip_ok);
         GroupRegs g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2, lane, strip_ok);
         GroupRegs g2 = group_load<FMT>(p.W, p.K, strip, gbase + 4, lane, strip_ok);
-        for (int i = 0; i < ksteps && ok; i += 3) {
+        GroupRegs g3 = group_load<FMT>(p.W, p.K, strip, gbase + 6, lane, strip_ok);
+        GroupRegs g4 = group_load<FMT>(p.W, p.K, strip, gbase + 8, lane, strip_ok);
+        GroupRegs g5 = group_load<FMT>(p.W, p.K, strip, gbase + 10, lane, strip_ok);
+        GroupRegs g6 = group_load<FMT>(p.W, p.K, strip, gbase + 12, lane, strip_ok);
+        GroupRegs g7 = group_load<FMT>(p.W, p.K, strip, gbase + 14, lane, strip_ok);
+        for (int i = 0; i < ksteps && ok; i += 8) {
             ok = convert_step(i, g0);
-#ifdef FDQP_TRACE
-            const unsigned long long pf_l0 = globaltimer_ns();
-#endif
-            g0 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 3), lane, strip_ok);
-#ifdef FDQP_TRACE
-            tr_load += globaltimer_ns() - pf_l0;
-#endif
+            g0 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 8), lane, strip_ok);
             if (ok && i + 1 < ksteps) {
                 ok = convert_step(i + 1, g1);
-                g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 4), lane, strip_ok);
+                g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 9), lane, strip_ok);
             }
             if (ok && i + 2 < ksteps) {
                 ok = convert_step(i + 2, g2);
-                g2 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 5), lane, strip_ok);
+                g2 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 10), lane, strip_ok);
+            }
+            if (ok && i + 3 < ksteps) {
+                ok = convert_step(i + 3, g3);
+                g3 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 11), lane, strip_ok);
+            }
+            if (ok && i + 4 < ksteps) {
+                ok = convert_step(i + 4, g4);
+                g4 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 12), lane, strip_ok);
+            }
+            if (ok && i + 5 < ksteps) {
+                ok = convert_step(i + 5, g5);
+                g5 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 13), lane, strip_ok);
+            }
+            if (ok && i + 6 < ksteps) {
+                ok = convert_step(i + 6, g6);
+                g6 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 14), lane, strip_ok);
+            }
+            if (ok && i + 7 < ksteps) {
+                ok = convert_step(i + 7, g7);
+                g7 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 15), lane, strip_ok);
             }
         }
 #ifdef FDQP_TRACE
@@ -902,7 +922,7 @@ __global__ void __launch_bounds__(kPfThreads, 1)
             if (lane == 0) mbar_arrive_cluster(full_a0 + 8u * s);
             return true;
         };
-        GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase, lane, strip_ok);
+        GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase + 0, lane, strip_ok);
         GroupRegs g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2, lane, strip_ok);
         GroupRegs g2 = group_load<FMT>(p.W, p.K, strip, gbase + 4, lane, strip_ok);
         for (int i = 0; i < ksteps && ok; i += 3) {
