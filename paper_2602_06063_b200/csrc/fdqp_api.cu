@@ -123,10 +123,11 @@ int prefill_slices(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
 
 // M >= 9: the tensor-core kernels, or the GEMV kernel eight token rows at a time -- whichever a small cost model
 // (microseconds, constants measured on B200) says is faster.
-//   GEMV: every chunk streams the whole matrix, at about 5.5 TB/s for 1-2 rows, 3.9 for 3-4, 3.2 for 5-8, plus ~5 us.
-//   Tensor-core kernels: per wave of tiles and 64-wide k-step ~0.72 us (one-SM kernel, 128-row tiles two to an SM, up
-//   to 128 tokens), ~0.78 us (256-row tiles) or ~0.95 us (two-SM kernel, which also has twice the tokens' MMAs to
-//   issue), nearly independent of M.
+//   GEMV: every chunk streams the whole matrix, at about 5.5 TB/s for 1-2 rows, 3.9 for 3-4, 3.2 for 5-8, plus ~8 us
+//   (back-to-back chunks of a small matrix: 2 x 15 us for 16 MB).
+//   Tensor-core kernels: per wave of tiles and 64-wide k-step ~0.64 us up to 64 tokens rising to ~0.72 us at 128
+//   (one-SM kernel, 128-row tiles two to an SM), ~0.78 us (256-row tiles) or ~0.95 us (two-SM kernel, which also has
+//   twice the tokens' MMAs to issue).
 bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     if (M <= kMaxTokens || ctx->p_path == 2) return false;
     if (ctx->p_path == 3) return true;
@@ -137,13 +138,13 @@ bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     const double mb = 0.625 * (double)K * (double)N / 1.0e6;  // packed weights, bytes per microsecond = TB/s * 1e6
     const int64_t last = M % kMaxTokens;                       // rows of the ragged last chunk (0: none)
     const double last_rate = last <= 2 ? 5.5 : (last <= 4 ? 3.9 : 3.2);
-    const double t_gemv = (double)(M / kMaxTokens) * (5.0 + mb / 3.2) + (last ? 5.0 + mb / last_rate : 0.0);
+    const double t_gemv = (double)(M / kMaxTokens) * (8.0 + mb / 3.2) + (last ? 8.0 + mb / last_rate : 0.0);
     const bool pair = use_pair(ctx, M);
     const int64_t tiles = ((N + 255) / 256) * (pair ? (M + 511) / 512 : (M + 255) / 256);
     const int64_t slots = pair ? ctx->sm_count / 2 : ctx->sm_count;
     const int Z = prefill_slices(ctx, M, K, N);
     const double waves = (double)((tiles * Z + slots - 1) / slots);
-    double t_tensor = 5.0 + waves * (double)(((K + 63) / 64 + Z - 1) / Z) * (pair ? 0.95 : (M <= 128 ? 0.72 : 0.78));
+    double t_tensor = 5.0 + waves * (double)(((K + 63) / 64 + Z - 1) / Z) * (pair ? 0.95 : (M <= 64 ? 0.64 : (M <= 128 ? 0.64 + 0.08 * (double)(M - 64) / 64.0 : 0.78)));
     if (Z > 1) t_tensor += 3.0 + (double)(Z + 1) * (double)M * (double)N * 4.0 / 5.0e6;  // partial results out and back
     if (M * K * 2 < kSpreadBelowBytes) t_tensor += 3.0;                                   // the spreading copy
     return t_tensor < t_gemv;
