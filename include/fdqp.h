@@ -327,6 +327,17 @@ FDQP_API fdqp_status fdqp_dequant_fmt(fdqp_ctx* ctx, int format, const void* W_p
  * nothing itself.  Cleared only by fdqp_destroy. */
 FDQP_API fdqp_status fdqp_last_status(fdqp_ctx* ctx);
 
+/* Exercises the give-up path that every device-side wait of the library shares
+ * (all of them are bounded; a wait that runs out records FDQP_ERR_TIMEOUT in the
+ * context's status word and the kernel returns normally, freeing what it holds):
+ * enqueues one warp that waits on a barrier nothing arrives on, with that same
+ * wait and a limit of `limit_us` microseconds (1 .. 100000).  After the caller has
+ * synchronised the stream, fdqp_last_status(ctx) is FDQP_ERR_TIMEOUT (sticky for
+ * this context); the device and other contexts are unaffected.  Nothing faults
+ * and nothing is left running.  Errors: FDQP_ERR_ARG (null ctx, limit out of
+ * range), FDQP_ERR_CUDA. */
+FDQP_API fdqp_status fdqp_selftest_bounded_wait(fdqp_ctx* ctx, int64_t limit_us, void* cuda_stream);
+
 /* Text of the last CUDA runtime error seen by this context ("" if none).  The
  * pointer stays valid until the next failing call or fdqp_destroy. */
 FDQP_API const char* fdqp_last_cuda_error(fdqp_ctx* ctx);

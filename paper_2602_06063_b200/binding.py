@@ -27,6 +27,7 @@ EXPORTS = [
     "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
     "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc", "q4nx_packed_bytes_fmt", "q4nx_pack_fmt",
     "q4nx_unpack_fmt", "fdqp_run_fmt", "fdqp_dequant_fmt", "fdqp_run_add_rmsnorm_epilogue",
+    "fdqp_selftest_bounded_wait",
 ]
 
 
@@ -91,6 +92,8 @@ def load_library():
     lib.fdqp_dequant.argtypes = [vp, vp, vp, ci, i64, i64, vp]
     lib.fdqp_last_status.restype = ci
     lib.fdqp_last_status.argtypes = [vp]
+    lib.fdqp_selftest_bounded_wait.restype = ci
+    lib.fdqp_selftest_bounded_wait.argtypes = [vp, ctypes.c_int64, vp]
     lib.fdqp_last_cuda_error.restype = ctypes.c_char_p
     lib.fdqp_last_cuda_error.argtypes = [vp]
     lib.fdqp_status_string.restype = ctypes.c_char_p
@@ -310,6 +313,10 @@ def fdqp_dequant_fmt(ctx: int, fmt: int, W_packed, out, out_is_bf16: bool, K: in
 
 def fdqp_last_status(ctx: int) -> int:
     return int(load_library().fdqp_last_status(ctx))
+
+
+def fdqp_selftest_bounded_wait(ctx: int, limit_us: int, stream=None) -> None:
+    _check(load_library().fdqp_selftest_bounded_wait(ctx, int(limit_us), _stream(stream)), "fdqp_selftest_bounded_wait", ctx)
 
 
 def fdqp_last_cuda_error(ctx: int) -> str:

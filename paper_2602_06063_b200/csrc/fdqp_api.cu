@@ -29,6 +29,7 @@ cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* residual, uint16_t
 cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* V, float* out, float* ws, int max_splits, int H,
                           int G, int d, int L, int pitch, int window, float scale, int sm_count, cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
+cudaError_t wait_selftest_launch(int* status, unsigned long long limit_ns, cudaStream_t stream);
 }  // namespace fdqp
 
 using namespace fdqp;
@@ -619,6 +620,16 @@ extern "C" fdqp_status fdqp_last_status(fdqp_ctx* ctx) {
     if (!ctx) return FDQP_ERR_ARG;
     const int v = *static_cast<volatile int*>(ctx->status_host);
     return v == 0 ? FDQP_OK : static_cast<fdqp_status>(v);
+}
+
+extern "C" fdqp_status fdqp_selftest_bounded_wait(fdqp_ctx* ctx, int64_t limit_us, void* cuda_stream) {
+    if (!ctx || limit_us < 1 || limit_us > 100000) return FDQP_ERR_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FDQP_ERR_CUDA;
+    cudaError_t e = wait_selftest_launch(ctx->status_dev, (unsigned long long)limit_us * 1000ull, static_cast<cudaStream_t>(cuda_stream));
+    if (e) return cuda_fail(ctx, e, "bounded-wait self-test launch");
+    ctx->launches += 1;
+    return FDQP_OK;
 }
 
 extern "C" const char* fdqp_last_cuda_error(fdqp_ctx* ctx) { return ctx ? ctx->last_err.c_str() : ""; }

@@ -55,18 +55,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait on a phase parity.  Returns false (after recording the timeout in *status) if
-// the barrier did not flip within kWaitLimitNs.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+// the barrier did not flip within `limit_ns`.
+__device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, int* status, unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = globaltimer_ns();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0u && globaltimer_ns() - t0 > kWaitLimitNs) {
+        if ((it & 63u) == 0u && globaltimer_ns() - t0 > limit_ns) {
             atomicExch(status, kStatusTimeout);
             __threadfence_system();
             return false;
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+    return mbar_wait_for(bar, parity, status, kWaitLimitNs);
 }
 
 // ---- bulk async copy global -> shared (1-D, no multicast) ---------------------------------

@@ -124,6 +124,22 @@ __global__ void __launch_bounds__(128) fdqp_plain_kernel(const uint8_t* __restri
         if (tk < mc) y[(int64_t)(m0 + tk) * N + s * kStripRows + lane] = acc[tk];
 }
 
+// Self-test of the give-up path every kernel of the library shares: one warp waits on a barrier that nothing ever
+// arrives on, with the same bounded wait and a short limit, records the timeout and returns normally.
+__global__ void __launch_bounds__(32) fdqp_wait_selftest_kernel(int* status, unsigned long long limit_ns) {
+    __shared__ __align__(8) uint64_t bar;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) mbar_init(b, 1);
+    mbar_fence_init();
+    __syncwarp();
+    mbar_wait_for(b, 0, status, limit_ns);
+}
+
+cudaError_t wait_selftest_launch(int* status, unsigned long long limit_ns, cudaStream_t stream) {
+    fdqp_wait_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_ns);
+    return cudaGetLastError();
+}
+
 template <int FMT>
 static cudaError_t dequant_fmt_launch_t(const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream) {
     const int64_t ctas = (int64_t)((N / kStripRows + 7) / 8) * (K / kGroup);

@@ -341,3 +341,38 @@ def test_run_host_result_paths_agree(fresh, K, N, M, params):
         assert np.array_equal(y_staged.numpy(), ref)
     finally:
         fd.fdqp_set_param(fresh, "host_direct_y", 1)
+
+
+# ------------------------------------------------------------------ the give-up path of the bounded waits
+
+def test_bounded_wait_gives_up_and_context_stays_usable():
+    """A wait that nothing satisfies returns after its limit, records FDQP_ERR_TIMEOUT in the context's sticky status
+    word and leaves the device usable: a second context on the same device computes a correct projection afterwards,
+    and so does the first one (its status stays set, its results are still right)."""
+    import time
+    K, N, M = 512, 96, 1
+    case = Case(K, N, M, seed=97)
+    own = fd.fdqp_create(0, 8, K, N)
+    other = fd.fdqp_create(0, 8, K, N)
+    try:
+        assert fd.fdqp_last_status(own) == 0
+        t0 = time.perf_counter()
+        fd.fdqp_selftest_bounded_wait(own, 500)      # microseconds
+        torch.cuda.synchronize()
+        assert time.perf_counter() - t0 < 5.0         # it returned by itself, well before the production limit
+        assert fd.fdqp_last_status(own) == 8          # FDQP_ERR_TIMEOUT
+        assert fd.fdqp_last_status(other) == 0
+        ref, a_ref = case.reference()
+        y = case.run(other)
+        assert_close(y, ref, a_ref)
+        yo = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        fd.fdqp_run(own, case.x_dev, case.W_dev, yo, M, K, N)
+        torch.cuda.synchronize()
+        assert fd.fdqp_last_status(own) == 8          # sticky
+        assert_close(yo.cpu().numpy(), ref, a_ref)
+        lib = fd.load_library()
+        assert lib.fdqp_selftest_bounded_wait(own, 0, None) == 1
+        assert lib.fdqp_selftest_bounded_wait(own, 100001, None) == 1
+    finally:
+        fd.fdqp_destroy(own)
+        fd.fdqp_destroy(other)
