@@ -59,6 +59,7 @@ struct PrefillParams {
     int epi;
     int Z;          // K slices; slice z covers k-steps [z * ksteps_z, (z + 1) * ksteps_z)
     int ksteps_z;   // 64-wide k-steps per slice
+    uint32_t x_box_bytes;  // one-SM kernel: bytes of one x box (64 k x the token rows that exist, rounded up to 16)
 };
 
 // ---- tcgen05 wrappers -----------------------------------------------------------------------------------------
@@ -454,7 +455,7 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
                 const int s = i % NB;
                 if (i >= NB) ok = mbar_wait(empty_b(s), ((i / NB) - 1) & 1, p.status);
                 if (!ok) break;
-                mbar_arrive_expect_tx(full_b(s), P::kBBytes);
+                mbar_arrive_expect_tx(full_b(s), p.x_box_bytes);
                 tma_load_2d(base + s * kBStride + kBOff, &x_map, (ks0 + i) * kPfK, tok0, full_b(s));
             }
         }
@@ -1118,7 +1119,10 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_by
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};      // innermost first
     const cuuint64_t strides[1] = {(cuuint64_t)x_row_bytes};        // bytes between token rows
-    const cuuint32_t box[2] = {(cuuint32_t)kPfK, (cuuint32_t)(pair ? kP2TokBox : (M <= Pf1<128>::kToks ? Pf1<128>::kToks : kPfToks))};
+    // one-SM kernel: the box holds only the token rows the MMAs read (M rounded up to 16), not the whole tile's
+    const int tile_toks = M <= Pf1<128>::kToks ? Pf1<128>::kToks : kPfToks;
+    const int box_rows = pair ? kP2TokBox : (M < tile_toks ? (M + 15) / 16 * 16 : tile_toks);
+    const cuuint32_t box[2] = {(cuuint32_t)kPfK, (cuuint32_t)box_rows};
     const cuuint32_t elem[2] = {1, 1};
     if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t*>(x), dims, strides, box, elem,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -1136,6 +1140,7 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_by
     p.K = K;
     p.N = N;
     p.ksteps_z = (ksteps_all + Z - 1) / Z;
+    p.x_box_bytes = (uint32_t)box_rows * kPfK * 2;
     p.Z = (ksteps_all + p.ksteps_z - 1) / p.ksteps_z;  // no empty slice
     Z = p.Z;
     cudaError_t err;
