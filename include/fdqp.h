@@ -365,7 +365,9 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "host_direct_y" fdqp_run_host*: 1 (default) = small x and y in device-addressable page-locked host memory are
  *                   read / written in place by the kernels, 0 = always through the staging buffers and copies
  *   "prefill_a_tmem" one-SM tensor-core kernel up to 128 token rows: 1 (default) = the converted weights are kept in
- *                   tensor memory and read from there by the MMAs, 0 = in shared memory; same results bit for bit
+ *                   tensor memory and read from there by the MMAs (two CTAs per SM; up to 64 token rows three smaller
+ *                   CTAs per SM when the call has that many to run), 2 = the three-CTA form whenever M <= 64,
+ *                   0 = weights in shared memory; same results bit for bit
  *   "debug"         measurement aid: 1 = the GEMV consumers skip the arithmetic (y is then undefined)
  * Unknown key or unusable value: FDQP_ERR_ARG.  Meant for benchmarks and tests. */
 FDQP_API fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t value);

@@ -122,6 +122,17 @@ int prefill_slices(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     return Z < 1 ? 1 : (int)Z;
 }
 
+// Up to 128 tokens the one-SM kernel keeps the converted weights in tensor memory (mode 1, two CTAs per SM).  Up to 64
+// tokens a variant with half the accumulator columns, two weight stages and a four-deep weight prefetch (64 registers)
+// fits three CTAs per SM (mode 2): 6 % faster when the call has at least three CTAs per SM to run (LM head 181 -> 170 us),
+// slower when it has not (12B gate|up at M = 32: 44 -> 47 us), so the automatic choice asks for that many.
+int prefill_tmem_mode(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
+    if (ctx->p_atmem != 1) return (int)ctx->p_atmem;
+    if (M > 64) return 1;
+    const int64_t ctas = ((N + 127) / 128) * prefill_slices(ctx, M, K, N);
+    return ctas >= 3 * (int64_t)ctx->sm_count ? 2 : 1;
+}
+
 // M >= 9: the tensor-core kernels, or the GEMV kernel eight token rows at a time -- whichever a small cost model
 // (microseconds, constants measured on B200) says is faster.
 //   GEMV: every chunk streams the whole matrix, at about 5.5 TB/s for 1-2 rows, 3.9 for 3-4, 3.2 for 5-8, plus ~8 us
@@ -145,7 +156,7 @@ bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     const int64_t slots = pair ? ctx->sm_count / 2 : ctx->sm_count;
     const int Z = prefill_slices(ctx, M, K, N);
     const double waves = (double)((tiles * Z + slots - 1) / slots);
-    double t_tensor = 5.0 + waves * (double)(((K + 63) / 64 + Z - 1) / Z) * (pair ? 0.95 : (M <= 64 ? 0.64 : (M <= 128 ? 0.64 + 0.08 * (double)(M - 64) / 64.0 : 0.78)));
+    double t_tensor = 5.0 + waves * (double)(((K + 63) / 64 + Z - 1) / Z) * (pair ? 0.95 : (M <= 64 ? (prefill_tmem_mode(ctx, M, K, N) == 2 ? 0.60 : 0.64) : (M <= 128 ? 0.64 + 0.08 * (double)(M - 64) / 64.0 : 0.78)));
     if (Z > 1) t_tensor += 3.0 + (double)(Z + 1) * (double)M * (double)N * 4.0 / 5.0e6;  // partial results out and back
     if (M * K * 2 < kSpreadBelowBytes) t_tensor += 3.0;                                   // the spreading copy
     return t_tensor < t_gemv;
@@ -426,7 +437,7 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
             xt = reinterpret_cast<const uint16_t*>(ctx->x_spread);
         }
         if ((e = prefill_launch(W, xt, x_row_bytes, y, y16, epi, ctx->pf_ws, ctx->status_dev, (int)M, (int)K, (int)N,
-                                use_pair(ctx, M) ? 1 : 0, prefill_slices(ctx, M, K, N), fmt, ctx->p_atmem != 0 ? 1 : 0, stream)))
+                                use_pair(ctx, M) ? 1 : 0, prefill_slices(ctx, M, K, N), fmt, prefill_tmem_mode(ctx, M, K, N), stream)))
             return cuda_fail(ctx, e, "prefill kernel launch");
         ctx->launches += prefill_slices(ctx, M, K, N) > 1 ? 2 : 1;
         return FDQP_OK;
@@ -659,7 +670,7 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
         if (v != 0 && v != 1) return FDQP_ERR_ARG;
         ctx->p_direct_y = v;
     } else if (!std::strcmp(key, "prefill_a_tmem")) {
-        if (v != 0 && v != 1) return FDQP_ERR_ARG;
+        if (v != 0 && v != 1 && v != 2) return FDQP_ERR_ARG;
         ctx->p_atmem = v;
     } else if (!std::strcmp(key, "prefill_pair")) {
         if (v > 1) return FDQP_ERR_ARG;
@@ -702,12 +713,16 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
                           "fdqp_prefill_pair_kernel grid=%lld cluster=2 block=320 tile=256x512 per pair stages=4 tmem_cols=512 "
                           "split_k=%d%s",
                           (long long)(2 * ((N + 255) / 256) * ((M + 511) / 512) * Z), Z, Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
-        else if (M <= 128)
+        else if (M <= 128) {
+            const int mode = prefill_tmem_mode(ctx, M, K, N);
+            const bool tri = mode == 2 && M <= 64;
             std::snprintf(buf, buf_bytes,
-                          "fdqp_prefill_kernel<128> grid=%lld block=320 tile=128x128 two CTAs per SM %s split_k=%d%s",
-                          (long long)(((N + 127) / 128) * Z),
-                          ctx->p_atmem ? "weights in TMEM (4 stages) x_stages=6 tmem_cols=256" : "stages=3 tmem_cols=128", Z,
-                          Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
+                          "fdqp_prefill_kernel<128> grid=%lld block=320 tile=128x128 %s CTAs per SM %s split_k=%d%s",
+                          (long long)(((N + 127) / 128) * Z), tri ? "three" : "two",
+                          tri ? "weights in TMEM (2 stages) x_stages=4 tmem_cols=128"
+                              : (mode ? "weights in TMEM (4 stages) x_stages=6 tmem_cols=256" : "stages=3 tmem_cols=128"),
+                          Z, Z > 1 ? " + fdqp_prefill_sum_kernel" : "");
+        }
         else
             std::snprintf(buf, buf_bytes,
                           "fdqp_prefill_kernel grid=%lld block=576 tile=256x256 stages=3 tmem_cols=512 split_k=%d%s",

@@ -48,6 +48,7 @@ struct Pf1 {
     static constexpr uint32_t kSmemBytes = kPfStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
     static constexpr int kCtasPerSm = ROWS == 256 ? 1 : 2;
     static constexpr uint32_t kSmemBytesTmemA = kPfTmemBStages * kBBytes + 1024 + 256;  // x stages only
+    static constexpr uint32_t kSmemBytesTri = 4 * kBBytes + 1024 + 256;                // three CTAs per SM: four x stages
 };
 
 struct PrefillParams {
@@ -382,19 +383,20 @@ extern "C" __attribute__((visibility("default"))) int fdqp_pf_trace_clear() {
 // MMA takes its A operand from there, which removes the weights' store and re-read from the shared-memory traffic (at
 // <= 128 tokens per MMA that traffic is what the tensor pipe waits for).  Shared memory then holds x stages only (six of
 // them); TMEM holds the accumulators (128 columns) and four weight stages of 32 columns (64 k as bf16 pairs).
-template <int FMT, int ROWS, bool ATMEM = false>
-__global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
+template <int FMT, int ROWS, bool ATMEM = false, bool TRI = false>
+__global__ void __launch_bounds__(Pf1<ROWS>::kThreads, TRI ? 3 : Pf1<ROWS>::kCtasPerSm)
     fdqp_prefill_kernel(const __grid_constant__ CUtensorMap x_map, const PrefillParams p) {
     using P = Pf1<ROWS>;
     static_assert(!ATMEM || ROWS == 128, "weights in tensor memory: 128-row tiles only");
     constexpr int CH = P::kToks / 2;  // token columns per epilogue warp of a quarter
-    constexpr int NA = ATMEM ? kPfTmemAStages : kPfStages;    // weight stages
-    constexpr int NB = ATMEM ? kPfTmemBStages : kPfStages;    // x stages
+    static_assert(!TRI || ATMEM, "three CTAs per SM: the tensor-memory variant only");
+    constexpr int NA = TRI ? 2 : (ATMEM ? kPfTmemAStages : kPfStages);    // weight stages
+    constexpr int NB = TRI ? 4 : (ATMEM ? kPfTmemBStages : kPfStages);    // x stages
     constexpr uint32_t kBStride = ATMEM ? P::kBBytes : P::kStageBytes;  // bytes from one x stage to the next
     constexpr uint32_t kBOff = ATMEM ? 0u : P::kABytes;                  // x tile inside its stage
     constexpr uint32_t kRing = NB * kBStride;
-    constexpr uint32_t kTmemCols = ATMEM ? 256u : P::kTmemCols;
-    constexpr uint32_t kTmemA = 128;  // ATMEM: first TMEM column of the weight stages
+    constexpr uint32_t kTmemCols = TRI ? 128u : (ATMEM ? 256u : P::kTmemCols);
+    constexpr uint32_t kTmemA = TRI ? 64 : 128;  // ATMEM: first TMEM column of the weight stages
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // tiles must start on a 1024-byte boundary (swizzle atom)
@@ -585,6 +587,28 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
 #endif
             return true;
         };
+        if (TRI) {
+            GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase + 0, lane, strip_ok);
+            GroupRegs g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2, lane, strip_ok);
+            GroupRegs g2 = group_load<FMT>(p.W, p.K, strip, gbase + 4, lane, strip_ok);
+            GroupRegs g3 = group_load<FMT>(p.W, p.K, strip, gbase + 6, lane, strip_ok);
+            for (int i = 0; i < ksteps && ok; i += 4) {
+                ok = convert_step(i, g0);
+                g0 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 4), lane, strip_ok);
+                if (ok && i + 1 < ksteps) {
+                    ok = convert_step(i + 1, g1);
+                    g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 5), lane, strip_ok);
+                }
+                if (ok && i + 2 < ksteps) {
+                    ok = convert_step(i + 2, g2);
+                    g2 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 6), lane, strip_ok);
+                }
+                if (ok && i + 3 < ksteps) {
+                    ok = convert_step(i + 3, g3);
+                    g3 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 7), lane, strip_ok);
+                }
+            }
+        } else {
         GroupRegs g0 = group_load<FMT>(p.W, p.K, strip, gbase + 0, lane, strip_ok);
         GroupRegs g1 = group_load<FMT>(p.W, p.K, strip, gbase + 2, lane, strip_ok);
         GroupRegs g2 = group_load<FMT>(p.W, p.K, strip, gbase + 4, lane, strip_ok);
@@ -624,6 +648,7 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, Pf1<ROWS>::kCtasPerSm)
                 ok = convert_step(i + 7, g7);
                 g7 = group_load<FMT>(p.W, p.K, strip, gbase + 2 * (i + 15), lane, strip_ok);
             }
+        }
         }
 #ifdef FDQP_TRACE
         if (dw == 0 && lane == 0) {
@@ -1062,6 +1087,7 @@ static cudaError_t prefill_set_smem_limit_fmt() {
     if (e) return e;
     if ((e = cudaFuncSetAttribute(fdqp_prefill_kernel<FMT, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Pf1<128>::kSmemBytes))) return e;
     if ((e = cudaFuncSetAttribute(fdqp_prefill_kernel<FMT, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Pf1<128>::kSmemBytesTmemA))) return e;
+    if ((e = cudaFuncSetAttribute(fdqp_prefill_kernel<FMT, 128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Pf1<128>::kSmemBytesTri))) return e;
     return cudaFuncSetAttribute(fdqp_prefill_pair_kernel<FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kP2SmemBytes);
 }
 
@@ -1094,7 +1120,9 @@ static cudaError_t prefill_launch_kernels(const CUtensorMap& map, const PrefillP
     }
     if (pair == 0 && M <= Pf1<128>::kToks) {  // small tiles, two CTAs per SM
         const int n_tiles = (N + 127) / 128;
-        if (a_tmem)
+        if (a_tmem == 2 && M <= 64)
+            fdqp_prefill_kernel<FMT, 128, true, true><<<n_tiles * Z, Pf1<128>::kThreads, Pf1<128>::kSmemBytesTri, stream>>>(map, p);
+        else if (a_tmem)
             fdqp_prefill_kernel<FMT, 128, true><<<n_tiles * Z, Pf1<128>::kThreads, Pf1<128>::kSmemBytesTmemA, stream>>>(map, p);
         else
             fdqp_prefill_kernel<FMT, 128><<<n_tiles * Z, Pf1<128>::kThreads, Pf1<128>::kSmemBytes, stream>>>(map, p);

@@ -26,9 +26,11 @@ def ctx():
 def fresh(ctx):
     for key in PARAMS:
         fd.fdqp_set_param(ctx, key, -1)
+    fd.fdqp_set_param(ctx, "prefill_a_tmem", 1)
     yield ctx
     for key in PARAMS:
         fd.fdqp_set_param(ctx, key, -1)
+    fd.fdqp_set_param(ctx, "prefill_a_tmem", 1)
 
 
 def bf16_rne_bits(f32: np.ndarray) -> np.ndarray:
@@ -71,6 +73,8 @@ CASES = [
     (1056, 320, 20, {"path": 2}),                        # GEMV eight rows at a time
     (1056, 320, 40, {"path": 3}),                        # one-SM tensor-core kernel
     (2048, 256, 64, {"path": 3, "prefill_split_k": 4}),  # ... with K slices + sum kernel
+    (1056, 320, 40, {"path": 3, "prefill_a_tmem": 2}),   # ... three CTAs per SM (up to 64 tokens)
+    (2048, 256, 64, {"path": 3, "prefill_a_tmem": 2, "prefill_split_k": 4}),
     (544, 1056, 300, {"path": 3}),                       # two-SM tensor-core kernel, ragged tokens
     (4096, 288, 512, {"path": 3, "prefill_split_k": 3}),
 ]

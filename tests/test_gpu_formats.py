@@ -107,7 +107,11 @@ def test_prefill_sized_projection_matches_oracle(ctx, fmt, K, N, M):
     fd.fdqp_set_param(ctx, "path", 3)       # the tensor-core kernels whatever the dispatch model would choose
     try:
         y = c.run(ctx)
+        if M <= 64:                         # the three-CTAs-per-SM form of the one-SM kernel: the same bits
+            fd.fdqp_set_param(ctx, "prefill_a_tmem", 2)
+            assert np.array_equal(c.run(ctx), y)
     finally:
+        fd.fdqp_set_param(ctx, "prefill_a_tmem", 1)
         fd.fdqp_set_param(ctx, "path", 0)
     n1 = min(N, 512)
     y_ref, a_ref = c.reference(0, n1)

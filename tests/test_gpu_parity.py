@@ -27,9 +27,11 @@ def fresh(ctx):
     """The shared context with every launch parameter back to automatic."""
     for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp", "prefill_pair", "prefill_split_k"):
         fd.fdqp_set_param(ctx, key, -1)
+    fd.fdqp_set_param(ctx, "prefill_a_tmem", 1)
     yield ctx
     for key in ("path", "ctas_per_sm", "consumer_warps", "stages", "split_k", "l2_evict_first", "prep_inline", "strip_aligned", "blocks_per_warp", "prefill_pair", "prefill_split_k"):
         fd.fdqp_set_param(ctx, key, -1)
+    fd.fdqp_set_param(ctx, "prefill_a_tmem", 1)
 
 
 # ------------------------------------------------------------------ dequantisation engine: bit-exact
@@ -129,6 +131,27 @@ def test_prefill_tensor_path_matches_oracle(fresh, K, N, M):
     fd.fdqp_set_param(fresh, "path", 2)
     assert "fdqp_gemv_kernel" in fd.fdqp_describe(fresh, M, K, N)
     assert_close(case.run(fresh), y_ref, a_ref, f"gemv-chunked K={K} N={N} M={M}")
+
+
+@pytest.mark.parametrize("K,N,M,Z", [(64, 32, 9, 1), (1056, 320, 20, 1), (2560, 1024, 64, 1), (544, 1056, 33, 1), (2048, 256, 64, 4),
+                                     (1024, 32, 40, 2), (2592, 160, 16, 3)])
+def test_prefill_three_ctas_per_sm_same_bits(fresh, K, N, M, Z):
+    # up to 64 token rows: the form with 64 accumulator columns, two weight stages and a four-deep weight prefetch that
+    # fits three CTAs per SM (chosen by itself for calls with that many CTAs; forced here) -- within the bound of the
+    # oracle and bit for bit what the two-CTA form computes
+    case = Case(K, N, M, seed=2500 + K + N + M)
+    fd.fdqp_set_param(fresh, "path", 3)
+    if Z > 1:
+        fd.fdqp_set_param(fresh, "prefill_split_k", Z)
+    fd.fdqp_set_param(fresh, "prefill_a_tmem", 2)
+    assert "three CTAs per SM" in fd.fdqp_describe(fresh, M, K, N)
+    y3 = case.run(fresh)
+    fd.fdqp_set_param(fresh, "prefill_a_tmem", 1)
+    assert "two CTAs per SM" in fd.fdqp_describe(fresh, M, K, N)
+    y2 = case.run(fresh)
+    y_ref, a_ref = case.reference()
+    assert_close(y3, y_ref, a_ref, f"three CTAs K={K} N={N} M={M} Z={Z}")
+    assert np.array_equal(y3, y2)
 
 
 @pytest.mark.parametrize("K,N,M,Z", [(2048, 256, 64, 4), (2112, 544, 300, 3), (4096, 288, 512, 8), (1024, 32, 40, 2)])
