@@ -5,17 +5,21 @@
 // (Sec. "Dequantization Engine", Sec. "Tiling-based MM").  Here the DRAM round trip is removed: the dequantised tile
 // only ever exists in shared memory, in the layout the tensor core reads.
 //
-// One CTA computes a 256 (output features) x 256 (tokens) tile of y:
+// The basic form: one CTA computes a 256 (output features) x 256 (tokens) tile of y:
 //   D[n][tok] = sum_k w16[k][n] * x[tok][k],   w16 = RNE_bf16( RN_fp32(d * q + m) )      (Eq. 3, then Eq. 14)
 //   - UMMA shape 128 x N_inst x 16 (kind::f16, bf16 inputs, fp32 accumulate), two accumulators (rows 0..127 and
 //     128..255 of the tile) of 256 TMEM columns each = all 512 columns;
-//   - A = dequantised weights, [256 rows][64 k] bf16 per pipeline stage, K-major, 128-byte swizzle, written by eight
-//     dequantisation warps (one 32-row strip each) with plain shared-memory stores;
-//   - B = x, [256 tokens][64 k] bf16 per stage, K-major, 128-byte swizzle, loaded by TMA (2-D tiled copy, no
+//   - A = dequantised weights, [256 rows][64 k] bf16 per pipeline stage, K-major, 128-byte swizzle, written by sixteen
+//     dequantisation warps (one 32-row strip and 32-wide group each) with plain shared-memory stores; each warp reads
+//     its codes, scale and offset straight from global memory, eight k-steps ahead;
+//   - B = x, [tokens][64 k] bf16 per stage, K-major, 128-byte swizzle, loaded by TMA (2-D tiled copy, no
 //     multicast); rows beyond M and columns beyond K are zero-filled by the copy engine;
 //   - one elected thread issues the MMAs; tcgen05.commit hands stages back and announces the finished accumulators;
-//   - epilogue: the eight dequantisation warps read TMEM (tcgen05.ld 32x32b) and store fp32 y, 128 contiguous bytes
-//     per warp store.
+//   - epilogue: the dequantisation warps read TMEM (tcgen05.ld 32x32b) and store fp32 y, 128 contiguous bytes
+//     per warp store (bf16 epilogues go through shared memory).
+// Up to 128 tokens: 128 x 128 tiles, two CTAs per SM, the converted weights kept in tensor memory (tcgen05.st) and read
+// from there by the MMAs; up to 64 tokens a smaller form of that fits three CTAs per SM.  More than 256 tokens: a pair
+// of SMs works on a 256 x 512 tile (cta_group::2).  Few tiles: K slices, summed by a second kernel.
 // Every wait is bounded; TMEM is released on every path.
 #include <cuda.h>
 
@@ -934,8 +938,8 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         const int sl = dw >> 1, gl = dw & 1;  // strip of this CTA's 128 rows, group of the 64-k stage
         const int64_t strip = (int64_t)(n0 / kStripRows) + sl;
         const bool strip_ok = strip < p.N / kStripRows;
-        // software pipeline: the loads of the next three stages are in flight while this one is converted (a stage
-        // lasts well under a microsecond here, less than one trip to L2 / HBM); groups past K load as zeros
+        // software pipeline: the loads of the next three k-steps are in flight while this one is converted (eight, as in
+        // the one-SM kernel, measured no faster here); groups past K load as zeros
         const int gbase = 2 * ks0 + gl;  // this warp's group in k-step i of the slice: gbase + 2 i
         // three register sets, each reloaded right after it has been converted (no rotation by moves: see the one-SM kernel)
         const uint32_t full_a0 = mapa_shared(full_a(0), 0);
