@@ -603,6 +603,22 @@ def run_ours(args, rank, local_rank, world):
                    "frac_of_burst": tflops / peaks["bf16_tflops"] if peaks.get("bf16_tflops") else None,
                    "frac_of_sustained": (tflops / peaks["bf16_tflops_sustained"]) if peaks.get("bf16_tflops_sustained") else None,
                    "launch": fd.fdqp_describe(pctx, PM, hk, hn)}
+        # smaller token counts on the same matrix (the one-SM forms of the kernel), same timing
+        other = {}
+        for om in (32, 128):
+            for _ in range(3):
+                fd.fdqp_run(pctx, px, hW, py, om, hk, hn, sraw)
+            p0.record(stream)
+            for _ in range(6):
+                fd.fdqp_run(pctx, px, hW, py, om, hk, hn, sraw)
+            p1.record(stream)
+            stream.synchronize()
+            if fd.fdqp_last_status(pctx) != 0:
+                raise SystemExit("bench.py: the prefill kernel reported " + fd.fdqp_status_string(fd.fdqp_last_status(pctx)))
+            o_ms = p0.elapsed_time(p1) / 6
+            other[f"M{om}"] = {"ms": o_ms, "tflops": 2.0 * om * hk * hn / (o_ms * 1e-3) / 1e12,
+                               "launch": fd.fdqp_describe(pctx, om, hk, hn)}
+        prefill["other_token_counts"] = other
         fd.fdqp_destroy(pctx)
         del px, py
 
