@@ -106,20 +106,49 @@ fdqp_status check_shape(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
 // More than 256 token rows: a pair of SMs works on a 256 x 512 tile (every converted weight serves 512 tokens).
 bool use_pair(const fdqp_ctx* ctx, int64_t M) { return ctx->p_pair >= 0 ? ctx->p_pair != 0 : M > 256; }
 
-// K slices of a tensor-core call: as many as fill one wave of SMs (or SM pairs), while every slice keeps at least eight
-// 64-wide k-steps and the partial results fit the context's workspace.
-int prefill_slices(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
+// Time model of a tensor-core call cut into Z K slices (microseconds, without the launch and the optional spreading
+// copy; constants measured on B200).  A CTA (pair) costs about c per 64-wide k-step when its SM is full: c = 0.64 up to
+// 64 tokens rising to 0.72 at 128 (128-row tiles, two CTAs per SM), 0.78 (256-row tiles, one CTA per SM), 0.95 (two-SM
+// kernel).  The busiest SM runs n = ceil(CTAs / SMs) of them, two at a time where two fit; a CTA that has the SM to
+// itself runs its k-steps in about 0.7 of that time.  Z > 1 adds the second kernel (~5 us) and the partial results:
+// written by the slices, read and summed by the second kernel.
+double prefill_time_model(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N, int64_t Z) {
     const bool pair = use_pair(ctx, M);
-    const int64_t tiles = ((N + 255) / 256) * (pair ? (M + 511) / 512 : (M + 255) / 256);
-    const int64_t slots = pair ? ctx->sm_count / 2 : ctx->sm_count;
+    const bool small = !pair && M <= 128;
+    const int64_t tiles = pair ? ((N + 255) / 256) * ((M + 511) / 512)
+                               : (small ? (N + 127) / 128 : ((N + 255) / 256) * ((M + 255) / 256));
+    const int64_t units = pair ? ctx->sm_count / 2 : ctx->sm_count;
+    const int64_t n = (tiles * Z + units - 1) / units;
+    const double rounds = small ? (double)(n / 2) + ((n & 1) ? 0.7 : 0.0) : (double)n;
+    const double c = pair ? 0.95 : (M <= 64 ? 0.64 : (M <= 128 ? 0.64 + 0.08 * (double)(M - 64) / 64.0 : 0.78));
+    const int64_t kz = ((K + 63) / 64 + Z - 1) / Z;
+    double t = rounds * (double)kz * c;
+    if (Z > 1) t += 5.0 + (double)(2 * Z + 1) * (double)M * (double)N * 4.0 / 5.0e6;
+    return t;
+}
+
+// K slices of a tensor-core call: the count the time model likes best (a larger count has to win by 8 %), while every
+// slice keeps at least eight 64-wide k-steps and the partial results fit the context's workspace.  Few tiles (27B down:
+// 42 of 128 rows) get as many slices as fill the SMs once; a tile count just above a multiple of the slots (12B-like
+// K = 5376, N = 43008 at M = 32: 336 CTAs on 296 slots) gets the slices that even out the last round (85 -> 70 us).
+int prefill_slices(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     const int64_t ksteps = (K + 63) / 64;
-    int64_t Z = slots / tiles;
-    if (ctx->p_pf_split > 0) Z = ctx->p_pf_split;
-    if (Z > kMaxSplit) Z = kMaxSplit;
-    if (Z > ksteps / 8) Z = ksteps / 8;
+    int64_t zmax = kMaxSplit;
+    if (zmax > ksteps / 8) zmax = ksteps / 8;
     const int64_t fit = (int64_t)(ctx->pf_ws_bytes / ((size_t)M * (size_t)N * 4));
-    if (Z > fit) Z = fit;
-    return Z < 1 ? 1 : (int)Z;
+    if (zmax > fit) zmax = fit;
+    if (zmax < 1) zmax = 1;
+    if (ctx->p_pf_split > 0) return (int)(ctx->p_pf_split < zmax ? ctx->p_pf_split : zmax);
+    int64_t best = 1;
+    double t_best = prefill_time_model(ctx, M, K, N, 1);
+    for (int64_t Z = 2; Z <= zmax; ++Z) {
+        const double t = prefill_time_model(ctx, M, K, N, Z);
+        if (t < 0.92 * t_best) {
+            best = Z;
+            t_best = t;
+        }
+    }
+    return (int)best;
 }
 
 // Up to 128 tokens the one-SM kernel keeps the converted weights in tensor memory (mode 1, two CTAs per SM).  Up to 64
@@ -137,9 +166,7 @@ int prefill_tmem_mode(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
 // (microseconds, constants measured on B200) says is faster.
 //   GEMV: every chunk streams the whole matrix, at about 5.5 TB/s for 1-2 rows, 3.9 for 3-4, 3.2 for 5-8, plus ~8 us
 //   (back-to-back chunks of a small matrix: 2 x 15 us for 16 MB).
-//   Tensor-core kernels: per wave of tiles and 64-wide k-step ~0.64 us up to 64 tokens rising to ~0.72 us at 128
-//   (one-SM kernel, 128-row tiles two to an SM), ~0.78 us (256-row tiles) or ~0.95 us (two-SM kernel, which also has
-//   twice the tokens' MMAs to issue).
+//   Tensor-core kernels: prefill_time_model above.
 bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     if (M <= kMaxTokens || ctx->p_path == 2) return false;
     if (ctx->p_path == 3) return true;
@@ -151,13 +178,8 @@ bool use_prefill(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     const int64_t last = M % kMaxTokens;                       // rows of the ragged last chunk (0: none)
     const double last_rate = last <= 2 ? 5.5 : (last <= 4 ? 3.9 : 3.2);
     const double t_gemv = (double)(M / kMaxTokens) * (8.0 + mb / 3.2) + (last ? 8.0 + mb / last_rate : 0.0);
-    const bool pair = use_pair(ctx, M);
-    const int64_t tiles = ((N + 255) / 256) * (pair ? (M + 511) / 512 : (M + 255) / 256);
-    const int64_t slots = pair ? ctx->sm_count / 2 : ctx->sm_count;
-    const int Z = prefill_slices(ctx, M, K, N);
-    const double waves = (double)((tiles * Z + slots - 1) / slots);
-    double t_tensor = 5.0 + waves * (double)(((K + 63) / 64 + Z - 1) / Z) * (pair ? 0.95 : (M <= 64 ? (prefill_tmem_mode(ctx, M, K, N) == 2 ? 0.60 : 0.64) : (M <= 128 ? 0.64 + 0.08 * (double)(M - 64) / 64.0 : 0.78)));
-    if (Z > 1) t_tensor += 3.0 + (double)(Z + 1) * (double)M * (double)N * 4.0 / 5.0e6;  // partial results out and back
+    double t_tensor = 5.0 + prefill_time_model(ctx, M, K, N, prefill_slices(ctx, M, K, N));
+    if (prefill_tmem_mode(ctx, M, K, N) == 2) t_tensor *= 0.94;  // three CTAs per SM
     if (M * K * 2 < kSpreadBelowBytes) t_tensor += 3.0;                                   // the spreading copy
     return t_tensor < t_gemv;
 }

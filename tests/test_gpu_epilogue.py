@@ -180,7 +180,8 @@ NORM_CASES = [
     (2560, 512, 2, {}, 3),                 # too many items for in-kernel preparation: norm kernel + preparation + GEMV
     (10240, 320, 1, {}, 3),
     (1056, 320, 20, {"path": 2}, 7),       # norm kernel, then three GEMV chunks with their preparation
-    (1056, 320, 40, {"path": 3}, 3),       # norm kernel + tensor-core kernel (K slices) + its sum kernel
+    (1056, 320, 40, {"path": 3, "prefill_split_k": 2}, 3),  # norm kernel + tensor-core kernel (K slices) + its sum kernel
+    (1056, 320, 40, {"path": 3}, 2),       # norm kernel + tensor-core kernel
     (544, 1056, 300, {"path": 3}, 2),
 ]
 

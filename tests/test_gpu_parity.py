@@ -161,7 +161,8 @@ def test_prefill_k_slices(fresh, K, N, M, Z):
     fd.fdqp_set_param(fresh, "path", 3)
     y_ref, a_ref = case.reference()
     auto = fd.fdqp_describe(fresh, M, K, N)
-    assert "split_k=" in auto and "split_k=1" not in auto      # such shapes are split without being asked
+    if K >= 2048:                                               # long reductions over few tiles are split without being
+        assert "split_k=" in auto and "split_k=1" not in auto  # asked (a short one is not worth the second kernel)
     y_auto = case.run(fresh)
     assert_close(y_auto, y_ref, a_ref, f"prefill auto split K={K} N={N} M={M}")
     fd.fdqp_set_param(fresh, "prefill_split_k", Z)
