@@ -348,7 +348,9 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
 /* Override a launch parameter; value < 0 restores the built-in choice.  Keys:
  *   "path"          0 = dispatch on M (default), 1 = force the plain CUDA-core kernel,
  *                   2 = run M >= 9 through the GEMV kernel eight token rows at a time,
- *                   3 = run every M >= 9 through the tensor-core prefill kernel
+ *                   3 = run every M >= 9 through the tensor-core prefill kernel (also K < 256, which the
+ *                   dispatch keeps off it: with so few terms the bf16 rounding of the weights does not average
+ *                   out and single outputs can land a few per cent outside the acceptance bound)
  *   "ctas_per_sm"   persistent CTAs per SM for the GEMV kernels (1 or 2; 2 implies 8 consumer warps)
  *   "consumer_warps" 8 or 16 consumer warps per CTA
  *   "stages"        shared-memory ring depth in stages (a stage holds consumer_warps / 8 * blocks_per_warp blocks)
