@@ -76,3 +76,21 @@ def test_gemma3_4b_lm_head_decode_and_prefill(ctx):
                                       nthreads=min(32, oracle.max_threads()))
         assert_close(y[:, n0:n0 + 32], y_ref, a_ref, f"LM head M=512 strip {s}")
     assert np.all(np.isfinite(y))
+
+
+@pytest.mark.parametrize("M,form", [(48, "three CTAs per SM"), (128, "two CTAs per SM")])
+def test_gemma3_4b_lm_head_small_prefill_chunks(ctx, M, form):
+    # the one-SM forms of the tensor-core kernel at full size, in the configuration the dispatch picks by itself:
+    # 32 strips spread over N (first and last included), all M rows
+    _, K, N, seed = synthgen.GEMMA3_4B_LM_HEAD
+    w = synthgen.weights(seed, K, N)
+    x = synthgen.activations(seed + 1, M, K)
+    base = Case(K, N, M, seed, weights=w, x=x)
+    assert form in fd.fdqp_describe(ctx, M, K, N)
+    y = base.run(ctx)
+    assert np.all(np.isfinite(y))
+    for s in np.unique(np.linspace(0, N // 32 - 1, 32).astype(np.int64)):
+        n0 = int(s) * 32
+        y_ref, a_ref = oracle.project(x, w.codes, w.scales, w.offsets, n0=n0, n1=n0 + 32,
+                                      nthreads=min(32, oracle.max_threads()))
+        assert_close(y[:, n0:n0 + 32], y_ref, a_ref, f"LM head M={M} strip {s}")
