@@ -283,7 +283,8 @@ FDQP_API fdqp_status fdqp_run_host_async(fdqp_ctx* ctx, const void* x_host_bf16,
  * counterpart: this is a packaging of fdqp_run's GEMV kernel, not another operation.)
  *   x_bf16, W_q4nx, y   device pointers, 16-byte aligned, as for fdqp_run; runs on the CURRENT device
  *   limits              M <= 8; N <= 262144; and the prepared activations must fit shared memory without
- *                       splitting K (about M*K <= 32768, e.g. K <= 3840 at M = 8); beyond them FDQP_ERR_SIZE
+ *                       splitting K (about M*K <= 32768, e.g. K <= 3840 at M = 8); beyond them FDQP_ERR_SIZE.
+ *                       A bounded wait that ran out inside the kernel is reported by fdqp_noalloc_last_status.
  * It takes no context and calls no cudaMalloc / cudaFree or any other allocating routine.  Its scratch -- the
  * partial-row slots of strips shared between CTAs, their arrival counters, a status word -- is a 688,384-byte
  * array inside the library image, resident on every device that loads the library until the process exits.
@@ -296,6 +297,15 @@ FDQP_API fdqp_status fdqp_run_host_async(fdqp_ctx* ctx, const void* x_host_bf16,
  * FDQP_ERR_SIZE, FDQP_ERR_ARCH, FDQP_ERR_CUDA. */
 FDQP_API fdqp_status fdqp_run_noalloc(const void* x_bf16, const void* W_q4nx, float* y, int64_t M, int64_t K,
                                       int64_t N, void* cuda_stream);
+
+/* Did a kernel of fdqp_run_noalloc give up on a bounded wait?  That entry point has no context to keep a status in,
+ * so its kernels record FDQP_ERR_TIMEOUT in a word of the scratch array; this call copies that word back from the
+ * CURRENT device (one blocking 4-byte device-to-host copy: call it after synchronising the stream; it allocates
+ * nothing).  FDQP_OK when no kernel gave up, or when fdqp_run_noalloc has not run on this device yet;
+ * FDQP_ERR_TIMEOUT once one did -- sticky until the process exits, and the y of that call is undefined (the next
+ * call clears the arrival counters it uses, so later calls are unaffected).  FDQP_ERR_CUDA if the copy fails.
+ * (The paper has no counterpart.) */
+FDQP_API fdqp_status fdqp_noalloc_last_status(void);
 
 /* ---- the dequantisation engine (Sec. "Dequantization Engine", Eq. 3) ------- */
 
@@ -370,7 +380,6 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *                   tensor memory and read from there by the MMAs (two CTAs per SM; up to 64 token rows three smaller
  *                   CTAs per SM when the call has that many to run), 2 = the three-CTA form whenever M <= 64,
  *                   0 = weights in shared memory; same results bit for bit
- *   "debug"         measurement aid: 1 = the GEMV consumers skip the arithmetic (y is then undefined)
  * Unknown key or unusable value: FDQP_ERR_ARG.  Meant for benchmarks and tests. */
 FDQP_API fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t value);
 

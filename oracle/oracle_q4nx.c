@@ -22,8 +22,7 @@
  * "M x K" matrix W has our N as its row count.
  *
  * Byte layout read here ("layout v1"; the paper fixes only the byte budget of
- * a block, every other choice is this build's reading and is listed in the
- * design notes):
+ * a block, every other choice is this build's reading):
  *   strip  s = n / 32, row r = n % 32; strips are stored one after another,
  *   a strip is 20*K bytes.  Inside a strip, blocks b = k / 256 follow each
  *   other; block b holds j_b = min(8, K/32 - 8*b) groups of 32 k-indices and
@@ -51,7 +50,7 @@
  * Microscaling specification defines them).  Pinned by the bit-field definitions of E2M1 / E8M0, exact rational
  * evaluation, equivalence with the group-32 routines on duplicated scales, hand-located bytes and a numpy matmul.
  *
- * Pins (tests/test_oracle_pins.py): the paper's 5120-byte block, hand-written
+ * Pins (checked by the CPU tests): the paper's 5120-byte block, hand-written
  * byte dumps, closed-form worked examples, exact rational evaluation of eq. 3
  * over all codes, an independent fp64 matmul, and invariants.  Parity with
  * the authors' on-disk files and with the NPU's own rounding of eq. 3 is

@@ -27,7 +27,7 @@ EXPORTS = [
     "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
     "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc", "q4nx_packed_bytes_fmt", "q4nx_pack_fmt",
     "q4nx_unpack_fmt", "fdqp_run_fmt", "fdqp_dequant_fmt", "fdqp_run_add_rmsnorm_epilogue",
-    "fdqp_selftest_bounded_wait",
+    "fdqp_selftest_bounded_wait", "fdqp_noalloc_last_status",
 ]
 
 
@@ -88,6 +88,8 @@ def load_library():
     lib.fdqp_run_host_async.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_run_noalloc.restype = ci
     lib.fdqp_run_noalloc.argtypes = [vp, vp, vp, i64, i64, i64, vp]
+    lib.fdqp_noalloc_last_status.restype = ci
+    lib.fdqp_noalloc_last_status.argtypes = []
     lib.fdqp_dequant.restype = ci
     lib.fdqp_dequant.argtypes = [vp, vp, vp, ci, i64, i64, vp]
     lib.fdqp_last_status.restype = ci
@@ -245,6 +247,12 @@ def fdqp_run_noalloc(x_bf16, W_q4nx, y, M: int, K: int, N: int, stream=None) -> 
     Runs on the current device; all calls share one scratch array, so keep them ordered on a stream."""
     _check(load_library().fdqp_run_noalloc(_addr(x_bf16), _addr(W_q4nx), _addr(y), M, K, N, _stream(stream)),
            "fdqp_run_noalloc")
+
+
+def fdqp_noalloc_last_status() -> int:
+    """Status word of fdqp_run_noalloc on the current device (0, or 8 once a kernel gave up on a bounded wait).
+    One blocking 4-byte copy: call it after synchronising the stream."""
+    return int(load_library().fdqp_noalloc_last_status())
 
 
 def fdqp_dequant(ctx: int, W_q4nx, out, out_is_bf16: bool, K: int, N: int, stream=None) -> None:

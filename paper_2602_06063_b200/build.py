@@ -1,40 +1,63 @@
-"""Builds libfdqp.so (CUDA kernels + C ABI) in-tree with nvcc for sm_100a."""
+"""Builds libfdqp.so (CUDA kernels + C ABI) in-tree with nvcc for sm_100a.
+
+Every source under csrc/ is compiled to an object of its own (in parallel, re-used while it is newer than every
+input) and the objects are linked into one shared library."""
 from __future__ import annotations
 
 import glob
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
+OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libfdqp.so")
 
-NVCC_FLAGS = [
+COMPILE_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-shared", "-cudart", "static",
+    "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
 ]
+LINK_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "static"]
 
 
 def sources() -> list[str]:
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")) + glob.glob(os.path.join(CSRC, "*.cpp")))
 
 
-def _newest_input() -> float:
-    files = sources() + glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh"))
-    files += glob.glob(os.path.join(ROOT, "include", "*.h")) + [os.path.abspath(__file__)]
+def _headers() -> list[str]:
+    files = glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh"))
+    return files + glob.glob(os.path.join(ROOT, "include", "*.h")) + [os.path.abspath(__file__)]
+
+
+def _newest(files) -> float:
     return max(os.path.getmtime(f) for f in files)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every source under csrc/ into libfdqp.so; no-op when it is up to date."""
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_input():
+    """Compile every source under csrc/ and link libfdqp.so; no-op when it is up to date."""
+    srcs = sources()
+    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest(srcs + _headers()):
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    os.makedirs(OBJ, exist_ok=True)
+    hdr_time = _newest(_headers())
+
+    def compile_one(src: str) -> str:
+        obj = os.path.join(OBJ, os.path.basename(src) + ".o")
+        if not force and os.path.exists(obj) and os.path.getmtime(obj) >= max(hdr_time, os.path.getmtime(src)):
+            return obj
+        cmd = [nvcc] + COMPILE_FLAGS + (["-Xptxas", "-v"] if verbose else [])
+        cmd += ["-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c", "-o", obj, src]
+        subprocess.check_call(cmd)
+        return obj
+
+    with ThreadPoolExecutor(max_workers=min(8, len(srcs))) as pool:
+        objs = list(pool.map(compile_one, srcs))
     tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp] + sources()
-    subprocess.check_call(cmd)
+    subprocess.check_call([nvcc] + LINK_FLAGS + ["-o", tmp] + objs)
     os.replace(tmp, LIB)
     return LIB
 

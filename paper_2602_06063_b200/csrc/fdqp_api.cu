@@ -23,7 +23,8 @@ cudaError_t dequant_launch(const uint8_t* W, void* out, bool out_bf16, int K, in
 cudaError_t dequant_fmt_launch(int fmt, const uint8_t* W, void* out, bool out_bf16, int K, int N, cudaStream_t stream);
 cudaError_t prefill_set_smem_limit();
 cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, uint16_t* y16, int epi, float* ws,
-                           int* status, int M, int K, int N, int pair, int Z, int fmt, int a_tmem, cudaStream_t stream);
+                           int* status, int M, int K, int N, int pair, int Z, int fmt, int a_tmem, cudaStream_t stream,
+                           int* kernels_launched);
 cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* residual, uint16_t* h_out, const uint16_t* gamma, float eps,
                            uint16_t* out, int M, int K, cudaStream_t stream);
 cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* V, float* out, float* ws, int max_splits, int H,
@@ -56,7 +57,7 @@ struct fdqp_ctx {
     int64_t launches = 0;
     std::string last_err;
     // overrides (-1 = automatic)
-    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_debug = -1, p_prep = -1, p_aligned = -1, p_bpw = -1, p_pair = -1, p_pf_split = -1;
+    int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_prep = -1, p_aligned = -1, p_bpw = -1, p_pair = -1, p_pf_split = -1;
     int64_t p_direct_y = 1;  // fdqp_run_host*: small results are stored straight into device-addressable host memory
     int64_t p_atmem = 1;  // tensor-core kernel up to 128 tokens: keep the converted weights in tensor memory
 };
@@ -281,7 +282,6 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     p->off_bar = p->off_part + round_up(L.part_bytes, 128);
     p->smem_bytes = p->off_bar + (2u * (uint32_t)nstage + 6u) * 8u + 512u;  // barriers, then the fused normalisation's sums
     p->evict_first = ctx->p_evict >= 0 ? (ctx->p_evict != 0) : 1;
-    p->debug = ctx->p_debug > 0 ? (int)ctx->p_debug : 0;
     // work items (8 activations each) per CTA if x is prepared in-kernel; beyond this a preparation kernel is cheaper
     p->prep_inline = ctx->p_prep >= 0 ? (int)(ctx->p_prep != 0) : ((int64_t)nbz * 8 * M * 4 <= (int64_t)cw * 32);
     p->ws_edge = ctx->ws_edge;
@@ -458,10 +458,12 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
                 return cuda_fail(ctx, e, "x spreading copy");
             xt = reinterpret_cast<const uint16_t*>(ctx->x_spread);
         }
+        int kernels = 0;
         if ((e = prefill_launch(W, xt, x_row_bytes, y, y16, epi, ctx->pf_ws, ctx->status_dev, (int)M, (int)K, (int)N,
-                                use_pair(ctx, M) ? 1 : 0, prefill_slices(ctx, M, K, N), fmt, prefill_tmem_mode(ctx, M, K, N), stream)))
+                                use_pair(ctx, M) ? 1 : 0, prefill_slices(ctx, M, K, N), fmt, prefill_tmem_mode(ctx, M, K, N), stream,
+                                &kernels)))
             return cuda_fail(ctx, e, "prefill kernel launch");
-        ctx->launches += prefill_slices(ctx, M, K, N) > 1 ? 2 : 1;
+        ctx->launches += kernels;
         return FDQP_OK;
     }
     // Token rows are processed eight at a time by the streaming GEMV kernel.
@@ -487,12 +489,6 @@ fdqp_status run_impl(fdqp_ctx* ctx, const void* x_bf16, const void* gamma_bf16, 
                 return cuda_fail(ctx, e, "x preparation launch");
             ctx->launches += 1;
         }
-#ifdef FDQP_TRACE
-        {
-            static int trace_seq = 0;  // trace builds only: launch slot of the per-CTA timeline
-            plan.debug |= (trace_seq++ & 31) << 8;
-        }
-#endif
         if ((e = gemv_launch(plan, cw, stream))) return cuda_fail(ctx, e, "gemv kernel launch");
         ctx->launches += 1;
         if (plan.Z > 1) {
@@ -700,8 +696,6 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
     } else if (!std::strcmp(key, "l2_evict_first")) {
         if (v > 1) return FDQP_ERR_ARG;
         ctx->p_evict = v;
-    } else if (!std::strcmp(key, "debug")) {
-        ctx->p_debug = v;
     } else if (!std::strcmp(key, "blocks_per_warp")) {
         if (v != -1 && v != 2 && v != 4) return FDQP_ERR_ARG;
         ctx->p_bpw = v;
@@ -775,6 +769,7 @@ namespace {
 
 constexpr int kNoAllocMaxCtas = 320;                  // partial-row slots: two per persistent CTA
 constexpr int64_t kNoAllocMaxN = 262144;              // arrival counters: one per 32-row strip
+constexpr int64_t kNoAllocMaxK = 1 << 20;             // far beyond what shared memory holds without a K split
 constexpr size_t kNoAllocEdgeBytes = (size_t)kNoAllocMaxCtas * 2 * kStripRows * kMaxTokens * sizeof(float);
 constexpr size_t kNoAllocTicketBytes = (size_t)(kNoAllocMaxN / kStripRows) * sizeof(int);
 constexpr size_t kNoAllocScratchBytes = kNoAllocEdgeBytes + kNoAllocTicketBytes + 256;  // + status word
@@ -800,7 +795,7 @@ extern "C" fdqp_status fdqp_run_noalloc(const void* x_bf16, const void* W_q4nx, 
                                         void* cuda_stream) {
     if (!x_bf16 || !W_q4nx || !y) return FDQP_ERR_ARG;
     if (M < 1 || K <= 0 || N <= 0 || (K % kGroup) != 0 || (N % kStripRows) != 0) return FDQP_ERR_SHAPE;
-    if (M > kMaxTokens || N > kNoAllocMaxN) return FDQP_ERR_SIZE;
+    if (M > kMaxTokens || N > kNoAllocMaxN || K > kNoAllocMaxK) return FDQP_ERR_SIZE;
     if (!aligned16(x_bf16) || !aligned16(W_q4nx) || !aligned16(y)) return FDQP_ERR_ALIGN;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoAllocMaxDevices) {
@@ -814,11 +809,13 @@ extern "C" fdqp_status fdqp_run_noalloc(const void* x_bf16, const void* W_q4nx, 
         NoAllocDevice& d = g_noalloc_devices[dev];
         if (!d.ready) {
             int major = 0;
-            if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return FDQP_ERR_CUDA;
+            if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) { cudaGetLastError(); return FDQP_ERR_CUDA; }
             if (major != 10) return FDQP_ERR_ARCH;
             if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-                cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+                cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+                cudaGetLastError();
                 return FDQP_ERR_CUDA;
+            }
             if (gemv_set_smem_limit(d.smem_optin) != cudaSuccess) { cudaGetLastError(); return FDQP_ERR_CUDA; }
             void* ptr = nullptr;
             if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) { cudaGetLastError(); return FDQP_ERR_CUDA; }
@@ -853,4 +850,26 @@ extern "C" fdqp_status fdqp_run_noalloc(const void* x_bf16, const void* W_q4nx, 
     if (cudaMemsetAsync(plan.tickets, 0, sizeof(int) * (size_t)plan.S, stream) != cudaSuccess) { cudaGetLastError(); return FDQP_ERR_CUDA; }
     if (gemv_launch(plan, cw, stream) != cudaSuccess) { cudaGetLastError(); return FDQP_ERR_CUDA; }
     return FDQP_OK;
+}
+
+// The status word of fdqp_run_noalloc lives in the scratch array (there is no context to hold it).  One blocking 4-byte
+// copy from the current device; allocates nothing.
+extern "C" fdqp_status fdqp_noalloc_last_status(void) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoAllocMaxDevices) {
+        cudaGetLastError();
+        return FDQP_ERR_CUDA;
+    }
+    unsigned char* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_devices[dev].ready) return FDQP_OK;  // no call on this device yet
+        scratch = g_noalloc_devices[dev].scratch;
+    }
+    int v = 0;
+    if (cudaMemcpy(&v, scratch + kNoAllocEdgeBytes + kNoAllocTicketBytes, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return FDQP_ERR_CUDA;
+    }
+    return v == 0 ? FDQP_OK : static_cast<fdqp_status>(v);
 }

@@ -73,13 +73,6 @@ __device__ __forceinline__ float* piece_slot(const GemvPlan& p, int z, int64_t c
     return p.ws_edge + (((int64_t)z * p.Gz + ci) * 2 + which) * (kStripRows * kMaxTokens);
 }
 
-#ifdef FDQP_TRACE
-// 32 launch slots (plan.debug bits 8..12) x 256 CTAs x 16 stamps
-__device__ unsigned long long g_fdqp_trace[32 * 256 * 16];
-#define FDQP_STAMP(i) do { if (lane == 0) g_fdqp_trace[(((p.debug >> 8) & 31) * 256 + (blockIdx.x & 255)) * 16 + (i)] = globaltimer_ns(); } while (0)
-#else
-#define FDQP_STAMP(i) do { } while (0)
-#endif
 
 // ---- activation preparation ------------------------------------------------------------------------
 //
@@ -485,7 +478,6 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
     const int nt = (npieces >= 2 && e < (s_last + 1) * len) ? (int)(e - tail_begin) : 0;
     const int bl_tail = (int)(tail_begin - s_last * len);
     const int nchunk = (nblk + CB - 1) / CB;
-    if (warp == 0) FDQP_STAMP(0);
 
     const uint32_t ring = smem_u32(smem);
     const uint32_t xs = ring + p.off_xs, xsc = ring + p.off_xsum;
@@ -507,7 +499,6 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
     float* const norm_q = reinterpret_cast<float*>(smem + p.off_bar + (2u * (uint32_t)nstage + 6u) * 8u);
     mbar_fence_init();
     __syncthreads();
-    if (warp == 0) FDQP_STAMP(1);
     // The next launch in the stream may begin as soon as SM slots free up: it streams weights (which nothing in this
     // library writes) and waits for this grid to complete before it touches activations, outputs or workspace.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -674,7 +665,6 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
 
         // Everything up to here touched only this CTA's shared memory.  x may come from the previous launch.
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        if (warp == 0) FDQP_STAMP(6);
         if (p.prep_inline) {
             // prepare this CTA's K slice of x straight into shared memory (cheap, and the first weights are still
             // on their way from HBM)
@@ -694,10 +684,6 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                     const int tm = idx >> 2;
                     v[u] = xprep_load(p.x, K, tile0 + (valid ? tm / M : 0), valid ? tm % M : 0, idx & 3, valid);
                 }
-#ifdef FDQP_TRACE
-                asm volatile("" ::"r"(v[0].x), "r"(v[kBatch - 1].x));
-                if (warp == 0 && base == 0) FDQP_STAMP(8);
-#endif
                 if (EPI && p.norm) {
                     // RMS normalisation in place (the plan guarantees one item per thread at most and the whole row in
                     // this CTA): sum of squares per token over all quads, then x <- bf16(x * r * (1 + gamma))
@@ -751,17 +737,14 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                     }
                 }
             }
-            if (warp == 0) FDQP_STAMP(9);
             asm volatile("bar.sync 1, %0;" ::"n"(CW * 32) : "memory");
         } else if (!mbar_wait(x_bar, 0, p.status)) {
             alive = false;
         }
-        if (warp == 0) FDQP_STAMP(2);
-        const bool work = !(p.debug & 1);
         // An "interior" stage -- both of the warp's blocks inside the range and the current strip, every block
         // full -- needs no bookkeeping beyond two tile indices.  `lim` is the first position that is not interior.
         const bool all_full = (groups_total & 7) == 0;
-        auto interior_limit = [&]() { return (all_full && work) ? (unit_next < nblk ? unit_next : nblk) : -1; };
+        auto interior_limit = [&]() { return all_full ? (unit_next < nblk ? unit_next : nblk) : -1; };
         int lim = interior_limit();
         int stage = 0;
         uint32_t phase = 0;
@@ -772,7 +755,6 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                 lim = interior_limit();
             }
             if (!mbar_wait(full0 + 8u * stage, phase, p.status)) { alive = false; break; }
-            if (warp == 0 && c == 0) FDQP_STAMP(3);
             const uint32_t sbase = ring + stage * kStageBytes + j0 * kBB;
             if (i0 + BPW - 1 < lim) {
                 const int tile = (i0 - unit_first) * 8 + tw;
@@ -790,7 +772,7 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                     }
                     tile_compute<MODE, FMT>(tb, acc, acc_m, lc);
                 }
-            } else if (all_full && work && i0 + BPW <= nblk && unit_next > i0 && unit_next - first_fix + len >= i0 + BPW) {
+            } else if (all_full && i0 + BPW <= nblk && unit_next > i0 && unit_next - first_fix + len >= i0 + BPW) {
                 // exactly one strip boundary inside the warp's blocks, every block full and inside the range: the blocks
                 // before it, the hand-off of the finished strip piece, the blocks after it -- two tiles in flight
                 // wherever two neighbours are on the same side
@@ -831,7 +813,7 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                     const int bl = i - unit_first;
                     const int rest = groups_total - 8 * (b_first + bl);
                     const int jb = rest < 8 ? rest : 8;
-                    if (work && tw < jb) {
+                    if (tw < jb) {
                         const uint32_t sb = sbase + jj * kBB;
                         const int tile = bl * 8 + tw;
                         TileIn ta;
@@ -847,16 +829,12 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             }
             if (++stage == nstage) { stage = 0; phase ^= 1u; }
         }
-        if (warp == 0) FDQP_STAMP(4);
         while (piece < npieces && alive) flush();
     } else {
         // =============================== reducer =================================================
         // The prepared activations of this CTA's K slice: one barrier, a few large copies.  They are written by
         // the preparation kernel this launch may overlap with, hence the dependency wait first.
         asm volatile("griddepcontrol.wait;" ::: "memory");  // before any global write of this grid
-#ifdef FDQP_TRACE
-        if (warp == CW + 1) { mbar_wait(full0, 0, p.status); FDQP_STAMP(7); }
-#endif
         if (warp == CW + 1 && lane == 0 && !p.prep_inline) {
             const int kbeg = b_first * kBlockK;
             const int kend_full = (b_first + len) * kBlockK;
@@ -973,7 +951,6 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                 }
             }
         }
-        if (warp == CW + 1) FDQP_STAMP(5);
     }
 }
 
@@ -993,11 +970,6 @@ __global__ void __launch_bounds__(256) fdqp_splitk_sum_kernel(const float* __res
     store_output(y, y16, epi, N, s, r, tok, acc);
 }
 
-#ifdef FDQP_TRACE
-extern "C" __attribute__((visibility("default"))) int fdqp_trace_read(unsigned long long* host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, g_fdqp_trace, sizeof(unsigned long long) * n);
-}
-#endif
 
 // RMS normalisation on its own (the calls whose activation preparation does not happen inside a GEMV CTA): one CTA per
 // token row, out[m][k] = bf16(x * rsqrt(mean(x^2) + eps) * (1 + gamma[k])).

@@ -51,7 +51,6 @@ struct GemvPlan {
     int evict_first;      // weight copies carry an evict-first L2 hint
     int strip_aligned;    // 1: CTA ranges are cut at strip boundaries (no strip is shared between CTAs of a slice)
     int prep_inline;      // 1: every CTA prepares its K slice of x itself; 0: a preparation kernel ran before
-    int debug;            // measurement aid: bit 0 = consumers skip the arithmetic (results are then undefined)
     uint32_t off_xs;      // shared-memory offsets (bytes): prepared-x records, per-token scalars,
     uint32_t off_xsum;    //   partial rows, barriers
     uint32_t off_part;

@@ -359,26 +359,8 @@ __device__ __forceinline__ void stage_copy_out(uint32_t stage, uint16_t* dst, in
 
 // ---- the kernel -------------------------------------------------------------------------------------------------------
 
-#ifdef FDQP_TRACE
-// trace builds only: 16 time stamps / counters for each of the first 512 CTAs of the last launch
-__device__ unsigned long long g_pf_trace[512 * 16];
-#define PF_STAMP(i) do { if (blockIdx.x < 512) g_pf_trace[blockIdx.x * 16 + (i)] = globaltimer_ns(); } while (0)
-#define PF_ADD(i, v) do { if (blockIdx.x < 512) g_pf_trace[blockIdx.x * 16 + (i)] += (v); } while (0)
-#define PF_T0() const unsigned long long pf_t0 = globaltimer_ns()
-#define PF_DT() (globaltimer_ns() - pf_t0)
-extern "C" __attribute__((visibility("default"))) int fdqp_pf_trace_read(unsigned long long* host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, g_pf_trace, sizeof(unsigned long long) * (size_t)n);
-}
-extern "C" __attribute__((visibility("default"))) int fdqp_pf_trace_clear() {
-    static unsigned long long zeros[512 * 16];
-    return (int)cudaMemcpyToSymbol(g_pf_trace, zeros, sizeof(zeros));
-}
-#else
-#define PF_STAMP(i) do { } while (0)
-#define PF_ADD(i, v) do { } while (0)
 #define PF_T0() do { } while (0)
 #define PF_DT() 0
-#endif
 
 // ROWS: output features per CTA tile.  256: the tile described above, one CTA per SM.  128 (for M <= 128): a 128 x 128
 // tile with half-size stages (16 KB + 16 KB), eight conversion warps and 128 TMEM columns, so that TWO CTAs share an SM:
@@ -428,7 +410,6 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, TRI ? 3 : Pf1<ROWS>::kCta
     const int ks0 = z * p.ksteps_z;                                                // first k-step of this slice
     const int ksteps = (ksteps_all - ks0) < p.ksteps_z ? (ksteps_all - ks0) : p.ksteps_z;
     float* const yout = p.y + (int64_t)z * p.M * p.N;
-    if (tid == 0) PF_STAMP(0);
 
     if (tid == 0) {
         for (int s = 0; s < NA; ++s) {
@@ -452,7 +433,6 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, TRI ? 3 : Pf1<ROWS>::kCta
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_g;
     bool ok = true;
-    if (tid == 0) PF_STAMP(1);
 
     if (warp == 0) {
         // =============================== TMA producer: x tiles ==============================================
@@ -472,32 +452,12 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, TRI ? 3 : Pf1<ROWS>::kCta
         {
             const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot_g, 0);
             const uint32_t idesc = umma_idesc(n_inst);
-#ifdef FDQP_TRACE
-            unsigned long long tr_wa = 0, tr_wb = 0, tr_is = 0;
-#endif
             for (int i = 0; i < ksteps && ok; ++i) {
                 const int sa = i % NA, sb = i % NB;
                 const uint32_t pha = (i / NA) & 1, phb = (i / NB) & 1;
-#ifdef FDQP_TRACE
-                {
-                    PF_T0();
-                    ok = mbar_wait(full_a(sa), pha, p.status);
-                    tr_wa += PF_DT();
-                }
-                {
-                    PF_T0();
-                    ok = ok && mbar_wait(full_b(sb), phb, p.status);
-                    tr_wb += PF_DT();
-                }
-                if (i == 0 && lane == 0) PF_STAMP(2);
-#else
                 ok = mbar_wait(full_a(sa), pha, p.status) && mbar_wait(full_b(sb), phb, p.status);
-#endif
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-#ifdef FDQP_TRACE
-                const unsigned long long pf_m0 = globaltimer_ns();
-#endif
                 tc_fence_after();
                 const uint32_t a_addr = base + sa * P::kStageBytes, b_addr = base + sb * kBStride + kBOff;
                 if (lane != 0) continue;
@@ -519,17 +479,8 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, TRI ? 3 : Pf1<ROWS>::kCta
                 }
                 umma_commit(empty_a(sa));  // the stages may be refilled once these MMAs have read them
                 umma_commit(empty_b(sb));
-#ifdef FDQP_TRACE
-                tr_is += globaltimer_ns() - pf_m0;
-#endif
             }
             if (lane == 0) {
-                PF_STAMP(6);
-#ifdef FDQP_TRACE
-                PF_ADD(12, tr_wa);
-                PF_ADD(13, tr_wb);
-                PF_ADD(14, tr_is);
-#endif
                 umma_commit(acc_done);
             }
         }
@@ -546,37 +497,17 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, TRI ? 3 : Pf1<ROWS>::kCta
         const int gbase = 2 * ks0 + gl;  // this warp's group in k-step i of the slice: gbase + 2 i
         // Eight register sets, each reloaded right after it has been converted.  (Rotating the sets with moves instead --
         // g0 = g1; g1 = g2; g2 = just-loaded -- makes the move wait for the load it follows, one trip to memory per k-step.)
-#ifdef FDQP_TRACE
-        unsigned long long tr_wait = 0, tr_conv = 0, tr_st = 0, tr_arr = 0, tr_load = 0;
-        unsigned long long tr_rt = 0, tr_arrived[4] = {0, 0, 0, 0};  // round trip: arrive on a stage -> the stage seen free again
-#endif
         auto convert_step = [&](int i, const GroupRegs& g) -> bool {
             const int s = i % NA;
-#ifdef FDQP_TRACE
-            const unsigned long long pf_w0 = globaltimer_ns();
-#endif
             if (i >= NA && !mbar_wait(empty_a(s), ((i / NA) - 1) & 1, p.status)) return false;
-#ifdef FDQP_TRACE
-            const unsigned long long pf_w1 = globaltimer_ns();
-            if (i >= NA) tr_rt += pf_w1 - tr_arrived[i & 3];
-#endif
             if (ATMEM) {
                 // this lane's row of the group, 16 bf16 pairs, into its TMEM lane; ordered against the MMAs that read the
                 // stage before (the barrier wait above) and after (the arrive below) by the tensor-core fences
                 uint32_t wreg[16];
                 group_convert<FMT>(g, wreg);
-#ifdef FDQP_TRACE
-                asm volatile("" ::"r"(wreg[0]), "r"(wreg[15]));
-                const unsigned long long pf_c1 = globaltimer_ns();
-                tr_conv += pf_c1 - pf_w1;
-#endif
                 tc_fence_after();
                 tmem_st_16cols(tmem_base + ((uint32_t)(sl * 32) << 16) + kTmemA + (uint32_t)(s * (kPfK / 2) + gl * 16), wreg);
                 tc_fence_before();
-#ifdef FDQP_TRACE
-                const unsigned long long pf_c2 = globaltimer_ns();
-                tr_st += pf_c2 - pf_c1;
-#endif
             } else {
                 group_store<FMT>(base + s * P::kStageBytes, g, sl, gl, lane);
                 // make the generic-proxy stores visible to the tensor core's (async-proxy) reads, then signal
@@ -584,11 +515,6 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, TRI ? 3 : Pf1<ROWS>::kCta
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(full_a(s));
-#ifdef FDQP_TRACE
-            tr_wait += pf_w1 - pf_w0;
-            tr_arrived[i & 3] = globaltimer_ns();
-            tr_arr += tr_arrived[i & 3] - pf_w1;
-#endif
             return true;
         };
         if (TRI) {
@@ -654,20 +580,9 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, TRI ? 3 : Pf1<ROWS>::kCta
             }
         }
         }
-#ifdef FDQP_TRACE
-        if (dw == 0 && lane == 0) {
-            PF_ADD(11, tr_wait);
-            PF_ADD(3, tr_conv);
-            PF_ADD(4, tr_st);
-            PF_ADD(15, tr_arr);
-            PF_ADD(5, tr_load);
-            PF_ADD(10, tr_rt);
-        }
-#endif
         // =============================== epilogue: TMEM -> y =================================================
         if (ok) ok = mbar_wait(acc_done, 0, p.status);
         ok = __all_sync(0xffffffffu, ok);
-        if (dw == 0 && lane == 0) PF_STAMP(7);
         const bool via_smem = p.epi != kEpiNone && p.Z == 1;  // bf16 epilogues (a K-split call leaves them to the sum)
         const bool geglu = p.epi == kEpiGegluBf16;
         const int cols = geglu ? P::kRows / 2 : P::kRows;       // bf16 values per token row of the staged tile
@@ -732,14 +647,12 @@ __global__ void __launch_bounds__(Pf1<ROWS>::kThreads, TRI ? 3 : Pf1<ROWS>::kCta
         }
     }
     // =============================== teardown: every path releases TMEM =====================================
-    if (warp == 2 && lane == 0) PF_STAMP(8);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
     }
-    if (tid == 0) PF_STAMP(9);
 }
 
 // ---- the two-SM kernel (M > 256) ----------------------------------------------------------------------------------
@@ -1144,8 +1057,11 @@ static cudaError_t prefill_launch_kernels(const CUtensorMap& map, const PrefillP
 // x_row_bytes: distance between token rows of x (K * 2 for a dense [M][K] array; a multiple of 16).
 // epi: kEpiNone writes fp32 y; the other epilogues write bf16 to y16 (see fdqp_plan.h).
 // fmt: the container's format (fdqp_format.h).
+// kernels_launched (may be null): receives 1, or 2 when the K slices needed the second kernel.
 cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_bytes, float* y, uint16_t* y16, int epi, float* ws,
-                           int* status, int M, int K, int N, int pair, int Z, int fmt, int a_tmem, cudaStream_t stream) {
+                           int* status, int M, int K, int N, int pair, int Z, int fmt, int a_tmem, cudaStream_t stream,
+                           int* kernels_launched) {
+    if (kernels_launched) *kernels_launched = 0;
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     CUtensorMap map;
@@ -1183,7 +1099,9 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_by
         case kFmtMxfp4: err = prefill_launch_kernels<kFmtMxfp4>(map, p, pair, a_tmem, M, N, Z, stream); break;
         default: return cudaErrorInvalidValue;
     }
-    if (err != cudaSuccess || Z == 1) return err;
+    if (err != cudaSuccess) return err;
+    if (kernels_launched) *kernels_launched = Z > 1 ? 2 : 1;
+    if (Z == 1) return err;
     if (epi != kEpiNone) {
         const int64_t total = (int64_t)M * N;
         fdqp_prefill_sum_epi_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(ws, y16, epi, Z, M, N);

@@ -231,8 +231,8 @@ def test_one_hot_reads_out_dequantised_rows(fresh):
     y = Case(K, N, 8, 0, weights=case.w, x=synthgen.bf16_bits(x)).run(fresh)
     want = w32[ks].astype(np.float64)
     assert np.all(np.abs(y - want) <= REL_TOL * np.abs(want) + ABS_TOL)
-    # (the GEMV forms d*S + (m - 128 d)*X with several roundings, so this read-out is close, not bit-equal;
-    # the bit-exact statement of Eq. 3 is fdqp_dequant's)
+    # (the GEMV forms d * 2^e * (integer sum) + m * (sum of x) with two roundings, so this read-out is close, not
+    # necessarily bit-equal; the bit-exact statement of Eq. 3 is fdqp_dequant's)
 
 
 def test_zero_and_offsets_only(fresh):
