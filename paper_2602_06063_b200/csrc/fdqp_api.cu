@@ -195,8 +195,8 @@ SmemLayout smem_layout(const fdqp_ctx* ctx, int M, int nbz, int cw, int ctas_per
     SmemLayout L;
     L.stage_bytes = (uint32_t)(cw / 8) * (uint32_t)bpw * (uint32_t)fmt_block_bytes(fmt);
     const uint32_t tiles = (uint32_t)nbz * 8u;
-    L.xs_bytes = tiles * 128u * (uint32_t)M;          // prepared activations of the K slice
-    L.xsum_bytes = M <= kColsMaxTokens ? 0u : tiles * 64u;         // per-token {sum x, unit} (plane mode only)
+    L.xs_bytes = tiles * (uint32_t)(M <= kColsMaxTokens ? kColsRecBytes : kPlaneRecBytes) * (uint32_t)M;  // prepared activations of the K slice
+    L.xsum_bytes = M <= kColsMaxTokens ? 0u : tiles * (uint32_t)kPlaneSumBytes;  // per-token sums of x (M >= 3 only)
     L.part_bytes = 2u * (uint32_t)cw * kStripRows * (uint32_t)M * 4u * (M <= kColsMaxTokens ? (uint32_t)kColsPartTerms : 1u);
     L.fixed = round_up(L.xs_bytes, 128) + round_up(L.xsum_bytes, 128) + round_up(L.part_bytes, 128) +
               (2u * kMaxStages + 6u) * 8u + 512u + 128u;
@@ -236,7 +236,7 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
             // (measured: pays up to M = 4, never when the larger stage would force a K split)
             bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (M <= 4 && blocks_per_cta >= 4 ? 4 : 2);
             L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw, fmt);
-            if (bpw == 4 && ctx->p_bpw != 4 && M > 1 && L.nstage < kMinStages) {
+            if (bpw == 4 && ctx->p_bpw != 4 && L.nstage < kMinStages) {  // smaller stages before another K slice
                 bpw = 2;
                 L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw, fmt);
             }
@@ -353,9 +353,9 @@ extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, in
         }
         if ((e = cudaMemset(ctx->tickets, 0, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
         const size_t tiles = (size_t)(max_K / kGroup), toks = (size_t)(max_M < kMaxTokens ? max_M : kMaxTokens);
-        if ((e = cudaMalloc(&ctx->xq, tiles * toks * 128))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMalloc(&ctx->xq, tiles * toks * kColsRecBytes))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->xsc, tiles * 64))) { st = cuda_fail(nullptr, e, ""); break; }
-        if ((e = cudaMemset(ctx->xq, 0, tiles * toks * 128))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMemset(ctx->xq, 0, tiles * toks * kColsRecBytes))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMemset(ctx->xsc, 0, tiles * 64))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaHostAlloc(&ctx->status_host, sizeof(int), cudaHostAllocMapped))) { st = cuda_fail(nullptr, e, ""); break; }
         *ctx->status_host = 0;

@@ -39,26 +39,9 @@
 // strip-aligned and added by fdqp_splitk_sum_kernel instead).  A CTA handles the shared strip at the END of its range FIRST, so that the exchange through
 // global memory is off its critical path and its last piece is a whole strip written directly.
 // No CTA ever waits for another CTA.
-#include "fdqp_device.cuh"
-#include "fdqp_format.h"
-#include "fdqp_plan.h"
+#include "fdqp_gemv_tile.cuh"
 
 namespace fdqp {
-
-// 32-bit arithmetic is exact (and an order of magnitude cheaper than a 64-bit division) while (G + 1)(T + 1) < 2^32.
-__device__ __forceinline__ bool fits32(int64_t G, int64_t T) { return (((uint64_t)(G + 1) * (uint64_t)(T + 1)) >> 32) == 0; }
-__device__ __forceinline__ int64_t div_floor(int64_t a, int64_t b, bool small) {
-    return small ? (int64_t)((uint32_t)a / (uint32_t)b) : a / b;
-}
-__device__ __forceinline__ int64_t range_begin(int64_t ci, int64_t G, int64_t T) {
-    if (fits32(G, T)) return (int64_t)(((uint32_t)ci * (uint32_t)T) / (uint32_t)G);
-    return (ci * T) / G;
-}
-// index of the CTA whose range [range_begin(ci), range_begin(ci+1)) contains L
-__device__ __forceinline__ int64_t cta_of(int64_t L, int64_t G, int64_t T) {
-    if (fits32(G, T)) return (int64_t)((((uint32_t)L + 1u) * (uint32_t)G - 1u) / (uint32_t)T);
-    return ((L + 1) * G - 1) / T;
-}
 
 __device__ __forceinline__ int slice_len(const GemvPlan& p, int z) {
     const int rest = p.nb - z * p.nbz;
@@ -74,100 +57,6 @@ __device__ __forceinline__ float* piece_slot(const GemvPlan& p, int z, int64_t c
 }
 
 
-// ---- activation preparation ------------------------------------------------------------------------
-//
-// One thread per (group-tile T, token, quarter q): eight consecutive activations, turned into fixed point
-// relative to the largest exponent of the 32-group and split into byte planes in MMA fragment order
-// ({bytes of even k, bytes of odd k} per plane).
-//
-// M >= 3 (SINGLE == false): 23-bit fixed point, planes 2 (signed), 1, 0 (unsigned).  Record of 32 bytes at
-//   xq[((T*M + tok)*4 + q)*32]: words 0..5 = planes 2, 1, 0; words 6, 7 = {sum of the group's x, unit 2^e_g};
-//   and xsc[T*16 + (tok/2)*4 + (tok%2)*2 + {0,1}] holds the same two scalars indexed by token.
-// M <= 2 (SINGLE == true, "column" layout): 23-bit fixed point in three SIGNED digits.  Per (tile, token) 128 bytes:
-//   [plane 2: 4 x 8 B by q][plane 1][plane 0][{sum x, unit}][8 zero bytes][16 bytes: see next line];
-//   the last 16 bytes of TOKEN 0's record start with the group sums of x of tokens 0 and 1 of that tile.
-// `tile` is the group-tile index in x, `slot` the tile's index in the destination (global: the same; shared
-// memory: relative to the CTA's K slice).  Must be called by whole quads (the four q of a (tile, token)).
-__device__ __forceinline__ uint4 xprep_load(const uint16_t* __restrict__ x, int K, int tile, int tok, int q, bool valid) {
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (valid) v = *reinterpret_cast<const uint4*>(x + (int64_t)tok * K + tile * kGroup + q * 8);
-    return v;
-}
-
-// Eight bf16 sums, each rounded once from the exact sum (the residual stream of a decoder layer stays in bf16).
-__device__ __forceinline__ uint4 add_bf16x8(uint4 a, uint4 b) {
-    uint4 r;
-    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r.x) : "r"(a.x), "r"(b.x));
-    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r.y) : "r"(a.y), "r"(b.y));
-    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r.z) : "r"(a.z), "r"(b.z));
-    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r.w) : "r"(a.w), "r"(b.w));
-    return r;
-}
-
-template <bool SINGLE>
-__device__ __forceinline__ void xprep_item(const uint4 v, int M, int slot, int tok, int q, bool valid,
-                                           uint32_t* __restrict__ xq, float* __restrict__ xsc) {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    float f[8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        f[2 * i] = __uint_as_float(w[i] << 16);
-        f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-    float amax = fmaxf(fmaxf(fmaxf(fabsf(f[0]), fabsf(f[1])), fmaxf(fabsf(f[2]), fabsf(f[3]))),
-                       fmaxf(fmaxf(fabsf(f[4]), fabsf(f[5])), fmaxf(fabsf(f[6]), fabsf(f[7]))));
-    float psum = ((f[0] + f[1]) + (f[2] + f[3])) + ((f[4] + f[5]) + (f[6] + f[7]));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-    psum += __shfl_xor_sync(0xffffffffu, psum, 1);
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-    psum += __shfl_xor_sync(0xffffffffu, psum, 2);
-    // exponent field of the group's largest magnitude, kept where both scale factors are normal floats
-    constexpr int kFrac = 21;  // |fixed-point value| <= 2^22: the plane sums of a group recombine inside an int32
-    int emax = (int)(__float_as_uint(amax) >> 23);
-    emax = emax < 24 ? 24 : (emax > 254 ? 254 : emax);
-    const float to_fixed = __uint_as_float((uint32_t)(254 + kFrac - emax) << 23);  // 2^(127 + kFrac - emax)
-    const float unit = __uint_as_float((uint32_t)(emax - kFrac) << 23);            // 2^(emax - 127 - kFrac)
-    // Round to the nearest integer I (ties to even) by adding 1.5 * 2^23: the sum's low mantissa bits are 2^22 + I.
-    // Column layout: bytes 0..2 of (I + 0x808080) ^ 0x808080 are the signed digits of I in base 256
-    // (I = 65536 d2 + 256 d1 + d0, each in [-128, 127]); plane layout: the two's-complement bytes of I themselves
-    // (top byte signed, lower bytes unsigned).
-    constexpr uint32_t kMagicBits = 0x4B400000u;  // bits of 12582912.0f
-    uint32_t J[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const uint32_t bits = __float_as_uint(fmaf(f[i], to_fixed, 12582912.0f));
-        J[i] = SINGLE ? ((bits - (kMagicBits - 0x00808080u)) ^ 0x00808080u) : (bits - kMagicBits);
-    }
-    uint32_t plane[3][2];  // [0] most significant; {even k, odd k}
-#pragma unroll
-    for (int pl = 0; pl < 3; ++pl) {
-        const uint32_t sel = (uint32_t)(2 - pl) | ((uint32_t)(6 - pl) << 4);  // byte 2 - pl of both operands
-        const uint32_t e01 = __byte_perm(J[0], J[2], sel), e23 = __byte_perm(J[4], J[6], sel);
-        const uint32_t o01 = __byte_perm(J[1], J[3], sel), o23 = __byte_perm(J[5], J[7], sel);
-        plane[pl][0] = __byte_perm(e01, e23, 0x5410);
-        plane[pl][1] = __byte_perm(o01, o23, 0x5410);
-    }
-    if (!valid) return;
-    if (SINGLE) {
-        uint32_t* rec = xq + ((int64_t)slot * M + tok) * 32;  // 128 bytes per (tile, token)
-#pragma unroll
-        for (int pl = 0; pl < 3; ++pl)
-            *reinterpret_cast<uint2*>(rec + pl * 8 + q * 2) = make_uint2(plane[pl][0], plane[pl][1]);
-        if (q == 0) *reinterpret_cast<uint2*>(rec + 24) = make_uint2(__float_as_uint(psum), __float_as_uint(unit));
-        if (q == 1) *reinterpret_cast<uint2*>(rec + 26) = make_uint2(0u, 0u);
-        if (q == 2) xq[(int64_t)slot * M * 32 + 28 + tok] = __float_as_uint(psum);
-    } else {
-        uint4* dst = reinterpret_cast<uint4*>(xq + ((int64_t)(slot * M + tok) * 4 + q) * 8);
-        dst[0] = make_uint4(plane[0][0], plane[0][1], plane[1][0], plane[1][1]);
-        dst[1] = make_uint4(plane[2][0], plane[2][1], __float_as_uint(psum), __float_as_uint(unit));
-        if (q == 0) {
-            float* sc = xsc + (int64_t)slot * 16 + (tok >> 1) * 4 + (tok & 1) * 2;
-            sc[0] = psum;
-            sc[1] = unit;
-        }
-    }
-}
-
 // Stand-alone preparation of a whole x, for calls whose K slice is too large to prepare inside every GEMV CTA.
 template <bool SINGLE>
 __global__ void __launch_bounds__(128) fdqp_xprep_kernel(const uint16_t* __restrict__ x, uint32_t* __restrict__ xq,
@@ -182,259 +71,6 @@ __global__ void __launch_bounds__(128) fdqp_xprep_kernel(const uint16_t* __restr
     const int q = idx & 3, tm = idx >> 2;
     const int tok = valid ? tm % M : 0, tile = valid ? tm / M : 0;
     xprep_item<SINGLE>(xprep_load(x, K, tile, tok, q, valid), M, tile, tok, q, valid, xq, xsc);
-}
-
-// ---- one 32 x 32 group-tile -------------------------------------------------------------------------
-
-
-// Kernel modes (see the header comment): derived constants.
-template <int MODE>
-struct ModeTraits {
-    static constexpr bool kCols = MODE != 2;     // planes as MMA columns (M <= kColsMaxTokens)
-    static constexpr int kAcc = kCols ? 1 : 2;   // accumulator columns per lane
-    static constexpr bool kXRow = MODE == 3;     // offset term needs the sums of x of both tokens
-    static constexpr int kAccM = MODE == 3 ? 2 : 1;
-};
-
-struct TileIn {
-    uint32_t c[4];   // code words: word q of rows g, g+8, g+16, g+24
-    uint32_t so[4];  // column modes: (d[g], d[g+8]), (d[g+16], d[g+24]); mode 2 also (m[g], m[g+8]), (m[g+16], m[g+24])
-    uint32_t b[6];   // B fragments {even k, odd k}: mode 2: planes 2, 1, 0; column modes: this lane's column
-    float sc[4];     // mode 2: {sum x, unit} of tokens 2q, 2q+1; column modes: {sum x, unit} of the lane's token
-    float xrow[2];   // mode 3: sum of x of tokens 0, 1 for this group
-    uint32_t m_row;  // column modes: bf16 offset of row `lane` (low half)
-};
-
-// Per-lane pieces of the shared-memory addresses of the prepared activations.
-struct LaneAddr {
-    uint32_t xs, x_stride;   // base and bytes per tile of the prepared-x records
-    uint32_t xb_off;         // column modes: this lane's B column inside the tile
-    uint32_t sc_off;         // column modes: {sum x, unit} of the token whose columns this lane accumulates
-    uint32_t x_lane, xsc_lane;  // mode 2: this lane's record / scalar quad inside tile 0
-};
-
-// Column modes: so_addr addresses the scale chunks only (lanes 0..15 matter); m_addr is this lane's own offset word.
-// MXFP4: so_addr is the byte address of row g's scale of this tile, m_addr that of row `lane`'s; so[0..3] then hold,
-// as fp32 bits, the scales 2^(e-127) of rows g, g+8, g+16, g+24 (a scale byte of 0, i.e. 2^-127, counts as 0 here),
-// m_row that of row `lane`; the B fragments are re-ordered to the natural k order the element look-up produces.
-__device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
-// {even k, odd k} byte order of a B fragment pair -> {k 0..3, k 4..7}
-__device__ __forceinline__ void mx_natural_order(uint32_t& b0, uint32_t& b1) {
-    const uint32_t e = b0, o = b1;
-    b0 = prmt(e, o, 0x5140u);
-    b1 = prmt(e, o, 0x7362u);
-}
-
-template <int MODE, int FMT = kFmtQ4nx>
-__device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_t so_addr, uint32_t m_addr, int tile,
-                                          const LaneAddr& la) {
-    using T = ModeTraits<MODE>;
-    constexpr bool kMx = FmtTraits<FMT>::kMx;
-    ldmatrix_x4(t.c, code_addr);
-    if (kMx) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) t.so[k] = lds_u8(so_addr + 8u * k) << 23;
-    }
-    if (T::kCols) {
-        if (kMx) {
-            t.m_row = lds_u8(m_addr) << 23;
-        } else {
-            uint32_t dd[2];
-            ldmatrix_x2_trans(dd, so_addr);
-            t.so[0] = dd[0];
-            t.so[1] = dd[1];
-            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(t.m_row) : "r"(m_addr));
-        }
-        const uint32_t tb = la.xs + (uint32_t)tile * la.x_stride;
-        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(t.b[0]), "=r"(t.b[1]) : "r"(tb + la.xb_off));
-        const float2 v = lds64f(tb + la.sc_off);
-        t.sc[0] = v.x;
-        t.sc[1] = v.y;
-        if (T::kXRow) {
-            const float2 xr = lds64f(tb + 112u);
-            t.xrow[0] = xr.x;
-            t.xrow[1] = xr.y;
-        }
-        if (kMx) mx_natural_order(t.b[0], t.b[1]);
-    } else {
-        if (!kMx) ldmatrix_x4_trans(t.so, so_addr);
-        const uint32_t x_addr = la.x_lane + (uint32_t)tile * la.x_stride;
-        const uint4 r0 = lds128(x_addr);
-        t.b[0] = r0.x; t.b[1] = r0.y; t.b[2] = r0.z; t.b[3] = r0.w;
-        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(t.b[4]), "=r"(t.b[5]) : "r"(x_addr + 16));
-        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
-                     : "=f"(t.sc[0]), "=f"(t.sc[1]), "=f"(t.sc[2]), "=f"(t.sc[3])
-                     : "r"(la.xsc_lane + (uint32_t)tile * 64u));
-        if (kMx) {
-            mx_natural_order(t.b[0], t.b[1]);
-            mx_natural_order(t.b[2], t.b[3]);
-            mx_natural_order(t.b[4], t.b[5]);
-        }
-    }
-}
-
-// Eight E2M1 codes of a word -> the unsigned bytes 2v + 12 (0 .. 24) of k 0..3 and k 4..7.  A 16-entry table as two
-// byte permutes: a selector nibble with bit 3 set returns the selected byte's sign fill, which is 0 for these bytes, so
-// the table of the non-negative codes answers only codes 0..7 and, with bit 3 flipped, that of the negative codes only
-// codes 8..15.
-// The two answers are disjoint (one of them is 0 in every byte), so they are not merged: each goes through the MMA and
-// the accumulator adds them.
-struct MxBytes {
-    uint32_t pos_lo, pos_hi, neg_lo, neg_hi;
-};
-// The four table words live in registers for the whole kernel (loaded through an opaque move, so that the compiler
-// does not re-create the constants in front of every permute).
-struct MxTables {
-    uint32_t pos0, pos1, neg0, neg1;
-};
-__device__ __forceinline__ MxTables mx_tables() {
-    MxTables t;
-    asm volatile("mov.b32 %0, 0x0F0E0D0C;" : "=r"(t.pos0));  // 12 + {0, 1, 2, 3}
-    asm volatile("mov.b32 %0, 0x18141210;" : "=r"(t.pos1));  // 12 + {4, 6, 8, 12}
-    asm volatile("mov.b32 %0, 0x090A0B0C;" : "=r"(t.neg0));  // 12 - {0, 1, 2, 3}
-    asm volatile("mov.b32 %0, 0x00040608;" : "=r"(t.neg1));  // 12 - {4, 6, 8, 12}
-    return t;
-}
-__device__ __forceinline__ MxBytes mx_codes_to_bytes(uint32_t w, const MxTables& tb) {
-    const uint32_t wn = w ^ 0x88888888u;
-    MxBytes r;
-    r.pos_lo = prmt(tb.pos0, tb.pos1, w);
-    r.neg_lo = prmt(tb.neg0, tb.neg1, wn);
-    r.pos_hi = prmt(tb.pos0, tb.pos1, w >> 16);
-    r.neg_hi = prmt(tb.neg0, tb.neg1, wn >> 16);
-    return r;
-}
-
-// d += A . B (same shapes and types as imma below)
-template <bool B_SIGNED>
-__device__ __forceinline__ void imma_acc(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                         uint32_t b1) {
-    if (B_SIGNED)
-        asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-            : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
-            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-    else
-        asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-            : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
-            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-template <bool B_SIGNED>
-__device__ __forceinline__ void imma(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                     uint32_t b1) {
-    const int zero = 0;  // accumulator start value
-    if (B_SIGNED)
-        asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-            : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
-            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(zero));
-    else
-        asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-            : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
-            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(zero));
-}
-
-// Per-lane constants of the column modes: which two MMA columns the lane holds.  Columns 4*(tok%2) + {0,1,2} are
-// planes 2, 1, 0 of token tok (of the pair), column 3 / 7 is zero; lane q holds columns 2q, 2q+1:
-//   q even: (plane 2, plane 1) -> 256 * s2 + s1, weighted 256 * unit;   q odd: (plane 0, zero) -> s0, weighted unit.
-struct LaneConst {
-    int k_first;       // weight of the first column relative to the second (256 or 1)
-    float w_unit;      // factor on `unit` (0 when the lane's token does not exist)
-    MxTables mx;       // MXFP4 only: the element look-up tables
-};
-
-// acc[row][.] += d * unit * (sum_k q_k X_k) + m * (sum_k x_k), fp32 (Eq. 3 applied per group).
-// `unit` (and 256 * unit) are powers of two, so d * unit is formed exactly by the mixed bf16 FMA.
-// Column modes keep the offset term sum_g m_g * X_g in a lane-per-row layout (acc_m[tok], row = lane).
-// MXFP4 (FMT): the element bytes 2v + 12 take the codes' place, half the power-of-two scale takes d's, and -12 times
-// that takes m's.
-template <int MODE, int FMT = kFmtQ4nx>
-__device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][ModeTraits<MODE>::kAcc],
-                                             float (&acc_m)[ModeTraits<MODE>::kAccM], const LaneConst& lc) {
-    using T = ModeTraits<MODE>;
-    constexpr bool kMx = FmtTraits<FMT>::kMx;
-    if (T::kCols) {
-        const float mw = kMx ? -0.5f * (float)kMxBias * __uint_as_float(t.m_row) : bf16lo_mul_f32hi(t.m_row, 1.0f);
-        if (T::kXRow) {
-#pragma unroll
-            for (int tk = 0; tk < T::kAccM; ++tk) acc_m[tk] = fmaf(mw, t.xrow[tk], acc_m[tk]);
-        } else {
-            acc_m[0] = fmaf(mw, t.sc[0], acc_m[0]);
-        }
-        const float uq = t.sc[1] * lc.w_unit;  // (MXFP4: w_unit carries the 1/2 of the elements' integer form)
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {  // rows (g, g+8) then (g+16, g+24)
-            const uint32_t w0 = t.c[2 * h], w1 = t.c[2 * h + 1];
-            int d[4];
-            if (kMx) {
-                const MxBytes m0 = mx_codes_to_bytes(w0, lc.mx), m1 = mx_codes_to_bytes(w1, lc.mx);  // lo: k 0..3, hi: k 4..7
-                imma<true>(d, m0.pos_lo, m1.pos_lo, m0.pos_hi, m1.pos_hi, t.b[0], t.b[1]);
-                imma_acc<true>(d, m0.neg_lo, m1.neg_lo, m0.neg_hi, m1.neg_hi, t.b[0], t.b[1]);
-            } else {
-                const uint32_t e0 = w0 & 0x0F0F0F0Fu, o0 = (w0 >> 4) & 0x0F0F0F0Fu;  // even-k codes, odd-k codes
-                const uint32_t e1 = w1 & 0x0F0F0F0Fu, o1 = (w1 >> 4) & 0x0F0F0F0Fu;
-                imma<true>(d, e0, e1, o0, o1, t.b[0], t.b[1]);
-            }
-            const float dq[2] = {kMx ? __uint_as_float(t.so[2 * h]) * uq : bf16lo_mul_f32hi(t.so[h], uq),
-                                 kMx ? __uint_as_float(t.so[2 * h + 1]) * uq : bf16hi_mul_f32hi(t.so[h], uq)};
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                // the lane's two columns combined in integers (exact, |.| < 2^24), one conversion
-                const float s = __int2float_rn(d[2 * r] * lc.k_first + d[2 * r + 1]);
-                acc[2 * h + r][0] = fmaf(dq[r], s, acc[2 * h + r][0]);
-            }
-        }
-        return;
-    }
-    constexpr float kMxOff = -0.5f * (float)kMxBias;
-    const float mof[4] = {kMx ? kMxOff * __uint_as_float(t.so[0]) : bf16lo_mul_f32hi(t.so[2], 1.0f),
-                          kMx ? kMxOff * __uint_as_float(t.so[1]) : bf16hi_mul_f32hi(t.so[2], 1.0f),
-                          kMx ? kMxOff * __uint_as_float(t.so[2]) : bf16lo_mul_f32hi(t.so[3], 1.0f),
-                          kMx ? kMxOff * __uint_as_float(t.so[3]) : bf16hi_mul_f32hi(t.so[3], 1.0f)};
-    const float half_unit[2] = {0.5f * t.sc[1], 0.5f * t.sc[3]};  // MXFP4: the 1/2 of the elements' integer form
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {  // rows (g, g+8) then (g+16, g+24)
-        const uint32_t w0 = t.c[2 * h], w1 = t.c[2 * h + 1];
-        int d2[4], d1[4], d0[4];
-        if (kMx) {
-            // three planes share the A operand: merging the two answers (four ORs) is cheaper than six more MMAs
-            const MxBytes m0 = mx_codes_to_bytes(w0, lc.mx), m1 = mx_codes_to_bytes(w1, lc.mx);  // lo: k 0..3, hi: k 4..7
-            const uint32_t e0 = m0.pos_lo | m0.neg_lo, o0 = m0.pos_hi | m0.neg_hi;
-            const uint32_t e1 = m1.pos_lo | m1.neg_lo, o1 = m1.pos_hi | m1.neg_hi;
-            imma<true>(d2, e0, e1, o0, o1, t.b[0], t.b[1]);
-            imma<false>(d1, e0, e1, o0, o1, t.b[2], t.b[3]);
-            imma<false>(d0, e0, e1, o0, o1, t.b[4], t.b[5]);
-        } else {
-            const uint32_t e0 = w0 & 0x0F0F0F0Fu, o0 = (w0 >> 4) & 0x0F0F0F0Fu;  // even-k codes, odd-k codes
-            const uint32_t e1 = w1 & 0x0F0F0F0Fu, o1 = (w1 >> 4) & 0x0F0F0F0Fu;
-            imma<true>(d2, e0, e1, o0, o1, t.b[0], t.b[1]);
-            imma<false>(d1, e0, e1, o0, o1, t.b[2], t.b[3]);
-            imma<false>(d0, e0, e1, o0, o1, t.b[4], t.b[5]);
-        }
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            const int i = 2 * h + r;
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int e = 2 * r + j;
-                // planes recombined in integers (|.| < 2^31), then one conversion (exact below 2^24, else one rounding)
-                const float s = __int2float_rn((d2[e] * 256 + d1[e]) * 256 + d0[e]);
-                const float dq = kMx ? __uint_as_float(t.so[i]) * half_unit[j]
-                                     : (r == 0 ? bf16lo_mul_f32hi(t.so[h], t.sc[2 * j + 1])
-                                               : bf16hi_mul_f32hi(t.so[h], t.sc[2 * j + 1]));
-                acc[i][j] = fmaf(dq, s, acc[i][j]);
-                acc[i][j] = fmaf(mof[i], t.sc[2 * j], acc[i][j]);
-            }
-        }
-    }
 }
 
 // CW consumer warps (8 or 16); MODE as above (1: M = 1, 3: M = 2, 2: M = 3..8); EPI: built with the bf16 epilogues
@@ -572,17 +208,16 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         LaneAddr la;
         LaneConst lc{};
         la.xs = xs;
-        la.x_stride = (uint32_t)M * 128u;
+        la.x_stride = (uint32_t)M * (uint32_t)(MT::kCols ? kColsRecBytes : kPlaneRecBytes);
         {
             const int gtok = g < M ? g : M - 1;
-            la.x_lane = xs + (uint32_t)(gtok * 4 + q) * 32u;
-            la.xsc_lane = xsc + q * 16;
-            lc.k_first = (q & 1) ? 1 : 256;
+            la.x_lane = xs + (uint32_t)(gtok * 4 + q) * 16u;
+            la.xsc_lane = xsc + q * 8;
             const int tok_b = g >> 2, pl = g & 3;
-            la.xb_off = (tok_b < M && pl < 3) ? (uint32_t)(tok_b * 128 + pl * 32 + q * 8) : 104u;
+            la.xb_off = tok_b < M ? (uint32_t)(tok_b * kColsRecBytes + pl * 32 + q * 8) : (uint32_t)kColsZeroOff;
             const int tok_d = q >> 1;
-            la.sc_off = (uint32_t)((tok_d < M ? tok_d : 0) * 128 + 96);
-            lc.w_unit = (tok_d < M ? ((q & 1) ? 1.f : 256.f) : 0.f) * (F::kMx ? 0.5f : 1.f);
+            la.sc_off = (uint32_t)((tok_d < M ? tok_d : 0) * kColsRecBytes + kColsSumOff);
+            lc.w_unit = (tok_d < M ? ((q & 1) ? 1.f : 65536.f) : 0.f) * (F::kMx ? 0.5f : 1.f);
             if (F::kMx) lc.mx = mx_tables();
         }
         float acc_m[MT::kAccM];  // column modes: offset term of row `lane`, per token
@@ -607,10 +242,53 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
 #pragma unroll
             for (int j = 0; j < NT; ++j) acc[i][j] = 0.f;
 
+        // Strip bookkeeping in processing order: position of block 0 of the current strip, position where
+        // the next strip starts, the in-slice index of the first block after the leading tail piece, and the position
+        // where the current piece began.
+        int unit_first = nt > 0 ? -bl_tail : -bl_first;
+        int unit_next = nt > 0 ? nt : unit_first + len;
+        int first_fix = nt > 0 ? bl_first : 0;
+        int piece_lo = 0;
+        auto next_unit = [&]() {
+            piece_lo = unit_next;
+            unit_first = unit_next - first_fix;
+            first_fix = 0;
+            unit_next = unit_first + len;
+        };
+        bool any_flagged = false;  // set once x is prepared: some group of the K slice takes the fp32 path
+
         int piece = 0;
         bool alive = true;
         // hand the warp's partial rows of the current strip piece to the reducer warp
         auto flush = [&]() {
+            if (MT::kCols && any_flagged && alive) {
+                // flagged groups among the tiles this warp processed for the piece: their contribution comes from the
+                // fp32 path (the tensor-core path added exactly zero for them)
+                const int hi = unit_next < nblk ? unit_next : nblk;
+                if (hi > piece_lo) {
+                    const int64_t s_cur = nt > 0 ? (piece == 0 ? s_last : s_first + piece - 1) : s_first + piece;
+                    ExactPiece ep;
+                    ep.blk0 = p.W + s_cur * strip_bytes + (int64_t)b_first * kBB;
+                    ep.groups_total = groups_total;
+                    ep.b_first = b_first;
+                    ep.bl_lo = piece_lo - unit_first;
+                    ep.bl_hi = hi - unit_first;
+                    ep.pos0 = unit_first;
+                    ep.CB = CB;
+                    ep.j0 = j0;
+                    ep.BPW = BPW;
+                    ep.tw = tw;
+                    ep.raw_tile_stride = la.x_stride;
+                    ep.unit_tile_stride = la.x_stride;
+                    ep.piece_stride = 16u;
+#pragma unroll
+                    for (int tk = 0; tk < MT::kAccM; ++tk) {
+                        ep.unit0 = xs + (uint32_t)(tk * kColsRecBytes + kColsUnitOff);
+                        ep.raw0 = xs + (uint32_t)(tk * kColsRecBytes);
+                        acc_m[tk] += piece_exact_token<FMT>(ep, lane);
+                    }
+                }
+            }
             const int par = piece & 1;
             if (piece >= 2 && !mbar_wait(red_empty0 + 8u * par, ((piece >> 1) - 1) & 1, p.status)) alive = false;
             constexpr int PT = MT::kCols ? kColsPartTerms : 1;
@@ -652,19 +330,9 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             ++piece;
         };
 
-        // Strip bookkeeping in processing order: position of block 0 of the current strip, position where
-        // the next strip starts, and the in-slice index of the first block after the leading tail piece.
-        int unit_first = nt > 0 ? -bl_tail : -bl_first;
-        int unit_next = nt > 0 ? nt : unit_first + len;
-        int first_fix = nt > 0 ? bl_first : 0;
-        auto next_unit = [&]() {
-            unit_first = unit_next - first_fix;
-            first_fix = 0;
-            unit_next = unit_first + len;
-        };
-
         // Everything up to here touched only this CTA's shared memory.  x may come from the previous launch.
         asm volatile("griddepcontrol.wait;" ::: "memory");
+        bool saw_flagged = false;
         if (p.prep_inline) {
             // prepare this CTA's K slice of x straight into shared memory (cheap, and the first weights are still
             // on their way from HBM)
@@ -733,14 +401,27 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                     if (base + u * CW * 32 < items) {  // warp-uniform: whole quads run the shuffles together
                         const bool valid = idx < items;
                         const int tm = idx >> 2;
-                        xprep_item<MT::kCols>(v[u], M, valid ? tm / M : 0, valid ? tm % M : 0, idx & 3, valid, xs_g, xsc_g);
+                        if (xprep_item<MT::kCols>(v[u], M, valid ? tm / M : 0, valid ? tm % M : 0, idx & 3, valid, xs_g, xsc_g))
+                            saw_flagged = true;
                     }
                 }
             }
-            asm volatile("bar.sync 1, %0;" ::"n"(CW * 32) : "memory");
-        } else if (!mbar_wait(x_bar, 0, p.status)) {
-            alive = false;
+        } else {
+            if (!mbar_wait(x_bar, 0, p.status)) alive = false;
+            // the preparation kernel's records: does this CTA's K slice hold a flagged group (unit == 0)?
+            if (MT::kCols) {
+                const int kend_full = (b_first + len) * kBlockK;
+                const int nrec = (((kend_full < K ? kend_full : K) - b_first * kBlockK) / kGroup) * M;
+                for (int r = tid; r < nrec && alive; r += CW * 32) {
+                    float unit;
+                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(unit) : "r"(xs + (uint32_t)(r * kColsRecBytes + kColsUnitOff)));
+                    if (unit == 0.f) saw_flagged = true;
+                }
+            }
         }
+        // all of x is in place; one barrier instruction also tells every consumer whether any group of the slice was
+        // flagged for the fp32 path (none in ordinary activations: the tile loop then never looks)
+        any_flagged = named_barrier_or(1, CW * 32, saw_flagged);
         // An "interior" stage -- both of the warp's blocks inside the range and the current strip, every block
         // full -- needs no bookkeeping beyond two tile indices.  `lim` is the first position that is not interior.
         const bool all_full = (groups_total & 7) == 0;
@@ -829,7 +510,7 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             }
             if (++stage == nstage) { stage = 0; phase ^= 1u; }
         }
-        while (piece < npieces && alive) flush();
+        while (piece < npieces && alive) { flush(); next_unit(); }
     } else {
         // =============================== reducer =================================================
         // The prepared activations of this CTA's K slice: one barrier, a few large copies.  They are written by
@@ -840,15 +521,16 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             const int kend_full = (b_first + len) * kBlockK;
             const int kend = kend_full < K ? kend_full : K;
             const uint32_t tile0 = (uint32_t)(kbeg / kGroup), ntiles = (uint32_t)((kend - kbeg) / kGroup);
-            const uint32_t rec_bytes = ntiles * (uint32_t)M * 128u, sc_bytes = MT::kCols ? 0u : ntiles * 64u;
+            constexpr uint32_t kRec = MT::kCols ? kColsRecBytes : kPlaneRecBytes;
+            const uint32_t rec_bytes = ntiles * (uint32_t)M * kRec, sc_bytes = MT::kCols ? 0u : ntiles * (uint32_t)kPlaneSumBytes;
             mbar_arrive_expect_tx(x_bar, rec_bytes + sc_bytes);
-            const uint8_t* src = reinterpret_cast<const uint8_t*>(p.xq) + (size_t)tile0 * M * 128u;
+            const uint8_t* src = reinterpret_cast<const uint8_t*>(p.xq) + (size_t)tile0 * M * kRec;
             for (uint32_t off = 0; off < rec_bytes; off += 32768u) {
                 const uint32_t n = rec_bytes - off < 32768u ? rec_bytes - off : 32768u;
                 bulk_g2s(xs + off, src + off, n, x_bar);
             }
             if constexpr (!MT::kCols) {
-                const uint8_t* s2 = reinterpret_cast<const uint8_t*>(p.xsc) + (size_t)tile0 * 64u;
+                const uint8_t* s2 = reinterpret_cast<const uint8_t*>(p.xsc) + (size_t)tile0 * kPlaneSumBytes;
                 for (uint32_t off = 0; off < sc_bytes; off += 32768u) {
                     const uint32_t n = sc_bytes - off < 32768u ? sc_bytes - off : 32768u;
                     bulk_g2s(xsc + off, s2 + off, n, x_bar);

@@ -19,14 +19,22 @@ constexpr int kEpiGegluBf16 = 2;  // bf16 [M][N/2]: gelu(row r) * (row r + 16) o
 constexpr int kColsMaxTokens = 2;
 // Column modes hand three partial terms per (row, token) to the reducer (two column halves + the offset term).
 constexpr int kColsPartTerms = 3;
+// Prepared activations in shared memory (written by xprep_item, read by the tile loop):
+//   column modes (M <= 2): one 160-byte record per (group-tile, token) -- four signed byte planes of the 31-bit fixed
+//   point (4 x 32 bytes), {sum of x, unit} at 128, eight zero bytes at 136 (the B column of a token that does not
+//   exist), and at 144 of token 0's record the sums of x of tokens 0 and 1;
+//   M >= 3: the bf16 activations themselves in MMA fragment order, 64 bytes per (group-tile, token), and the sums of x
+//   of the (up to eight) tokens, 32 bytes per group-tile.
+constexpr int kColsRecBytes = 160, kColsSumOff = 128, kColsUnitOff = 132, kColsZeroOff = 136, kColsRowSumOff = 144;
+constexpr int kPlaneRecBytes = 64, kPlaneSumBytes = 32;
 constexpr int kMaxSplit = 8;        // K slices
 constexpr int kMaxCtasPerSm = 2;
 
 struct GemvPlan {
     const uint8_t* W;     // device, packed Q4NX
     const uint16_t* x;    // device, [M][K] bf16 bits
-    const uint32_t* xq;   // device, prepared activations: 32-byte records [K/32][M][4] (see fdqp_xprep_kernel)
-    const float* xsc;     // device, per-group {sum x, unit} by token: [K/32][8][2]
+    const uint32_t* xq;   // device, prepared activations of a call whose x is prepared by fdqp_xprep_kernel (layout above)
+    const float* xsc;     // device, M >= 3: per group-tile the sums of x by token, [K/32][8]
     float* y;             // device, fp32 output [M][N] (epilogue kEpiNone)
     uint16_t* y16;        // device, bf16 output (other epilogues)
     int epi;
