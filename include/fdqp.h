@@ -254,6 +254,44 @@ FDQP_API fdqp_status fdqp_flowkv_decode(fdqp_ctx* ctx, const void* q_bf16, const
                                int64_t H, int64_t G, int64_t d, int64_t L, int64_t pitch, int64_t window, float scale,
                                void* cuda_stream);
 
+/* One step of fdqp_run_chain: a projection as fdqp_run_add_rmsnorm_epilogue describes it (x, optional RMS
+ * normalisation with optional residual addition, W, epilogue, out), with M common to the chain. */
+typedef struct {
+    const void* x_bf16;        /* device, [M][K] bf16, 16-byte aligned */
+    const void* W_q4nx;        /* device, q4nx_packed_bytes(K, N) bytes, 16-byte aligned */
+    void* out;                 /* device, 16-byte aligned: fp32 [M][N], bf16 [M][N] or bf16 [M][N/2] as `epilogue` says */
+    int64_t K, N;
+    int epilogue;              /* fdqp_epilogue */
+    int depends_on_previous;   /* 1: x_bf16 (or residual_bf16) is the `out` / h_out of the PREVIOUS step of this chain */
+    const void* gamma_bf16;    /* not null: RMS-normalise x first (scale 1 + gamma), device [K] bf16 */
+    float eps;
+    const void* residual_bf16; /* with gamma: h = bf16(x + residual) is what gets normalised; device [M][K] bf16 or null */
+    void* h_out_bf16;          /* with residual: receives h, device [M][K] bf16, or null */
+} fdqp_chain_step;
+
+/* A chain of projections at M = 1 .. 8 token rows in as few launches as possible: ONE persistent kernel walks up to
+ * 64 steps (longer chains are cut into several launches).  The paper keeps all kernels of a decoder layer resident
+ * and pipelined on its tile array, the vectors between them staying on chip (its section on mapping the decoder;
+ * Sec. "FusedDQP"); here the weight stream of step i + 1 is already filling shared memory while step i finishes, so
+ * launch latency and the first trip to HBM are paid once per chain.  Each step computes exactly what
+ * fdqp_run_add_rmsnorm_epilogue computes for the same arguments (Eq. 14 / 15 with Eq. 3 fused; same acceptance
+ * bound; results reproducible run to run, though the summation order may differ from the single call's).
+ *   depends_on_previous = 1  the step starts its activations only after every output of the previous step is in
+ *                            global memory (a bounded wait on a counter: FDQP_ERR_TIMEOUT in fdqp_last_status if it
+ *                            runs out).  Example: gate|up with FDQP_EPI_GEGLU_BF16 followed by the down projection
+ *                            on its output.  A dependency on any EARLIER step than the previous one is not tracked.
+ *   depends_on_previous = 0  the step's inputs must not be written by any step of the chain.
+ * A step's outputs must not alias the inputs of another step unless that step depends on it.
+ * Limits: 1 <= M <= 8; Q4NX only; a normalised step needs its whole row in one K slice (about M * K <= 16384, e.g.
+ * every K = 2560 projection up to M = 4... see FDQP_ERR_SIZE below); shapes within the context's maxima.
+ * Asynchronous on `cuda_stream`; no allocation; uses the context's chain workspace, so calls that share a context
+ * must be ordered on one stream.
+ * Errors (nothing is launched): FDQP_ERR_ARG (null pointers, n_steps < 1, unknown epilogue, dependency flag on the
+ * first step, residual without gamma), FDQP_ERR_SHAPE, FDQP_ERR_ALIGN, FDQP_ERR_SIZE (beyond the context's maxima,
+ * M > 8, a normalised step whose row does not fit one K slice, workspace exhausted), FDQP_ERR_CUDA. */
+FDQP_API fdqp_status fdqp_run_chain(fdqp_ctx* ctx, const fdqp_chain_step* steps, int64_t n_steps, int64_t M,
+                                    void* cuda_stream);
+
 /* Same projection with HOST activations and result: copies x (host, [M][K] bf16)
  * to the context's device staging buffer, runs fdqp_run, copies y back to `y_host`
  * (host, [M][N] fp32) and synchronises the stream before returning.  W stays a
@@ -369,6 +407,10 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "l2_evict_first" 1 = weight copies carry an evict-first L2 hint
  *   "strip_aligned" 1 = CTA work ranges are cut at strip boundaries, 0 = equal block counts per CTA
  *   "prep_inline"   1 = every GEMV CTA prepares its slice of x itself, 0 = a preparation kernel runs first
+ *   "chain_launch"  fdqp_run_chain: bit 0 = programmatic stream serialisation (default on), bit 1 = cooperative launch
+ *   "chain_steps"   fdqp_run_chain: most steps per launch (1 .. 64, default 64)
+ *   "chain_wide"    fdqp_run_chain: 1 (default) = a launch none of whose steps depends on another is cut into CTA ranges
+ *                   as one sequence of blocks, 0 = every step is cut on its own
  *   "prefill_split_k" 1..8 K slices for the tensor-core kernels (their partial results are added by a second
  *                   kernel); default: as many as fill the SMs when a shape has few output tiles
  *   "prefill_pair"  1 = prefill-sized calls use the two-SM kernel (256 x 512 tile per CTA pair), 0 = the one-SM kernel

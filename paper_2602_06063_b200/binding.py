@@ -27,7 +27,7 @@ EXPORTS = [
     "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
     "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc", "q4nx_packed_bytes_fmt", "q4nx_pack_fmt",
     "q4nx_unpack_fmt", "fdqp_run_fmt", "fdqp_dequant_fmt", "fdqp_run_add_rmsnorm_epilogue",
-    "fdqp_selftest_bounded_wait", "fdqp_noalloc_last_status",
+    "fdqp_selftest_bounded_wait", "fdqp_noalloc_last_status", "fdqp_run_chain",
 ]
 
 
@@ -88,6 +88,8 @@ def load_library():
     lib.fdqp_run_host_async.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_run_noalloc.restype = ci
     lib.fdqp_run_noalloc.argtypes = [vp, vp, vp, i64, i64, i64, vp]
+    lib.fdqp_run_chain.restype = ci
+    lib.fdqp_run_chain.argtypes = [vp, vp, i64, i64, vp]
     lib.fdqp_noalloc_last_status.restype = ci
     lib.fdqp_noalloc_last_status.argtypes = []
     lib.fdqp_dequant.restype = ci
@@ -220,6 +222,35 @@ def fdqp_run_add_rmsnorm_epilogue(ctx: int, x_bf16, residual_bf16, h_out_bf16, g
                                                         _addr(gamma_bf16), float(eps), _addr(W_q4nx), _addr(out),
                                                         int(epilogue), M, K, N, _stream(stream)),
            "fdqp_run_add_rmsnorm_epilogue", ctx)
+
+
+class ChainStepC(ctypes.Structure):
+    """fdqp_chain_step of include/fdqp.h."""
+    _fields_ = [("x_bf16", ctypes.c_void_p), ("W_q4nx", ctypes.c_void_p), ("out", ctypes.c_void_p),
+                ("K", ctypes.c_int64), ("N", ctypes.c_int64), ("epilogue", ctypes.c_int),
+                ("depends_on_previous", ctypes.c_int), ("gamma_bf16", ctypes.c_void_p), ("eps", ctypes.c_float),
+                ("residual_bf16", ctypes.c_void_p), ("h_out_bf16", ctypes.c_void_p)]
+
+
+def chain_step(x_bf16, W_q4nx, out, K: int, N: int, epilogue: int = 0, depends_on_previous: bool = False,
+               gamma_bf16=None, eps: float = 0.0, residual_bf16=None, h_out_bf16=None) -> ChainStepC:
+    """One step of fdqp_run_chain (device tensors or addresses; see fdqp_chain_step in fdqp.h)."""
+    return ChainStepC(_addr(x_bf16) or None, _addr(W_q4nx) or None, _addr(out) or None, K, N, int(epilogue),
+                      int(bool(depends_on_previous)), _addr(gamma_bf16) or None, float(eps),
+                      _addr(residual_bf16) or None, _addr(h_out_bf16) or None)
+
+
+def make_chain(steps):
+    """A C array of fdqp_chain_step from a list of chain_step(...) values (keep it alive for the call)."""
+    return (ChainStepC * len(steps))(*steps)
+
+
+def fdqp_run_chain(ctx: int, steps, M: int, stream=None) -> None:
+    """Run a chain of projections (a list of chain_step(...) or an array from make_chain) at M token rows in as few
+    persistent launches as possible.  Asynchronous on `stream`."""
+    arr = steps if isinstance(steps, ctypes.Array) else make_chain(steps)
+    _check(load_library().fdqp_run_chain(ctx, ctypes.cast(arr, ctypes.c_void_p), len(arr), M, _stream(stream)),
+           "fdqp_run_chain", ctx)
 
 
 def fdqp_flowkv_decode(ctx: int, q_bf16, K_bf16, V_bf16, out, H: int, G: int, d: int, L: int, pitch: int, window: int,

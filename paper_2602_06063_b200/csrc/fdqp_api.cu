@@ -8,6 +8,7 @@
 #include <mutex>
 #include <new>
 #include <string>
+#include <vector>
 
 #include "fdqp.h"
 #include "fdqp_format.h"
@@ -31,6 +32,8 @@ cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* 
                           int G, int d, int L, int pitch, int window, float scale, int sm_count, cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
 cudaError_t wait_selftest_launch(int* status, unsigned long long limit_ns, cudaStream_t stream);
+cudaError_t chain_set_smem_limit(int bytes);
+cudaError_t chain_launch(const ChainPlan& cp, int grid, bool epi, int launch_mode, cudaStream_t stream);
 }  // namespace fdqp
 
 using namespace fdqp;
@@ -58,6 +61,14 @@ struct fdqp_ctx {
     std::string last_err;
     // overrides (-1 = automatic)
     int64_t p_path = -1, p_ctas_per_sm = -1, p_cw = -1, p_stages = -1, p_split_k = -1, p_evict = -1, p_prep = -1, p_aligned = -1, p_bpw = -1, p_pair = -1, p_pf_split = -1;
+    // fdqp_run_chain: partial rows of shared strips (2 per CTA and step), of whole strip-slices, arrival counters per
+    // (step, strip), and the per-step completion counters followed by the exit counter
+    float* chain_edge = nullptr;
+    float* chain_full = nullptr;
+    int* chain_tickets = nullptr;
+    int* chain_done = nullptr;
+    size_t chain_ticket_cap = 0;
+    int64_t p_chain_launch = 1, p_chain_steps = kMaxChainSteps, p_chain_wide = 1;
     int64_t p_direct_y = 1;  // fdqp_run_host*: small results are stored straight into device-addressable host memory
     int64_t p_atmem = 1;  // tensor-core kernel up to 128 tokens: keep the converted weights in tensor memory
 };
@@ -76,6 +87,11 @@ constexpr size_t kDirectHostBytes = 1u << 20;  // results up to this size go str
 constexpr int kKvMaxHeads = 64, kKvMaxSplits = 148, kKvMaxDim = 256;  // decode attention workspace
 constexpr size_t kPrefillWsCap = 128u << 20;  // bytes of partial results a context keeps for K-split tensor-core calls
 constexpr int kMinStages = 3;  // ring depth below which another K slice is preferred
+// fdqp_run_chain: shared memory a step's prepared activations may take (K is cut into slices beyond it), activation
+// items (8 values) one CTA prepares per step at most, and the partial-row slots for steps with K slices
+constexpr uint32_t kChainXsCap = 64u << 10;
+constexpr int kChainPrepItems = 8 * 16 * 32;
+constexpr size_t kChainFullSlots = 16384;
 
 struct DeviceGuard {
     int prev = -1;
@@ -360,6 +376,17 @@ extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, in
         if ((e = cudaHostAlloc(&ctx->status_host, sizeof(int), cudaHostAllocMapped))) { st = cuda_fail(nullptr, e, ""); break; }
         *ctx->status_host = 0;
         if ((e = cudaHostGetDevicePointer(&ctx->status_dev, ctx->status_host, 0))) { st = cuda_fail(nullptr, e, ""); break; }
+        {
+            const size_t slot_b = sizeof(float) * kStripRows * kMaxTokens;
+            ctx->chain_ticket_cap = (size_t)16 * (size_t)S < 65536 ? 65536 : (size_t)16 * (size_t)S;
+            if ((e = cudaMalloc(&ctx->chain_edge, slot_b * 2 * (size_t)ctx->sm_count * kMaxChainSteps))) { st = cuda_fail(nullptr, e, ""); break; }
+            if ((e = cudaMalloc(&ctx->chain_full, slot_b * kChainFullSlots))) { st = cuda_fail(nullptr, e, ""); break; }
+            if ((e = cudaMalloc(&ctx->chain_tickets, sizeof(int) * ctx->chain_ticket_cap))) { st = cuda_fail(nullptr, e, ""); break; }
+            if ((e = cudaMalloc(&ctx->chain_done, sizeof(int) * (kMaxChainSteps + 1)))) { st = cuda_fail(nullptr, e, ""); break; }
+            if ((e = cudaMemset(ctx->chain_tickets, 0, sizeof(int) * ctx->chain_ticket_cap))) { st = cuda_fail(nullptr, e, ""); break; }
+            if ((e = cudaMemset(ctx->chain_done, 0, sizeof(int) * (kMaxChainSteps + 1)))) { st = cuda_fail(nullptr, e, ""); break; }
+        }
+        if ((e = chain_set_smem_limit(ctx->smem_optin))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = gemv_set_smem_limit(ctx->smem_optin))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = prefill_set_smem_limit())) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaDeviceSynchronize())) { st = cuda_fail(nullptr, e, ""); break; }
@@ -382,6 +409,10 @@ extern "C" fdqp_status fdqp_destroy(fdqp_ctx* ctx) {
     if (ctx->x_norm) cudaFree(ctx->x_norm);
     if (ctx->kv_ws) cudaFree(ctx->kv_ws);
     if (ctx->tickets) cudaFree(ctx->tickets);
+    if (ctx->chain_edge) cudaFree(ctx->chain_edge);
+    if (ctx->chain_full) cudaFree(ctx->chain_full);
+    if (ctx->chain_tickets) cudaFree(ctx->chain_tickets);
+    if (ctx->chain_done) cudaFree(ctx->chain_done);
     if (ctx->xq) cudaFree(ctx->xq);
     if (ctx->xsc) cudaFree(ctx->xsc);
     if (ctx->x_stage) cudaFree(ctx->x_stage);
@@ -702,6 +733,15 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
     } else if (!std::strcmp(key, "strip_aligned")) {
         if (v > 1) return FDQP_ERR_ARG;
         ctx->p_aligned = v;
+    } else if (!std::strcmp(key, "chain_launch")) {
+        if (v > 3) return FDQP_ERR_ARG;
+        ctx->p_chain_launch = v < 0 ? 1 : v;
+    } else if (!std::strcmp(key, "chain_wide")) {
+        if (v > 1) return FDQP_ERR_ARG;
+        ctx->p_chain_wide = v < 0 ? 1 : v;
+    } else if (!std::strcmp(key, "chain_steps")) {
+        if (v == 0 || v > kMaxChainSteps) return FDQP_ERR_ARG;
+        ctx->p_chain_steps = v < 0 ? kMaxChainSteps : v;
     } else if (!std::strcmp(key, "prep_inline")) {
         if (v > 1) return FDQP_ERR_ARG;
         ctx->p_prep = v;
@@ -754,6 +794,156 @@ extern "C" fdqp_status fdqp_describe(fdqp_ctx* ctx, int64_t M, int64_t K, int64_
                   "evict_first=%d strip_aligned=%d blocks_per_warp=%d",
                   plan.prep_inline ? "" : "fdqp_xprep_kernel + ", cw, mc == 1 ? 1 : (mc > kColsMaxTokens ? 2 : (mc == 2 ? 3 : 1)), (long long)((M + kMaxTokens - 1) / kMaxTokens), plan.Z * plan.Gz, (cw + 1 + cw / 8) * 32,
                   plan.smem_bytes, plan.nstage, plan.Z, plan.Gz, plan.evict_first, plan.strip_aligned, plan.bpw);
+    return FDQP_OK;
+}
+
+// ---- a chain of projections in one persistent launch -----------------------------------------------------------------
+
+extern "C" fdqp_status fdqp_run_chain(fdqp_ctx* ctx, const fdqp_chain_step* steps, int64_t n_steps, int64_t M,
+                                      void* cuda_stream) {
+    if (!ctx || !steps || n_steps < 1) return FDQP_ERR_ARG;
+    if (M < 1) return FDQP_ERR_SHAPE;
+    if (M > kMaxTokens) return FDQP_ERR_SIZE;
+    for (int64_t i = 0; i < n_steps; ++i) {
+        const fdqp_chain_step& u = steps[i];
+        if (!u.x_bf16 || !u.W_q4nx || !u.out) return FDQP_ERR_ARG;
+        if (u.epilogue != kEpiNone && u.epilogue != kEpiBf16 && u.epilogue != kEpiGegluBf16) return FDQP_ERR_ARG;
+        if ((u.residual_bf16 || u.h_out_bf16) && !u.gamma_bf16) return FDQP_ERR_ARG;
+        if (u.h_out_bf16 && !u.residual_bf16) return FDQP_ERR_ARG;
+        if (u.h_out_bf16 && (u.h_out_bf16 == u.x_bf16 || u.h_out_bf16 == u.residual_bf16)) return FDQP_ERR_ARG;
+        if (u.gamma_bf16 && !(u.eps >= 0.f)) return FDQP_ERR_ARG;
+        if (u.depends_on_previous != 0 && (u.depends_on_previous != 1 || i == 0)) return FDQP_ERR_ARG;
+        const fdqp_status st = check_shape(ctx, M, u.K, u.N);
+        if (st != FDQP_OK) return st;
+        if (!aligned16(u.x_bf16) || !aligned16(u.W_q4nx) || !aligned16(u.out) || (u.gamma_bf16 && !aligned16(u.gamma_bf16)) ||
+            (u.residual_bf16 && !aligned16(u.residual_bf16)) || (u.h_out_bf16 && !aligned16(u.h_out_bf16)))
+            return FDQP_ERR_ALIGN;
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FDQP_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int grid = ctx->sm_count;
+    const int m = (int)M;
+    const bool cols = m <= kColsMaxTokens;
+    const uint32_t rec = (uint32_t)(cols ? kColsRecBytes : kPlaneRecBytes);
+    // blocks of a K slice whose prepared activations fit the shared-memory budget and one preparation pass
+    int cap_blocks = (int)(kChainXsCap / (8u * rec * (uint32_t)m));
+    if (cap_blocks > kChainPrepItems / (8 * m * 4)) cap_blocks = kChainPrepItems / (8 * m * 4);
+    if (cap_blocks < 1) return FDQP_ERR_SIZE;
+    const int per_launch = (int)ctx->p_chain_steps;
+    // plan every launch before the first one goes out, so that an error launches nothing
+    std::vector<ChainPlan> plans;
+    std::vector<char> plan_epi;
+    for (int64_t first = 0; first < n_steps; first += per_launch) {
+        const int n = (int)((n_steps - first) < per_launch ? (n_steps - first) : per_launch);
+        ChainPlan cp;
+        std::memset(&cp, 0, sizeof(cp));
+        cp.nsteps = n;
+        cp.M = m;
+        cp.ws_edge = ctx->chain_edge;
+        cp.ws_full = ctx->chain_full;
+        cp.tickets = ctx->chain_tickets;
+        cp.done = ctx->chain_done;
+        cp.exit_count = ctx->chain_done + kMaxChainSteps;
+        cp.status = ctx->status_dev;
+        cp.evict_first = ctx->p_evict >= 0 ? (ctx->p_evict != 0) : 1;
+        uint32_t xs_bytes = 0, xsum_bytes = 0;
+        size_t ticket_off = 0, edge_off = 0, full_off = 0, blocks = 0;
+        bool epi = false, dependent = false;
+        for (int i = 0; i < n; ++i) {
+            const fdqp_chain_step& u = steps[first + i];
+            ChainStep& c = cp.step[i];
+            c.W = static_cast<const uint8_t*>(u.W_q4nx);
+            c.x = static_cast<const uint16_t*>(u.x_bf16);
+            c.y = u.epilogue == kEpiNone ? static_cast<float*>(u.out) : nullptr;
+            c.y16 = u.epilogue == kEpiNone ? nullptr : static_cast<uint16_t*>(u.out);
+            c.gamma = static_cast<const uint16_t*>(u.gamma_bf16);
+            c.residual = static_cast<const uint16_t*>(u.residual_bf16);
+            c.h_out = static_cast<uint16_t*>(u.h_out_bf16);
+            c.eps = u.eps;
+            c.epi = u.epilogue;
+            c.norm = u.gamma_bf16 ? 1 : 0;
+            if (c.epi != kEpiNone || c.norm) epi = true;
+            c.K = (int)u.K;
+            c.N = (int)u.N;
+            c.S = c.N / kStripRows;
+            c.nb = (c.K + kBlockK - 1) / kBlockK;
+            int Z = (c.nb + cap_blocks - 1) / cap_blocks;
+            c.nbz = (c.nb + Z - 1) / Z;
+            Z = (c.nb + c.nbz - 1) / c.nbz;
+            c.Z = Z;
+            if (c.norm && Z > 1) return FDQP_ERR_SIZE;  // the normalisation needs the whole row in every CTA
+            if (Z > grid) return FDQP_ERR_SIZE;
+            const int len_last = c.nb - (Z - 1) * c.nbz;
+            int64_t Gz = grid / Z;
+            if (Gz > (int64_t)c.S * len_last) Gz = (int64_t)c.S * len_last;
+            if (Gz < 1) Gz = 1;
+            // whole strips per CTA when that costs at most 3 % of imbalance (nothing is exchanged between CTAs then)
+            c.strip_aligned = 0;
+            if (c.S >= Gz && (double)((c.S + Gz - 1) / Gz) * (double)Gz <= 1.03 * (double)c.S) c.strip_aligned = 1;
+            if (ctx->p_aligned >= 0 && (ctx->p_aligned == 0 || c.S >= Gz)) c.strip_aligned = ctx->p_aligned != 0;
+            c.Gz = (int)Gz;
+            c.wait_prev = (u.depends_on_previous && i > 0) ? 1 : 0;  // across launches the stream order is the dependency
+            if (c.wait_prev) {
+                cp.step[i - 1].signal = 1;
+                dependent = true;
+            }
+            c.B = (uint32_t)blocks;
+            blocks += (size_t)c.S * c.nb;
+            for (int z = 0; z < Z; ++z) {
+                if (cp.nunits >= kMaxChainUnits) return FDQP_ERR_SIZE;
+                cp.unit_step[cp.nunits] = (uint8_t)i;
+                cp.unit_slice[cp.nunits] = (uint8_t)z;
+                ++cp.nunits;
+            }
+            c.ticket_off = (uint32_t)ticket_off;
+            c.edge_off = (uint32_t)edge_off;
+            c.full_off = (uint32_t)full_off;
+            ticket_off += (size_t)c.S;
+            edge_off += (size_t)2 * Z * c.Gz;
+            if (Z > 1) full_off += (size_t)Z * c.S;
+            const uint32_t xb = (uint32_t)c.nbz * 8u * rec * (uint32_t)m;
+            if (xb > xs_bytes) xs_bytes = xb;
+            if (!cols && (uint32_t)c.nbz * 8u * (uint32_t)kPlaneSumBytes > xsum_bytes) xsum_bytes = (uint32_t)c.nbz * 8u * (uint32_t)kPlaneSumBytes;
+        }
+        // No step of this launch waits for another one: cut the whole chain, not every step, into equal CTA ranges.
+        cp.Wtot = (uint32_t)blocks;
+        cp.wide = (!dependent && blocks >= (size_t)grid && blocks < (1u << 31) && ctx->p_chain_wide != 0) ? 1 : 0;
+        if (ticket_off > ctx->chain_ticket_cap || full_off > kChainFullSlots ||
+            edge_off > (size_t)2 * ctx->sm_count * kMaxChainSteps)
+            return FDQP_ERR_SIZE;
+        const uint32_t part_bytes = 2u * 16u * kStripRows * (uint32_t)m * 4u * (cols ? (uint32_t)kColsPartTerms : 1u);
+        const uint32_t norm_bytes = (uint32_t)(kChainPrepItems / 4) * 4u + 64u;
+        const uint32_t fixed = round_up(xs_bytes, 128) + round_up(xsum_bytes, 128) + round_up(part_bytes, 128) +
+                               round_up(norm_bytes, 128) + (2u * kMaxStages + 4u) * 8u + 128u;
+        // four blocks per warp and stage (half the barrier round trips per tile) while the ring keeps three stages
+        int bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (m <= 4 ? 4 : 2);
+        uint32_t stage_bytes = 2u * (uint32_t)bpw * kBlockBytes;
+        int nstage = (uint32_t)ctx->smem_optin > fixed ? (int)(((uint32_t)ctx->smem_optin - fixed) / stage_bytes) : 0;
+        if (bpw == 4 && ctx->p_bpw != 4 && nstage < kMinStages) {
+            bpw = 2;
+            stage_bytes = 2u * (uint32_t)bpw * kBlockBytes;
+            nstage = (uint32_t)ctx->smem_optin > fixed ? (int)(((uint32_t)ctx->smem_optin - fixed) / stage_bytes) : 0;
+        }
+        cp.bpw = bpw;
+        if (nstage > kMaxStages) nstage = kMaxStages;
+        if (ctx->p_stages > 0 && ctx->p_stages < nstage) nstage = (int)ctx->p_stages;
+        if (nstage < 2) return FDQP_ERR_SIZE;
+        cp.nstage = nstage;
+        cp.off_xs = (uint32_t)nstage * stage_bytes;
+        cp.off_xsum = cp.off_xs + round_up(xs_bytes, 128);
+        cp.off_part = cp.off_xsum + round_up(xsum_bytes, 128);
+        cp.off_norm = cp.off_part + round_up(part_bytes, 128);
+        cp.off_bar = cp.off_norm + round_up(norm_bytes, 128);
+        cp.smem_bytes = cp.off_bar + (2u * (uint32_t)nstage + 4u) * 8u;
+        plans.push_back(cp);
+        plan_epi.push_back(epi ? 1 : 0);
+    }
+    for (size_t i = 0; i < plans.size(); ++i) {
+        const cudaError_t e = chain_launch(plans[i], grid, plan_epi[i] != 0, (int)ctx->p_chain_launch, stream);
+        if (e) return cuda_fail(ctx, e, "chain kernel launch");
+        ctx->launches += 1;
+    }
     return FDQP_OK;
 }
 

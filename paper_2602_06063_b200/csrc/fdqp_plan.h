@@ -66,4 +66,50 @@ struct GemvPlan {
     uint32_t smem_bytes;
 };
 
+// ---- a chain of projections in one persistent launch (fdqp_chain.cu) ---------------------------------------------
+constexpr int kMaxChainSteps = 64;   // projections one launch walks (a longer chain is cut into several launches)
+constexpr int kMaxChainUnits = 160;  // (step, K slice) pairs of one launch
+
+struct ChainStep {
+    const uint8_t* W;          // device, packed Q4NX
+    const uint16_t* x;         // device, [M][K] bf16 bits (may be written by the previous step: wait_prev)
+    float* y;                  // device, fp32 output [M][N] (epilogue kEpiNone)
+    uint16_t* y16;             // device, bf16 output (other epilogues)
+    const uint16_t* gamma;     // RMS normalisation of x in the activation preparation (norm != 0)
+    const uint16_t* residual;  // with norm: x + residual is what gets normalised ...
+    uint16_t* h_out;           // ... and, when not null, is also written here by the grid's first CTA
+    float eps;
+    int epi, norm;
+    int K, N;
+    int S;                     // strips = N / 32
+    int nb;                    // blocks per strip = ceil(K / 256)
+    int Z, nbz;                // K slices and blocks per slice (the prepared x of a slice must fit shared memory)
+    int Gz;                    // CTAs per slice (Z * Gz <= grid; the rest of the grid idles during this step)
+    int strip_aligned;         // 1: CTA ranges are cut at strip boundaries
+    uint32_t B;                // chain-wide cut: position of this step's first block in the chain's block sequence
+    int wait_prev;             // 1: the step's input is the previous step's output: wait for all of its strips
+    int signal;                // 1: the next step waits on this one: count the stored strips in done[step]
+    uint32_t ticket_off;       // this step's arrival counters inside ChainPlan::tickets
+    uint32_t edge_off;         // this step's slots inside ChainPlan::ws_edge (2 per CTA) ...
+    uint32_t full_off;         // ... and inside ChainPlan::ws_full (Z * S, used when Z > 1)
+};
+
+struct ChainPlan {
+    int nsteps, M;
+    float* ws_edge;            // device, partial rows of strips shared between CTAs
+    float* ws_full;            // device, partial rows of whole strip-slices (steps with K slices)
+    int* tickets;              // device, arrival counters per (step, strip), zero between launches
+    int* done;                 // device, [kMaxChainSteps] strips stored per step, zero between launches
+    int* exit_count;           // device, CTAs that have finished (the last one resets `done`)
+    int* status;               // host-mapped sticky status word
+    int nstage, evict_first;
+    int bpw;                   // blocks per consumer warp and ring stage (2 or 4; a stage holds twice as many blocks)
+    int wide;                  // 1: chain-wide cut into CTA ranges (no step waits for another), 0: every step cut on its own
+    uint32_t Wtot;             // chain-wide cut: blocks of all steps together
+    int nunits;                // (step, K slice) pairs in processing order
+    uint8_t unit_step[kMaxChainUnits], unit_slice[kMaxChainUnits];
+    uint32_t off_xs, off_xsum, off_part, off_norm, off_bar, smem_bytes;  // shared-memory carve-up (bytes)
+    ChainStep step[kMaxChainSteps];
+};
+
 }  // namespace fdqp
