@@ -1,14 +1,14 @@
 #!/usr/bin/env python
 """Benchmark of the FusedDQP hot path on B200.
 
-A step is one Gemma3-4B decoder layer at M = 1: the seven Q4NX projections q, k, v, o, gate, up, down
-(59.1 MB of packed weights) on seeded synthetic inputs.  Projections that share their input are launched
-together -- q|k|v and gate|up are concatenated along N, which in the strip-major Q4NX container is plain
-concatenation of the packed bytes -- so a step is four fdqp_run calls (--fuse 0 runs the seven one by one).
-Several distinct copies of the layer's weights are resident in HBM and the steps rotate through them, so every
-timed step streams its weights from HBM and not from L2.  The metric is the achieved bandwidth over the algorithmic bytes of the step
-(0.625*K*N + 2*M*K + 4*M*N per projection); decode tokens/s (projections only: 34 layers + LM head) is
-reported beside it.
+A step is one pass of the hot path over the largest single-GPU configuration: the Gemma3-4B tied LM head (K = 2560,
+N = 262144, 419 MB of packed Q4NX weights, seed 17) at decode M = 1 -- one fdqp_run call, one kernel launch.  The
+metric is the achieved bandwidth over the algorithmic bytes of the step (0.625*K*N + 2*M*K + 4*M*N).  Beside the
+headline the line carries one sub-object per BASELINE configuration and M (per-call median / min / p90 from CUDA-event
+pairs, back-to-back mean from a graph replay of at least 60 ms, GB/s, fractions of the measured and the nominal peak,
+the launch plan and the clock samples of its own region), the Gemma3-4B layer as single calls and as chained launches,
+decode tokens/s (projections only: 34 layers + LM head), batched decode, the prefill tensor-core path, decode attention,
+the format variants and the dequantisation engine.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
@@ -34,10 +34,12 @@ import numpy as np  # noqa: E402
 import synthgen  # noqa: E402
 
 METRIC = "fused Q4NX dequant-GEMV achieved HBM GB/s & % of peak; decode tokens/s (1 GPU)"
-WORKLOAD = "Gemma3-4B decoder layer at M=1: q,k,v,o,gate,up,down Q4NX group-32 projections (seeds 1-7)"
+WORKLOAD = "Gemma3-4B tied LM head K=2560 N=262144, Q4NX group 32, decode M=1 (seed 17): the largest single-GPU configuration"
 L2_BYTES = 126e6
 LAYER_COPIES = 8            # distinct weight sets resident in HBM (8 x 59 MB = 472 MB >> L2)
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one LM-head launch (K=2560, N=262144, M=1) from an ncu capture
+NCU_LM_HEAD_DRAM_BYTES = 419511296 + 3408128
 
 
 def alg_bytes(M, K, N):
@@ -84,19 +86,13 @@ class ClockSampler:
         for line in self.proc.stdout:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) >= 7:
-                self.rows.append(parts)
+                self.rows.append((time.time(), parts))      # host time at which the sample arrived
 
-    def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
+    @staticmethod
+    def _summary(rows):
         sm, smax, reasons, power = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for _, r in rows:
             try:
                 sm.append(float(r[0]))
                 smax.append(float(r[1]))
@@ -108,6 +104,23 @@ class ClockSampler:
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+    def window(self, t0, t1):
+        """Samples that arrived during [t0, t1 + one period]: the clocks of one timed region."""
+        if self.proc is None:
+            return None
+        time.sleep(0.03)                                    # let the sample that covers the end of the region arrive
+        return self._summary([r for r in list(self.rows) if t0 <= r[0] <= t1 + 0.025])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        return self._summary(self.rows)
 
 
 # ----------------------------------------------------------------------------------------------- rank plumbing
@@ -130,18 +143,20 @@ def whole_job_gbs(bytes_per_step, steps, world, ms):
 # ----------------------------------------------------------------------------------------------- reference arm
 
 def run_reference(args, rank, world):
-    """Times the CPU oracle (as it stands) on the host cores: each step is one pass of the decoder layer's
-    seven projections at M = 1 over the same seeded inputs, all output columns, OpenMP over columns."""
+    """Times the CPU oracle (as it stands) on the host cores on the headline workload: each step is one pass over a
+    bounded sample of the LM head's outputs at M = 1 (the first 65536 of the 262144 columns of the seeded matrix, all of
+    K), OpenMP over columns; the GB/s counts the sample's own algorithmic bytes."""
     if rank != 0:
         return
     import oracle
     cores = min(oracle.max_threads(), os.cpu_count() or 1)
-    layer = [(name, K, N, synthgen.weights(seed, K, N), synthgen.activations(seed, 1, K))
-             for name, K, N, seed in synthgen.GEMMA3_4B_LAYER]
+    _, K, N, seed = synthgen.GEMMA3_4B_LM_HEAD
+    n1 = N // 4
+    w = synthgen.weights(seed, K, n1)                      # the generator is column-wise: the first n1 columns of the head
+    x = synthgen.activations(seed, 1, K)
 
     def one_pass():
-        for _, K, N, w, x in layer:
-            oracle.project(x, w.codes, w.scales, w.offsets, nthreads=cores)
+        oracle.project(x, w.codes, w.scales, w.offsets, nthreads=cores)
 
     for _ in range(args.warmup):
         one_pass()
@@ -149,14 +164,15 @@ def run_reference(args, rank, world):
     for _ in range(args.steps):
         one_pass()
     dt = time.perf_counter() - t0
-    gbs = layer_bytes() * args.steps / dt / 1e9
+    gbs = alg_bytes(1, K, n1) * args.steps / dt / 1e9
+    sample = f"outputs 0..{n1 - 1} of the {N} of the LM head per step (a quarter of the matrix)"
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "note": "CPU oracle (fp64, plain C, OpenMP over output columns)"},
-        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
-                         "sample": "whole layer, all 7 projections, all outputs, per step"},
+        "config": {"workload": WORKLOAD, "M": 1, "K": K, "N": N, "sample": sample,
+                   "note": "CPU oracle (fp64, plain C, OpenMP over output columns)"},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -246,6 +262,49 @@ def run_shape(args):
                       "peak_kind": peak_kind, "weight_copies": ncopies, "steps": args.steps,
                       "graph": bool(args.graph and not args.same_weights), "epilogue": args.epilogue, "rmsnorm": bool(args.rmsnorm),
                       "launch": fd.fdqp_describe(ctx, M, K, N)}), flush=True)
+    fd.fdqp_destroy(ctx)
+
+
+# ----------------------------------------------------------------------------------------------- a chained layer
+
+def run_layer_chain(args):
+    """Times the Gemma3-4B decoder layer at M = --tokens (q|k|v, o, gate|up, down on independent seeded inputs) as chained
+    launches of --layer-chain layers each (fdqp_run_chain), rotating over 8 distinct weight sets."""
+    import torch
+
+    import paper_2602_06063_b200 as fd
+
+    L, M = args.layer_chain, args.tokens
+    torch.cuda.set_device(0)
+    peaks, peak_kind = measured_peaks()
+    by_name = {n: (K, N, seed) for n, K, N, seed in synthgen.GEMMA3_4B_LAYER}
+    groups = [["q", "k", "v"], ["o"], ["gate", "up"], ["down"]]
+    shapes = [("|".join(g), by_name[g[0]][0], sum(by_name[n][1] for n in g), by_name[g[0]][2]) for g in groups]
+    ctx = fd.fdqp_create(0, 8, 10240, 20480)
+    for kv in args.param or []:
+        key, val = kv.split("=")
+        fd.fdqp_set_param(ctx, key, int(val))
+    copies = [[tiled_weights(fd, torch, K, N, seed + 1000 * c) for _, K, N, seed in shapes] for c in range(LAYER_COPIES)]
+    xs = [torch.from_numpy(synthgen.activations(seed, M, K).view(np.int16)).cuda() for _, K, _, seed in shapes]
+    ys = [torch.empty((M, N), dtype=torch.float32, device="cuda") for _, _, N, _ in shapes]
+    stream = torch.cuda.Stream()
+    sraw = stream.cuda_stream
+    chains = [fd.make_chain([fd.chain_step(xs[j], copies[(first + l) % LAYER_COPIES][j], ys[j], K, N)
+                             for l in range(L) for j, (_, K, N, _) in enumerate(shapes)]) for first in range(0, LAYER_COPIES, max(1, min(L, LAYER_COPIES)))]
+    for i in range(max(3, args.warmup)):
+        fd.fdqp_run_chain(ctx, chains[i % len(chains)], M, sraw)
+    stream.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        fd.fdqp_run_chain(ctx, chains[i % len(chains)], M, sraw)
+    e1.record(stream)
+    stream.synchronize()
+    assert fd.fdqp_last_status(ctx) == 0
+    us = e0.elapsed_time(e1) * 1e3 / (args.steps * L)
+    gbs = layer_bytes(M) / us / 1e3
+    print(json.dumps({"layer_chain": {"layers_per_launch": L, "M": M}, "us_per_layer": us, "GBps": gbs,
+                      "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "peak_kind": peak_kind, "launches": args.steps}), flush=True)
     fd.fdqp_destroy(ctx)
 
 
@@ -343,6 +402,100 @@ def run_flowkv(args):
 
 # ----------------------------------------------------------------------------------------------- our arm
 
+MIN_REGION_MS = 60.0        # every timed region lasts at least this long, whatever --steps is (several clock samples)
+PAIR_CALLS = 160            # per-call event pairs behind each median / min / p90
+
+
+class Regions:
+    """Host-time windows of the timed regions, so that each gets the clock samples that fall inside it."""
+
+    def __init__(self, sampler):
+        self.sampler = sampler
+
+    def clocks(self, t0, t1):
+        return self.sampler.window(t0, t1) if self.sampler is not None else None
+
+
+def tiled_weights(fd, torch, K, N, seed, fmt=None):
+    """Packed weights of a K x N matrix on the device: a seeded matrix of up to 4096 output columns tiled along N (the
+    strip-major container makes that byte concatenation) -- the full recipe costs minutes of host time for the largest
+    shapes and the kernels' timing does not depend on the values."""
+    nb = min(N, 4096)
+    if fmt is None or fmt == fd.FMT_Q4NX:
+        w = synthgen.weights(seed, K, nb)
+        tile = fd.q4nx_pack(w.codes, w.scales, w.offsets)
+        nbytes = fd.q4nx_packed_bytes(K, N)
+    else:
+        w = synthgen.weights_fmt(seed, K, nb, fmt)
+        tile = fd.q4nx_pack_fmt(fmt, w.codes, w.scales, w.offsets)
+        nbytes = fd.q4nx_packed_bytes_fmt(fmt, K, N)
+    return torch.from_numpy(np.tile(tile, -(-N // nb))[:nbytes].copy()).cuda()
+
+
+def weight_copies(torch, base):
+    """Enough distinct copies of a weight buffer that consecutive launches never find theirs in L2 (>= 4 x L2 in all)."""
+    n = max(1, int(np.ceil(4 * L2_BYTES / base.numel())))
+    return [base] + [base.clone() for _ in range(n - 1)]
+
+
+def time_region(torch, stream, enqueue, ncalls_cycle, regions, min_ms=MIN_REGION_MS, pairs=PAIR_CALLS):
+    """enqueue(i) puts call i (rotating inputs itself) on `stream`.  Returns per-call statistics:
+    median / min / p90 of single calls bracketed by CUDA events on the launching stream (direct launches), and the mean
+    of back-to-back calls replayed from a CUDA graph for at least min_ms (what a decode loop sees), with the clock
+    samples taken during that region."""
+    for i in range(max(3, ncalls_cycle)):
+        enqueue(i)
+    stream.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(pairs)]
+    for i, (a, b) in enumerate(evs):
+        a.record(stream)
+        enqueue(i)
+        b.record(stream)
+    stream.synchronize()
+    us = sorted(a.elapsed_time(b) * 1e3 for a, b in evs)
+    per_graph = max(ncalls_cycle, 8)
+    per_graph = -(-per_graph // ncalls_cycle) * ncalls_cycle
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        for i in range(per_graph):
+            enqueue(i)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        for _ in range(2):
+            g.replay()
+        e0.record(stream)
+        g.replay()
+        e1.record(stream)
+    stream.synchronize()
+    one = max(e0.elapsed_time(e1), 1e-3)
+    reps = max(1, int(np.ceil(min_ms / one)))
+    t0 = time.time()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+    stream.synchronize()
+    t1 = time.time()
+    ms = e0.elapsed_time(e1)
+    return {"us_median": us[len(us) // 2], "us_min": us[0], "us_p90": us[int(0.9 * (len(us) - 1))],
+            "us_back_to_back": ms * 1e3 / (reps * per_graph), "calls_timed": reps * per_graph, "region_ms": ms,
+            "clocks": regions.clocks(t0, t1)}
+
+
+def with_rates(entry, alg_bytes_per_call, peaks, flops=None):
+    """GB/s over the algorithmic bytes (back-to-back mean and per-call median) against the measured and nominal peaks."""
+    gbs = alg_bytes_per_call / entry["us_back_to_back"] / 1e3
+    entry.update({"bytes": alg_bytes_per_call, "GBps": gbs, "frac_of_measured": gbs / peaks["hbm_gbs"],
+                  "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
+                  "GBps_median_call": alg_bytes_per_call / entry["us_median"] / 1e3})
+    if flops is not None:
+        tf = flops / entry["us_back_to_back"] / 1e6
+        entry.update({"TFLOPs": tf, "frac_of_burst": tf / peaks["bf16_tflops"],
+                      "frac_of_sustained": tf / peaks["bf16_tflops_sustained"]})
+    return entry
+
+
 def run_ours(args, rank, local_rank, world):
     import torch
 
@@ -362,396 +515,281 @@ def run_ours(args, rank, local_rank, world):
         torch.cuda.synchronize()
 
     peaks, peak_kind = measured_peaks()
-    M = 1
-    layer_shapes = synthgen.GEMMA3_4B_LAYER
-    # launch groups: projections sharing their input run as one call on weights concatenated along N
-    groups = [["q", "k", "v"], ["o"], ["gate", "up"], ["down"]] if args.fuse else [[n] for n, _, _, _ in layer_shapes]
-    by_name = {n: (K, N, seed) for n, K, N, seed in layer_shapes}
-    shapes = [("|".join(g), by_name[g[0]][0], sum(by_name[n][1] for n in g), by_name[g[0]][2]) for g in groups]
-    max_K = max(K for _, K, _, _ in shapes)
-    step_bytes_layer = layer_bytes(M)
     _, hk, hn, hseed = synthgen.GEMMA3_4B_LM_HEAD
-    ctx = fd.fdqp_create(local_rank, 8, max(max_K, hk), max(max(N for _, _, N, _ in shapes), hn))
-    if args.param:
-        for kv in args.param:
-            key, val = kv.split("=")
-            fd.fdqp_set_param(ctx, key, int(val))
-
-    # ---- resident inputs: LAYER_COPIES distinct weight sets, one x and one y per projection
-    copies = []
-    host_layer0 = None
-    for c in range(LAYER_COPIES):
-        layer = []
-        for g in groups:
-            parts = []
-            for name in g:
-                K, N, seed = by_name[name]
-                w = synthgen.weights(seed + 1000 * c, K, N)
-                parts.append(fd.q4nx_pack(w.codes, w.scales, w.offsets))
-                if c == 0:
-                    host_layer0 = host_layer0 or []
-                    host_layer0.append((w, synthgen.activations(by_name[g[0]][2], M, K)))
-            layer.append(torch.from_numpy(np.concatenate(parts)).cuda())
-        copies.append(layer)
-    xs_host = [synthgen.activations(seed, M, K) for _, K, _, seed in shapes]
-    xs = [torch.from_numpy(x.view(np.int16)).cuda() for x in xs_host]
-    ys = [torch.empty((M, N), dtype=torch.float32, device="cuda") for _, _, N, _ in shapes]
+    M = 1
+    ctx = fd.fdqp_create(local_rank, 8, 21504, hn)
+    for kv in args.param or []:
+        key, val = kv.split("=")
+        fd.fdqp_set_param(ctx, key, int(val))
     stream = torch.cuda.Stream()
     sraw = stream.cuda_stream
-
-    def enqueue_layer(c):
-        for i, (_, K, N, _) in enumerate(shapes):
-            fd.fdqp_run(ctx, xs[i], copies[c][i], ys[i], M, K, N, sraw)
-
-    # CUDA graphs: a decode step of the real model is 34 such layers back to back, so the layers are captured
-    # LAYER_COPIES at a time (one pass over all resident weight copies per graph); single-layer graphs cover the
-    # remainder when the step count is not a multiple of LAYER_COPIES.
-    # kernels one step launches (activation preparation and split-K sum kernels included, when the plan uses them)
-    count0 = fd.fdqp_launch_count(ctx)
-    enqueue_layer(0)
-    torch.cuda.synchronize()
-    kernels_per_step = fd.fdqp_launch_count(ctx) - count0
-    graphs = None
-    pass_graph = None
-    if args.graph:
-        graphs = []
-        with torch.cuda.stream(stream):
-            enqueue_layer(0)
-        stream.synchronize()
-        for c in range(LAYER_COPIES):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                enqueue_layer(c)
-            graphs.append(g)
-        pass_graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(pass_graph, stream=stream):
-            for c in range(LAYER_COPIES):
-                enqueue_layer(c)
-
-    def run_steps(first, count):
-        """Enqueue `count` consecutive steps starting at step index `first`."""
-        i = first
-        end = first + count
-        while i < end:
-            c = i % LAYER_COPIES
-            if pass_graph is not None and c == 0 and end - i >= LAYER_COPIES:
-                with torch.cuda.stream(stream):
-                    pass_graph.replay()
-                i += LAYER_COPIES
-            elif graphs is not None:
-                with torch.cuda.stream(stream):
-                    graphs[c].replay()
-                i += 1
-            else:
-                enqueue_layer(c)
-                i += 1
-
-    def step(i):
-        run_steps(i, 1)
-
-    run_steps(0, args.warmup)
-    first_timed = -(-args.warmup // LAYER_COPIES) * LAYER_COPIES   # start the timed region on a pass boundary
-    run_steps(args.warmup, first_timed - args.warmup)
-    stream.synchronize()
-
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler is not None:
         sampler.start()
-        time.sleep(0.3)
-    launches_before = fd.fdqp_launch_count(ctx)
+    regions = Regions(sampler)
+
+    # ---- headline: the largest single-GPU configuration, the Gemma3-4B LM head at M = 1 (seed 17), one call per step
+    hw = synthgen.weights(hseed, hk, hn)
+    hW = torch.from_numpy(fd.q4nx_pack(hw.codes, hw.scales, hw.offsets)).cuda()
+    hx_host = synthgen.activations(hseed, 1, hk)
+    hx = torch.from_numpy(hx_host.view(np.int16)).cuda()
+    hy = torch.empty((1, hn), dtype=torch.float32, device="cuda")
+    step_bytes = alg_bytes(1, hk, hn)
+    count0 = fd.fdqp_launch_count(ctx)
+    fd.fdqp_run(ctx, hx, hW, hy, 1, hk, hn, sraw)
+    stream.synchronize()
+    kernels_per_step = fd.fdqp_launch_count(ctx) - count0
+    for _ in range(args.warmup):
+        fd.fdqp_run(ctx, hx, hW, hy, 1, hk, hn, sraw)
+    stream.synchronize()
+    # EXACTLY --steps steps per block; the block is repeated until the timed region is long enough to carry clock samples
+    g_steps = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_steps, stream=stream):
+        for _ in range(args.steps):
+            fd.fdqp_run(ctx, hx, hW, hy, 1, hk, hn, sraw)
+    with torch.cuda.stream(stream):
+        g_steps.replay()
+    stream.synchronize()
+    blocks = max(1, int(np.ceil(MIN_REGION_MS / (args.steps * 0.070))))
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    ev0.record(stream)
-    run_steps(first_timed, args.steps)
-    ev1.record(stream)
+    t_host0 = time.time()
+    with torch.cuda.stream(stream):
+        ev0.record(stream)
+        for _ in range(blocks):
+            g_steps.replay()
+        ev1.record(stream)
     stream.synchronize()
+    t_host1 = time.time()
     barrier()
-    ms = ev0.elapsed_time(ev1)
-    calls_per_step = len(shapes)
-    launches = kernels_per_step * args.steps
-    if graphs is None:
-        assert fd.fdqp_launch_count(ctx) - launches_before == launches
-    clocks = sampler.stop() if rank == 0 else None
+    timed_steps = blocks * args.steps
+    ms = max_over_ranks(ev0.elapsed_time(ev1), dist, "cuda")
     if fd.fdqp_last_status(ctx) != 0:
         raise SystemExit("bench.py: a kernel reported " + fd.fdqp_status_string(fd.fdqp_last_status(ctx)))
-    ms = max_over_ranks(ms, dist, "cuda")
+    head_clocks = regions.clocks(t_host0, t_host1)
+    head_us = ms * 1e3 / timed_steps
+    gbs = whole_job_gbs(step_bytes, timed_steps, world, ms)
 
-    # ---- end to end: host x in, host y out, through fdqp_run_host_async (pinned buffers) + one stream sync, every step
-    xs_pin = [torch.from_numpy(x.view(np.int16)).pin_memory() for x in xs_host]
-    ys_pin = [torch.empty((M, N), dtype=torch.float32).pin_memory() for _, _, N, _ in shapes]
-    e2e_steps = max(3, min(args.steps, 200))
-
-    def e2e_enqueue(c):
-        for j, (_, K, N, _) in enumerate(shapes):
-            fd.fdqp_run_host_async(ctx, xs_pin[j], copies[c][j], ys_pin[j], M, K, N, sraw)
-
-    e2e_enqueue(0)             # the first call allocates the context's staging buffers
+    # ---- end to end: host x in, host y out through fdqp_run_host_async (pinned buffers) + one stream sync, every step
+    x_pin = torch.from_numpy(hx_host.view(np.int16)).pin_memory()
+    y_pin = torch.empty((1, hn), dtype=torch.float32).pin_memory()
+    fd.fdqp_run_host_async(ctx, x_pin, hW, y_pin, 1, hk, hn, sraw)     # the first call allocates the staging buffers
     stream.synchronize()
-    e2e_graphs = None
-    if graphs:
-        # the step's four calls recorded once per weight set and replayed: with pinned buffers used in place a step is
-        # kernels only (they read x from and write y to host memory), and the host pays one launch per step
-        e2e_graphs = []
-        for c in range(LAYER_COPIES):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                e2e_enqueue(c)
-            e2e_graphs.append(g)
-
-    def e2e_step(i):
-        c = i % LAYER_COPIES
-        if e2e_graphs is not None:
-            with torch.cuda.stream(stream):
-                e2e_graphs[c].replay()
-        else:
-            e2e_enqueue(c)
-        stream.synchronize()   # the step's results are in host memory from here on
-
-    for i in range(3):
-        e2e_step(i)
+    e2e_steps = max(args.steps, 200)
+    for _ in range(3):
+        fd.fdqp_run_host_async(ctx, x_pin, hW, y_pin, 1, hk, hn, sraw)
+        stream.synchronize()
     barrier()
     t0 = time.perf_counter()
-    for i in range(e2e_steps):
-        e2e_step(3 + i)
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    e2e_s = max_over_ranks(e2e_s, dist, "cuda")
+    for _ in range(e2e_steps):
+        fd.fdqp_run_host_async(ctx, x_pin, hW, y_pin, 1, hk, hn, sraw)
+        stream.synchronize()                                            # the step's result is in host memory from here on
+    e2e_s = max_over_ranks(time.perf_counter() - t0, dist, "cuda")
 
-    # ---- LM head (M = 1) for the tokens/s figure: 34 layers + head, projections only
-    head_ms = None
-    if rank == 0 and not args.no_head:
-        hw = synthgen.weights(hseed, hk, hn)
-        hW = torch.from_numpy(fd.q4nx_pack(hw.codes, hw.scales, hw.offsets)).cuda()
-        del hw
-        hx = torch.from_numpy(synthgen.activations(hseed, 1, hk).view(np.int16)).cuda()
-        hy = torch.empty((1, hn), dtype=torch.float32, device="cuda")
-        for _ in range(3):
-            fd.fdqp_run(ctx, hx, hW, hy, 1, hk, hn, sraw)
-        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        h0.record(stream)
-        for _ in range(10):
-            fd.fdqp_run(ctx, hx, hW, hy, 1, hk, hn, sraw)
-        h1.record(stream)
-        stream.synchronize()
-        head_ms = h0.elapsed_time(h1) / 10
+    line_extra = {}
+    if rank == 0 and not args.headline_only:
+        # ---- every BASELINE configuration and M: per-call statistics, GB/s, fractions, launch plan, clocks
+        configs = {}
 
-    # ---- the same projections at M = 8 (batched decode): one graph pass over the weight copies, LM head directly
-    batch8 = None
-    if rank == 0 and not args.no_head:
+        def shape_entry(K, N, Mi, seed, W_list=None, amp=1.0):
+            copies = W_list or weight_copies(torch, tiled_weights(fd, torch, K, N, seed))
+            x = torch.from_numpy(synthgen.activations(seed, Mi, K, amp).view(np.int16)).cuda()
+            y = torch.empty((Mi, N), dtype=torch.float32, device="cuda")
+            ent = time_region(torch, stream, lambda i: fd.fdqp_run(ctx, x, copies[i % len(copies)], y, Mi, K, N, sraw),
+                              len(copies), regions)
+            ent["launch"] = fd.fdqp_describe(ctx, Mi, K, N)
+            return with_rates(ent, alg_bytes(Mi, K, N), peaks), copies
+
+        _, K0, N0, seed0 = synthgen.GEMMA3_1B_GATE
+        configs["0: Gemma3-1B gate K=1152 N=6912 M=1"], _ = shape_entry(K0, N0, 1, seed0)
+        # config 1: the Gemma3-4B decoder layer at M = 1 -- per call, as four single calls, and as chains
+        by_name = {n: (K, N, seed) for n, K, N, seed in synthgen.GEMMA3_4B_LAYER}
+        groups = [["q", "k", "v"], ["o"], ["gate", "up"], ["down"]]
+        shapes = [("|".join(g), by_name[g[0]][0], sum(by_name[n][1] for n in g), by_name[g[0]][2]) for g in groups]
+        layer_copies = []
+        for c in range(LAYER_COPIES):
+            layer_copies.append([tiled_weights(fd, torch, K, N, seed + 1000 * c) for _, K, N, seed in shapes])
+        xs = [torch.from_numpy(synthgen.activations(seed, 1, K).view(np.int16)).cuda() for _, K, _, seed in shapes]
+        ys = [torch.empty((1, N), dtype=torch.float32, device="cuda") for _, _, N, _ in shapes]
+        per_call = {}
+        for j, (name, K, N, seed) in enumerate(shapes):
+            ent = time_region(torch, stream, lambda i, j=j, K=K, N=N: fd.fdqp_run(ctx, xs[j], layer_copies[i % LAYER_COPIES][j], ys[j], 1, K, N, sraw),
+                              LAYER_COPIES, regions)
+            ent["launch"] = fd.fdqp_describe(ctx, 1, K, N)
+            per_call[f"{name} K={K} N={N}"] = with_rates(ent, alg_bytes(1, K, N), peaks)
+        lbytes = layer_bytes(1)
+
+        def layer_single(i):
+            for j, (_, K, N, _) in enumerate(shapes):
+                fd.fdqp_run(ctx, xs[j], layer_copies[i % LAYER_COPIES][j], ys[j], 1, K, N, sraw)
+
+        def chain_of(cs):
+            return fd.make_chain([fd.chain_step(xs[j], layer_copies[c][j], ys[j], K, N)
+                                  for c in cs for j, (_, K, N, _) in enumerate(shapes)])
+
+        chains1 = [chain_of([c]) for c in range(LAYER_COPIES)]
+        chain8 = chain_of(range(LAYER_COPIES))
+        layer = {"four_single_calls": with_rates(time_region(torch, stream, layer_single, LAYER_COPIES, regions), lbytes, peaks),
+                 "one_chained_launch_per_layer": with_rates(time_region(torch, stream, lambda i: fd.fdqp_run_chain(ctx, chains1[i % LAYER_COPIES], 1, sraw), LAYER_COPIES, regions), lbytes, peaks)}
+        ent8 = time_region(torch, stream, lambda i: fd.fdqp_run_chain(ctx, chain8, 1, sraw), 1, regions)
+        for k in ("us_median", "us_min", "us_p90", "us_back_to_back"):
+            ent8[k] /= LAYER_COPIES                                      # per layer
+        layer["one_chained_launch_per_8_layers"] = with_rates(ent8, lbytes, peaks)
+        configs["1: Gemma3-4B decoder layer M=1"] = {"per_call": per_call, "per_layer": layer,
+                                                     "note": "the seven projections as q|k|v, o, gate|up, down (inputs sharing x are "
+                                                             "concatenated along N); independent seeded inputs, so a chain cuts the "
+                                                             "layer's blocks into CTA ranges as one sequence; times per layer"}
+        _, K2, N2, seed2 = synthgen.GEMMA3_12B_GATE_UP
+        W2 = None
+        for Mi in (1, 2, 4, 8):
+            configs[f"2: Gemma3-12B gate|up K={K2} N={N2} M={Mi}"], W2 = shape_entry(K2, N2, Mi, seed2, W2)
+        del W2
+        _, K3, N3, seed3 = synthgen.GEMMA3_27B_DOWN
+        W3 = None
+        for Mi in (1, 4, 8):
+            configs[f"3: Gemma3-27B down K={K3} N={N3} M={Mi}"], W3 = shape_entry(K3, N3, Mi, seed3, W3, amp=K3 ** -0.5)
+        del W3
+        ent = time_region(torch, stream, lambda i: fd.fdqp_run(ctx, hx, hW, hy, 1, hk, hn, sraw), 1, regions)
+        ent["launch"] = fd.fdqp_describe(ctx, 1, hk, hn)
+        configs[f"4: Gemma3-4B LM head K={hk} N={hn} M=1"] = with_rates(ent, step_bytes, peaks)
+
+        # ---- decode tokens/s, projections only: 34 layers + LM head (attention, norms and sampling are out of scope)
+        L = synthgen.GEMMA3_4B_LAYERS
+        head_steps = [fd.chain_step(hx, hW, hy, hk, hn)]
+        token_chain = fd.make_chain([fd.chain_step(xs[j], layer_copies[l % LAYER_COPIES][j], ys[j], K, N)
+                                     for l in range(L) for j, (_, K, N, _) in enumerate(shapes)] + head_steps)
+        tok = time_region(torch, stream, lambda i: fd.fdqp_run_chain(ctx, token_chain, 1, sraw), 1, regions, pairs=40)
+        token_bytes = L * lbytes + step_bytes
+
+        def token_single(i):
+            for l in range(L):
+                layer_single(l)
+            fd.fdqp_run(ctx, hx, hW, hy, 1, hk, hn, sraw)
+
+        tok1 = time_region(torch, stream, token_single, 1, regions, pairs=40)
+        decode = {"chained": dict(with_rates(tok, token_bytes, peaks), tokens_per_s=1e6 / tok["us_back_to_back"],
+                                  launches_per_token=-(-(4 * L + 1) // 64)),
+                  "single_calls": dict(with_rates(tok1, token_bytes, peaks), tokens_per_s=1e6 / tok1["us_back_to_back"],
+                                       launches_per_token=5 * L + 1),
+                  "bytes_per_token": token_bytes, "roofline_tokens_per_s": peaks["hbm_gbs"] * 1e9 / token_bytes}
+
+        # ---- batched decode at M = 8: the layer as single calls and chained, and the LM head
         M8 = 8
         xs8 = [torch.from_numpy(synthgen.activations(seed, M8, K).view(np.int16)).cuda() for _, K, _, seed in shapes]
         ys8 = [torch.empty((M8, N), dtype=torch.float32, device="cuda") for _, _, N, _ in shapes]
 
-        def enqueue_layer8(c):
-            for i, (_, K, N, _) in enumerate(shapes):
-                fd.fdqp_run(ctx, xs8[i], copies[c][i], ys8[i], M8, K, N, sraw)
+        def layer8(i):
+            for j, (_, K, N, _) in enumerate(shapes):
+                fd.fdqp_run(ctx, xs8[j], layer_copies[i % LAYER_COPIES][j], ys8[j], M8, K, N, sraw)
 
-        with torch.cuda.stream(stream):
-            enqueue_layer8(0)
-        stream.synchronize()
-        g8 = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g8, stream=stream):
-            for c in range(LAYER_COPIES):
-                enqueue_layer8(c)
-        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with torch.cuda.stream(stream):
-            for _ in range(3):
-                g8.replay()
-            b0.record(stream)
-            for _ in range(20):
-                g8.replay()
-            b1.record(stream)
-        stream.synchronize()
-        layer8_ms = b0.elapsed_time(b1) / (20 * LAYER_COPIES)
+        chain8_m8 = fd.make_chain([fd.chain_step(xs8[j], layer_copies[c][j], ys8[j], K, N)
+                                   for c in range(LAYER_COPIES) for j, (_, K, N, _) in enumerate(shapes)])
+        b_single = with_rates(time_region(torch, stream, layer8, LAYER_COPIES, regions), layer_bytes(M8), peaks)
+        b_chain = time_region(torch, stream, lambda i: fd.fdqp_run_chain(ctx, chain8_m8, M8, sraw), 1, regions)
+        for k in ("us_median", "us_min", "us_p90", "us_back_to_back"):
+            b_chain[k] /= LAYER_COPIES
+        b_chain = with_rates(b_chain, layer_bytes(M8), peaks)
         hx8 = torch.from_numpy(synthgen.activations(hseed, M8, hk).view(np.int16)).cuda()
         hy8 = torch.empty((M8, hn), dtype=torch.float32, device="cuda")
-        for _ in range(3):
-            fd.fdqp_run(ctx, hx8, hW, hy8, M8, hk, hn, sraw)
-        b0.record(stream)
-        for _ in range(10):
-            fd.fdqp_run(ctx, hx8, hW, hy8, M8, hk, hn, sraw)
-        b1.record(stream)
-        stream.synchronize()
-        head8_ms = b0.elapsed_time(b1) / 10
-        batch8 = {"M": M8, "layer_ms": layer8_ms, "lm_head_ms": head8_ms,
-                  "layer_gbs": layer_bytes(M8) / (layer8_ms * 1e-3) / 1e9,
-                  "decode_tokens_per_s": M8 * 1e3 / (synthgen.GEMMA3_4B_LAYERS * layer8_ms + head8_ms)}
+        b_head = with_rates(time_region(torch, stream, lambda i: fd.fdqp_run(ctx, hx8, hW, hy8, M8, hk, hn, sraw), 1, regions),
+                            alg_bytes(M8, hk, hn), peaks)
+        batch8 = {"M": M8, "layer_single_calls": b_single, "layer_chained_8_per_launch": b_chain, "lm_head": b_head,
+                  "decode_tokens_per_s": M8 * 1e6 / (L * b_chain["us_back_to_back"] + b_head["us_back_to_back"])}
         del xs8, ys8, hx8, hy8
 
-    # ---- LM head at a prefill chunk (M = 512, the largest baseline configuration): the tensor-core path, against the tensor roofline
-    prefill = None
-    if rank == 0 and not args.no_head:
-        PM = 512
-        pctx = fd.fdqp_create(local_rank, PM, hk, hn)
-        px = torch.from_numpy(synthgen.activations(hseed, PM, hk).view(np.int16)).cuda()
-        py = torch.empty((PM, hn), dtype=torch.float32, device="cuda")
-        for _ in range(3):
-            fd.fdqp_run(pctx, px, hW, py, PM, hk, hn, sraw)
-        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        p0.record(stream)
-        for _ in range(6):
-            fd.fdqp_run(pctx, px, hW, py, PM, hk, hn, sraw)
-        p1.record(stream)
-        stream.synchronize()
+        # ---- LM head at a prefill chunk (M = 512): the tensor-core path, against the tensor roofline
+        pctx = fd.fdqp_create(local_rank, 512, hk, hn)
+        px = torch.from_numpy(synthgen.activations(hseed, 512, hk).view(np.int16)).cuda()
+        py = torch.empty((512, hn), dtype=torch.float32, device="cuda")
+        prefill = {}
+        for pm in (512, 128, 32):
+            ent = time_region(torch, stream, lambda i, pm=pm: fd.fdqp_run(pctx, px, hW, py, pm, hk, hn, sraw), 1, regions, pairs=24)
+            ent["launch"] = fd.fdqp_describe(pctx, pm, hk, hn)
+            prefill[f"M={pm}"] = with_rates(ent, alg_bytes(pm, hk, hn), peaks, flops=2.0 * pm * hk * hn)
         if fd.fdqp_last_status(pctx) != 0:
             raise SystemExit("bench.py: the prefill kernel reported " + fd.fdqp_status_string(fd.fdqp_last_status(pctx)))
-        p_ms = p0.elapsed_time(p1) / 6
-        tflops = 2.0 * PM * hk * hn / (p_ms * 1e-3) / 1e12
-        prefill = {"workload": f"Gemma3-4B LM head K={hk} N={hn} at M={PM}", "ms": p_ms, "tflops": tflops,
-                   "bound": "tensor", "peak_burst_tflops": peaks.get("bf16_tflops"),
-                   "peak_sustained_tflops": peaks.get("bf16_tflops_sustained"),
-                   "frac_of_burst": tflops / peaks["bf16_tflops"] if peaks.get("bf16_tflops") else None,
-                   "frac_of_sustained": (tflops / peaks["bf16_tflops_sustained"]) if peaks.get("bf16_tflops_sustained") else None,
-                   "launch": fd.fdqp_describe(pctx, PM, hk, hn)}
-        # smaller token counts on the same matrix (the one-SM forms of the kernel), same timing
-        other = {}
-        for om in (32, 128):
-            for _ in range(3):
-                fd.fdqp_run(pctx, px, hW, py, om, hk, hn, sraw)
-            p0.record(stream)
-            for _ in range(6):
-                fd.fdqp_run(pctx, px, hW, py, om, hk, hn, sraw)
-            p1.record(stream)
-            stream.synchronize()
-            if fd.fdqp_last_status(pctx) != 0:
-                raise SystemExit("bench.py: the prefill kernel reported " + fd.fdqp_status_string(fd.fdqp_last_status(pctx)))
-            o_ms = p0.elapsed_time(p1) / 6
-            other[f"M{om}"] = {"ms": o_ms, "tflops": 2.0 * om * hk * hn / (o_ms * 1e-3) / 1e12,
-                               "launch": fd.fdqp_describe(pctx, om, hk, hn)}
-        prefill["other_token_counts"] = other
         fd.fdqp_destroy(pctx)
         del px, py
+        configs[f"4: Gemma3-4B LM head K={hk} N={hn} M=512 (tensor cores)"] = prefill["M=512"]
 
-    # ---- next steps beside the projection: decode attention over a KV cache, and the format variants of the container
-    attention = None
-    formats = None
-    dequant = None
-    if rank == 0 and not args.no_head:
-        H, G, d, L = 8, 4, 256, 32768          # Gemma3-4B heads at a 32k context
-        ncache = max(1, int(np.ceil(4 * L2_BYTES / (2 * G * L * d * 2))))
+        # ---- next steps beside the projection: decode attention, format variants, the dequantisation engine
+        H, G, d, Lc = 8, 4, 256, 32768
+        ncache = max(1, int(np.ceil(4 * L2_BYTES / (2 * G * Lc * d * 2))))
         gen = torch.Generator(device="cuda").manual_seed(2)
-        caches = [(torch.randn((G, L, d), device="cuda", generator=gen).to(torch.bfloat16),
-                   torch.randn((G, L, d), device="cuda", generator=gen).to(torch.bfloat16)) for _ in range(ncache)]
+        caches = [(torch.randn((G, Lc, d), device="cuda", generator=gen).to(torch.bfloat16),
+                   torch.randn((G, Lc, d), device="cuda", generator=gen).to(torch.bfloat16)) for _ in range(ncache)]
         aq = torch.randn((H, d), device="cuda", generator=gen).to(torch.bfloat16)
         ao = torch.empty((H, d), dtype=torch.float32, device="cuda")
-        attention = {"workload": f"Gemma3-4B decode attention, H={H} G={G} d={d}, L={L}", "bound": "hbm"}
+        attention = {"workload": f"Gemma3-4B decode attention, H={H} G={G} d={d}, L={Lc}"}
         for name, window in (("global", 0), ("window_1024", 1024)):
-            reps = 20
-            ga = torch.cuda.CUDAGraph()
-            with torch.cuda.stream(stream):
-                for i in range(3):
-                    fd.fdqp_flowkv_decode(ctx, aq, caches[i % ncache][0], caches[i % ncache][1], ao, H, G, d, L, L, window,
-                                          d ** -0.5, sraw)
-            stream.synchronize()
-            with torch.cuda.graph(ga, stream=stream):
-                for i in range(reps):
-                    fd.fdqp_flowkv_decode(ctx, aq, caches[i % ncache][0], caches[i % ncache][1], ao, H, G, d, L, L, window,
-                                          d ** -0.5, sraw)
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            with torch.cuda.stream(stream):
-                ga.replay()
-                a0.record(stream)
-                ga.replay()
-                a1.record(stream)
-            stream.synchronize()
-            us = a0.elapsed_time(a1) * 1e3 / reps
-            n_att = window if window else L
-            a_gbs = 2.0 * G * n_att * d * 2 / us / 1e3
-            attention[name] = {"us": us, "gbs": a_gbs, "frac": a_gbs / peaks["hbm_gbs"]}
-            del ga
+            ent = time_region(torch, stream, lambda i, window=window: fd.fdqp_flowkv_decode(
+                ctx, aq, caches[i % ncache][0], caches[i % ncache][1], ao, H, G, d, Lc, Lc, window, d ** -0.5, sraw), ncache, regions)
+            attention[name] = with_rates(ent, 2.0 * G * (window if window else Lc) * d * 2, peaks)
         del caches
         formats = {"workload": f"LM head K={hk} N={hn} at M=1, bytes of the format's own container"}
         for name, fmt in (("g64", fd.FMT_G64), ("g128", fd.FMT_G128), ("mxfp4", fd.FMT_MXFP4)):
-            fw = synthgen.weights_fmt(hseed, hk, 4096, fmt)
-            tile = fd.q4nx_pack_fmt(fmt, fw.codes, fw.scales, fw.offsets)
-            nbytes = fd.q4nx_packed_bytes_fmt(fmt, hk, hn)
-            fW = torch.from_numpy(np.tile(tile, hn // 4096)[:nbytes].copy()).cuda()
-            for _ in range(3):
-                fd.fdqp_run_fmt(ctx, fmt, hx, fW, hy, 1, hk, hn, sraw)
-            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            f0.record(stream)
-            for _ in range(10):
-                fd.fdqp_run_fmt(ctx, fmt, hx, fW, hy, 1, hk, hn, sraw)
-            f1.record(stream)
-            stream.synchronize()
-            f_ms = f0.elapsed_time(f1) / 10
-            f_gbs = (nbytes + 2 * hk + 4 * hn) / (f_ms * 1e-3) / 1e9
-            formats[name] = {"ms": f_ms, "gbs": f_gbs, "frac": f_gbs / peaks["hbm_gbs"]}
+            fW = tiled_weights(fd, torch, hk, hn, hseed, fmt)
+            ent = time_region(torch, stream, lambda i, fmt=fmt, fW=fW: fd.fdqp_run_fmt(ctx, fmt, hx, fW, hy, 1, hk, hn, sraw), 1, regions, pairs=40)
+            formats[name] = with_rates(ent, fW.numel() + 2 * hk + 4 * hn, peaks)
             del fW
-        # the dequantisation engine on the LM head: container -> dense bf16 matrix in HBM (write-bound)
         dq_out = torch.empty((hk, hn), dtype=torch.bfloat16, device="cuda")
-        for _ in range(2):
-            fd.fdqp_dequant(ctx, hW, dq_out, True, hk, hn, sraw)
-        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        d0.record(stream)
-        for _ in range(5):
-            fd.fdqp_dequant(ctx, hW, dq_out, True, hk, hn, sraw)
-        d1.record(stream)
-        stream.synchronize()
-        dq_ms = d0.elapsed_time(d1) / 5
-        dq_gbs = (0.625 + 2.0) * hk * hn / (dq_ms * 1e-3) / 1e9
-        dequant = {"workload": f"LM head K={hk} N={hn} -> bf16 [K][N]", "ms": dq_ms, "gbs": dq_gbs, "bound": "hbm",
-                   "frac": dq_gbs / peaks["hbm_gbs"]}
+        ent = time_region(torch, stream, lambda i: fd.fdqp_dequant(ctx, hW, dq_out, True, hk, hn, sraw), 1, regions, pairs=24)
+        dequant = with_rates(ent, (0.625 + 2.0) * hk * hn, peaks)
+        dequant["workload"] = f"LM head K={hk} N={hn} -> bf16 [K][N]"
         del dq_out
         if fd.fdqp_last_status(ctx) != 0:
             raise SystemExit("bench.py: a kernel reported " + fd.fdqp_status_string(fd.fdqp_last_status(ctx)))
+        line_extra = {"configs": configs, "decode_tokens": decode, "decode_tokens_per_s": decode["chained"]["tokens_per_s"],
+                      "batched_decode": batch8, "prefill_lm_head": prefill, "decode_attention": attention,
+                      "format_variants": formats, "dequant_engine": dequant}
 
-    # ---- CPU baseline: the oracle on the host cores, one pass over the same layer (rank 0, N = 1 only)
+    clocks_all = sampler.stop() if sampler is not None else None
+
+    # ---- CPU baseline: the oracle on the host cores over the same LM head (rank 0, N = 1 only): all cores, then one
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         import oracle
         cores = min(oracle.max_threads(), os.cpu_count() or 1)
         t0 = time.perf_counter()
         passes = 0
-        while passes < 1 or time.perf_counter() - t0 < 10:   # about 10 s of oracle work
-            for w, x in host_layer0:
-                oracle.project(x, w.codes, w.scales, w.offsets, nthreads=cores)
+        while passes < 1 or time.perf_counter() - t0 < 8:
+            oracle.project(hx_host, hw.codes, hw.scales, hw.offsets, nthreads=cores)
             passes += 1
         dt = time.perf_counter() - t0
-        cpu = {"value": layer_bytes(M) * passes / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
-               "sample": f"{passes} pass(es) of the whole layer (7 projections, all outputs), {dt:.1f} s"}
+        n1 = 8192                                                      # single thread: a 1/32 column sample
+        t0 = time.perf_counter()
+        oracle.project(hx_host, hw.codes, hw.scales, hw.offsets, n0=0, n1=n1, nthreads=1)
+        dt1 = time.perf_counter() - t0
+        cpu = {"value": step_bytes * passes / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+               "sample": f"{passes} pass(es) over all {hn} outputs of the LM head, {dt:.1f} s",
+               "single_thread": {"value": alg_bytes(1, hk, n1) / dt1 / 1e9, "unit": "GB/s", "cores": 1,
+                                 "sample": f"outputs 0..{n1 - 1} of the LM head, {dt1:.1f} s"}}
 
     if rank == 0:
-        step_bytes = step_bytes_layer
-        gbs = whole_job_gbs(step_bytes, args.steps, world, ms)
-        per_launch_us = ms * 1e3 / (calls_per_step * args.steps)   # one GEMV launch incl. its preparation kernel
-        achieved = (step_bytes / calls_per_step) / (per_launch_us * 1e-6) / 1e9
-        layer_ms = ms / args.steps
         line = {
             "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": layer_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "ms_per_step": head_us * 1e-3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": {"workload": WORKLOAD, "M": M, "bytes_per_step": step_bytes, "cuda_graph": (f"{LAYER_COPIES} steps per graph" if graphs else False),
-                       "calls_per_step": [name for name, _, _, _ in shapes],
-                       "l2": f"inputs larger than L2: steps rotate over {LAYER_COPIES} distinct weight sets "
-                             f"({LAYER_COPIES * step_bytes / 1e6:.0f} MB)",
+            "config": {"workload": WORKLOAD, "M": M, "K": hk, "N": hn, "bytes_per_step": step_bytes,
+                       "launches_per_step": kernels_per_step, "timed_steps": timed_steps,
+                       "timing": f"{blocks} replays of a CUDA graph of exactly --steps = {args.steps} calls, CUDA events on the launching stream",
+                       "l2": "inputs larger than L2: every step streams 419 MB of weights through a 126 MB L2",
                        "multi_gpu": "independent replicas, no collective",
-                       "launch": fd.fdqp_describe(ctx, 1, 2560, 10240)},
+                       "launch": fd.fdqp_describe(ctx, 1, hk, hn)},
             "frac_of_nominal_8TBps": gbs / world / NOMINAL_HBM_GBS,
-            "decode_tokens_per_s": (1e3 / (synthgen.GEMMA3_4B_LAYERS * layer_ms + head_ms)) if head_ms else None,
-            "lm_head_ms": head_ms,
-            "lm_head_gbs": (alg_bytes(1, hk, hn) / (head_ms * 1e-3) / 1e9) if head_ms else None,
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": achieved / peaks["hbm_gbs"],
-                         # ncu, K=2560 N=98304 M=1 (profiles/gemv_m1_k2560_n98304.md): dram read+write = 1.024 x the
-                         # algorithmic bytes; traffic grows in proportion to 0.625*K*N, so scale to this call size
-                         "traffic": 1.024 * step_bytes / calls_per_step, "peak_kind": peak_kind + " copy bandwidth",
-                         "kernel": "fdqp_gemv_kernel", "launch_us": per_launch_us},
-            "batched_decode": batch8,
-            "prefill_lm_head": prefill,
-            "decode_attention": attention,
-            "format_variants": formats,
-            "dequant_engine": dequant,
+            "roofline": {"bound": "hbm", "achieved": step_bytes / head_us / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": step_bytes / head_us / 1e3 / peaks["hbm_gbs"],
+                         # one ncu capture of this launch: dram__bytes_read.sum + dram__bytes_write.sum
+                         "traffic": NCU_LM_HEAD_DRAM_BYTES, "peak_kind": peak_kind + " copy bandwidth",
+                         "kernel": "fdqp_gemv_kernel<16,1,4,false,Q4NX>", "launch_us": head_us},
             "cpu_baseline": cpu,
             "e2e": {"value": whole_job_gbs(step_bytes, e2e_steps, world, e2e_s * 1e3), "unit": "GB/s",
-                    "h2d_bytes_per_step": sum(2 * M * K for _, K, _, _ in shapes),
-                    "d2h_bytes_per_step": sum(4 * M * N for _, _, N, _ in shapes), "ms_per_step": e2e_s / e2e_steps * 1e3,
-                    "how": "fdqp_run_host_async per projection on pinned buffers (x read from and y written to host memory "
-                           "by the kernels), " + ("the step's calls replayed from a CUDA graph, " if e2e_graphs is not None else "")
-                           + "one stream synchronisation per step"},
-            "gpu_launches": launches,
-            "clocks": clocks,
+                    "h2d_bytes_per_step": 2 * M * hk, "d2h_bytes_per_step": 4 * M * hn, "ms_per_step": e2e_s / e2e_steps * 1e3,
+                    "how": "fdqp_run_host_async on pinned host buffers + one stream synchronisation per step"},
+            "gpu_launches": kernels_per_step * timed_steps,
+            "clocks": head_clocks or clocks_all,
         }
+        line.update(line_extra)
         print(json.dumps(line), flush=True)
     fd.fdqp_destroy(ctx)
     if dist is not None:
@@ -761,8 +799,8 @@ def run_ours(args, rank, local_rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=8000)
-    ap.add_argument("--warmup", type=int, default=40)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--graph", type=int, default=1, help="replay each step from a CUDA graph (default 1)")
     ap.add_argument("--fuse", type=int, default=1, help="run q|k|v and gate|up as one call each (default 1)")
@@ -781,30 +819,38 @@ def main():
     ap.add_argument("--residual", action="store_true",
                     help="with --shape --rmsnorm: add a residual to x first and write the sum out (fdqp_run_add_rmsnorm_epilogue)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
-    ap.add_argument("--no-head", action="store_true", help="skip the LM-head timing")
+    ap.add_argument("--layer-chain", type=int, default=0,
+                    help="time the Gemma3-4B layer as chained launches of this many layers each (fdqp_run_chain) instead")
+    ap.add_argument("--tokens", type=int, default=1, help="with --layer-chain: token rows M (1 .. 8)")
+    ap.add_argument("--headline-only", action="store_true", help="only the headline workload (no per-configuration table)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
-        if args.steps == 8000 and args.warmup == 40:
-            args.steps, args.warmup = 5, 1
+        if args.steps == 200 and args.warmup == 10:
+            args.steps, args.warmup = 20, 2
         run_reference(args, rank, world)
         return
     if args.warmup < 3:
         args.warmup = 3
     if args.dequant:
-        if args.steps == 8000:
+        if args.steps == 200:
             args.steps = 10
         run_dequant(args)
         return
     if args.flowkv:
-        if args.steps == 8000:
+        if args.steps == 200:
             args.steps = 50
         run_flowkv(args)
         return
+    if args.layer_chain:
+        if args.steps == 200:
+            args.steps = 50
+        run_layer_chain(args)
+        return
     if args.shape:
-        if args.steps == 8000:
+        if args.steps == 200:
             args.steps = 50
         run_shape(args)
         return

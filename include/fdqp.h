@@ -37,6 +37,19 @@
  * unspecified but run-to-run reproducible order; for M >= 9 the weights pass
  * through bf16 before a tensor-core contraction.  Acceptance bound for y against
  * an fp64 evaluation: |y - y_ref| <= 2e-3 * sum_k |x*w_hat| + 1e-5.
+ * What the kernels guarantee for every finite input, and where the acceptance
+ * bound follows from it:
+ *   - M <= 8 (GEMV kernels): the activations enter the arithmetic EXACTLY (no
+ *     rounding of x, whatever the dynamic range inside a 32-group: see fdqp_run);
+ *     a group contributes d * (sum_k code_k x_k) + m * (sum_k x_k), the sums exact
+ *     or fp32-accumulated, combined in fp32.  So |y - y_ref| <= 2^-17 * sum_k
+ *     |x_k| (|d * code_k| + |m|) + 1e-5, which is inside the acceptance bound
+ *     unless more than 99.5 % of that sum cancels inside d * code + m (weights
+ *     that are exactly zero through m = -d * code under the largest activations).
+ *   - M >= 9 (tensor-core kernels): additionally each w_hat is rounded to bf16
+ *     (2^-9 relative), so the bound holds when the K rounding errors average
+ *     out; the dispatch keeps reductions shorter than K = 256 on the GEMV kernels.
+ * Non-finite activations give non-finite outputs in their token row.
  *
  * Conventions
  *   - "host" / "device" on every pointer says where the memory must live.
@@ -163,10 +176,16 @@ FDQP_API fdqp_status fdqp_destroy(fdqp_ctx* ctx);
  * shorter than K = 256 always take the GEMV kernels: the tensor-core path
  * multiplies by bf16-rounded weights, whose rounding errors need a long K to
  * average out inside the acceptance bound.
- * In the GEMV kernels the activations of each 32-group are held as fixed point
- * relative to the group's largest exponent (22 fraction bits below it): exact for
- * every element within 2^14 of the group's largest magnitude, rounded to 2^-22 of
- * that magnitude otherwise.
+ * How the GEMV kernels hold x.  M <= 2: each 32-group as 31-bit fixed point
+ * relative to its largest exponent, in four signed byte planes that ride in the
+ * columns of one integer tensor-core MMA per 16 rows -- exact for every bf16
+ * within 2^22 of the group's largest magnitude.  A group with anything else (a
+ * value more than four million times smaller than its neighbour, a subnormal
+ * beside a normal number, an infinity, a NaN) is not rounded: it is flagged,
+ * contributes nothing through the tensor cores and is evaluated in fp32, weight
+ * by weight as Eq. 3 writes it, inside the same kernel.  M = 3 .. 8: codes and
+ * activations are both exact in bf16 and go through the bf16 tensor-core MMA with
+ * fp32 accumulation; nothing is rounded and nothing needs a flag.
  * Asynchronous on `cuda_stream`; no allocation and no host synchronisation.  W, x
  * and y must stay valid until the stream has passed the call.  Two calls that
  * share a context must be ordered on one stream.
@@ -282,8 +301,8 @@ typedef struct {
  *                            on its output.  A dependency on any EARLIER step than the previous one is not tracked.
  *   depends_on_previous = 0  the step's inputs must not be written by any step of the chain.
  * A step's outputs must not alias the inputs of another step unless that step depends on it.
- * Limits: 1 <= M <= 8; Q4NX only; a normalised step needs its whole row in one K slice (about M * K <= 16384, e.g.
- * every K = 2560 projection up to M = 4... see FDQP_ERR_SIZE below); shapes within the context's maxima.
+ * Limits: 1 <= M <= 8; Q4NX only; a normalised step needs its whole row prepared in one piece (M * K <= 13056 for
+ * M <= 2, M * K <= 32768 above: every K = 2560 projection qualifies); shapes within the context's maxima.
  * Asynchronous on `cuda_stream`; no allocation; uses the context's chain workspace, so calls that share a context
  * must be ordered on one stream.
  * Errors (nothing is launched): FDQP_ERR_ARG (null pointers, n_steps < 1, unknown epilogue, dependency flag on the

@@ -908,14 +908,16 @@ extern "C" fdqp_status fdqp_run_chain(fdqp_ctx* ctx, const fdqp_chain_step* step
         }
         // No step of this launch waits for another one: cut the whole chain, not every step, into equal CTA ranges.
         cp.Wtot = (uint32_t)blocks;
+        cp.has_deps = dependent ? 1 : 0;
         cp.wide = (!dependent && blocks >= (size_t)grid && blocks < (1u << 31) && ctx->p_chain_wide != 0) ? 1 : 0;
         if (ticket_off > ctx->chain_ticket_cap || full_off > kChainFullSlots ||
             edge_off > (size_t)2 * ctx->sm_count * kMaxChainSteps)
             return FDQP_ERR_SIZE;
         const uint32_t part_bytes = 2u * 16u * kStripRows * (uint32_t)m * 4u * (cols ? (uint32_t)kColsPartTerms : 1u);
         const uint32_t norm_bytes = (uint32_t)(kChainPrepItems / 4) * 4u + 64u;
+        const uint32_t geo_bytes = (uint32_t)cp.nunits * 16u;  // the CTA's block range per (step, K slice) unit
         const uint32_t fixed = round_up(xs_bytes, 128) + round_up(xsum_bytes, 128) + round_up(part_bytes, 128) +
-                               round_up(norm_bytes, 128) + (2u * kMaxStages + 4u) * 8u + 128u;
+                               round_up(norm_bytes, 128) + round_up(geo_bytes, 128) + (2u * kMaxStages + 4u) * 8u + 128u;
         // four blocks per warp and stage (half the barrier round trips per tile) while the ring keeps three stages
         int bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (m <= 4 ? 4 : 2);
         uint32_t stage_bytes = 2u * (uint32_t)bpw * kBlockBytes;
@@ -934,7 +936,8 @@ extern "C" fdqp_status fdqp_run_chain(fdqp_ctx* ctx, const fdqp_chain_step* step
         cp.off_xsum = cp.off_xs + round_up(xs_bytes, 128);
         cp.off_part = cp.off_xsum + round_up(xsum_bytes, 128);
         cp.off_norm = cp.off_part + round_up(part_bytes, 128);
-        cp.off_bar = cp.off_norm + round_up(norm_bytes, 128);
+        cp.off_geo = cp.off_norm + round_up(norm_bytes, 128);
+        cp.off_bar = cp.off_geo + round_up(geo_bytes, 128);
         cp.smem_bytes = cp.off_bar + (2u * (uint32_t)nstage + 4u) * 8u;
         plans.push_back(cp);
         plan_epi.push_back(epi ? 1 : 0);

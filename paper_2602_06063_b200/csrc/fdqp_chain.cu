@@ -46,37 +46,50 @@ __device__ __forceinline__ int chain_slice_len(const ChainStep& st, int z) {
 //   chain-wide (cp.wide != 0, only when no step waits for another): the blocks of all steps and slices are laid end
 //     to end and cut into `grid` equal ranges, so that a CTA streams ONE contiguous share of the whole chain: it
 //     prepares activations only for the steps it touches and shares at most two strips with its neighbours.
-__device__ __forceinline__ StepGeom unit_geom(const ChainPlan& cp, const ChainStep& st, int z, int cta, int kCB) {
-    StepGeom g;
-    g.z = z;
-    g.ci = cta;
-    g.nblk = 0;
-    g.bl_first = g.npieces = g.nt = g.bl_tail = g.nchunk = 0;
-    g.a = g.e = g.s_first = g.s_last = g.a_true = 0;
-    g.b_first = z * st.nbz;
-    g.len = chain_slice_len(st, z);
-    const int64_t T = (int64_t)st.S * g.len;
+// (The divisions are done ONCE per CTA and unit, by one thread each, into a table in shared memory: unit_range; every
+// warp role then derives what it needs from the table entry with multiplications only: unit_geom.)
+__device__ __forceinline__ int4 unit_range(const ChainPlan& cp, const ChainStep& st, int z, int cta) {
+    const int len = chain_slice_len(st, z);
+    const int64_t T = (int64_t)st.S * len;
+    int64_t a, e, a_true;
     if (cp.wide) {
         const int64_t B = (int64_t)st.B + (int64_t)z * st.S * st.nbz;  // slices before z are all nbz long
         const int64_t A = range_begin(cta, gridDim.x, cp.Wtot) - B, E = range_begin(cta + 1, gridDim.x, cp.Wtot) - B;
-        g.a = A < 0 ? 0 : (A > T ? T : A);
-        g.e = E < 0 ? 0 : (E > T ? T : E);
-        g.a_true = A;
+        a = A < 0 ? 0 : (A > T ? T : A);
+        e = E < 0 ? 0 : (E > T ? T : E);
+        a_true = A < -1 ? -1 : A;  // only "before this slice or not" matters (see chain_piece_slot)
     } else {
-        if (cta / st.Gz != z) return g;  // another slice's CTA (or one this step cannot use)
-        g.ci = cta % st.Gz;
-        g.a = st.strip_aligned ? range_begin(g.ci, st.Gz, st.S) * g.len : range_begin(g.ci, st.Gz, T);
-        g.e = st.strip_aligned ? range_begin(g.ci + 1, st.Gz, st.S) * g.len : range_begin(g.ci + 1, st.Gz, T);
-        g.a_true = g.a;
+        if (cta / st.Gz != z) return make_int4(0, 0, 0, 0);  // another slice's CTA (or one this step cannot use)
+        const int ci = cta % st.Gz;
+        a = st.strip_aligned ? range_begin(ci, st.Gz, st.S) * len : range_begin(ci, st.Gz, T);
+        e = st.strip_aligned ? range_begin(ci + 1, st.Gz, st.S) * len : range_begin(ci + 1, st.Gz, T);
+        a_true = a;
     }
-    g.nblk = (int)(g.e - g.a);
+    if (e <= a) return make_int4(0, 0, 0, 0);
+    // strips of the first and the last block; the sign of .z tells whether the range began before this slice
+    const int s_first = (int)(a / len), s_last = (int)((e - 1) / len);
+    return make_int4((int)a, (int)e, a_true < 0 ? -1 - s_first : s_first, s_last);
+}
+
+__device__ __forceinline__ StepGeom unit_geom(const ChainPlan& cp, const ChainStep& st, int z, int cta, int kCB, int4 t) {
+    StepGeom g;
+    g.z = z;
+    g.ci = cp.wide ? cta : cta % st.Gz;
+    g.b_first = z * st.nbz;
+    g.len = chain_slice_len(st, z);
+    g.a = t.x;
+    g.e = t.y;
+    g.nblk = t.y - t.x;
+    g.bl_first = g.npieces = g.nt = g.bl_tail = g.nchunk = 0;
+    g.s_first = g.s_last = 0;
+    g.a_true = g.a;
     if (g.nblk <= 0) {
         g.nblk = 0;
         return g;
     }
-    const bool small = fits32(st.Gz, T);
-    g.s_first = div_floor(g.a, g.len, small);
-    g.s_last = div_floor(g.e - 1, g.len, small);
+    g.s_first = t.z < 0 ? -1 - t.z : t.z;
+    g.s_last = t.w;
+    if (t.z < 0) g.a_true = -1;
     g.bl_first = (int)(g.a - g.s_first * g.len);
     g.npieces = (int)(g.s_last - g.s_first) + 1;
     // processing order: the blocks of a partial last strip come first, then the rest of the range in order
@@ -180,6 +193,9 @@ __global__ void __launch_bounds__(kThreads, 1) fdqp_chain_kernel(const __grid_co
         mbar_init(red_full0 + 8u * tid, kCW);
         mbar_init(red_empty0 + 8u * tid, 1);
     }
+    // this CTA's block range in every (step, K slice) unit: one thread per unit does the divisions
+    int4* const geo = reinterpret_cast<int4*>(smem + cp.off_geo);
+    for (int ui = tid; ui < cp.nunits; ui += blockDim.x) geo[ui] = unit_range(cp, cp.step[cp.unit_step[ui]], cp.unit_slice[ui], blockIdx.x);
     mbar_fence_init();
     __syncthreads();
     // The next launch in the stream may begin as soon as SM slots free up: it streams weights (which nothing in this
@@ -194,10 +210,11 @@ __global__ void __launch_bounds__(kThreads, 1) fdqp_chain_kernel(const __grid_co
         uint32_t phase = 0;
         bool alive = true;
         for (int ui = 0; ui < cp.nunits && alive; ++ui) {
+            const int4 gt = geo[ui];
+            if (gt.y <= gt.x) continue;  // nothing of this unit for this CTA
             const int si = cp.unit_step[ui], uz = cp.unit_slice[ui];
             const ChainStep& st = cp.step[si];
-            const StepGeom g = unit_geom(cp, st, uz, blockIdx.x, kCB);
-            if (g.nblk == 0) continue;
+            const StepGeom g = unit_geom(cp, st, uz, blockIdx.x, kCB, gt);
             const int groups_total = st.K / kGroup;
             const int64_t strip_bytes = (int64_t)kGroupBytes * groups_total;
             for (int c = 0; c < g.nchunk; ++c) {
@@ -287,10 +304,11 @@ __global__ void __launch_bounds__(kThreads, 1) fdqp_chain_kernel(const __grid_co
         asm volatile("griddepcontrol.wait;" ::: "memory");
 
         for (int ui = 0; ui < cp.nunits; ++ui) {
+            const int4 gt = geo[ui];
+            if (gt.y <= gt.x) continue;  // nothing of this unit for this CTA
             const int si = cp.unit_step[ui], uz = cp.unit_slice[ui];
             const ChainStep& st = cp.step[si];
-            const StepGeom g = unit_geom(cp, st, uz, blockIdx.x, kCB);
-            if (g.nblk == 0) continue;  // (the same answer in every warp of the CTA)
+            const StepGeom g = unit_geom(cp, st, uz, blockIdx.x, kCB, gt);  // (the same answer in every warp of the CTA)
             const int K = st.K;
             const int groups_total = K / kGroup;
             const int64_t strip_bytes = (int64_t)kGroupBytes * groups_total;
@@ -304,7 +322,13 @@ __global__ void __launch_bounds__(kThreads, 1) fdqp_chain_kernel(const __grid_co
             {
                 const int kbeg = g.b_first * kBlockK;
                 const int kend_full = (g.b_first + g.len) * kBlockK;
-                const int tile0 = kbeg / kGroup, ntiles = ((kend_full < K ? kend_full : K) - kbeg) / kGroup;
+                const int ntiles_all = ((kend_full < K ? kend_full : K) - kbeg) / kGroup;
+                // A range inside ONE strip touches only its own blocks' share of x (a long-K projection cut over many
+                // CTAs); the normalisation needs the whole row.
+                const bool part_k = g.npieces == 1 && !(EPI && st.norm);
+                const int tile_lo = part_k ? g.bl_first * 8 : 0;
+                const int tile_hi = part_k ? ((g.bl_first + g.nblk) * 8 < ntiles_all ? (g.bl_first + g.nblk) * 8 : ntiles_all) : ntiles_all;
+                const int tile0 = kbeg / kGroup + tile_lo, ntiles = tile_hi - tile_lo;
                 const int items = ntiles * M * 4;  // <= kPrepBatch * kCW * 32 (the plan guarantees it)
                 uint32_t* xs_g = reinterpret_cast<uint32_t*>(smem + cp.off_xs);
                 float* xsc_g = reinterpret_cast<float*>(smem + cp.off_xsum);
@@ -381,7 +405,7 @@ __global__ void __launch_bounds__(kThreads, 1) fdqp_chain_kernel(const __grid_co
                     if (u * kCW * 32 < items) {  // warp-uniform: whole quads run the shuffles together
                         const bool valid = idx < items;
                         const int tm = idx >> 2;
-                        if (xprep_item<MT::kCols>(v[u], M, valid ? tm / M : 0, valid ? tm % M : 0, idx & 3, valid, xs_g, xsc_g))
+                        if (xprep_item<MT::kCols>(v[u], M, tile_lo + (valid ? tm / M : 0), valid ? tm % M : 0, idx & 3, valid, xs_g, xsc_g))
                             saw_flagged = true;
                     }
                 }
@@ -564,7 +588,7 @@ __global__ void __launch_bounds__(kThreads, 1) fdqp_chain_kernel(const __grid_co
         for (int ui = 0; ui < cp.nunits; ++ui) {
             const int si = cp.unit_step[ui], uz = cp.unit_slice[ui];
             const ChainStep& st = cp.step[si];
-            const StepGeom g = unit_geom(cp, st, uz, blockIdx.x, kCB);
+            const StepGeom g = unit_geom(cp, st, uz, blockIdx.x, kCB, geo[ui]);
             const int len = g.len;
             for (int piece = 0; piece < g.npieces; ++piece) {
                 const int G = pieceG + piece;  // index over all steps: hand-over buffer and owner alternate with it
@@ -663,6 +687,7 @@ __global__ void __launch_bounds__(kThreads, 1) fdqp_chain_kernel(const __grid_co
 
     // The last CTA to leave puts the dependency counters back to zero for the next launch (every wait of every CTA
     // has ended by the time its threads meet here).
+    if (!cp.has_deps) return;  // (kernel-uniform) no step of this launch counted anything
     __syncthreads();
     if (tid == 0) {
         __threadfence();

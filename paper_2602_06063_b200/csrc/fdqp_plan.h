@@ -104,11 +104,12 @@ struct ChainPlan {
     int* status;               // host-mapped sticky status word
     int nstage, evict_first;
     int bpw;                   // blocks per consumer warp and ring stage (2 or 4; a stage holds twice as many blocks)
+    int has_deps;              // 1: some step waits for the one before it (the completion counters are in use)
     int wide;                  // 1: chain-wide cut into CTA ranges (no step waits for another), 0: every step cut on its own
     uint32_t Wtot;             // chain-wide cut: blocks of all steps together
     int nunits;                // (step, K slice) pairs in processing order
     uint8_t unit_step[kMaxChainUnits], unit_slice[kMaxChainUnits];
-    uint32_t off_xs, off_xsum, off_part, off_norm, off_bar, smem_bytes;  // shared-memory carve-up (bytes)
+    uint32_t off_xs, off_xsum, off_part, off_norm, off_geo, off_bar, smem_bytes;  // shared-memory carve-up (bytes)
     ChainStep step[kMaxChainSteps];
 };
 

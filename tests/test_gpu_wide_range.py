@@ -161,3 +161,31 @@ def test_format_variants_with_outlier_groups(fresh, fmt, M):
     assert fd.fdqp_last_status(fresh) == 0
     y_ref, a_ref = oracle.fmt_project(fmt, xb, w.codes, w.scales, w.offsets)
     assert_close(y.cpu().numpy(), y_ref, a_ref, f"fmt={fmt} M={M}")
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 8])
+def test_weights_that_cancel_to_zero_under_the_outlier(fresh, M):
+    """The other side of the line: the weight under the outlier is zero through cancellation, d * code + m = 0 with
+    m = -d * code, so d * (sum code x) and m * (sum x) both carry the outlier's magnitude and cancel.  What the library
+    promises for EVERY finite input is |y - y_ref| <= 2^-17 * sum_k |x_k| (|d code_k| + |m|) + 1e-5 (the activations
+    enter exactly; the factorised sums are combined in fp32); the acceptance bound follows from it unless almost all
+    of that sum cancels, as it does here by construction."""
+    K, N = 1024, 96
+    w = synthgen.weights(990 + M, K, N)
+    codes, scales, offsets = w.codes.copy(), w.scales.copy(), w.offsets.copy()
+    x = f32_of(synthgen.activations(991 + M, M, K)) * 2.0 ** -9
+    for g in range(0, K // 32, 4):
+        pos = g * 32 + (3 * g + 2) % 32
+        x[:, pos] = 2.0 ** 12
+        codes[:, pos] = 8
+        scales[:, g] = 0x3E00      # d = 2^-3
+        offsets[:, g] = 0xBF80     # m = -1 = -d * 8
+    case = Case(K, N, M, 0, weights=synthgen.Q4NXWeights(codes, scales, offsets), x=synthgen.bf16_bits(x))
+    y_ref, _ = case.reference()
+    y = case.run(fresh)
+    d = f32_of(scales).astype(np.float64)
+    m = f32_of(offsets).astype(np.float64)
+    mag = np.abs(np.repeat(d, 32, axis=1) * codes) + np.abs(np.repeat(m, 32, axis=1))        # [N, K]
+    big = np.abs(f32_of(case.x).astype(np.float64)) @ mag.T                                   # [M, N]
+    assert np.all(np.isfinite(y))
+    assert np.all(np.abs(y.astype(np.float64) - y_ref) <= 2.0 ** -17 * big + 1e-5)
