@@ -421,7 +421,7 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "ctas_per_sm"   persistent CTAs per SM for the GEMV kernels (1 or 2; 2 implies 8 consumer warps)
  *   "consumer_warps" 8 or 16 consumer warps per CTA
  *   "stages"        shared-memory ring depth in stages (a stage holds consumer_warps / 8 * blocks_per_warp blocks)
- *   "blocks_per_warp" 2 or 4 Q4NX blocks per consumer warp per stage (4 only at M = 1)
+ *   "blocks_per_warp" 2 or 4 Q4NX blocks per consumer warp per stage
  *   "split_k"       number of K slices (1, 2, 4 or 8)
  *   "l2_evict_first" 1 = weight copies carry an evict-first L2 hint
  *   "strip_aligned" 1 = CTA work ranges are cut at strip boundaries, 0 = equal block counts per CTA

@@ -249,8 +249,9 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
             nbz = (p->nb + Z - 1) / Z;
             // four blocks per warp per stage halve the barrier traffic per tile
             const int64_t blocks_per_cta = (int64_t)p->S * p->nb / ((int64_t)ctx->sm_count * ctas_per_sm);
-            // (measured: pays up to M = 4, never when the larger stage would force a K split)
-            bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (M <= 4 && blocks_per_cta >= 4 ? 4 : 2);
+            // (measured: LM head 68 against 91 us at M = 1, 101 against 119 us at M = 8; never when the larger stage would
+            // force a K split)
+            bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (blocks_per_cta >= 4 ? 4 : 2);
             L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw, fmt);
             if (bpw == 4 && ctx->p_bpw != 4 && L.nstage < kMinStages) {  // smaller stages before another K slice
                 bpw = 2;
@@ -275,9 +276,9 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     {
         const double t_block = 0.125 * ctas_per_sm;  // one 5 KB block at an SM's share of HBM bandwidth
         const int64_t blocks_bal = (total_blocks / Z + Gz - 1) / Gz;
-        // (measured: ranges cut inside strips also stream ~4 % slower up to M = 4 -- strip boundaries then fall at odd
-        // places inside the stages, and more stages take the bookkeeping path)
-        const double cost_bal = blocks_bal * t_block * (M <= 4 ? 1.04 : 1.0) + (blocks_bal >= 2 * (int64_t)nbz ? 0.6 : 2.0);
+        // (measured: ranges cut inside strips also stream 3-4 % slower -- strip boundaries then fall at odd places inside
+        // the stages, and more stages take the bookkeeping path)
+        const double cost_bal = blocks_bal * t_block * 1.04 + (blocks_bal >= 2 * (int64_t)nbz ? 0.6 : 2.0);
         const int Ga = Gz < p->S ? Gz : p->S;
         const int64_t blocks_al = (int64_t)((p->S + Ga - 1) / Ga) * nbz;
         const double cost_al = blocks_al * t_block + (Z > 1 ? 2.0 : 0.4);
@@ -369,9 +370,9 @@ extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, in
         }
         if ((e = cudaMemset(ctx->tickets, 0, sizeof(int) * (size_t)S))) { st = cuda_fail(nullptr, e, ""); break; }
         const size_t tiles = (size_t)(max_K / kGroup), toks = (size_t)(max_M < kMaxTokens ? max_M : kMaxTokens);
-        if ((e = cudaMalloc(&ctx->xq, tiles * toks * kColsRecBytes))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMalloc(&ctx->xq, tiles * toks * kColsRecBytes + 16))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMalloc(&ctx->xsc, tiles * 64))) { st = cuda_fail(nullptr, e, ""); break; }
-        if ((e = cudaMemset(ctx->xq, 0, tiles * toks * kColsRecBytes))) { st = cuda_fail(nullptr, e, ""); break; }
+        if ((e = cudaMemset(ctx->xq, 0, tiles * toks * kColsRecBytes + 16))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaMemset(ctx->xsc, 0, tiles * 64))) { st = cuda_fail(nullptr, e, ""); break; }
         if ((e = cudaHostAlloc(&ctx->status_host, sizeof(int), cudaHostAllocMapped))) { st = cuda_fail(nullptr, e, ""); break; }
         *ctx->status_host = 0;
@@ -919,7 +920,7 @@ extern "C" fdqp_status fdqp_run_chain(fdqp_ctx* ctx, const fdqp_chain_step* step
         const uint32_t fixed = round_up(xs_bytes, 128) + round_up(xsum_bytes, 128) + round_up(part_bytes, 128) +
                                round_up(norm_bytes, 128) + round_up(geo_bytes, 128) + (2u * kMaxStages + 4u) * 8u + 128u;
         // four blocks per warp and stage (half the barrier round trips per tile) while the ring keeps three stages
-        int bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (m <= 4 ? 4 : 2);
+        int bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : 4;
         uint32_t stage_bytes = 2u * (uint32_t)bpw * kBlockBytes;
         int nstage = (uint32_t)ctx->smem_optin > fixed ? (int)(((uint32_t)ctx->smem_optin - fixed) / stage_bytes) : 0;
         if (bpw == 4 && ctx->p_bpw != 4 && nstage < kMinStages) {

@@ -271,10 +271,12 @@ __global__ void __launch_bounds__(kThreads, 1) fdqp_chain_kernel(const __grid_co
             la.x_lane = xs + (uint32_t)(gtok * 4 + q) * 16u;
             la.xsc_lane = xsc + q * 8;
             const int tok_b = g8 >> 2, pl = g8 & 3;
-            la.xb_off = tok_b < M ? (uint32_t)(tok_b * kColsRecBytes + pl * 32 + q * 8) : (uint32_t)kColsZeroOff;
+            la.xb_off = tok_b < M ? (uint32_t)(tok_b * kColsRecBytes + pl * 32 + q * 8) : 0u;  // (no such token: weight 0 below)
             const int tok_d = q >> 1;
             la.sc_off = (uint32_t)((tok_d < M ? tok_d : 0) * kColsRecBytes + kColsSumOff);
             lc.w_unit = tok_d < M ? ((q & 1) ? 1.f : 65536.f) : 0.f;
+            asm volatile("mov.b32 %0, 0x000F000F;" : "=r"(lc.nib_mask));
+            asm volatile("mov.b32 %0, 0x43004300;" : "=r"(lc.nib_magic));
         }
         // ldmatrix source rows (see the single-call kernel): codes = row `lane` of the tile; scales / offsets = the
         // 16-byte chunks of the tile's scale and offset words

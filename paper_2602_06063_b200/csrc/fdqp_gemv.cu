@@ -214,11 +214,14 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             la.x_lane = xs + (uint32_t)(gtok * 4 + q) * 16u;
             la.xsc_lane = xsc + q * 8;
             const int tok_b = g >> 2, pl = g & 3;
-            la.xb_off = tok_b < M ? (uint32_t)(tok_b * kColsRecBytes + pl * 32 + q * 8) : (uint32_t)kColsZeroOff;
+            la.xb_off = tok_b < M ? (uint32_t)(tok_b * kColsRecBytes + pl * 32 + q * 8) : 0u;  // (no such token: weight 0 below)
             const int tok_d = q >> 1;
             la.sc_off = (uint32_t)((tok_d < M ? tok_d : 0) * kColsRecBytes + kColsSumOff);
             lc.w_unit = (tok_d < M ? ((q & 1) ? 1.f : 65536.f) : 0.f) * (F::kMx ? 0.5f : 1.f);
             if (F::kMx) lc.mx = mx_tables();
+            // (opaque moves: the compiler keeps the two constants in registers instead of re-creating them per use)
+            asm volatile("mov.b32 %0, 0x000F000F;" : "=r"(lc.nib_mask));
+            asm volatile("mov.b32 %0, 0x43004300;" : "=r"(lc.nib_magic));
         }
         float acc_m[MT::kAccM];  // column modes: offset term of row `lane`, per token
 #pragma unroll
@@ -522,7 +525,9 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             const int kend = kend_full < K ? kend_full : K;
             const uint32_t tile0 = (uint32_t)(kbeg / kGroup), ntiles = (uint32_t)((kend - kbeg) / kGroup);
             constexpr uint32_t kRec = MT::kCols ? kColsRecBytes : kPlaneRecBytes;
-            const uint32_t rec_bytes = ntiles * (uint32_t)M * kRec, sc_bytes = MT::kCols ? 0u : ntiles * (uint32_t)kPlaneSumBytes;
+            // (a bulk copy moves multiples of 16 bytes: an odd number of 136-byte records is rounded up into the slack
+            // both buffers keep behind the records)
+            const uint32_t rec_bytes = (ntiles * (uint32_t)M * kRec + 15u) & ~15u, sc_bytes = MT::kCols ? 0u : ntiles * (uint32_t)kPlaneSumBytes;
             mbar_arrive_expect_tx(x_bar, rec_bytes + sc_bytes);
             const uint8_t* src = reinterpret_cast<const uint8_t*>(p.xq) + (size_t)tile0 * M * kRec;
             for (uint32_t off = 0; off < rec_bytes; off += 32768u) {

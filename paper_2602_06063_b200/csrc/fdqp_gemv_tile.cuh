@@ -30,8 +30,7 @@ __device__ __forceinline__ int64_t cta_of(int64_t L, int64_t G, int64_t T) {
 //
 // M <= 2 (SINGLE == true, "column" layout): the group as 31-bit fixed point relative to its largest exponent, in four
 //   SIGNED base-256 digits, each digit plane in MMA fragment order ({bytes of even k, bytes of odd k}).  Per (tile,
-//   token) a 160-byte record: [plane 3 (most significant): 4 x 8 B by q][plane 2][plane 1][plane 0][{sum x, unit}]
-//   [8 zero bytes][at 144 of TOKEN 0's record: the group sums of x of tokens 0 and 1][pad].
+//   token) a 136-byte record: [plane 3 (most significant): 4 x 8 B by q][plane 2][plane 1][plane 0][{sum x, unit}].
 // M >= 3 (SINGLE == false): no fixed point -- the bf16 activations themselves, permuted into the B-fragment order of
 //   the bf16 MMA (this thread's 16 bytes become (x0,x4), (x1,x5), (x2,x6), (x3,x7)), 64 bytes per (tile, token) at
 //   xq[((T*M + tok)*4 + q)*4], and the group's sum of x at xsc[T*8 + tok].
@@ -60,7 +59,7 @@ __device__ __forceinline__ uint4 add_bf16x8(uint4 a, uint4 b) {
 // is not (a value more than four million times smaller than an outlier beside it, a subnormal beside a normal
 // number), or with a non-finite element, is FLAGGED instead of rounded: its record carries unit = 0 and sum = 0, so
 // that the tensor-core path contributes exactly nothing for it, and the raw bf16 activations in k order in bytes
-// 0..63.  The GEMV kernels then evaluate that group in fp32 straight from Eq. 3 (piece_exact_token below).
+// 0..63 (where the planes would be).  The GEMV kernels then evaluate that group in fp32 straight from Eq. 3 (piece_exact_token below).
 template <bool SINGLE>
 __device__ __forceinline__ bool xprep_item(const uint4 v, int M, int slot, int tok, int q, bool valid,
                                            uint32_t* __restrict__ xq, float* __restrict__ xsc) {
@@ -126,16 +125,15 @@ __device__ __forceinline__ bool xprep_item(const uint4 v, int M, int slot, int t
     }
     constexpr int kRecWords = kColsRecBytes / 4;
     uint32_t* rec = xq + ((int64_t)slot * M + tok) * kRecWords;
-    if (flagged) {
-        *reinterpret_cast<uint4*>(rec + q * 4) = v;  // raw activations 8q .. 8q+7
+    if (flagged) {  // raw activations 8q .. 8q+7 (records are 8-byte aligned)
+        *reinterpret_cast<uint2*>(rec + q * 4) = make_uint2(v.x, v.y);
+        *reinterpret_cast<uint2*>(rec + q * 4 + 2) = make_uint2(v.z, v.w);
     } else {
 #pragma unroll
         for (int pl = 0; pl < 4; ++pl)
             *reinterpret_cast<uint2*>(rec + pl * 8 + q * 2) = make_uint2(plane[pl][0], plane[pl][1]);
     }
     if (q == 0) *reinterpret_cast<uint2*>(rec + kColsSumOff / 4) = make_uint2(__float_as_uint(psum), __float_as_uint(unit));
-    if (q == 1) *reinterpret_cast<uint2*>(rec + kColsZeroOff / 4) = make_uint2(0u, 0u);
-    if (q == 2) xq[(int64_t)slot * M * kRecWords + kColsRowSumOff / 4 + tok] = __float_as_uint(psum);
     return flagged;
 }
 
@@ -214,10 +212,9 @@ __device__ __forceinline__ void tile_load(TileIn& t, uint32_t code_addr, uint32_
         const float2 v = lds64f(tb + la.sc_off);
         t.sc[0] = v.x;
         t.sc[1] = v.y;
-        if (T::kXRow) {
-            const float2 xr = lds64f(tb + (uint32_t)kColsRowSumOff);
-            t.xrow[0] = xr.x;
-            t.xrow[1] = xr.y;
+        if (T::kXRow) {  // the sums of x of both tokens (each in its own record)
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(t.xrow[0]) : "r"(tb + (uint32_t)kColsSumOff));
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(t.xrow[1]) : "r"(tb + (uint32_t)(kColsRecBytes + kColsSumOff)));
         }
         if (kMx) mx_natural_order(t.b[0], t.b[1]);
     } else {
@@ -296,6 +293,7 @@ __device__ __forceinline__ void imma(int (&d)[4], uint32_t a0, uint32_t a1, uint
 //   weighted unit.
 struct LaneConst {
     float w_unit;      // factor on `unit` (0 when the lane's token does not exist)
+    uint32_t nib_mask, nib_magic;  // mode 2: 0x000F000F and 0x43004300, held in registers for the whole kernel
     MxTables mx;       // MXFP4 only: the element look-up tables
 };
 
@@ -306,12 +304,21 @@ __device__ __forceinline__ void mma_bf16_acc(float (&d)[4], uint32_t a0, uint32_
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// D = A * B (accumulator starts at zero: no registers to clear)
+__device__ __forceinline__ void mma_bf16_zero(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                              uint32_t b1) {
+    const float zero = 0.f;
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(zero));
+}
 // Two exact small integers as a bf16 pair: nibbles i and i + 4 of a code word.  (w >> 4i) & 0x000F000F | 0x43004300 is
 // the pair (128 + n_i, 128 + n_{i+4}) -- in bf16 the ulp at 128 is 1 -- and the packed subtraction removes the 128.
-__device__ __forceinline__ uint32_t nibble_pair_bf16(uint32_t w, int i) {
-    const uint32_t biased = ((w >> (4 * i)) & 0x000F000Fu) | 0x43004300u;
-    uint32_t r;
-    asm("sub.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(biased), "r"(0x43004300u));
+// The AND and the OR are ONE three-input logic instruction (look-up table 0xEA = (a & b) | c).
+__device__ __forceinline__ uint32_t nibble_pair_bf16(uint32_t w, int i, uint32_t mask, uint32_t magic) {
+    uint32_t biased, r;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(biased) : "r"(w >> (4 * i)), "r"(mask), "r"(magic));
+    asm("sub.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(biased), "r"(magic));
     return r;
 }
 // The same from two bytes (values up to 127) minus `bias`: bytes `sel` picks from {lo, hi} become the low bytes of the
@@ -401,12 +408,12 @@ __device__ __forceinline__ void tile_compute(const TileIn& t, float (&acc)[4][Mo
         } else {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                a0[i] = nibble_pair_bf16(w0, i);
-                a1[i] = nibble_pair_bf16(w1, i);
+                a0[i] = nibble_pair_bf16(w0, i, lc.nib_mask, lc.nib_magic);
+                a1[i] = nibble_pair_bf16(w1, i, lc.nib_mask, lc.nib_magic);
             }
         }
-        float cc[4] = {0.f, 0.f, 0.f, 0.f};  // (row g+16h, tok 2q), (same row, tok 2q+1), (row g+8+16h, tok 2q), (.., 2q+1)
-        mma_bf16_acc(cc, a0[0], a1[0], a0[1], a1[1], t.b[0], t.b[1]);
+        float cc[4];  // (row g+16h, tok 2q), (same row, tok 2q+1), (row g+8+16h, tok 2q), (.., 2q+1)
+        mma_bf16_zero(cc, a0[0], a1[0], a0[1], a1[1], t.b[0], t.b[1]);
         mma_bf16_acc(cc, a0[2], a1[2], a0[3], a1[3], t.b[2], t.b[3]);
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
@@ -478,8 +485,9 @@ __device__ __noinline__ float piece_exact_token(const ExactPiece e, int lane) {
         const uint32_t raw = e.raw0 + (uint32_t)tile * e.raw_tile_stride;
 #pragma unroll 1
         for (int p4 = 0; p4 < 4; ++p4) {
-            const uint4 xr = lds128(raw + (uint32_t)p4 * e.piece_stride);
-            const uint32_t xw[4] = {xr.x, xr.y, xr.z, xr.w};
+            uint32_t xw[4];  // (the records are 8-byte aligned)
+            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(xw[0]), "=r"(xw[1]) : "r"(raw + (uint32_t)p4 * e.piece_stride));
+            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(xw[2]), "=r"(xw[3]) : "r"(raw + (uint32_t)p4 * e.piece_stride + 8u));
 #pragma unroll
             for (int j = 0; j < 4; ++j) {  // byte j of code word p4: k = 8 p4 + 2j in the low nibble, k + 1 in the high one
                 const uint32_t byte = (cw[p4] >> (8 * j)) & 0xffu;

@@ -20,12 +20,11 @@ constexpr int kColsMaxTokens = 2;
 // Column modes hand three partial terms per (row, token) to the reducer (two column halves + the offset term).
 constexpr int kColsPartTerms = 3;
 // Prepared activations in shared memory (written by xprep_item, read by the tile loop):
-//   column modes (M <= 2): one 160-byte record per (group-tile, token) -- four signed byte planes of the 31-bit fixed
-//   point (4 x 32 bytes), {sum of x, unit} at 128, eight zero bytes at 136 (the B column of a token that does not
-//   exist), and at 144 of token 0's record the sums of x of tokens 0 and 1;
+//   column modes (M <= 2): one 136-byte record per (group-tile, token) -- four signed byte planes of the 31-bit fixed
+//   point (4 x 32 bytes) and {sum of x, unit} at 128;
 //   M >= 3: the bf16 activations themselves in MMA fragment order, 64 bytes per (group-tile, token), and the sums of x
 //   of the (up to eight) tokens, 32 bytes per group-tile.
-constexpr int kColsRecBytes = 160, kColsSumOff = 128, kColsUnitOff = 132, kColsZeroOff = 136, kColsRowSumOff = 144;
+constexpr int kColsRecBytes = 136, kColsSumOff = 128, kColsUnitOff = 132;
 constexpr int kPlaneRecBytes = 64, kPlaneSumBytes = 32;
 constexpr int kMaxSplit = 8;        // K slices
 constexpr int kMaxCtasPerSm = 2;

@@ -16,7 +16,7 @@ PREP_ITEMS = 8 * 16 * 32
 
 
 def plan_step(M, K, N, grid=GRID):
-    rec = 160 if M <= 2 else 64
+    rec = 136 if M <= 2 else 64
     cap = min(XS_CAP // (8 * rec * M), PREP_ITEMS // (8 * M * 4))
     assert cap >= 1
     S, nb = N // 32, -(-K // 256)
@@ -82,7 +82,7 @@ SHAPES = [(2560, 4096), (2048, 2560), (2560, 20480), (10240, 2560), (1152, 6912)
 @pytest.mark.parametrize("K,N", SHAPES)
 def test_chain_step_split(M, K, N):
     p = plan_step(M, K, N)
-    rec = 160 if M <= 2 else 64
+    rec = 136 if M <= 2 else 64
     assert p["nbz"] * 8 * rec * M <= XS_CAP and p["nbz"] * 8 * M * 4 <= PREP_ITEMS
     assert p["Z"] * p["Gz"] <= GRID
     pieces = pieces_of(p)
