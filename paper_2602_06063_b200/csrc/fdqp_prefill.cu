@@ -230,6 +230,15 @@ __device__ __forceinline__ uint32_t pf_prmt(uint32_t a, uint32_t b, uint32_t sel
     return d;
 }
 
+// (x & 0x000F000F) | 0x43004300 as ONE three-input logic instruction (look-up table 0xEA = (a & b) | c): the bf16 pair
+// (128 + nibble 0, 128 + nibble 4) of x; the packed subtraction removes the 128 exactly.
+__device__ __forceinline__ uint32_t pf_nibble_pair(uint32_t x) {
+    uint32_t biased, r;
+    asm("lop3.b32 %0, %1, 0x000F000F, 0x43004300, 0xEA;" : "=r"(biased) : "r"(x));
+    asm("sub.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(biased), "r"(0x43004300u));
+    return r;
+}
+
 template <int FMT>
 __device__ __forceinline__ void group_store(uint32_t a_tile, const GroupRegs& r, int strip_local, int gl, int lane) {
     const int row = strip_local * 32 + lane;
@@ -269,8 +278,7 @@ __device__ __forceinline__ void group_store(uint32_t a_tile, const GroupRegs& r,
         float f[8];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            uint32_t q2 = ((w >> (4 * i)) & 0x000F000Fu) | 0x43004300u;  // bf16x2 (128 + q_i, 128 + q_{i+4})
-            asm("sub.bf16x2 %0, %0, %1;" : "+r"(q2) : "r"(0x43004300u));  // exact: (q_i, q_{i+4})
+            uint32_t q2 = pf_nibble_pair(w >> (4 * i));  // bf16x2 (q_i, q_{i+4}), exact
             f[i] = dequant_lo(q2, r.d_bits, m);
             f[i + 4] = dequant_hi(q2, r.d_bits, m);
         }
@@ -323,8 +331,7 @@ __device__ __forceinline__ void group_convert(const GroupRegs& r, uint32_t (&out
         float f[8];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            uint32_t q2 = ((w >> (4 * i)) & 0x000F000Fu) | 0x43004300u;
-            asm("sub.bf16x2 %0, %0, %1;" : "+r"(q2) : "r"(0x43004300u));
+            const uint32_t q2 = pf_nibble_pair(w >> (4 * i));
             f[i] = dequant_lo(q2, r.d_bits, m);
             f[i + 4] = dequant_hi(q2, r.d_bits, m);
         }
