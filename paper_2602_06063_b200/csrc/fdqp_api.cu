@@ -879,9 +879,16 @@ extern "C" fdqp_status fdqp_run_chain(fdqp_ctx* ctx, const fdqp_chain_step* step
             int64_t Gz = grid / Z;
             if (Gz > (int64_t)c.S * len_last) Gz = (int64_t)c.S * len_last;
             if (Gz < 1) Gz = 1;
-            // whole strips per CTA when that costs at most 3 % of imbalance (nothing is exchanged between CTAs then)
+            // whole strips per CTA when that costs at most 3 % of imbalance (nothing is exchanged between CTAs then) --
+            // or, for a step another one waits on, when the extra blocks of the busiest CTA (0.125 us each) cost less
+            // than the exchange of shared strips that the waiting step would have to sit out (about 2 us)
             c.strip_aligned = 0;
-            if (c.S >= Gz && (double)((c.S + Gz - 1) / Gz) * (double)Gz <= 1.03 * (double)c.S) c.strip_aligned = 1;
+            if (c.S >= Gz) {
+                const int64_t per = (c.S + Gz - 1) / Gz;
+                const double extra_blocks = ((double)per - (double)c.S / (double)Gz) * (double)c.nbz;
+                const bool waited_on = first + i + 1 < n_steps && steps[first + i + 1].depends_on_previous != 0;
+                if ((double)per * (double)Gz <= 1.03 * (double)c.S || (waited_on && extra_blocks * 0.125 < 2.0)) c.strip_aligned = 1;
+            }
             if (ctx->p_aligned >= 0 && (ctx->p_aligned == 0 || c.S >= Gz)) c.strip_aligned = ctx->p_aligned != 0;
             c.Gz = (int)Gz;
             c.wait_prev = (u.depends_on_previous && i > 0) ? 1 : 0;  // across launches the stream order is the dependency

@@ -325,12 +325,27 @@ __global__ void __launch_bounds__(kThreads, 1) fdqp_chain_kernel(const __grid_co
                 const int kbeg = g.b_first * kBlockK;
                 const int kend_full = (g.b_first + g.len) * kBlockK;
                 const int ntiles_all = ((kend_full < K ? kend_full : K) - kbeg) / kGroup;
-                // A range inside ONE strip touches only its own blocks' share of x (a long-K projection cut over many
-                // CTAs); the normalisation needs the whole row.
-                const bool part_k = g.npieces == 1 && !(EPI && st.norm);
-                const int tile_lo = part_k ? g.bl_first * 8 : 0;
-                const int tile_hi = part_k ? ((g.bl_first + g.nblk) * 8 < ntiles_all ? (g.bl_first + g.nblk) * 8 : ntiles_all) : ntiles_all;
-                const int tile0 = kbeg / kGroup + tile_lo, ntiles = tile_hi - tile_lo;
+                // A range inside one strip, or in the end of one strip and the beginning of the next, touches only its own
+                // blocks' share of x (a long-K projection cut over many CTAs): up to two tile ranges [lo1, hi1), [lo2, hi2).
+                // The normalisation needs the whole row.
+                int lo1 = 0, hi1 = ntiles_all, lo2 = 0, hi2 = 0;
+                if (!(EPI && st.norm)) {
+                    if (g.npieces == 1) {
+                        lo1 = g.bl_first * 8;
+                        hi1 = (g.bl_first + g.nblk) * 8;
+                    } else if (g.npieces == 2 && g.nblk - (g.len - g.bl_first) <= g.bl_first) {
+                        hi1 = (g.nblk - (g.len - g.bl_first)) * 8;  // the second strip's first blocks
+                        lo2 = g.bl_first * 8;                        // the first strip's last blocks
+                        hi2 = g.len * 8;
+                    }
+                    hi1 = hi1 < ntiles_all ? hi1 : ntiles_all;
+                    hi2 = hi2 < ntiles_all ? hi2 : ntiles_all;
+                    if (hi2 < lo2) hi2 = lo2;
+                }
+                const int n1 = hi1 - lo1, ntiles = n1 + (hi2 - lo2);
+                // tile (relative to the K slice) of the t-th tile prepared
+                auto tile_rel = [&](int t) { return t < n1 ? lo1 + t : lo2 + (t - n1); };
+                const int tile0 = kbeg / kGroup;
                 const int items = ntiles * M * 4;  // <= kPrepBatch * kCW * 32 (the plan guarantees it)
                 uint32_t* xs_g = reinterpret_cast<uint32_t*>(smem + cp.off_xs);
                 float* xsc_g = reinterpret_cast<float*>(smem + cp.off_xsum);
@@ -340,7 +355,7 @@ __global__ void __launch_bounds__(kThreads, 1) fdqp_chain_kernel(const __grid_co
                     const int idx = u * kCW * 32 + tid;
                     v[u] = make_uint4(0, 0, 0, 0);
                     if (idx < items) {
-                        const int tm = idx >> 2, tile = tile0 + tm / M, tok = tm % M, qq = idx & 3;
+                        const int tm = idx >> 2, tile = tile0 + tile_rel(tm / M), tok = tm % M, qq = idx & 3;
                         v[u] = ldcg128(st.x + (int64_t)tok * K + tile * kGroup + qq * 8);
                     }
                 }
@@ -407,7 +422,7 @@ __global__ void __launch_bounds__(kThreads, 1) fdqp_chain_kernel(const __grid_co
                     if (u * kCW * 32 < items) {  // warp-uniform: whole quads run the shuffles together
                         const bool valid = idx < items;
                         const int tm = idx >> 2;
-                        if (xprep_item<MT::kCols>(v[u], M, tile_lo + (valid ? tm / M : 0), valid ? tm % M : 0, idx & 3, valid, xs_g, xsc_g))
+                        if (xprep_item<MT::kCols>(v[u], M, valid ? tile_rel(tm / M) : 0, valid ? tm % M : 0, idx & 3, valid, xs_g, xsc_g))
                             saw_flagged = true;
                     }
                 }

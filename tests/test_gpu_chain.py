@@ -220,3 +220,34 @@ def test_chain_argument_errors(fresh):
     assert lib.fdqp_run_chain(fresh, None, 1, 1, s) == 1
     torch.cuda.synchronize()
     assert fd.fdqp_last_status(fresh) == 0
+
+
+@pytest.mark.parametrize("M", [1, 4])
+def test_chain_through_two_layers_and_the_full_size_lm_head(M):
+    """Nine steps in one launch at BASELINE sizes: the four calls of a Gemma3-4B layer twice (seeded weights of two
+    different layers) and the tied LM head (K = 2560, N = 262144, seed 17).  Every output of the layer calls and a
+    sample of strips spread over the LM head's outputs are checked against the oracle."""
+    _, hk, hn, hseed = synthgen.GEMMA3_4B_LM_HEAD
+    ctx = fd.fdqp_create(0, 8, 10240, hn)
+    try:
+        shapes = [(2560, 4096), (2048, 2560), (2560, 20480), (10240, 2560)]
+        cases = [Case(K, N, M, seed=7700 + 10 * layer + j) for layer in range(2) for j, (K, N) in enumerate(shapes)]
+        head = Case(hk, hn, M, hseed)
+        outs = [torch.full((M, c.N), float("nan"), dtype=torch.float32, device="cuda") for c in cases + [head]]
+        steps = [fd.chain_step(c.x_dev, c.W_dev, o, c.K, c.N) for c, o in zip(cases + [head], outs)]
+        before = fd.fdqp_launch_count(ctx)
+        fd.fdqp_run_chain(ctx, steps, M)
+        torch.cuda.synchronize()
+        assert fd.fdqp_last_status(ctx) == 0
+        assert fd.fdqp_launch_count(ctx) - before == 1
+        for c, o in zip(cases, outs):
+            y_ref, a_ref = c.reference()
+            assert_close(o.cpu().numpy(), y_ref, a_ref, f"layer call K={c.K} N={c.N} M={M}")
+        y = outs[-1].cpu().numpy()
+        assert np.all(np.isfinite(y))
+        for n0 in (0, 4096, 99968, 131072 - 64, 200000 - 200000 % 32, hn - 128):
+            y_ref, a_ref = head.reference(n0=n0, n1=n0 + 128)
+            assert_close(y[:, n0:n0 + 128], y_ref, a_ref, f"LM head columns {n0}.. M={M}")
+    finally:
+        torch.cuda.synchronize()
+        fd.fdqp_destroy(ctx)
