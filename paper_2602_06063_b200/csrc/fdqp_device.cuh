@@ -54,13 +54,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
+// The same test, but the thread may stay suspended for up to about a microsecond (it resumes at once when the phase
+// completes): a waiting warp then spends few issue slots on polling.
+__device__ __forceinline__ bool mbar_try_wait_suspended(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(1000u)
+        : "memory");
+    return ok != 0;
+}
+
 // Bounded wait on a phase parity.  Returns false (after recording the timeout in *status) if
 // the barrier did not flip within `limit_ns`.
 __device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, int* status, unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = globaltimer_ns();
     for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_suspended(bar, parity)) return true;
         if ((it & 63u) == 0u && globaltimer_ns() - t0 > limit_ns) {
             atomicExch(status, kStatusTimeout);
             __threadfence_system();

@@ -260,6 +260,12 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
         };
         bool any_flagged = false;  // set once x is prepared: some group of the K slice takes the fp32 path
 
+        // where this lane's partial sums go in the reducer's buffer (parity 0; parity 1 lies part_par_bytes further)
+        constexpr int PT = MT::kCols ? kColsPartTerms : 1;
+        const uint32_t part_par_bytes = (uint32_t)(CW * PT * kStripRows * M) * 4u;
+        const uint32_t part_warp = part + (uint32_t)(warp * PT * kStripRows * M) * 4u;
+        const uint32_t st_acc = part_warp + (uint32_t)(MT::kCols ? ((q & 1) * M + (q >> 1)) * kStripRows + g : 2 * q * kStripRows + g) * 4u;
+        const uint32_t st_m = part_warp + (uint32_t)(2 * M * kStripRows + lane) * 4u;
         int piece = 0;
         bool alive = true;
         // hand the warp's partial rows of the current strip piece to the reducer warp
@@ -294,23 +300,18 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             }
             const int par = piece & 1;
             if (piece >= 2 && !mbar_wait(red_empty0 + 8u * par, ((piece >> 1) - 1) & 1, p.status)) alive = false;
-            constexpr int PT = MT::kCols ? kColsPartTerms : 1;
-            const uint32_t slot = part + (uint32_t)((par * CW + warp) * PT * kStripRows * M) * 4u;
+            const uint32_t pslot = par ? part_par_bytes : 0u;
             if (MT::kCols) {
                 // Lanes q and q^1 hold the two column halves of each row's sum for token q/2, lane r holds row r's
                 // offset terms: all three go to the reducer as they are ([term][token][row]); it adds them.
-                const int tok = q >> 1;
-                if (tok < M) {
+                if ((q >> 1) < M) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
-                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(slot + (uint32_t)((((q & 1) * M + tok) * kStripRows) + g + 8 * i) * 4u),
-                                     "f"(acc[i][0])
-                                     : "memory");
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(st_acc + pslot + 32u * i), "f"(acc[i][0]) : "memory");
                 }
 #pragma unroll
                 for (int tk = 0; tk < MT::kAccM; ++tk) {
-                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(slot + (uint32_t)((2 * M + tk) * kStripRows + lane) * 4u), "f"(acc_m[tk])
-                                 : "memory");
+                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(st_m + pslot + (uint32_t)(tk * kStripRows * 4)), "f"(acc_m[tk]) : "memory");
                     acc_m[tk] = 0.f;
                 }
 #pragma unroll
@@ -320,10 +321,8 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                 for (int i = 0; i < 4; ++i)
 #pragma unroll
                     for (int j = 0; j < NT; ++j) {
-                        const int tok = 2 * q + j;
-                        if (tok < M)
-                            asm volatile("st.shared.f32 [%0], %1;" ::"r"(slot + (uint32_t)(tok * kStripRows + g + 8 * i) * 4u),
-                                         "f"(acc[i][j])
+                        if (2 * q + j < M)
+                            asm volatile("st.shared.f32 [%0], %1;" ::"r"(st_acc + pslot + (uint32_t)((j * kStripRows + 8 * i) * 4)), "f"(acc[i][j])
                                          : "memory");
                         acc[i][j] = 0.f;
                     }
@@ -461,27 +460,46 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
                 // before it, the hand-off of the finished strip piece, the blocks after it -- two tiles in flight
                 // wherever two neighbours are on the same side
                 const int pb = unit_next - i0;  // first block of the next strip piece, 1 .. BPW - 1
-#pragma unroll 1
-                for (int jj = 0; jj < BPW;) {
-                    if (jj == pb) {
-                        flush();
-                        next_unit();
-                        lim = interior_limit();
-                    }
+                auto one = [&](int jj) {
+                    const uint32_t sb = sbase + jj * kBB;
+                    TileIn ta;
+                    tile_load<MODE, FMT>(ta, sb + code_lane, sb + so_full, sb + m_full, (i0 + jj - unit_first) * 8 + tw, la);
+                    tile_compute<MODE, FMT>(ta, acc, acc_m, lc);
+                };
+                auto two = [&](int jj) {
                     const uint32_t sb = sbase + jj * kBB;
                     const int tile = (i0 + jj - unit_first) * 8 + tw;
-                    TileIn ta;
+                    TileIn ta, tb;
                     tile_load<MODE, FMT>(ta, sb + code_lane, sb + so_full, sb + m_full, tile, la);
-                    if (jj + 1 < BPW && jj + 1 != pb) {
-                        TileIn tb;
-                        tile_load<MODE, FMT>(tb, sb + kBB + code_lane, sb + kBB + so_full, sb + kBB + m_full, tile + 8, la);
-                        tile_compute<MODE, FMT>(ta, acc, acc_m, lc);
-                        tile_compute<MODE, FMT>(tb, acc, acc_m, lc);
-                        jj += 2;
+                    tile_load<MODE, FMT>(tb, sb + kBB + code_lane, sb + kBB + so_full, sb + kBB + m_full, tile + 8, la);
+                    tile_compute<MODE, FMT>(ta, acc, acc_m, lc);
+                    tile_compute<MODE, FMT>(tb, acc, acc_m, lc);
+                };
+                auto hand_over = [&]() {
+                    flush();
+                    next_unit();
+                    lim = interior_limit();
+                };
+                if (BPW == 4) {
+                    if (pb == 2) {
+                        two(0);
+                        hand_over();
+                        two(2);
+                    } else if (pb == 1) {
+                        one(0);
+                        hand_over();
+                        two(1);
+                        one(3);
                     } else {
-                        tile_compute<MODE, FMT>(ta, acc, acc_m, lc);
-                        jj += 1;
+                        two(0);
+                        one(2);
+                        hand_over();
+                        one(3);
                     }
+                } else {  // two blocks per warp: the boundary is between them
+                    one(0);
+                    hand_over();
+                    one(1);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8u * stage);
