@@ -359,6 +359,9 @@ def run_flowkv(args):
     torch.cuda.set_device(0)
     peaks, peak_kind = measured_peaks()
     ctx = fd.fdqp_create(0, 8, 256, 256)
+    for kv in args.param or []:
+        k, v = kv.split("=")
+        fd.fdqp_set_param(ctx, k, int(v))
     n = window if 0 < window < L else L
     cache_bytes = 2 * G * L * d * 2
     ncopies = max(1, int(np.ceil(4 * L2_BYTES / cache_bytes)))

@@ -257,7 +257,9 @@ FDQP_API fdqp_status fdqp_run_add_rmsnorm_epilogue(fdqp_ctx* ctx, const void* x_
  * over positions j = 0 .. L-1, or only the last `window` of them (window > 0 and
  * < L: sliding-window attention); evaluated chunk by chunk with a running maximum
  * and a running sum, K and V each read once.  (The paper's equation for the
- * decoding step omits the scale; it is an argument here.)
+ * decoding step omits the scale; it is an argument here.)  Short ranges (a sliding
+ * window, a young cache; see the "flowkv_cluster" parameter) are one kernel
+ * launch, longer ones two.
  *   q_bf16  device, [H][d] bf16
  *   K_bf16, V_bf16  device, [G][pitch][d] bf16: position j of KV head g at
  *           (g * pitch + j) * d; pitch >= L is the cache's capacity in positions
@@ -430,6 +432,9 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "chain_steps"   fdqp_run_chain: most steps per launch (1 .. 64, default 64)
  *   "chain_wide"    fdqp_run_chain: 1 (default) = a launch none of whose steps depends on another is cut into CTA ranges
  *                   as one sequence of blocks, 0 = every step is cut on its own
+ *   "flowkv_cluster" fdqp_flowkv_decode: ranges of up to this many positions (default 2048; 0 = never) run as ONE launch,
+ *                   the splits of a KV head as a thread-block cluster merged through distributed shared memory;
+ *                   longer ranges take the two-launch route (split kernel + merge kernel)
  *   "prefill_split_k" 1..8 K slices for the tensor-core kernels (their partial results are added by a second
  *                   kernel); default: as many as fill the SMs when a shape has few output tiles
  *   "prefill_pair"  1 = prefill-sized calls use the two-SM kernel (256 x 512 tile per CTA pair), 0 = the one-SM kernel

@@ -29,7 +29,8 @@ cudaError_t prefill_launch(const uint8_t* W, const uint16_t* x, int64_t x_row_by
 cudaError_t rmsnorm_launch(const uint16_t* x, const uint16_t* residual, uint16_t* h_out, const uint16_t* gamma, float eps,
                            uint16_t* out, int M, int K, cudaStream_t stream);
 cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* V, float* out, float* ws, int max_splits, int H,
-                          int G, int d, int L, int pitch, int window, float scale, int sm_count, cudaStream_t stream);
+                          int G, int d, int L, int pitch, int window, float scale, int sm_count, int cluster_max_positions,
+                          int* launches, cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
 cudaError_t wait_selftest_launch(int* status, unsigned long long limit_ns, cudaStream_t stream);
 cudaError_t chain_set_smem_limit(int bytes);
@@ -37,6 +38,8 @@ cudaError_t chain_launch(const ChainPlan& cp, int grid, bool epi, int launch_mod
 }  // namespace fdqp
 
 using namespace fdqp;
+
+constexpr int kFlowKvClusterPositions = 2048;  // default of the "flowkv_cluster" parameter
 
 struct fdqp_ctx {
     int device = 0;
@@ -69,6 +72,7 @@ struct fdqp_ctx {
     int* chain_done = nullptr;
     size_t chain_ticket_cap = 0;
     int64_t p_chain_launch = 1, p_chain_steps = kMaxChainSteps, p_chain_wide = 1;
+    int64_t p_flowkv_cluster = kFlowKvClusterPositions;  // ranges up to this many positions take the one-launch attention
     int64_t p_direct_y = 1;  // fdqp_run_host*: small results are stored straight into device-addressable host memory
     int64_t p_atmem = 1;  // tensor-core kernel up to 128 tokens: keep the converted weights in tensor memory
 };
@@ -574,12 +578,13 @@ extern "C" fdqp_status fdqp_flowkv_decode(fdqp_ctx* ctx, const void* q_bf16, con
     if (!aligned16(q_bf16) || !aligned16(K_bf16) || !aligned16(V_bf16) || !aligned16(out)) return FDQP_ERR_ALIGN;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FDQP_ERR_CUDA;
+    int launches = 0;
     const cudaError_t e = flowkv_launch(static_cast<const uint16_t*>(q_bf16), static_cast<const uint16_t*>(K_bf16),
                                         static_cast<const uint16_t*>(V_bf16), out, ctx->kv_ws, kKvMaxSplits, (int)H, (int)G, (int)d,
-                                        (int)L, (int)pitch, (int)window, scale, ctx->sm_count,
-                                        static_cast<cudaStream_t>(cuda_stream));
+                                        (int)L, (int)pitch, (int)window, scale, ctx->sm_count, (int)ctx->p_flowkv_cluster,
+                                        &launches, static_cast<cudaStream_t>(cuda_stream));
     if (e) return cuda_fail(ctx, e, "decode attention launch");
-    ctx->launches += 2;
+    ctx->launches += launches;
     return FDQP_OK;
 }
 
@@ -737,6 +742,9 @@ extern "C" fdqp_status fdqp_set_param(fdqp_ctx* ctx, const char* key, int64_t va
     } else if (!std::strcmp(key, "chain_launch")) {
         if (v > 3) return FDQP_ERR_ARG;
         ctx->p_chain_launch = v < 0 ? 1 : v;
+    } else if (!std::strcmp(key, "flowkv_cluster")) {
+        if (v > (int64_t)1 << 20) return FDQP_ERR_ARG;
+        ctx->p_flowkv_cluster = v < 0 ? kFlowKvClusterPositions : v;
     } else if (!std::strcmp(key, "chain_wide")) {
         if (v > 1) return FDQP_ERR_ARG;
         ctx->p_chain_wide = v < 0 ? 1 : v;

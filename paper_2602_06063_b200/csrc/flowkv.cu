@@ -14,6 +14,9 @@
 //   - O^T[d][8 heads] += V_tile^T (d x 16, ldmatrix.trans) . P (16 x 8), fp32 accumulators in registers;
 //   - the four warps' (m, l, O) are merged through shared memory and written as one partial per (split, head);
 //     flowkv_merge_kernel combines the splits' partials in split order and normalises.
+//   - short ranges (a sliding window, a young cache) are one launch: the splits of a KV head form a thread-block cluster
+//     of up to 16 CTAs, every CTA leaves its partial in its own shared memory and, after a cluster barrier, each CTA
+//     combines one slice of the head's outputs across all partials through distributed shared memory, in split order.
 // Each cache byte is read once.  Everything is deterministic (fixed merge orders).
 #include "fdqp_device.cuh"
 
@@ -25,12 +28,14 @@ constexpr int kKvStages = 3;
 constexpr int kKvMaxGroup = 8;  // query heads per KV head
 constexpr int kKvMergeThreads = 1024;
 constexpr int kKvMaxSplitsDev = 160;  // upper bound of the split count the merge kernel handles (a multiple of 32)
+constexpr int kKvMaxCluster = 16;     // splits of the one-launch variant: one thread-block cluster per KV head
 
 struct FlowKvParams {
     const uint16_t* q;  // [H][d]
     const uint16_t* K;  // [G][pitch][d]
     const uint16_t* V;
     float* ws;          // [H][splits][d + 4]: partial O (unnormalised), running maximum, running sum, 2 unused
+    float* out;         // [H][d]: written by the one-launch variant only
     int H, G, L, pitch;
     int j0;             // first position attended to (0, or L - window)
     int chunk;          // positions per split (a multiple of kKvWarps * kKvTile)
@@ -54,7 +59,21 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return r;
 }
 
-template <int D>
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// a float of CTA `rank`'s shared memory, at the address `local` has in this CTA's
+__device__ __forceinline__ float ld_cluster_f32(uint32_t local, uint32_t rank) {
+    uint32_t remote;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+
+// CLUSTER: the grid's x dimension is one cluster (splits <= kKvMaxCluster); the kernel writes `out` itself.
+template <int D, bool CLUSTER>
 __global__ void __launch_bounds__(kKvWarps * 32, 1) flowkv_decode_kernel(const FlowKvParams p) {
     constexpr int kRowBytes = D * 2;
     constexpr int kChunksPerRow = kRowBytes / 16;            // 32 (d = 256) or 16 (d = 128)
@@ -77,19 +96,6 @@ __global__ void __launch_bounds__(kKvWarps * 32, 1) flowkv_decode_kernel(const F
     const uint8_t* Kg = reinterpret_cast<const uint8_t*>(p.K) + (size_t)kvh * p.pitch * kRowBytes;
     const uint8_t* Vg = reinterpret_cast<const uint8_t*>(p.V) + (size_t)kvh * p.pitch * kRowBytes;
     const uint32_t ring = smem_u32(smem) + warp * (kKvStages * kStageBytes);
-
-    // ---- Q^T as B fragments: lane (g4, q4) holds head g4, dims 16 kk + 2 q4 (+1) and + 8 (+9)
-    uint32_t qf[D / 16][2];
-    {
-        const uint16_t* qh = p.q + (size_t)(kvh * R + (g4 < R ? g4 : 0)) * D;
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t lo = *reinterpret_cast<const uint32_t*>(qh + kk * 16 + 2 * q4);
-            const uint32_t hi = *reinterpret_cast<const uint32_t*>(qh + kk * 16 + 2 * q4 + 8);
-            qf[kk][0] = g4 < R ? lo : 0u;
-            qf[kk][1] = g4 < R ? hi : 0u;
-        }
-    }
 
     // the copies of tile t (this warp's t-th tile) into ring stage t % kKvStages
     auto issue = [&](int t) {
@@ -117,6 +123,20 @@ __global__ void __launch_bounds__(kKvWarps * 32, 1) flowkv_decode_kernel(const F
 
 #pragma unroll
     for (int t = 0; t < kKvStages - 1; ++t) issue(t);
+
+    // ---- Q^T as B fragments (loaded while the first tiles are on their way): lane (g4, q4) holds head g4, dims 16 kk + 2 q4 (+1) and + 8 (+9)
+    uint32_t qf[D / 16][2];
+    {
+        const uint16_t* qh = p.q + (size_t)(kvh * R + (g4 < R ? g4 : 0)) * D;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t lo = *reinterpret_cast<const uint32_t*>(qh + kk * 16 + 2 * q4);
+            const uint32_t hi = *reinterpret_cast<const uint32_t*>(qh + kk * 16 + 2 * q4 + 8);
+            qf[kk][0] = g4 < R ? lo : 0u;
+            qf[kk][1] = g4 < R ? hi : 0u;
+        }
+    }
+
 
     // ldmatrix source rows/chunks of this lane: matrix mi = lane / 8
     const int mi = lane >> 3, r8 = lane & 7;
@@ -220,6 +240,9 @@ __global__ void __launch_bounds__(kKvWarps * 32, 1) flowkv_decode_kernel(const F
         base[D + g4 + 8] = o[dt][3];
     }
     __syncthreads();
+    // this CTA's partial: to the workspace, or (one-launch variant) to shared memory behind the warps' partials
+    float* cl_o = stats + kKvWarps * kKvMaxGroup * 2;  // [R][D]
+    float* cl_st = cl_o + kKvMaxGroup * D;             // [R][2]: running maximum, running sum
     for (int idx = tid; idx < R * D; idx += kKvWarps * 32) {
         const int h = idx / D, i = idx % D;
         float m = -INFINITY;
@@ -233,12 +256,49 @@ __global__ void __launch_bounds__(kKvWarps * 32, 1) flowkv_decode_kernel(const F
             acc += part[(size_t)(w * kKvMaxGroup + h) * D + i] * f;
             l += stats[(w * kKvMaxGroup + h) * 2 + 1] * f;
         }
-        float* dst = p.ws + ((size_t)(kvh * R + h) * p.splits + split) * (D + 4);
-        dst[i] = acc;
-        if (i == 0) {
-            dst[D] = m;
-            dst[D + 1] = l;
+        if (CLUSTER) {
+            cl_o[idx] = acc;
+            if (i == 0) {
+                cl_st[h * 2] = m;
+                cl_st[h * 2 + 1] = l;
+            }
+        } else {
+            float* dst = p.ws + ((size_t)(kvh * R + h) * p.splits + split) * (D + 4);
+            dst[i] = acc;
+            if (i == 0) {
+                dst[D] = m;
+                dst[D + 1] = l;
+            }
         }
+    }
+    if (CLUSTER) {
+        // every CTA of the cluster has its partial in place; CTA `split` combines outputs split, split + S, ... of the
+        // head group (a thread per output) over all S partials in split order and normalises
+        cluster_sync();
+        const int S = p.splits;
+        const uint32_t o_addr = smem_u32(cl_o), st_addr = smem_u32(cl_st);
+        for (int idx = split * (kKvWarps * 32) + tid; idx < R * D; idx += S * (kKvWarps * 32)) {
+            const int h = idx / D;
+            float ms[kKvMaxCluster], ls[kKvMaxCluster], os[kKvMaxCluster];
+            float m = -INFINITY;
+#pragma unroll
+            for (int s2 = 0; s2 < kKvMaxCluster; ++s2) {
+                const bool on = s2 < S;
+                ms[s2] = on ? ld_cluster_f32(st_addr + (uint32_t)(h * 8), (uint32_t)s2) : -INFINITY;
+                ls[s2] = on ? ld_cluster_f32(st_addr + (uint32_t)(h * 8 + 4), (uint32_t)s2) : 0.f;
+                os[s2] = on ? ld_cluster_f32(o_addr + (uint32_t)idx * 4u, (uint32_t)s2) : 0.f;
+                m = fmaxf(m, ms[s2]);
+            }
+            float acc = 0.f, l = 0.f;
+#pragma unroll
+            for (int s2 = 0; s2 < kKvMaxCluster; ++s2) {
+                const float f = ms[s2] == -INFINITY ? 0.f : exp2f(ms[s2] - m);
+                acc += os[s2] * f;
+                l += ls[s2] * f;
+            }
+            p.out[(size_t)kvh * R * D + idx] = acc / l;
+        }
+        cluster_sync();  // nobody leaves while its shared memory may still be read
     }
 }
 
@@ -312,14 +372,19 @@ __global__ void __launch_bounds__(kKvMergeThreads) flowkv_merge_kernel(const flo
 // ---- host side ------------------------------------------------------------------------------------------------------
 
 template <int D>
-static cudaError_t flowkv_launch_d(const FlowKvParams& p, float* out, cudaStream_t stream) {
+constexpr int flowkv_smem_bytes() {
     constexpr int kRing = kKvWarps * kKvStages * 2 * kKvTile * D * 2;
-    constexpr int kMerge = (kKvWarps * kKvMaxGroup * D + kKvWarps * kKvMaxGroup * 2) * 4;
-    constexpr int kSmem = kRing > kMerge ? kRing : kMerge;
+    constexpr int kMerge = (kKvWarps * kKvMaxGroup * D + kKvWarps * kKvMaxGroup * 2 + kKvMaxGroup * D + kKvMaxGroup * 2) * 4;
+    return kRing > kMerge ? kRing : kMerge;
+}
+
+template <int D>
+static cudaError_t flowkv_launch_d(const FlowKvParams& p, float* out, cudaStream_t stream) {
+    constexpr int kSmem = flowkv_smem_bytes<D>();
     static bool attr_set = false;  // per process; the attribute is per device function
     cudaError_t e;
     if (!attr_set) {
-        if ((e = cudaFuncSetAttribute(flowkv_decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem))) return e;
+        if ((e = cudaFuncSetAttribute(flowkv_decode_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem))) return e;
         attr_set = true;
     }
     cudaLaunchAttribute attr;
@@ -332,7 +397,7 @@ static cudaError_t flowkv_launch_d(const FlowKvParams& p, float* out, cudaStream
     cfg.stream = stream;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    if ((e = cudaLaunchKernelEx(&cfg, flowkv_decode_kernel<D>, p))) return e;
+    if ((e = cudaLaunchKernelEx(&cfg, flowkv_decode_kernel<D, false>, p))) return e;
     cfg.gridDim = dim3((unsigned)p.H);
     cfg.blockDim = dim3(kKvMergeThreads);
     cfg.dynamicSmemBytes = 0;
@@ -341,14 +406,76 @@ static cudaError_t flowkv_launch_d(const FlowKvParams& p, float* out, cudaStream
     return cudaLaunchKernelEx(&cfg, flowkv_merge_kernel<D>, ws, out, splits);
 }
 
+// The one-launch variant: grid (S, G) in clusters of S CTAs.  `*usable` is set to the number of such clusters the
+// device can hold at once (0: this cluster size cannot be launched here; the caller then takes the two-launch route).
+template <int D>
+static cudaError_t flowkv_cluster_config(int S, cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attrs) {
+    constexpr int kSmem = flowkv_smem_bytes<D>();
+    static bool attr_set = false;
+    cudaError_t e;
+    if (!attr_set) {
+        if ((e = cudaFuncSetAttribute(flowkv_decode_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem))) return e;
+        if ((e = cudaFuncSetAttribute(flowkv_decode_kernel<D, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1))) return e;
+        attr_set = true;
+    }
+    attrs[0].id = cudaLaunchAttributeClusterDimension;
+    attrs[0].val.clusterDim.x = (unsigned)S;
+    attrs[0].val.clusterDim.y = 1;
+    attrs[0].val.clusterDim.z = 1;
+    attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[1].val.programmaticStreamSerializationAllowed = 1;
+    *cfg = cudaLaunchConfig_t{};
+    cfg->blockDim = dim3(kKvWarps * 32);
+    cfg->dynamicSmemBytes = kSmem;
+    cfg->attrs = attrs;
+    cfg->numAttrs = 2;
+    return cudaSuccess;
+}
+
+template <int D>
+static cudaError_t flowkv_cluster_usable(int S, int G, int* usable) {
+    static int cached[kKvMaxCluster + 1];  // 0: not asked yet; else 1 + the number of co-resident clusters
+    if (!cached[S]) {
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attrs[2];
+        cudaError_t e = flowkv_cluster_config<D>(S, &cfg, attrs);
+        if (e) return e;
+        cfg.gridDim = dim3((unsigned)S, (unsigned)G);
+        cfg.numAttrs = 1;  // the cluster shape alone
+        int n = 0;
+        e = cudaOccupancyMaxActiveClusters(&n, flowkv_decode_kernel<D, true>, &cfg);
+        if (e) {
+            (void)cudaGetLastError();
+            n = 0;
+        }
+        cached[S] = 1 + n;
+    }
+    *usable = cached[S] - 1;
+    return cudaSuccess;
+}
+
+template <int D>
+static cudaError_t flowkv_launch_cluster_d(const FlowKvParams& p, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attrs[2];
+    cudaError_t e = flowkv_cluster_config<D>(p.splits, &cfg, attrs);
+    if (e) return e;
+    cfg.gridDim = dim3((unsigned)p.splits, (unsigned)p.G);
+    cfg.stream = stream;
+    return cudaLaunchKernelEx(&cfg, flowkv_decode_kernel<D, true>, p);
+}
+
 // ws must hold H * max_splits * (d + 4) floats; max_splits <= kKvMaxSplitsDev.
 cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* V, float* out, float* ws, int max_splits, int H,
-                          int G, int d, int L, int pitch, int window, float scale, int sm_count, cudaStream_t stream) {
+                          int G, int d, int L, int pitch, int window, float scale, int sm_count, int cluster_max_positions,
+                          int* launches, cudaStream_t stream) {
+    if (d != 128 && d != 256) return cudaErrorInvalidValue;
     FlowKvParams p;
     p.q = q;
     p.K = K;
     p.V = V;
     p.ws = ws;
+    p.out = out;
     p.H = H;
     p.G = G;
     p.L = L;
@@ -356,6 +483,21 @@ cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* 
     p.j0 = (window > 0 && window < L) ? L - window : 0;
     const int n = L - p.j0;
     const int gran = kKvWarps * kKvTile;
+    p.scale_log2e = scale * 1.4426950408889634f;
+    if (n <= cluster_max_positions) {
+        // one launch: S splits (a power of two, at most 16) of equal length, one cluster per KV head
+        int S = 1;
+        while (S < kKvMaxCluster && S * gran < n) S *= 2;
+        int usable = 0;
+        cudaError_t e = d == 256 ? flowkv_cluster_usable<256>(S, G, &usable) : flowkv_cluster_usable<128>(S, G, &usable);
+        if (e) return e;
+        if (usable >= 1) {
+            p.splits = S;
+            p.chunk = ((n + S - 1) / S + gran - 1) / gran * gran;
+            *launches = 1;
+            return d == 256 ? flowkv_launch_cluster_d<256>(p, stream) : flowkv_launch_cluster_d<128>(p, stream);
+        }
+    }
     // CTAs over all KV heads: as many as are resident at once (one per SM at d = 256, whose rings take 192 KB; two at
     // d = 128), never more -- a CTA that has to wait for a free SM would double the time.
     const int resident = sm_count * (d == 128 ? 2 : 1);
@@ -366,10 +508,9 @@ cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* 
     p.chunk = chunk;
     p.splits = (n + chunk - 1) / chunk;
     if (p.splits > kKvMaxSplitsDev) return cudaErrorInvalidValue;
-    p.scale_log2e = scale * 1.4426950408889634f;
+    *launches = 2;
     if (d == 256) return flowkv_launch_d<256>(p, out, stream);
-    if (d == 128) return flowkv_launch_d<128>(p, out, stream);
-    return cudaErrorInvalidValue;
+    return flowkv_launch_d<128>(p, out, stream);
 }
 
 }  // namespace fdqp

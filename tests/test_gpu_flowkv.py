@@ -88,6 +88,29 @@ def test_full_size_caches(ctx, H, G, d, L, window):
     assert not bad.any(), f"{bad.sum()} of {bad.size} outside the bound; worst {(err / (absw + 1e-30)).max():.2e}"
 
 
+@pytest.mark.parametrize("H,G,d,L,window", [(8, 4, 256, 5000, 1024), (8, 4, 256, 1024, 0), (8, 4, 256, 2048, 0), (8, 4, 256, 65, 0),
+                                            (32, 16, 128, 777, 0), (16, 2, 128, 3001, 512), (7, 1, 256, 1500, 0), (8, 1, 128, 1, 0)])
+def test_one_launch_and_two_launch_routes(ctx, H, G, d, L, window):
+    """Short ranges run as one launch (a cluster per KV head merges its splits through distributed shared memory), or,
+    with the "flowkv_cluster" parameter at 0, as the split kernel and the merge kernel; both within the bound."""
+    q, K, V = make(7600 + L + H, H, G, d, L)
+    scale = d ** -0.5
+    ref, absw = oracle.decode_attention(q, K, V, L, window, scale)
+    outs = []
+    try:
+        for limit in (-1, 0, 1 << 20):
+            fd.fdqp_set_param(ctx, "flowkv_cluster", limit)
+            before = fd.fdqp_launch_count(ctx)
+            out = run(ctx, q, K, V, L, window, scale)
+            n = fd.fdqp_launch_count(ctx) - before
+            assert n == (2 if limit == 0 else 1)
+            assert np.all(np.abs(out.astype(np.float64) - ref) <= REL * absw + ABS), f"limit {limit}"
+            assert np.array_equal(out, run(ctx, q, K, V, L, window, scale))      # fixed merge order on either route
+            outs.append(out)
+    finally:
+        fd.fdqp_set_param(ctx, "flowkv_cluster", -1)
+
+
 def test_peaked_scores_and_large_magnitudes(ctx):
     # a large scale makes the distribution collapse onto few positions (running-maximum updates matter)
     H, G, d, L = 8, 4, 256, 1500
