@@ -661,6 +661,9 @@ def run_ours(args, rank, local_rank, world):
         head_steps = [fd.chain_step(hx, hW, hy, hk, hn)]
         token_chain = fd.make_chain([fd.chain_step(xs[j], layer_copies[l % LAYER_COPIES][j], ys[j], K, N)
                                      for l in range(L) for j, (_, K, N, _) in enumerate(shapes)] + head_steps)
+        n_before = fd.fdqp_launch_count(ctx)
+        fd.fdqp_run_chain(ctx, token_chain, 1, sraw)
+        token_launches = fd.fdqp_launch_count(ctx) - n_before
         tok = time_region(torch, stream, lambda i: fd.fdqp_run_chain(ctx, token_chain, 1, sraw), 1, regions, pairs=40)
         token_bytes = L * lbytes + step_bytes
 
@@ -671,7 +674,7 @@ def run_ours(args, rank, local_rank, world):
 
         tok1 = time_region(torch, stream, token_single, 1, regions, pairs=40)
         decode = {"chained": dict(with_rates(tok, token_bytes, peaks), tokens_per_s=1e6 / tok["us_back_to_back"],
-                                  launches_per_token=-(-(4 * L + 1) // 64)),
+                                  launches_per_token=token_launches),
                   "single_calls": dict(with_rates(tok1, token_bytes, peaks), tokens_per_s=1e6 / tok1["us_back_to_back"],
                                        launches_per_token=5 * L + 1),
                   "bytes_per_token": token_bytes, "roofline_tokens_per_s": peaks["hbm_gbs"] * 1e9 / token_bytes}

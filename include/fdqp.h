@@ -291,7 +291,8 @@ typedef struct {
 } fdqp_chain_step;
 
 /* A chain of projections at M = 1 .. 8 token rows in as few launches as possible: ONE persistent kernel walks up to
- * 64 steps (longer chains are cut into several launches).  The paper keeps all kernels of a decoder layer resident
+ * 160 steps (longer chains, and chains whose steps together need more arrival counters or partial-row slots than the
+ * context's workspace holds, are cut into several launches).  The paper keeps all kernels of a decoder layer resident
  * and pipelined on its tile array, the vectors between them staying on chip (its section on mapping the decoder;
  * Sec. "FusedDQP"); here the weight stream of step i + 1 is already filling shared memory while step i finishes, so
  * launch latency and the first trip to HBM are paid once per chain.  Each step computes exactly what
@@ -429,7 +430,7 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "strip_aligned" 1 = CTA work ranges are cut at strip boundaries, 0 = equal block counts per CTA
  *   "prep_inline"   1 = every GEMV CTA prepares its slice of x itself, 0 = a preparation kernel runs first
  *   "chain_launch"  fdqp_run_chain: bit 0 = programmatic stream serialisation (default on), bit 1 = cooperative launch
- *   "chain_steps"   fdqp_run_chain: most steps per launch (1 .. 64, default 64)
+ *   "chain_steps"   fdqp_run_chain: most steps per launch (1 .. 160, default 160)
  *   "chain_wide"    fdqp_run_chain: 1 (default) = a launch none of whose steps depends on another is cut into CTA ranges
  *                   as one sequence of blocks, 0 = every step is cut on its own
  *   "flowkv_cluster" fdqp_flowkv_decode: ranges of up to this many positions (default 2048; 0 = never) run as ONE launch,

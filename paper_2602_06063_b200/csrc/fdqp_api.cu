@@ -384,7 +384,7 @@ extern "C" fdqp_status fdqp_create(fdqp_ctx** out, int device, int64_t max_M, in
         {
             const size_t slot_b = sizeof(float) * kStripRows * kMaxTokens;
             ctx->chain_ticket_cap = (size_t)16 * (size_t)S < 65536 ? 65536 : (size_t)16 * (size_t)S;
-            if ((e = cudaMalloc(&ctx->chain_edge, slot_b * 2 * (size_t)ctx->sm_count * kMaxChainSteps))) { st = cuda_fail(nullptr, e, ""); break; }
+            if ((e = cudaMalloc(&ctx->chain_edge, slot_b * 2 * (size_t)ctx->sm_count * kChainEdgeSteps))) { st = cuda_fail(nullptr, e, ""); break; }
             if ((e = cudaMalloc(&ctx->chain_full, slot_b * kChainFullSlots))) { st = cuda_fail(nullptr, e, ""); break; }
             if ((e = cudaMalloc(&ctx->chain_tickets, sizeof(int) * ctx->chain_ticket_cap))) { st = cuda_fail(nullptr, e, ""); break; }
             if ((e = cudaMalloc(&ctx->chain_done, sizeof(int) * (kMaxChainSteps + 1)))) { st = cuda_fail(nullptr, e, ""); break; }
@@ -839,10 +839,13 @@ extern "C" fdqp_status fdqp_run_chain(fdqp_ctx* ctx, const fdqp_chain_step* step
     int cap_blocks = (int)(kChainXsCap / (8u * rec * (uint32_t)m));
     if (cap_blocks > kChainPrepItems / (8 * m * 4)) cap_blocks = kChainPrepItems / (8 * m * 4);
     if (cap_blocks < 1) return FDQP_ERR_SIZE;
-    const int per_launch = (int)ctx->p_chain_steps;
-    // plan every launch before the first one goes out, so that an error launches nothing
+    // plan every launch before the first one goes out, so that an error launches nothing; where the steps of a launch
+    // need more counters or partial-row slots than the workspace holds, the chain is cut into shorter launches
     std::vector<ChainPlan> plans;
     std::vector<char> plan_epi;
+    auto plan_all = [&](const int per_launch) -> fdqp_status {
+    plans.clear();
+    plan_epi.clear();
     for (int64_t first = 0; first < n_steps; first += per_launch) {
         const int n = (int)((n_steps - first) < per_launch ? (n_steps - first) : per_launch);
         ChainPlan cp;
@@ -927,7 +930,7 @@ extern "C" fdqp_status fdqp_run_chain(fdqp_ctx* ctx, const fdqp_chain_step* step
         cp.has_deps = dependent ? 1 : 0;
         cp.wide = (!dependent && blocks >= (size_t)grid && blocks < (1u << 31) && ctx->p_chain_wide != 0) ? 1 : 0;
         if (ticket_off > ctx->chain_ticket_cap || full_off > kChainFullSlots ||
-            edge_off > (size_t)2 * ctx->sm_count * kMaxChainSteps)
+            (cp.wide ? (size_t)2 * grid : edge_off) > (size_t)2 * ctx->sm_count * kChainEdgeSteps)
             return FDQP_ERR_SIZE;
         const uint32_t part_bytes = 2u * 16u * kStripRows * (uint32_t)m * 4u * (cols ? (uint32_t)kColsPartTerms : 1u);
         const uint32_t norm_bytes = (uint32_t)(kChainPrepItems / 4) * 4u + 64u;
@@ -958,6 +961,14 @@ extern "C" fdqp_status fdqp_run_chain(fdqp_ctx* ctx, const fdqp_chain_step* step
         plans.push_back(cp);
         plan_epi.push_back(epi ? 1 : 0);
     }
+    return FDQP_OK;
+    };
+    fdqp_status planned = FDQP_ERR_SIZE;
+    for (int per_launch = (int)ctx->p_chain_steps; per_launch >= 1; per_launch = per_launch > 1 ? (per_launch + 1) / 2 : 0) {
+        planned = plan_all(per_launch);
+        if (planned != FDQP_ERR_SIZE) break;
+    }
+    if (planned != FDQP_OK) return planned;
     for (size_t i = 0; i < plans.size(); ++i) {
         const cudaError_t e = chain_launch(plans[i], grid, plan_epi[i] != 0, (int)ctx->p_chain_launch, stream);
         if (e) return cuda_fail(ctx, e, "chain kernel launch");

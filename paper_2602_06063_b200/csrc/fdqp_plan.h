@@ -66,8 +66,9 @@ struct GemvPlan {
 };
 
 // ---- a chain of projections in one persistent launch (fdqp_chain.cu) ---------------------------------------------
-constexpr int kMaxChainSteps = 64;   // projections one launch walks (a longer chain is cut into several launches)
-constexpr int kMaxChainUnits = 160;  // (step, K slice) pairs of one launch
+constexpr int kMaxChainSteps = 160;  // projections one launch walks (a longer chain is cut into several launches)
+constexpr int kMaxChainUnits = 240;  // (step, K slice) pairs of one launch
+constexpr int kChainEdgeSteps = 64;  // partial-row slots for strips shared between CTAs: two per CTA for this many steps
 
 struct ChainStep {
     const uint8_t* W;          // device, packed Q4NX

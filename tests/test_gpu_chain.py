@@ -251,3 +251,42 @@ def test_chain_through_two_layers_and_the_full_size_lm_head(M):
     finally:
         torch.cuda.synchronize()
         fd.fdqp_destroy(ctx)
+
+
+def test_a_whole_token_of_projections_is_one_launch_and_large_chains_are_cut(fresh):
+    """137 steps (34 layers of four projections and a head, here with small shapes) run as one launch; a chain whose
+    steps together have more strips than the context has arrival counters is cut into shorter launches by the library."""
+    M = 1
+    shapes = [(256, 416), (416, 256), (256, 2048), (1024, 256)]
+    cases = [Case(K, N, M, seed=4100 + i) for i, (K, N) in enumerate(shapes)]
+    head = Case(256, 8192, M, seed=4105)
+    steps, outs, refs = [], [], []
+    for l in range(34):
+        for c in cases:
+            y = torch.empty((M, c.N), dtype=torch.float32, device="cuda")
+            steps.append(fd.chain_step(c.x_dev, c.W_dev, y, c.K, c.N))
+            outs.append(y)
+            refs.append(c)
+    y = torch.empty((M, head.N), dtype=torch.float32, device="cuda")
+    steps.append(fd.chain_step(head.x_dev, head.W_dev, y, head.K, head.N))
+    outs.append(y)
+    refs.append(head)
+    before = fd.fdqp_launch_count(fresh)
+    fd.fdqp_run_chain(fresh, fd.make_chain(steps), M)
+    torch.cuda.synchronize()
+    assert fd.fdqp_last_status(fresh) == 0
+    assert fd.fdqp_launch_count(fresh) - before == 1
+    for y, c in zip(outs, refs):
+        y_ref, a_ref = c.reference()
+        assert_close(y.cpu().numpy(), y_ref, a_ref, f"K={c.K} N={c.N}")
+    # 80 steps of 1024 strips each: more strips than arrival counters (65536) -> two launches, same results
+    big = Case(64, 32768, M, seed=4110)
+    ys = [torch.empty((M, big.N), dtype=torch.float32, device="cuda") for _ in range(80)]
+    before = fd.fdqp_launch_count(fresh)
+    fd.fdqp_run_chain(fresh, fd.make_chain([fd.chain_step(big.x_dev, big.W_dev, y, big.K, big.N) for y in ys]), M)
+    torch.cuda.synchronize()
+    assert fd.fdqp_last_status(fresh) == 0
+    assert fd.fdqp_launch_count(fresh) - before == 2
+    y_ref, a_ref = big.reference()
+    for y in (ys[0], ys[39], ys[40], ys[79]):
+        assert_close(y.cpu().numpy(), y_ref, a_ref, "cut chain")
