@@ -1,11 +1,12 @@
 """Activations with a wide dynamic range inside a 32-group, through the GEMV kernels (M = 1 .. 8).
 
-The kernels hold the activations of a quantisation group as fixed point relative to the group's largest exponent.
-That is exact only for values within 2^14 of the largest; a group with anything else -- a small value next to an
-outlier channel, a subnormal next to a normal number, an infinity or a NaN -- is flagged by the activation preparation
-and evaluated in fp32 straight from Eq. 3 inside the same kernel.  These tests go to both sides of that line and
-check the stated acceptance bound against the fp64 oracle on inputs built to break a rounded fixed point: the outlier's
-own weight is zero, so everything the output is made of comes from the small elements.
+At one and two token rows the kernels hold the activations of a quantisation group as 31-bit fixed point relative to
+the group's largest exponent.  That is exact for values within 2^22 of the largest; a group with anything else -- a
+tiny value next to an outlier channel, a subnormal next to a normal number, an infinity or a NaN -- is flagged by the
+activation preparation and evaluated in fp32 straight from Eq. 3 inside the same kernel.  At three to eight rows the
+activations enter the tensor cores as the bf16 numbers they are.  These tests go to both sides of that line and check
+the stated acceptance bound against the fp64 oracle on inputs built to break a rounded fixed point: the outlier's own
+weight is zero, so everything the output is made of comes from the small elements.
 """
 import numpy as np
 import pytest
