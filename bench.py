@@ -743,9 +743,16 @@ def run_ours(args, rank, local_rank, world):
         dequant = with_rates(ent, (0.625 + 2.0) * hk * hn, peaks)
         dequant["workload"] = f"LM head K={hk} N={hn} -> bf16 [K][N]"
         del dq_out
+        # ---- what the weight stream could reach at most: the same bulk-copy ring with nothing behind it, over 2 GiB
+        probe_bytes = 2 << 30
+        probe = torch.empty(probe_bytes, dtype=torch.uint8, device="cuda")
+        ent = time_region(torch, stream, lambda i: fd.fdqp_stream_read(ctx, probe, probe_bytes, sraw), 1, regions, pairs=24)
+        read_ref = with_rates(ent, float(probe_bytes // 40960 * 40960), peaks)
+        read_ref["workload"] = "2 GiB read once by fdqp_stream_read (bulk copies into a shared-memory ring, data dropped)"
+        del probe
         if fd.fdqp_last_status(ctx) != 0:
             raise SystemExit("bench.py: a kernel reported " + fd.fdqp_status_string(fd.fdqp_last_status(ctx)))
-        line_extra = {"configs": configs, "decode_tokens": decode, "decode_tokens_per_s": decode["chained"]["tokens_per_s"],
+        line_extra = {"read_stream_reference": read_ref, "configs": configs, "decode_tokens": decode, "decode_tokens_per_s": decode["chained"]["tokens_per_s"],
                       "batched_decode": batch8, "prefill_lm_head": prefill, "decode_attention": attention,
                       "format_variants": formats, "dequant_engine": dequant}
 

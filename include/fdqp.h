@@ -251,6 +251,14 @@ FDQP_API fdqp_status fdqp_run_add_rmsnorm_epilogue(fdqp_ctx* ctx, const void* x_
                                           void* h_out_bf16, const void* gamma_bf16, float eps, const void* W_q4nx,
                                           void* out, int epilogue, int64_t M, int64_t K, int64_t N, void* cuda_stream);
 
+/* Measurement aid (the paper has no counterpart): reads the first floor(bytes / 40960) * 40960 bytes of `buf` (device,
+ * 16-byte aligned) once, one persistent CTA per SM pulling its contiguous share through a shared-memory ring with the
+ * bulk copies the projection kernels stream their weights with, and drops the data.  Timed by the caller, it gives the
+ * read rate that stream can reach at most on this device (a copy's bandwidth counts a read and a write per byte).
+ * Asynchronous on `cuda_stream`; writes nothing but the status word on a timed-out wait.
+ * Errors: FDQP_ERR_ARG, FDQP_ERR_ALIGN, FDQP_ERR_CUDA. */
+FDQP_API fdqp_status fdqp_stream_read(fdqp_ctx* ctx, const void* buf, int64_t bytes, void* cuda_stream);
+
 /* Decode attention over a KV cache (the paper's FlowKV, and FlowKV-SWA for local
  * layers): the attention of ONE new token at decoding step L,
  *     out[h] = sum_j softmax_j( scale * q[h] . K[g][j] ) V[g][j],   g = h / (H / G),

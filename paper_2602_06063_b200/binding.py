@@ -23,7 +23,7 @@ STATUS = {
 
 EXPORTS = [
     "q4nx_packed_bytes", "q4nx_pack", "q4nx_unpack", "fdqp_create", "fdqp_destroy", "fdqp_run", "fdqp_run_host",
-    "fdqp_run_host_async", "fdqp_run_epilogue", "fdqp_run_rmsnorm_epilogue", "fdqp_flowkv_decode",
+    "fdqp_run_host_async", "fdqp_run_epilogue", "fdqp_run_rmsnorm_epilogue", "fdqp_flowkv_decode", "fdqp_stream_read",
     "fdqp_dequant", "fdqp_last_status", "fdqp_last_cuda_error", "fdqp_status_string", "fdqp_set_param",
     "fdqp_launch_count", "fdqp_describe", "fdqp_run_noalloc", "q4nx_packed_bytes_fmt", "q4nx_pack_fmt",
     "q4nx_unpack_fmt", "fdqp_run_fmt", "fdqp_dequant_fmt", "fdqp_run_add_rmsnorm_epilogue",
@@ -84,6 +84,8 @@ def load_library():
     lib.fdqp_run_add_rmsnorm_epilogue.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, ci, i64, i64, i64, vp]
     lib.fdqp_flowkv_decode.restype = ci
     lib.fdqp_flowkv_decode.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, ctypes.c_float, vp]
+    lib.fdqp_stream_read.restype = ci
+    lib.fdqp_stream_read.argtypes = [vp, vp, i64, vp]
     lib.fdqp_run_host_async.restype = ci
     lib.fdqp_run_host_async.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.fdqp_run_noalloc.restype = ci
@@ -259,6 +261,11 @@ def fdqp_flowkv_decode(ctx: int, q_bf16, K_bf16, V_bf16, out, H: int, G: int, d:
     fp32); window > 0 restricts it to the last `window` positions."""
     _check(load_library().fdqp_flowkv_decode(ctx, _addr(q_bf16), _addr(K_bf16), _addr(V_bf16), _addr(out), H, G, d, L,
                                              pitch, window, float(scale), _stream(stream)), "fdqp_flowkv_decode", ctx)
+
+
+def fdqp_stream_read(ctx: int, buf, nbytes: int, stream=None) -> None:
+    """Measurement aid: reads `nbytes` of a device buffer once through the projection kernels' bulk-copy ring."""
+    _check(load_library().fdqp_stream_read(ctx, _addr(buf), nbytes, _stream(stream)), "fdqp_stream_read", ctx)
 
 
 def fdqp_run_host(ctx: int, x_host_bf16, W_q4nx, y_host, M: int, K: int, N: int, stream=None) -> None:

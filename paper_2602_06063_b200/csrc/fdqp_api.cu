@@ -32,6 +32,7 @@ cudaError_t flowkv_launch(const uint16_t* q, const uint16_t* K, const uint16_t* 
                           int G, int d, int L, int pitch, int window, float scale, int sm_count, int cluster_max_positions,
                           int* launches, cudaStream_t stream);
 cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, int K, int N, cudaStream_t stream);
+cudaError_t stream_read_launch(const uint8_t* buf, int64_t bytes, int sm_count, int* status, cudaStream_t stream);
 cudaError_t wait_selftest_launch(int* status, unsigned long long limit_ns, cudaStream_t stream);
 cudaError_t chain_set_smem_limit(int bytes);
 cudaError_t chain_launch(const ChainPlan& cp, int grid, bool epi, int launch_mode, cudaStream_t stream);
@@ -567,6 +568,18 @@ extern "C" fdqp_status fdqp_run_add_rmsnorm_epilogue(fdqp_ctx* ctx, const void* 
     if (!gamma_bf16 || !residual_bf16) return FDQP_ERR_ARG;
     return run_impl(ctx, x_bf16, gamma_bf16, eps, W_q4nx, out, epilogue, M, K, N, cuda_stream, kFmtQ4nx, residual_bf16,
                     h_out_bf16);
+}
+
+extern "C" fdqp_status fdqp_stream_read(fdqp_ctx* ctx, const void* buf, int64_t bytes, void* cuda_stream) {
+    if (!ctx || !buf || bytes < 0) return FDQP_ERR_ARG;
+    if (!aligned16(buf)) return FDQP_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FDQP_ERR_CUDA;
+    const cudaError_t e = stream_read_launch(static_cast<const uint8_t*>(buf), bytes, ctx->sm_count, ctx->status_dev,
+                                             static_cast<cudaStream_t>(cuda_stream));
+    if (e) return cuda_fail(ctx, e, "read-stream kernel launch");
+    ctx->launches += 1;
+    return FDQP_OK;
 }
 
 extern "C" fdqp_status fdqp_flowkv_decode(fdqp_ctx* ctx, const void* q_bf16, const void* K_bf16, const void* V_bf16, float* out,

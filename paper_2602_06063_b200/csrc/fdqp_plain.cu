@@ -171,4 +171,52 @@ cudaError_t plain_launch(const uint8_t* W, const uint16_t* x, float* y, int M, i
     return cudaGetLastError();
 }
 
+// ---- read-stream reference ------------------------------------------------------------------------------------------
+//
+// What the weight stream of the projection kernels could reach at most: one persistent CTA per SM pulls its share of a
+// buffer through a shared-memory ring with the same 1-D bulk copies (40 KB per stage, evict-first) and drops the data.
+// A measurement aid: the copy bandwidth counts a read and a write per byte, this one only reads.
+constexpr int kStreamStages = 5;
+constexpr uint32_t kStreamChunk = 8u * kBlockBytes;  // one ring stage of the projection kernels
+
+__global__ void __launch_bounds__(32, 1) fdqp_stream_read_kernel(const uint8_t* __restrict__ buf, int64_t chunks, int* status) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const uint32_t ring = smem_u32(smem);
+    const uint32_t bars = ring + kStreamStages * kStreamChunk;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStreamStages; ++s) mbar_init(bars + 8u * s, 1);
+        mbar_fence_init();
+    }
+    __syncwarp();
+    if (threadIdx.x != 0) return;
+    // this CTA's chunks: c0, c0 + 1, ... (equal contiguous shares)
+    const int64_t c0 = chunks * blockIdx.x / gridDim.x, c1 = chunks * (blockIdx.x + 1) / gridDim.x;
+    const int64_t n = c1 - c0;
+    const uint64_t policy = l2_policy_evict_first();
+    auto issue = [&](int64_t k) {
+        const uint32_t bar = bars + 8u * (uint32_t)(k % kStreamStages);
+        mbar_arrive_expect_tx(bar, kStreamChunk);
+        bulk_g2s_hint(ring + (uint32_t)(k % kStreamStages) * kStreamChunk, buf + (c0 + k) * (int64_t)kStreamChunk, kStreamChunk, bar, policy);
+    };
+    for (int64_t k = 0; k < n && k < kStreamStages; ++k) issue(k);
+    for (int64_t k = 0; k < n; ++k) {
+        if (!mbar_wait(bars + 8u * (uint32_t)(k % kStreamStages), (uint32_t)(k / kStreamStages) & 1u, status)) break;
+        if (k + kStreamStages < n) issue(k + kStreamStages);
+    }
+}
+
+cudaError_t stream_read_launch(const uint8_t* buf, int64_t bytes, int sm_count, int* status, cudaStream_t stream) {
+    static bool attr_set = false;
+    constexpr int kSmem = kStreamStages * (int)kStreamChunk + 64;
+    cudaError_t e;
+    if (!attr_set) {
+        if ((e = cudaFuncSetAttribute(fdqp_stream_read_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem))) return e;
+        attr_set = true;
+    }
+    const int64_t chunks = bytes / (int64_t)kStreamChunk;
+    if (chunks < 1) return cudaSuccess;
+    fdqp_stream_read_kernel<<<sm_count, 32, kSmem, stream>>>(buf, chunks, status);
+    return cudaGetLastError();
+}
+
 }  // namespace fdqp

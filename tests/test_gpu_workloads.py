@@ -94,3 +94,20 @@ def test_gemma3_4b_lm_head_small_prefill_chunks(ctx, M, form):
         y_ref, a_ref = oracle.project(x, w.codes, w.scales, w.offsets, n0=n0, n1=n0 + 32,
                                       nthreads=min(32, oracle.max_threads()))
         assert_close(y[:, n0:n0 + 32], y_ref, a_ref, f"LM head M={M} strip {s}")
+
+
+def test_read_stream_reference_runs_and_reports_no_error():
+    """The measurement aid reads whole 40 KB chunks of a buffer through the projection kernels' bulk-copy ring; sizes
+    below a chunk read nothing; a misaligned buffer is refused."""
+    ctx = fd.fdqp_create(0, 8, 256, 256)
+    try:
+        buf = torch.zeros(64 * 1024 * 1024 + 48, dtype=torch.uint8, device="cuda")
+        for nbytes in (0, 16, 40960, 40960 * 3 + 16, 64 * 1024 * 1024):
+            fd.fdqp_stream_read(ctx, buf, nbytes)
+        torch.cuda.synchronize()
+        assert fd.fdqp_last_status(ctx) == 0
+        with pytest.raises(fd.FdqpError):
+            fd.fdqp_stream_read(ctx, buf[8:], 40960)
+    finally:
+        torch.cuda.synchronize()
+        fd.fdqp_destroy(ctx)
