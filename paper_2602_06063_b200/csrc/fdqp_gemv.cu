@@ -177,13 +177,24 @@ __global__ void __launch_bounds__((CW + 1 + CW / 8) * 32, CW == 8 ? 2 : 1)
             const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
             if (lane == 0) mbar_arrive_expect_tx(full0 + 8u * stage, total);
             __syncwarp();
-            if (bytes) {
-                const uint8_t* src = p.W + ps * strip_bytes + (int64_t)(b_first + pbl) * kBB;
+            // Blocks that follow each other in the container AND in the stage go out as ONE copy (strips follow each other
+            // in memory, so that is usually the whole stage): the memory system serves 20-40 KB copies faster than 5 KB ones
+            // (bare read stream: 7.28 against 6.93 TB/s).  A run ends after a short block (its slot in the stage is not filled).
+            const uint8_t* src = p.W + ps * strip_bytes + (int64_t)(b_first + pbl) * kBB;
+            const uint64_t src_prev = __shfl_up_sync(0xffffffffu, (uint64_t)(uintptr_t)src, 1);
+            const uint32_t bytes_prev = __shfl_up_sync(0xffffffffu, bytes, 1);
+            const bool first_of_run = bytes != 0 && (lane == 0 || bytes_prev != kBB || (uint64_t)(uintptr_t)src != src_prev + kBB);
+            const uint32_t firsts = __ballot_sync(0xffffffffu, first_of_run), filled = __ballot_sync(0xffffffffu, bytes != 0);
+            const uint32_t later = firsts & ~((2u << lane) - 1u);                       // runs that begin after this lane
+            const int run_end = later ? __ffs(later) - 1 : 32 - __clz(filled | 1u);    // one past the run's last lane
+            const uint32_t bytes_last = __shfl_sync(0xffffffffu, bytes, (run_end - 1) & 31);
+            if (first_of_run) {
+                const uint32_t run_bytes = (uint32_t)(run_end - 1 - lane) * kBB + bytes_last;
                 const uint32_t dst = ring + stage * kStageBytes + lane * kBB;
                 if (p.evict_first)
-                    bulk_g2s_hint(dst, src, bytes, full0 + 8u * stage, policy);
+                    bulk_g2s_hint(dst, src, run_bytes, full0 + 8u * stage, policy);
                 else
-                    bulk_g2s(dst, src, bytes, full0 + 8u * stage);
+                    bulk_g2s(dst, src, run_bytes, full0 + 8u * stage);
             }
             if (++stage == nstage) { stage = 0; phase ^= 1u; }
         }
