@@ -258,7 +258,12 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
             // force a K split)
             bpw = ctx->p_bpw == 2 || ctx->p_bpw == 4 ? (int)ctx->p_bpw : (blocks_per_cta >= 4 ? 4 : 2);
             L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw, fmt);
-            if (bpw == 4 && ctx->p_bpw != 4 && L.nstage < kMinStages) {  // smaller stages before another K slice
+            if (bpw == 4 && ctx->p_bpw != 4 && L.nstage < kMinStages) {
+                // The larger stages do not fit beside this slice's activations.  Another K slice keeps them (measured on
+                // the 27B down projection, K = 21504: M = 4 23.3 us with four slices against 32.7 us with two slices
+                // and the smaller stages; M = 3 23.1 against 27.2, M = 8 24.9 against 29.4); the smaller stages are
+                // what is left when K cannot be cut further.
+                if (ctx->p_split_k <= 0 && Z * 2 <= kMaxSplit && Z * 2 <= p->nb) continue;
                 bpw = 2;
                 L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw, fmt);
             }
@@ -267,6 +272,29 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
         if (L.nstage >= 2 || ctas_per_sm == 1) break;
     }
     if (L.nstage < 2) return false;
+    // K slices are strip-aligned, so the busiest CTA of a slice works on ceil(strips / CTAs of the slice) whole strip
+    // slices: with few strips per CTA the number of slices decides how uneven that is (27B down, 168 strips: 3 x 42 blocks
+    // with two slices, 5 x 21 with four, 10 x 11 with eight; measured at M = 3: 26.0 / 23.0 / 23.8 us).  Once K has to be
+    // cut, take the count, up to four times the necessary one, whose busiest CTA has the least to do.
+    if (Z > 1 && ctx->p_split_k <= 0) {
+        const int grid_all = ctx->sm_count * ctas_per_sm;
+        auto busiest = [&](int z) {
+            const int nbz_c = (p->nb + z - 1) / z;
+            const int z_eff = (p->nb + nbz_c - 1) / nbz_c;
+            int gz = grid_all / z_eff;
+            if (gz < 1) gz = 1;
+            if (gz > p->S) gz = (int)p->S;
+            return (int64_t)((p->S + gz - 1) / gz) * nbz_c;
+        };
+        int best = Z;
+        for (int cand = Z * 2; cand <= Z * 4 && cand <= kMaxSplit && cand <= p->nb; cand *= 2)
+            if (busiest(cand) < busiest(best)) best = cand;
+        if (best != Z) {
+            Z = best;
+            nbz = (p->nb + Z - 1) / Z;
+            L = smem_layout(ctx, M, nbz, cw, ctas_per_sm, bpw, fmt);  // (a shorter slice: at least as many stages)
+        }
+    }
     Z = (p->nb + nbz - 1) / nbz;  // drop slices that would be empty
     p->Z = Z;
     p->nbz = nbz;
