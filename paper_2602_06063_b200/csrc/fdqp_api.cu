@@ -307,14 +307,19 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     // global memory (~2 us on the critical path unless the CTA also owns whole strips to do afterwards).  Cutting at
     // strip boundaries avoids that at the price of imbalance.  Estimate both (us) and take the cheaper.
     {
-        const double t_block = 0.125 * ctas_per_sm;  // one 5 KB block at an SM's share of HBM bandwidth
+        // Time to stream the busiest CTA's blocks (us): an SM alone pulls a 5 KB block in about 0.085 us (60 GB/s), all SMs
+        // together are held to the HBM rate (0.79 ns per block over the whole grid) -- so when few CTAs have work, or the
+        // work is uneven, the busiest one is not slowed down by the others' share.
+        const double t_sm = 0.085 * ctas_per_sm, t_all = (double)(total_blocks / Z) * 5120.0 / 6.5e6;
         const int64_t blocks_bal = (total_blocks / Z + Gz - 1) / Gz;
         // (measured: ranges cut inside strips also stream 3-4 % slower -- strip boundaries then fall at odd places inside
         // the stages, and more stages take the bookkeeping path)
-        const double cost_bal = blocks_bal * t_block * 1.04 + (blocks_bal >= 2 * (int64_t)nbz ? 0.6 : 2.0);
+        const double stream_bal = (double)blocks_bal * t_sm > t_all ? (double)blocks_bal * t_sm : t_all;
+        const double cost_bal = stream_bal * 1.04 + (blocks_bal >= 2 * (int64_t)nbz ? 0.6 : 2.0);
         const int Ga = Gz < p->S ? Gz : p->S;
         const int64_t blocks_al = (int64_t)((p->S + Ga - 1) / Ga) * nbz;
-        const double cost_al = blocks_al * t_block + (Z > 1 ? 2.0 : 0.4);
+        const double stream_al = (double)blocks_al * t_sm > t_all ? (double)blocks_al * t_sm : t_all;
+        const double cost_al = stream_al + (Z > 1 ? 2.0 : 0.4);
         // K slices are always strip-aligned: every (slice, strip) then has one owner and the slices are added by a
         // second small kernel instead of through arrival counters
         const bool aligned = Z > 1 || (ctx->p_aligned >= 0 ? ctx->p_aligned != 0 : cost_al < cost_bal);
@@ -333,7 +338,7 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
     p->smem_bytes = p->off_bar + (2u * (uint32_t)nstage + 6u) * 8u + 512u;  // barriers, then the fused normalisation's sums
     p->evict_first = ctx->p_evict >= 0 ? (ctx->p_evict != 0) : 1;
     // work items (8 activations each) per CTA if x is prepared in-kernel; beyond this a preparation kernel is cheaper
-    p->prep_inline = ctx->p_prep >= 0 ? (int)(ctx->p_prep != 0) : ((int64_t)nbz * 8 * M * 4 <= (int64_t)cw * 32);
+    p->prep_inline = ctx->p_prep >= 0 ? (int)(ctx->p_prep != 0) : ((int64_t)nbz * 8 * M * 4 <= (int64_t)2 * cw * 32);
     p->ws_edge = ctx->ws_edge;
     p->ws_full = ctx->ws_full;
     p->tickets = ctx->tickets;

@@ -177,9 +177,9 @@ def run_norm(ctx, case, gamma_dev, eps, epi, M=None):
 NORM_CASES = [
     (2560, 2048, 1, {}, 1),                # fused into the GEMV launch
     (1152, 288, 3, {}, 1),                 # fused, three token rows, tail block
-    (2560, 512, 2, {}, 3),                 # too many items for in-kernel preparation: norm kernel + preparation + GEMV
-    (10240, 320, 1, {}, 3),
-    (1056, 320, 20, {"path": 2}, 7),       # norm kernel, then three GEMV chunks with their preparation
+    (2560, 512, 2, {}, 2),                 # more than one item per thread: norm kernel + GEMV (which prepares in-kernel)
+    (10240, 320, 1, {}, 3),                # too many items for in-kernel preparation: norm kernel + preparation + GEMV
+    (1056, 320, 20, {"path": 2}, 6),       # norm kernel, two GEMV chunks of eight rows with their preparation, one of four without
     (1056, 320, 40, {"path": 3, "prefill_split_k": 2}, 3),  # norm kernel + tensor-core kernel (K slices) + its sum kernel
     (1056, 320, 40, {"path": 3}, 2),       # norm kernel + tensor-core kernel
     (544, 1056, 300, {"path": 3}, 2),
