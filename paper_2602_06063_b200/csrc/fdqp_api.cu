@@ -132,7 +132,7 @@ bool use_pair(const fdqp_ctx* ctx, int64_t M) { return ctx->p_pair >= 0 ? ctx->p
 // copy; constants measured on B200).  A CTA (pair) costs about c per 64-wide k-step when its SM is full: c = 0.64 up to
 // 64 tokens rising to 0.72 at 128 (128-row tiles, two CTAs per SM), 0.78 (256-row tiles, one CTA per SM), 0.95 (two-SM
 // kernel).  The busiest SM runs n = ceil(CTAs / SMs) of them, two at a time where two fit; a CTA that has the SM to
-// itself runs its k-steps in about 0.7 of that time.  Z > 1 adds the second kernel (~5 us) and the partial results:
+// itself runs its k-steps in about 0.7 of that time.  Z > 1 adds the second kernel (2-3 us on the stream: it overlaps the first one's tail) and the partial results:
 // written by the slices, read and summed by the second kernel.
 double prefill_time_model(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N, int64_t Z) {
     const bool pair = use_pair(ctx, M);
@@ -145,7 +145,7 @@ double prefill_time_model(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N, 
     const double c = pair ? 0.95 : (M <= 64 ? 0.64 : (M <= 128 ? 0.64 + 0.08 * (double)(M - 64) / 64.0 : 0.78));
     const int64_t kz = ((K + 63) / 64 + Z - 1) / Z;
     double t = rounds * (double)kz * c;
-    if (Z > 1) t += 5.0 + (double)(2 * Z + 1) * (double)M * (double)N * 4.0 / 5.0e6;
+    if (Z > 1) t += 2.5 + (double)(2 * Z + 1) * (double)M * (double)N * 4.0 / 5.0e6;
     return t;
 }
 
@@ -165,7 +165,7 @@ int prefill_slices(const fdqp_ctx* ctx, int64_t M, int64_t K, int64_t N) {
     double t_best = prefill_time_model(ctx, M, K, N, 1);
     for (int64_t Z = 2; Z <= zmax; ++Z) {
         const double t = prefill_time_model(ctx, M, K, N, Z);
-        if (t < 0.92 * t_best) {
+        if (t < 0.95 * t_best) {
             best = Z;
             t_best = t;
         }
