@@ -181,8 +181,8 @@ NORM_CASES = [
     (10240, 320, 1, {}, 3),                # too many items for in-kernel preparation: norm kernel + preparation + GEMV
     (1056, 320, 20, {"path": 2}, 6),       # norm kernel, two GEMV chunks of eight rows with their preparation, one of four without
     (1056, 320, 40, {"path": 3, "prefill_split_k": 2}, 3),  # norm kernel + tensor-core kernel (K slices) + its sum kernel
-    (1056, 320, 40, {"path": 3}, 2),       # norm kernel + tensor-core kernel
-    (544, 1056, 300, {"path": 3}, 2),
+    (1056, 320, 40, {"path": 3, "prefill_split_k": 1}, 2),       # norm kernel + tensor-core kernel
+    (544, 1056, 300, {"path": 3, "prefill_split_k": 1}, 2),
 ]
 
 
