@@ -712,10 +712,14 @@ def run_ours(args, rank, local_rank, world):
             ent = time_region(torch, stream, lambda i, pm=pm: fd.fdqp_run(pctx, px, hW, py, pm, hk, hn, sraw), 1, regions, pairs=24)
             ent["launch"] = fd.fdqp_describe(pctx, pm, hk, hn)
             prefill[f"M={pm}"] = with_rates(ent, alg_bytes(pm, hk, hn), peaks, flops=2.0 * pm * hk * hn)
+        # the same call with bf16 outputs (what a prefill pipeline hands on): the fp32 result of M = 512 is 537 MB of stores
+        py16 = torch.empty((512, hn), dtype=torch.bfloat16, device="cuda")
+        ent = time_region(torch, stream, lambda i: fd.fdqp_run_epilogue(pctx, px, hW, py16, fd.EPI_BF16, 512, hk, hn, sraw), 1, regions, pairs=24)
+        prefill["M=512, bf16 outputs"] = with_rates(ent, alg_bytes(512, hk, hn) - 2.0 * 512 * hn, peaks, flops=2.0 * 512 * hk * hn)
         if fd.fdqp_last_status(pctx) != 0:
             raise SystemExit("bench.py: the prefill kernel reported " + fd.fdqp_status_string(fd.fdqp_last_status(pctx)))
         fd.fdqp_destroy(pctx)
-        del px, py
+        del px, py, py16
         configs[f"4: Gemma3-4B LM head K={hk} N={hn} M=512 (tensor cores)"] = prefill["M=512"]
 
         # ---- next steps beside the projection: decode attention, format variants, the dequantisation engine
