@@ -307,16 +307,21 @@ typedef struct {
  * fdqp_run_add_rmsnorm_epilogue computes for the same arguments (Eq. 14 / 15 with Eq. 3 fused; same acceptance
  * bound; results reproducible run to run, though the summation order may differ from the single call's).
  *   depends_on_previous = 1  the step starts its activations only after every output of the previous step is in
- *                            global memory (a bounded wait on a counter: FDQP_ERR_TIMEOUT in fdqp_last_status if it
- *                            runs out).  Example: gate|up with FDQP_EPI_GEGLU_BF16 followed by the down projection
+ *                            global memory.  Example: gate|up with FDQP_EPI_GEGLU_BF16 followed by the down projection
  *                            on its output.  A dependency on any EARLIER step than the previous one is not tracked.
+ *                            By default such a step begins a new launch (the stream order is the dependency; a step
+ *                            alone in its launch goes out as the single call it is equivalent to), which measured
+ *                            faster than the alternative the "chain_dependent" parameter selects: the step stays in
+ *                            the same launch and waits on a counter of the previous step's stored outputs (a bounded
+ *                            wait: FDQP_ERR_TIMEOUT in fdqp_last_status if it runs out).
  *   depends_on_previous = 0  the step's inputs must not be written by any step of the chain.
  * A step's outputs must not alias the inputs of another step unless that step depends on it.
- * Limits: 1 <= M <= 8; Q4NX only; a normalised step needs its whole row prepared in one piece (M * K <= 13056 for
- * M <= 2, M * K <= 32768 above: every K = 2560 projection qualifies); shapes within the context's maxima.
+ * Limits: 1 <= M <= 8; Q4NX only; a normalised step that shares its launch with others needs its whole row prepared in
+ * one piece (M * K <= 13056 for M <= 2, M * K <= 32768 above: every K = 2560 projection qualifies); shapes within the
+ * context's maxima.
  * Asynchronous on `cuda_stream`; no allocation; uses the context's chain workspace, so calls that share a context
  * must be ordered on one stream.
- * Errors (nothing is launched): FDQP_ERR_ARG (null pointers, n_steps < 1, unknown epilogue, dependency flag on the
+ * Errors (found before anything is launched): FDQP_ERR_ARG (null pointers, n_steps < 1, unknown epilogue, dependency flag on the
  * first step, residual without gamma), FDQP_ERR_SHAPE, FDQP_ERR_ALIGN, FDQP_ERR_SIZE (beyond the context's maxima,
  * M > 8, a normalised step whose row does not fit one K slice, workspace exhausted), FDQP_ERR_CUDA. */
 FDQP_API fdqp_status fdqp_run_chain(fdqp_ctx* ctx, const fdqp_chain_step* steps, int64_t n_steps, int64_t M,
@@ -439,6 +444,8 @@ FDQP_API const char* fdqp_status_string(fdqp_status s);
  *   "prep_inline"   1 = every GEMV CTA prepares its slice of x itself, 0 = a preparation kernel runs first
  *   "chain_launch"  fdqp_run_chain: bit 0 = programmatic stream serialisation (default on), bit 1 = cooperative launch
  *   "chain_steps"   fdqp_run_chain: most steps per launch (1 .. 160, default 160)
+ *   "chain_dependent" fdqp_run_chain: 0 (default) = a step with depends_on_previous begins a new launch; 1 = it stays in
+ *                   the launch and waits on the previous step's completion counter
  *   "chain_wide"    fdqp_run_chain: 1 (default) = a launch none of whose steps depends on another is cut into CTA ranges
  *                   as one sequence of blocks, 0 = every step is cut on its own
  *   "flowkv_cluster" fdqp_flowkv_decode: ranges of up to this many positions (default 2048; 0 = never) run as ONE launch,

@@ -17,7 +17,7 @@ from test_gpu_epilogue import geglu_bound
 
 pytestmark = pytest.mark.gpu
 
-PARAMS = ("stages", "l2_evict_first", "strip_aligned", "chain_launch", "chain_steps", "chain_wide", "blocks_per_warp")
+PARAMS = ("stages", "l2_evict_first", "strip_aligned", "chain_launch", "chain_steps", "chain_wide", "chain_dependent", "blocks_per_warp")
 
 
 @pytest.fixture(scope="module")
@@ -106,9 +106,13 @@ def interleave_gate_up(w_gate, w_up):
     return synthgen.Q4NXWeights(cat(w_gate.codes, w_up.codes), cat(w_gate.scales, w_up.scales), cat(w_gate.offsets, w_up.offsets))
 
 
+@pytest.mark.parametrize("in_kernel", [1, 0])
 @pytest.mark.parametrize("D,inner,M", [(1024, 1536, 1), (1024, 1536, 2), (1024, 1536, 8), (1152, 512, 3),
                                        (2560, 10240, 1), (2560, 10240, 2), (2560, 10240, 8)])
-def test_mlp_block_as_a_dependent_chain(fresh, D, inner, M):
+def test_mlp_block_as_a_dependent_chain(fresh, D, inner, M, in_kernel):
+    """normalise(x + residual) -> gate|up -> gated GELU -> down.  in_kernel = 1: both steps in ONE launch, the second
+    waits on the first's completion counter; 0 (the library's default): the dependent step begins a new launch."""
+    fd.fdqp_set_param(fresh, "chain_dependent", in_kernel)
     seed = 7300 + D + M
     w_gu = interleave_gate_up(synthgen.weights(seed, D, inner), synthgen.weights(seed + 1, D, inner))
     w_dn = synthgen.weights(seed + 2, inner, D, sigma_d=0.002, sigma_m=0.001)
@@ -128,7 +132,8 @@ def test_mlp_block_as_a_dependent_chain(fresh, D, inner, M):
     ])
     before = fd.fdqp_launch_count(fresh)
     run_chain(fresh, steps, M)
-    assert fd.fdqp_launch_count(fresh) - before == 1
+    launches = fd.fdqp_launch_count(fresh) - before
+    assert launches == 1 if in_kernel else launches >= 2
     # the oracle chain
     h_ref = oracle.add_residual(x, res)
     assert np.array_equal(h_dev.cpu().numpy().view(np.uint16), h_ref)
@@ -155,6 +160,7 @@ def test_dependent_chain_across_launches(fresh):
     is the counter, across launches the stream order."""
     M, D = 2, 512
     fd.fdqp_set_param(fresh, "chain_steps", 4)
+    fd.fdqp_set_param(fresh, "chain_dependent", 1)
     ws = [synthgen.weights(7500 + i, D, D, sigma_d=0.002, sigma_m=0.001) for i in range(6)]
     Ws = [dev_bytes(fd.q4nx_pack(w.codes, w.scales, w.offsets)) for w in ws]
     x0 = synthgen.activations(7510, M, D)
@@ -290,3 +296,45 @@ def test_a_whole_token_of_projections_is_one_launch_and_large_chains_are_cut(fre
     y_ref, a_ref = big.reference()
     for y in (ys[0], ys[39], ys[40], ys[79]):
         assert_close(y.cpu().numpy(), y_ref, a_ref, "cut chain")
+
+
+def test_dependent_steps_begin_new_launches_by_default(fresh):
+    """q, k, v (independent) -> o (depends) -> gate|up (depends, normalised, gated GELU) -> down (depends): by default the
+    three independent steps are one launch and every dependent step a launch (or a single call) of its own."""
+    M, D = 2, 512
+    shapes = [(D, 512), (D, 256), (D, 256), (512, D), (D, 2048), (1024, D)]
+    ws = [synthgen.weights(7700 + i, K, N, sigma_d=0.002, sigma_m=0.001) for i, (K, N) in enumerate(shapes)]
+    ws[4] = interleave_gate_up(synthgen.weights(7710, D, 1024), synthgen.weights(7711, D, 1024))
+    Ws = [dev_bytes(fd.q4nx_pack(w.codes, w.scales, w.offsets)) for w in ws]
+    x0 = synthgen.activations(7720, M, D)
+    gamma = synthgen.bf16_bits((0.25 * synthgen.bf16_to_f32(synthgen.activations(7721, 1, D))[0]).astype(np.float32))
+    q = torch.full((M, 512), 0x7FC0, dtype=torch.int16, device="cuda")
+    k = torch.full((M, 256), float("nan"), dtype=torch.float32, device="cuda")
+    v = torch.full((M, 256), float("nan"), dtype=torch.float32, device="cuda")
+    o = torch.full((M, D), 0x7FC0, dtype=torch.int16, device="cuda")
+    act = torch.full((M, 1024), 0x7FC0, dtype=torch.int16, device="cuda")
+    y = torch.full((M, D), float("nan"), dtype=torch.float32, device="cuda")
+    x_dev, gamma_dev = dev_bytes(x0), dev_bytes(gamma)
+    steps = [fd.chain_step(x_dev, Ws[0], q, D, 512, fd.EPI_BF16),
+             fd.chain_step(x_dev, Ws[1], k, D, 256),
+             fd.chain_step(x_dev, Ws[2], v, D, 256),
+             fd.chain_step(q, Ws[3], o, 512, D, fd.EPI_BF16, True),
+             fd.chain_step(o, Ws[4], act, D, 2048, fd.EPI_GEGLU_BF16, True, gamma_dev, 1e-6),
+             fd.chain_step(act, Ws[5], y, 1024, D, fd.EPI_NONE, True)]
+    outs = {}
+    for in_kernel in (0, 1):
+        fd.fdqp_set_param(fresh, "chain_dependent", in_kernel)
+        before = fd.fdqp_launch_count(fresh)
+        run_chain(fresh, steps, M)
+        launches = fd.fdqp_launch_count(fresh) - before
+        assert launches == 1 if in_kernel else launches >= 4
+        outs[in_kernel] = (q.cpu().numpy().copy(), k.cpu().numpy().copy(), o.cpu().numpy().copy(), act.cpu().numpy().copy(), y.cpu().numpy().copy())
+        # every step against the oracle's projection of the input the GPU handed on
+        def check(prev_bits, w, got, bf16, label):
+            y_ref, a_ref = oracle.project(prev_bits, w.codes, w.scales, w.offsets)
+            g = synthgen.bf16_to_f32(got.view(np.uint16)).astype(np.float64) if bf16 else got.astype(np.float64)
+            assert np.all(np.abs(g - y_ref) <= REL_TOL * a_ref + ABS_TOL + (2.0 ** -8 * np.abs(y_ref) if bf16 else 0)), label
+        check(x0, ws[0], outs[in_kernel][0], True, "q")
+        check(x0, ws[1], outs[in_kernel][1], False, "k")
+        check(outs[in_kernel][0].view(np.uint16), ws[3], outs[in_kernel][2], True, "o")
+        check(outs[in_kernel][3].view(np.uint16), ws[5], outs[in_kernel][4], False, "down")
