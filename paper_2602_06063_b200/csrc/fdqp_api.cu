@@ -315,10 +315,14 @@ bool plan_gemv(const fdqp_ctx* ctx, int M, int K, int N, int* consumer_warps, Ge
         // (measured: ranges cut inside strips also stream 3-4 % slower -- strip boundaries then fall at odd places inside
         // the stages, and more stages take the bookkeeping path)
         const double stream_bal = (double)blocks_bal * t_sm > t_all ? (double)blocks_bal * t_sm : t_all;
-        const double cost_bal = stream_bal * 1.04 + (blocks_bal >= 2 * (int64_t)nbz ? 0.6 : 2.0);
+        const double cost_bal = stream_bal * 1.04 + (blocks_bal >= 2 * (int64_t)nbz ? 1.0 : 2.0);
         const int Ga = Gz < p->S ? Gz : p->S;
         const int64_t blocks_al = (int64_t)((p->S + Ga - 1) / Ga) * nbz;
-        const double stream_al = (double)blocks_al * t_sm > t_all ? (double)blocks_al * t_sm : t_all;
+        // (when the grid as a whole is held to the HBM rate, what the busiest CTA has beyond the average it streams
+        // alone, at its own rate, after the others have finished)
+        const double beyond = (double)blocks_al - (double)(total_blocks / Z) / (double)Ga;
+        const double held = t_all + (beyond > 0 ? beyond : 0) * t_sm;
+        const double stream_al = (double)blocks_al * t_sm > held ? (double)blocks_al * t_sm : held;
         const double cost_al = stream_al + (Z > 1 ? 2.0 : 0.4);
         // K slices are always strip-aligned: every (slice, strip) then has one owner and the slices are added by a
         // second small kernel instead of through arrival counters
